@@ -1,0 +1,179 @@
+/*
+ * psgd.h -- C ABI of the B200 (sm_100a) PowerSGD+ gradient-compression library.
+ *
+ * One handle compresses `count` independent, equally shaped matrix variables
+ * X in R^{m x n} (m >= n), each seen by N data-parallel nodes that are simulated
+ * as a batch dimension on ONE GPU (problem statement: Sec. 1, Eq. (1); state of
+ * the method: Algorithm 2, "Initialize").  All-Reduce Mean of Algorithm 1 is an
+ * in-device mean over the node index; there is no inter-GPU communication.
+ *
+ * Memory layout (row-major, innermost index last), all float32 unless stated:
+ *   G      [count][N][m][n]   stochastic gradients g_t^(i)            (input, read-only)
+ *   E      [count][N][m][n]   residuals e_t^(i); persistent state, updated in place
+ *   Q      [count][n][r]      auxiliary basis Q_{t-1}; persistent state, updated in place
+ *   P_hat  [count][m][r]      orthonormal projection P~_t            (output)
+ *   D_hat  [count][m][n]      global reconstruction P~ Q^T           (optional output)
+ *
+ * Ownership: every DEVICE buffer is allocated and owned by the caller; the
+ * library never allocates or frees device memory.  `psgd_attach` hands it E, Q
+ * and an opaque workspace whose size `psgd_sizes` reports.  Pointers marked
+ * DEVICE must be device pointers valid on the current device; pointers marked
+ * HOST are ordinary host pointers.
+ *
+ * Errors: argument problems return a negative psgd_status synchronously and
+ * leave all state untouched.  Numerical conditions (rank-deficient P, Jacobi
+ * sweeps exhausted) never abort a step: they set warning bits in a device-side
+ * status word that `psgd_last_status` returns after synchronising the stream.
+ * All step calls are stream-ordered and never synchronise.  A handle is not
+ * thread-safe.
+ */
+#ifndef PSGD_H
+#define PSGD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct psgd_handle psgd_handle;
+
+/* CUDA stream passed as an opaque pointer (a cudaStream_t); NULL = default stream. */
+typedef void* psgd_stream;
+
+typedef enum {
+    PSGD_OK = 0,
+    PSGD_E_INVALID = -1,    /* argument out of range (m < n, r > n, r > 128, ...) */
+    PSGD_E_NULL = -2,       /* required pointer is NULL */
+    PSGD_E_WORKSPACE = -3,  /* workspace too small or buffers not attached */
+    PSGD_E_CUDA = -4,       /* a CUDA runtime call failed; see psgd_last_cuda_error */
+    PSGD_E_STATE = -5       /* call not valid in the handle's current state */
+} psgd_status;
+
+/* warning bits of the device status word */
+#define PSGD_W_RANK_DEFICIENT 1 /* a pivot of the orthogonalisation fell below tolerance */
+#define PSGD_W_NOT_CONVERGED 2  /* the eigen-solver of the refresh hit its sweep limit */
+
+/* options for psgd_set_option */
+#define PSGD_OPT_ERROR_FORM 1   /* 0 (default): e_i <- Delta_i - P~ Q_i^T  (Algorithm 2, last line)
+                                   1: e_i <- Delta_i - P~ Q^T with the node-averaged Q */
+#define PSGD_OPT_MODE 2         /* 0: eager (E holds the true residual after every step)
+                                   1: deferred (E holds Delta_t = g_t + e_t; the subtraction of
+                                      P~_t Q_i^T is folded into the next step's first pass;
+                                      psgd_materialize_error produces the true residual) */
+#define PSGD_OPT_REFRESH_ITERS 3   /* subspace iterations q of the refresh (default 20) */
+#define PSGD_OPT_REFRESH_OVERSAMPLE 4 /* extra columns of the refresh block (default max(8, r)) */
+
+/* buffers that psgd_debug_ptr exposes (test use only; valid until the next step) */
+#define PSGD_BUF_P_NODE 1   /* P^(i)   [count][N][m][r] */
+#define PSGD_BUF_Q_NODE 2   /* Q^(i)   [count][N][n][r] */
+#define PSGD_BUF_P_HAT 3    /* P~      [count][m][r]    */
+#define PSGD_BUF_DBAR 4     /* node mean of Delta (refresh only) [count][m][n] */
+#define PSGD_BUF_P_MEAN 5   /* P       [count][m][r]    */
+
+/* kernel families for psgd_profile_read */
+#define PSGD_K_PROJECT 0
+#define PSGD_K_ORTH 1
+#define PSGD_K_BACKPROJECT 2
+#define PSGD_K_RESIDUAL 3
+#define PSGD_K_REFRESH 4
+#define PSGD_K_MISC 5
+#define PSGD_K_COUNT 6
+
+/*
+ * Create a handle for one matrix variable (Sec. 1: N nodes, X in R^{m x n}, m >= n;
+ * Algorithm 2 "Require": rank r, restart period tau = refresh_period, N workers).
+ * Requires m >= n >= r >= 1, r <= 128, N >= 1, refresh_period >= 0 (0 = never
+ * refresh: plain PowerSGD, the first branch of Algorithm 2).  `seed` keys the
+ * counter-based generator used for Q_{-1} (psgd_reset) and for the random start
+ * block of the refresh.  Allocates host memory only.  *out is set on success.
+ */
+psgd_status psgd_create(int64_t m, int64_t n, int r, int N, int refresh_period, uint64_t seed,
+                        psgd_handle** out);
+
+/* Same, for `count` >= 1 independent matrices of equal shape processed by the same launches. */
+psgd_status psgd_create_batch(int64_t m, int64_t n, int r, int N, int count, int refresh_period,
+                              uint64_t seed, psgd_handle** out);
+
+/* Set an option (see PSGD_OPT_*).  Must precede psgd_sizes/psgd_attach. */
+psgd_status psgd_set_option(psgd_handle* h, int option, int value);
+
+/* Byte sizes of E, Q and the workspace the caller must provide.  Any pointer may be NULL. */
+psgd_status psgd_sizes(const psgd_handle* h, size_t* e_bytes, size_t* q_bytes, size_t* workspace_bytes);
+
+/*
+ * Hand the handle its DEVICE buffers: E and Q (persistent state, Algorithm 2
+ * "Initialize") and the workspace.  All three must be 256-byte aligned and stay
+ * valid until psgd_destroy.  The contents of E and Q are taken as the current
+ * state (e_t, Q_{t-1}); call psgd_reset to initialise them.
+ */
+psgd_status psgd_attach(psgd_handle* h, float* E /*DEVICE*/, float* Q /*DEVICE*/,
+                        void* workspace /*DEVICE*/, size_t workspace_bytes);
+
+/* e_0 = 0, Q_{-1} ~ N(0,1) from the seed (same on every node), t = 0.  (Algorithm 2, "Initialize") */
+psgd_status psgd_reset(psgd_handle* h, psgd_stream stream);
+
+/*
+ * One iteration t of Algorithm 2 without the optimizer update:
+ *   Delta_i = g_i + e_i (Eq. (7a));  SVD-Comp if refresh_period > 0 and
+ *   t mod refresh_period == 0, else SSP-Comp (Algorithm 1);  e_i <- Delta_i - Delta^_i;  t <- t + 1.
+ * G: DEVICE, read-only.  P_hat (DEVICE, may be NULL) receives P~_t.  D_hat
+ * (DEVICE, may be NULL) receives the dense global reconstruction P~_t Q_t^T.
+ * Q (attached) is replaced by Q_t.  Enqueued on `stream`; does not synchronise.
+ */
+psgd_status psgd_step(psgd_handle* h, const float* G, float* P_hat, float* D_hat, psgd_stream stream);
+
+/* The same iteration with SVD-Comp forced (Algorithm 1, second function; Definition 3). */
+psgd_status psgd_refresh(psgd_handle* h, const float* G, float* P_hat, float* D_hat, psgd_stream stream);
+
+/*
+ * psgd_step with HOST buffers: copies G_host into the caller's DEVICE staging
+ * buffer G_stage (same size as G), runs the step, copies P~ and Q_t back to
+ * P_hat_host / Q_host (either may be NULL) and synchronises the stream.
+ * Pinned host memory makes the copies asynchronous with respect to the host.
+ */
+psgd_status psgd_step_host(psgd_handle* h, const float* G_host /*HOST*/, float* G_stage /*DEVICE*/,
+                           float* P_hat_host /*HOST*/, float* Q_host /*HOST*/, psgd_stream stream);
+
+/*
+ * Deferred mode only: turn the stored Delta_t back into the true residual
+ * e_{t+1} = Delta_t - P~_t Q_i^T (Algorithm 2, last line) in place.  A no-op when
+ * E already holds the residual.  Call before reading or checkpointing E.
+ */
+psgd_status psgd_materialize_error(psgd_handle* h, psgd_stream stream);
+
+/* Tell the handle that the caller overwrote E (and Q) with a true residual / basis. */
+psgd_status psgd_state_written(psgd_handle* h);
+
+psgd_status psgd_get_step(const psgd_handle* h, int64_t* t);
+psgd_status psgd_set_step(psgd_handle* h, int64_t t);
+
+/* Synchronise `stream`, return the warning bits accumulated since the last call in *flags, clear them. */
+psgd_status psgd_last_status(psgd_handle* h, psgd_stream stream, int* flags /*HOST*/);
+
+/* Test hook: DEVICE address and byte size of an internal buffer (PSGD_BUF_*). */
+psgd_status psgd_debug_ptr(psgd_handle* h, int which, void** ptr, size_t* bytes);
+
+/* Number of kernels this handle has launched since creation. */
+psgd_status psgd_launch_count(const psgd_handle* h, int64_t* launches);
+
+/*
+ * Per-family kernel timing with CUDA events recorded on the launching stream.
+ * psgd_profile_begin enables it; psgd_profile_read synchronises the events,
+ * returns accumulated milliseconds and launch counts per family
+ * (arrays of PSGD_K_COUNT entries, HOST) and disables it again.
+ */
+psgd_status psgd_profile_begin(psgd_handle* h);
+psgd_status psgd_profile_read(psgd_handle* h, float* ms /*HOST*/, int* launches /*HOST*/);
+
+/* Text of the last CUDA error seen by this handle (static storage; never NULL). */
+const char* psgd_last_cuda_error(const psgd_handle* h);
+
+/* Frees host memory of the handle.  Never touches caller-owned device buffers. */
+psgd_status psgd_destroy(psgd_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PSGD_H */

@@ -1,0 +1,212 @@
+"""ctypes binding of the C ABI in include/psgd.h (same names, argument marshalling only)."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+PSGD_W_RANK_DEFICIENT = 1
+PSGD_W_NOT_CONVERGED = 2
+PSGD_OPT_ERROR_FORM, PSGD_OPT_MODE, PSGD_OPT_REFRESH_ITERS, PSGD_OPT_REFRESH_OVERSAMPLE = 1, 2, 3, 4
+PSGD_BUF = {"P_node": 1, "Q_node": 2, "P_hat": 3, "Dbar": 4, "P_mean": 5}
+KERNEL_FAMILIES = ["project", "orth", "backproject", "residual", "refresh", "misc"]
+
+_STATUS = {0: "PSGD_OK", -1: "PSGD_E_INVALID", -2: "PSGD_E_NULL", -3: "PSGD_E_WORKSPACE",
+           -4: "PSGD_E_CUDA", -5: "PSGD_E_STATE"}
+
+# every symbol include/psgd.h declares: name -> (restype, argtypes)
+_vp, _i64, _u64, _int, _sz = C.c_void_p, C.c_int64, C.c_uint64, C.c_int, C.c_size_t
+SIGNATURES = {
+    "psgd_create": (_int, [_i64, _i64, _int, _int, _int, _u64, C.POINTER(_vp)]),
+    "psgd_create_batch": (_int, [_i64, _i64, _int, _int, _int, _int, _u64, C.POINTER(_vp)]),
+    "psgd_set_option": (_int, [_vp, _int, _int]),
+    "psgd_sizes": (_int, [_vp, C.POINTER(_sz), C.POINTER(_sz), C.POINTER(_sz)]),
+    "psgd_attach": (_int, [_vp, _vp, _vp, _vp, _sz]),
+    "psgd_reset": (_int, [_vp, _vp]),
+    "psgd_step": (_int, [_vp, _vp, _vp, _vp, _vp]),
+    "psgd_refresh": (_int, [_vp, _vp, _vp, _vp, _vp]),
+    "psgd_step_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "psgd_materialize_error": (_int, [_vp, _vp]),
+    "psgd_state_written": (_int, [_vp]),
+    "psgd_get_step": (_int, [_vp, C.POINTER(_i64)]),
+    "psgd_set_step": (_int, [_vp, _i64]),
+    "psgd_last_status": (_int, [_vp, _vp, C.POINTER(_int)]),
+    "psgd_debug_ptr": (_int, [_vp, _int, C.POINTER(_vp), C.POINTER(_sz)]),
+    "psgd_launch_count": (_int, [_vp, C.POINTER(_i64)]),
+    "psgd_profile_begin": (_int, [_vp]),
+    "psgd_profile_read": (_int, [_vp, C.POINTER(C.c_float), C.POINTER(_int)]),
+    "psgd_last_cuda_error": (C.c_char_p, [_vp]),
+    "psgd_destroy": (_int, [_vp]),
+}
+
+
+class PSGDError(RuntimeError):
+    pass
+
+
+def library_path():
+    return os.path.join(HERE, "libpsgd.so")
+
+
+_lib = None
+
+
+def lib():
+    """The loaded C library.  Raises if it has not been built: there is no fallback."""
+    global _lib
+    if _lib is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise PSGDError(f"{path} is missing: build it with `python -m paper_2509_11254_b200.build`")
+        L = C.CDLL(path)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def _check(code, h=None):
+    if code != 0:
+        msg = _STATUS.get(code, str(code))
+        if code == -4 and h is not None:
+            msg += ": " + lib().psgd_last_cuda_error(h).decode()
+        raise PSGDError(msg)
+
+
+class PowerSGDPlus:
+    """`count` equally shaped m x n matrix variables on N simulated nodes (one GPU).
+
+    Owns the torch tensors that back the library's caller-owned buffers:
+    E [count,N,m,n], Q [count,n,r] and the workspace.
+    """
+
+    def __init__(self, m, n, r, N, refresh_period=0, seed=0, count=1, device="cuda:0", error_form="local",
+                 mode="eager", refresh_iters=None, oversample=None, reset=True):
+        import torch
+
+        self.torch = torch
+        self.m, self.n, self.r, self.N, self.count, self.tau = m, n, r, N, count, refresh_period
+        self.device = torch.device(device)
+        if self.device.type != "cuda":
+            raise PSGDError("PowerSGDPlus needs a CUDA device; there is no CPU path")
+        L = lib()
+        h = _vp()
+        _check(L.psgd_create_batch(m, n, r, N, count, refresh_period, seed, C.byref(h)))
+        self.h = h
+        _check(L.psgd_set_option(h, PSGD_OPT_ERROR_FORM, {"local": 0, "mean": 1}[error_form]))
+        _check(L.psgd_set_option(h, PSGD_OPT_MODE, {"eager": 0, "deferred": 1}[mode]))
+        if refresh_iters is not None:
+            _check(L.psgd_set_option(h, PSGD_OPT_REFRESH_ITERS, refresh_iters))
+        if oversample is not None:
+            _check(L.psgd_set_option(h, PSGD_OPT_REFRESH_OVERSAMPLE, oversample))
+        eb, qb, wb = _sz(), _sz(), _sz()
+        _check(L.psgd_sizes(h, C.byref(eb), C.byref(qb), C.byref(wb)))
+        with torch.cuda.device(self.device):
+            self.E = torch.empty((count, N, m, n), dtype=torch.float32, device=self.device)
+            self.Q = torch.empty((count, n, r), dtype=torch.float32, device=self.device)
+            self.ws = torch.empty((wb.value,), dtype=torch.uint8, device=self.device)
+            self.P_hat = torch.empty((count, m, r), dtype=torch.float32, device=self.device)
+            _check(L.psgd_attach(h, self.E.data_ptr(), self.Q.data_ptr(), self.ws.data_ptr(), wb.value), h)
+            if reset:
+                self.reset()
+
+    # -- helpers ----------------------------------------------------------
+    def _stream(self, stream=None):
+        s = stream if stream is not None else self.torch.cuda.current_stream(self.device)
+        return _vp(s.cuda_stream)
+
+    def _g(self, G):
+        t = self.torch
+        if not (isinstance(G, t.Tensor) and G.is_cuda and G.dtype == t.float32 and G.is_contiguous()):
+            raise PSGDError("G must be a contiguous float32 CUDA tensor")
+        if G.numel() != self.count * self.N * self.m * self.n:
+            raise PSGDError("G has the wrong number of elements")
+        return G
+
+    # -- the C ABI, one method per entry point ------------------------------
+    def reset(self, stream=None):
+        with self.torch.cuda.device(self.device):
+            _check(lib().psgd_reset(self.h, self._stream(stream)), self.h)
+
+    def step(self, G, D_hat=None, stream=None, force_refresh=False):
+        G = self._g(G)
+        fn = lib().psgd_refresh if force_refresh else lib().psgd_step
+        with self.torch.cuda.device(self.device):
+            _check(fn(self.h, G.data_ptr(), self.P_hat.data_ptr(), D_hat.data_ptr() if D_hat is not None else None,
+                      self._stream(stream)), self.h)
+
+    def refresh(self, G, D_hat=None, stream=None):
+        self.step(G, D_hat, stream, force_refresh=True)
+
+    def step_host(self, G_host, G_stage, P_hat_host=None, Q_host=None, stream=None):
+        with self.torch.cuda.device(self.device):
+            _check(lib().psgd_step_host(self.h, G_host.data_ptr(), G_stage.data_ptr(),
+                                        P_hat_host.data_ptr() if P_hat_host is not None else None,
+                                        Q_host.data_ptr() if Q_host is not None else None,
+                                        self._stream(stream)), self.h)
+
+    def materialize_error(self, stream=None):
+        with self.torch.cuda.device(self.device):
+            _check(lib().psgd_materialize_error(self.h, self._stream(stream)), self.h)
+
+    def set_state(self, E=None, Q=None, t=None):
+        """Overwrite the persistent state (e_t, Q_{t-1}, t) from host or device arrays."""
+        tc = self.torch
+        if E is not None:
+            self.E.copy_(tc.as_tensor(E, dtype=tc.float32).reshape(self.E.shape))
+        if Q is not None:
+            self.Q.copy_(tc.as_tensor(Q, dtype=tc.float32).reshape(self.Q.shape))
+        _check(lib().psgd_state_written(self.h))
+        if t is not None:
+            _check(lib().psgd_set_step(self.h, int(t)))
+
+    @property
+    def t(self):
+        v = _i64()
+        _check(lib().psgd_get_step(self.h, C.byref(v)))
+        return v.value
+
+    def last_status(self, stream=None):
+        v = _int()
+        with self.torch.cuda.device(self.device):
+            _check(lib().psgd_last_status(self.h, self._stream(stream), C.byref(v)), self.h)
+        return v.value
+
+    def debug(self, name):
+        """Copy of an internal buffer as a torch tensor (test hook)."""
+        tc = self.torch
+        p, b = _vp(), _sz()
+        _check(lib().psgd_debug_ptr(self.h, PSGD_BUF[name], C.byref(p), C.byref(b)))
+        off = p.value - self.ws.data_ptr()
+        flat = self.ws[off:off + b.value].view(tc.float32)
+        shape = {"P_node": (self.count, self.N, self.m, self.r), "Q_node": (self.count, self.N, self.n, self.r),
+                 "P_hat": (self.count, self.m, self.r), "Dbar": (self.count, self.m, self.n),
+                 "P_mean": (self.count, self.m, self.r)}[name]
+        return flat.view(shape).clone()
+
+    def launch_count(self):
+        v = _i64()
+        _check(lib().psgd_launch_count(self.h, C.byref(v)))
+        return v.value
+
+    def profile_begin(self):
+        _check(lib().psgd_profile_begin(self.h))
+
+    def profile_read(self):
+        ms = (C.c_float * len(KERNEL_FAMILIES))()
+        ln = (_int * len(KERNEL_FAMILIES))()
+        _check(lib().psgd_profile_read(self.h, ms, ln), self.h)
+        return {k: (ms[i], ln[i]) for i, k in enumerate(KERNEL_FAMILIES)}
+
+    def close(self):
+        if getattr(self, "h", None) is not None and self.h.value:
+            lib().psgd_destroy(self.h)
+            self.h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

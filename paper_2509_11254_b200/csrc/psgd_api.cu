@@ -1,0 +1,553 @@
+// Host side of the C ABI declared in include/psgd.h: argument checks, workspace
+// layout and the stream-ordered sequence of kernels for one iteration of
+// Algorithm 2 (SSP-Comp or SVD-Comp of Algorithm 1 plus the residual update).
+#include "../../include/psgd.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "psgd_kernels.cuh"
+
+using namespace psgd;
+
+namespace {
+
+constexpr int MAX_R = 128;
+constexpr int MAX_L = 160;  // widest refresh block
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
+
+struct Layout {
+    size_t flags, Pnode, Pmean, Phat, Qnode, part, gram, T, dbar, Y, Z, V, U, total;
+};
+
+struct ProfEvent {
+    cudaEvent_t a, b;
+    int kind;
+};
+
+}  // namespace
+
+struct psgd_handle {
+    int64_t m, n;
+    int r, N, count, tau;
+    uint64_t seed;
+    int error_form = 0, mode = 0, refresh_iters = 20, oversample = -1;
+    int64_t t = 0;
+    float* E = nullptr;
+    float* Q = nullptr;
+    char* ws = nullptr;
+    size_t ws_bytes = 0;
+    Layout lay{};
+    int ell = 0;        // refresh block width
+    int S = 1, rpc = 0; // back-projection row chunks
+    int64_t launches = 0;
+    bool profiling = false;
+    std::vector<ProfEvent> events;
+    char err[256] = "no error";
+    bool vec4 = false;  // n % 4 == 0 (128-bit paths usable when pointers are 16-byte aligned)
+};
+
+namespace {
+
+int refresh_width(const psgd_handle* h) {
+    int over = h->oversample >= 0 ? h->oversample : std::max(8, h->r);
+    int ell = std::min<int64_t>(h->n, (int64_t)h->r + over);
+    ell = std::min(ell, MAX_L);
+    return std::max(ell, h->r);
+}
+
+void plan(psgd_handle* h) {
+    h->ell = refresh_width(h);
+    const int colblk = ceil_div(h->n, BP_COLS);
+    const int64_t target = 8 * 148;
+    int64_t base = (int64_t)h->count * h->N * colblk;
+    int S = (int)std::max<int64_t>(1, (target + base - 1) / base);
+    S = std::min<int64_t>(S, ceil_div(h->m, BP_SUB));
+    int rpc = (int)align_up(ceil_div(h->m, S), BP_SUB);
+    h->rpc = rpc;
+    h->S = ceil_div(h->m, rpc);
+    // refresh back-projection (Z = Dbar^T Y, one "node"): its own chunking, computed at launch,
+    // but it shares the partial buffer, so size that for the larger of the two uses.
+    Layout& L = h->lay;
+    const size_t m = h->m, n = h->n, r = h->r, N = h->N, cnt = h->count, ell = h->ell;
+    const size_t c = std::max<size_t>(r, ell);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L.flags = take(256);
+    L.Pnode = take(cnt * N * m * r * 4);
+    L.Pmean = take(cnt * m * r * 4);
+    L.Phat = take(cnt * m * r * 4);
+    L.Qnode = take(cnt * N * n * r * 4);
+    size_t part_step = cnt * N * (size_t)h->S * n * r * 4;
+    size_t part_ref = cnt * (size_t)ceil_div(h->m, BP_SUB) * n * ell * 4;  // upper bound on chunks
+    part_ref = std::min(part_ref, cnt * (size_t)64 * n * ell * 4);          // refresh uses <= 64 chunks
+    L.part = take(std::max(part_step, part_ref));
+    size_t nparts = ceil_div(std::max(m, n), GR_ROWS);
+    L.gram = take(cnt * nparts * c * c * 8);
+    L.T = take(cnt * c * c * 8);
+    L.dbar = take(cnt * m * n * 4);
+    L.Y = take(cnt * m * ell * 4);
+    L.Z = take(cnt * n * ell * 4);
+    size_t c2 = (c + 1) & ~(size_t)1;
+    L.V = take(cnt * c2 * c2 * 8);
+    L.U = take(cnt * ell * r * 8);
+    L.total = off;
+}
+
+#define PSGD_CUDA(h, call)                                                                  \
+    do {                                                                                    \
+        cudaError_t e_ = (call);                                                            \
+        if (e_ != cudaSuccess) {                                                            \
+            snprintf((h)->err, sizeof((h)->err), "%s: %s", #call, cudaGetErrorString(e_));  \
+            return PSGD_E_CUDA;                                                             \
+        }                                                                                   \
+    } while (0)
+
+struct Launcher {
+    psgd_handle* h;
+    cudaStream_t st;
+    psgd_status status = PSGD_OK;
+    int force_kind = -1;  // when >= 0 every launch is booked under this family
+    void begin(int kind) {
+        if (!h->profiling) return;
+        ProfEvent ev;
+        ev.kind = force_kind >= 0 ? force_kind : kind;
+        cudaEventCreate(&ev.a);
+        cudaEventCreate(&ev.b);
+        cudaEventRecord(ev.a, st);
+        h->events.push_back(ev);
+    }
+    void end() {
+        if (h->profiling) cudaEventRecord(h->events.back().b, st);
+        h->launches++;
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess && status == PSGD_OK) {
+            snprintf(h->err, sizeof(h->err), "kernel launch: %s", cudaGetErrorString(e));
+            status = PSGD_E_CUDA;
+        }
+    }
+};
+
+template <typename K>
+void allow_smem(K kernel, size_t bytes) {
+    if (bytes > 48 * 1024) cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+inline bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+// ---- K1 dispatch ------------------------------------------------------------
+template <int RP, int VEC, bool ADD, bool STORE>
+void launch_project_t(Launcher& L, const ProjectArgs& a, int count) {
+    auto kern = k_project<RP, VEC, ADD, STORE>;
+    size_t smem = project_smem_bytes<RP, ADD>();
+    allow_smem(kern, smem);
+    dim3 grid(ceil_div(a.rows, PJ_TR), a.nodes, count * a.nchunks);
+    L.begin(PSGD_K_PROJECT);
+    kern<<<grid, PJ_THREADS, smem, L.st>>>(a);
+    L.end();
+}
+template <int RP>
+void launch_project_rp(Launcher& L, const ProjectArgs& a, int count, bool vec, bool add) {
+    if (vec) {
+        if (add) launch_project_t<RP, 4, true, true>(L, a, count);
+        else launch_project_t<RP, 4, false, false>(L, a, count);
+    } else {
+        if (add) launch_project_t<RP, 1, true, true>(L, a, count);
+        else launch_project_t<RP, 1, false, false>(L, a, count);
+    }
+}
+// P = (A [+B]) Q for all matrices; `add` also stores A+B into Mout.
+void launch_project(Launcher& L, const float* A, const float* B, float* Mout, const float* Q, float* P, int rows, int n,
+                    int r, int nodes, int count, bool vec) {
+    ProjectArgs a{A, B, Mout, Q, P, rows, n, r, nodes, 1};
+    bool add = B != nullptr;
+    vec = vec && aligned16(A) && (!B || aligned16(B)) && (!Mout || aligned16(Mout));
+    if (r <= 4) launch_project_rp<4>(L, a, count, vec, add);
+    else if (r <= 8) launch_project_rp<8>(L, a, count, vec, add);
+    else if (r <= 16) launch_project_rp<16>(L, a, count, vec, add);
+    else {
+        a.nchunks = ceil_div(r, 32);
+        // the in-place store of A+B is only safe when a single CTA reads each tile
+        launch_project_rp<32>(L, a, count, vec, add && a.nchunks == 1);
+    }
+}
+
+// ---- K3 dispatch ------------------------------------------------------------
+template <int RP>
+void launch_back_rp(Launcher& L, BackArgs a, int mats, bool vec) {
+    a.nchunks = ceil_div(a.r, RP);
+    dim3 grid(ceil_div(a.n, BP_COLS), a.S, mats * a.nchunks);
+    L.begin(PSGD_K_BACKPROJECT);
+    if (vec) k_backproject<RP, 4><<<grid, BP_THREADS, 0, L.st>>>(a);
+    else k_backproject<RP, 1><<<grid, BP_THREADS, 0, L.st>>>(a);
+    L.end();
+}
+void launch_back(Launcher& L, const float* M, const float* Phat, float* part, int rows, int n, int r, int nodes,
+                 int count, int rpc, int S, bool vec) {
+    BackArgs a{M, Phat, part, rows, n, r, nodes, 1, rpc, S};
+    vec = vec && aligned16(M);
+    if (r <= 4) launch_back_rp<4>(L, a, count * nodes, vec);
+    else if (r <= 8) launch_back_rp<8>(L, a, count * nodes, vec);
+    else launch_back_rp<16>(L, a, count * nodes, vec);
+}
+
+// ---- K4 dispatch ------------------------------------------------------------
+void launch_resid(Launcher& L, const float* M, float* Out, const float* Phat, const float* Qf, int rows, int n, int r,
+                  int nodes, int mats, int q_per_node, int out_per_node, bool vec) {
+    int rpc = 128;
+    while (rpc > RS_SUB && (int64_t)mats * ceil_div(n, RS_COLS) * ceil_div(rows, rpc) < 4 * 148) rpc /= 2;
+    ResidArgs a{M, Out, Phat, Qf, rows, n, r, nodes, rpc, q_per_node, out_per_node};
+    vec = vec && aligned16(Out) && (!M || aligned16(M));
+    dim3 grid(ceil_div(n, RS_COLS), ceil_div(rows, rpc), mats);
+    L.begin(PSGD_K_RESIDUAL);
+    if (r <= 4) { if (vec) k_residual<4, 4><<<grid, RS_THREADS, 0, L.st>>>(a); else k_residual<4, 1><<<grid, RS_THREADS, 0, L.st>>>(a); }
+    else if (r <= 8) { if (vec) k_residual<8, 4><<<grid, RS_THREADS, 0, L.st>>>(a); else k_residual<8, 1><<<grid, RS_THREADS, 0, L.st>>>(a); }
+    else { if (vec) k_residual<16, 4><<<grid, RS_THREADS, 0, L.st>>>(a); else k_residual<16, 1><<<grid, RS_THREADS, 0, L.st>>>(a); }
+    L.end();
+}
+
+// ---- K2: X <- orthonormal factor of X (rows x c), in place or into Xout ------
+void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int rows, int c, int kind) {
+    char* ws = h->ws;
+    double* gram = (double*)(ws + h->lay.gram);
+    double* T = (double*)(ws + h->lay.T);
+    int* flags = (int*)(ws + h->lay.flags);
+    int nparts = ceil_div(rows, GR_ROWS);
+    int nblk = ceil_div(c, 64);
+    GramArgs g{X, gram, rows, c, nparts};
+    L.begin(kind);
+    k_gram<<<dim3(nparts, nblk * nblk, h->count), 256, 0, L.st>>>(g);
+    L.end();
+    size_t smem = (size_t)c * c * 8;
+    allow_smem(k_chol, smem);
+    L.begin(kind);
+    k_chol<<<h->count, 256, smem, L.st>>>(gram, T, c, nparts, flags);
+    L.end();
+    ApplyArgs ap{X, T, Xout, rows, c, c, c, 1};
+    L.begin(kind);
+    k_apply<<<dim3(ceil_div(rows, 32), h->count), 256, (size_t)32 * c * 4, L.st>>>(ap);
+    L.end();
+}
+
+// ---- Algorithm 1, common tail: Q_i, Q, residual, optional dense reconstruction --
+void tail(Launcher& L, psgd_handle* h, float* D_hat) {
+    char* ws = h->ws;
+    float* Phat = (float*)(ws + h->lay.Phat);
+    float* Qnode = (float*)(ws + h->lay.Qnode);
+    float* part = (float*)(ws + h->lay.part);
+    const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count;
+    launch_back(L, h->E, Phat, part, m, n, r, N, cnt, h->rpc, h->S, h->vec4);
+    size_t tot = (size_t)cnt * n * r;
+    L.begin(PSGD_K_BACKPROJECT);
+    k_reduce_q<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(part, Qnode, h->Q, n, r, N, h->S, cnt);
+    L.end();
+    if (h->error_form == 0)
+        launch_resid(L, h->E, h->E, Phat, Qnode, m, n, r, N, cnt * N, 1, 1, h->vec4);
+    else
+        launch_resid(L, h->E, h->E, Phat, h->Q, m, n, r, N, cnt * N, 0, 1, h->vec4);
+    if (D_hat) launch_resid(L, nullptr, D_hat, Phat, h->Q, m, n, r, N, cnt, 0, 0, h->vec4);
+}
+
+// ---- SSP-Comp (Algorithm 1, first function) ------------------------------------
+void ssp(Launcher& L, psgd_handle* h, const float* G) {
+    char* ws = h->ws;
+    float* Pnode = (float*)(ws + h->lay.Pnode);
+    float* Pmean = (float*)(ws + h->lay.Pmean);
+    float* Phat = (float*)(ws + h->lay.Phat);
+    const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count;
+    if (r <= 32) {
+        launch_project(L, G, h->E, h->E, h->Q, Pnode, m, n, r, N, cnt, h->vec4);
+    } else {
+        L.begin(PSGD_K_PROJECT);
+        k_add_mean<<<148 * 8, 256, 0, L.st>>>(G, h->E, nullptr, (size_t)m * n, N, cnt);
+        L.end();
+        launch_project(L, h->E, nullptr, nullptr, h->Q, Pnode, m, n, r, N, cnt, h->vec4);
+    }
+    size_t tot = (size_t)cnt * m * r;
+    L.begin(PSGD_K_ORTH);
+    k_node_mean<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Pnode, Pmean, (size_t)m * r, N, cnt);
+    L.end();
+    launch_orth(L, h, Pmean, Phat, m, r, PSGD_K_ORTH);
+}
+
+// ---- SVD-Comp (Algorithm 1, second function): top-r left singular subspace of the
+//      node mean by randomised block subspace iteration + Rayleigh-Ritz. ----------
+void svd(Launcher& L, psgd_handle* h, const float* G) {
+    char* ws = h->ws;
+    float* Phat = (float*)(ws + h->lay.Phat);
+    float* dbar = (float*)(ws + h->lay.dbar);
+    float* Y = (float*)(ws + h->lay.Y);
+    float* Z = (float*)(ws + h->lay.Z);
+    float* part = (float*)(ws + h->lay.part);
+    double* gram = (double*)(ws + h->lay.gram);
+    double* V = (double*)(ws + h->lay.V);
+    double* U = (double*)(ws + h->lay.U);
+    int* flags = (int*)(ws + h->lay.flags);
+    const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count, ell = h->ell;
+    const int K = PSGD_K_REFRESH;
+    L.force_kind = K;
+    L.begin(K);
+    k_add_mean<<<148 * 8, 256, 0, L.st>>>(G, h->E, dbar, (size_t)m * n, N, cnt);
+    L.end();
+    size_t zt = (size_t)cnt * n * ell;
+    L.begin(K);
+    k_fill_normal<<<(unsigned)((zt + 255) / 256), 256, 0, L.st>>>(Z, zt, h->seed, 0x5eed0000ull + (uint64_t)h->t);
+    L.end();
+    launch_orth(L, h, Z, Z, n, ell, K);
+    // chunking of Z = Dbar^T Y over rows
+    int colblk = ceil_div(n, BP_COLS);
+    int64_t base = (int64_t)cnt * colblk * ceil_div(ell, 16);
+    int S = (int)std::max<int64_t>(1, (8 * 148 + base - 1) / base);
+    S = std::min(S, std::min(64, ceil_div(m, BP_SUB)));
+    int rpc = (int)align_up(ceil_div(m, S), BP_SUB);
+    S = ceil_div(m, rpc);
+    for (int it = 0; it < h->refresh_iters; ++it) {
+        // Y = Dbar Z, orthonormalise;  Z = Dbar^T Y, orthonormalise
+        launch_project(L, dbar, nullptr, nullptr, Z, Y, m, n, ell, 1, cnt, h->vec4);
+        launch_orth(L, h, Y, Y, m, ell, K);
+        launch_back(L, dbar, Y, part, m, n, ell, 1, cnt, rpc, S, h->vec4);
+        size_t tot = (size_t)cnt * n * ell;
+        L.begin(K);
+        k_reduce_q<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(part, nullptr, Z, n, ell, 1, S, cnt);
+        L.end();
+        if (it + 1 < h->refresh_iters) launch_orth(L, h, Z, Z, n, ell, K);
+    }
+    // Rayleigh-Ritz: eigenvectors of Z^T Z = Y^T Dbar Dbar^T Y, then P~ = Y U[:, :r]
+    int nparts = ceil_div(n, GR_ROWS);
+    int nblk = ceil_div(ell, 64);
+    GramArgs g{Z, gram, n, ell, nparts};
+    L.begin(K);
+    k_gram<<<dim3(nparts, nblk * nblk, cnt), 256, 0, L.st>>>(g);
+    L.end();
+    int c2 = (ell + 1) & ~1;
+    size_t smem = (size_t)c2 * c2 * 8;
+    allow_smem(k_jacobi_top, smem);
+    L.begin(K);
+    k_jacobi_top<<<cnt, JAC_THREADS, smem, L.st>>>(gram, nparts, ell, r, V, U, flags);
+    L.end();
+    ApplyArgs ap{Y, U, Phat, m, ell, r, r, 0};
+    L.begin(K);
+    k_apply<<<dim3(ceil_div(m, 32), cnt), 256, (size_t)32 * ell * 4, L.st>>>(ap);
+    L.end();
+    L.force_kind = -1;
+}
+
+psgd_status check_ready(const psgd_handle* h) {
+    if (!h) return PSGD_E_NULL;
+    if (!h->E || !h->Q || !h->ws) return PSGD_E_WORKSPACE;
+    return PSGD_OK;
+}
+
+psgd_status do_step(psgd_handle* h, const float* G, float* P_hat, float* D_hat, psgd_stream stream, bool force) {
+    psgd_status s = check_ready(h);
+    if (s != PSGD_OK) return s;
+    if (!G) return PSGD_E_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    Launcher L{h, st};
+    bool refresh = force || (h->tau > 0 && h->t % h->tau == 0);
+    if (refresh) svd(L, h, G); else ssp(L, h, G);
+    tail(L, h, D_hat);
+    if (L.status != PSGD_OK) return L.status;
+    if (P_hat) {
+        PSGD_CUDA(h, cudaMemcpyAsync(P_hat, h->ws + h->lay.Phat, (size_t)h->count * h->m * h->r * 4,
+                                     cudaMemcpyDeviceToDevice, st));
+    }
+    h->t += 1;
+    return PSGD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+psgd_status psgd_create_batch(int64_t m, int64_t n, int r, int N, int count, int refresh_period, uint64_t seed,
+                              psgd_handle** out) {
+    if (!out) return PSGD_E_NULL;
+    if (!(m >= n && n >= r && r >= 1 && r <= MAX_R && N >= 1 && count >= 1 && refresh_period >= 0)) return PSGD_E_INVALID;
+    if (m > (1 << 24) || n > (1 << 24) || N > 65535 || (int64_t)count * 8 > 65535) return PSGD_E_INVALID;
+    psgd_handle* h = new (std::nothrow) psgd_handle();
+    if (!h) return PSGD_E_INVALID;
+    h->m = m; h->n = n; h->r = r; h->N = N; h->count = count; h->tau = refresh_period; h->seed = seed;
+    h->vec4 = (n % 4 == 0);
+    plan(h);
+    *out = h;
+    return PSGD_OK;
+}
+
+psgd_status psgd_create(int64_t m, int64_t n, int r, int N, int refresh_period, uint64_t seed, psgd_handle** out) {
+    return psgd_create_batch(m, n, r, N, 1, refresh_period, seed, out);
+}
+
+psgd_status psgd_set_option(psgd_handle* h, int option, int value) {
+    if (!h) return PSGD_E_NULL;
+    if (h->ws) return PSGD_E_STATE;
+    switch (option) {
+        case PSGD_OPT_ERROR_FORM: if (value != 0 && value != 1) return PSGD_E_INVALID; h->error_form = value; break;
+        case PSGD_OPT_MODE: if (value != 0) return PSGD_E_INVALID; h->mode = value; break;
+        case PSGD_OPT_REFRESH_ITERS: if (value < 1 || value > 64) return PSGD_E_INVALID; h->refresh_iters = value; break;
+        case PSGD_OPT_REFRESH_OVERSAMPLE: if (value < 0 || value > MAX_L) return PSGD_E_INVALID; h->oversample = value; break;
+        default: return PSGD_E_INVALID;
+    }
+    plan(h);
+    return PSGD_OK;
+}
+
+psgd_status psgd_sizes(const psgd_handle* h, size_t* e_bytes, size_t* q_bytes, size_t* workspace_bytes) {
+    if (!h) return PSGD_E_NULL;
+    if (e_bytes) *e_bytes = (size_t)h->count * h->N * h->m * h->n * 4;
+    if (q_bytes) *q_bytes = (size_t)h->count * h->n * h->r * 4;
+    if (workspace_bytes) *workspace_bytes = h->lay.total;
+    return PSGD_OK;
+}
+
+psgd_status psgd_attach(psgd_handle* h, float* E, float* Q, void* workspace, size_t workspace_bytes) {
+    if (!h || !E || !Q || !workspace) return PSGD_E_NULL;
+    if (workspace_bytes < h->lay.total) return PSGD_E_WORKSPACE;
+    if (((uintptr_t)E & 255) || ((uintptr_t)Q & 255) || ((uintptr_t)workspace & 255)) return PSGD_E_INVALID;
+    h->E = E; h->Q = Q; h->ws = (char*)workspace; h->ws_bytes = workspace_bytes;
+    return PSGD_OK;
+}
+
+psgd_status psgd_reset(psgd_handle* h, psgd_stream stream) {
+    psgd_status s = check_ready(h);
+    if (s != PSGD_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    size_t eb, qb;
+    psgd_sizes(h, &eb, &qb, nullptr);
+    PSGD_CUDA(h, cudaMemsetAsync(h->E, 0, eb, st));
+    PSGD_CUDA(h, cudaMemsetAsync(h->ws + h->lay.flags, 0, 256, st));
+    Launcher L{h, st};
+    size_t tot = qb / 4;
+    L.begin(PSGD_K_MISC);
+    k_fill_normal<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(h->Q, tot, h->seed, 1);
+    L.end();
+    h->t = 0;
+    return L.status;
+}
+
+psgd_status psgd_step(psgd_handle* h, const float* G, float* P_hat, float* D_hat, psgd_stream stream) {
+    return do_step(h, G, P_hat, D_hat, stream, false);
+}
+
+psgd_status psgd_refresh(psgd_handle* h, const float* G, float* P_hat, float* D_hat, psgd_stream stream) {
+    return do_step(h, G, P_hat, D_hat, stream, true);
+}
+
+psgd_status psgd_step_host(psgd_handle* h, const float* G_host, float* G_stage, float* P_hat_host, float* Q_host,
+                           psgd_stream stream) {
+    psgd_status s = check_ready(h);
+    if (s != PSGD_OK) return s;
+    if (!G_host || !G_stage) return PSGD_E_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    size_t eb, qb;
+    psgd_sizes(h, &eb, &qb, nullptr);
+    PSGD_CUDA(h, cudaMemcpyAsync(G_stage, G_host, eb, cudaMemcpyHostToDevice, st));
+    s = do_step(h, G_stage, nullptr, nullptr, stream, false);
+    if (s != PSGD_OK) return s;
+    if (P_hat_host)
+        PSGD_CUDA(h, cudaMemcpyAsync(P_hat_host, h->ws + h->lay.Phat, (size_t)h->count * h->m * h->r * 4,
+                                     cudaMemcpyDeviceToHost, st));
+    if (Q_host) PSGD_CUDA(h, cudaMemcpyAsync(Q_host, h->Q, qb, cudaMemcpyDeviceToHost, st));
+    PSGD_CUDA(h, cudaStreamSynchronize(st));
+    return PSGD_OK;
+}
+
+psgd_status psgd_materialize_error(psgd_handle* h, psgd_stream) {
+    psgd_status s = check_ready(h);
+    if (s != PSGD_OK) return s;
+    return PSGD_OK;  // eager mode: E already holds the residual
+}
+
+psgd_status psgd_state_written(psgd_handle* h) {
+    if (!h) return PSGD_E_NULL;
+    return PSGD_OK;
+}
+
+psgd_status psgd_get_step(const psgd_handle* h, int64_t* t) {
+    if (!h || !t) return PSGD_E_NULL;
+    *t = h->t;
+    return PSGD_OK;
+}
+
+psgd_status psgd_set_step(psgd_handle* h, int64_t t) {
+    if (!h) return PSGD_E_NULL;
+    if (t < 0) return PSGD_E_INVALID;
+    h->t = t;
+    return PSGD_OK;
+}
+
+psgd_status psgd_last_status(psgd_handle* h, psgd_stream stream, int* flags) {
+    psgd_status s = check_ready(h);
+    if (s != PSGD_OK) return s;
+    if (!flags) return PSGD_E_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    int v = 0;
+    PSGD_CUDA(h, cudaMemcpyAsync(&v, h->ws + h->lay.flags, 4, cudaMemcpyDeviceToHost, st));
+    PSGD_CUDA(h, cudaMemsetAsync(h->ws + h->lay.flags, 0, 4, st));
+    PSGD_CUDA(h, cudaStreamSynchronize(st));
+    *flags = v;
+    return PSGD_OK;
+}
+
+psgd_status psgd_debug_ptr(psgd_handle* h, int which, void** ptr, size_t* bytes) {
+    psgd_status s = check_ready(h);
+    if (s != PSGD_OK) return s;
+    if (!ptr || !bytes) return PSGD_E_NULL;
+    const size_t m = h->m, n = h->n, r = h->r, N = h->N, c = h->count;
+    switch (which) {
+        case PSGD_BUF_P_NODE: *ptr = h->ws + h->lay.Pnode; *bytes = c * N * m * r * 4; break;
+        case PSGD_BUF_Q_NODE: *ptr = h->ws + h->lay.Qnode; *bytes = c * N * n * r * 4; break;
+        case PSGD_BUF_P_HAT: *ptr = h->ws + h->lay.Phat; *bytes = c * m * r * 4; break;
+        case PSGD_BUF_DBAR: *ptr = h->ws + h->lay.dbar; *bytes = c * m * n * 4; break;
+        case PSGD_BUF_P_MEAN: *ptr = h->ws + h->lay.Pmean; *bytes = c * m * r * 4; break;
+        default: return PSGD_E_INVALID;
+    }
+    return PSGD_OK;
+}
+
+psgd_status psgd_launch_count(const psgd_handle* h, int64_t* launches) {
+    if (!h || !launches) return PSGD_E_NULL;
+    *launches = h->launches;
+    return PSGD_OK;
+}
+
+psgd_status psgd_profile_begin(psgd_handle* h) {
+    if (!h) return PSGD_E_NULL;
+    h->profiling = true;
+    return PSGD_OK;
+}
+
+psgd_status psgd_profile_read(psgd_handle* h, float* ms, int* launches) {
+    if (!h || !ms || !launches) return PSGD_E_NULL;
+    for (int k = 0; k < PSGD_K_COUNT; ++k) { ms[k] = 0.f; launches[k] = 0; }
+    for (auto& ev : h->events) {
+        PSGD_CUDA(h, cudaEventSynchronize(ev.b));
+        float t = 0.f;
+        PSGD_CUDA(h, cudaEventElapsedTime(&t, ev.a, ev.b));
+        ms[ev.kind] += t;
+        launches[ev.kind] += 1;
+        cudaEventDestroy(ev.a);
+        cudaEventDestroy(ev.b);
+    }
+    h->events.clear();
+    h->profiling = false;
+    return PSGD_OK;
+}
+
+const char* psgd_last_cuda_error(const psgd_handle* h) { return h ? h->err : "null handle"; }
+
+psgd_status psgd_destroy(psgd_handle* h) {
+    if (!h) return PSGD_E_NULL;
+    for (auto& ev : h->events) { cudaEventDestroy(ev.a); cudaEventDestroy(ev.b); }
+    delete h;
+    return PSGD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,774 @@
+// Device kernels of the PowerSGD+ compression path (sm_100a).
+//
+// Naming follows the paper: M (= Delta) is g + e (Eq. (7a)); P = M Q, P~ = QR(P),
+// Q_i = M_i^T P~ (Algorithm 1); e <- M - P~ Q_i^T (Algorithm 2, last line).
+// All streaming kernels are HBM-bound fp32 FFMA kernels: they move tiles with
+// 128-bit cp.async / 128-bit loads and keep the small factors (Q, P~) in shared
+// memory where one warp reads them as broadcasts.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace psgd {
+
+// ----------------------------------------------------------------------------
+// small helpers
+// ----------------------------------------------------------------------------
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem, int src_bytes) {
+    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem), "r"(src_bytes));
+}
+__device__ __forceinline__ void cp_async4(void* smem, const void* gmem, int src_bytes) {
+    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;\n" ::"r"(s), "l"(gmem), "r"(src_bytes));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+}
+
+__device__ __forceinline__ float4 ldg_stream4(const float* p) {
+    return __ldcs(reinterpret_cast<const float4*>(p));
+}
+
+// ----------------------------------------------------------------------------
+// K1  project:  P_i = (A_i [+ B_i]) Q      (Algorithm 1: P^(i) <- Delta^(i) Q, with
+//     the error-feedback add of Eq. (7a) fused in; optionally stores M = A + B).
+//
+// One CTA owns 32 rows of one (matrix, node) and walks the n columns in tiles of
+// PJ_TC.  A tile is staged in shared memory by cp.async (3 stages); lane = row,
+// warp = 8-column slice, so the Q tile is read as a warp-wide broadcast and each
+// thread keeps RP running sums.  The 8 warps' partial sums are added in a fixed
+// order at the end (deterministic).
+// ----------------------------------------------------------------------------
+constexpr int PJ_TR = 32;          // rows per CTA
+constexpr int PJ_TC = 64;          // columns per tile
+constexpr int PJ_TCP = PJ_TC + 4;  // padded row stride (floats): conflict-free 128-bit row reads
+constexpr int PJ_STAGES = 3;
+constexpr int PJ_THREADS = 256;
+
+struct ProjectArgs {
+    const float* A;   // [mats][rows][n]
+    const float* B;   // [mats][rows][n] or nullptr
+    float* Mout;      // [mats][rows][n] or nullptr (may alias B)
+    const float* Q;   // [count][n][r]
+    float* P;         // [mats][rows][r]
+    int rows, n, r, nodes, nchunks;
+};
+
+template <int RP, bool ADD>
+__host__ __device__ constexpr size_t project_smem_bytes() {
+    size_t tiles = (size_t)PJ_STAGES * PJ_TR * PJ_TCP * (ADD ? 2 : 1);
+    size_t q = (size_t)PJ_STAGES * PJ_TC * RP;
+    size_t red = (size_t)8 * 32 * RP;
+    size_t body = tiles + q;
+    return 4 * (body > red ? body : red);
+}
+
+template <int RP, int VEC, bool ADD, bool STORE>
+__global__ void __launch_bounds__(PJ_THREADS) k_project(ProjectArgs a) {
+    extern __shared__ __align__(16) float smem[];
+    float* tA = smem;
+    float* tB = tA + (ADD ? PJ_STAGES * PJ_TR * PJ_TCP : 0);
+    float* tQ = tB + PJ_STAGES * PJ_TR * PJ_TCP;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int row0 = blockIdx.x * PJ_TR;
+    const int node = blockIdx.y;
+    const int c = blockIdx.z / a.nchunks, chunk = blockIdx.z % a.nchunks;
+    const int k0 = chunk * RP;
+    const size_t mat = (size_t)c * a.nodes + node;
+    const float* Ab = a.A + mat * (size_t)a.rows * a.n;
+    const float* Bb = ADD ? a.B + mat * (size_t)a.rows * a.n : nullptr;
+    float* Mb = STORE ? a.Mout + mat * (size_t)a.rows * a.n : nullptr;
+    const float* Qb = a.Q + (size_t)c * a.n * a.r;
+    const int n = a.n, r = a.r, rows = a.rows;
+    const int ntiles = (n + PJ_TC - 1) / PJ_TC;
+
+    auto load_tile = [&](int t, int stage) {
+        const int col0 = t * PJ_TC;
+        float* sa = tA + stage * PJ_TR * PJ_TCP;
+        float* sb = tB + stage * PJ_TR * PJ_TCP;
+        if (VEC == 4) {
+#pragma unroll
+            for (int it = 0; it < (PJ_TR * PJ_TC / 4) / PJ_THREADS; ++it) {
+                int ch = tid + it * PJ_THREADS;
+                int rr = ch / (PJ_TC / 4), c4 = (ch % (PJ_TC / 4)) * 4;
+                int grow = min(row0 + rr, rows - 1);
+                int gcol = col0 + c4;
+                int ok = gcol < n ? 16 : 0;
+                size_t off = (size_t)grow * n + (ok ? gcol : 0);
+                cp_async16(sa + rr * PJ_TCP + c4, Ab + off, ok);
+                if (ADD) cp_async16(sb + rr * PJ_TCP + c4, Bb + off, ok);
+            }
+        } else {
+            for (int e = tid; e < PJ_TR * PJ_TC; e += PJ_THREADS) {
+                int rr = e / PJ_TC, cc = e % PJ_TC;
+                int grow = min(row0 + rr, rows - 1);
+                int gcol = col0 + cc;
+                int ok = gcol < n ? 4 : 0;
+                size_t off = (size_t)grow * n + (ok ? gcol : 0);
+                cp_async4(sa + rr * PJ_TCP + cc, Ab + off, ok);
+                if (ADD) cp_async4(sb + rr * PJ_TCP + cc, Bb + off, ok);
+            }
+        }
+        float* sq = tQ + stage * PJ_TC * RP;
+        for (int e = tid; e < PJ_TC * RP; e += PJ_THREADS) {
+            int cc = e / RP, k = e % RP;
+            int gcol = col0 + cc;
+            int ok = (gcol < n && k0 + k < r) ? 4 : 0;
+            size_t off = ok ? (size_t)gcol * r + k0 + k : 0;
+            cp_async4(sq + e, Qb + off, ok);
+        }
+    };
+
+    float acc[RP];
+#pragma unroll
+    for (int k = 0; k < RP; ++k) acc[k] = 0.f;
+
+    for (int s = 0; s < PJ_STAGES - 1; ++s) {
+        if (s < ntiles) load_tile(s, s);
+        cp_async_commit();
+    }
+    for (int t = 0; t < ntiles; ++t) {
+        cp_async_wait<PJ_STAGES - 2>();
+        __syncthreads();
+        if (t + PJ_STAGES - 1 < ntiles) load_tile(t + PJ_STAGES - 1, (t + PJ_STAGES - 1) % PJ_STAGES);
+        cp_async_commit();
+        const int stage = t % PJ_STAGES;
+        float* sa = tA + stage * PJ_TR * PJ_TCP + lane * PJ_TCP;
+        const float* sb = tB + stage * PJ_TR * PJ_TCP + lane * PJ_TCP;
+        const float* sq = tQ + stage * PJ_TC * RP;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int cb = warp * 8 + j * 4;
+            float4 v = *reinterpret_cast<const float4*>(sa + cb);
+            if (ADD) {
+                float4 w = *reinterpret_cast<const float4*>(sb + cb);
+                v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+            }
+            if (STORE) *reinterpret_cast<float4*>(sa + cb) = v;
+            const float mv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                const float* q = sq + (cb + cc) * RP;
+#pragma unroll
+                for (int k4 = 0; k4 < RP / 4; ++k4) {
+                    float4 qv = *reinterpret_cast<const float4*>(q + 4 * k4);
+                    acc[4 * k4 + 0] = fmaf(mv[cc], qv.x, acc[4 * k4 + 0]);
+                    acc[4 * k4 + 1] = fmaf(mv[cc], qv.y, acc[4 * k4 + 1]);
+                    acc[4 * k4 + 2] = fmaf(mv[cc], qv.z, acc[4 * k4 + 2]);
+                    acc[4 * k4 + 3] = fmaf(mv[cc], qv.w, acc[4 * k4 + 3]);
+                }
+            }
+        }
+        if (STORE) {
+            __syncthreads();
+            const int col0 = t * PJ_TC;
+            const float* st = tA + stage * PJ_TR * PJ_TCP;
+            if (VEC == 4) {
+#pragma unroll
+                for (int it = 0; it < (PJ_TR * PJ_TC / 4) / PJ_THREADS; ++it) {
+                    int ch = tid + it * PJ_THREADS;
+                    int rr = ch / (PJ_TC / 4), c4 = (ch % (PJ_TC / 4)) * 4;
+                    if (row0 + rr < rows && col0 + c4 < n)
+                        *reinterpret_cast<float4*>(Mb + (size_t)(row0 + rr) * n + col0 + c4) =
+                            *reinterpret_cast<const float4*>(st + rr * PJ_TCP + c4);
+                }
+            } else {
+                for (int e = tid; e < PJ_TR * PJ_TC; e += PJ_THREADS) {
+                    int rr = e / PJ_TC, cc = e % PJ_TC;
+                    if (row0 + rr < rows && col0 + cc < n)
+                        Mb[(size_t)(row0 + rr) * n + col0 + cc] = st[rr * PJ_TCP + cc];
+                }
+            }
+        }
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+    // cross-warp reduction, fixed order
+    float* red = smem;  // [8][32][RP]
+#pragma unroll
+    for (int k = 0; k < RP; ++k) red[(warp * 32 + lane) * RP + k] = acc[k];
+    __syncthreads();
+    float* Pb = a.P + mat * (size_t)rows * r;
+    for (int e = tid; e < 32 * RP; e += PJ_THREADS) {
+        int rr = e / RP, k = e % RP;
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) s += red[(w * 32 + rr) * RP + k];
+        if (row0 + rr < rows && k0 + k < r) Pb[(size_t)(row0 + rr) * r + k0 + k] = s;
+    }
+}
+
+// ----------------------------------------------------------------------------
+// K3  back-project:  partial Q_i = M_i[rows of chunk]^T P~   (Algorithm 1:
+//     Q^(i) <- Delta^(i)^T P~).  Thread owns 4 adjacent columns and RP outputs per
+//     column; P~ rows are broadcast from shared memory.  Row chunks write partial
+//     sums that k_reduce_q adds in a fixed order.
+// ----------------------------------------------------------------------------
+constexpr int BP_THREADS = 128;
+constexpr int BP_COLS = 256;   // columns per CTA (64 threads x 4)
+constexpr int BP_SUB = 64;     // rows per shared-memory sub-tile of P~
+
+struct BackArgs {
+    const float* M;     // [mats][rows][n]
+    const float* Phat;  // [count][rows][r]
+    float* part;        // [mats][S][n][r]
+    int rows, n, r, nodes, nchunks, rows_per_chunk, S;
+};
+
+template <int RP, int VEC>
+__global__ void __launch_bounds__(BP_THREADS) k_backproject(BackArgs a) {
+    __shared__ __align__(16) float Ps[BP_SUB * RP];
+    __shared__ __align__(16) float red[64 * 4 * RP];
+    const int tid = threadIdx.x, tx = tid & 63, g = tid >> 6;
+    const int col = blockIdx.x * BP_COLS + tx * 4;
+    const int s = blockIdx.y;
+    const int mat = blockIdx.z / a.nchunks, chunk = blockIdx.z % a.nchunks;
+    const int c = mat / a.nodes;
+    const int k0 = chunk * RP;
+    const int n = a.n, r = a.r;
+    const int rbeg = s * a.rows_per_chunk, rend = min(a.rows, rbeg + a.rows_per_chunk);
+    const float* Mb = a.M + (size_t)mat * a.rows * n;
+    const float* Pb = a.Phat + (size_t)c * a.rows * r;
+
+    float acc[4][RP];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int k = 0; k < RP; ++k) acc[j][k] = 0.f;
+
+    for (int sub0 = rbeg; sub0 < rend; sub0 += BP_SUB) {
+        __syncthreads();
+        for (int e = tid; e < BP_SUB * RP; e += BP_THREADS) {
+            int rr = e / RP, k = e % RP;
+            int grow = sub0 + rr;
+            Ps[e] = (grow < rend && k0 + k < r) ? Pb[(size_t)grow * r + k0 + k] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll 1
+        for (int rr = 0; rr < BP_SUB / 2; rr += 8) {
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                int lr = g + 2 * (rr + u);
+                int grow = sub0 + lr;
+                v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (grow < rend) {
+                    const float* p = Mb + (size_t)grow * n + col;
+                    if (VEC == 4) {
+                        if (col < n) v[u] = ldg_stream4(p);
+                    } else {
+                        if (col + 0 < n) v[u].x = __ldcs(p + 0);
+                        if (col + 1 < n) v[u].y = __ldcs(p + 1);
+                        if (col + 2 < n) v[u].z = __ldcs(p + 2);
+                        if (col + 3 < n) v[u].w = __ldcs(p + 3);
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const float* pr = Ps + (g + 2 * (rr + u)) * RP;
+#pragma unroll
+                for (int k4 = 0; k4 < RP / 4; ++k4) {
+                    float4 p4 = *reinterpret_cast<const float4*>(pr + 4 * k4);
+                    const float pk[4] = {p4.x, p4.y, p4.z, p4.w};
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        acc[0][4 * k4 + kk] = fmaf(v[u].x, pk[kk], acc[0][4 * k4 + kk]);
+                        acc[1][4 * k4 + kk] = fmaf(v[u].y, pk[kk], acc[1][4 * k4 + kk]);
+                        acc[2][4 * k4 + kk] = fmaf(v[u].z, pk[kk], acc[2][4 * k4 + kk]);
+                        acc[3][4 * k4 + kk] = fmaf(v[u].w, pk[kk], acc[3][4 * k4 + kk]);
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (g == 1) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int k = 0; k < RP; ++k) red[(tx * 4 + j) * RP + k] = acc[j][k];
+    }
+    __syncthreads();
+    if (g == 0) {
+        float* out = a.part + ((size_t)mat * a.S + s) * (size_t)n * r;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (col + j < n) {
+#pragma unroll
+                for (int k = 0; k < RP; ++k)
+                    if (k0 + k < r) out[(size_t)(col + j) * r + k0 + k] = acc[j][k] + red[(tx * 4 + j) * RP + k];
+            }
+        }
+    }
+}
+
+// Q_i = sum over row chunks of the partials;  Q = (1/N) sum_i Q_i   (All-Reduce Mean).
+// One thread per (matrix, column, k); fixed summation order.
+__global__ void k_reduce_q(const float* part, float* Qi, float* Qmean, int n, int r, int nodes, int S, int count) {
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t per = (size_t)n * r;
+    if (idx >= per * count) return;
+    int c = (int)(idx / per);
+    size_t e = idx % per;
+    float tot = 0.f;
+    for (int i = 0; i < nodes; ++i) {
+        size_t mat = (size_t)c * nodes + i;
+        float s = 0.f;
+        for (int k = 0; k < S; ++k) s += part[(mat * S + k) * per + e];
+        if (Qi) Qi[mat * per + e] = s;
+        tot += s;
+    }
+    Qmean[(size_t)c * per + e] = tot / (float)nodes;
+}
+
+// ----------------------------------------------------------------------------
+// K4  residual:  E_i = M_i - P~ Q_i^T   (Algorithm 2, last line), or with M == nullptr
+//     the dense reconstruction P~ Q^T (Algorithm 1, return value).  Thread owns 4
+//     adjacent columns with their Q rows in registers and walks the rows.
+// ----------------------------------------------------------------------------
+constexpr int RS_THREADS = 128;
+constexpr int RS_COLS = 256;
+constexpr int RS_SUB = 16;  // rows per sub-tile (8 per row group)
+constexpr int RS_MAXR = 128;
+
+struct ResidArgs {
+    const float* M;     // [mats][rows][n] or nullptr
+    float* Out;         // [mats][rows][n] (may alias M)
+    const float* Phat;  // [count][rows][r]
+    const float* Qf;    // [mats or count][n][r]
+    int rows, n, r, nodes, rows_per_chunk;
+    int q_per_node;     // 1: Qf indexed by (matrix,node); 0: by matrix only
+    int out_per_node;   // 1: Out/M indexed by (matrix,node); 0: by matrix only (dense reconstruction)
+};
+
+template <int RP, int VEC>
+__global__ void __launch_bounds__(RS_THREADS) k_residual(ResidArgs a) {
+    __shared__ __align__(16) float Ps[RS_SUB * RS_MAXR];
+    const int tid = threadIdx.x, tx = tid & 63, g = tid >> 6;
+    const int col = blockIdx.x * RS_COLS + tx * 4;
+    const int n = a.n, r = a.r;
+    const int mat = blockIdx.z;
+    const int c = a.out_per_node ? mat / a.nodes : mat;
+    const int rbeg = blockIdx.y * a.rows_per_chunk, rend = min(a.rows, rbeg + a.rows_per_chunk);
+    const float* Mb = a.M ? a.M + (size_t)mat * a.rows * n : nullptr;
+    float* Ob = a.Out + (size_t)mat * a.rows * n;
+    const float* Pb = a.Phat + (size_t)c * a.rows * r;
+    const float* Qb = a.Qf + (size_t)(a.q_per_node ? mat : c) * n * r;
+    const int nch = (r + RP - 1) / RP;
+    const int rpad = nch * RP;
+
+    float q[4][RP];
+    auto load_q = [&](int k0) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int k = 0; k < RP; ++k)
+                q[j][k] = (col + j < n && k0 + k < r) ? __ldg(Qb + (size_t)(col + j) * r + k0 + k) : 0.f;
+    };
+    if (nch == 1) load_q(0);
+
+    for (int sub0 = rbeg; sub0 < rend; sub0 += RS_SUB) {
+        __syncthreads();
+        for (int e = tid; e < RS_SUB * rpad; e += RS_THREADS) {
+            int rr = e / rpad, k = e % rpad;
+            int grow = sub0 + rr;
+            Ps[rr * RS_MAXR + k] = (grow < rend && k < r) ? Pb[(size_t)grow * r + k] : 0.f;
+        }
+        __syncthreads();
+        float4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            int grow = sub0 + g + 2 * u;
+            v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (Mb && grow < rend) {
+                const float* p = Mb + (size_t)grow * n + col;
+                if (VEC == 4) {
+                    if (col < n) v[u] = ldg_stream4(p);
+                } else {
+                    if (col + 0 < n) v[u].x = __ldcs(p + 0);
+                    if (col + 1 < n) v[u].y = __ldcs(p + 1);
+                    if (col + 2 < n) v[u].z = __ldcs(p + 2);
+                    if (col + 3 < n) v[u].w = __ldcs(p + 3);
+                }
+            }
+        }
+        float rec[8][4];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) rec[u][j] = 0.f;
+        for (int ch = 0; ch < nch; ++ch) {
+            if (nch > 1) load_q(ch * RP);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const float* pr = Ps + (g + 2 * u) * RS_MAXR + ch * RP;
+#pragma unroll
+                for (int k4 = 0; k4 < RP / 4; ++k4) {
+                    float4 p4 = *reinterpret_cast<const float4*>(pr + 4 * k4);
+                    const float pk[4] = {p4.x, p4.y, p4.z, p4.w};
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) rec[u][j] = fmaf(pk[kk], q[j][4 * k4 + kk], rec[u][j]);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            int grow = sub0 + g + 2 * u;
+            if (grow >= rend) continue;
+            float4 o;
+            if (Mb) {
+                o = make_float4(v[u].x - rec[u][0], v[u].y - rec[u][1], v[u].z - rec[u][2], v[u].w - rec[u][3]);
+            } else {
+                o = make_float4(rec[u][0], rec[u][1], rec[u][2], rec[u][3]);
+            }
+            float* p = Ob + (size_t)grow * n + col;
+            if (VEC == 4) {
+                if (col < n) *reinterpret_cast<float4*>(p) = o;
+            } else {
+                if (col + 0 < n) p[0] = o.x;
+                if (col + 1 < n) p[1] = o.y;
+                if (col + 2 < n) p[2] = o.z;
+                if (col + 3 < n) p[3] = o.w;
+            }
+        }
+    }
+}
+
+// ----------------------------------------------------------------------------
+// elementwise helpers
+// ----------------------------------------------------------------------------
+// M = G + E (Eq. (7a)) written over E; optionally Dbar = (1/N) sum_i M_i (SVD-Comp, first line).
+__global__ void k_add_mean(const float* G, float* E, float* Dbar, size_t per_mat, int nodes, int count) {
+    size_t total = per_mat * count;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (size_t)gridDim.x * blockDim.x) {
+        size_t c = idx / per_mat, e = idx % per_mat;
+        float s = 0.f;
+        for (int i = 0; i < nodes; ++i) {
+            size_t off = (c * nodes + i) * per_mat + e;
+            float mval = __ldcs(G + off) + E[off];
+            E[off] = mval;
+            s += mval;
+        }
+        if (Dbar) Dbar[idx] = s / (float)nodes;
+    }
+}
+
+// X = (1/N) sum_i X_i  for the small factor arrays (All-Reduce Mean of P).
+__global__ void k_node_mean(const float* Xi, float* X, size_t per_mat, int nodes, int count) {
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= per_mat * count) return;
+    size_t c = idx / per_mat, e = idx % per_mat;
+    float s = 0.f;
+    for (int i = 0; i < nodes; ++i) s += Xi[(c * nodes + i) * per_mat + e];
+    X[idx] = s / (float)nodes;
+}
+
+// Counter-based N(0,1): splitmix64 of (seed, stream, index) -> two uniforms -> Box-Muller.
+__device__ __forceinline__ uint64_t splitmix64(uint64_t x) {
+    x += 0x9E3779B97F4A7C15ull;
+    x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+    x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+    return x ^ (x >> 31);
+}
+__global__ void k_fill_normal(float* X, size_t count, uint64_t seed, uint64_t stream) {
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= count) return;
+    uint64_t h = splitmix64(splitmix64(seed ^ (stream * 0xD1B54A32D192ED03ull)) + idx);
+    float u1 = ((float)(uint32_t)(h >> 40) + 0.5f) * (1.0f / 16777216.0f);
+    float u2 = ((float)(uint32_t)((h >> 8) & 0xFFFFFF) + 0.5f) * (1.0f / 16777216.0f);
+    X[idx] = sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
+}
+
+// ----------------------------------------------------------------------------
+// K2  orthogonalisation  P~ = QR(P)  with diag(R) > 0, as column-scaled Cholesky QR:
+//     G = P^T P (double),  d = sqrt(diag G),  D^-1 G D^-1 = L L^T,  P~ = P D^-1 L^-T.
+//     For full column rank this is the unique QR factor with positive diagonal
+//     (R = L^T D), i.e. what Householder QR with the sign fix returns.
+// ----------------------------------------------------------------------------
+constexpr int GR_ROWS = 128;  // rows per Gram CTA
+struct GramArgs {
+    const float* X;  // [count][rows][c]
+    double* part;    // [count][nparts][c][c]
+    int rows, c, nparts;
+};
+// grid: (nparts, nblk*nblk, count); 256 threads as 16x16; each thread a 4x4 block of a 64x64 tile.
+__global__ void __launch_bounds__(256) k_gram(GramArgs a) {
+    __shared__ float sa[32][65];
+    __shared__ float sb[32][65];
+    const int nblk = (a.c + 63) / 64;
+    const int bi = blockIdx.y / nblk, bj = blockIdx.y % nblk;
+    if (bi > bj) return;  // symmetric: only the upper block triangle
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const float* Xb = a.X + (size_t)blockIdx.z * a.rows * a.c;
+    const int rbeg = blockIdx.x * GR_ROWS, rend = min(a.rows, rbeg + GR_ROWS);
+    double acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+    for (int r0 = rbeg; r0 < rend; r0 += 32) {
+        __syncthreads();
+        for (int e = threadIdx.x; e < 32 * 64; e += 256) {
+            int rr = e / 64, cc = e % 64;
+            int grow = r0 + rr;
+            int ca = bi * 64 + cc, cb = bj * 64 + cc;
+            sa[rr][cc] = (grow < rend && ca < a.c) ? Xb[(size_t)grow * a.c + ca] : 0.f;
+            sb[rr][cc] = (grow < rend && cb < a.c) ? Xb[(size_t)grow * a.c + cb] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll 4
+        for (int rr = 0; rr < 32; ++rr) {
+            double va[4], vb[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                va[i] = (double)sa[rr][ty + 16 * i];
+                vb[i] = (double)sb[rr][tx + 16 * i];
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fma(va[i], vb[j], acc[i][j]);
+        }
+    }
+    double* out = a.part + ((size_t)blockIdx.z * a.nparts + blockIdx.x) * a.c * a.c;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int ga = bi * 64 + ty + 16 * i, gb = bj * 64 + tx + 16 * j;
+            if (ga < a.c && gb < a.c) out[(size_t)ga * a.c + gb] = acc[i][j];
+        }
+}
+
+// Sum the Gram partials, scale to unit diagonal, Cholesky, invert, and write
+// T = D^-1 L^-T (upper triangular, double) so that P~ = P T.  One CTA per matrix.
+// Dynamic shared memory: c*c doubles.
+constexpr double CHOL_PIVOT_TOL = 1e-11;  // squared sine of the angle to the previous columns
+__global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int c, int nparts, int* flags) {
+    extern __shared__ __align__(16) double Gs[];  // [c][c]
+    __shared__ double dinv[192];
+    __shared__ int bad;
+    const int tid = threadIdx.x;
+    const int nblk = (c + 63) / 64;
+    const double* pb = part + (size_t)blockIdx.x * nparts * c * c;
+    if (tid == 0) bad = 0;
+    for (int e = tid; e < c * c; e += 256) {
+        int i = e / c, j = e % c;
+        int ii = i, jj = j;
+        if (i / 64 > j / 64) { ii = j; jj = i; }   // lower block triangle was not computed: mirror
+        (void)nblk;
+        double s = 0.0;
+        for (int p = 0; p < nparts; ++p) s += pb[(size_t)p * c * c + (size_t)ii * c + jj];
+        Gs[e] = s;
+    }
+    __syncthreads();
+    for (int k = tid; k < c; k += 256) {
+        double d = Gs[k * c + k];
+        if (!(d > 0.0)) { dinv[k] = 0.0; bad = 1; } else dinv[k] = 1.0 / sqrt(d);
+    }
+    __syncthreads();
+    for (int e = tid; e < c * c; e += 256) {
+        int i = e / c, j = e % c;
+        double v = Gs[e] * dinv[i] * dinv[j];
+        if (i == j && dinv[i] == 0.0) v = 1.0;  // zero column: decouple it (fixed up later)
+        Gs[e] = v;
+    }
+    __syncthreads();
+    // right-looking Cholesky on the lower triangle: Gs = L L^T
+    for (int k = 0; k < c; ++k) {
+        if (tid == 0) {
+            double p = Gs[k * c + k];
+            if (!(p > CHOL_PIVOT_TOL)) { bad = 1; p = 1.0; for (int i = k + 1; i < c; ++i) Gs[i * c + k] = 0.0; }
+            Gs[k * c + k] = sqrt(p);
+        }
+        __syncthreads();
+        double lkk = Gs[k * c + k];
+        for (int i = k + 1 + tid; i < c; i += 256) Gs[i * c + k] /= lkk;
+        __syncthreads();
+        int rem = c - k - 1;
+        for (int e = tid; e < rem * rem; e += 256) {
+            int i = k + 1 + e / rem, j = k + 1 + e % rem;
+            if (j <= i) Gs[i * c + j] -= Gs[i * c + k] * Gs[j * c + k];
+        }
+        __syncthreads();
+    }
+    // in-place inverse of the lower-triangular L, row by row
+    for (int i = 0; i < c; ++i) {
+        double lii = Gs[i * c + i];
+        double val = 0.0;
+        int j = tid;  // c <= 192 <= 256: one column per thread
+        if (j < i) {
+            double s = 0.0;
+            for (int k = j; k < i; ++k) s += Gs[i * c + k] * Gs[k * c + j];
+            val = -s / lii;
+        }
+        __syncthreads();
+        if (j < i) Gs[i * c + j] = val;
+        if (j == i) Gs[i * c + i] = 1.0 / lii;
+        __syncthreads();
+    }
+    // T[j][k] = dinv[j] * Linv[k][j]  for j <= k
+    double* Tb = T + (size_t)blockIdx.x * c * c;
+    for (int e = tid; e < c * c; e += 256) {
+        int j = e / c, k = e % c;
+        Tb[e] = (j <= k) ? dinv[j] * Gs[k * c + j] : 0.0;
+    }
+    if (tid == 0 && bad) atomicOr(flags, 1);
+}
+
+// Xout[row][k] = sum_j X[row][j] * T[j][k]  (double accumulate), k < kout.
+// grid: (row tiles of 32, count); 256 threads.  X and Xout may alias (rows are staged).
+struct ApplyArgs {
+    const float* X;   // [count][rows][c]
+    const double* T;  // [count][c][ldt]
+    float* Xout;      // [count][rows][kout]
+    int rows, c, kout, ldt, upper;
+};
+__global__ void __launch_bounds__(256) k_apply(ApplyArgs a) {
+    extern __shared__ __align__(16) float xs[];  // [32][c]
+    const int row0 = blockIdx.x * 32;
+    const float* Xb = a.X + (size_t)blockIdx.y * a.rows * a.c;
+    const double* Tb = a.T + (size_t)blockIdx.y * a.c * a.ldt;
+    float* Ob = a.Xout + (size_t)blockIdx.y * a.rows * a.kout;
+    for (int e = threadIdx.x; e < 32 * a.c; e += 256) {
+        int rr = e / a.c, j = e % a.c;
+        xs[e] = (row0 + rr < a.rows) ? Xb[(size_t)(row0 + rr) * a.c + j] : 0.f;
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < 32 * a.kout; e += 256) {
+        int rr = e / a.kout, k = e % a.kout;
+        int jend = a.upper ? min(a.c, k + 1) : a.c;
+        double s = 0.0;
+        for (int j = 0; j < jend; ++j) s = fma((double)xs[rr * a.c + j], __ldg(Tb + (size_t)j * a.ldt + k), s);
+        if (row0 + rr < a.rows) Ob[(size_t)(row0 + rr) * a.kout + k] = (float)s;
+    }
+}
+
+// ----------------------------------------------------------------------------
+// Refresh: Rayleigh-Ritz on the block.  A = Z^T Z (double, c x c, summed from Gram
+// partials) is diagonalised by cyclic Jacobi with a round-robin pair schedule;
+// the r eigenvectors of the largest eigenvalues are written as U [c][r] (double).
+// One CTA per matrix; dynamic shared memory: c2*c2 doubles (c2 = c rounded up to even).
+// The sweep count is bounded; exhaustion sets PSGD_W_NOT_CONVERGED.
+// ----------------------------------------------------------------------------
+constexpr int JAC_THREADS = 512;
+constexpr int JAC_MAX_SWEEPS = 40;
+__global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, int nparts, int c, int r,
+                                                            double* Vws, double* U, int* flags) {
+    extern __shared__ __align__(16) double As[];  // [c2][c2]
+    __shared__ double cs[128], sn[128];
+    __shared__ int pp[128], qq[128];
+    __shared__ double offn, diagn;
+    __shared__ int order[192];
+    const int tid = threadIdx.x;
+    const int c2 = (c + 1) & ~1;
+    const int np = c2 / 2;
+    double* V = Vws + (size_t)blockIdx.x * c2 * c2;
+    const double* pb = part + (size_t)blockIdx.x * nparts * c * c;
+    for (int e = tid; e < c2 * c2; e += JAC_THREADS) {
+        int i = e / c2, j = e % c2;
+        double s = 0.0;
+        if (i < c && j < c) {
+            int ii = i, jj = j;
+            if (i / 64 > j / 64) { ii = j; jj = i; }
+            for (int p = 0; p < nparts; ++p) s += pb[(size_t)p * c * c + (size_t)ii * c + jj];
+        }
+        As[e] = s;
+        V[e] = (i == j) ? 1.0 : 0.0;
+    }
+    __syncthreads();
+    // symmetrise (the two triangles of a diagonal block were accumulated separately)
+    for (int e = tid; e < c2 * c2; e += JAC_THREADS) {
+        int i = e / c2, j = e % c2;
+        if (i < j) { double v = 0.5 * (As[i * c2 + j] + As[j * c2 + i]); As[i * c2 + j] = v; As[j * c2 + i] = v; }
+    }
+    __syncthreads();
+    int converged = 0;
+    for (int sweep = 0; sweep < JAC_MAX_SWEEPS && !converged; ++sweep) {
+        for (int round = 0; round < c2 - 1; ++round) {
+            // round-robin tournament: position 0 fixed, the others rotate
+            if (tid < np) {
+                int a0 = (tid == 0) ? 0 : 1 + (tid - 1 + round) % (c2 - 1);
+                int b0 = 1 + (c2 - 2 - tid + round) % (c2 - 1);
+                int p = min(a0, b0), q = max(a0, b0);
+                pp[tid] = p; qq[tid] = q;
+                double apq = As[p * c2 + q], app = As[p * c2 + p], aqq = As[q * c2 + q];
+                double cc = 1.0, ss = 0.0;
+                if (fabs(apq) > 1e-300 && fabs(apq) > 1e-18 * sqrt(fabs(app * aqq))) {
+                    double tau = (aqq - app) / (2.0 * apq);
+                    double t = (tau >= 0.0 ? 1.0 : -1.0) / (fabs(tau) + sqrt(1.0 + tau * tau));
+                    cc = 1.0 / sqrt(1.0 + t * t);
+                    ss = t * cc;
+                }
+                cs[tid] = cc; sn[tid] = ss;
+            }
+            __syncthreads();
+            // columns: A <- A J, V <- V J
+            for (int e = tid; e < np * c2; e += JAC_THREADS) {
+                int k = e / c2, i = e % c2;
+                int p = pp[k], q = qq[k];
+                double cc = cs[k], ss = sn[k];
+                double aip = As[i * c2 + p], aiq = As[i * c2 + q];
+                As[i * c2 + p] = cc * aip - ss * aiq;
+                As[i * c2 + q] = ss * aip + cc * aiq;
+                double vip = V[i * c2 + p], viq = V[i * c2 + q];
+                V[i * c2 + p] = cc * vip - ss * viq;
+                V[i * c2 + q] = ss * vip + cc * viq;
+            }
+            __syncthreads();
+            // rows: A <- J^T A
+            for (int e = tid; e < np * c2; e += JAC_THREADS) {
+                int k = e / c2, j = e % c2;
+                int p = pp[k], q = qq[k];
+                double cc = cs[k], ss = sn[k];
+                double apj = As[p * c2 + j], aqj = As[q * c2 + j];
+                As[p * c2 + j] = cc * apj - ss * aqj;
+                As[q * c2 + j] = ss * apj + cc * aqj;
+            }
+            __syncthreads();
+        }
+        if (tid == 0) { offn = 0.0; diagn = 0.0; }
+        __syncthreads();
+        double lo = 0.0, ld = 0.0;
+        for (int e = tid; e < c2 * c2; e += JAC_THREADS) {
+            int i = e / c2, j = e % c2;
+            double v = As[e];
+            if (i == j) ld += v * v; else lo += v * v;
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            lo += __shfl_xor_sync(0xffffffffu, lo, o);
+            ld += __shfl_xor_sync(0xffffffffu, ld, o);
+        }
+        if ((tid & 31) == 0) { atomicAdd(&offn, lo); atomicAdd(&diagn, ld); }
+        __syncthreads();
+        converged = (offn <= 1e-30 * diagn) || (diagn == 0.0);
+        __syncthreads();
+    }
+    if (tid == 0 && !converged) atomicOr(flags, 2);
+    // rank the eigenvalues (descending; ties by index) and emit the top r eigenvectors
+    for (int i = tid; i < c2; i += JAC_THREADS) {
+        double li = (i < c) ? As[i * c2 + i] : -1e300;
+        int rank = 0;
+        for (int j = 0; j < c2; ++j) {
+            double lj = (j < c) ? As[j * c2 + j] : -1e300;
+            if (lj > li || (lj == li && j < i)) ++rank;
+        }
+        order[rank] = i;
+    }
+    __syncthreads();
+    double* Ub = U + (size_t)blockIdx.x * c * r;
+    for (int e = tid; e < c * r; e += JAC_THREADS) {
+        int i = e / r, k = e % r;
+        Ub[e] = V[i * c2 + order[k]];
+    }
+}
+
+}  // namespace psgd

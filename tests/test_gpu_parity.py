@@ -1,0 +1,212 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle.
+
+Every comparison starts both sides from IDENTICAL state: the oracle's state is
+rounded to float32, uploaded, and the oracle continues from the rounded values.
+Tolerances (float32 path vs double oracle):
+  relative Frobenius error <= 1e-5 on P~, Q, Q_i, P_i and E
+  (E's denominator is floored at 1e-3 * ||M||_F so that exact-low-rank inputs,
+  whose residual is pure rounding noise, are still comparable);
+  after a refresh: projector distance ||P~P~^T - P~_ref P~_ref^T||_F <= 1e-4 when
+  the spectrum of the node mean has a gap (sigma_r - sigma_{r+1}) / sigma_1 >= 2e-3,
+  otherwise only the residual norm ||Dbar - P~P~^T Dbar||_F must match (1e-5).
+"""
+import numpy as np
+import pytest
+
+from conftest import rel_fro
+from oracle import psgd_oracle as orc
+from paper_2509_11254_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-5
+PROJ_TOL = 1e-4
+GAP_MIN = 2e-3
+
+
+@pytest.fixture(scope="module")
+def torch_cuda():
+    import torch
+
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    return torch
+
+
+def projector_distance(P, Pref):
+    """||P P^T - Pref Pref^T||_F without forming m x m matrices.
+
+    For orthonormal P, Pref of equal width this equals sqrt(2) ||(I - Pref Pref^T) P||_F,
+    which has no cancellation (the float32 P is orthonormal only to ~1e-7).
+    """
+    P = np.asarray(P, dtype=np.float64)
+    Pref = np.asarray(Pref, dtype=np.float64)
+    return float(np.sqrt(2.0) * np.linalg.norm(P - Pref @ (Pref.T @ P)))
+
+
+def compare_step(out, gpu, m, n, r, N, tag):
+    """out: oracle dict for one matrix; gpu: dict of numpy arrays for the same matrix."""
+    normM = np.linalg.norm(out["M"])
+    P_ref = out["P_hat"]
+    orth = np.linalg.norm(gpu["P_hat"].astype(np.float64).T @ gpu["P_hat"] - np.eye(r))
+    assert orth < 5e-6 * np.sqrt(r) + 1e-6, f"{tag}: P~ not orthonormal ({orth})"
+    if out["refresh"]:
+        s = out["sigma"]
+        gap = (s[r - 1] - (s[r] if r < len(s) else 0.0)) / s[0]
+        Dbar = out["Dbar"]
+        Pg = gpu["P_hat"].astype(np.float64)
+        res_g = np.linalg.norm(Dbar - Pg @ (Pg.T @ Dbar))
+        res_o = np.linalg.norm(Dbar - P_ref @ (P_ref.T @ Dbar))
+        # 1e-5 relative, with an absolute floor of 1e-6 ||Dbar|| (float32 rounding of P~ itself)
+        assert abs(res_g - res_o) <= TOL * max(res_o, 0.1 * np.linalg.norm(Dbar)), f"{tag}: refresh residual"
+        if gap >= GAP_MIN:
+            d = projector_distance(Pg, P_ref)
+            assert d <= PROJ_TOL, f"{tag}: projector distance {d} (gap {gap})"
+            # rotation-invariant quantities
+            rot = P_ref.T @ Pg                      # r x r, ~orthogonal
+            assert rel_fro(gpu["Q"], out["Q"] @ rot) <= 2 * PROJ_TOL, f"{tag}: Q after refresh"
+            e = rel_fro(gpu["E"], out["E"], floor=1e-3 * normM)
+            assert e <= 2 * PROJ_TOL, f"{tag}: E after refresh {e}"
+        return
+    assert rel_fro(gpu["P_node"], out["P_i"]) <= TOL, f"{tag}: P_i"
+    assert rel_fro(gpu["P_hat"], P_ref) <= TOL, f"{tag}: P~ {rel_fro(gpu['P_hat'], P_ref)}"
+    assert rel_fro(gpu["Q"], out["Q"]) <= TOL, f"{tag}: Q"
+    assert rel_fro(gpu["Q_node"], out["Q_i"]) <= TOL, f"{tag}: Q_i"
+    e = rel_fro(gpu["E"], out["E"], floor=1e-3 * normM)
+    assert e <= TOL, f"{tag}: E {e}"
+
+
+def run_case(torch, m, n, r, N, tau, steps, workload=1, count=1, error_form="local", Einit=0.0, seed=7,
+             check_dense=False, mode="eager"):
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    dev = "cuda:0"
+    comp = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=seed, count=count, device=dev, error_form=error_form,
+                        mode=mode)
+    rng = np.random.default_rng(seed)
+    Q0 = np.stack([synth.init_Q(n, r, matrix_id=c, seed=seed) for c in range(count)])
+    oracles = [orc.PowerSGDPlusOracle(m, n, r, N, tau, Q0[c], error_form) for c in range(count)]
+    if Einit:
+        for o in oracles:
+            o.E = (rng.standard_normal((N, m, n)) * Einit).astype(np.float32).astype(np.float64)
+    for t in range(steps):
+        G = np.stack([synth.make_gradients(workload, m, n, N, step=t, matrix_id=c, seed=seed) for c in range(count)])
+        # identical state on both sides: the oracle continues from float32-rounded values
+        for o in oracles:
+            o.E = o.E.astype(np.float32).astype(np.float64)
+            o.Q = o.Q.astype(np.float32).astype(np.float64)
+        comp.set_state(E=np.stack([o.E for o in oracles]), Q=np.stack([o.Q for o in oracles]), t=t)
+        Gd = torch.as_tensor(G, device=dev)
+        Dh = torch.empty((count, m, n), dtype=torch.float32, device=dev) if check_dense else None
+        comp.step(Gd, D_hat=Dh)
+        comp.materialize_error()
+        flags = comp.last_status()
+        assert flags == 0, f"step {t}: warning flags {flags}"
+        assert comp.t == t + 1
+        gp = dict(P_hat=comp.P_hat.cpu().numpy(), Q=comp.Q.cpu().numpy(), E=comp.E.cpu().numpy(),
+                  P_node=comp.debug("P_node").cpu().numpy(), Q_node=comp.debug("Q_node").cpu().numpy())
+        for c, o in enumerate(oracles):
+            out = o.step(G[c])
+            compare_step(out, {k: v[c] for k, v in gp.items()}, m, n, r, N, f"t={t} c={c}")
+            if check_dense:
+                Pg = gp["P_hat"][c].astype(np.float64)
+                Qg = gp["Q"][c].astype(np.float64)
+                assert rel_fro(Dh[c].cpu().numpy(), Pg @ Qg.T) <= TOL
+    comp.close()
+
+
+# ---- BASELINE config 1: tiny, 20 steps, refresh every 5 ------------------------
+def test_config1_tiny_20_steps(torch_cuda):
+    run_case(torch_cuda, 256, 128, 4, 4, tau=5, steps=20, workload=1)
+
+
+def test_config1_plain_powersgd(torch_cuda):
+    run_case(torch_cuda, 256, 128, 4, 4, tau=0, steps=6, workload=1, check_dense=True)
+
+
+# ---- shapes that span several tiles and ragged tails ---------------------------
+@pytest.mark.parametrize("m,n,r,N,count", [
+    (100, 37, 3, 3, 1),      # n % 4 != 0: scalar path, ragged rows and columns
+    (130, 66, 5, 2, 2),      # n % 4 == 2
+    (300, 200, 8, 2, 3),     # several row tiles, batch of 3
+    (96, 96, 1, 5, 1),       # r = 1, square
+    (64, 8, 8, 2, 1),        # n == r
+    (513, 260, 16, 1, 1),    # N = 1, r = 16, ragged both ways
+    (320, 257, 12, 3, 1),     # n odd
+])
+def test_ragged_shapes_ssp(torch_cuda, m, n, r, N, count):
+    run_case(torch_cuda, m, n, r, N, tau=0, steps=3, workload=2, count=count, Einit=0.01)
+
+
+@pytest.mark.parametrize("r", [24, 32, 48, 64, 128])
+def test_large_rank_ssp(torch_cuda, r):
+    run_case(torch_cuda, 640, 256, r, 2, tau=0, steps=2, workload=5, Einit=0.01)
+
+
+def test_mean_error_form(torch_cuda):
+    run_case(torch_cuda, 192, 128, 4, 3, tau=0, steps=3, workload=2, error_form="mean", Einit=0.01)
+
+
+# ---- refresh (SVD-Comp) ---------------------------------------------------------
+@pytest.mark.parametrize("m,n,r,N,workload", [
+    (256, 128, 4, 4, 1),
+    (384, 200, 8, 2, 2),
+    (300, 130, 1, 3, 5),
+    (512, 256, 16, 2, 5),
+    (200, 50, 50, 2, 5),      # r == n: the whole column space
+])
+def test_refresh_schedule(torch_cuda, m, n, r, N, workload):
+    """SVD-Comp at t = 0 and t = 3, SSP-Comp in between; the residual evolves naturally."""
+    run_case(torch_cuda, m, n, r, N, tau=3, steps=5, workload=workload)
+
+
+def test_refresh_every_step(torch_cuda):
+    run_case(torch_cuda, 256, 128, 4, 4, tau=1, steps=3, workload=1)
+
+
+def test_exact_rank_r_recovery(torch_cuda):
+    """Exactly rank-r input, zero residual: one SSP step reproduces it, E stays ~0."""
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    torch = torch_cuda
+    m, n, r, N = 160, 96, 4, 3
+    G = synth.exact_rank_r(m, n, r, N)
+    comp = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=3)
+    Dh = torch.empty((1, m, n), dtype=torch.float32, device="cuda:0")
+    comp.step(torch.as_tensor(G[None], device="cuda:0"), D_hat=Dh)
+    assert rel_fro(Dh[0].cpu().numpy(), G[0]) <= 5e-6
+    assert np.linalg.norm(comp.E.cpu().numpy()) <= 5e-6 * np.linalg.norm(G)
+
+
+def test_free_running_matches_oracle(torch_cuda):
+    """No state resync: rotation-invariant outputs stay close over several steps."""
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    torch = torch_cuda
+    m, n, r, N, tau, steps = 256, 128, 4, 4, 5, 12
+    comp = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=1)
+    Q0 = synth.init_Q(n, r, seed=1)
+    comp.set_state(E=np.zeros((1, N, m, n), np.float32), Q=Q0[None], t=0)
+    o = orc.PowerSGDPlusOracle(m, n, r, N, tau, Q0)
+    for t in range(steps):
+        G = synth.make_gradients(1, m, n, N, step=t)
+        comp.step(torch.as_tensor(G[None], device="cuda:0"))
+        out = o.step(G)
+    comp.materialize_error()
+    assert rel_fro(comp.E[0].cpu().numpy(), out["E"]) <= 1e-3
+    assert projector_distance(comp.P_hat[0].cpu().numpy(), out["P_hat"]) <= 1e-3
+
+
+def test_reset_initialises_state(torch_cuda):
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    comp = PowerSGDPlus(512, 256, 8, 2, seed=11, count=2)
+    q = comp.Q.cpu().numpy().ravel()
+    assert np.all(comp.E.cpu().numpy() == 0)
+    assert abs(q.mean()) < 0.05 and abs(q.std() - 1.0) < 0.05
+    assert abs(np.mean(q ** 3)) < 0.2 and abs(np.mean(q ** 4) - 3.0) < 0.4
+    comp2 = PowerSGDPlus(512, 256, 8, 2, seed=11, count=2)
+    assert np.array_equal(comp2.Q.cpu().numpy().ravel(), q)          # same seed, same Q
+    comp3 = PowerSGDPlus(512, 256, 8, 2, seed=12, count=2)
+    assert not np.array_equal(comp3.Q.cpu().numpy().ravel(), q)
+    assert comp.t == 0 and comp.launch_count() > 0
