@@ -48,7 +48,8 @@ typedef enum {
     PSGD_E_NULL = -2,       /* required pointer is NULL */
     PSGD_E_WORKSPACE = -3,  /* workspace too small or buffers not attached */
     PSGD_E_CUDA = -4,       /* a CUDA runtime call failed; see psgd_last_cuda_error */
-    PSGD_E_STATE = -5       /* call not valid in the handle's current state */
+    PSGD_E_STATE = -5,      /* call not valid in the handle's current state */
+    PSGD_E_TOO_LARGE = -6   /* problem does not fit the fixed scratch of psgd_backproject_static */
 } psgd_status;
 
 /* warning bits of the device status word */
@@ -172,6 +173,38 @@ const char* psgd_last_cuda_error(const psgd_handle* h);
 
 /* Frees host memory of the handle.  Never touches caller-owned device buffers. */
 psgd_status psgd_destroy(psgd_handle* h);
+
+/*
+ * Back-projection without a workspace.  (An addition of this library: the paper has no
+ * counterpart; the operation itself is the Q^(i) <- Delta^(i)^T P~ / All-Reduce-Mean pair of
+ * Algorithm 1.)
+ *
+ * Some callers cannot allocate device memory at all: a plug-in running inside a serving
+ * process whose memory pool already owns the whole GPU, code that runs where cudaMalloc is
+ * not allowed or would stall every stream on the device, or a tightly budgeted job that was
+ * given fixed input/output buffers and nothing else.  The handle API above needs a workspace
+ * from them; this call does not.  It computes, for ONE matrix on N nodes,
+ *     Q_node[i] = M[i]^T P_hat   (i = 0..N-1)      and      Q_mean = (1/N) sum_i Q_node[i]
+ * with M [N][m][n], P_hat [m][r], Q_node [N][n][r] (may be NULL), Q_mean [n][r]; all DEVICE,
+ * float32, row-major, caller-owned.  The partial sums over row chunks go to a fixed array of
+ * PSGD_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU that loads the
+ * library gives up that much memory until the process exits.
+ *
+ * Limits and rules:
+ *  - N * n * r * 4 bytes must not exceed PSGD_STATIC_SCRATCH_BYTES, otherwise PSGD_E_TOO_LARGE
+ *    is returned and nothing is launched; m >= n >= r >= 1, r <= 128 as elsewhere.
+ *  - The first call on each device looks up the array's device address (a CUDA runtime query,
+ *    no allocation); make that first call outside any stream capture.
+ *  - The call allocates and frees nothing and does not synchronise.
+ *  - All calls on a device share the one array, and it keeps whatever the previous call left
+ *    there.  Each call overwrites every entry it later reads, so stale contents are harmless,
+ *    but two calls that may run at the same time on the GPU (different streams) race on it:
+ *    keep all calls on one stream or order them yourself.
+ */
+#define PSGD_STATIC_SCRATCH_BYTES (8u << 20)
+psgd_status psgd_backproject_static(const float* M /*DEVICE*/, const float* P_hat /*DEVICE*/,
+                                    float* Q_node /*DEVICE*/, float* Q_mean /*DEVICE*/,
+                                    int64_t m, int64_t n, int r, int N, psgd_stream stream);
 
 #ifdef __cplusplus
 }

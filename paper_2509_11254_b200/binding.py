@@ -13,7 +13,7 @@ PSGD_BUF = {"P_node": 1, "Q_node": 2, "P_hat": 3, "Dbar": 4, "P_mean": 5}
 KERNEL_FAMILIES = ["project", "orth", "backproject", "residual", "refresh", "misc"]
 
 _STATUS = {0: "PSGD_OK", -1: "PSGD_E_INVALID", -2: "PSGD_E_NULL", -3: "PSGD_E_WORKSPACE",
-           -4: "PSGD_E_CUDA", -5: "PSGD_E_STATE"}
+           -4: "PSGD_E_CUDA", -5: "PSGD_E_STATE", -6: "PSGD_E_TOO_LARGE"}
 
 # every symbol include/psgd.h declares: name -> (restype, argtypes)
 _vp, _i64, _u64, _int, _sz = C.c_void_p, C.c_int64, C.c_uint64, C.c_int, C.c_size_t
@@ -38,6 +38,7 @@ SIGNATURES = {
     "psgd_profile_read": (_int, [_vp, C.POINTER(C.c_float), C.POINTER(_int)]),
     "psgd_last_cuda_error": (C.c_char_p, [_vp]),
     "psgd_destroy": (_int, [_vp]),
+    "psgd_backproject_static": (_int, [_vp, _vp, _vp, _vp, _i64, _i64, _int, _int, _vp]),
 }
 
 
@@ -210,3 +211,23 @@ class PowerSGDPlus:
             self.close()
         except Exception:
             pass
+
+
+def backproject_static(M, P_hat, Q_mean, Q_node=None, stream=None):
+    """Q_node[i] = M[i]^T P_hat and their mean, through the entry point that allocates nothing.
+
+    M [N,m,n], P_hat [m,r], Q_mean [n,r], Q_node [N,n,r] or None: contiguous float32 CUDA tensors
+    owned by the caller.  Raises PSGDError(PSGD_E_TOO_LARGE) when N*n*r*4 exceeds the fixed scratch.
+    """
+    import torch
+
+    N, m, n = M.shape
+    r = P_hat.shape[1]
+    for t in (M, P_hat, Q_mean) + ((Q_node,) if Q_node is not None else ()):
+        if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+            raise PSGDError("tensors must be contiguous float32 CUDA tensors")
+    s = stream if stream is not None else torch.cuda.current_stream(M.device)
+    with torch.cuda.device(M.device):
+        _check(lib().psgd_backproject_static(M.data_ptr(), P_hat.data_ptr(),
+                                             Q_node.data_ptr() if Q_node is not None else None,
+                                             Q_mean.data_ptr(), m, n, r, N, _vp(s.cuda_stream)))

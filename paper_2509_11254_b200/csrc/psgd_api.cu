@@ -551,3 +551,5 @@ psgd_status psgd_destroy(psgd_handle* h) {
 }
 
 }  // extern "C"
+
+#include "psgd_noalloc.cu"
