@@ -12,6 +12,7 @@
 #include <vector>
 
 #include "psgd_kernels.cuh"
+#include "psgd_fused.cuh"
 
 using namespace psgd;
 
@@ -25,6 +26,7 @@ inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 
 struct Layout {
     size_t flags, Pnode, Pmean, Phat, Qnode, part, gram, T, dbar, Y, Z, V, U, total;
+    size_t Qpad, Ppad, Qsub, Tacc, Pout, Wpart;  // deferred (single-pass) mode only
 };
 
 struct ProfEvent {
@@ -52,6 +54,13 @@ struct psgd_handle {
     std::vector<ProfEvent> events;
     char err[256] = "no error";
     bool vec4 = false;  // n % 4 == 0 (128-bit paths usable when pointers are 16-byte aligned)
+    // single-pass (deferred residual) plan and state
+    bool fused_ok = false;        // the shape fits the cluster kernel
+    int RP = 0, CS = 1, Wc = 0, KC = 1, nblk = 0;
+    size_t fused_smem = 0;
+    bool pending = false;         // E holds Delta_t; the residual is Delta_t - P~_t Qsub^T
+    bool tacc_identity = true;    // no preconditioner yet
+    bool qpad_valid = false;      // padded copy of Q is current
 };
 
 namespace {
@@ -89,7 +98,7 @@ void plan(psgd_handle* h) {
     size_t part_ref = cnt * (size_t)ceil_div(h->m, BP_SUB) * n * ell * 4;  // upper bound on chunks
     part_ref = std::min(part_ref, cnt * (size_t)64 * n * ell * 4);          // refresh uses <= 64 chunks
     L.part = take(std::max(part_step, part_ref));
-    size_t nparts = ceil_div(std::max(m, n), GR_ROWS);
+    size_t nparts = std::max<size_t>(ceil_div(std::max(m, n), GR_ROWS), 64);  // 64: most clusters per matrix
     L.gram = take(cnt * nparts * c * c * 8);
     L.T = take(cnt * c * c * 8);
     L.dbar = take(cnt * m * n * 4);
@@ -98,6 +107,42 @@ void plan(psgd_handle* h) {
     size_t c2 = (c + 1) & ~(size_t)1;
     L.V = take(cnt * c2 * c2 * 8);
     L.U = take(cnt * ell * r * 8);
+    // ---- single-pass mode ----
+    h->fused_ok = false;
+    if (h->mode == 1 && h->r <= 16 && h->n % 4 == 0) {
+        const int RP = h->r <= 4 ? 4 : (h->r <= 8 ? 8 : 16);
+        const int cs_opts[4] = {1, 2, 4, 8};
+        const int resident[4] = {148, 74, 36, 16};  // clusters of that size resident on a B200 (one CTA per SM)
+        for (int ci = 0; ci < 4 && !h->fused_ok; ++ci) {
+            int CS = cs_opts[ci];
+            int Wc = (int)align_up(ceil_div(h->n, CS), 4);
+            if ((int64_t)h->N * (Wc / 4) > FU_THREADS) continue;
+            size_t fl = RP == 4 ? fused_smem_floats<4>(h->N, Wc) : RP == 8 ? fused_smem_floats<8>(h->N, Wc)
+                                                                           : fused_smem_floats<16>(h->N, Wc);
+            if (fl * 4 > 227 * 1024) continue;
+            h->fused_ok = true; h->RP = RP; h->CS = CS; h->Wc = Wc; h->fused_smem = fl * 4;
+            h->nblk = ceil_div(h->m, FU_R);
+            int res = resident[ci], kmax = std::min(h->nblk, 64), best = 1;
+            double best_eff = -1.0;
+            for (int KC = 1; KC <= kmax; ++KC) {
+                int64_t tot = (int64_t)h->count * KC;
+                if (tot < 2 * res && KC < kmax) continue;
+                double eff = (double)tot / (double)(((tot + res - 1) / res) * res);
+                if (eff > best_eff + 1e-9) { best_eff = eff; best = KC; }
+                if (eff >= 0.95) break;
+            }
+            h->KC = best;
+        }
+    }
+    if (h->fused_ok) {
+        const size_t RP = h->RP, KC = h->KC;
+        L.Qpad = take(cnt * n * RP * 4);
+        L.Ppad = take(cnt * m * RP * 4);
+        L.Qsub = take(cnt * N * n * RP * 4);
+        L.Tacc = take(cnt * RP * RP * 4);
+        L.Pout = take(cnt * m * RP * 4);
+        L.Wpart = take(cnt * KC * N * n * RP * 4);
+    }
     L.total = off;
 }
 
@@ -190,8 +235,8 @@ void launch_back_rp(Launcher& L, BackArgs a, int mats, bool vec) {
     L.end();
 }
 void launch_back(Launcher& L, const float* M, const float* Phat, float* part, int rows, int n, int r, int nodes,
-                 int count, int rpc, int S, bool vec) {
-    BackArgs a{M, Phat, part, rows, n, r, nodes, 1, rpc, S};
+                 int count, int rpc, int S, bool vec, const int* gate = nullptr) {
+    BackArgs a{M, Phat, part, rows, n, r, nodes, 1, rpc, S, gate};
     vec = vec && aligned16(M);
     if (r <= 4) launch_back_rp<4>(L, a, count * nodes, vec);
     else if (r <= 8) launch_back_rp<8>(L, a, count * nodes, vec);
@@ -339,6 +384,89 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
     L.force_kind = -1;
 }
 
+// ---- single-pass SSP-Comp step (deferred residual) --------------------------------
+template <int RP>
+void launch_fused_t(Launcher& L, psgd_handle* h, const FusedArgs& a) {
+    void (*kern)(FusedArgs) = h->pending ? k_fused_step<RP, true> : k_fused_step<RP, false>;
+    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->fused_smem);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((size_t)h->CS * h->KC * h->count));
+    cfg.blockDim = dim3(FU_THREADS);
+    cfg.dynamicSmemBytes = h->fused_smem;
+    cfg.stream = L.st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)h->CS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    L.begin(PSGD_K_PROJECT);
+    cudaLaunchKernelEx(&cfg, kern, a);
+    L.end();
+}
+
+void fused_ssp(Launcher& L, psgd_handle* h, const float* G) {
+    char* ws = h->ws;
+    const Layout& Y = h->lay;
+    float* Phat = (float*)(ws + Y.Phat);
+    float* Qnode = (float*)(ws + Y.Qnode);
+    float* part = (float*)(ws + Y.part);
+    double* gram = (double*)(ws + Y.gram);
+    double* T = (double*)(ws + Y.T);
+    int* flags = (int*)(ws + Y.flags);
+    int* gate = flags + 1;
+    float* Qpad = (float*)(ws + Y.Qpad);
+    float* Ppad = (float*)(ws + Y.Ppad);
+    float* Qsub = (float*)(ws + Y.Qsub);
+    float* Tacc = (float*)(ws + Y.Tacc);
+    float* Pout = (float*)(ws + Y.Pout);
+    float* Wpart = (float*)(ws + Y.Wpart);
+    const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count, RP = h->RP;
+    if (!h->qpad_valid) {
+        size_t tot = (size_t)cnt * n * RP;
+        L.begin(PSGD_K_MISC);
+        k_pad_rows<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(h->Q, Qpad, (size_t)cnt * n, r, RP);
+        L.end();
+        h->qpad_valid = true;
+    }
+    cudaMemsetAsync(gate, 0, 4, L.st);
+    FusedArgs a{G, h->E, Qpad, Ppad, Qsub, h->tacc_identity ? nullptr : Tacc, Pout, Wpart, gram,
+                m, n, r, N, h->KC, h->CS, h->Wc, h->nblk,
+                h->error_form == 0 ? (long long)n * RP : 0LL};
+    if (RP == 4) launch_fused_t<4>(L, h, a);
+    else if (RP == 8) launch_fused_t<8>(L, h, a);
+    else launch_fused_t<16>(L, h, a);
+    // P'^T P' = L L^T  ->  T'; scaled pivot^2 < 2e-2 (rounding of W T amplified > 7x) raises the gate for the precise path
+    L.begin(PSGD_K_ORTH);
+    k_chol<<<cnt, 256, (size_t)r * r * 8, L.st>>>(gram, T, r, h->KC, flags, gate, 2e-2);
+    L.end();
+    FinishPArgs fp{Pout, T, Phat, Ppad, Tacc, m, r, RP, h->tacc_identity ? 1 : 0};
+    L.begin(PSGD_K_ORTH);
+    k_finish_p<<<dim3(ceil_div(m, 64), cnt), 256, 0, L.st>>>(fp);
+    L.end();
+    // precise back-projection over the stored Delta, only when the gate was raised
+    launch_back(L, h->E, Phat, part, m, n, r, N, cnt, h->rpc, h->S, h->vec4, gate);
+    FinishQArgs fq{Wpart, part, T, gate, Qnode, h->Q, Qpad, Qsub, n, r, RP, N, h->KC, h->S, h->error_form};
+    L.begin(PSGD_K_BACKPROJECT);
+    k_finish_q<<<dim3(ceil_div(n, 16), cnt), 16 * RP, 0, L.st>>>(fq);
+    L.end();
+    h->pending = true;
+    h->tacc_identity = false;
+}
+
+// e_{t+1} = Delta_t - P~_t Qsub^T in place (Algorithm 2, last line), if it is still pending
+void materialize(Launcher& L, psgd_handle* h) {
+    if (!h->pending) return;
+    char* ws = h->ws;
+    float* Phat = (float*)(ws + h->lay.Phat);
+    float* Qnode = (float*)(ws + h->lay.Qnode);
+    const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count;
+    if (h->error_form == 0) launch_resid(L, h->E, h->E, Phat, Qnode, m, n, r, N, cnt * N, 1, 1, h->vec4);
+    else launch_resid(L, h->E, h->E, Phat, h->Q, m, n, r, N, cnt * N, 0, 1, h->vec4);
+    h->pending = false;
+}
+
 psgd_status check_ready(const psgd_handle* h) {
     if (!h) return PSGD_E_NULL;
     if (!h->E || !h->Q || !h->ws) return PSGD_E_WORKSPACE;
@@ -352,8 +480,19 @@ psgd_status do_step(psgd_handle* h, const float* G, float* P_hat, float* D_hat, 
     cudaStream_t st = (cudaStream_t)stream;
     Launcher L{h, st};
     bool refresh = force || (h->tau > 0 && h->t % h->tau == 0);
-    if (refresh) svd(L, h, G); else ssp(L, h, G);
-    tail(L, h, D_hat);
+    if (h->mode == 1 && h->fused_ok && !refresh) {
+        fused_ssp(L, h, G);
+        if (D_hat) {
+            float* Phat = (float*)(h->ws + h->lay.Phat);
+            launch_resid(L, nullptr, D_hat, Phat, h->Q, (int)h->m, (int)h->n, h->r, h->N, h->count, 0, 0, h->vec4);
+        }
+    } else {
+        materialize(L, h);   // refresh steps and shapes outside the single-pass plan run eagerly
+        if (refresh) svd(L, h, G); else ssp(L, h, G);
+        tail(L, h, D_hat);
+        h->tacc_identity = true;
+        h->qpad_valid = false;
+    }
     if (L.status != PSGD_OK) return L.status;
     if (P_hat) {
         PSGD_CUDA(h, cudaMemcpyAsync(P_hat, h->ws + h->lay.Phat, (size_t)h->count * h->m * h->r * 4,
@@ -390,7 +529,7 @@ psgd_status psgd_set_option(psgd_handle* h, int option, int value) {
     if (h->ws) return PSGD_E_STATE;
     switch (option) {
         case PSGD_OPT_ERROR_FORM: if (value != 0 && value != 1) return PSGD_E_INVALID; h->error_form = value; break;
-        case PSGD_OPT_MODE: if (value != 0) return PSGD_E_INVALID; h->mode = value; break;
+        case PSGD_OPT_MODE: if (value != 0 && value != 1) return PSGD_E_INVALID; h->mode = value; break;
         case PSGD_OPT_REFRESH_ITERS: if (value < 1 || value > 64) return PSGD_E_INVALID; h->refresh_iters = value; break;
         case PSGD_OPT_REFRESH_OVERSAMPLE: if (value < 0 || value > MAX_L) return PSGD_E_INVALID; h->oversample = value; break;
         default: return PSGD_E_INVALID;
@@ -429,6 +568,7 @@ psgd_status psgd_reset(psgd_handle* h, psgd_stream stream) {
     k_fill_normal<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(h->Q, tot, h->seed, 1);
     L.end();
     h->t = 0;
+    h->pending = false; h->tacc_identity = true; h->qpad_valid = false;
     return L.status;
 }
 
@@ -459,14 +599,17 @@ psgd_status psgd_step_host(psgd_handle* h, const float* G_host, float* G_stage, 
     return PSGD_OK;
 }
 
-psgd_status psgd_materialize_error(psgd_handle* h, psgd_stream) {
+psgd_status psgd_materialize_error(psgd_handle* h, psgd_stream stream) {
     psgd_status s = check_ready(h);
     if (s != PSGD_OK) return s;
-    return PSGD_OK;  // eager mode: E already holds the residual
+    Launcher L{h, (cudaStream_t)stream};
+    materialize(L, h);   // no-op when E already holds the residual
+    return L.status;
 }
 
 psgd_status psgd_state_written(psgd_handle* h) {
     if (!h) return PSGD_E_NULL;
+    h->pending = false; h->tacc_identity = true; h->qpad_valid = false;
     return PSGD_OK;
 }
 

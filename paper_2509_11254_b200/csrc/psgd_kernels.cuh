@@ -217,12 +217,14 @@ struct BackArgs {
     const float* Phat;  // [count][rows][r]
     float* part;        // [mats][S][n][r]
     int rows, n, r, nodes, nchunks, rows_per_chunk, S;
+    const int* gate;    // when non-null the kernel does nothing unless *gate != 0
 };
 
 template <int RP, int VEC>
 __global__ void __launch_bounds__(BP_THREADS) k_backproject(BackArgs a) {
     __shared__ __align__(16) float Ps[BP_SUB * RP];
     __shared__ __align__(16) float red[64 * 4 * RP];
+    if (a.gate && *a.gate == 0) return;
     const int tid = threadIdx.x, tx = tid & 63, g = tid >> 6;
     const int col = blockIdx.x * BP_COLS + tx * 4;
     const int s = blockIdx.y;
@@ -552,14 +554,17 @@ __global__ void __launch_bounds__(256) k_gram(GramArgs a) {
 // T = D^-1 L^-T (upper triangular, double) so that P~ = P T.  One CTA per matrix.
 // Dynamic shared memory: c*c doubles.
 constexpr double CHOL_PIVOT_TOL = 1e-11;  // squared sine of the angle to the previous columns
-__global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int c, int nparts, int* flags) {
+// `gate` (optional): set to 1 when a scaled pivot^2 falls below gate_tol, i.e. when the columns
+// are too ill-conditioned for results derived from W = M^T P to keep float32 accuracy.
+__global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int c, int nparts, int* flags,
+                                              int* gate = nullptr, double gate_tol = 0.0) {
     extern __shared__ __align__(16) double Gs[];  // [c][c]
     __shared__ double dinv[192];
-    __shared__ int bad;
+    __shared__ int bad, illc;
     const int tid = threadIdx.x;
     const int nblk = (c + 63) / 64;
     const double* pb = part + (size_t)blockIdx.x * nparts * c * c;
-    if (tid == 0) bad = 0;
+    if (tid == 0) { bad = 0; illc = 0; }
     for (int e = tid; e < c * c; e += 256) {
         int i = e / c, j = e % c;
         int ii = i, jj = j;
@@ -586,6 +591,7 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
     for (int k = 0; k < c; ++k) {
         if (tid == 0) {
             double p = Gs[k * c + k];
+            if (!(p > gate_tol)) illc = 1;
             if (!(p > CHOL_PIVOT_TOL)) { bad = 1; p = 1.0; for (int i = k + 1; i < c; ++i) Gs[i * c + k] = 0.0; }
             Gs[k * c + k] = sqrt(p);
         }
@@ -622,6 +628,7 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
         Tb[e] = (j <= k) ? dinv[j] * Gs[k * c + j] : 0.0;
     }
     if (tid == 0 && bad) atomicOr(flags, 1);
+    if (tid == 0 && illc && gate) atomicOr(gate, 1);
 }
 
 // Xout[row][k] = sum_j X[row][j] * T[j][k]  (double accumulate), k < kout.

@@ -4,8 +4,9 @@ Every comparison starts both sides from IDENTICAL state: the oracle's state is
 rounded to float32, uploaded, and the oracle continues from the rounded values.
 Tolerances (float32 path vs double oracle):
   relative Frobenius error <= 1e-5 on P~, Q, Q_i, P_i and E
-  (E's denominator is floored at 1e-3 * ||M||_F so that exact-low-rank inputs,
-  whose residual is pure rounding noise, are still comparable);
+  (E's denominator is floored at 1e-2 * ||M||_F: E = M - P~Q_i^T is a cancellation whose
+  float32 rounding error is about eps * ||M||_F ~ 1e-7 ||M||_F whatever the size of E, so a
+  relative bound of 1e-5 is only meaningful down to ||E||_F ~ 1e-2 ||M||_F);
   after a refresh: projector distance ||P~P~^T - P~_ref P~_ref^T||_F <= 1e-4 when
   the spectrum of the node mean has a gap (sigma_r - sigma_{r+1}) / sigma_1 >= 2e-3,
   otherwise only the residual norm ||Dbar - P~P~^T Dbar||_F must match (1e-5).
@@ -65,14 +66,15 @@ def compare_step(out, gpu, m, n, r, N, tag):
             # rotation-invariant quantities
             rot = P_ref.T @ Pg                      # r x r, ~orthogonal
             assert rel_fro(gpu["Q"], out["Q"] @ rot) <= 2 * PROJ_TOL, f"{tag}: Q after refresh"
-            e = rel_fro(gpu["E"], out["E"], floor=1e-3 * normM)
+            e = rel_fro(gpu["E"], out["E"], floor=1e-2 * normM)
             assert e <= 2 * PROJ_TOL, f"{tag}: E after refresh {e}"
         return
-    assert rel_fro(gpu["P_node"], out["P_i"]) <= TOL, f"{tag}: P_i"
+    if "P_node" in gpu:
+        assert rel_fro(gpu["P_node"], out["P_i"]) <= TOL, f"{tag}: P_i"
     assert rel_fro(gpu["P_hat"], P_ref) <= TOL, f"{tag}: P~ {rel_fro(gpu['P_hat'], P_ref)}"
     assert rel_fro(gpu["Q"], out["Q"]) <= TOL, f"{tag}: Q"
     assert rel_fro(gpu["Q_node"], out["Q_i"]) <= TOL, f"{tag}: Q_i"
-    e = rel_fro(gpu["E"], out["E"], floor=1e-3 * normM)
+    e = rel_fro(gpu["E"], out["E"], floor=1e-2 * normM)
     assert e <= TOL, f"{tag}: E {e}"
 
 
@@ -104,7 +106,9 @@ def run_case(torch, m, n, r, N, tau, steps, workload=1, count=1, error_form="loc
         assert flags == 0, f"step {t}: warning flags {flags}"
         assert comp.t == t + 1
         gp = dict(P_hat=comp.P_hat.cpu().numpy(), Q=comp.Q.cpu().numpy(), E=comp.E.cpu().numpy(),
-                  P_node=comp.debug("P_node").cpu().numpy(), Q_node=comp.debug("Q_node").cpu().numpy())
+                  Q_node=comp.debug("Q_node").cpu().numpy())
+        if mode == "eager":   # the single-pass kernel never materialises the per-node P_i
+            gp["P_node"] = comp.debug("P_node").cpu().numpy()
         for c, o in enumerate(oracles):
             out = o.step(G[c])
             compare_step(out, {k: v[c] for k, v in gp.items()}, m, n, r, N, f"t={t} c={c}")
@@ -210,3 +214,60 @@ def test_reset_initialises_state(torch_cuda):
     comp3 = PowerSGDPlus(512, 256, 8, 2, seed=12, count=2)
     assert not np.array_equal(comp3.Q.cpu().numpy().ravel(), q)
     assert comp.t == 0 and comp.launch_count() > 0
+
+
+# ---- single-pass (deferred residual) mode -------------------------------------------
+def test_deferred_config1_tiny_20_steps(torch_cuda):
+    run_case(torch_cuda, 256, 128, 4, 4, tau=5, steps=20, workload=1, mode="deferred")
+
+
+@pytest.mark.parametrize("m,n,r,N,count,workload", [
+    (300, 200, 8, 2, 3, 2),      # one CTA per cluster, ragged rows, batch of 3
+    (96, 96, 1, 5, 1, 2),        # r = 1
+    (64, 8, 8, 2, 1, 2),         # n == r
+    (513, 260, 16, 1, 1, 5),     # N = 1, r = 16, ragged rows, partial last chunk
+    (768, 768, 8, 8, 2, 2),      # cluster of 4 CTAs (config-2 shape)
+    (4112, 4096, 16, 4, 1, 5),   # cluster of 8 CTAs (config-5 columns), ragged last row block
+    (784, 768, 16, 16, 1, 3),    # 16 nodes, cluster of 8, slice narrower than two chunks
+    (130, 66, 5, 2, 2, 2),       # n % 4 != 0: falls back to the eager kernels
+])
+def test_deferred_step_by_step(torch_cuda, m, n, r, N, count, workload):
+    run_case(torch_cuda, m, n, r, N, tau=0, steps=3, workload=workload, count=count, Einit=0.01, mode="deferred")
+
+
+def test_deferred_mean_error_form(torch_cuda):
+    run_case(torch_cuda, 192, 128, 4, 3, tau=0, steps=3, workload=2, error_form="mean", Einit=0.01, mode="deferred")
+
+
+@pytest.mark.parametrize("m,n,r,N,workload,tau", [(256, 128, 4, 4, 1, 5), (768, 768, 8, 8, 2, 0), (1040, 1024, 16, 4, 5, 4)])
+def test_deferred_free_running(torch_cuda, m, n, r, N, workload, tau):
+    """Several steps without resync: pending residuals and the preconditioner are in play."""
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    torch = torch_cuda
+    steps = 9
+    comp = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=1, mode="deferred")
+    eager = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=1, mode="eager")
+    Q0 = synth.init_Q(n, r, seed=1)
+    for cpt in (comp, eager):
+        cpt.set_state(E=np.zeros((1, N, m, n), np.float32), Q=Q0[None], t=0)
+    o = orc.PowerSGDPlusOracle(m, n, r, N, tau, Q0)
+    for t in range(steps):
+        G = synth.make_gradients(workload, m, n, N, step=t)
+        Gd = torch.as_tensor(G[None], device="cuda:0")
+        comp.step(Gd)
+        eager.step(Gd)
+        out = o.step(G)
+    comp.materialize_error()
+    assert comp.last_status() == 0
+    normM = np.linalg.norm(out["M"])
+    Pd, Pe = comp.P_hat[0].cpu().numpy(), eager.P_hat[0].cpu().numpy()
+    assert projector_distance(Pd, out["P_hat"]) <= 1e-3
+    assert rel_fro(comp.E[0].cpu().numpy(), out["E"], floor=1e-2 * normM) <= 1e-3
+    # the two GPU modes compute the same thing with different rounding
+    assert projector_distance(Pd, Pe) <= 1e-3
+    assert rel_fro(comp.E[0].cpu().numpy(), eager.E[0].cpu().numpy(), floor=1e-2 * normM) <= 1e-3
+    # idempotent
+    e1 = comp.E.clone()
+    comp.materialize_error()
+    assert torch.equal(e1, comp.E)
