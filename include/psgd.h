@@ -55,6 +55,7 @@ typedef enum {
 /* warning bits of the device status word */
 #define PSGD_W_RANK_DEFICIENT 1 /* a pivot of the orthogonalisation fell below tolerance */
 #define PSGD_W_NOT_CONVERGED 2  /* the eigen-solver of the refresh hit its sweep limit */
+#define PSGD_W_TIMEOUT 4        /* a bounded wait inside a kernel ran out (results of that step are invalid) */
 
 /* options for psgd_set_option */
 #define PSGD_OPT_ERROR_FORM 1   /* 0 (default): e_i <- Delta_i - P~ Q_i^T  (Algorithm 2, last line)
@@ -155,6 +156,14 @@ psgd_status psgd_last_status(psgd_handle* h, psgd_stream stream, int* flags /*HO
 
 /* Test hook: DEVICE address and byte size of an internal buffer (PSGD_BUF_*). */
 psgd_status psgd_debug_ptr(psgd_handle* h, int which, void** ptr, size_t* bytes);
+
+/*
+ * Launch plan of the handle, 8 ints (HOST): [0] 1 if the single-pass kernel serves this shape in
+ * deferred mode, [1] rank padding, [2] columns per CTA, [3] CTAs per cluster, [4] row slots per
+ * matrix, [5] clusters resident at once (-1 before the first single-pass launch), [6] its dynamic
+ * shared memory in bytes, [7] row chunks of the eager back-projection.
+ */
+psgd_status psgd_plan_info(const psgd_handle* h, int* info /*HOST*/);
 
 /* Number of kernels this handle has launched since creation. */
 psgd_status psgd_launch_count(const psgd_handle* h, int64_t* launches);

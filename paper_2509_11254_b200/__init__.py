@@ -11,5 +11,6 @@ from .binding import (  # noqa: F401
     library_path,
     PSGD_W_RANK_DEFICIENT,
     PSGD_W_NOT_CONVERGED,
+    PSGD_W_TIMEOUT,
     KERNEL_FAMILIES,
 )

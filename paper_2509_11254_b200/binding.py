@@ -8,6 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 
 PSGD_W_RANK_DEFICIENT = 1
 PSGD_W_NOT_CONVERGED = 2
+PSGD_W_TIMEOUT = 4
 PSGD_OPT_ERROR_FORM, PSGD_OPT_MODE, PSGD_OPT_REFRESH_ITERS, PSGD_OPT_REFRESH_OVERSAMPLE = 1, 2, 3, 4
 PSGD_BUF = {"P_node": 1, "Q_node": 2, "P_hat": 3, "Dbar": 4, "P_mean": 5}
 KERNEL_FAMILIES = ["project", "orth", "backproject", "residual", "refresh", "misc"]
@@ -33,6 +34,7 @@ SIGNATURES = {
     "psgd_set_step": (_int, [_vp, _i64]),
     "psgd_last_status": (_int, [_vp, _vp, C.POINTER(_int)]),
     "psgd_debug_ptr": (_int, [_vp, _int, C.POINTER(_vp), C.POINTER(_sz)]),
+    "psgd_plan_info": (_int, [_vp, C.POINTER(_int)]),
     "psgd_launch_count": (_int, [_vp, C.POINTER(_i64)]),
     "psgd_profile_begin": (_int, [_vp]),
     "psgd_profile_read": (_int, [_vp, C.POINTER(C.c_float), C.POINTER(_int)]),
@@ -186,6 +188,12 @@ class PowerSGDPlus:
                  "P_hat": (self.count, self.m, self.r), "Dbar": (self.count, self.m, self.n),
                  "P_mean": (self.count, self.m, self.r)}[name]
         return flat.view(shape).clone()
+
+    def plan_info(self):
+        v = (_int * 8)()
+        _check(lib().psgd_plan_info(self.h, v))
+        keys = ("single_pass", "RP", "WC", "CS", "KC", "active_clusters", "smem_bytes", "S")
+        return dict(zip(keys, list(v)))
 
     def launch_count(self):
         v = _i64()

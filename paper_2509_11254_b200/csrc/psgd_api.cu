@@ -3,6 +3,7 @@
 // Algorithm 2 (SSP-Comp or SVD-Comp of Algorithm 1 plus the residual update).
 #include "../../include/psgd.h"
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -26,7 +27,7 @@ inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 
 struct Layout {
     size_t flags, Pnode, Pmean, Phat, Qnode, part, gram, T, dbar, Y, Z, V, U, total;
-    size_t Qpad, Ppad, Qsub, Tacc, Pout, Wpart;  // deferred (single-pass) mode only
+    size_t Qpad, Ppad, Qsub, Tacc, Pout, Wpart, Cmat, Cpart;  // deferred (single-pass) mode only
 };
 
 struct ProfEvent {
@@ -56,8 +57,9 @@ struct psgd_handle {
     bool vec4 = false;  // n % 4 == 0 (128-bit paths usable when pointers are 16-byte aligned)
     // single-pass (deferred residual) plan and state
     bool fused_ok = false;        // the shape fits the cluster kernel
-    int RP = 0, CS = 1, Wc = 0, KC = 1, nblk = 0;
+    int RP = 0, CS = 1, WC = 0, KC = 1, KCmax = 1, nblk = 0;
     size_t fused_smem = 0;
+    int active_clusters = -1;     // clusters of the single-pass kernel resident at once (known after its first launch)
     bool pending = false;         // E holds Delta_t; the residual is Delta_t - P~_t Qsub^T
     bool tacc_identity = true;    // no preconditioner yet
     bool qpad_valid = false;      // padded copy of Q is current
@@ -108,40 +110,45 @@ void plan(psgd_handle* h) {
     L.V = take(cnt * c2 * c2 * 8);
     L.U = take(cnt * ell * r * 8);
     // ---- single-pass mode ----
+    // A CTA owns WC in {128, 256, 512} columns of every node; the tile of S it keeps on chip and the
+    // registers of its back-projection bound N * WC by 2048.  CS = ceil(n / WC) CTAs form a cluster.
     h->fused_ok = false;
-    if (h->mode == 1 && h->r <= 16 && h->n % 4 == 0) {
-        const int RP = h->r <= 4 ? 4 : (h->r <= 8 ? 8 : 16);
-        const int cs_opts[4] = {1, 2, 4, 8};
-        const int resident[4] = {148, 74, 36, 16};  // clusters of that size resident on a B200 (one CTA per SM)
-        for (int ci = 0; ci < 4 && !h->fused_ok; ++ci) {
-            int CS = cs_opts[ci];
-            int Wc = (int)align_up(ceil_div(h->n, CS), 4);
-            if ((int64_t)h->N * (Wc / 4) > FU_THREADS) continue;
-            size_t fl = RP == 4 ? fused_smem_floats<4>(h->N, Wc) : RP == 8 ? fused_smem_floats<8>(h->N, Wc)
-                                                                           : fused_smem_floats<16>(h->N, Wc);
-            if (fl * 4 > 227 * 1024) continue;
-            h->fused_ok = true; h->RP = RP; h->CS = CS; h->Wc = Wc; h->fused_smem = fl * 4;
+    if (h->mode == 1 && h->r <= 8 && h->n % 4 == 0 && h->N <= 16) {
+        const int RP = h->r <= 4 ? 4 : 8;
+        const int wcmax = h->N <= 4 ? 512 : (h->N <= 8 ? 256 : 128);
+        int bestWC = 0, bestCS = 0;
+        int64_t bestWaste = -1;
+        for (int WC = 128; WC <= wcmax; WC *= 2) {
+            int CS = ceil_div(h->n, WC);
+            if (CS > FU_MAXCS) continue;
+            int64_t waste = (int64_t)CS * WC - h->n;
+            if (bestWaste < 0 || waste <= bestWaste) { bestWaste = waste; bestWC = WC; bestCS = CS; }
+        }
+        if (bestWC) {
+            h->fused_ok = true; h->RP = RP; h->CS = bestCS; h->WC = bestWC;
+            h->fused_smem = RP == 4 ? (bestWC == 128 ? fused_smem_bytes<4, 128>(h->N) : bestWC == 256 ? fused_smem_bytes<4, 256>(h->N) : fused_smem_bytes<4, 512>(h->N))
+                                    : (bestWC == 128 ? fused_smem_bytes<8, 128>(h->N) : bestWC == 256 ? fused_smem_bytes<8, 256>(h->N) : fused_smem_bytes<8, 512>(h->N));
             h->nblk = ceil_div(h->m, FU_R);
-            int res = resident[ci], kmax = std::min(h->nblk, 64), best = 1;
-            double best_eff = -1.0;
-            for (int KC = 1; KC <= kmax; ++KC) {
-                int64_t tot = (int64_t)h->count * KC;
-                if (tot < 2 * res && KC < kmax) continue;
-                double eff = (double)tot / (double)(((tot + res - 1) / res) * res);
-                if (eff > best_eff + 1e-9) { best_eff = eff; best = KC; }
-                if (eff >= 0.95) break;
-            }
-            h->KC = best;
+            // Row slots per matrix.  The workspace is sized here, on the host, for KCmax slots from a table of
+            // the clusters of each size that a B200 keeps resident (one CTA per SM); the first launch asks the
+            // device for the real number and picks KC <= KCmax for whole waves.
+            static const int resident[FU_MAXCS + 1] = {0, 148, 74, 48, 36, 28, 24, 20, 16};
+            h->KCmax = (int)std::max<int64_t>(1, std::min<int64_t>(std::min(std::max(1, h->nblk / 4), 64),
+                                                                   (16 * resident[bestCS] + h->count - 1) / h->count));
+            h->KC = h->KCmax;
+            h->active_clusters = -1;
         }
     }
     if (h->fused_ok) {
-        const size_t RP = h->RP, KC = h->KC;
+        const size_t RP = h->RP, KC = h->KCmax;
         L.Qpad = take(cnt * n * RP * 4);
         L.Ppad = take(cnt * m * RP * 4);
         L.Qsub = take(cnt * N * n * RP * 4);
         L.Tacc = take(cnt * RP * RP * 4);
         L.Pout = take(cnt * m * RP * 4);
         L.Wpart = take(cnt * KC * N * n * RP * 4);
+        L.Cmat = take(cnt * RP * RP * 4);
+        L.Cpart = take(cnt * (size_t)ceil_div(h->n, 16) * RP * RP * 8);
     }
     L.total = off;
 }
@@ -385,12 +392,37 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
 }
 
 // ---- single-pass SSP-Comp step (deferred residual) --------------------------------
-template <int RP>
-void launch_fused_t(Launcher& L, psgd_handle* h, const FusedArgs& a) {
-    void (*kern)(FusedArgs) = h->pending ? k_fused_step<RP, true> : k_fused_step<RP, false>;
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+// Rank-3 map over [count*N][m][n] float32 with tiles of 8 rows x bw columns of one node; out-of-range reads give zeros.
+bool make_tile_map(CUtensorMap* map, const float* base, int64_t n, int64_t m, int64_t mats, int bw) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)n, (cuuint64_t)m, (cuuint64_t)mats};
+    cuuint64_t strides[2] = {(cuuint64_t)n * 4, (cuuint64_t)m * (cuuint64_t)n * 4};
+    cuuint32_t box[3] = {(cuuint32_t)bw, (cuuint32_t)FU_R, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int RP, int WC>
+void launch_fused_t(Launcher& L, psgd_handle* h, const float* G, FusedArgs a) {
+    void (*kern)(CUtensorMap, CUtensorMap, FusedArgs) = h->pending ? k_fused_step<RP, WC, true> : k_fused_step<RP, WC, false>;
     cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->fused_smem);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)((size_t)h->CS * h->KC * h->count));
     cfg.blockDim = dim3(FU_THREADS);
     cfg.dynamicSmemBytes = h->fused_smem;
     cfg.stream = L.st;
@@ -401,9 +433,44 @@ void launch_fused_t(Launcher& L, psgd_handle* h, const FusedArgs& a) {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (h->active_clusters < 0) {
+        cfg.gridDim = dim3((unsigned)((size_t)h->CS * h->KCmax * h->count));
+        int nc = 0;
+        if (cudaOccupancyMaxActiveClusters(&nc, kern, &cfg) != cudaSuccess) { nc = 0; cudaGetLastError(); }
+        h->active_clusters = nc;
+        // row slots: trade the idle tail of the last wave of clusters against the traffic of the
+        // per-slot partial W (written and read once: 2 KC RP / (3 m) of the step's 12 bytes per element)
+        int best = h->KCmax;
+        if (nc > 0) {
+            double best_cost = 1e30;
+            for (int KC = 1; KC <= h->KCmax; ++KC) {
+                int64_t tot = (int64_t)h->count * KC;
+                double eff = (double)tot / (double)(((tot + nc - 1) / nc) * nc);
+                double cost = 1.0 / eff + 2.0 * KC * RP / (3.0 * (double)h->m);
+                if (cost < best_cost - 1e-9) { best_cost = cost; best = KC; }
+            }
+        }
+        h->KC = best;
+    }
+    a.KC = h->KC;
+    cfg.gridDim = dim3((unsigned)((size_t)h->CS * h->KC * h->count));
+    CUtensorMap tmG, tmM;
+    const int bw = FusedGeom<WC>::BW;
+    if (!make_tile_map(&tmG, G, h->n, h->m, (int64_t)h->count * h->N, bw) ||
+        !make_tile_map(&tmM, h->E, h->n, h->m, (int64_t)h->count * h->N, bw)) {
+        snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
+        L.status = PSGD_E_CUDA;
+        return;
+    }
     L.begin(PSGD_K_PROJECT);
-    cudaLaunchKernelEx(&cfg, kern, a);
+    cudaLaunchKernelEx(&cfg, kern, tmG, tmM, a);
     L.end();
+}
+template <int RP>
+void launch_fused_rp(Launcher& L, psgd_handle* h, const float* G, const FusedArgs& a) {
+    if (h->WC == 128) launch_fused_t<RP, 128>(L, h, G, a);
+    else if (h->WC == 256) launch_fused_t<RP, 256>(L, h, G, a);
+    else launch_fused_t<RP, 512>(L, h, G, a);
 }
 
 void fused_ssp(Launcher& L, psgd_handle* h, const float* G) {
@@ -422,8 +489,10 @@ void fused_ssp(Launcher& L, psgd_handle* h, const float* G) {
     float* Tacc = (float*)(ws + Y.Tacc);
     float* Pout = (float*)(ws + Y.Pout);
     float* Wpart = (float*)(ws + Y.Wpart);
+    float* Cmat = (float*)(ws + Y.Cmat);
+    double* Cpart = (double*)(ws + Y.Cpart);
     const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count, RP = h->RP;
-    if (!h->qpad_valid) {
+    if (!h->qpad_valid) {   // first single-pass step after an eager one: no accumulated transform yet, Q' = Q
         size_t tot = (size_t)cnt * n * RP;
         L.begin(PSGD_K_MISC);
         k_pad_rows<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(h->Q, Qpad, (size_t)cnt * n, r, RP);
@@ -431,25 +500,29 @@ void fused_ssp(Launcher& L, psgd_handle* h, const float* G) {
         h->qpad_valid = true;
     }
     cudaMemsetAsync(gate, 0, 4, L.st);
-    FusedArgs a{G, h->E, Qpad, Ppad, Qsub, h->tacc_identity ? nullptr : Tacc, Pout, Wpart, gram,
-                m, n, r, N, h->KC, h->CS, h->Wc, h->nblk,
+    FusedArgs a{h->E, Qpad, Ppad, Qsub, Cmat, Pout, Wpart, gram, flags,
+                m, n, r, N, h->KC, h->CS, h->nblk,
                 h->error_form == 0 ? (long long)n * RP : 0LL};
-    if (RP == 4) launch_fused_t<4>(L, h, a);
-    else if (RP == 8) launch_fused_t<8>(L, h, a);
-    else launch_fused_t<16>(L, h, a);
+    if (RP == 4) launch_fused_rp<4>(L, h, G, a);
+    else launch_fused_rp<8>(L, h, G, a);
+    if (L.status != PSGD_OK) return;
     // P'^T P' = L L^T  ->  T'; scaled pivot^2 < 2e-2 (rounding of W T amplified > 7x) raises the gate for the precise path
     L.begin(PSGD_K_ORTH);
     k_chol<<<cnt, 256, (size_t)r * r * 8, L.st>>>(gram, T, r, h->KC, flags, gate, 2e-2);
     L.end();
-    FinishPArgs fp{Pout, T, Phat, Ppad, Tacc, m, r, RP, h->tacc_identity ? 1 : 0};
+    FinishPArgs fp{Pout, T, Phat, Ppad, Tacc, Tacc, m, r, RP, h->tacc_identity ? 1 : 0};
     L.begin(PSGD_K_ORTH);
     k_finish_p<<<dim3(ceil_div(m, 64), cnt), 256, 0, L.st>>>(fp);
     L.end();
     // precise back-projection over the stored Delta, only when the gate was raised
     launch_back(L, h->E, Phat, part, m, n, r, N, cnt, h->rpc, h->S, h->vec4, gate);
-    FinishQArgs fq{Wpart, part, T, gate, Qnode, h->Q, Qpad, Qsub, n, r, RP, N, h->KC, h->S, h->error_form};
+    const int qblocks = ceil_div(n, 16);
+    FinishQArgs fq{Wpart, part, T, Tacc, gate, Qnode, h->Q, Qpad, Qsub, Cpart, n, r, RP, N, h->KC, h->S, h->error_form};
     L.begin(PSGD_K_BACKPROJECT);
-    k_finish_q<<<dim3(ceil_div(n, 16), cnt), 16 * RP, 0, L.st>>>(fq);
+    k_finish_q<<<dim3(qblocks, cnt), 16 * RP, 0, L.st>>>(fq);
+    L.end();
+    L.begin(PSGD_K_BACKPROJECT);
+    k_sum_c<<<cnt, RP * RP, 0, L.st>>>(Cpart, Cmat, qblocks, RP);
     L.end();
     h->pending = true;
     h->tacc_identity = false;
@@ -480,7 +553,7 @@ psgd_status do_step(psgd_handle* h, const float* G, float* P_hat, float* D_hat, 
     cudaStream_t st = (cudaStream_t)stream;
     Launcher L{h, st};
     bool refresh = force || (h->tau > 0 && h->t % h->tau == 0);
-    if (h->mode == 1 && h->fused_ok && !refresh) {
+    if (h->mode == 1 && h->fused_ok && !refresh && aligned16(G)) {
         fused_ssp(L, h, G);
         if (D_hat) {
             float* Phat = (float*)(h->ws + h->lay.Phat);
@@ -652,6 +725,13 @@ psgd_status psgd_debug_ptr(psgd_handle* h, int which, void** ptr, size_t* bytes)
         case PSGD_BUF_P_MEAN: *ptr = h->ws + h->lay.Pmean; *bytes = c * m * r * 4; break;
         default: return PSGD_E_INVALID;
     }
+    return PSGD_OK;
+}
+
+psgd_status psgd_plan_info(const psgd_handle* h, int* info) {
+    if (!h || !info) return PSGD_E_NULL;
+    info[0] = h->fused_ok ? 1 : 0; info[1] = h->RP; info[2] = h->WC; info[3] = h->CS; info[4] = h->KC;
+    info[5] = h->active_clusters; info[6] = (int)h->fused_smem; info[7] = h->S;
     return PSGD_OK;
 }
 

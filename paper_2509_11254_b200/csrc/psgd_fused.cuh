@@ -5,325 +5,516 @@
 // literally.  This kernel does the whole iteration in ONE pass over HBM (read G, read the
 // stored Delta of the previous step, write the new Delta = 12 bytes per element):
 //
-//   * the residual of the previous step is never stored: E_t = Delta_{t-1} - P~_{t-1} Q_{i,t-1}^T is
-//     rebuilt on the fly from the small factors (Algorithm 2, last line, folded into Eq. (7a));
-//   * a row block's node-mean P[b] = (1/N) sum_i M_i[b,:] Q only needs that row block, so the
-//     contraction W_i += M_i[b,:]^T P[b] can follow while the tile is still in shared memory;
-//   * because P~ = P T for an upper-triangular T (Cholesky QR), Q_i = M_i^T P~ = W_i T is obtained
-//     afterwards from the small matrices alone (k_finish_q), as is P~ itself (k_finish_p).
+//   * the residual of the previous step is never stored: the buffer holds Delta_{t-1} and
+//     e_t = Delta_{t-1} - P~_{t-1} Q_{i,t-1}^T is rebuilt from the small factors (Algorithm 2,
+//     last line, folded into Eq. (7a)):  Delta_t = S - P~_{t-1} Qsub_i^T  with  S = g_t + Delta_{t-1};
+//   * the projection is linear, so it is taken of S and corrected in the small space:
+//         P = (1/N) sum_i Delta_t,i Q = (1/N) sum_i S_i Q  -  P~_{t-1} C,   C = (1/N) sum_i Qsub_i^T Q  (r x r);
+//   * a row block's P only needs that row block, so the contraction W_i += Delta_t,i[b,:]^T P[b]
+//     follows while the block is still in shared memory;
+//   * because P~ = P T for an upper-triangular T (Cholesky QR), Q_i = Delta_i^T P~ = W_i T is obtained
+//     afterwards from the small matrices alone (k_finish_q), as is P~ itself (k_finish_p).  The
+//     previous step's accumulated T is folded into Q beforehand (Q' = Q T), so that P' = P T
+//     comes out nearly orthonormal and W = Delta^T P' keeps float32 accuracy.
 //
-// A thread-block CLUSTER owns a row block of 16 rows for all N nodes; each CTA of the cluster
-// owns a column slice, keeps its slice of the tile in shared memory and exchanges the 16 x r
-// partial sums of P through distributed shared memory.  Float sums are formed in a fixed
-// order everywhere (deterministic results).
+// A thread-block CLUSTER owns row blocks of 8 rows for all N nodes; each CTA of the cluster
+// owns a column slice of WC columns.  G and the stored Delta arrive as TMA tiles (8 rows x up to
+// 256 columns of one node, cp.async.bulk.tensor with zero fill beyond the matrix edges) in a
+// ring of shared-memory stages whose completion is tracked by mbarriers; the warps take turns
+// issuing the copies.  S is kept in a double-buffered shared-memory tile; the 8 x r partial
+// sums of P are pushed to the peers' shared memory (DSMEM) and the cluster barrier is split
+// into arrive / wait so that its latency is covered by the next block's loads and arithmetic.
+// Float sums are formed in a fixed order everywhere (bit-reproducible results).  Every
+// mbarrier wait is bounded; a wait that runs out sets PSGD_W_TIMEOUT in the status word and
+// the kernel carries on to its end.
 #pragma once
 #include <cooperative_groups.h>
+#include <cuda.h>
 
 #include "psgd_kernels.cuh"
 
 namespace psgd {
 namespace cg = cooperative_groups;
 
-constexpr int FU_THREADS = 512;
-constexpr int FU_R = 16;      // rows per block
-constexpr int FU_CH = 64;     // columns per pipeline stage
-constexpr int FU_CHP = 68;    // padded stage row stride (floats)
-constexpr int FU_STAGES = 3;
+constexpr int FU_THREADS = 256;
+constexpr int FU_R = 8;        // rows per block
+constexpr int FU_RG = 4;       // rows per warp task
+constexpr int FU_MAXCS = 8;    // largest cluster
+constexpr unsigned FU_WAIT_LIMIT = 1u << 20;   // polls of one mbarrier wait before giving up
+constexpr int FU_W_TIMEOUT = 4;                // == PSGD_W_TIMEOUT
 
 struct FusedArgs {
-    const float* G;      // [count][N][m][n]
     float* Mbuf;         // [count][N][m][n]  in: Delta_{t-1} (or e_t if !PENDING); out: Delta_t
-    const float* Qpad;   // [count][n][RP]    Q_{t-1}, rows padded to RP
+    const float* Qpad;   // [count][n][RP]    Q' = Q_{t-1} T (preconditioned), rows padded to RP
     const float* Ppad;   // [count][m][RP]    P~_{t-1}           (PENDING only)
     const float* Qsub;   // [count][N or 1][n][RP] factor the pending residual subtracts (PENDING only)
-    const float* Tprev;  // [count][RP][RP] upper-triangular preconditioner, or nullptr (identity)
-    float* Pout;         // [count][m][RP]    P' = P * Tprev (node mean, preconditioned)
-    float* Wpart;        // [count][KC][N][n][RP]  partial W_i = M_i^T P'
+    const float* Cmat;   // [count][RP][RP]   C' = mean_i Qsub_i^T Q'                    (PENDING only)
+    float* Pout;         // [count][m][RP]    P' = P T (node mean, preconditioned)
+    float* Wpart;        // [count][KC][N][n][RP]  partial W_i = Delta_i^T P'
     double* gram;        // [count][KC][r][r]      partial P'^T P'
-    int m, n, r, N, KC, CS, Wc, nblk;
+    int* flags;          // device status word
+    int m, n, r, N, KC, CS, nblk;
     long long qsub_node_stride;  // n*RP, or 0 when all nodes subtract the same factor
 };
 
-template <int RP>
-__host__ __device__ inline size_t fused_smem_floats(int N, int Wc) {
-    size_t Wt = (size_t)Wc + 4;
-    size_t tile = (size_t)N * FU_R * Wt;
-    size_t stage = (size_t)2 * FU_R * FU_CHP + (size_t)FU_CH * RP + (size_t)FU_R * RP;  // G, Mprev, Qsub chunk, P~prev rows
-    size_t qs = (size_t)((Wc + FU_CH - 1) / FU_CH) * FU_CH * RP;   // padded to whole chunks, zero-filled
-    size_t red = (size_t)8 * FU_R * RP;
-    size_t small = (size_t)2 * FU_R * RP /*Ppart*/ + (size_t)FU_R * RP /*Praw*/ + (size_t)FU_R * RP /*Pb*/ + (size_t)RP * RP /*T*/;
-    return tile + FU_STAGES * stage + qs + red + small;
+template <int WC>
+struct FusedGeom {
+    static constexpr int BW = WC >= 256 ? 256 : WC;      // columns of one TMA tile = one stage
+    static constexpr int NH = WC / BW;                   // stages per node and block
+    static constexpr int CPL = BW / 128;                 // columns per lane in the projection phase
+    static constexpr int NCG = 4;                        // column groups per stage (one warp each, two row groups)
+    static constexpr int NST = BW == 256 ? 5 : 8;        // ring depth
+    static constexpr int TPN = WC / 8;                   // back-projection threads per node
+    static constexpr int STAGE_FLOATS = 2 * FU_R * BW;   // G tile, then stored-Delta tile
+};
+
+template <int RP, int WC>
+__host__ __device__ inline size_t fused_smem_bytes(int N) {
+    using Ge = FusedGeom<WC>;
+    size_t fl = (size_t)2 * N * FU_R * WC            // S tile, double-buffered
+              + (size_t)Ge::NST * Ge::STAGE_FLOATS   // ring
+              + (size_t)2 * 2 * Ge::NH * Ge::NCG * 32   // per-warp partial sums of P
+              + (size_t)2 * FU_MAXCS * FU_R * RP     // partial sums received from the cluster
+              + (size_t)2 * FU_R * RP                // P' rows
+              + (size_t)2 * FU_R * RP                // P~_{t-1} rows
+              + (size_t)RP * RP;                     // C'
+    return fl * 4 + (size_t)(2 * Ge::NST + 2) * 8 + 128;   // + alignment slack for the TMA destinations
 }
 
-template <int RP, bool PENDING>
-__global__ void __launch_bounds__(FU_THREADS, 1) k_fused_step(FusedArgs a) {
-    extern __shared__ __align__(16) float smem[];
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after FU_WAIT_LIMIT polls, records it and lets the caller go on; a thread
+// that has given up once no longer waits at all (`dead`), so a broken pipeline still ends quickly.
+__device__ __forceinline__ void mbar_wait(unsigned bar, unsigned parity, int* flags, bool& dead) {
+    if (dead) return;
+    for (unsigned it = 0; it < FU_WAIT_LIMIT; ++it)
+        if (mbar_try_wait(bar, parity)) return;
+    dead = true;
+    atomicOr(flags, FU_W_TIMEOUT);
+}
+// TMA: one tile {x: columns, y: rows, z: (matrix, node)} of a rank-3 tensor map into shared memory.
+// x must be a multiple of 4 floats (16 bytes); coordinates past the extents read zeros.
+__device__ __forceinline__ void tma_load_3d(unsigned dst, const CUtensorMap* map, int x, int y, int z, unsigned bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void cluster_arrive_release() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait_acquire() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void st_cluster_f32(unsigned local_addr, unsigned rank, float v) {
+    unsigned remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("st.shared::cluster.f32 [%0], %1;\n" ::"r"(remote), "f"(v) : "memory");
+}
+
+// Sum over the 32 lanes of NV per-lane values with a halving butterfly (fixed order).
+// On return lane l holds the total of value index l (NV == 32) or l >> 1 (NV == 16) in v[0].
+template <int NV>
+__device__ __forceinline__ void butterfly_reduce(float (&v)[NV], int lane) {
+#pragma unroll
+    for (int o = 16, cnt = NV; cnt > 1; o >>= 1, cnt >>= 1) {
+        const bool up = (lane & o) != 0;
+#pragma unroll
+        for (int j = 0; j < cnt / 2; ++j) {
+            float send = up ? v[j] : v[j + cnt / 2];
+            float keep = up ? v[j + cnt / 2] : v[j];
+            v[j] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+        }
+    }
+    if (NV == 16) v[0] += __shfl_xor_sync(0xffffffffu, v[0], 1);
+}
+
+// d = a * b + c on two packed floats (one instruction slot on sm_100)
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+    float2 d;
+    asm("{\n.reg .b64 ra, rb, rc, rd;\n"
+        "mov.b64 ra, {%2, %3};\nmov.b64 rb, {%4, %5};\nmov.b64 rc, {%6, %7};\n"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n"
+        "mov.b64 {%0, %1}, rd;\n}\n"
+        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+    return d;
+}
+
+// A float delivered to a peer CTA's shared memory; the peer's mbarrier counts the 4 bytes.
+__device__ __forceinline__ void st_async_cluster_f32(unsigned local_addr, unsigned local_bar, unsigned rank, float v) {
+    unsigned raddr, rbar;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(raddr) : "r"(local_addr), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(rbar) : "r"(local_bar), "r"(rank));
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];\n"
+                 ::"r"(raddr), "r"(__float_as_uint(v)), "r"(rbar) : "memory");
+}
+
+template <int RP, int WC, bool PENDING>
+__global__ void __launch_bounds__(FU_THREADS, 1)
+k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmM, FusedArgs a) {
+    using Ge = FusedGeom<WC>;
+    constexpr int BW = Ge::BW, NH = Ge::NH, CPL = Ge::CPL, NCG = Ge::NCG, NST = Ge::NST, TPN = Ge::TPN;
+    constexpr int NV = FU_RG * RP;         // per-lane partial sums of one warp task
+    constexpr int PR = FU_R * RP;          // entries of one block of P
+    constexpr int RP2 = RP / 2;
+    constexpr unsigned STAGE_BYTES = Ge::STAGE_FLOATS * 4;
+
+    extern __shared__ __align__(16) float smem_raw[];
+    float* smem = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
     cg::cluster_group cluster = cg::this_cluster();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int CS = a.CS, N = a.N, n = a.n, m = a.m, Wc = a.Wc;
-    const int q = (int)(blockIdx.x % CS);
+    const int CS = a.CS, N = a.N, n = a.n, m = a.m;
+    const int q = (int)(blockIdx.x % CS);              // rank in the cluster = column slice
     const int cid = (int)(blockIdx.x / CS);
     const int c = cid / a.KC, slot = cid % a.KC;
-    const int Wt = Wc + 4;
-    const int nch = (Wc + FU_CH - 1) / FU_CH;
-    const int colbase = q * Wc;                       // first global column of this CTA
-    const int colend = min(n, colbase + Wc);          // one past its last valid column
+    const int colbase = q * WC;
+    const int colend = min(n, colbase + WC);
+    const int ncols = max(0, colend - colbase);
 
     // ---- shared memory carve-up ----
-    float* tile = smem;                                       // [N][16][Wt]
-    float* stg = tile + (size_t)N * FU_R * Wt;                // stages
-    constexpr int STG_G = 0, STG_M = FU_R * FU_CHP, STG_Q = 2 * FU_R * FU_CHP, STG_P = STG_Q + FU_CH * RP;
-    constexpr int STG_SZ = STG_P + FU_R * RP;
-    float* Qs = stg + FU_STAGES * STG_SZ;                     // [nch*64][RP], zero beyond the slice
-    float* red = Qs + (size_t)nch * FU_CH * RP;               // [8][16][RP]
-    float* Ppart = red + 8 * FU_R * RP;                       // [2][16][RP]
-    float* Praw = Ppart + 2 * FU_R * RP;                      // [16][RP]
-    float* Pb = Praw + FU_R * RP;                             // [16][RP]
-    float* Tp = Pb + FU_R * RP;                               // [RP][RP]
+    float* ring = smem;                                        // [NST][2][8][BW]   (128-byte aligned)
+    float* tile = ring + (size_t)NST * Ge::STAGE_FLOATS;       // [2][N][8][WC]
+    float* PpartW = tile + (size_t)2 * N * FU_R * WC;          // [2][2][NH*NCG][32]
+    float* Precv = PpartW + 2 * 2 * NH * NCG * 32;             // [2][FU_MAXCS][PR]
+    float* Pb = Precv + 2 * FU_MAXCS * PR;                     // [2][PR]   P' rows
+    float* Pp = Pb + 2 * PR;                                   // [2][PR]   P~_{t-1} rows
+    float* Cm = Pp + 2 * PR;                                   // [RP][RP]
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(Cm + RP * RP);
+    const unsigned bar_full = smem_u32(bars), bar_empty = smem_u32(bars + NST), bar_recv = smem_u32(bars + 2 * NST);
 
-    const float* Gc = a.G + (size_t)c * N * m * n;
     float* Mc = a.Mbuf + (size_t)c * N * m * n;
     const float* Qc = a.Qpad + (size_t)c * n * RP;
     const float* Ppc = PENDING ? a.Ppad + (size_t)c * m * RP : nullptr;
     const float* Qsc = PENDING ? a.Qsub + (size_t)c * (a.qsub_node_stride ? N : 1) * n * RP : nullptr;
 
-    // resident slice of Q_{t-1} and the preconditioner
-    for (int e = tid; e < nch * FU_CH * RP / 4; e += FU_THREADS) {
-        int col = (e * 4) / RP;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (col < Wc && colbase + col < colend) v = *reinterpret_cast<const float4*>(Qc + (size_t)(colbase + col) * RP + (e * 4) % RP);
-        *reinterpret_cast<float4*>(Qs + e * 4) = v;
-    }
-    const bool precond = a.Tprev != nullptr;
-    for (int e = tid; e < RP * RP; e += FU_THREADS) Tp[e] = precond ? a.Tprev[(size_t)c * RP * RP + e] : 0.f;
-
-    // number of row blocks this cluster owns: slot, slot+KC, ...
+    // row blocks this cluster owns: slot, slot + KC, ...
     const int nb = (a.nblk > slot) ? (a.nblk - slot + a.KC - 1) / a.KC : 0;
-    const int per_block = nch * N;
-    const int T = nb * per_block;
+    const int nstb = NH * N;               // stages per block: column half outer, node inner
+    const int T = nb * nstb;
 
-    auto issue = [&](int s) {   // cp.async loads of stage s (all threads take part)
-        int bl = s / per_block, rem = s % per_block;
-        int j = rem / N, i = rem % N;
-        int row0 = (slot + bl * a.KC) * FU_R;
-        float* sb = stg + (s % FU_STAGES) * STG_SZ;
-        int cbase = colbase + j * FU_CH;
-        if (tid < 256) {
-            int rr = tid >> 4, c4 = (tid & 15) * 4;
-            int ok = (row0 + rr < m && cbase + c4 < colend) ? 16 : 0;
-            size_t off = ok ? ((size_t)i * m + row0 + rr) * n + cbase + c4 : 0;
-            cp_async16(sb + STG_G + rr * FU_CHP + c4, Gc + off, ok);
+    // ---- one-time set-up ----
+    if (tid == 0) {
+        for (int s = 0; s < NST; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, FU_THREADS / 32);
+        }
+        mbar_init(bar_recv, 1);
+        mbar_init(bar_recv + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (PENDING)
+        for (int e = tid; e < RP * RP; e += FU_THREADS) Cm[e] = a.Cmat[(size_t)c * RP * RP + e];
+    cluster.sync();   // every CTA's barriers exist before a peer sends to them
+    bool dead = false;
+
+    // projection phase: warp -> (column group, row group) of a stage, lane -> CPL adjacent columns
+    const int cgp = warp % NCG, rgl = warp / NCG;
+    const int acol = cgp * 32 * CPL + lane * CPL;      // column within the stage
+    // back-projection phase: thread -> (node, 4 + 4 columns)
+    const int bi = tid / TPN, tc = tid % TPN;
+    const bool btask = bi < N;
+    const int bc0 = 4 * tc, bc1 = WC / 2 + 4 * tc;
+    const bool bok0 = btask && bc0 < ncols, bok1 = btask && bc1 < ncols;
+    float2 wacc[8][RP2];                   // W for 8 columns, pairs over k
+    constexpr int QSN = PENDING ? 4 : 1;
+    float2 qs[QSN][RP];                    // Qsub for column pairs (2j, 2j+1), per k
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+#pragma unroll
+        for (int k = 0; k < RP2; ++k) wacc[j][k] = make_float2(0.f, 0.f);
+    if (PENDING) {
+        float t8[8][RP];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int col = (j < 4 ? bc0 : bc1) + (j & 3);
+#pragma unroll
+            for (int k4 = 0; k4 < RP / 4; ++k4) {
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (btask && col < ncols)
+                    v = __ldg(reinterpret_cast<const float4*>(Qsc + (size_t)bi * a.qsub_node_stride + (size_t)(colbase + col) * RP + 4 * k4));
+                t8[j][4 * k4 + 0] = v.x; t8[j][4 * k4 + 1] = v.y; t8[j][4 * k4 + 2] = v.z; t8[j][4 * k4 + 3] = v.w;
+            }
+        }
+#pragma unroll
+        for (int j2 = 0; j2 < QSN; ++j2)
+#pragma unroll
+            for (int k = 0; k < RP; ++k) qs[j2][k] = make_float2(t8[(2 * j2) % 8][k], t8[(2 * j2 + 1) % 8][k]);
+    }
+
+    // ---- producer role (taken in turn by the warps): two TMA tiles per stage ----
+    // state of the next stage to issue, advanced by every thread in step with the main loop
+    int p_bl = 0, p_h = 0, p_i = 0, p_ss = 0, p_par = 1;   // p_par: parity of the slot's previous release
+    auto issue_next = [&]() {      // called by one whole warp; the slot must have been released
+        if (lane == 0) {
+            const int row = (slot + p_bl * a.KC) * FU_R;
+            const unsigned bar = bar_full + 8 * p_ss;
+            const unsigned dst = smem_u32(ring + (size_t)p_ss * Ge::STAGE_FLOATS);
+            mbar_expect_tx(bar, STAGE_BYTES);
+            tma_load_3d(dst, &tmG, colbase + p_h * BW, row, c * N + p_i, bar);
+            tma_load_3d(dst + STAGE_BYTES / 2, &tmM, colbase + p_h * BW, row, c * N + p_i, bar);
+        }
+        __syncwarp();
+    };
+    auto advance_next = [&]() {
+        if (++p_i == N) { p_i = 0; if (++p_h == NH) { p_h = 0; ++p_bl; } }
+        if (++p_ss == NST) { p_ss = 0; p_par ^= 1; }
+    };
+    for (int s = 0; s < NST - 1; ++s) {
+        if (s < T && warp == 0) issue_next();
+        advance_next();
+    }
+
+    // P' of one finished block: node mean of the received partial sums, small-space correction.
+    // Every thread waits for the cluster's partial sums itself (bounded), so no barrier follows the wait.
+    auto finish_block = [&](int bl) {
+        const int pb = bl & 1;
+        const int prow0 = (slot + bl * a.KC) * FU_R;
+        mbar_wait(bar_recv + 8 * pb, (unsigned)((bl >> 1) & 1), a.flags, dead);
+        if (tid < PR) {
+            const int rr = tid / RP, k = tid % RP;
+            float sum = 0.f;
+            for (int qq = 0; qq < CS; ++qq) sum += Precv[(pb * FU_MAXCS + qq) * PR + tid];
+            float v = sum / (float)N;
             if (PENDING) {
-                // chunk of the factor that the pending residual subtracts: [64 cols][RP]
-                for (int e = tid; e < FU_CH * RP / 4; e += 256) {
-                    int col = (e * 4) / RP;
-                    int okq = (cbase + col < colend) ? 16 : 0;
-                    size_t offq = okq ? (size_t)i * a.qsub_node_stride + (size_t)(cbase + col) * RP + (e * 4) % RP : 0;
-                    cp_async16(sb + STG_Q + e * 4, Qsc + offq, okq);
+                const float* pp = Pp + pb * PR + rr * RP;
+#pragma unroll
+                for (int j = 0; j < RP; ++j) v = fmaf(-pp[j], Cm[j * RP + k], v);
+            }
+            if (prow0 + rr >= m) v = 0.f;
+            Pb[pb * PR + tid] = v;
+            if (q == 0 && prow0 + rr < m) a.Pout[((size_t)c * m + prow0 + rr) * RP + k] = v;
+        }
+        __syncthreads();
+    };
+    double gacc = 0.0;   // rank 0, threads 64 .. 64 + r*r: one entry of P'^T P'
+    auto gram_block = [&](int bl) {
+        const int pb = bl & 1;
+        const int t2 = tid - 64;
+        if (q == 0 && t2 >= 0 && t2 < a.r * a.r) {
+            const int ga = t2 / a.r, gb = t2 % a.r;
+#pragma unroll
+            for (int rr = 0; rr < FU_R; ++rr)
+                gacc = fma((double)Pb[pb * PR + rr * RP + ga], (double)Pb[pb * PR + rr * RP + gb], gacc);
+        }
+    };
+    // back-projection of row rr of block bl: Delta = S - P~_{t-1} Qsub^T, W += Delta^T P', store Delta
+    auto back_row = [&](int bl, int rr) {
+        if (!btask) return;
+        const int pb = bl & 1;
+        const int prow = (slot + bl * a.KC) * FU_R + rr;
+        const float* tp = tile + (((size_t)pb * N + bi) * FU_R + rr) * WC;
+        const float4 v0 = *reinterpret_cast<const float4*>(tp + bc0);
+        const float4 v1 = *reinterpret_cast<const float4*>(tp + bc1);
+        float2 mv[4] = {make_float2(v0.x, v0.y), make_float2(v0.z, v0.w), make_float2(v1.x, v1.y), make_float2(v1.z, v1.w)};
+        if (PENDING) {
+            const float* pp = Pp + pb * PR + rr * RP;
+#pragma unroll
+            for (int k4 = 0; k4 < RP / 4; ++k4) {
+                const float4 p4 = *reinterpret_cast<const float4*>(pp + 4 * k4);
+                const float pk[4] = {-p4.x, -p4.y, -p4.z, -p4.w};
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const float2 pd = make_float2(pk[kk], pk[kk]);
+#pragma unroll
+                    for (int j2 = 0; j2 < 4; ++j2) mv[j2] = ffma2(pd, qs[j2 % QSN][4 * k4 + kk], mv[j2]);
                 }
             }
-        } else {
-            int t2 = tid - 256;
-            int rr = t2 >> 4, c4 = (t2 & 15) * 4;
-            int ok = (row0 + rr < m && cbase + c4 < colend) ? 16 : 0;
-            size_t off = ok ? ((size_t)i * m + row0 + rr) * n + cbase + c4 : 0;
-            cp_async16(sb + STG_M + rr * FU_CHP + c4, Mc + off, ok);
-            if (PENDING && rem == 0) {
-                // rows of P~_{t-1} for this block, once per block
-                for (int e = t2; e < FU_R * RP / 4; e += 256) {
-                    int rr2 = (e * 4) / RP;
-                    int okp = (row0 + rr2 < m) ? 16 : 0;
-                    size_t offp = okp ? (size_t)(row0 + rr2) * RP + (e * 4) % RP : 0;
-                    cp_async16(sb + STG_P + e * 4, Ppc + offp, okp);
-                }
+        }
+        const float* pr = Pb + pb * PR + rr * RP;
+        float2 pk2[RP2];
+#pragma unroll
+        for (int k4 = 0; k4 < RP / 4; ++k4) {
+            const float4 p4 = *reinterpret_cast<const float4*>(pr + 4 * k4);
+            pk2[2 * k4] = make_float2(p4.x, p4.y);
+            pk2[2 * k4 + 1] = make_float2(p4.z, p4.w);
+        }
+#pragma unroll
+        for (int j2 = 0; j2 < 4; ++j2) {
+            const float2 mx = make_float2(mv[j2].x, mv[j2].x), my = make_float2(mv[j2].y, mv[j2].y);
+#pragma unroll
+            for (int k2 = 0; k2 < RP2; ++k2) {
+                wacc[2 * j2][k2] = ffma2(mx, pk2[k2], wacc[2 * j2][k2]);
+                wacc[2 * j2 + 1][k2] = ffma2(my, pk2[k2], wacc[2 * j2 + 1][k2]);
             }
+        }
+        if (prow < m) {
+            float* go = Mc + ((size_t)bi * m + prow) * n + colbase;
+            if (bok0) *reinterpret_cast<float4*>(go + bc0) = make_float4(mv[0].x, mv[0].y, mv[1].x, mv[1].y);
+            if (bok1) *reinterpret_cast<float4*>(go + bc1) = make_float4(mv[2].x, mv[2].y, mv[3].x, mv[3].y);
         }
     };
 
-    // phase-A mapping: lane -> (row, half); warp -> 4 columns of the chunk; thread -> 2 columns
-    const int arow = lane & 15, ahalf = lane >> 4;
-    const int acol = warp * 4 + ahalf * 2;  // column within the chunk
-    // phase-B mapping: thread -> (node, 4 columns)
-    const int Wc4 = Wc / 4;
-    const bool btask = tid < N * Wc4;
-    const int bnode = btask ? tid / Wc4 : 0;
-    const int bcol = btask ? (tid % Wc4) * 4 : 0;   // column within the slice
-    const bool bcol_ok = btask && (colbase + bcol < colend);
-
-    float pacc[RP], pprev[RP];
-    float wacc[4][RP];
+    float2 sacc[FU_RG][RP2];
 #pragma unroll
-    for (int k = 0; k < RP; ++k) { pacc[k] = 0.f; pprev[k] = 0.f; }
+    for (int rr = 0; rr < FU_RG; ++rr)
 #pragma unroll
-    for (int jj = 0; jj < 4; ++jj)
-#pragma unroll
-        for (int k = 0; k < RP; ++k) wacc[jj][k] = 0.f;
-    double gacc = 0.0;  // rank 0 only: one entry of P'^T P' per thread
+        for (int k = 0; k < RP2; ++k) sacc[rr][k] = make_float2(0.f, 0.f);
+    float2 Qr[CPL][RP2];     // rows of Q' for this lane's columns of the current column half, pairs over k
+    float pprev_reg = 0.f;   // thread < PR: its entry of P~_{t-1} for the block being projected
 
-    for (int s = 0; s < FU_STAGES - 1; ++s) {
-        if (s < T) issue(s);
-        cp_async_commit();
-    }
-    __syncthreads();   // Qs, Tp visible
-
-    for (int s = 0; s < T; ++s) {
-        cp_async_wait<FU_STAGES - 2>();
-        __syncthreads();
-        if (s + FU_STAGES - 1 < T) issue(s + FU_STAGES - 1);
-        cp_async_commit();
-
-        const int bl = s / per_block, rem = s % per_block;
-        const int j = rem / N, i = rem % N;
+    const int k0 = nstb >= 3 ? 1 : 0;   // stage of a block at which the previous block's P' is finished
+    const int span = nstb - k0;         // stages over which the previous block's 8 rows are back-projected
+    int ss = 0, par = 0;                // ring slot and parity of the stage being consumed
+    int sg = 0;
+    for (int bl = 0; bl < nb; ++bl) {
         const int row0 = (slot + bl * a.KC) * FU_R;
-        float* sb = stg + (s % FU_STAGES) * STG_SZ;
-        if (PENDING && rem == 0) {
-#pragma unroll
-            for (int k4 = 0; k4 < RP / 4; ++k4) {
-                float4 v = *reinterpret_cast<const float4*>(sb + STG_P + arow * RP + 4 * k4);
-                pprev[4 * k4 + 0] = v.x; pprev[4 * k4 + 1] = v.y; pprev[4 * k4 + 2] = v.z; pprev[4 * k4 + 3] = v.w;
-            }
+        const int pbuf = bl & 1;
+        int brow = 0, bacc = 0;         // rows of the previous block done so far; Bresenham accumulator
+        if (tid == 0) mbar_expect_tx(bar_recv + 8 * pbuf, (unsigned)(CS * PR * 4));
+        if (PENDING && tid < PR) {
+            const int rr = tid / RP;
+            pprev_reg = (row0 + rr < m) ? __ldg(Ppc + (size_t)(row0 + rr) * RP + tid % RP) : 0.f;
         }
-        // ---- phase A: M = G + (Mprev - P~prev Qsub^T);  pacc += M Q ----
-        {
-            float2 g2 = *reinterpret_cast<const float2*>(sb + STG_G + arow * FU_CHP + acol);
-            float2 m2 = *reinterpret_cast<const float2*>(sb + STG_M + arow * FU_CHP + acol);
-            float mv[2] = {m2.x, m2.y};
-            const float gv[2] = {g2.x, g2.y};
+        int sl = 0;
+        for (int h = 0; h < NH; ++h) {
+            if (NH > 1 || bl == 0) {   // (re)load this lane's rows of Q' for the column half
 #pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
-                if (PENDING) {
-                    const float* qp = sb + STG_Q + (acol + cc) * RP;
-                    float r0 = 0.f, r1 = 0.f, r2 = 0.f, r3 = 0.f;
+                for (int j = 0; j < CPL; ++j)
 #pragma unroll
                     for (int k4 = 0; k4 < RP / 4; ++k4) {
-                        float4 qv = *reinterpret_cast<const float4*>(qp + 4 * k4);
-                        r0 = fmaf(pprev[4 * k4 + 0], qv.x, r0);
-                        r1 = fmaf(pprev[4 * k4 + 1], qv.y, r1);
-                        r2 = fmaf(pprev[4 * k4 + 2], qv.z, r2);
-                        r3 = fmaf(pprev[4 * k4 + 3], qv.w, r3);
+                        const int col = h * BW + acol + j;
+                        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (col < ncols) v = __ldg(reinterpret_cast<const float4*>(Qc + (size_t)(colbase + col) * RP + 4 * k4));
+                        Qr[j][2 * k4] = make_float2(v.x, v.y);
+                        Qr[j][2 * k4 + 1] = make_float2(v.z, v.w);
                     }
-                    mv[cc] = mv[cc] - ((r0 + r1) + (r2 + r3));
-                }
-                mv[cc] += gv[cc];
-                const float* qq = Qs + (size_t)(j * FU_CH + acol + cc) * RP;
-#pragma unroll
-                for (int k4 = 0; k4 < RP / 4; ++k4) {
-                    float4 qv = *reinterpret_cast<const float4*>(qq + 4 * k4);
-                    pacc[4 * k4 + 0] = fmaf(mv[cc], qv.x, pacc[4 * k4 + 0]);
-                    pacc[4 * k4 + 1] = fmaf(mv[cc], qv.y, pacc[4 * k4 + 1]);
-                    pacc[4 * k4 + 2] = fmaf(mv[cc], qv.z, pacc[4 * k4 + 2]);
-                    pacc[4 * k4 + 3] = fmaf(mv[cc], qv.w, pacc[4 * k4 + 3]);
-                }
             }
-            if (j * FU_CH + acol < Wc)
-                *reinterpret_cast<float2*>(tile + ((size_t)i * FU_R + arow) * Wt + j * FU_CH + acol) = make_float2(mv[0], mv[1]);
-        }
-        if (rem != per_block - 1) continue;
+            for (int i = 0; i < N; ++i, ++sl, ++sg) {
+                if (warp == (sg & 7)) {           // this warp's turn to refill the ring
+                    if (sg + NST - 1 < T) {
+                        if (sg > 0) mbar_wait(bar_empty + 8 * p_ss, (unsigned)p_par, a.flags, dead);
+                        issue_next();
+                    }
+                }
+                advance_next();
+                if (bl > 0 && sl == k0) {
+                    finish_block(bl - 1);
+                    gram_block(bl - 1);
+                }
 
-        // ---- end of a row block: reduce P over the CTA, the cluster, then phase B ----
-        const int par = bl & 1;
+                // ---- projection: S = g + stored Delta -> tile; sacc += S Q' ----
+                mbar_wait(bar_full + 8 * ss, (unsigned)par, a.flags, dead);
+                {
+                    const float* sgp = ring + (size_t)ss * Ge::STAGE_FLOATS + (size_t)(rgl * FU_RG) * BW + acol;
+                    const float* smp = sgp + FU_R * BW;
+                    float* tp = tile + (((size_t)pbuf * N + i) * FU_R + rgl * FU_RG) * WC + h * BW + acol;
+                    float sv[FU_RG][CPL];
 #pragma unroll
-        for (int k = 0; k < RP; ++k) pacc[k] += __shfl_xor_sync(0xffffffffu, pacc[k], 16);
-        if (warp >= 8 && lane < 16) {
-#pragma unroll
-            for (int k = 0; k < RP; ++k) red[((warp - 8) * FU_R + arow) * RP + k] = pacc[k];
-        }
-        __syncthreads();
-        if (warp < 8 && lane < 16) {
-#pragma unroll
-            for (int k = 0; k < RP; ++k) pacc[k] += red[(warp * FU_R + arow) * RP + k];
-        }
-        __syncthreads();
-        if (warp < 8 && lane < 16) {
-#pragma unroll
-            for (int k = 0; k < RP; ++k) red[(warp * FU_R + arow) * RP + k] = pacc[k];
-        }
-        __syncthreads();
-        if (tid < FU_R * RP) {
-            float sum = 0.f;
-#pragma unroll
-            for (int w = 0; w < 8; ++w) sum += red[w * FU_R * RP + tid];
-            Ppart[par * FU_R * RP + tid] = sum;
-        }
-        cluster.sync();
-        if (tid < FU_R * RP) {
-            float sum = 0.f;
-            for (int qq = 0; qq < CS; ++qq) {
-                const float* rp = cluster.map_shared_rank(Ppart, qq);
-                sum += rp[par * FU_R * RP + tid];
-            }
-            Praw[tid] = sum / (float)N;
-        }
-        __syncthreads();
-        if (tid < FU_R * RP) {
-            int rr = tid / RP, k = tid % RP;
-            float v;
-            if (precond) {
-                v = 0.f;
-                for (int jj = 0; jj <= k; ++jj) v = fmaf(Praw[rr * RP + jj], Tp[jj * RP + k], v);
-            } else {
-                v = Praw[tid];
-            }
-            Pb[tid] = v;
-            if (q == 0 && row0 + rr < m) a.Pout[((size_t)c * m + row0 + rr) * RP + k] = v;
-        }
-        __syncthreads();
-        if (q == 0 && tid < a.r * a.r) {
-            int ga = tid / a.r, gb = tid % a.r;
-#pragma unroll
-            for (int rr = 0; rr < FU_R; ++rr) gacc = fma((double)Pb[rr * RP + ga], (double)Pb[rr * RP + gb], gacc);
-        }
-        // ---- phase B: W_i += M_i[b,:]^T P'[b];  store M ----
-        if (btask) {
-            const float* tp = tile + (size_t)bnode * FU_R * Wt + bcol;
-            float* gout = Mc + ((size_t)bnode * m + row0) * n + colbase + bcol;
-#pragma unroll 4
-            for (int rr = 0; rr < FU_R; ++rr) {
-                float4 v = *reinterpret_cast<const float4*>(tp + rr * Wt);
-                if (bcol_ok && row0 + rr < m) *reinterpret_cast<float4*>(gout + (size_t)rr * n) = v;
-                const float* pr = Pb + rr * RP;
-#pragma unroll
-                for (int k4 = 0; k4 < RP / 4; ++k4) {
-                    float4 p4 = *reinterpret_cast<const float4*>(pr + 4 * k4);
-                    const float pk[4] = {p4.x, p4.y, p4.z, p4.w};
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        wacc[0][4 * k4 + kk] = fmaf(v.x, pk[kk], wacc[0][4 * k4 + kk]);
-                        wacc[1][4 * k4 + kk] = fmaf(v.y, pk[kk], wacc[1][4 * k4 + kk]);
-                        wacc[2][4 * k4 + kk] = fmaf(v.z, pk[kk], wacc[2][4 * k4 + kk]);
-                        wacc[3][4 * k4 + kk] = fmaf(v.w, pk[kk], wacc[3][4 * k4 + kk]);
+                    for (int rr = 0; rr < FU_RG; ++rr) {
+                        if (CPL == 2) {
+                            const float2 g2 = *reinterpret_cast<const float2*>(sgp + rr * BW);
+                            const float2 m2 = *reinterpret_cast<const float2*>(smp + rr * BW);
+                            sv[rr][0] = g2.x + m2.x; sv[rr][CPL - 1] = g2.y + m2.y;
+                        } else {
+                            sv[rr][0] = sgp[rr * BW] + smp[rr * BW];
+                        }
                     }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_empty + 8 * ss);   // the stage is in registers: release the slot
+#pragma unroll
+                    for (int rr = 0; rr < FU_RG; ++rr) {
+                        if (CPL == 2) *reinterpret_cast<float2*>(tp + rr * WC) = make_float2(sv[rr][0], sv[rr][CPL - 1]);
+                        else tp[rr * WC] = sv[rr][0];
+#pragma unroll
+                        for (int j = 0; j < CPL; ++j) {
+                            const float2 sd = make_float2(sv[rr][j], sv[rr][j]);
+#pragma unroll
+                            for (int k2 = 0; k2 < RP2; ++k2) sacc[rr][k2] = ffma2(sd, Qr[j][k2], sacc[rr][k2]);
+                        }
+                    }
+                }
+                if (++ss == NST) { ss = 0; par ^= 1; }
+
+                if (i == N - 1) {   // the column half is complete for every node: reduce over the warp's columns
+                    float v[NV];
+#pragma unroll
+                    for (int rr = 0; rr < FU_RG; ++rr)
+#pragma unroll
+                        for (int k2 = 0; k2 < RP2; ++k2) {
+                            v[rr * RP + 2 * k2] = sacc[rr][k2].x;
+                            v[rr * RP + 2 * k2 + 1] = sacc[rr][k2].y;
+                            sacc[rr][k2] = make_float2(0.f, 0.f);
+                        }
+                    butterfly_reduce<NV>(v, lane);
+                    if (NV == 32 || (lane & 1) == 0)
+                        PpartW[((pbuf * 2 + rgl) * (NH * NCG) + h * NCG + cgp) * 32 + (NV == 32 ? lane : lane >> 1)] = v[0];
+                }
+
+                // ---- back-projection of the previous block, spread over this block's stages ----
+                if (bl > 0 && sl >= k0) {
+                    bacc += FU_R;
+                    while (bacc >= span && brow < FU_R) { back_row(bl - 1, brow); ++brow; bacc -= span; }
                 }
             }
         }
+        // block projected: CTA sum of the partial P, sent to every CTA of the cluster
+        if (PENDING && tid < PR) Pp[pbuf * PR + tid] = pprev_reg;
+        __syncthreads();
+        if (tid < PR) {
+            const int rr = tid / RP, k = tid % RP;
+            const int rgi = rr / FU_RG, j = (rr % FU_RG) * RP + k;
+            float sum = 0.f;
 #pragma unroll
-        for (int k = 0; k < RP; ++k) pacc[k] = 0.f;
+            for (int g = 0; g < NH * NCG; ++g) sum += PpartW[((pbuf * 2 + rgi) * (NH * NCG) + g) * 32 + j];
+            const unsigned dst = smem_u32(Precv + (pbuf * FU_MAXCS + q) * PR + tid);
+            for (int qq = 0; qq < CS; ++qq) st_async_cluster_f32(dst, bar_recv + 8 * pbuf, (unsigned)qq, sum);
+        }
     }
-    cp_async_wait<0>();
+    if (nb > 0) {
+        finish_block(nb - 1);
+        gram_block(nb - 1);
+#pragma unroll 1
+        for (int rr = 0; rr < FU_R; ++rr) back_row(nb - 1, rr);
+    }
 
     // ---- flush this cluster's partial W and Gram ----
-    if (bcol_ok) {
-        float* wp = a.Wpart + ((((size_t)c * a.KC + slot) * N + bnode) * n + colbase + bcol) * RP;
+    if (btask) {
 #pragma unroll
-        for (int jj = 0; jj < 4; ++jj)
+        for (int j = 0; j < 8; ++j) {
+            const int col = (j < 4 ? bc0 : bc1) + (j & 3);
+            if (col < ncols) {
+                float* wp = a.Wpart + ((((size_t)c * a.KC + slot) * N + bi) * n + colbase + col) * RP;
 #pragma unroll
-            for (int k4 = 0; k4 < RP / 4; ++k4)
-                *reinterpret_cast<float4*>(wp + (size_t)jj * RP + 4 * k4) =
-                    make_float4(wacc[jj][4 * k4 + 0], wacc[jj][4 * k4 + 1], wacc[jj][4 * k4 + 2], wacc[jj][4 * k4 + 3]);
+                for (int k4 = 0; k4 < RP / 4; ++k4)
+                    *reinterpret_cast<float4*>(wp + 4 * k4) =
+                        make_float4(wacc[j][2 * k4].x, wacc[j][2 * k4].y, wacc[j][2 * k4 + 1].x, wacc[j][2 * k4 + 1].y);
+            }
+        }
     }
-    if (q == 0 && tid < a.r * a.r) a.gram[((size_t)c * a.KC + slot) * a.r * a.r + tid] = gacc;
-    cluster.sync();   // nobody leaves while a peer may still read its shared memory
+    {
+        const int t2 = tid - 64;
+        if (q == 0 && t2 >= 0 && t2 < a.r * a.r) a.gram[((size_t)c * a.KC + slot) * a.r * a.r + t2] = gacc;
+    }
+    cluster.sync();   // nobody leaves while a peer may still address its shared memory
 }
 
 // P~ = P' T' (double accumulate).  Writes the user layout [m][r] and the padded copy [m][RP];
-// block 0 of each matrix also advances the preconditioner Tacc <- Tprev * T'.
+// block 0 of each matrix also advances the accumulated transform Tacc <- Tacc * T'.
 // grid: (ceil(m/64), count), 256 threads.
 struct FinishPArgs {
     const float* Pout;   // [count][m][RP]
     const double* T;     // [count][r][r]
     float* Phat;         // [count][m][r]
     float* Ppad;         // [count][m][RP]
-    float* Tacc;         // [count][RP][RP]
+    const float* Tacc_in;   // [count][RP][RP]  (ignored when tprev_identity)
+    float* Tacc_out;        // [count][RP][RP]
     int m, r, RP, tprev_identity;
 };
 __global__ void __launch_bounds__(256) k_finish_p(FinishPArgs a) {
@@ -347,45 +538,54 @@ __global__ void __launch_bounds__(256) k_finish_p(FinishPArgs a) {
         a.Ppad[((size_t)c * a.m + row) * RP + k] = (float)s;
     }
     if (blockIdx.x == 0) {
-        float* Ta = a.Tacc + (size_t)c * RP * RP;
+        const float* Ti = a.Tacc_in + (size_t)c * RP * RP;
+        float* To = a.Tacc_out + (size_t)c * RP * RP;
         for (int e = threadIdx.x; e < r * r; e += 256) {
             int j = e / r, k = e % r;
             double s = 0.0;
             if (a.tprev_identity) s = Ts[e];
-            else for (int l = j; l <= k; ++l) s = fma((double)Ta[j * RP + l], Ts[l * r + k], s);
+            else for (int l = j; l <= k; ++l) s = fma((double)Ti[j * RP + l], Ts[l * r + k], s);
             Tn[e] = s;
         }
         __syncthreads();
         for (int e = threadIdx.x; e < RP * RP; e += 256) {
             int j = e / RP, k = e % RP;
-            Ta[e] = (j < r && k < r) ? (float)Tn[j * r + k] : 0.f;
+            To[e] = (j < r && k < r) ? (float)Tn[j * r + k] : 0.f;
         }
     }
 }
 
 // Q_i = (sum over clusters of W_i) T'   (or, when *gate != 0, the sum of the precise
-// back-projection partials), Q = (1/N) sum_i Q_i.  Writes the user layouts and the padded
-// copies the next fused step reads.  grid: (ceil(n/16), count), 16*RP threads.
+// back-projection partials), Q = (1/N) sum_i Q_i.  Writes the user layouts, the factor the
+// pending residual subtracts (Qsub), the preconditioned basis Q' = Q Tacc the next fused step
+// projects with, and this block's share of C' = mean_i Qsub_i^T Q'.
+// grid: (ceil(n/16), count), 16*RP threads.
 struct FinishQArgs {
     const float* Wpart;  // [count][KC][N][n][RP]
     const float* part;   // [count][N][S][n][r]   precise partials (gate != 0)
     const double* T;     // [count][r][r]
+    const float* Tacc;   // [count][RP][RP]  accumulated transform (already advanced by k_finish_p)
     const int* gate;
     float* Qnode;        // [count][N][n][r]
     float* Qmean;        // [count][n][r]
-    float* Qpad;         // [count][n][RP]
+    float* Qpad;         // [count][n][RP]   Q'
     float* Qsub;         // [count][N or 1][n][RP]
+    double* Cpart;       // [count][nblocks][RP][RP]
     int n, r, RP, N, KC, S, sub_is_mean;
 };
 __global__ void k_finish_q(FinishQArgs a) {
     __shared__ double Ts[16 * 16];
+    __shared__ float Ta[16 * 16];
     __shared__ float Ws[16][17];
+    __shared__ float Qs_[16][17];     // Q' of this block's columns
+    __shared__ float Qi_[16][16][17]; // [node chunk of 16][column][k]  Qsub values
     const int c = blockIdx.y, r = a.r, RP = a.RP, n = a.n, N = a.N;
     const int cl = threadIdx.x / RP, k = threadIdx.x % RP;
     const int col = blockIdx.x * 16 + cl;
     const bool precise = a.gate && *a.gate != 0;
     const double* Tb = a.T + (size_t)c * r * r;
     for (int e = threadIdx.x; e < r * r; e += blockDim.x) Ts[e] = Tb[e];
+    for (int e = threadIdx.x; e < RP * RP; e += blockDim.x) Ta[e] = a.Tacc[(size_t)c * RP * RP + e];
     __syncthreads();
     double mean = 0.0;
     for (int i = 0; i < N; ++i) {
@@ -413,14 +613,47 @@ __global__ void k_finish_q(FinishQArgs a) {
             if (k < r) a.Qnode[(((size_t)c * N + i) * n + col) * r + k] = qv;
             if (!a.sub_is_mean) a.Qsub[(((size_t)c * N + i) * n + col) * RP + k] = (k < r) ? qv : 0.f;
         }
+        Qi_[i & 15][cl][k] = (col < n && k < r) ? qv : 0.f;   // kept until Q' is known (N <= 16)
         mean += (double)qv;
     }
+    float qm = (float)(mean / (double)N);
     if (col < n) {
-        float qm = (float)(mean / (double)N);
         if (k < r) a.Qmean[((size_t)c * n + col) * r + k] = qm;
-        a.Qpad[((size_t)c * n + col) * RP + k] = (k < r) ? qm : 0.f;
         if (a.sub_is_mean) a.Qsub[((size_t)c * n + col) * RP + k] = (k < r) ? qm : 0.f;
     }
+    // Q' = Q Tacc (upper triangular): needs the whole row of Q
+    __syncthreads();
+    Ws[cl][k] = (col < n && k < r) ? qm : 0.f;
+    __syncthreads();
+    float qp = 0.f;
+    for (int j = 0; j <= k; ++j) qp = fmaf(Ws[cl][j], Ta[j * RP + k], qp);
+    if (!(col < n && k < r)) qp = 0.f;
+    if (col < n) a.Qpad[((size_t)c * n + col) * RP + k] = qp;
+    Qs_[cl][k] = qp;
+    __syncthreads();
+    // this block's share of C'[j][k] = (1/Nsub) sum_i sum_col Qsub_i[col][j] Q'[col][k]:
+    // thread (cl, k) with cl < RP takes entry (j = cl, k).  Needs N <= 16 (the fused plan guarantees it).
+    if (cl < RP) {
+        const int j = cl;
+        double s = 0.0;
+        if (a.sub_is_mean) {
+            for (int cc = 0; cc < 16; ++cc) s = fma((double)Ws[cc][j], (double)Qs_[cc][k], s);
+        } else {
+            for (int i = 0; i < N; ++i)
+                for (int cc = 0; cc < 16; ++cc) s = fma((double)Qi_[i][cc][j], (double)Qs_[cc][k], s);
+            s /= (double)N;
+        }
+        a.Cpart[(((size_t)c * gridDim.x + blockIdx.x) * RP + j) * RP + k] = s;
+    }
+}
+
+// C' = sum of the per-block shares (fixed order), float32 [count][RP][RP].  grid: count, RP*RP threads.
+__global__ void k_sum_c(const double* Cpart, float* Cmat, int nparts, int RP) {
+    const int c = blockIdx.x, e = threadIdx.x;
+    if (e >= RP * RP) return;
+    double s = 0.0;
+    for (int p = 0; p < nparts; ++p) s += Cpart[((size_t)c * nparts + p) * RP * RP + e];
+    Cmat[(size_t)c * RP * RP + e] = (float)s;
 }
 
 // Padded copies of the state for the fused kernel: Qpad [count][n][RP] from Q [count][n][r].

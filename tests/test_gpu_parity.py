@@ -222,13 +222,17 @@ def test_deferred_config1_tiny_20_steps(torch_cuda):
 
 
 @pytest.mark.parametrize("m,n,r,N,count,workload", [
-    (300, 200, 8, 2, 3, 2),      # one CTA per cluster, ragged rows, batch of 3
-    (96, 96, 1, 5, 1, 2),        # r = 1
+    (300, 200, 8, 2, 3, 2),      # one CTA per cluster, 256-column slice, ragged rows, batch of 3
+    (96, 96, 1, 5, 1, 2),        # r = 1, five nodes, 128-column slice
     (64, 8, 8, 2, 1, 2),         # n == r
-    (513, 260, 16, 1, 1, 5),     # N = 1, r = 16, ragged rows, partial last chunk
-    (768, 768, 8, 8, 2, 2),      # cluster of 4 CTAs (config-2 shape)
-    (4112, 4096, 16, 4, 1, 5),   # cluster of 8 CTAs (config-5 columns), ragged last row block
-    (784, 768, 16, 16, 1, 3),    # 16 nodes, cluster of 8, slice narrower than two chunks
+    (513, 260, 7, 1, 1, 5),      # N = 1 (two stages per block), ragged rows, slice of 4 valid columns in the last CTA
+    (768, 768, 8, 8, 2, 2),      # cluster of 3 CTAs x 256 columns (config-2 shape)
+    (2056, 768, 8, 8, 1, 2),     # config-2 FFN shape, m % 8 == 0 with several row slots
+    (4099, 4096, 8, 4, 1, 5),    # cluster of 8 CTAs x 512 columns (config-5 columns), last block has 3 valid rows
+    (2054, 2048, 4, 8, 1, 4),    # cluster of 8 CTAs x 256 columns (config-4 columns), r = 4
+    (784, 768, 4, 16, 1, 3),     # 16 nodes: cluster of 6 CTAs x 128 columns
+    (1004, 1000, 6, 4, 2, 2),    # n not a multiple of the slice: padded columns, last row chunk empty
+    (513, 260, 16, 1, 1, 5),     # r = 16: outside the single-pass plan, runs the eager kernels
     (130, 66, 5, 2, 2, 2),       # n % 4 != 0: falls back to the eager kernels
 ])
 def test_deferred_step_by_step(torch_cuda, m, n, r, N, count, workload):
@@ -239,7 +243,8 @@ def test_deferred_mean_error_form(torch_cuda):
     run_case(torch_cuda, 192, 128, 4, 3, tau=0, steps=3, workload=2, error_form="mean", Einit=0.01, mode="deferred")
 
 
-@pytest.mark.parametrize("m,n,r,N,workload,tau", [(256, 128, 4, 4, 1, 5), (768, 768, 8, 8, 2, 0), (1040, 1024, 16, 4, 5, 4)])
+@pytest.mark.parametrize("m,n,r,N,workload,tau", [(256, 128, 4, 4, 1, 5), (768, 768, 8, 8, 2, 0), (1040, 1024, 8, 4, 5, 4),
+                                                  (1040, 1024, 16, 4, 5, 4)])
 def test_deferred_free_running(torch_cuda, m, n, r, N, workload, tau):
     """Several steps without resync: pending residuals and the preconditioner are in play."""
     from paper_2509_11254_b200 import PowerSGDPlus
