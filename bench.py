@@ -42,7 +42,7 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=2)
     ap.add_argument("--rank", type=int, default=None)
-    ap.add_argument("--mode", default="eager", choices=["eager", "deferred"])
+    ap.add_argument("--mode", default="deferred", choices=["eager", "deferred"])
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

@@ -276,7 +276,9 @@ k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CU
         if (++p_i == N) { p_i = 0; if (++p_h == NH) { p_h = 0; ++p_bl; } }
         if (++p_ss == NST) { p_ss = 0; p_par ^= 1; }
     };
-    for (int s = 0; s < NST - 1; ++s) {
+    // The ring runs NST - 2 stages ahead: the slot refilled at stage sg is the one released two stages
+    // earlier, so the warp on duty practically never waits for a slower warp.
+    for (int s = 0; s < NST - 2; ++s) {
         if (s < T && warp == 0) issue_next();
         advance_next();
     }
@@ -369,7 +371,7 @@ k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CU
     float2 Qr[CPL][RP2];     // rows of Q' for this lane's columns of the current column half, pairs over k
     float pprev_reg = 0.f;   // thread < PR: its entry of P~_{t-1} for the block being projected
 
-    const int k0 = nstb >= 3 ? 1 : 0;   // stage of a block at which the previous block's P' is finished
+    const int k0 = nstb / 2;            // stage of a block at which the previous block's P' is finished
     const int span = nstb - k0;         // stages over which the previous block's 8 rows are back-projected
     int ss = 0, par = 0;                // ring slot and parity of the stage being consumed
     int sg = 0;
@@ -398,8 +400,8 @@ k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CU
             }
             for (int i = 0; i < N; ++i, ++sl, ++sg) {
                 if (warp == (sg & 7)) {           // this warp's turn to refill the ring
-                    if (sg + NST - 1 < T) {
-                        if (sg > 0) mbar_wait(bar_empty + 8 * p_ss, (unsigned)p_par, a.flags, dead);
+                    if (sg + NST - 2 < T) {
+                        if (sg > 1) mbar_wait(bar_empty + 8 * p_ss, (unsigned)p_par, a.flags, dead);
                         issue_next();
                     }
                 }
