@@ -406,13 +406,13 @@ EncodeTiledFn encode_tiled_fn() {
     }
     return fn;
 }
-// Rank-3 map over [count*N][m][n] float32 with tiles of 8 rows x bw columns of one node; out-of-range reads give zeros.
-bool make_tile_map(CUtensorMap* map, const float* base, int64_t n, int64_t m, int64_t mats, int bw) {
+// Rank-3 map over [count*N][m][n] float32 with tiles of `rows` rows x bw columns of one node; out-of-range reads give zeros.
+bool make_tile_map(CUtensorMap* map, const float* base, int64_t n, int64_t m, int64_t mats, int bw, int rows) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {(cuuint64_t)n, (cuuint64_t)m, (cuuint64_t)mats};
     cuuint64_t strides[2] = {(cuuint64_t)n * 4, (cuuint64_t)m * (cuuint64_t)n * 4};
-    cuuint32_t box[3] = {(cuuint32_t)bw, (cuuint32_t)FU_R, 1};
+    cuuint32_t box[3] = {(cuuint32_t)bw, (cuuint32_t)rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -455,9 +455,9 @@ void launch_fused_t(Launcher& L, psgd_handle* h, const float* G, FusedArgs a) {
     a.KC = h->KC;
     cfg.gridDim = dim3((unsigned)((size_t)h->CS * h->KC * h->count));
     CUtensorMap tmG, tmM;
-    const int bw = FusedGeom<WC>::BW;
-    if (!make_tile_map(&tmG, G, h->n, h->m, (int64_t)h->count * h->N, bw) ||
-        !make_tile_map(&tmM, h->E, h->n, h->m, (int64_t)h->count * h->N, bw)) {
+    const int bw = FusedGeom<WC>::BW, rs = FusedGeom<WC>::RS;
+    if (!make_tile_map(&tmG, G, h->n, h->m, (int64_t)h->count * h->N, bw, rs) ||
+        !make_tile_map(&tmM, h->E, h->n, h->m, (int64_t)h->count * h->N, bw, rs)) {
         snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
         L.status = PSGD_E_CUDA;
         return;

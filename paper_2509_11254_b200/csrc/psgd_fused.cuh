@@ -18,12 +18,17 @@
 //     comes out nearly orthonormal and W = Delta^T P' keeps float32 accuracy.
 //
 // A thread-block CLUSTER owns row blocks of 8 rows for all N nodes; each CTA of the cluster
-// owns a column slice of WC columns.  G and the stored Delta arrive as TMA tiles (8 rows x up to
-// 256 columns of one node, cp.async.bulk.tensor with zero fill beyond the matrix edges) in a
-// ring of shared-memory stages whose completion is tracked by mbarriers; the warps take turns
-// issuing the copies.  S is kept in a double-buffered shared-memory tile; the 8 x r partial
-// sums of P are pushed to the peers' shared memory (DSMEM) and the cluster barrier is split
-// into arrive / wait so that its latency is covered by the next block's loads and arithmetic.
+// owns a column slice of WC columns.  The CTA's 16 warps are split into two roles with their
+// own register budgets (setmaxnreg):
+//   * 8 projection warps: G and the stored Delta arrive as TMA tiles (cp.async.bulk.tensor,
+//     zero fill beyond the matrix edges) in a ring of shared-memory stages tracked by
+//     mbarriers; the warps take turns issuing the copies, form S, keep it in a double-buffered
+//     shared-memory tile, accumulate S Q' and send the 8 x r partial sums of P to every CTA
+//     of the cluster (st.async into the peers' shared memory, counted by their mbarriers);
+//   * 8 back-projection warps: one block behind, they finish P' of a block, apply the
+//     correction to the tile, accumulate W in registers and write Delta_t to HBM.
+// The two roles meet only through mbarriers (tile written / tile free), so the latency of
+// the cluster exchange and of either role is covered by the other.
 // Float sums are formed in a fixed order everywhere (bit-reproducible results).  Every
 // mbarrier wait is bounded; a wait that runs out sets PSGD_W_TIMEOUT in the status word and
 // the kernel carries on to its end.
@@ -36,7 +41,8 @@
 namespace psgd {
 namespace cg = cooperative_groups;
 
-constexpr int FU_THREADS = 256;
+constexpr int FU_THREADS = 512;     // 8 projection warps + 8 back-projection warps
+constexpr int FU_ROLE = 256;        // threads per role
 constexpr int FU_R = 8;        // rows per block
 constexpr int FU_RG = 4;       // rows per warp task
 constexpr int FU_MAXCS = 8;    // largest cluster
@@ -59,13 +65,17 @@ struct FusedArgs {
 
 template <int WC>
 struct FusedGeom {
-    static constexpr int BW = WC >= 256 ? 256 : WC;      // columns of one TMA tile = one stage
-    static constexpr int NH = WC / BW;                   // stages per node and block
-    static constexpr int CPL = BW / 128;                 // columns per lane in the projection phase
-    static constexpr int NCG = 4;                        // column groups per stage (one warp each, two row groups)
-    static constexpr int NST = BW == 256 ? 5 : 8;        // ring depth
+    static constexpr int BW = WC >= 256 ? 256 : WC;      // columns of one TMA tile
+    static constexpr int NBX = WC / BW;                  // TMA tiles per array and stage
+    static constexpr int CPL = WC >= 256 ? 2 : 1;        // columns per lane in the projection role
+    static constexpr int NCG = WC / (32 * CPL);          // column groups of a stage (one warp each)
+    static constexpr int NRG = 8 / NCG;                  // row groups of a stage
+    static constexpr int RS = FU_RG * NRG;               // rows of a stage
+    static constexpr int NRC = FU_R / RS;                // stages (row chunks) per node and block
+    static constexpr int NST = WC >= 256 ? 5 : 8;        // ring depth
     static constexpr int TPN = WC / 8;                   // back-projection threads per node
-    static constexpr int STAGE_FLOATS = 2 * FU_R * BW;   // G tile, then stored-Delta tile
+    static constexpr int STAGE_FLOATS = 2 * RS * WC;     // G rows, then stored-Delta rows; each array as NBX tiles [RS][BW]
+    static constexpr int NBAR = 2 * NST + 6;             // full/empty per stage, 2 x (received, tile written, tile free)
 };
 
 template <int RP, int WC>
@@ -73,12 +83,11 @@ __host__ __device__ inline size_t fused_smem_bytes(int N) {
     using Ge = FusedGeom<WC>;
     size_t fl = (size_t)2 * N * FU_R * WC            // S tile, double-buffered
               + (size_t)Ge::NST * Ge::STAGE_FLOATS   // ring
-              + (size_t)2 * 2 * Ge::NH * Ge::NCG * 32   // per-warp partial sums of P
+              + (size_t)2 * 2 * Ge::NCG * 32         // per-warp partial sums of P
               + (size_t)2 * FU_MAXCS * FU_R * RP     // partial sums received from the cluster
-              + (size_t)2 * FU_R * RP                // P' rows
-              + (size_t)2 * FU_R * RP                // P~_{t-1} rows
+              + (size_t)3 * 2 * FU_R * RP            // P' rows, P' rows with swapped pairs, -P~_{t-1} rows
               + (size_t)RP * RP;                     // C'
-    return fl * 4 + (size_t)(2 * Ge::NST + 2) * 8 + 128;   // + alignment slack for the TMA destinations
+    return fl * 4 + (size_t)Ge::NBAR * 8 + 128;      // + alignment slack for the TMA destinations
 }
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -146,14 +155,23 @@ __device__ __forceinline__ void butterfly_reduce(float (&v)[NV], int lane) {
     if (NV == 16) v[0] += __shfl_xor_sync(0xffffffffu, v[0], 1);
 }
 
-// d = a * b + c on two packed floats (one instruction slot on sm_100)
-__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+// Two packed floats in one 64-bit register (low half = .x), kept packed from the load to the last use so
+// that no pack / unpack moves are needed around the packed FMA.
+typedef unsigned long long f2p;
+__device__ __forceinline__ f2p pack2(float x, float y) {
+    f2p d;
+    asm("mov.b64 %0, {%1, %2};\n" : "=l"(d) : "f"(x), "f"(y));
+    return d;
+}
+__device__ __forceinline__ float2 unpack2(f2p v) {
     float2 d;
-    asm("{\n.reg .b64 ra, rb, rc, rd;\n"
-        "mov.b64 ra, {%2, %3};\nmov.b64 rb, {%4, %5};\nmov.b64 rc, {%6, %7};\n"
-        "fma.rn.f32x2 rd, ra, rb, rc;\n"
-        "mov.b64 {%0, %1}, rd;\n}\n"
-        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+    asm("mov.b64 {%0, %1}, %2;\n" : "=f"(d.x), "=f"(d.y) : "l"(v));
+    return d;
+}
+// d = a * b + c on two packed floats (one instruction slot on sm_100)
+__device__ __forceinline__ f2p ffma2(f2p a, f2p b, f2p c) {
+    f2p d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(d) : "l"(a), "l"(b), "l"(c));
     return d;
 }
 
@@ -166,15 +184,20 @@ __device__ __forceinline__ void st_async_cluster_f32(unsigned local_addr, unsign
                  ::"r"(raddr), "r"(__float_as_uint(v)), "r"(rbar) : "memory");
 }
 
+__device__ __forceinline__ void role_barrier(int id) {   // barrier among the 256 threads of one role
+    asm volatile("bar.sync %0, 256;\n" ::"r"(id) : "memory");
+}
+
 template <int RP, int WC, bool PENDING>
 __global__ void __launch_bounds__(FU_THREADS, 1)
 k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmM, FusedArgs a) {
     using Ge = FusedGeom<WC>;
-    constexpr int BW = Ge::BW, NH = Ge::NH, CPL = Ge::CPL, NCG = Ge::NCG, NST = Ge::NST, TPN = Ge::TPN;
+    constexpr int BW = Ge::BW, NBX = Ge::NBX, CPL = Ge::CPL, NCG = Ge::NCG, RS = Ge::RS, NRC = Ge::NRC, NST = Ge::NST, TPN = Ge::TPN;
     constexpr int NV = FU_RG * RP;         // per-lane partial sums of one warp task
     constexpr int PR = FU_R * RP;          // entries of one block of P
     constexpr int RP2 = RP / 2;
     constexpr unsigned STAGE_BYTES = Ge::STAGE_FLOATS * 4;
+    constexpr unsigned BOX_BYTES = RS * BW * 4;
 
     extern __shared__ __align__(16) float smem_raw[];
     float* smem = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
@@ -189,234 +212,121 @@ k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CU
     const int ncols = max(0, colend - colbase);
 
     // ---- shared memory carve-up ----
-    float* ring = smem;                                        // [NST][2][8][BW]   (128-byte aligned)
+    float* ring = smem;                                        // [NST][2][NBX][RS][BW]   (128-byte aligned)
     float* tile = ring + (size_t)NST * Ge::STAGE_FLOATS;       // [2][N][8][WC]
-    float* PpartW = tile + (size_t)2 * N * FU_R * WC;          // [2][2][NH*NCG][32]
-    float* Precv = PpartW + 2 * 2 * NH * NCG * 32;             // [2][FU_MAXCS][PR]
+    float* PpartW = tile + (size_t)2 * N * FU_R * WC;          // [2][2][NCG][32]
+    float* Precv = PpartW + 2 * 2 * NCG * 32;                  // [2][FU_MAXCS][PR]
     float* Pb = Precv + 2 * FU_MAXCS * PR;                     // [2][PR]   P' rows
-    float* Pp = Pb + 2 * PR;                                   // [2][PR]   P~_{t-1} rows
-    float* Cm = Pp + 2 * PR;                                   // [RP][RP]
+    float* Pbs = Pb + 2 * PR;                                  // [2][PR]   P' rows, neighbours (2k, 2k+1) swapped
+    float* Ppn = Pbs + 2 * PR;                                 // [2][PR]   -P~_{t-1} rows
+    float* Cm = Ppn + 2 * PR;                                  // [RP][RP]
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(Cm + RP * RP);
-    const unsigned bar_full = smem_u32(bars), bar_empty = smem_u32(bars + NST), bar_recv = smem_u32(bars + 2 * NST);
+    const unsigned bar_full = smem_u32(bars), bar_empty = bar_full + 8 * NST, bar_recv = bar_empty + 8 * NST;
+    const unsigned bar_tfull = bar_recv + 16, bar_tfree = bar_tfull + 16;
 
     float* Mc = a.Mbuf + (size_t)c * N * m * n;
-    const float* Qc = a.Qpad + (size_t)c * n * RP;
-    const float* Ppc = PENDING ? a.Ppad + (size_t)c * m * RP : nullptr;
-    const float* Qsc = PENDING ? a.Qsub + (size_t)c * (a.qsub_node_stride ? N : 1) * n * RP : nullptr;
 
     // row blocks this cluster owns: slot, slot + KC, ...
     const int nb = (a.nblk > slot) ? (a.nblk - slot + a.KC - 1) / a.KC : 0;
-    const int nstb = NH * N;               // stages per block: column half outer, node inner
+    const int nstb = NRC * N;              // stages per block: row chunk outer, node inner
     const int T = nb * nstb;
 
     // ---- one-time set-up ----
     if (tid == 0) {
         for (int s = 0; s < NST; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, FU_THREADS / 32);
+            mbar_init(bar_empty + 8 * s, FU_ROLE / 32);
         }
-        mbar_init(bar_recv, 1);
-        mbar_init(bar_recv + 8, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_recv + 8 * b, 1);
+            mbar_init(bar_tfull + 8 * b, FU_ROLE / 32);
+            mbar_init(bar_tfree + 8 * b, FU_ROLE / 32);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     if (PENDING)
         for (int e = tid; e < RP * RP; e += FU_THREADS) Cm[e] = a.Cmat[(size_t)c * RP * RP + e];
     cluster.sync();   // every CTA's barriers exist before a peer sends to them
     bool dead = false;
+    const f2p ZERO2 = 0ull;
 
-    // projection phase: warp -> (column group, row group) of a stage, lane -> CPL adjacent columns
-    const int cgp = warp % NCG, rgl = warp / NCG;
-    const int acol = cgp * 32 * CPL + lane * CPL;      // column within the stage
-    // back-projection phase: thread -> (node, 4 + 4 columns)
-    const int bi = tid / TPN, tc = tid % TPN;
-    const bool btask = bi < N;
-    const int bc0 = 4 * tc, bc1 = WC / 2 + 4 * tc;
-    const bool bok0 = btask && bc0 < ncols, bok1 = btask && bc1 < ncols;
-    float2 wacc[8][RP2];                   // W for 8 columns, pairs over k
-    constexpr int QSN = PENDING ? 4 : 1;
-    float2 qs[QSN][RP];                    // Qsub for column pairs (2j, 2j+1), per k
+    if (warp < FU_ROLE / 32) {
+        // =====================================================================================
+        // projection role
+        // =====================================================================================
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 88;\n");
+        const float* Qc = a.Qpad + (size_t)c * n * RP;
+        // warp -> (column group, row group) of a stage, lane -> CPL adjacent columns (fixed for the kernel)
+        const int cgp = warp % NCG, rgl = warp / NCG;
+        const int acol = cgp * 32 * CPL + lane * CPL;                       // column within the slice
+        const int abox = acol / BW, aboxcol = acol % BW;                    // TMA tile and column inside it
+        f2p Qr[CPL][RP2];        // rows of Q' for this lane's columns, pairs over k
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
-#pragma unroll
-        for (int k = 0; k < RP2; ++k) wacc[j][k] = make_float2(0.f, 0.f);
-    if (PENDING) {
-        float t8[8][RP];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int col = (j < 4 ? bc0 : bc1) + (j & 3);
+        for (int j = 0; j < CPL; ++j)
 #pragma unroll
             for (int k4 = 0; k4 < RP / 4; ++k4) {
-                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (btask && col < ncols)
-                    v = __ldg(reinterpret_cast<const float4*>(Qsc + (size_t)bi * a.qsub_node_stride + (size_t)(colbase + col) * RP + 4 * k4));
-                t8[j][4 * k4 + 0] = v.x; t8[j][4 * k4 + 1] = v.y; t8[j][4 * k4 + 2] = v.z; t8[j][4 * k4 + 3] = v.w;
+                ulonglong2 v = make_ulonglong2(0ull, 0ull);
+                if (acol + j < ncols) v = __ldg(reinterpret_cast<const ulonglong2*>(Qc + (size_t)(colbase + acol + j) * RP + 4 * k4));
+                Qr[j][2 * k4] = v.x;
+                Qr[j][2 * k4 + 1] = v.y;
             }
-        }
-#pragma unroll
-        for (int j2 = 0; j2 < QSN; ++j2)
-#pragma unroll
-            for (int k = 0; k < RP; ++k) qs[j2][k] = make_float2(t8[(2 * j2) % 8][k], t8[(2 * j2 + 1) % 8][k]);
-    }
 
-    // ---- producer role (taken in turn by the warps): two TMA tiles per stage ----
-    // state of the next stage to issue, advanced by every thread in step with the main loop
-    int p_bl = 0, p_h = 0, p_i = 0, p_ss = 0, p_par = 1;   // p_par: parity of the slot's previous release
-    auto issue_next = [&]() {      // called by one whole warp; the slot must have been released
-        if (lane == 0) {
-            const int row = (slot + p_bl * a.KC) * FU_R;
-            const unsigned bar = bar_full + 8 * p_ss;
-            const unsigned dst = smem_u32(ring + (size_t)p_ss * Ge::STAGE_FLOATS);
-            mbar_expect_tx(bar, STAGE_BYTES);
-            tma_load_3d(dst, &tmG, colbase + p_h * BW, row, c * N + p_i, bar);
-            tma_load_3d(dst + STAGE_BYTES / 2, &tmM, colbase + p_h * BW, row, c * N + p_i, bar);
-        }
-        __syncwarp();
-    };
-    auto advance_next = [&]() {
-        if (++p_i == N) { p_i = 0; if (++p_h == NH) { p_h = 0; ++p_bl; } }
-        if (++p_ss == NST) { p_ss = 0; p_par ^= 1; }
-    };
-    // The ring runs NST - 2 stages ahead: the slot refilled at stage sg is the one released two stages
-    // earlier, so the warp on duty practically never waits for a slower warp.
-    for (int s = 0; s < NST - 2; ++s) {
-        if (s < T && warp == 0) issue_next();
-        advance_next();
-    }
-
-    // P' of one finished block: node mean of the received partial sums, small-space correction.
-    // Every thread waits for the cluster's partial sums itself (bounded), so no barrier follows the wait.
-    auto finish_block = [&](int bl) {
-        const int pb = bl & 1;
-        const int prow0 = (slot + bl * a.KC) * FU_R;
-        mbar_wait(bar_recv + 8 * pb, (unsigned)((bl >> 1) & 1), a.flags, dead);
-        if (tid < PR) {
-            const int rr = tid / RP, k = tid % RP;
-            float sum = 0.f;
-            for (int qq = 0; qq < CS; ++qq) sum += Precv[(pb * FU_MAXCS + qq) * PR + tid];
-            float v = sum / (float)N;
-            if (PENDING) {
-                const float* pp = Pp + pb * PR + rr * RP;
+        // producer duty (taken in turn by the warps): 2 * NBX TMA tiles per stage.
+        // State of the next stage to issue, advanced by every thread in step with the main loop.
+        int p_bl = 0, p_rc = 0, p_i = 0, p_ss = 0, p_par = 1;   // p_par: parity of the slot's previous release
+        auto issue_next = [&]() {      // called by one whole warp; the slot must have been released
+            if (lane == 0) {
+                const int row = (slot + p_bl * a.KC) * FU_R + p_rc * RS;
+                const unsigned bar = bar_full + 8 * p_ss;
+                const unsigned dst = smem_u32(ring + (size_t)p_ss * Ge::STAGE_FLOATS);
+                mbar_expect_tx(bar, STAGE_BYTES);
 #pragma unroll
-                for (int j = 0; j < RP; ++j) v = fmaf(-pp[j], Cm[j * RP + k], v);
-            }
-            if (prow0 + rr >= m) v = 0.f;
-            Pb[pb * PR + tid] = v;
-            if (q == 0 && prow0 + rr < m) a.Pout[((size_t)c * m + prow0 + rr) * RP + k] = v;
-        }
-        __syncthreads();
-    };
-    double gacc = 0.0;   // rank 0, threads 64 .. 64 + r*r: one entry of P'^T P'
-    auto gram_block = [&](int bl) {
-        const int pb = bl & 1;
-        const int t2 = tid - 64;
-        if (q == 0 && t2 >= 0 && t2 < a.r * a.r) {
-            const int ga = t2 / a.r, gb = t2 % a.r;
-#pragma unroll
-            for (int rr = 0; rr < FU_R; ++rr)
-                gacc = fma((double)Pb[pb * PR + rr * RP + ga], (double)Pb[pb * PR + rr * RP + gb], gacc);
-        }
-    };
-    // back-projection of row rr of block bl: Delta = S - P~_{t-1} Qsub^T, W += Delta^T P', store Delta
-    auto back_row = [&](int bl, int rr) {
-        if (!btask) return;
-        const int pb = bl & 1;
-        const int prow = (slot + bl * a.KC) * FU_R + rr;
-        const float* tp = tile + (((size_t)pb * N + bi) * FU_R + rr) * WC;
-        const float4 v0 = *reinterpret_cast<const float4*>(tp + bc0);
-        const float4 v1 = *reinterpret_cast<const float4*>(tp + bc1);
-        float2 mv[4] = {make_float2(v0.x, v0.y), make_float2(v0.z, v0.w), make_float2(v1.x, v1.y), make_float2(v1.z, v1.w)};
-        if (PENDING) {
-            const float* pp = Pp + pb * PR + rr * RP;
-#pragma unroll
-            for (int k4 = 0; k4 < RP / 4; ++k4) {
-                const float4 p4 = *reinterpret_cast<const float4*>(pp + 4 * k4);
-                const float pk[4] = {-p4.x, -p4.y, -p4.z, -p4.w};
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const float2 pd = make_float2(pk[kk], pk[kk]);
-#pragma unroll
-                    for (int j2 = 0; j2 < 4; ++j2) mv[j2] = ffma2(pd, qs[j2 % QSN][4 * k4 + kk], mv[j2]);
+                for (int x = 0; x < NBX; ++x) {
+                    tma_load_3d(dst + x * BOX_BYTES, &tmG, colbase + x * BW, row, c * N + p_i, bar);
+                    tma_load_3d(dst + STAGE_BYTES / 2 + x * BOX_BYTES, &tmM, colbase + x * BW, row, c * N + p_i, bar);
                 }
             }
+            __syncwarp();
+        };
+        auto advance_next = [&]() {
+            if (++p_i == N) { p_i = 0; if (++p_rc == NRC) { p_rc = 0; ++p_bl; } }
+            if (++p_ss == NST) { p_ss = 0; p_par ^= 1; }
+        };
+        // The ring runs NST - 2 stages ahead: the slot refilled at stage sg is the one released two stages
+        // earlier, so the warp on duty practically never waits for a slower warp.
+        for (int s = 0; s < NST - 2; ++s) {
+            if (s < T && warp == 0) issue_next();
+            advance_next();
         }
-        const float* pr = Pb + pb * PR + rr * RP;
-        float2 pk2[RP2];
-#pragma unroll
-        for (int k4 = 0; k4 < RP / 4; ++k4) {
-            const float4 p4 = *reinterpret_cast<const float4*>(pr + 4 * k4);
-            pk2[2 * k4] = make_float2(p4.x, p4.y);
-            pk2[2 * k4 + 1] = make_float2(p4.z, p4.w);
-        }
-#pragma unroll
-        for (int j2 = 0; j2 < 4; ++j2) {
-            const float2 mx = make_float2(mv[j2].x, mv[j2].x), my = make_float2(mv[j2].y, mv[j2].y);
-#pragma unroll
-            for (int k2 = 0; k2 < RP2; ++k2) {
-                wacc[2 * j2][k2] = ffma2(mx, pk2[k2], wacc[2 * j2][k2]);
-                wacc[2 * j2 + 1][k2] = ffma2(my, pk2[k2], wacc[2 * j2 + 1][k2]);
-            }
-        }
-        if (prow < m) {
-            float* go = Mc + ((size_t)bi * m + prow) * n + colbase;
-            if (bok0) *reinterpret_cast<float4*>(go + bc0) = make_float4(mv[0].x, mv[0].y, mv[1].x, mv[1].y);
-            if (bok1) *reinterpret_cast<float4*>(go + bc1) = make_float4(mv[2].x, mv[2].y, mv[3].x, mv[3].y);
-        }
-    };
 
-    float2 sacc[FU_RG][RP2];
+        f2p sacc[FU_RG][RP2];
 #pragma unroll
-    for (int rr = 0; rr < FU_RG; ++rr)
+        for (int rr = 0; rr < FU_RG; ++rr)
 #pragma unroll
-        for (int k = 0; k < RP2; ++k) sacc[rr][k] = make_float2(0.f, 0.f);
-    float2 Qr[CPL][RP2];     // rows of Q' for this lane's columns of the current column half, pairs over k
-    float pprev_reg = 0.f;   // thread < PR: its entry of P~_{t-1} for the block being projected
-
-    const int k0 = nstb / 2;            // stage of a block at which the previous block's P' is finished
-    const int span = nstb - k0;         // stages over which the previous block's 8 rows are back-projected
-    int ss = 0, par = 0;                // ring slot and parity of the stage being consumed
-    int sg = 0;
-    for (int bl = 0; bl < nb; ++bl) {
-        const int row0 = (slot + bl * a.KC) * FU_R;
-        const int pbuf = bl & 1;
-        int brow = 0, bacc = 0;         // rows of the previous block done so far; Bresenham accumulator
-        if (tid == 0) mbar_expect_tx(bar_recv + 8 * pbuf, (unsigned)(CS * PR * 4));
-        if (PENDING && tid < PR) {
-            const int rr = tid / RP;
-            pprev_reg = (row0 + rr < m) ? __ldg(Ppc + (size_t)(row0 + rr) * RP + tid % RP) : 0.f;
-        }
-        int sl = 0;
-        for (int h = 0; h < NH; ++h) {
-            if (NH > 1 || bl == 0) {   // (re)load this lane's rows of Q' for the column half
-#pragma unroll
-                for (int j = 0; j < CPL; ++j)
-#pragma unroll
-                    for (int k4 = 0; k4 < RP / 4; ++k4) {
-                        const int col = h * BW + acol + j;
-                        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (col < ncols) v = __ldg(reinterpret_cast<const float4*>(Qc + (size_t)(colbase + col) * RP + 4 * k4));
-                        Qr[j][2 * k4] = make_float2(v.x, v.y);
-                        Qr[j][2 * k4 + 1] = make_float2(v.z, v.w);
+            for (int k = 0; k < RP2; ++k) sacc[rr][k] = ZERO2;
+        int ss = 0, par = 0;                // ring slot and parity of the stage being consumed
+        int sg = 0;
+        for (int bl = 0; bl < nb; ++bl) {
+            const int pbuf = bl & 1;
+            // the tile buffer was last read by the back-projection of block bl - 2
+            if (bl >= 2) mbar_wait(bar_tfree + 8 * pbuf, (unsigned)(((bl >> 1) - 1) & 1), a.flags, dead);
+#pragma unroll 1
+            for (int rc = 0; rc < NRC; ++rc) {
+#pragma unroll 1
+                for (int i = 0; i < N; ++i, ++sg) {
+                    if (warp == (sg & 7)) {           // this warp's turn to refill the ring
+                        if (sg + NST - 2 < T) {
+                            if (sg > 1) mbar_wait(bar_empty + 8 * p_ss, (unsigned)p_par, a.flags, dead);
+                            issue_next();
+                        }
                     }
-            }
-            for (int i = 0; i < N; ++i, ++sl, ++sg) {
-                if (warp == (sg & 7)) {           // this warp's turn to refill the ring
-                    if (sg + NST - 2 < T) {
-                        if (sg > 1) mbar_wait(bar_empty + 8 * p_ss, (unsigned)p_par, a.flags, dead);
-                        issue_next();
-                    }
-                }
-                advance_next();
-                if (bl > 0 && sl == k0) {
-                    finish_block(bl - 1);
-                    gram_block(bl - 1);
-                }
+                    advance_next();
 
-                // ---- projection: S = g + stored Delta -> tile; sacc += S Q' ----
-                mbar_wait(bar_full + 8 * ss, (unsigned)par, a.flags, dead);
-                {
-                    const float* sgp = ring + (size_t)ss * Ge::STAGE_FLOATS + (size_t)(rgl * FU_RG) * BW + acol;
-                    const float* smp = sgp + FU_R * BW;
-                    float* tp = tile + (((size_t)pbuf * N + i) * FU_R + rgl * FU_RG) * WC + h * BW + acol;
+                    // ---- S = g + stored Delta -> tile; sacc += S Q' ----
+                    mbar_wait(bar_full + 8 * ss, (unsigned)par, a.flags, dead);
+                    const float* sgp = ring + (size_t)ss * Ge::STAGE_FLOATS + (size_t)abox * (RS * BW) + (size_t)(rgl * FU_RG) * BW + aboxcol;
+                    const float* smp = sgp + RS * WC;
+                    float* tp = tile + (((size_t)pbuf * N + i) * FU_R + rc * RS + rgl * FU_RG) * WC + acol;
                     float sv[FU_RG][CPL];
 #pragma unroll
                     for (int rr = 0; rr < FU_RG; ++rr) {
@@ -436,73 +346,201 @@ k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CU
                         else tp[rr * WC] = sv[rr][0];
 #pragma unroll
                         for (int j = 0; j < CPL; ++j) {
-                            const float2 sd = make_float2(sv[rr][j], sv[rr][j]);
+                            const f2p sd = pack2(sv[rr][j], sv[rr][j]);
 #pragma unroll
                             for (int k2 = 0; k2 < RP2; ++k2) sacc[rr][k2] = ffma2(sd, Qr[j][k2], sacc[rr][k2]);
                         }
                     }
-                }
-                if (++ss == NST) { ss = 0; par ^= 1; }
+                    if (++ss == NST) { ss = 0; par ^= 1; }
 
-                if (i == N - 1) {   // the column half is complete for every node: reduce over the warp's columns
-                    float v[NV];
+                    if (i == N - 1) {   // the row chunk is complete for every node: reduce over the warp's columns
+                        float v[NV];
 #pragma unroll
-                    for (int rr = 0; rr < FU_RG; ++rr)
+                        for (int rr = 0; rr < FU_RG; ++rr)
 #pragma unroll
-                        for (int k2 = 0; k2 < RP2; ++k2) {
-                            v[rr * RP + 2 * k2] = sacc[rr][k2].x;
-                            v[rr * RP + 2 * k2 + 1] = sacc[rr][k2].y;
-                            sacc[rr][k2] = make_float2(0.f, 0.f);
-                        }
-                    butterfly_reduce<NV>(v, lane);
-                    if (NV == 32 || (lane & 1) == 0)
-                        PpartW[((pbuf * 2 + rgl) * (NH * NCG) + h * NCG + cgp) * 32 + (NV == 32 ? lane : lane >> 1)] = v[0];
+                            for (int k2 = 0; k2 < RP2; ++k2) {
+                                const float2 u = unpack2(sacc[rr][k2]);
+                                v[rr * RP + 2 * k2] = u.x;
+                                v[rr * RP + 2 * k2 + 1] = u.y;
+                                sacc[rr][k2] = ZERO2;
+                            }
+                        butterfly_reduce<NV>(v, lane);
+                        const int rgi = rc * Ge::NRG + rgl;     // row group within the block (0 or 1)
+                        if (NV == 32 || (lane & 1) == 0)
+                            PpartW[((pbuf * 2 + rgi) * NCG + cgp) * 32 + (NV == 32 ? lane : lane >> 1)] = v[0];
+                    }
                 }
-
-                // ---- back-projection of the previous block, spread over this block's stages ----
-                if (bl > 0 && sl >= k0) {
-                    bacc += FU_R;
-                    while (bacc >= span && brow < FU_R) { back_row(bl - 1, brow); ++brow; bacc -= span; }
+            }
+            // block projected: the tile is complete; CTA sum of the partial P, sent to every CTA of the cluster
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tfull + 8 * pbuf);
+            role_barrier(1);
+            if (tid < PR) {
+                const int rr = tid / RP, k = tid % RP;
+                const int rgi = rr / FU_RG, j = (rr % FU_RG) * RP + k;
+                float sum = 0.f;
+#pragma unroll
+                for (int g = 0; g < NCG; ++g) sum += PpartW[((pbuf * 2 + rgi) * NCG + g) * 32 + j];
+                const unsigned dst = smem_u32(Precv + (pbuf * FU_MAXCS + q) * PR + tid);
+                for (int qq = 0; qq < CS; ++qq) st_async_cluster_f32(dst, bar_recv + 8 * pbuf, (unsigned)qq, sum);
+            }
+        }
+    } else {
+        // =====================================================================================
+        // back-projection role (one block behind the projection)
+        // =====================================================================================
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 168;\n");
+        const int tb = tid - FU_ROLE;
+        const float* Ppc = PENDING ? a.Ppad + (size_t)c * m * RP : nullptr;
+        const float* Qsc = PENDING ? a.Qsub + (size_t)c * (a.qsub_node_stride ? N : 1) * n * RP : nullptr;
+        // thread -> (node, 4 + 4 columns)
+        const int bi = tb / TPN, tc = tb % TPN;
+        const bool btask = bi < N;
+        const int bc0 = 4 * tc, bc1 = WC / 2 + 4 * tc;
+        const bool bok0 = btask && bc0 < ncols, bok1 = btask && bc1 < ncols;
+        // W for 8 columns in "diagonal" pairs: wd[j2][k2][0] = {w[2j2][2k2], w[2j2+1][2k2+1]}, [1] = {w[2j2][2k2+1], w[2j2+1][2k2]}
+        f2p wd[4][RP2][2];
+        constexpr int QSN = PENDING ? 8 : 1;
+        f2p qs[QSN][RP2];                      // Qsub rows of the 8 columns, pairs over k
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int k = 0; k < RP2; ++k) { wd[j][k][0] = ZERO2; wd[j][k][1] = ZERO2; }
+        if (PENDING) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int col = (j < 4 ? bc0 : bc1) + (j & 3);
+#pragma unroll
+                for (int k4 = 0; k4 < RP / 4; ++k4) {
+                    ulonglong2 v = make_ulonglong2(0ull, 0ull);
+                    if (btask && col < ncols)
+                        v = __ldg(reinterpret_cast<const ulonglong2*>(Qsc + (size_t)bi * a.qsub_node_stride + (size_t)(colbase + col) * RP + 4 * k4));
+                    qs[j % QSN][2 * k4] = v.x;
+                    qs[j % QSN][2 * k4 + 1] = v.y;
                 }
             }
         }
-        // block projected: CTA sum of the partial P, sent to every CTA of the cluster
-        if (PENDING && tid < PR) Pp[pbuf * PR + tid] = pprev_reg;
-        __syncthreads();
-        if (tid < PR) {
-            const int rr = tid / RP, k = tid % RP;
-            const int rgi = rr / FU_RG, j = (rr % FU_RG) * RP + k;
-            float sum = 0.f;
+        double gacc = 0.0;   // rank 0, threads 64 .. 64 + r*r of the role: one entry of P'^T P'
+
+        for (int bl = 0; bl < nb; ++bl) {
+            const int pb = bl & 1;
+            const int prow0 = (slot + bl * a.KC) * FU_R;
+            const unsigned ph = (unsigned)((bl >> 1) & 1);
+            float pprev = 0.f;
+            if (PENDING && tb < PR) {
+                const int rr = tb / RP;
+                pprev = (prow0 + rr < m) ? __ldg(Ppc + (size_t)(prow0 + rr) * RP + tb % RP) : 0.f;
+            }
+            if (tb == 0) mbar_expect_tx(bar_recv + 8 * pb, (unsigned)(CS * PR * 4));
+            if (PENDING && tb < PR) Ppn[pb * PR + tb] = -pprev;
+            role_barrier(2);                      // -P~_{t-1} rows visible to the role
+            // P' of the block: node mean of the cluster's partial sums, small-space correction.
+            // Every thread waits for the sums itself (bounded), so no barrier precedes the reads.
+            mbar_wait(bar_recv + 8 * pb, ph, a.flags, dead);
+            if (tb < PR) {
+                const int rr = tb / RP, k = tb % RP;
+                float sum = 0.f;
+                for (int qq = 0; qq < CS; ++qq) sum += Precv[(pb * FU_MAXCS + qq) * PR + tb];
+                float v = sum / (float)N;
+                if (PENDING) {
+                    const float* pp = Ppn + pb * PR + rr * RP;
 #pragma unroll
-            for (int g = 0; g < NH * NCG; ++g) sum += PpartW[((pbuf * 2 + rgi) * (NH * NCG) + g) * 32 + j];
-            const unsigned dst = smem_u32(Precv + (pbuf * FU_MAXCS + q) * PR + tid);
-            for (int qq = 0; qq < CS; ++qq) st_async_cluster_f32(dst, bar_recv + 8 * pbuf, (unsigned)qq, sum);
-        }
-    }
-    if (nb > 0) {
-        finish_block(nb - 1);
-        gram_block(nb - 1);
+                    for (int j = 0; j < RP; ++j) v = fmaf(pp[j], Cm[j * RP + k], v);
+                }
+                if (prow0 + rr >= m) v = 0.f;
+                Pb[pb * PR + tb] = v;
+                Pbs[pb * PR + (tb ^ 1)] = v;
+                if (q == 0 && prow0 + rr < m) a.Pout[((size_t)c * m + prow0 + rr) * RP + k] = v;
+            }
+            role_barrier(2);                      // P' rows visible to the role
+            {
+                const int t2 = tb - 64;
+                if (q == 0 && t2 >= 0 && t2 < a.r * a.r) {
+                    const int ga = t2 / a.r, gb = t2 % a.r;
+#pragma unroll
+                    for (int rr = 0; rr < FU_R; ++rr)
+                        gacc = fma((double)Pb[pb * PR + rr * RP + ga], (double)Pb[pb * PR + rr * RP + gb], gacc);
+                }
+            }
+            mbar_wait(bar_tfull + 8 * pb, ph, a.flags, dead);   // all of S of this block is in the tile
+            if (btask) {
+                // rows of the block: Delta = S - P~_{t-1} Qsub^T, W += Delta^T P', store Delta
 #pragma unroll 1
-        for (int rr = 0; rr < FU_R; ++rr) back_row(nb - 1, rr);
-    }
+                for (int rr = 0; rr < FU_R; ++rr) {
+                    const float* tp = tile + (((size_t)pb * N + bi) * FU_R + rr) * WC;
+                    const float4 v0 = *reinterpret_cast<const float4*>(tp + bc0);
+                    const float4 v1 = *reinterpret_cast<const float4*>(tp + bc1);
+                    float mvs[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+                    if (PENDING) {
+                        const float* pp = Ppn + pb * PR + rr * RP;
+                        f2p pn2[RP2];
+#pragma unroll
+                        for (int k4 = 0; k4 < RP / 4; ++k4) {
+                            const ulonglong2 p4 = *reinterpret_cast<const ulonglong2*>(pp + 4 * k4);
+                            pn2[2 * k4] = p4.x;
+                            pn2[2 * k4 + 1] = p4.y;
+                        }
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            f2p acc = ffma2(pn2[0], qs[j % QSN][0], ZERO2);
+#pragma unroll
+                            for (int k2 = 1; k2 < RP2; ++k2) acc = ffma2(pn2[k2], qs[j % QSN][k2], acc);
+                            const float2 u = unpack2(acc);
+                            mvs[j] += u.x + u.y;
+                        }
+                    }
+                    const float* pr = Pb + pb * PR + rr * RP;
+                    const float* prs = Pbs + pb * PR + rr * RP;
+#pragma unroll
+                    for (int k4 = 0; k4 < RP / 4; ++k4) {
+                        const ulonglong2 p4 = *reinterpret_cast<const ulonglong2*>(pr + 4 * k4);
+                        const ulonglong2 s4 = *reinterpret_cast<const ulonglong2*>(prs + 4 * k4);
+                        const f2p pk2[2] = {p4.x, p4.y};
+                        const f2p pks2[2] = {s4.x, s4.y};
+#pragma unroll
+                        for (int j2 = 0; j2 < 4; ++j2) {
+                            const f2p mp = pack2(mvs[2 * j2], mvs[2 * j2 + 1]);
+#pragma unroll
+                            for (int u = 0; u < 2; ++u) {
+                                wd[j2][2 * k4 + u][0] = ffma2(mp, pk2[u], wd[j2][2 * k4 + u][0]);
+                                wd[j2][2 * k4 + u][1] = ffma2(mp, pks2[u], wd[j2][2 * k4 + u][1]);
+                            }
+                        }
+                    }
+                    if (prow0 + rr < m) {
+                        float* go = Mc + ((size_t)bi * m + prow0 + rr) * n + colbase;
+                        if (bok0) *reinterpret_cast<float4*>(go + bc0) = make_float4(mvs[0], mvs[1], mvs[2], mvs[3]);
+                        if (bok1) *reinterpret_cast<float4*>(go + bc1) = make_float4(mvs[4], mvs[5], mvs[6], mvs[7]);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tfree + 8 * pb);   // the projection may overwrite this tile buffer
+        }
 
-    // ---- flush this cluster's partial W and Gram ----
-    if (btask) {
+        // ---- flush this cluster's partial W and Gram ----
+        if (btask) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int col = (j < 4 ? bc0 : bc1) + (j & 3);
-            if (col < ncols) {
-                float* wp = a.Wpart + ((((size_t)c * a.KC + slot) * N + bi) * n + colbase + col) * RP;
+            for (int j = 0; j < 8; ++j) {
+                const int col = (j < 4 ? bc0 : bc1) + (j & 3);
+                if (col < ncols) {
+                    float* wp = a.Wpart + ((((size_t)c * a.KC + slot) * N + bi) * n + colbase + col) * RP;
+                    const int j2 = j >> 1, odd = j & 1;
 #pragma unroll
-                for (int k4 = 0; k4 < RP / 4; ++k4)
-                    *reinterpret_cast<float4*>(wp + 4 * k4) =
-                        make_float4(wacc[j][2 * k4].x, wacc[j][2 * k4].y, wacc[j][2 * k4 + 1].x, wacc[j][2 * k4 + 1].y);
+                    for (int k4 = 0; k4 < RP / 4; ++k4) {
+                        // w[j][2k2] and w[j][2k2+1] out of the diagonal pairs
+                        const float2 a0 = unpack2(wd[j2][2 * k4][0]), b0 = unpack2(wd[j2][2 * k4][1]);
+                        const float2 a1 = unpack2(wd[j2][2 * k4 + 1][0]), b1 = unpack2(wd[j2][2 * k4 + 1][1]);
+                        *reinterpret_cast<float4*>(wp + 4 * k4) = odd ? make_float4(b0.y, a0.y, b1.y, a1.y)
+                                                                       : make_float4(a0.x, b0.x, a1.x, b1.x);
+                    }
+                }
             }
         }
-    }
-    {
-        const int t2 = tid - 64;
-        if (q == 0 && t2 >= 0 && t2 < a.r * a.r) a.gram[((size_t)c * a.KC + slot) * a.r * a.r + t2] = gacc;
+        {
+            const int t2 = tb - 64;
+            if (q == 0 && t2 >= 0 && t2 < a.r * a.r) a.gram[((size_t)c * a.KC + slot) * a.r * a.r + t2] = gacc;
+        }
     }
     cluster.sync();   // nobody leaves while a peer may still address its shared memory
 }
