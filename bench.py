@@ -29,6 +29,9 @@ sys.path.insert(0, ROOT)
 METRIC = "powersgd_plus_step_gradient_throughput"
 UNIT = "GB/s"
 FALLBACK_HBM = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per element of one launch, from the ncu captures summarised under
+# profiles/ (taken on the 16384x4096, N=4 workload, where traffic grows in proportion to the elements)
+TRAFFIC_BYTES_PER_ELEMENT = {"k_fused_step": 11.86}
 
 # default (rank, nodes, refresh period) per workload id
 DEFAULTS = {2: (8, 8, 50), 3: (16, 16, 20), 4: (32, 8, 100), 5: (16, 4, 0), 1: (4, 4, 5)}
@@ -233,7 +236,7 @@ def timed_steps(torch, handles, bufs, steps, dist_barrier):
     return ev0.elapsed_time(ev1)
 
 
-def sweep_config5(torch, device, peak):
+def sweep_config5(torch, device, peak, mode):
     """BASELINE config 5: m=16384, n=4096, N=4, per-rank step and refresh latency."""
     from paper_2509_11254_b200 import PowerSGDPlus, synth
 
@@ -241,7 +244,7 @@ def sweep_config5(torch, device, peak):
     bufs = [synth.make_gradients_torch(5, m, n, N, 1, step=b, device=device) for b in range(2)]
     out = []
     for r in (1, 4, 16, 64, 128):
-        h = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=5, device=device)
+        h = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=5, device=device, mode=mode)
         for s in range(3):
             h.step(bufs[s % 2])
         steps = 10
@@ -263,7 +266,8 @@ def sweep_config5(torch, device, peak):
         rms = ev0.elapsed_time(ev1) / 2
         flags = h.last_status()
         alg, gb = algorithmic_bytes([(m, n, 1)], r, N)
-        out.append({"r": r, "step_ms": round(ms, 4), "grad_GBps": round(gb / ms / 1e6, 1),
+        plan = h.plan_info()
+        out.append({"r": r, "kernel": "single-pass" if (mode == "deferred" and plan["single_pass"]) else "eager", "step_ms": round(ms, 4), "grad_GBps": round(gb / ms / 1e6, 1),
                     "north_star_frac": round(alg / ms / 1e6 / peak, 4), "refresh_ms": round(rms, 3),
                     "flags": flags})
         h.close()
@@ -350,8 +354,15 @@ def run_ours(args):
     if dom != "project":
         ssp_frac = 1.0  # the tail kernels run on refresh steps too
     achieved = per_family_bytes[dom] * ssp_frac / dom_ms_per_step / 1e6 if dom_ms_per_step else None
-    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak if achieved else None, "traffic": None, "peak_source": f"of {peak_kind}",
+    plans = [h.plan_info() for h in handles]
+    single_pass = args.mode == "deferred" and all(p["single_pass"] for p in plans)
+    kernel_name = "k_fused_step" if (dom == "project" and single_pass) else "k_" + dom
+    # DRAM bytes per element of the dominant kernel from the committed ncu capture (profiles/), scaled to this
+    # workload's elements; None for kernels without a current capture
+    traffic = TRAFFIC_BYTES_PER_ELEMENT.get(kernel_name)
+    traffic = traffic * el * ssp_frac if traffic is not None else None
+    roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak if achieved else None, "traffic": traffic, "peak_source": f"of {peak_kind}",
                 "algorithmic_bytes_per_launch_set": per_family_bytes[dom],
                 "per_family_ms_per_step": {k: round(v[0] / prof_steps, 4) for k, v in fam.items()},
                 "note": "second pass of the same steps with per-launch CUDA events on the launching stream"}
@@ -361,6 +372,7 @@ def run_ours(args):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": synth.WORKLOADS[args.workload]["name"], "matrices": [list(s) for s in shapes],
                        "r": r, "N": N, "refresh_period": tau, "mode": args.mode,
+                       "launch_plan": [{k: p[k] for k in ("single_pass", "WC", "CS", "KC", "active_clusters")} for p in plans],
                        "l2": "inputs (%.2f GB of G per step, 2 alternating sets) exceed L2" % (g_bytes / 1e9),
                        "parallelism": "replicas" if world > 1 else "single"},
             "north_star_frac": alg_bytes / ms_step / 1e6 / peak,
@@ -396,7 +408,7 @@ def run_ours(args):
     torch.cuda.empty_cache()
 
     if rank == 0 and world == 1 and not args.no_sweep:
-        line["sweep_config5"] = sweep_config5(torch, device, peak)
+        line["sweep_config5"] = sweep_config5(torch, device, peak, args.mode)
     if rank == 0 and world == 1 and not args.no_cpu:
         line["cpu_baseline"] = cpu_baseline(args.workload if args.workload != 4 else 4, r, N)
     if rank == 0:

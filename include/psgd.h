@@ -66,6 +66,8 @@ typedef enum {
                                       psgd_materialize_error produces the true residual) */
 #define PSGD_OPT_REFRESH_ITERS 3   /* subspace iterations q of the refresh (default 20) */
 #define PSGD_OPT_REFRESH_OVERSAMPLE 4 /* extra columns of the refresh block (default max(8, r)) */
+#define PSGD_OPT_REFRESH_TC 5      /* 1 (default): the early sweeps of a refresh whose block has >= 32 columns run
+                                      on the tensor cores in TF32, the last 8 in float32; 0: float32 throughout */
 
 /* buffers that psgd_debug_ptr exposes (test use only; valid until the next step) */
 #define PSGD_BUF_P_NODE 1   /* P^(i)   [count][N][m][r] */
@@ -182,6 +184,21 @@ const char* psgd_last_cuda_error(const psgd_handle* h);
 
 /* Frees host memory of the handle.  Never touches caller-owned device buffers. */
 psgd_status psgd_destroy(psgd_handle* h);
+
+/*
+ * The tensor-core contraction the refresh uses for its early subspace sweeps (SVD-Comp of
+ * Algorithm 1 computed by block subspace iteration; Definition 3 fixes what it converges to):
+ *     C[c] = A[c] B[c]^T,   A [count][M][K],  B [count][Nc][K],  C [count][M][Nc],
+ * all DEVICE, float32, row-major.  Operands are read as TF32 (the 13 low mantissa bits are
+ * ignored), products are accumulated in float32.  Requires Nc <= 256, K % 4 == 0, A and B
+ * 16-byte aligned.  `scratch` (DEVICE, 256-byte aligned) must hold the bytes that
+ * psgd_gemm_nt_tf32_scratch reports; its first word is used as a status word.  Synchronises the
+ * stream before returning; PSGD_E_STATE means a bounded wait inside the kernel ran out.
+ */
+psgd_status psgd_gemm_nt_tf32_scratch(int64_t M, int64_t Nc, int64_t K, int count, size_t* scratch_bytes /*HOST*/);
+psgd_status psgd_gemm_nt_tf32(const float* A /*DEVICE*/, const float* B /*DEVICE*/, float* C /*DEVICE*/, int64_t M,
+                              int64_t Nc, int64_t K, int count, void* scratch /*DEVICE*/, size_t scratch_bytes,
+                              psgd_stream stream);
 
 /*
  * Back-projection without a workspace.  (An addition of this library: the paper has no

@@ -102,6 +102,23 @@ def svd_top_r(W, r):
 
 
 # --------------------------------------------------------------------------
+# Product with TF32 operands: what the tensor-core sweeps of the refresh compute
+# for one contraction of the subspace iteration (any basis of the subspace is a
+# valid SVD-Comp result, so the sweeps themselves need no oracle; this function
+# defines the single product so that the kernel can be checked in isolation).
+# --------------------------------------------------------------------------
+def tf32_truncate(X):
+    """float32 values with the 13 low mantissa bits cleared (TF32: 1 + 8 + 10 bits), as float64."""
+    bits = np.ascontiguousarray(X, dtype=np.float32).view(np.uint32) & np.uint32(0xFFFFE000)
+    return bits.view(np.float32).astype(F64)
+
+
+def gemm_nt_tf32(A, B):
+    """C = A B^T with both operands truncated to TF32 and exact (double) accumulation."""
+    return tf32_truncate(A) @ tf32_truncate(B).T
+
+
+# --------------------------------------------------------------------------
 # Algorithm 1, both compressors.  Delta has shape [N, m, n].
 # --------------------------------------------------------------------------
 def ssp_comp(Q, Delta):

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 PSGD_W_RANK_DEFICIENT = 1
 PSGD_W_NOT_CONVERGED = 2
 PSGD_W_TIMEOUT = 4
-PSGD_OPT_ERROR_FORM, PSGD_OPT_MODE, PSGD_OPT_REFRESH_ITERS, PSGD_OPT_REFRESH_OVERSAMPLE = 1, 2, 3, 4
+PSGD_OPT_ERROR_FORM, PSGD_OPT_MODE, PSGD_OPT_REFRESH_ITERS, PSGD_OPT_REFRESH_OVERSAMPLE, PSGD_OPT_REFRESH_TC = 1, 2, 3, 4, 5
 PSGD_BUF = {"P_node": 1, "Q_node": 2, "P_hat": 3, "Dbar": 4, "P_mean": 5}
 KERNEL_FAMILIES = ["project", "orth", "backproject", "residual", "refresh", "misc"]
 
@@ -40,6 +40,8 @@ SIGNATURES = {
     "psgd_profile_read": (_int, [_vp, C.POINTER(C.c_float), C.POINTER(_int)]),
     "psgd_last_cuda_error": (C.c_char_p, [_vp]),
     "psgd_destroy": (_int, [_vp]),
+    "psgd_gemm_nt_tf32_scratch": (_int, [_i64, _i64, _i64, _int, C.POINTER(_sz)]),
+    "psgd_gemm_nt_tf32": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _int, _vp, _sz, _vp]),
     "psgd_backproject_static": (_int, [_vp, _vp, _vp, _vp, _i64, _i64, _int, _int, _vp]),
 }
 
@@ -86,7 +88,7 @@ class PowerSGDPlus:
     """
 
     def __init__(self, m, n, r, N, refresh_period=0, seed=0, count=1, device="cuda:0", error_form="local",
-                 mode="eager", refresh_iters=None, oversample=None, reset=True):
+                 mode="eager", refresh_iters=None, oversample=None, reset=True, refresh_tc=None):
         import torch
 
         self.torch = torch
@@ -104,6 +106,8 @@ class PowerSGDPlus:
             _check(L.psgd_set_option(h, PSGD_OPT_REFRESH_ITERS, refresh_iters))
         if oversample is not None:
             _check(L.psgd_set_option(h, PSGD_OPT_REFRESH_OVERSAMPLE, oversample))
+        if refresh_tc is not None:
+            _check(L.psgd_set_option(h, PSGD_OPT_REFRESH_TC, int(bool(refresh_tc))))
         eb, qb, wb = _sz(), _sz(), _sz()
         _check(L.psgd_sizes(h, C.byref(eb), C.byref(qb), C.byref(wb)))
         with torch.cuda.device(self.device):
@@ -219,6 +223,29 @@ class PowerSGDPlus:
             self.close()
         except Exception:
             pass
+
+
+def gemm_nt_tf32(A, B, stream=None):
+    """C[c] = A[c] @ B[c].T on the tensor cores (TF32 operands, float32 accumulation).
+
+    A [count,M,K], B [count,Nc,K]: contiguous float32 CUDA tensors.  Returns C [count,M,Nc].
+    """
+    import torch
+
+    count, M, K = A.shape
+    Nc = B.shape[1]
+    for t in (A, B):
+        if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+            raise PSGDError("tensors must be contiguous float32 CUDA tensors")
+    nb = _sz()
+    _check(lib().psgd_gemm_nt_tf32_scratch(M, Nc, K, count, C.byref(nb)))
+    s = stream if stream is not None else torch.cuda.current_stream(A.device)
+    with torch.cuda.device(A.device):
+        scratch = torch.empty((nb.value,), dtype=torch.uint8, device=A.device)
+        out = torch.empty((count, M, Nc), dtype=torch.float32, device=A.device)
+        _check(lib().psgd_gemm_nt_tf32(A.data_ptr(), B.data_ptr(), out.data_ptr(), M, Nc, K, count,
+                                       scratch.data_ptr(), nb.value, _vp(s.cuda_stream)))
+    return out
 
 
 def backproject_static(M, P_hat, Q_mean, Q_node=None, stream=None):

@@ -14,6 +14,7 @@
 
 #include "psgd_kernels.cuh"
 #include "psgd_fused.cuh"
+#include "psgd_gemm_tc.cuh"
 
 using namespace psgd;
 
@@ -28,6 +29,7 @@ inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 struct Layout {
     size_t flags, Pnode, Pmean, Phat, Qnode, part, gram, T, dbar, Y, Z, V, U, total;
     size_t Qpad, Ppad, Qsub, Tacc, Pout, Wpart, Cmat, Cpart;  // deferred (single-pass) mode only
+    size_t dbarT, Yt, Zt, gpart;                              // tensor-core refresh only
 };
 
 struct ProfEvent {
@@ -41,7 +43,9 @@ struct psgd_handle {
     int64_t m, n;
     int r, N, count, tau;
     uint64_t seed;
-    int error_form = 0, mode = 0, refresh_iters = 20, oversample = -1;
+    int error_form = 0, mode = 0, refresh_iters = 20, oversample = -1, refresh_tc = 1;
+    bool tc_ok = false;           // the refresh block is wide enough for the tensor-core sweeps
+    size_t gpart_floats = 0;
     int64_t t = 0;
     float* E = nullptr;
     float* Q = nullptr;
@@ -66,6 +70,16 @@ struct psgd_handle {
 };
 
 namespace {
+
+// K splits of the tensor-core product with M rows and K columns: enough CTAs for about two per SM,
+// at least 8 K-blocks of 32 each
+int gemm_tc_splits(int64_t M, int64_t K, int count) {
+    int64_t tiles = ((M + TC_BM - 1) / TC_BM) * count;
+    int64_t KB = (K + TC_BK - 1) / TC_BK;
+    int64_t S = std::max<int64_t>(1, std::min<int64_t>((2 * 148 + tiles - 1) / tiles, std::max<int64_t>(1, KB / 8)));
+    int64_t kbps = (KB + S - 1) / S;
+    return (int)((KB + kbps - 1) / kbps);
+}
 
 int refresh_width(const psgd_handle* h) {
     int over = h->oversample >= 0 ? h->oversample : std::max(8, h->r);
@@ -109,6 +123,18 @@ void plan(psgd_handle* h) {
     size_t c2 = (c + 1) & ~(size_t)1;
     L.V = take(cnt * c2 * c2 * 8);
     L.U = take(cnt * ell * r * 8);
+    // ---- tensor-core sweeps of the refresh: block of >= 32 columns, 16-byte row strides for TMA ----
+    h->tc_ok = h->refresh_tc && ell >= 32 && ell <= TC_MAXN && h->n % 4 == 0 && h->m % 4 == 0;
+    if (h->tc_ok) {
+        const size_t ncp = align_up(ell, 16);
+        L.dbarT = take(cnt * m * n * 4);
+        L.Yt = take(cnt * ell * m * 4);
+        L.Zt = take(cnt * ell * n * 4);
+        size_t g1 = gemm_tc_splits(h->m, h->n, h->count) * cnt * m * ncp;
+        size_t g2 = gemm_tc_splits(h->n, h->m, h->count) * cnt * n * ncp;
+        h->gpart_floats = std::max(g1, g2);
+        L.gpart = take(h->gpart_floats * 4);
+    }
     // ---- single-pass mode ----
     // A CTA owns WC in {128, 256, 512} columns of every node; the tile of S it keeps on chip and the
     // registers of its back-projection bound N * WC by 2048.  CS = ceil(n / WC) CTAs form a cluster.
@@ -194,6 +220,63 @@ void allow_smem(K kernel, size_t bytes) {
 
 inline bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
 
+// ---- TMA tensor maps ----------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+// Rank-3 map over [count*N][m][n] float32 with tiles of `rows` rows x bw columns of one node; out-of-range reads give zeros.
+bool make_tile_map(CUtensorMap* map, const float* base, int64_t n, int64_t m, int64_t mats, int bw, int rows,
+                   CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_NONE) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)n, (cuuint64_t)m, (cuuint64_t)mats};
+    cuuint64_t strides[2] = {(cuuint64_t)n * 4, (cuuint64_t)m * (cuuint64_t)n * 4};
+    cuuint32_t box[3] = {(cuuint32_t)bw, (cuuint32_t)rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+
+// C = A B^T on the tensor cores: A [count][M][K], B [count][Nc][K] (both K-major), C [count][M][Nc].
+void launch_gemm_tc(Launcher& L, psgd_handle* h, const float* A, const float* B, float* C, int M, int Nc, int K, int kind) {
+    const int cnt = h->count;
+    const int Ncp = (int)align_up(Nc, 16);
+    const int KB = ceil_div(K, TC_BK);
+    const int S = gemm_tc_splits(M, K, cnt);
+    const int kbps = ceil_div(KB, S);
+    float* Cpart = (float*)(h->ws + h->lay.gpart);
+    if ((size_t)cnt * S * M * Ncp > h->gpart_floats) { L.status = PSGD_E_WORKSPACE; return; }
+    CUtensorMap tmA, tmB;
+    if (!make_tile_map(&tmA, A, K, M, cnt, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tile_map(&tmB, B, K, Nc, cnt, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B)) {
+        snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
+        L.status = PSGD_E_CUDA;
+        return;
+    }
+    GemmTcArgs g{Cpart, M, Ncp, K, S, kbps, (int*)(h->ws + h->lay.flags)};
+    size_t smem = gemm_tc_smem_bytes(Ncp);
+    cudaFuncSetAttribute(k_gemm_tf32, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    L.begin(kind);
+    k_gemm_tf32<<<dim3(ceil_div(M, TC_BM), S, cnt), TC_THREADS, smem, L.st>>>(tmA, tmB, g);
+    L.end();
+    size_t tot = (size_t)cnt * M * Nc;
+    L.begin(kind);
+    k_gemm_reduce<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Cpart, C, M, Nc, Ncp, S, cnt);
+    L.end();
+}
+
 // ---- K1 dispatch ------------------------------------------------------------
 template <int RP, int VEC, bool ADD, bool STORE>
 void launch_project_t(Launcher& L, const ProjectArgs& a, int count) {
@@ -266,7 +349,7 @@ void launch_resid(Launcher& L, const float* M, float* Out, const float* Phat, co
 }
 
 // ---- K2: X <- orthonormal factor of X (rows x c), in place or into Xout ------
-void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int rows, int c, int kind) {
+void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int rows, int c, int kind, float* XoutT = nullptr) {
     char* ws = h->ws;
     double* gram = (double*)(ws + h->lay.gram);
     double* T = (double*)(ws + h->lay.T);
@@ -282,7 +365,7 @@ void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int r
     L.begin(kind);
     k_chol<<<h->count, 256, smem, L.st>>>(gram, T, c, nparts, flags);
     L.end();
-    ApplyArgs ap{X, T, Xout, rows, c, c, c, 1};
+    ApplyArgs ap{X, T, Xout, rows, c, c, c, 1, XoutT};
     L.begin(kind);
     k_apply<<<dim3(ceil_div(rows, 32), h->count), 256, (size_t)32 * c * 4, L.st>>>(ap);
     L.end();
@@ -352,7 +435,25 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
     L.begin(K);
     k_fill_normal<<<(unsigned)((zt + 255) / 256), 256, 0, L.st>>>(Z, zt, h->seed, 0x5eed0000ull + (uint64_t)h->t);
     L.end();
-    launch_orth(L, h, Z, Z, n, ell, K);
+    // Early sweeps on the tensor cores (TF32 operands): they bring the block close to the subspace, the
+    // float32 sweeps that follow remove the TF32 rounding.  Needs Dbar^T and transposed copies of the blocks.
+    int it0 = 0;
+    const bool tc = h->tc_ok && aligned16(dbar) && h->refresh_iters > 8;
+    float* dbarT = tc ? (float*)(ws + h->lay.dbarT) : nullptr;
+    float* Yt = tc ? (float*)(ws + h->lay.Yt) : nullptr;
+    float* Zt = tc ? (float*)(ws + h->lay.Zt) : nullptr;
+    launch_orth(L, h, Z, Z, n, ell, K, Zt);
+    if (tc) {
+        L.begin(K);
+        k_transpose<<<dim3(ceil_div(n, 32), ceil_div(m, 32), cnt), dim3(32, 8), 0, L.st>>>(dbar, dbarT, m, n);
+        L.end();
+        for (; it0 < h->refresh_iters - 8; ++it0) {
+            launch_gemm_tc(L, h, dbar, Zt, Y, m, ell, n, K);       // Y = Dbar Z
+            launch_orth(L, h, Y, Y, m, ell, K, Yt);
+            launch_gemm_tc(L, h, dbarT, Yt, Z, n, ell, m, K);      // Z = Dbar^T Y
+            launch_orth(L, h, Z, Z, n, ell, K, Zt);
+        }
+    }
     // chunking of Z = Dbar^T Y over rows
     int colblk = ceil_div(n, BP_COLS);
     int64_t base = (int64_t)cnt * colblk * ceil_div(ell, 16);
@@ -360,7 +461,7 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
     S = std::min(S, std::min(64, ceil_div(m, BP_SUB)));
     int rpc = (int)align_up(ceil_div(m, S), BP_SUB);
     S = ceil_div(m, rpc);
-    for (int it = 0; it < h->refresh_iters; ++it) {
+    for (int it = it0; it < h->refresh_iters; ++it) {
         // Y = Dbar Z, orthonormalise;  Z = Dbar^T Y, orthonormalise
         launch_project(L, dbar, nullptr, nullptr, Z, Y, m, n, ell, 1, cnt, h->vec4);
         launch_orth(L, h, Y, Y, m, ell, K);
@@ -384,7 +485,7 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
     L.begin(K);
     k_jacobi_top<<<cnt, JAC_THREADS, smem, L.st>>>(gram, nparts, ell, r, V, U, flags);
     L.end();
-    ApplyArgs ap{Y, U, Phat, m, ell, r, r, 0};
+    ApplyArgs ap{Y, U, Phat, m, ell, r, r, 0, nullptr};
     L.begin(K);
     k_apply<<<dim3(ceil_div(m, 32), cnt), 256, (size_t)32 * ell * 4, L.st>>>(ap);
     L.end();
@@ -392,32 +493,6 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
 }
 
 // ---- single-pass SSP-Comp step (deferred residual) --------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qr;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
-            qr == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-    }
-    return fn;
-}
-// Rank-3 map over [count*N][m][n] float32 with tiles of `rows` rows x bw columns of one node; out-of-range reads give zeros.
-bool make_tile_map(CUtensorMap* map, const float* base, int64_t n, int64_t m, int64_t mats, int bw, int rows) {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)n, (cuuint64_t)m, (cuuint64_t)mats};
-    cuuint64_t strides[2] = {(cuuint64_t)n * 4, (cuuint64_t)m * (cuuint64_t)n * 4};
-    cuuint32_t box[3] = {(cuuint32_t)bw, (cuuint32_t)rows, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int RP, int WC>
 void launch_fused_t(Launcher& L, psgd_handle* h, const float* G, FusedArgs a) {
     void (*kern)(CUtensorMap, CUtensorMap, FusedArgs) = h->pending ? k_fused_step<RP, WC, true> : k_fused_step<RP, WC, false>;
@@ -605,6 +680,7 @@ psgd_status psgd_set_option(psgd_handle* h, int option, int value) {
         case PSGD_OPT_MODE: if (value != 0 && value != 1) return PSGD_E_INVALID; h->mode = value; break;
         case PSGD_OPT_REFRESH_ITERS: if (value < 1 || value > 64) return PSGD_E_INVALID; h->refresh_iters = value; break;
         case PSGD_OPT_REFRESH_OVERSAMPLE: if (value < 0 || value > MAX_L) return PSGD_E_INVALID; h->oversample = value; break;
+        case PSGD_OPT_REFRESH_TC: if (value != 0 && value != 1) return PSGD_E_INVALID; h->refresh_tc = value; break;
         default: return PSGD_E_INVALID;
     }
     plan(h);
@@ -771,6 +847,50 @@ psgd_status psgd_destroy(psgd_handle* h) {
     for (auto& ev : h->events) { cudaEventDestroy(ev.a); cudaEventDestroy(ev.b); }
     delete h;
     return PSGD_OK;
+}
+
+}  // extern "C"
+
+extern "C" {
+
+psgd_status psgd_gemm_nt_tf32_scratch(int64_t M, int64_t Nc, int64_t K, int count, size_t* scratch_bytes) {
+    if (!scratch_bytes) return PSGD_E_NULL;
+    if (!(M >= 1 && Nc >= 1 && Nc <= TC_MAXN && K >= 4 && K % 4 == 0 && count >= 1 && count <= 65535)) return PSGD_E_INVALID;
+    *scratch_bytes = (size_t)gemm_tc_splits(M, K, count) * count * M * align_up(Nc, 16) * 4 + 256;
+    return PSGD_OK;
+}
+
+psgd_status psgd_gemm_nt_tf32(const float* A, const float* B, float* C, int64_t M, int64_t Nc, int64_t K, int count,
+                              void* scratch, size_t scratch_bytes, psgd_stream stream) {
+    size_t need = 0;
+    psgd_status st = psgd_gemm_nt_tf32_scratch(M, Nc, K, count, &need);
+    if (st != PSGD_OK) return st;
+    if (!A || !B || !C || !scratch) return PSGD_E_NULL;
+    if (scratch_bytes < need) return PSGD_E_WORKSPACE;
+    if (!aligned16(A) || !aligned16(B) || ((uintptr_t)scratch & 255)) return PSGD_E_INVALID;
+    cudaStream_t cs = (cudaStream_t)stream;
+    const int Ncp = (int)align_up(Nc, 16);
+    const int KB = ceil_div(K, TC_BK);
+    const int S = gemm_tc_splits(M, K, count);
+    const int kbps = ceil_div(KB, S);
+    int* flags = (int*)scratch;                       // first 256 bytes: status word
+    float* Cpart = (float*)((char*)scratch + 256);
+    CUtensorMap tmA, tmB;
+    if (!make_tile_map(&tmA, A, K, M, count, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tile_map(&tmB, B, K, Nc, count, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B))
+        return PSGD_E_CUDA;
+    if (cudaMemsetAsync(flags, 0, 4, cs) != cudaSuccess) return PSGD_E_CUDA;
+    GemmTcArgs g{Cpart, (int)M, Ncp, (int)K, S, kbps, flags};
+    size_t smem = gemm_tc_smem_bytes(Ncp);
+    cudaFuncSetAttribute(k_gemm_tf32, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    k_gemm_tf32<<<dim3(ceil_div(M, TC_BM), S, count), TC_THREADS, smem, cs>>>(tmA, tmB, g);
+    size_t tot = (size_t)count * M * Nc;
+    k_gemm_reduce<<<(unsigned)((tot + 255) / 256), 256, 0, cs>>>(Cpart, C, (int)M, (int)Nc, Ncp, S, count);
+    if (cudaGetLastError() != cudaSuccess) return PSGD_E_CUDA;
+    int hflags = 0;
+    if (cudaMemcpyAsync(&hflags, flags, 4, cudaMemcpyDeviceToHost, cs) != cudaSuccess || cudaStreamSynchronize(cs) != cudaSuccess)
+        return PSGD_E_CUDA;
+    return hflags ? PSGD_E_STATE : PSGD_OK;
 }
 
 }  // extern "C"

@@ -1,0 +1,194 @@
+// Tensor-core contraction for the refresh (SVD-Comp of Algorithm 1, computed as a block
+// subspace iteration):  C = A B^T  with A [M][K] and B [Nc][K] both row-major float32, i.e. both
+// operands K-major.  The two products of one iteration have this form,
+//     Y = Dbar Z      (A = Dbar  [m][n],  B = Z^T [l][n]),
+//     Z = Dbar^T Y    (A = Dbar^T [n][m], B = Y^T [l][m]),
+// once a transposed copy of the node mean Dbar is kept.
+//
+// sm_100 path: TMA loads 128-byte-swizzled tiles (128 x 32 floats of A, Ncp x 32 of B) into a
+// 4-stage shared-memory ring; one thread issues tcgen05.mma (kind::tf32, M = 128, N = Ncp,
+// K = 8 per instruction) with the accumulator in tensor memory; four warps read the
+// accumulator back with tcgen05.ld and store it.  Inputs are read as TF32 (the low 13 mantissa
+// bits of the float32 operands are ignored), which is why the refresh only runs its early
+// sweeps here and finishes with float32 sweeps.  K is split over blockIdx.y; the partial
+// products are summed in a fixed order by k_gemm_reduce.
+// Every wait is bounded: a wait that runs out sets PSGD_W_TIMEOUT and the kernel carries on,
+// frees its tensor memory and returns.
+#pragma once
+#include <cuda.h>
+
+#include "psgd_fused.cuh"
+
+namespace psgd {
+
+constexpr int TC_BM = 128;       // rows of A per CTA (= UMMA M)
+constexpr int TC_BK = 32;        // floats of K per stage (= one 128-byte swizzle row)
+constexpr int TC_STAGES = 4;
+constexpr int TC_THREADS = 192;  // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-5: epilogue
+constexpr int TC_MAXN = 256;
+
+struct GemmTcArgs {
+    float* Cpart;     // [count][S][M][Ncp]
+    int M, Ncp, K, S, kb_per_split;
+    int* flags;
+};
+
+__host__ __device__ inline size_t gemm_tc_smem_bytes(int Ncp) {
+    return (size_t)TC_STAGES * ((size_t)TC_BM * TC_BK * 4 + (size_t)Ncp * TC_BK * 4) + 1024 /*alignment*/ + 128 /*barriers, tmem address*/;
+}
+
+// shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzled:
+// 8-row groups 1024 bytes apart (stride offset), leading offset unused (1), descriptor version 1.
+__device__ __forceinline__ unsigned long long tc_smem_desc(unsigned addr) {
+    unsigned long long d = 0;
+    d |= (unsigned long long)((addr >> 4) & 0x3FFF);
+    d |= (unsigned long long)1 << 16;
+    d |= (unsigned long long)(1024 >> 4) << 32;
+    d |= (unsigned long long)1 << 46;
+    d |= (unsigned long long)2 << 61;    // SWIZZLE_128B
+    return d;
+}
+// instruction descriptor: D = F32, A = B = TF32, both K-major, N and M encoded as N/8 and M/16
+__device__ __forceinline__ unsigned tc_idesc(int n) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(TC_BM >> 4) << 24);
+}
+__device__ __forceinline__ void tma_load_3d_sw(unsigned dst, const CUtensorMap* map, int x, int y, int z, unsigned bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+k_gemm_tf32(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmTcArgs a) {
+    extern __shared__ __align__(16) unsigned char tc_smem_raw[];
+    unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned a_bytes = TC_BM * TC_BK * 4, b_bytes = (unsigned)a.Ncp * TC_BK * 4;
+    const unsigned stage_bytes = a_bytes + b_bytes;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(base + (size_t)TC_STAGES * stage_bytes);
+    const unsigned bar_full = smem_u32(bars), bar_empty = bar_full + 8 * TC_STAGES, bar_acc = bar_empty + 8 * TC_STAGES;
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 2 * TC_STAGES + 1);
+    const unsigned smem_base = smem_u32(base);
+
+    const int mt = blockIdx.x, sp = blockIdx.y, c = blockIdx.z;
+    const int KB = (a.K + TC_BK - 1) / TC_BK;
+    const int kb0 = sp * a.kb_per_split;
+    const int nkb = max(0, min(KB, kb0 + a.kb_per_split) - kb0);
+    unsigned ncols = 32;                       // tensor-memory columns: power of two >= Ncp
+    while ((int)ncols < a.Ncp) ncols <<= 1;
+
+    if (tid == 0) {
+        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        mbar_init(bar_acc, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(ncols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    const unsigned tmem = *tmem_slot;
+    bool dead = false;
+
+    if (warp == 0) {
+        // ---- TMA producer ----
+        if (lane == 0) {
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % TC_STAGES;
+                if (kb >= TC_STAGES) mbar_wait(bar_empty + 8 * s, (unsigned)((kb / TC_STAGES - 1) & 1), a.flags, dead);
+                const unsigned dst = smem_base + s * stage_bytes;
+                mbar_expect_tx(bar_full + 8 * s, stage_bytes);
+                tma_load_3d_sw(dst, &tmA, (kb0 + kb) * TC_BK, mt * TC_BM, c, bar_full + 8 * s);
+                tma_load_3d_sw(dst + a_bytes, &tmB, (kb0 + kb) * TC_BK, 0, c, bar_full + 8 * s);
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer ----
+        if (lane == 0) {
+            const unsigned idesc = tc_idesc(a.Ncp);
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % TC_STAGES;
+                mbar_wait(bar_full + 8 * s, (unsigned)((kb / TC_STAGES) & 1), a.flags, dead);
+                asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                const unsigned long long da = tc_smem_desc(smem_base + s * stage_bytes);
+                const unsigned long long db = tc_smem_desc(smem_base + s * stage_bytes + a_bytes);
+#pragma unroll
+                for (int k = 0; k < TC_BK / 8; ++k) {
+                    const unsigned acc = (kb > 0 || k > 0) ? 1u : 0u;
+                    // 8 floats of K = 32 bytes further along the swizzled row: start address field + 2
+                    asm volatile(
+                        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+                        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
+                        ::"r"(tmem), "l"(da + (unsigned long long)(2 * k)), "l"(db + (unsigned long long)(2 * k)), "r"(idesc), "r"(acc) : "memory");
+                }
+                // the stage may be refilled once these MMAs have read it
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_empty + 8 * s) : "memory");
+            }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_acc) : "memory");
+        }
+    } else {
+        // ---- epilogue: tensor memory -> registers -> Cpart ----
+        mbar_wait(bar_acc, 0u, a.flags, dead);
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        const int quarter = warp & 3;                    // the tensor-memory lanes this warp may read
+        const int row = mt * TC_BM + quarter * 32 + lane;
+        float* out = a.Cpart + (((size_t)c * a.S + sp) * a.M + row) * a.Ncp;
+        for (int col = 0; col < a.Ncp; col += 8) {
+            unsigned r[8];
+            const unsigned taddr = tmem + ((unsigned)(quarter * 32) << 16) + (unsigned)col;
+            if (nkb > 0) {
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
+                             : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                             : "r"(taddr) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) r[j] = 0u;
+            }
+            if (row < a.M) {
+                *reinterpret_cast<uint4*>(out + col) = make_uint4(r[0], r[1], r[2], r[3]);
+                *reinterpret_cast<uint4*>(out + col + 4) = make_uint4(r[4], r[5], r[6], r[7]);
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(ncols) : "memory");
+    }
+}
+
+// C[c][row][col] = sum_s Cpart[c][s][row][col], col < Nc  (fixed order).  One thread per output.
+__global__ void k_gemm_reduce(const float* Cpart, float* C, int M, int Nc, int Ncp, int S, int count) {
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t per = (size_t)M * Nc;
+    if (idx >= per * count) return;
+    int c = (int)(idx / per);
+    size_t e = idx % per;
+    int row = (int)(e / Nc), col = (int)(e % Nc);
+    float s = 0.f;
+    for (int k = 0; k < S; ++k) s += Cpart[(((size_t)c * S + k) * M + row) * Ncp + col];
+    C[idx] = s;
+}
+
+// Out[c][j][i] = In[c][i][j]  (rows x cols -> cols x rows), 32 x 32 tiles through shared memory.
+__global__ void k_transpose(const float* In, float* Out, int rows, int cols) {
+    __shared__ float t[32][33];
+    const float* ib = In + (size_t)blockIdx.z * rows * cols;
+    float* ob = Out + (size_t)blockIdx.z * rows * cols;
+    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+        int r = r0 + j, cidx = c0 + threadIdx.x;
+        t[j][threadIdx.x] = (r < rows && cidx < cols) ? ib[(size_t)r * cols + cidx] : 0.f;
+    }
+    __syncthreads();
+    for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+        int cidx = c0 + j, r = r0 + threadIdx.x;
+        if (cidx < cols && r < rows) ob[(size_t)cidx * rows + r] = t[threadIdx.x][j];
+    }
+}
+
+}  // namespace psgd

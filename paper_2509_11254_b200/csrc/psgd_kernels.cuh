@@ -638,6 +638,7 @@ struct ApplyArgs {
     const double* T;  // [count][c][ldt]
     float* Xout;      // [count][rows][kout]
     int rows, c, kout, ldt, upper;
+    float* XoutT;     // optional transposed copy [count][kout][rows]
 };
 __global__ void __launch_bounds__(256) k_apply(ApplyArgs a) {
     extern __shared__ __align__(16) float xs[];  // [32][c]
@@ -655,7 +656,10 @@ __global__ void __launch_bounds__(256) k_apply(ApplyArgs a) {
         int jend = a.upper ? min(a.c, k + 1) : a.c;
         double s = 0.0;
         for (int j = 0; j < jend; ++j) s = fma((double)xs[rr * a.c + j], __ldg(Tb + (size_t)j * a.ldt + k), s);
-        if (row0 + rr < a.rows) Ob[(size_t)(row0 + rr) * a.kout + k] = (float)s;
+        if (row0 + rr < a.rows) {
+            Ob[(size_t)(row0 + rr) * a.kout + k] = (float)s;
+            if (a.XoutT) a.XoutT[((size_t)blockIdx.y * a.kout + k) * a.rows + row0 + rr] = (float)s;
+        }
     }
 }
 

@@ -21,7 +21,7 @@ def test_every_declared_symbol_is_exported(L):
     from paper_2509_11254_b200 import binding
 
     header = open(os.path.join(ROOT, "include", "psgd.h")).read()
-    declared = set(re.findall(r"\b(psgd_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(psgd_[a-z0-9_]+)\s*\(", header))
     declared -= {"psgd_status", "psgd_handle", "psgd_stream"}
     assert declared, "no declarations found"
     for name in sorted(declared):

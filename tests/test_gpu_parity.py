@@ -164,6 +164,17 @@ def test_refresh_schedule(torch_cuda, m, n, r, N, workload):
     run_case(torch_cuda, m, n, r, N, tau=3, steps=5, workload=workload)
 
 
+@pytest.mark.parametrize("m,n,r,N,workload", [
+    (1000, 520, 32, 2, 5),     # block of 64 columns: tensor-core sweeps, ragged row tile, K tail
+    (768, 768, 24, 3, 2),      # block of 48 columns (padded to 48 = 3 x 16)
+    (1536, 1024, 64, 2, 5),    # block of 128 columns, several K splits
+    (900, 644, 100, 2, 5),     # block of 160 columns (widest), K not a multiple of 32
+])
+def test_refresh_tensor_core_sweeps(torch_cuda, m, n, r, N, workload):
+    """SVD-Comp whose early subspace sweeps run as TF32 tcgen05 products, finished in float32."""
+    run_case(torch_cuda, m, n, r, N, tau=2, steps=3, workload=workload)
+
+
 def test_refresh_every_step(torch_cuda):
     run_case(torch_cuda, 256, 128, 4, 4, tau=1, steps=3, workload=1)
 
@@ -276,3 +287,32 @@ def test_deferred_free_running(torch_cuda, m, n, r, N, workload, tau):
     e1 = comp.E.clone()
     comp.materialize_error()
     assert torch.equal(e1, comp.E)
+
+
+# ---- the tensor-core contraction of the refresh, in isolation ------------------------------
+@pytest.mark.parametrize("M,Nc,K,count", [
+    (128, 16, 32, 1),        # one tile, one K block, one MMA group
+    (300, 48, 520, 2),       # ragged rows, K tail (520 = 16 * 32 + 8), batch of 2
+    (1000, 64, 4096, 1),     # several K splits
+    (129, 160, 100, 1),      # widest block, K smaller than four stages
+    (4096, 128, 16384, 1),   # config-5 back-projection shape of the refresh (Z = Dbar^T Y)
+])
+def test_gemm_nt_tf32_matches_definition(torch_cuda, M, Nc, K, count):
+    """C = A B^T with TF32 operands: element-wise against the definition evaluated in double.
+
+    The products of TF32 operands are exact in float32; what remains is the float32 accumulation
+    over K terms, far below 1e-5 of |a_row| |b_row|, while a dropped or misplaced K block would
+    show up at 1e-2.
+    """
+    from paper_2509_11254_b200 import binding
+
+    torch = torch_cuda
+    rng = np.random.default_rng(M + Nc + K)
+    A = rng.standard_normal((count, M, K)).astype(np.float32)
+    B = rng.standard_normal((count, Nc, K)).astype(np.float32)
+    C = binding.gemm_nt_tf32(torch.as_tensor(A, device="cuda:0"), torch.as_tensor(B, device="cuda:0")).cpu().numpy()
+    for c in range(count):
+        ref = orc.gemm_nt_tf32(A[c], B[c])
+        scale = np.linalg.norm(orc.tf32_truncate(A[c]), axis=1)[:, None] * np.linalg.norm(orc.tf32_truncate(B[c]), axis=1)[None, :]
+        err = np.abs(C[c] - ref) / scale
+        assert err.max() <= 1e-5, f"max scaled error {err.max()}"
