@@ -360,7 +360,7 @@ void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int r
     L.begin(kind);
     k_gram<<<dim3(nparts, nblk * nblk, h->count), 256, 0, L.st>>>(g);
     L.end();
-    size_t smem = (size_t)c * c * 8;
+    size_t smem = (size_t)c * chol_ld(c) * 8;
     allow_smem(k_chol, smem);
     L.begin(kind);
     k_chol<<<h->count, 256, smem, L.st>>>(gram, T, c, nparts, flags);
@@ -480,7 +480,7 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
     k_gram<<<dim3(nparts, nblk * nblk, cnt), 256, 0, L.st>>>(g);
     L.end();
     int c2 = (ell + 1) & ~1;
-    size_t smem = (size_t)c2 * c2 * 8;
+    size_t smem = (size_t)c2 * jac_ld(c2) * 8;
     allow_smem(k_jacobi_top, smem);
     L.begin(K);
     k_jacobi_top<<<cnt, JAC_THREADS, smem, L.st>>>(gram, nparts, ell, r, V, U, flags);
@@ -583,7 +583,7 @@ void fused_ssp(Launcher& L, psgd_handle* h, const float* G) {
     if (L.status != PSGD_OK) return;
     // P'^T P' = L L^T  ->  T'; scaled pivot^2 < 2e-2 (rounding of W T amplified > 7x) raises the gate for the precise path
     L.begin(PSGD_K_ORTH);
-    k_chol<<<cnt, 256, (size_t)r * r * 8, L.st>>>(gram, T, r, h->KC, flags, gate, 2e-2);
+    k_chol<<<cnt, 256, (size_t)r * chol_ld(r) * 8, L.st>>>(gram, T, r, h->KC, flags, gate, 2e-2);
     L.end();
     FinishPArgs fp{Pout, T, Phat, Ppad, Tacc, Tacc, m, r, RP, h->tacc_identity ? 1 : 0};
     L.begin(PSGD_K_ORTH);

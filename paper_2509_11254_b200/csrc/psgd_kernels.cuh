@@ -552,80 +552,83 @@ __global__ void __launch_bounds__(256) k_gram(GramArgs a) {
 
 // Sum the Gram partials, scale to unit diagonal, Cholesky, invert, and write
 // T = D^-1 L^-T (upper triangular, double) so that P~ = P T.  One CTA per matrix.
-// Dynamic shared memory: c*c doubles.
+// Dynamic shared memory: c * chol_ld(c) doubles (rows padded to an odd number of doubles so that
+// walking down a column is free of bank conflicts).
 constexpr double CHOL_PIVOT_TOL = 1e-11;  // squared sine of the angle to the previous columns
+__host__ __device__ inline int chol_ld(int c) { return c | 1; }
 // `gate` (optional): set to 1 when a scaled pivot^2 falls below gate_tol, i.e. when the columns
 // are too ill-conditioned for results derived from W = M^T P to keep float32 accuracy.
 __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int c, int nparts, int* flags,
                                               int* gate = nullptr, double gate_tol = 0.0) {
-    extern __shared__ __align__(16) double Gs[];  // [c][c]
+    extern __shared__ __align__(16) double Gs[];  // [c][ld]
     __shared__ double dinv[192];
     __shared__ int bad, illc;
     const int tid = threadIdx.x;
-    const int nblk = (c + 63) / 64;
+    const int ld = chol_ld(c);
     const double* pb = part + (size_t)blockIdx.x * nparts * c * c;
     if (tid == 0) { bad = 0; illc = 0; }
     for (int e = tid; e < c * c; e += 256) {
         int i = e / c, j = e % c;
         int ii = i, jj = j;
         if (i / 64 > j / 64) { ii = j; jj = i; }   // lower block triangle was not computed: mirror
-        (void)nblk;
         double s = 0.0;
         for (int p = 0; p < nparts; ++p) s += pb[(size_t)p * c * c + (size_t)ii * c + jj];
-        Gs[e] = s;
+        Gs[i * ld + j] = s;
     }
     __syncthreads();
     for (int k = tid; k < c; k += 256) {
-        double d = Gs[k * c + k];
+        double d = Gs[k * ld + k];
         if (!(d > 0.0)) { dinv[k] = 0.0; bad = 1; } else dinv[k] = 1.0 / sqrt(d);
     }
     __syncthreads();
     for (int e = tid; e < c * c; e += 256) {
         int i = e / c, j = e % c;
-        double v = Gs[e] * dinv[i] * dinv[j];
+        double v = Gs[i * ld + j] * dinv[i] * dinv[j];
         if (i == j && dinv[i] == 0.0) v = 1.0;  // zero column: decouple it (fixed up later)
-        Gs[e] = v;
+        Gs[i * ld + j] = v;
     }
     __syncthreads();
     // right-looking Cholesky on the lower triangle: Gs = L L^T
     for (int k = 0; k < c; ++k) {
         if (tid == 0) {
-            double p = Gs[k * c + k];
+            double p = Gs[k * ld + k];
             if (!(p > gate_tol)) illc = 1;
-            if (!(p > CHOL_PIVOT_TOL)) { bad = 1; p = 1.0; for (int i = k + 1; i < c; ++i) Gs[i * c + k] = 0.0; }
-            Gs[k * c + k] = sqrt(p);
+            if (!(p > CHOL_PIVOT_TOL)) { bad = 1; p = 1.0; for (int i = k + 1; i < c; ++i) Gs[i * ld + k] = 0.0; }
+            Gs[k * ld + k] = sqrt(p);
         }
         __syncthreads();
-        double lkk = Gs[k * c + k];
-        for (int i = k + 1 + tid; i < c; i += 256) Gs[i * c + k] /= lkk;
+        double lkk = Gs[k * ld + k];
+        for (int i = k + 1 + tid; i < c; i += 256) Gs[i * ld + k] /= lkk;
         __syncthreads();
-        int rem = c - k - 1;
-        for (int e = tid; e < rem * rem; e += 256) {
-            int i = k + 1 + e / rem, j = k + 1 + e % rem;
-            if (j <= i) Gs[i * c + j] -= Gs[i * c + k] * Gs[j * c + k];
+        // trailing update, one row per warp pass: lanes walk along the row
+        const int rem = c - k - 1;
+        for (int ri = (tid >> 5); ri < rem; ri += 8) {
+            const int i = k + 1 + ri;
+            const double lik = Gs[i * ld + k];
+            for (int j = k + 1 + (tid & 31); j <= i; j += 32) Gs[i * ld + j] -= lik * Gs[j * ld + k];
         }
         __syncthreads();
     }
     // in-place inverse of the lower-triangular L, row by row
     for (int i = 0; i < c; ++i) {
-        double lii = Gs[i * c + i];
+        double lii = Gs[i * ld + i];
         double val = 0.0;
         int j = tid;  // c <= 192 <= 256: one column per thread
         if (j < i) {
             double s = 0.0;
-            for (int k = j; k < i; ++k) s += Gs[i * c + k] * Gs[k * c + j];
+            for (int k = j; k < i; ++k) s += Gs[i * ld + k] * Gs[k * ld + j];
             val = -s / lii;
         }
         __syncthreads();
-        if (j < i) Gs[i * c + j] = val;
-        if (j == i) Gs[i * c + i] = 1.0 / lii;
+        if (j < i) Gs[i * ld + j] = val;
+        if (j == i) Gs[i * ld + i] = 1.0 / lii;
         __syncthreads();
     }
     // T[j][k] = dinv[j] * Linv[k][j]  for j <= k
     double* Tb = T + (size_t)blockIdx.x * c * c;
     for (int e = tid; e < c * c; e += 256) {
         int j = e / c, k = e % c;
-        Tb[e] = (j <= k) ? dinv[j] * Gs[k * c + j] : 0.0;
+        Tb[e] = (j <= k) ? dinv[j] * Gs[k * ld + j] : 0.0;
     }
     if (tid == 0 && bad) atomicOr(flags, 1);
     if (tid == 0 && illc && gate) atomicOr(gate, 1);
@@ -672,17 +675,20 @@ __global__ void __launch_bounds__(256) k_apply(ApplyArgs a) {
 // ----------------------------------------------------------------------------
 constexpr int JAC_THREADS = 512;
 constexpr int JAC_MAX_SWEEPS = 40;
+// leading dimension of the shared-memory matrix: odd number of doubles (no bank conflicts down a column)
+__host__ __device__ inline int jac_ld(int c2) { return c2 | 1; }
 __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, int nparts, int c, int r,
                                                             double* Vws, double* U, int* flags) {
-    extern __shared__ __align__(16) double As[];  // [c2][c2]
+    extern __shared__ __align__(16) double As[];  // [c2][ld]
     __shared__ double cs[128], sn[128];
     __shared__ int pp[128], qq[128];
     __shared__ double offn, diagn;
     __shared__ int order[192];
     const int tid = threadIdx.x;
     const int c2 = (c + 1) & ~1;
+    const int ld = jac_ld(c2);
     const int np = c2 / 2;
-    double* V = Vws + (size_t)blockIdx.x * c2 * c2;
+    double* Vt = Vws + (size_t)blockIdx.x * c2 * c2;   // eigenvector matrix, stored transposed: Vt[p][i] = V[i][p]
     const double* pb = part + (size_t)blockIdx.x * nparts * c * c;
     for (int e = tid; e < c2 * c2; e += JAC_THREADS) {
         int i = e / c2, j = e % c2;
@@ -692,14 +698,14 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
             if (i / 64 > j / 64) { ii = j; jj = i; }
             for (int p = 0; p < nparts; ++p) s += pb[(size_t)p * c * c + (size_t)ii * c + jj];
         }
-        As[e] = s;
-        V[e] = (i == j) ? 1.0 : 0.0;
+        As[i * ld + j] = s;
+        Vt[e] = (i == j) ? 1.0 : 0.0;
     }
     __syncthreads();
     // symmetrise (the two triangles of a diagonal block were accumulated separately)
     for (int e = tid; e < c2 * c2; e += JAC_THREADS) {
         int i = e / c2, j = e % c2;
-        if (i < j) { double v = 0.5 * (As[i * c2 + j] + As[j * c2 + i]); As[i * c2 + j] = v; As[j * c2 + i] = v; }
+        if (i < j) { double v = 0.5 * (As[i * ld + j] + As[j * ld + i]); As[i * ld + j] = v; As[j * ld + i] = v; }
     }
     __syncthreads();
     int converged = 0;
@@ -711,7 +717,7 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
                 int b0 = 1 + (c2 - 2 - tid + round) % (c2 - 1);
                 int p = min(a0, b0), q = max(a0, b0);
                 pp[tid] = p; qq[tid] = q;
-                double apq = As[p * c2 + q], app = As[p * c2 + p], aqq = As[q * c2 + q];
+                double apq = As[p * ld + q], app = As[p * ld + p], aqq = As[q * ld + q];
                 double cc = 1.0, ss = 0.0;
                 if (fabs(apq) > 1e-300 && fabs(apq) > 1e-18 * sqrt(fabs(app * aqq))) {
                     double tau = (aqq - app) / (2.0 * apq);
@@ -722,17 +728,17 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
                 cs[tid] = cc; sn[tid] = ss;
             }
             __syncthreads();
-            // columns: A <- A J, V <- V J
+            // columns: A <- A J, V <- V J   (thread index runs down the column)
             for (int e = tid; e < np * c2; e += JAC_THREADS) {
                 int k = e / c2, i = e % c2;
                 int p = pp[k], q = qq[k];
                 double cc = cs[k], ss = sn[k];
-                double aip = As[i * c2 + p], aiq = As[i * c2 + q];
-                As[i * c2 + p] = cc * aip - ss * aiq;
-                As[i * c2 + q] = ss * aip + cc * aiq;
-                double vip = V[i * c2 + p], viq = V[i * c2 + q];
-                V[i * c2 + p] = cc * vip - ss * viq;
-                V[i * c2 + q] = ss * vip + cc * viq;
+                double aip = As[i * ld + p], aiq = As[i * ld + q];
+                As[i * ld + p] = cc * aip - ss * aiq;
+                As[i * ld + q] = ss * aip + cc * aiq;
+                double vip = Vt[p * c2 + i], viq = Vt[q * c2 + i];
+                Vt[p * c2 + i] = cc * vip - ss * viq;
+                Vt[q * c2 + i] = ss * vip + cc * viq;
             }
             __syncthreads();
             // rows: A <- J^T A
@@ -740,25 +746,25 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
                 int k = e / c2, j = e % c2;
                 int p = pp[k], q = qq[k];
                 double cc = cs[k], ss = sn[k];
-                double apj = As[p * c2 + j], aqj = As[q * c2 + j];
-                As[p * c2 + j] = cc * apj - ss * aqj;
-                As[q * c2 + j] = ss * apj + cc * aqj;
+                double apj = As[p * ld + j], aqj = As[q * ld + j];
+                As[p * ld + j] = cc * apj - ss * aqj;
+                As[q * ld + j] = ss * apj + cc * aqj;
             }
             __syncthreads();
         }
         if (tid == 0) { offn = 0.0; diagn = 0.0; }
         __syncthreads();
-        double lo = 0.0, ld = 0.0;
+        double lo = 0.0, ldg = 0.0;
         for (int e = tid; e < c2 * c2; e += JAC_THREADS) {
             int i = e / c2, j = e % c2;
-            double v = As[e];
-            if (i == j) ld += v * v; else lo += v * v;
+            double v = As[i * ld + j];
+            if (i == j) ldg += v * v; else lo += v * v;
         }
         for (int o = 16; o > 0; o >>= 1) {
             lo += __shfl_xor_sync(0xffffffffu, lo, o);
-            ld += __shfl_xor_sync(0xffffffffu, ld, o);
+            ldg += __shfl_xor_sync(0xffffffffu, ldg, o);
         }
-        if ((tid & 31) == 0) { atomicAdd(&offn, lo); atomicAdd(&diagn, ld); }
+        if ((tid & 31) == 0) { atomicAdd(&offn, lo); atomicAdd(&diagn, ldg); }
         __syncthreads();
         converged = (offn <= 1e-30 * diagn) || (diagn == 0.0);
         __syncthreads();
@@ -766,10 +772,10 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
     if (tid == 0 && !converged) atomicOr(flags, 2);
     // rank the eigenvalues (descending; ties by index) and emit the top r eigenvectors
     for (int i = tid; i < c2; i += JAC_THREADS) {
-        double li = (i < c) ? As[i * c2 + i] : -1e300;
+        double li = (i < c) ? As[i * ld + i] : -1e300;
         int rank = 0;
         for (int j = 0; j < c2; ++j) {
-            double lj = (j < c) ? As[j * c2 + j] : -1e300;
+            double lj = (j < c) ? As[j * ld + j] : -1e300;
             if (lj > li || (lj == li && j < i)) ++rank;
         }
         order[rank] = i;
@@ -778,7 +784,7 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
     double* Ub = U + (size_t)blockIdx.x * c * r;
     for (int e = tid; e < c * r; e += JAC_THREADS) {
         int i = e / r, k = e % r;
-        Ub[e] = V[i * c2 + order[k]];
+        Ub[e] = Vt[order[k] * c2 + i];
     }
 }
 
