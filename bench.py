@@ -50,6 +50,7 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-refresh", action="store_true", help="tau = 0 (plain PowerSGD steps only)")
+    ap.add_argument("--refresh-period", type=int, default=None, help="override the workload's refresh period tau")
     return ap.parse_args()
 
 
@@ -298,6 +299,8 @@ def run_ours(args):
 
     r, N, tau = DEFAULTS[args.workload]
     r = args.rank or r
+    if args.refresh_period is not None:
+        tau = args.refresh_period
     if args.no_refresh:
         tau = 0
     shapes = stack_for(args.workload)

@@ -360,10 +360,16 @@ void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int r
     L.begin(kind);
     k_gram<<<dim3(nparts, nblk * nblk, h->count), 256, 0, L.st>>>(g);
     L.end();
+    if (nparts > 4) {   // fold the partials in parallel first; k_chol then reads partial 0 with the original stride
+        size_t tot = (size_t)c * c * h->count;
+        L.begin(kind);
+        k_gram_sum<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(gram, c * c, nparts, h->count);
+        L.end();
+    }
     size_t smem = (size_t)c * chol_ld(c) * 8;
     allow_smem(k_chol, smem);
     L.begin(kind);
-    k_chol<<<h->count, 256, smem, L.st>>>(gram, T, c, nparts, flags);
+    k_chol<<<h->count, 256, smem, L.st>>>(gram, T, c, nparts > 4 ? -nparts : nparts, flags);
     L.end();
     ApplyArgs ap{X, T, Xout, rows, c, c, c, 1, XoutT};
     L.begin(kind);
@@ -483,7 +489,13 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
     size_t smem = (size_t)c2 * jac_ld(c2) * 8;
     allow_smem(k_jacobi_top, smem);
     L.begin(K);
-    k_jacobi_top<<<cnt, JAC_THREADS, smem, L.st>>>(gram, nparts, ell, r, V, U, flags);
+    if (nparts > 4) {
+        size_t tot = (size_t)ell * ell * cnt;
+        L.begin(K);
+        k_gram_sum<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(gram, ell * ell, nparts, cnt);
+        L.end();
+    }
+    k_jacobi_top<<<cnt, JAC_THREADS, smem, L.st>>>(gram, nparts > 4 ? -nparts : nparts, ell, r, V, U, flags);
     L.end();
     ApplyArgs ap{Y, U, Phat, m, ell, r, r, 0, nullptr};
     L.begin(K);

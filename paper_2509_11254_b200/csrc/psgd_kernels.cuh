@@ -550,6 +550,18 @@ __global__ void __launch_bounds__(256) k_gram(GramArgs a) {
         }
 }
 
+// part[c][0][e] <- sum_p part[c][p][e]  (fixed order), so that the single-CTA kernels below read one
+// matrix instead of streaming every partial through one SM.  One thread per entry.
+__global__ void k_gram_sum(double* part, int cc, int nparts, int count) {
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)cc * count) return;
+    size_t c = idx / cc, e = idx % cc;
+    double* pb = part + c * (size_t)nparts * cc;
+    double s = 0.0;
+    for (int p = 0; p < nparts; ++p) s += pb[(size_t)p * cc + e];
+    pb[e] = s;
+}
+
 // Sum the Gram partials, scale to unit diagonal, Cholesky, invert, and write
 // T = D^-1 L^-T (upper triangular, double) so that P~ = P T.  One CTA per matrix.
 // Dynamic shared memory: c * chol_ld(c) doubles (rows padded to an odd number of doubles so that
@@ -565,7 +577,10 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
     __shared__ int bad, illc;
     const int tid = threadIdx.x;
     const int ld = chol_ld(c);
-    const double* pb = part + (size_t)blockIdx.x * nparts * c * c;
+    // nparts < 0: the partials were already folded into partial 0 (k_gram_sum); matrices stay |nparts| partials apart
+    const int pstride = nparts < 0 ? -nparts : nparts;
+    if (nparts < 0) nparts = 1;
+    const double* pb = part + (size_t)blockIdx.x * pstride * c * c;
     if (tid == 0) { bad = 0; illc = 0; }
     for (int e = tid; e < c * c; e += 256) {
         int i = e / c, j = e % c;
@@ -689,7 +704,9 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
     const int ld = jac_ld(c2);
     const int np = c2 / 2;
     double* Vt = Vws + (size_t)blockIdx.x * c2 * c2;   // eigenvector matrix, stored transposed: Vt[p][i] = V[i][p]
-    const double* pb = part + (size_t)blockIdx.x * nparts * c * c;
+    const int pstride = nparts < 0 ? -nparts : nparts;   // nparts < 0: partials already folded into partial 0
+    if (nparts < 0) nparts = 1;
+    const double* pb = part + (size_t)blockIdx.x * pstride * c * c;
     for (int e = tid; e < c2 * c2; e += JAC_THREADS) {
         int i = e / c2, j = e % c2;
         double s = 0.0;
