@@ -279,21 +279,16 @@ def sweep_config5(torch, device, peak, mode):
 
 def run_ours(args):
     import torch
-    import torch.distributed as dist
 
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2509_11254_b200.replicas import Replicas, env_rank
+
+    rank, local, world = env_rank()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
     torch.cuda.set_device(local)
     device = f"cuda:{local}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(device))
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
+    reps = Replicas("nccl", device)
+    barrier = reps.barrier
 
     from paper_2509_11254_b200 import synth
 
@@ -324,12 +319,9 @@ def run_ours(args):
     ms_total = timed_steps(torch, handles, bufs, args.steps, barrier)
     l1 = sum(h.launch_count() for h in handles)
     clocks = sampler.stop()
-    if world > 1:
-        t = torch.tensor([ms_total], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = reps.max_over_ranks(ms_total)
     ms_step = ms_total / args.steps
-    value = world * g_bytes / ms_step / 1e6  # GB/s of gradient, all replicas
+    value = reps.job_throughput(g_bytes, ms_step) / 1e9  # GB/s of gradient, all replicas
 
     # second pass over the same number of steps with per-launch CUDA events (roofline of the dominant kernel)
     for h in handles:
@@ -416,8 +408,7 @@ def run_ours(args):
         line["cpu_baseline"] = cpu_baseline(args.workload if args.workload != 4 else 4, r, N)
     if rank == 0:
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    reps.close()
 
 
 def main():

@@ -316,3 +316,66 @@ def test_gemm_nt_tf32_matches_definition(torch_cuda, M, Nc, K, count):
         scale = np.linalg.norm(orc.tf32_truncate(A[c]), axis=1)[:, None] * np.linalg.norm(orc.tf32_truncate(B[c]), axis=1)[None, :]
         err = np.abs(C[c] - ref) / scale
         assert err.max() <= 1e-5, f"max scaled error {err.max()}"
+
+
+# ---- full-size workloads in the benchmark's launch configuration, checked on sampled matrices ----
+def _full_size_case(torch, workload, m, n, r, N, count, tau, sample, free_steps):
+    """Deferred mode as bench.py runs it: free-running steps against the oracle on the sampled
+    matrices (rotation-invariant outputs, 1e-3), then one more step from identical state (1e-5)."""
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    dev = "cuda:0"
+    comp = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=3, count=count, device=dev, mode="deferred")
+    Q0 = comp.Q.cpu().numpy()
+    oracles = {c: orc.PowerSGDPlusOracle(m, n, r, N, tau, Q0[c]) for c in sample}
+    out = {}
+    for t in range(free_steps):
+        G = synth.make_gradients_torch(workload, m, n, N, count, step=t, device=dev)
+        comp.step(G)
+        for c in sample:
+            out[c] = oracles[c].step(G[c].cpu().numpy())
+        del G
+    comp.materialize_error()
+    assert comp.last_status() == 0
+    for c in sample:
+        normM = np.linalg.norm(out[c]["M"])
+        assert projector_distance(comp.P_hat[c].cpu().numpy(), out[c]["P_hat"]) <= 1e-3, f"matrix {c}: projector"
+        assert rel_fro(comp.E[c].cpu().numpy(), out[c]["E"], floor=1e-2 * normM) <= 1e-3, f"matrix {c}: residual"
+    # one step from identical state: the oracle continues from the GPU's float32 state
+    t = free_steps
+    for c in sample:
+        oracles[c].E = comp.E[c].cpu().numpy().astype(np.float64)
+        oracles[c].Q = comp.Q[c].cpu().numpy().astype(np.float64)
+        oracles[c].t = t
+    G = synth.make_gradients_torch(workload, m, n, N, count, step=t, device=dev)
+    comp.step(G)
+    comp.materialize_error()
+    assert comp.last_status() == 0
+    Qn = comp.debug("Q_node")
+    for c in sample:
+        o = oracles[c].step(G[c].cpu().numpy())
+        gp = dict(P_hat=comp.P_hat[c].cpu().numpy(), Q=comp.Q[c].cpu().numpy(), E=comp.E[c].cpu().numpy(),
+                  Q_node=Qn[c].cpu().numpy())
+        compare_step(o, gp, m, n, r, N, f"full size, matrix {c}")
+    plan = comp.plan_info()
+    comp.close()
+    return plan
+
+
+def test_full_size_config2_attention_class(torch_cuda):
+    """BASELINE config 2, the 48 matrices of 768 x 768 (r = 8, N = 8, refresh at t = 0), three sampled."""
+    plan = _full_size_case(torch_cuda, 2, 768, 768, 8, 8, 48, tau=50, sample=(0, 17, 47), free_steps=4)
+    assert plan["single_pass"] == 1 and plan["CS"] == 3 and plan["WC"] == 256
+
+
+def test_full_size_config2_ffn_class(torch_cuda):
+    """BASELINE config 2, the 36 matrices of 2048 x 768, two sampled."""
+    plan = _full_size_case(torch_cuda, 2, 2048, 768, 8, 8, 36, tau=50, sample=(5, 35), free_steps=3)
+    assert plan["single_pass"] == 1
+
+
+@pytest.mark.parametrize("r", [4, 8])
+def test_full_size_config5(torch_cuda, r):
+    """BASELINE config 5: one 16384 x 4096 matrix on 4 nodes, plain PowerSGD steps (the step the sweep times)."""
+    plan = _full_size_case(torch_cuda, 5, 16384, 4096, r, 4, 1, tau=0, sample=(0,), free_steps=3)
+    assert plan["single_pass"] == 1 and plan["CS"] == 8 and plan["WC"] == 512
