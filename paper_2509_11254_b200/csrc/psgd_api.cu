@@ -30,6 +30,7 @@ struct Layout {
     size_t flags, Pnode, Pmean, Phat, Qnode, part, gram, T, dbar, Y, Z, V, U, total;
     size_t Qpad, Ppad, Qsub, Tacc, Pout, Wpart, Cmat, Cpart;  // deferred (single-pass) mode only
     size_t dbarT, Yt, Zt, gpart;                              // tensor-core refresh only
+    size_t rtP, rtQ;                                          // tensor-core residual (r > 16) only
 };
 
 struct ProfEvent {
@@ -46,6 +47,8 @@ struct psgd_handle {
     int error_form = 0, mode = 0, refresh_iters = 20, oversample = -1, refresh_tc = 1;
     bool tc_ok = false;           // the refresh block is wide enough for the tensor-core sweeps
     size_t gpart_floats = 0;
+    bool rtc_ok = false;          // ranks above 16 with 16-byte row strides: residual update on the tensor cores
+    int rtc_KP = 0;
     int64_t t = 0;
     float* E = nullptr;
     float* Q = nullptr;
@@ -134,6 +137,14 @@ void plan(psgd_handle* h) {
         size_t g2 = gemm_tc_splits(h->n, h->m, h->count) * cnt * n * ncp;
         h->gpart_floats = std::max(g1, g2);
         L.gpart = take(h->gpart_floats * 4);
+    }
+    // ---- residual update on the tensor cores: split (head + tail) padded copies of P~ and Q_i ----
+    h->rtc_ok = h->r > 16 && h->n % 4 == 0;
+    if (h->rtc_ok) {
+        h->rtc_KP = (int)align_up(r, TC_BK);
+        const size_t KP = h->rtc_KP;
+        L.rtP = take(3 * cnt * m * KP * 4);       // the three TF32 terms of P~, padded to KP columns
+        L.rtQ = take(3 * cnt * N * n * KP * 4);   // the same for Q_i
     }
     // ---- single-pass mode ----
     // A CTA owns WC in {128, 256, 512} columns of every node; the tile of S it keeps on chip and the
@@ -334,8 +345,43 @@ void launch_back(Launcher& L, const float* M, const float* Phat, float* part, in
 }
 
 // ---- K4 dispatch ------------------------------------------------------------
+// Tensor-core form for ranks above 16 (exactly split TF32 rank-r product in tensor memory, see psgd_gemm_tc.cuh).
+bool launch_resid_tc(Launcher& L, const float* M, float* Out, const float* Phat, const float* Qf, int rows, int n, int r,
+                     int nodes, int mats, int q_per_node, int out_per_node) {
+    psgd_handle* h = L.h;
+    if (!h->rtc_ok || !aligned16(Out) || (M && !aligned16(M))) return false;
+    const int KP = h->rtc_KP, cnt = h->count;
+    const int qmats = q_per_node ? mats : cnt;
+    const size_t tp = (size_t)cnt * rows * KP, tq = (size_t)qmats * n * KP;
+    float* Pt[3] = {(float*)(h->ws + h->lay.rtP), (float*)(h->ws + h->lay.rtP) + tp, (float*)(h->ws + h->lay.rtP) + 2 * tp};
+    float* Qt[3] = {(float*)(h->ws + h->lay.rtQ), (float*)(h->ws + h->lay.rtQ) + tq, (float*)(h->ws + h->lay.rtQ) + 2 * tq};
+    L.begin(PSGD_K_RESIDUAL);
+    k_split_pad<<<(unsigned)((tp + 255) / 256), 256, 0, L.st>>>(Phat, Pt[0], Pt[1], Pt[2], (size_t)cnt * rows, r, KP);
+    L.end();
+    L.begin(PSGD_K_RESIDUAL);
+    k_split_pad<<<(unsigned)((tq + 255) / 256), 256, 0, L.st>>>(Qf, Qt[0], Qt[1], Qt[2], (size_t)qmats * n, r, KP);
+    L.end();
+    CUtensorMap tP[3], tQ[3];
+    for (int t = 0; t < 3; ++t) {
+        if (!make_tile_map(&tP[t], Pt[t], KP, rows, cnt, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tile_map(&tQ[t], Qt[t], KP, n, qmats, TC_BK, RT_BN, CU_TENSOR_MAP_SWIZZLE_128B)) {
+            snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
+            L.status = PSGD_E_CUDA;
+            return true;
+        }
+    }
+    ResidTcArgs a{M, Out, rows, n, KP, out_per_node ? nodes : 1, q_per_node, (int*)(h->ws + h->lay.flags)};
+    size_t smem = resid_tc_smem_bytes();
+    cudaFuncSetAttribute(k_residual_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    L.begin(PSGD_K_RESIDUAL);
+    k_residual_tc<<<dim3(ceil_div(rows, TC_BM), mats), RT_THREADS, smem, L.st>>>(tP[0], tP[1], tP[2], tQ[0], tQ[1], tQ[2], a);
+    L.end();
+    return true;
+}
+
 void launch_resid(Launcher& L, const float* M, float* Out, const float* Phat, const float* Qf, int rows, int n, int r,
                   int nodes, int mats, int q_per_node, int out_per_node, bool vec) {
+    if (r > 16 && launch_resid_tc(L, M, Out, Phat, Qf, rows, n, r, nodes, mats, q_per_node, out_per_node)) return;
     int rpc = 128;
     while (rpc > RS_SUB && (int64_t)mats * ceil_div(n, RS_COLS) * ceil_div(rows, rpc) < 4 * 148) rpc /= 2;
     ResidArgs a{M, Out, Phat, Qf, rows, n, r, nodes, rpc, q_per_node, out_per_node};

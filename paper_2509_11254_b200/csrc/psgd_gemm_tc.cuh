@@ -192,3 +192,200 @@ __global__ void k_transpose(const float* In, float* Out, int rows, int cols) {
 }
 
 }  // namespace psgd
+
+namespace psgd {
+
+// ---------------------------------------------------------------------------------------------
+// Residual update on the tensor cores for ranks above 16:  E_i = M_i - P~ Q_i^T  (Algorithm 2, last
+// line; with M == nullptr the dense reconstruction P~ Q^T of Algorithm 1).  The rank-r product is a
+// 128 x 128 output tile with K = r, accumulated in tensor memory; float32 accuracy comes from
+// splitting both small factors exactly into three TF32 numbers (x = h + m + l, 11 + 11 + 2 mantissa
+// bits) and issuing the six products down to 2^-22 (l*h, h*l, m*m, m*h, h*m, h*h, small terms
+// first), so that what is dropped (m*l, l*m, l*l) is below 2^-33 relative.  The epilogue
+// warps read the accumulator back (tcgen05.ld), subtract it from M and store E.  Tensor memory
+// holds two accumulators, so the MMAs of the next column tile overlap the epilogue of this one.
+// ---------------------------------------------------------------------------------------------
+constexpr int RT_BN = 128;        // columns per output tile (= UMMA N)
+constexpr int RT_STAGES = 2;
+constexpr int RT_THREADS = 192;   // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-5: epilogue
+
+struct ResidTcArgs {
+    const float* M;     // [mats][rows][n] or nullptr
+    float* Out;         // [mats][rows][n] (may alias M)
+    int rows, n, KP;    // KP: rank padded to a multiple of 32
+    int nodes;          // matrices per P~ (node count), 1 when Out is per matrix only
+    int q_per_node;     // 1: Q indexed like Out (matrix, node); 0: by matrix only
+    int* flags;
+};
+
+__host__ __device__ inline size_t resid_tc_smem_bytes() {
+    return (size_t)RT_STAGES * (3 * TC_BM * TC_BK * 4 + 3 * RT_BN * TC_BK * 4) + 1024 + 256;
+}
+
+// X [rows][r] -> Xh, Xm, Xl [rows][KP], zero padded: x = h + m + l exactly, each term a TF32 number
+// (h: x with its 13 low mantissa bits cleared; m: the same of x - h; l: what is left, at most 2 bits).
+__global__ void k_split_pad(const float* X, float* Xh, float* Xm, float* Xl, size_t rows, int r, int KP) {
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= rows * KP) return;
+    size_t row = idx / KP;
+    int k = (int)(idx % KP);
+    float x = (k < r) ? X[row * r + k] : 0.f;
+    float h = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
+    float r1 = x - h;
+    float mm = __uint_as_float(__float_as_uint(r1) & 0xFFFFE000u);
+    Xh[idx] = h;
+    Xm[idx] = mm;
+    Xl[idx] = r1 - mm;
+}
+
+__global__ void __launch_bounds__(RT_THREADS, 1)
+k_residual_tc(const __grid_constant__ CUtensorMap tmPh, const __grid_constant__ CUtensorMap tmPm, const __grid_constant__ CUtensorMap tmPl,
+              const __grid_constant__ CUtensorMap tmQh, const __grid_constant__ CUtensorMap tmQm, const __grid_constant__ CUtensorMap tmQl,
+              ResidTcArgs a) {
+    extern __shared__ __align__(16) unsigned char rt_smem_raw[];
+    unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(rt_smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr unsigned A_BYTES = TC_BM * TC_BK * 4, B_BYTES = RT_BN * TC_BK * 4;
+    constexpr unsigned STAGE_BYTES = 3 * A_BYTES + 3 * B_BYTES;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(base + (size_t)RT_STAGES * STAGE_BYTES);
+    const unsigned bar_full = smem_u32(bars), bar_empty = bar_full + 8 * RT_STAGES;
+    const unsigned bar_accf = bar_empty + 8 * RT_STAGES, bar_acce = bar_accf + 16;   // accumulator full / free, 2 each
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 2 * RT_STAGES + 4);
+    const unsigned smem_base = smem_u32(base);
+
+    const int rt = blockIdx.x, mat = blockIdx.y;
+    const int c = mat / a.nodes;                    // matrix index of P~
+    const int qz = a.q_per_node ? mat : c;          // which Q
+    const int nct = (a.n + RT_BN - 1) / RT_BN;      // column tiles
+    const int nkc = a.KP / TC_BK;                   // K chunks per tile
+    const int total = nct * nkc;
+
+    if (tid == 0) {
+        for (int s = 0; s < RT_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(bar_accf + 8 * b, 1); mbar_init(bar_acce + 8 * b, 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(4u * RT_BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    const unsigned tmem = *tmem_slot;
+    bool dead = false;
+
+    if (warp == 0) {
+        // ---- TMA producer: per (column tile, K chunk) the heads and tails of both factors ----
+        if (lane == 0) {
+            for (int it = 0; it < total; ++it) {
+                const int s = it % RT_STAGES;
+                const int ct = it / nkc, kc = it % nkc;
+                if (it >= RT_STAGES) mbar_wait(bar_empty + 8 * s, (unsigned)((it / RT_STAGES - 1) & 1), a.flags, dead);
+                const unsigned dst = smem_base + s * STAGE_BYTES;
+                const unsigned bar = bar_full + 8 * s;
+                mbar_expect_tx(bar, STAGE_BYTES);
+                tma_load_3d_sw(dst, &tmPh, kc * TC_BK, rt * TC_BM, c, bar);
+                tma_load_3d_sw(dst + A_BYTES, &tmPm, kc * TC_BK, rt * TC_BM, c, bar);
+                tma_load_3d_sw(dst + 2 * A_BYTES, &tmPl, kc * TC_BK, rt * TC_BM, c, bar);
+                tma_load_3d_sw(dst + 3 * A_BYTES, &tmQh, kc * TC_BK, ct * RT_BN, qz, bar);
+                tma_load_3d_sw(dst + 3 * A_BYTES + B_BYTES, &tmQm, kc * TC_BK, ct * RT_BN, qz, bar);
+                tma_load_3d_sw(dst + 3 * A_BYTES + 2 * B_BYTES, &tmQl, kc * TC_BK, ct * RT_BN, qz, bar);
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer ----
+        if (lane == 0) {
+            const unsigned idesc = tc_idesc(RT_BN);
+            for (int it = 0; it < total; ++it) {
+                const int s = it % RT_STAGES;
+                const int ct = it / nkc, kc = it % nkc;
+                const int ab = ct & 1;                                   // accumulator buffer
+                if (kc == 0 && ct >= 2) mbar_wait(bar_acce + 8 * ab, (unsigned)(((ct >> 1) - 1) & 1), a.flags, dead);
+                mbar_wait(bar_full + 8 * s, (unsigned)((it / RT_STAGES) & 1), a.flags, dead);
+                asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                const unsigned sb = smem_base + s * STAGE_BYTES;
+                const unsigned long long dP[3] = {tc_smem_desc(sb), tc_smem_desc(sb + A_BYTES), tc_smem_desc(sb + 2 * A_BYTES)};
+                const unsigned long long dQ[3] = {tc_smem_desc(sb + 3 * A_BYTES), tc_smem_desc(sb + 3 * A_BYTES + B_BYTES),
+                                                  tc_smem_desc(sb + 3 * A_BYTES + 2 * B_BYTES)};
+                // two accumulators per tile: the h*h products (8 adds per 64 of K) and the five small products,
+                // so that the rounding of the tensor core's float32 adds hits the large running sum as rarely as possible
+                const unsigned d_big = tmem + (unsigned)(ab * 2 * RT_BN), d_small = d_big + RT_BN;
+                // (index of the P term, index of the Q term) with h = 0, m = 1, l = 2; small products first
+                const int tp[6] = {2, 0, 1, 1, 0, 0}, tq[6] = {0, 2, 1, 0, 1, 0};
+#pragma unroll
+                for (int k = 0; k < TC_BK / 8; ++k) {
+                    const unsigned long long o = (unsigned long long)(2 * k);
+#pragma unroll
+                    for (int t = 0; t < 6; ++t) {
+                        const unsigned acc = (kc > 0 || k > 0 || (t > 0 && t < 5)) ? 1u : 0u;
+                        asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
+                                     ::"r"(t == 5 ? d_big : d_small), "l"(dP[tp[t]] + o), "l"(dQ[tq[t]] + o), "r"(idesc), "r"(acc) : "memory");
+                    }
+                }
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_empty + 8 * s) : "memory");
+                if (kc == nkc - 1)
+                    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_accf + 8 * ab) : "memory");
+            }
+        }
+    } else {
+        // ---- epilogue: E = M - accumulator ----
+        const int quarter = warp & 3;
+        const int row = rt * TC_BM + quarter * 32 + lane;
+        const bool rok = row < a.rows;
+        const float* Mr = a.M ? a.M + ((size_t)mat * a.rows + (rok ? row : 0)) * a.n : nullptr;
+        float* Or = a.Out + ((size_t)mat * a.rows + (rok ? row : 0)) * a.n;
+        for (int ct = 0; ct < nct; ++ct) {
+            const int ab = ct & 1;
+            mbar_wait(bar_accf + 8 * ab, (unsigned)((ct >> 1) & 1), a.flags, dead);
+            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+#pragma unroll 1
+            for (int cc = 0; cc < RT_BN; cc += 32) {
+                const int col0 = ct * RT_BN + cc;
+                if (col0 >= a.n) break;
+                unsigned r[32], rs[32];
+                const unsigned taddr = tmem + ((unsigned)(quarter * 32) << 16) + (unsigned)(ab * 2 * RT_BN + cc);
+#define PSGD_TMEM_LD32(R, ADDR)                                                                                             \
+                asm volatile(                                                                                                  \
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "  \
+                    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"              \
+                    : "=r"(R[0]), "=r"(R[1]), "=r"(R[2]), "=r"(R[3]), "=r"(R[4]), "=r"(R[5]), "=r"(R[6]), "=r"(R[7]),          \
+                      "=r"(R[8]), "=r"(R[9]), "=r"(R[10]), "=r"(R[11]), "=r"(R[12]), "=r"(R[13]), "=r"(R[14]), "=r"(R[15]),    \
+                      "=r"(R[16]), "=r"(R[17]), "=r"(R[18]), "=r"(R[19]), "=r"(R[20]), "=r"(R[21]), "=r"(R[22]), "=r"(R[23]),  \
+                      "=r"(R[24]), "=r"(R[25]), "=r"(R[26]), "=r"(R[27]), "=r"(R[28]), "=r"(R[29]), "=r"(R[30]), "=r"(R[31])   \
+                    : "r"(ADDR) : "memory")
+                PSGD_TMEM_LD32(r, taddr);
+                PSGD_TMEM_LD32(rs, taddr + (unsigned)RT_BN);
+#undef PSGD_TMEM_LD32
+                asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(rs[j]));
+                if (rok) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        if (col0 + j < a.n) {      // n % 4 == 0: a group of 4 columns is all in or all out
+                            float4 mv = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (Mr) mv = ldg_stream4(Mr + col0 + j);
+                            float4 o;
+                            if (Mr) o = make_float4(mv.x - __uint_as_float(r[j]), mv.y - __uint_as_float(r[j + 1]),
+                                                    mv.z - __uint_as_float(r[j + 2]), mv.w - __uint_as_float(r[j + 3]));
+                            else o = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                            *reinterpret_cast<float4*>(Or + col0 + j) = o;
+                        }
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acce + 8 * ab);      // this warp is done with the accumulator buffer
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(4u * RT_BN) : "memory");
+    }
+}
+
+}  // namespace psgd

@@ -144,7 +144,17 @@ def test_ragged_shapes_ssp(torch_cuda, m, n, r, N, count):
 
 @pytest.mark.parametrize("r", [24, 32, 48, 64, 128])
 def test_large_rank_ssp(torch_cuda, r):
-    run_case(torch_cuda, 640, 256, r, 2, tau=0, steps=2, workload=5, Einit=0.01)
+    run_case(torch_cuda, 640, 256, r, 2, tau=0, steps=2, workload=5, Einit=0.01, check_dense=True)
+
+
+@pytest.mark.parametrize("m,n,r,N,count,form", [
+    (1000, 520, 20, 3, 2, "local"),     # rank padded 20 -> 32, ragged row tile, 3 column tiles with a ragged last one
+    (300, 260, 40, 2, 1, "mean"),       # node-averaged Q in the residual, rank padded 40 -> 64
+    (2048, 2048, 32, 2, 1, "local"),    # config-4 attention shape and rank
+])
+def test_residual_on_tensor_cores(torch_cuda, m, n, r, N, count, form):
+    """Ranks above 16: E = M - P~ Q_i^T as a split-TF32 tcgen05 product, against the oracle at 1e-5."""
+    run_case(torch_cuda, m, n, r, N, tau=0, steps=2, workload=4, count=count, Einit=0.01, error_form=form, check_dense=True)
 
 
 def test_mean_error_form(torch_cuda):
