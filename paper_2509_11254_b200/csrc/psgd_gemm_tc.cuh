@@ -207,7 +207,7 @@ namespace psgd {
 // ---------------------------------------------------------------------------------------------
 constexpr int RT_BN = 128;        // columns per output tile (= UMMA N)
 constexpr int RT_STAGES = 2;
-constexpr int RT_THREADS = 192;   // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-5: epilogue
+constexpr int RT_THREADS = 320;   // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-9: epilogue (two per lane quarter)
 
 struct ResidTcArgs {
     const float* M;     // [mats][rows][n] or nullptr
@@ -262,7 +262,7 @@ k_residual_tc(const __grid_constant__ CUtensorMap tmPh, const __grid_constant__ 
 
     if (tid == 0) {
         for (int s = 0; s < RT_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(bar_accf + 8 * b, 1); mbar_init(bar_acce + 8 * b, 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(bar_accf + 8 * b, 1); mbar_init(bar_acce + 8 * b, 8); }
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     if (warp == 1) {
@@ -330,17 +330,26 @@ k_residual_tc(const __grid_constant__ CUtensorMap tmPh, const __grid_constant__ 
         }
     } else {
         // ---- epilogue: E = M - accumulator ----
+        // Eight warps: warp w reads the tensor-memory lanes of quarter w % 4 (its accumulator rows) and the
+        // 32-column chunks of parity (w - 2) / 4.  The M values of a chunk are requested before the
+        // accumulator is read so that more loads are in flight.
         const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int row = rt * TC_BM + quarter * 32 + lane;
         const bool rok = row < a.rows;
         const float* Mr = a.M ? a.M + ((size_t)mat * a.rows + (rok ? row : 0)) * a.n : nullptr;
         float* Or = a.Out + ((size_t)mat * a.rows + (rok ? row : 0)) * a.n;
         for (int ct = 0; ct < nct; ++ct) {
             const int ab = ct & 1;
+            float4 mv[8];
+            const int cfirst = ct * RT_BN + half * 32;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                mv[j] = (Mr && rok && cfirst + 4 * j < a.n) ? ldg_stream4(Mr + cfirst + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
             mbar_wait(bar_accf + 8 * ab, (unsigned)((ct >> 1) & 1), a.flags, dead);
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
 #pragma unroll 1
-            for (int cc = 0; cc < RT_BN; cc += 32) {
+            for (int cc = half * 32; cc < RT_BN; cc += 64) {
                 const int col0 = ct * RT_BN + cc;
                 if (col0 >= a.n) break;
                 unsigned r[32], rs[32];
@@ -358,22 +367,31 @@ k_residual_tc(const __grid_constant__ CUtensorMap tmPh, const __grid_constant__ 
                 PSGD_TMEM_LD32(rs, taddr + (unsigned)RT_BN);
 #undef PSGD_TMEM_LD32
                 asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+                // request the next chunk's M values (the next chunk of this tile, else nothing: the next tile's
+                // first chunk is requested at the top of the tile loop)
+                float4 mn[8];
+                const int cnext = col0 + 64;
+                const bool more = cc + 64 < RT_BN;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(rs[j]));
+                for (int j = 0; j < 8; ++j)
+                    mn[j] = (more && Mr && rok && cnext + 4 * j < a.n) ? ldg_stream4(Mr + cnext + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
                 if (rok) {
 #pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
-                        if (col0 + j < a.n) {      // n % 4 == 0: a group of 4 columns is all in or all out
-                            float4 mv = make_float4(0.f, 0.f, 0.f, 0.f);
-                            if (Mr) mv = ldg_stream4(Mr + col0 + j);
+                    for (int j = 0; j < 8; ++j) {
+                        if (col0 + 4 * j < a.n) {      // n % 4 == 0: a group of 4 columns is all in or all out
+                            const float a0 = __uint_as_float(r[4 * j]) + __uint_as_float(rs[4 * j]);
+                            const float a1 = __uint_as_float(r[4 * j + 1]) + __uint_as_float(rs[4 * j + 1]);
+                            const float a2 = __uint_as_float(r[4 * j + 2]) + __uint_as_float(rs[4 * j + 2]);
+                            const float a3 = __uint_as_float(r[4 * j + 3]) + __uint_as_float(rs[4 * j + 3]);
                             float4 o;
-                            if (Mr) o = make_float4(mv.x - __uint_as_float(r[j]), mv.y - __uint_as_float(r[j + 1]),
-                                                    mv.z - __uint_as_float(r[j + 2]), mv.w - __uint_as_float(r[j + 3]));
-                            else o = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-                            *reinterpret_cast<float4*>(Or + col0 + j) = o;
+                            if (Mr) o = make_float4(mv[j].x - a0, mv[j].y - a1, mv[j].z - a2, mv[j].w - a3);
+                            else o = make_float4(a0, a1, a2, a3);
+                            *reinterpret_cast<float4*>(Or + col0 + 4 * j) = o;
                         }
                     }
                 }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) mv[j] = mn[j];
             }
             asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
             __syncwarp();
