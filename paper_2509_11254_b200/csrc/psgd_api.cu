@@ -27,7 +27,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 
 struct Layout {
-    size_t flags, Pnode, Pmean, Phat, Qnode, part, gram, T, dbar, Y, Z, V, U, total;
+    size_t flags, defic, Pnode, Pmean, Phat, Qnode, part, gram, T, dbar, Y, Z, V, U, total;
     size_t Qpad, Ppad, Qsub, Tacc, Pout, Wpart, Cmat, Cpart;  // deferred (single-pass) mode only
     size_t dbarT, Yt, Zt, gpart;                              // tensor-core refresh only
     size_t rtP, rtQ;                                          // tensor-core residual (r > 16) only
@@ -109,6 +109,7 @@ void plan(psgd_handle* h) {
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
     L.flags = take(256);
+    L.defic = take(cnt * 192 * 4);
     L.Pnode = take(cnt * N * m * r * 4);
     L.Pmean = take(cnt * m * r * 4);
     L.Phat = take(cnt * m * r * 4);
@@ -395,7 +396,8 @@ void launch_resid(Launcher& L, const float* M, float* Out, const float* Phat, co
 }
 
 // ---- K2: X <- orthonormal factor of X (rows x c), in place or into Xout ------
-void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int rows, int c, int kind, float* XoutT = nullptr) {
+void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int rows, int c, int kind, float* XoutT = nullptr,
+                 bool complete = false) {
     char* ws = h->ws;
     double* gram = (double*)(ws + h->lay.gram);
     double* T = (double*)(ws + h->lay.T);
@@ -415,12 +417,18 @@ void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int r
     size_t smem = (size_t)c * chol_ld(c) * 8;
     allow_smem(k_chol, smem);
     L.begin(kind);
-    k_chol<<<h->count, 256, smem, L.st>>>(gram, T, c, nparts > 4 ? -nparts : nparts, flags);
+    int* defic = (int*)(ws + h->lay.defic);
+    k_chol<<<h->count, 256, smem, L.st>>>(gram, T, c, nparts > 4 ? -nparts : nparts, flags, nullptr, 0.0, complete ? defic : nullptr);
     L.end();
     ApplyArgs ap{X, T, Xout, rows, c, c, c, 1, XoutT};
     L.begin(kind);
     k_apply<<<dim3(ceil_div(rows, 32), h->count), 256, (size_t)32 * c * 4, L.st>>>(ap);
     L.end();
+    if (complete) {   // rank-deficient P: replace the rejected columns by an orthonormal completion (no-op otherwise)
+        L.begin(kind);
+        k_complete<<<h->count, 256, 0, L.st>>>(Xout, nullptr, defic, flags, rows, c, 0, h->seed + (uint64_t)h->t);
+        L.end();
+    }
 }
 
 // ---- Algorithm 1, common tail: Q_i, Q, residual, optional dense reconstruction --
@@ -461,7 +469,7 @@ void ssp(Launcher& L, psgd_handle* h, const float* G) {
     L.begin(PSGD_K_ORTH);
     k_node_mean<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Pnode, Pmean, (size_t)m * r, N, cnt);
     L.end();
-    launch_orth(L, h, Pmean, Phat, m, r, PSGD_K_ORTH);
+    launch_orth(L, h, Pmean, Phat, m, r, PSGD_K_ORTH, nullptr, true);
 }
 
 // ---- SVD-Comp (Algorithm 1, second function): top-r left singular subspace of the
@@ -641,11 +649,15 @@ void fused_ssp(Launcher& L, psgd_handle* h, const float* G) {
     if (L.status != PSGD_OK) return;
     // P'^T P' = L L^T  ->  T'; scaled pivot^2 < 2e-2 (rounding of W T amplified > 7x) raises the gate for the precise path
     L.begin(PSGD_K_ORTH);
-    k_chol<<<cnt, 256, (size_t)r * chol_ld(r) * 8, L.st>>>(gram, T, r, h->KC, flags, gate, 2e-2);
+    int* defic = (int*)(ws + Y.defic);
+    k_chol<<<cnt, 256, (size_t)r * chol_ld(r) * 8, L.st>>>(gram, T, r, h->KC, flags, gate, 2e-2, defic);
     L.end();
     FinishPArgs fp{Pout, T, Phat, Ppad, Tacc, Tacc, m, r, RP, h->tacc_identity ? 1 : 0};
     L.begin(PSGD_K_ORTH);
     k_finish_p<<<dim3(ceil_div(m, 64), cnt), 256, 0, L.st>>>(fp);
+    L.end();
+    L.begin(PSGD_K_ORTH);   // rank-deficient P': orthonormal completion of P~ and of its padded copy (no-op otherwise)
+    k_complete<<<cnt, 256, 0, L.st>>>(Phat, Ppad, defic, flags, m, r, RP, h->seed + (uint64_t)h->t);
     L.end();
     // precise back-projection over the stored Delta, only when the gate was raised
     launch_back(L, h->E, Phat, part, m, n, r, N, cnt, h->rpc, h->S, h->vec4, gate);

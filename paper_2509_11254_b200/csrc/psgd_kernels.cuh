@@ -570,10 +570,13 @@ constexpr double CHOL_PIVOT_TOL = 1e-11;  // squared sine of the angle to the pr
 __host__ __device__ inline int chol_ld(int c) { return c | 1; }
 // `gate` (optional): set to 1 when a scaled pivot^2 falls below gate_tol, i.e. when the columns
 // are too ill-conditioned for results derived from W = M^T P to keep float32 accuracy.
+// `defic` (optional, [count][c]): 1 for every column whose pivot was rejected (zero or dependent column);
+// k_complete replaces those columns of P~ by an orthonormal completion.
 __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int c, int nparts, int* flags,
-                                              int* gate = nullptr, double gate_tol = 0.0) {
+                                              int* gate = nullptr, double gate_tol = 0.0, int* defic = nullptr) {
     extern __shared__ __align__(16) double Gs[];  // [c][ld]
     __shared__ double dinv[192];
+    __shared__ int dcol[192];
     __shared__ int bad, illc;
     const int tid = threadIdx.x;
     const int ld = chol_ld(c);
@@ -593,7 +596,8 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
     __syncthreads();
     for (int k = tid; k < c; k += 256) {
         double d = Gs[k * ld + k];
-        if (!(d > 0.0)) { dinv[k] = 0.0; bad = 1; } else dinv[k] = 1.0 / sqrt(d);
+        dcol[k] = 0;
+        if (!(d > 0.0)) { dinv[k] = 0.0; bad = 1; dcol[k] = 1; } else dinv[k] = 1.0 / sqrt(d);
     }
     __syncthreads();
     for (int e = tid; e < c * c; e += 256) {
@@ -608,7 +612,7 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
         if (tid == 0) {
             double p = Gs[k * ld + k];
             if (!(p > gate_tol)) illc = 1;
-            if (!(p > CHOL_PIVOT_TOL)) { bad = 1; p = 1.0; for (int i = k + 1; i < c; ++i) Gs[i * ld + k] = 0.0; }
+            if (!(p > CHOL_PIVOT_TOL)) { bad = 1; dcol[k] = 1; p = 1.0; for (int i = k + 1; i < c; ++i) Gs[i * ld + k] = 0.0; }
             Gs[k * ld + k] = sqrt(p);
         }
         __syncthreads();
@@ -645,8 +649,62 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
         int j = e / c, k = e % c;
         Tb[e] = (j <= k) ? dinv[j] * Gs[k * ld + j] : 0.0;
     }
+    if (defic)
+        for (int k = tid; k < c; k += 256) defic[(size_t)blockIdx.x * c + k] = dcol[k];
     if (tid == 0 && bad) atomicOr(flags, 1);
     if (tid == 0 && illc && gate) atomicOr(gate, 1);
+}
+
+// Orthonormal completion of a rank-deficient factor (the paper is silent on QR of a rank-deficient P; any
+// orthonormal P~ whose span contains range(P) is a valid result).  Every column that k_chol rejected is
+// replaced by a seeded pseudo-random vector, orthogonalised twice (modified Gram-Schmidt, double sums)
+// against the valid columns and normalised.  One CTA per matrix; does nothing unless the status word
+// carries PSGD_W_RANK_DEFICIENT.  Ppad (optional) is the padded copy [count][rows][RP] kept in step.
+__global__ void __launch_bounds__(256) k_complete(float* Phat, float* Ppad, const int* defic, const int* flags, int rows, int r,
+                                                  int RP, uint64_t seed) {
+    if (!(*flags & 1)) return;
+    __shared__ double red[8];
+    __shared__ double bc;
+    const int c = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float* Pb = Phat + (size_t)c * rows * r;
+    const int* db = defic + (size_t)c * r;
+    auto block_sum = [&](double v) -> double {
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        __syncthreads();
+        if (lane == 0) red[warp] = v;
+        __syncthreads();
+        if (tid == 0) { double t = 0.0; for (int w = 0; w < 8; ++w) t += red[w]; bc = t; }
+        __syncthreads();
+        return bc;
+    };
+    for (int k = 0; k < r; ++k) {
+        if (!db[k]) continue;
+        for (int row = tid; row < rows; row += 256) {
+            uint64_t h = splitmix64(splitmix64(seed ^ (0xC0FFEEull + (uint64_t)c * 1315423911ull + (uint64_t)k)) + (uint64_t)row);
+            float u1 = ((float)(uint32_t)(h >> 40) + 0.5f) * (1.0f / 16777216.0f);
+            float u2 = ((float)(uint32_t)((h >> 8) & 0xFFFFFF) + 0.5f) * (1.0f / 16777216.0f);
+            Pb[(size_t)row * r + k] = sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
+        }
+        __syncthreads();
+        for (int pass = 0; pass < 2; ++pass)
+            for (int j = 0; j < r; ++j) {
+                if (j == k || (db[j] && j > k)) continue;      // columns not yet completed hold nothing useful
+                double s = 0.0;
+                for (int row = tid; row < rows; row += 256) s += (double)Pb[(size_t)row * r + j] * (double)Pb[(size_t)row * r + k];
+                const double cj = block_sum(s);
+                for (int row = tid; row < rows; row += 256) Pb[(size_t)row * r + k] -= (float)(cj * (double)Pb[(size_t)row * r + j]);
+                __syncthreads();
+            }
+        double s = 0.0;
+        for (int row = tid; row < rows; row += 256) { double v = Pb[(size_t)row * r + k]; s += v * v; }
+        const double inv = 1.0 / sqrt(fmax(block_sum(s), 1e-300));
+        for (int row = tid; row < rows; row += 256) {
+            float v = (float)((double)Pb[(size_t)row * r + k] * inv);
+            Pb[(size_t)row * r + k] = v;
+            if (Ppad) Ppad[((size_t)c * rows + row) * RP + k] = v;
+        }
+        __syncthreads();
+    }
 }
 
 // Xout[row][k] = sum_j X[row][j] * T[j][k]  (double accumulate), k < kout.

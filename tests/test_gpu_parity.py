@@ -389,3 +389,77 @@ def test_full_size_config5(torch_cuda, r):
     """BASELINE config 5: one 16384 x 4096 matrix on 4 nodes, plain PowerSGD steps (the step the sweep times)."""
     plan = _full_size_case(torch_cuda, 5, 16384, 4096, r, 4, 1, tau=0, sample=(0,), free_steps=3)
     assert plan["single_pass"] == 1 and plan["CS"] == 8 and plan["WC"] == 512
+
+
+# ---- degenerate inputs ------------------------------------------------------------------------
+def _invariants(comp, M, P_mean, r, tag):
+    """What must hold for ANY valid orthonormal factor (several are correct when P is rank deficient)."""
+    P = comp.P_hat[0].cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(P.T @ P - np.eye(r)) <= 1e-5, f"{tag}: P~ not orthonormal"
+    assert np.linalg.norm(P_mean - P @ (P.T @ P_mean)) <= 1e-5 * max(np.linalg.norm(P_mean), 1e-30) + 1e-6, f"{tag}: range(P) not in range(P~)"
+    E = comp.E[0].cpu().numpy().astype(np.float64)
+    Qn = comp.debug("Q_node")[0].cpu().numpy().astype(np.float64)
+    for i in range(M.shape[0]):
+        nm = np.linalg.norm(M[i])
+        assert np.linalg.norm(E[i] + P @ Qn[i].T - M[i]) <= 1e-5 * nm, f"{tag}: E + P~Q_i^T != M (node {i})"
+        assert np.linalg.norm(P.T @ E[i]) <= 1e-5 * nm, f"{tag}: P~^T E != 0 (node {i})"
+
+
+@pytest.mark.parametrize("mode", ["eager", "deferred"])
+def test_rank_deficient_projection(torch_cuda, mode):
+    """P = mean_i M_i Q of rank 2 < r = 4: any orthonormal completion is valid; the warning bit is set."""
+    from paper_2509_11254_b200 import PowerSGDPlus, PSGD_W_RANK_DEFICIENT
+
+    torch = torch_cuda
+    m, n, r, N = 200, 96, 4, 3
+    G = synth.exact_rank_r(m, n, 2, N)                      # every node: the same exactly rank-2 matrix
+    comp = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=3, mode=mode)
+    Q0 = synth.init_Q(n, r, seed=3)
+    comp.set_state(E=np.zeros((1, N, m, n), np.float32), Q=Q0[None], t=1)
+    comp.step(torch.as_tensor(G[None], device="cuda:0"))
+    comp.materialize_error()
+    flags = comp.last_status()
+    assert flags & PSGD_W_RANK_DEFICIENT
+    M = G.astype(np.float64)
+    _invariants(comp, M, M.mean(axis=0) @ Q0.astype(np.float64), r, mode)
+
+
+def test_zero_gradient_step(torch_cuda):
+    """G = 0 and E = 0 (P = 0, the case the counterexample's induction can hit): outputs stay finite, E stays 0."""
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    torch = torch_cuda
+    m, n, r, N = 128, 64, 4, 2
+    comp = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=3)
+    comp.step(torch.zeros((1, N, m, n), device="cuda:0"))
+    assert torch.isfinite(comp.P_hat).all() and torch.isfinite(comp.Q).all()
+    assert float(comp.E.abs().max()) == 0.0
+    P = comp.P_hat[0].cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(P.T @ P - np.eye(r)) <= 1e-5
+
+
+def test_ill_conditioned_projection_takes_the_precise_path(torch_cuda):
+    """Deferred mode with a nearly dependent basis Q: the Cholesky pivot test raises the gate and the
+    step still matches the oracle at 1e-5 (Q_i from the precise back-projection)."""
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    torch = torch_cuda
+    m, n, r, N = 520, 256, 4, 2
+    rng = np.random.default_rng(5)
+    Q0 = synth.init_Q(n, r, seed=9)
+    Q0[:, 3] = Q0[:, 2] + 0.02 * Q0[:, 3]          # columns 2 and 3 at an angle of about 0.02
+    Q0 = Q0.astype(np.float32)
+    E0 = (rng.standard_normal((N, m, n)) * 0.01).astype(np.float32)
+    G = synth.make_gradients(2, m, n, N, step=0, seed=9)
+    comp = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=9, mode="deferred")
+    comp.set_state(E=E0[None], Q=Q0[None], t=1)
+    o = orc.PowerSGDPlusOracle(m, n, r, N, 0, Q0)
+    o.E = E0.astype(np.float64)
+    o.t = 1
+    comp.step(torch.as_tensor(G[None], device="cuda:0"))
+    comp.materialize_error()
+    assert comp.last_status() == 0
+    out = o.step(G)
+    gp = dict(P_hat=comp.P_hat[0].cpu().numpy(), Q=comp.Q[0].cpu().numpy(), E=comp.E[0].cpu().numpy(),
+              Q_node=comp.debug("Q_node")[0].cpu().numpy())
+    compare_step(out, gp, m, n, r, N, "ill-conditioned Q")
