@@ -68,6 +68,8 @@ typedef enum {
 #define PSGD_OPT_REFRESH_OVERSAMPLE 4 /* extra columns of the refresh block (default max(8, r)) */
 #define PSGD_OPT_REFRESH_TC 5      /* 1 (default): the early sweeps of a refresh whose block has >= 32 columns run
                                       on the tensor cores in TF32, the last 8 in float32; 0: float32 throughout */
+#define PSGD_OPT_POWER_STEPS 6     /* K >= 1 power steps per SSP iteration (Eq. (8)); 1 (default) is PowerSGD's single
+                                      step (Eq. (9)); K > 1 runs the three-pass kernels */
 
 /* buffers that psgd_debug_ptr exposes (test use only; valid until the next step) */
 #define PSGD_BUF_P_NODE 1   /* P^(i)   [count][N][m][r] */

@@ -121,11 +121,18 @@ def gemm_nt_tf32(A, B):
 # --------------------------------------------------------------------------
 # Algorithm 1, both compressors.  Delta has shape [N, m, n].
 # --------------------------------------------------------------------------
-def ssp_comp(Q, Delta):
-    """SSP-Comp of Algorithm 1.  Returns a dict of every intermediate."""
+def ssp_comp(Q, Delta, power_steps=1):
+    """SSP-Comp of Algorithm 1.  Returns a dict of every intermediate.
+
+    power_steps = K > 1 runs the K-step power iteration of Eq. (8) across the nodes: the first K - 1
+    rounds only carry Q forward (Q <- mean_i Delta_i^T P~), the K-th is the round Algorithm 1 states.
+    """
     Delta = np.asarray(Delta, dtype=F64)
     Q = np.asarray(Q, dtype=F64)
     N = Delta.shape[0]
+    for _ in range(power_steps - 1):
+        P_hat = qr_orth(_mean(np.stack([Delta[i] @ Q for i in range(N)])))
+        Q = _mean(np.stack([Delta[i].T @ P_hat for i in range(N)]))
     P_i = np.stack([Delta[i] @ Q for i in range(N)])           # P^(i) <- Delta^(i) Q
     P = _mean(P_i)                                              # All-Reduce Mean
     P_hat, R = householder_qr(P)                                # P~ <- QR(P)
@@ -185,13 +192,14 @@ class PowerSGDPlusOracle:
     subtracts P~ Q^T with the node-averaged Q instead.
     """
 
-    def __init__(self, m, n, r, N, tau, Q_init, error_form="local"):
+    def __init__(self, m, n, r, N, tau, Q_init, error_form="local", power_steps=1):
         if not (m >= n >= r >= 1 and N >= 1 and tau >= 0):
             raise ValueError("need m >= n >= r >= 1, N >= 1, tau >= 0")
         if error_form not in ("local", "mean"):
             raise ValueError("error_form")
         self.m, self.n, self.r, self.N, self.tau = m, n, r, N, tau
         self.error_form = error_form
+        self.power_steps = power_steps
         self.t = 0
         self.Q = np.array(Q_init, dtype=F64).reshape(n, r).copy()
         self.E = np.zeros((N, m, n), dtype=F64)                 # e_0^(i) = 0
@@ -208,7 +216,7 @@ class PowerSGDPlusOracle:
         G = np.asarray(G, dtype=F64).reshape(self.N, self.m, self.n)
         M = G + self.E                                          # Eq. (7a)
         refresh = force_svd or self.is_refresh_step()
-        out = svd_comp(M, self.r) if refresh else ssp_comp(self.Q, M)
+        out = svd_comp(M, self.r) if refresh else ssp_comp(self.Q, M, self.power_steps)
         if self.error_form == "local":
             E_new = M - out["Dhat_i"]                           # e_{t+1}^(i)
         else:

@@ -44,7 +44,7 @@ struct psgd_handle {
     int64_t m, n;
     int r, N, count, tau;
     uint64_t seed;
-    int error_form = 0, mode = 0, refresh_iters = 20, oversample = -1, refresh_tc = 1;
+    int error_form = 0, mode = 0, refresh_iters = 20, oversample = -1, refresh_tc = 1, power_steps = 1;
     bool tc_ok = false;           // the refresh block is wide enough for the tensor-core sweeps
     size_t gpart_floats = 0;
     bool rtc_ok = false;          // ranks above 16 with 16-byte row strides: residual update on the tensor cores
@@ -470,6 +470,22 @@ void ssp(Launcher& L, psgd_handle* h, const float* G) {
     k_node_mean<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Pnode, Pmean, (size_t)m * r, N, cnt);
     L.end();
     launch_orth(L, h, Pmean, Phat, m, r, PSGD_K_ORTH, nullptr, true);
+    // K-step power iteration (Eq. (8)): K - 1 more rounds Q <- mean_i M_i^T P~, P~ <- QR(mean_i M_i Q) on the
+    // stored M before the usual last back-projection
+    float* Qnode = (float*)(ws + h->lay.Qnode);
+    float* part = (float*)(ws + h->lay.part);
+    for (int k = 1; k < h->power_steps; ++k) {
+        launch_back(L, h->E, Phat, part, m, n, r, N, cnt, h->rpc, h->S, h->vec4);
+        size_t tq = (size_t)cnt * n * r;
+        L.begin(PSGD_K_BACKPROJECT);
+        k_reduce_q<<<(unsigned)((tq + 255) / 256), 256, 0, L.st>>>(part, Qnode, h->Q, n, r, N, h->S, cnt);
+        L.end();
+        launch_project(L, h->E, nullptr, nullptr, h->Q, Pnode, m, n, r, N, cnt, h->vec4);
+        L.begin(PSGD_K_ORTH);
+        k_node_mean<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Pnode, Pmean, (size_t)m * r, N, cnt);
+        L.end();
+        launch_orth(L, h, Pmean, Phat, m, r, PSGD_K_ORTH, nullptr, true);
+    }
 }
 
 // ---- SVD-Comp (Algorithm 1, second function): top-r left singular subspace of the
@@ -698,7 +714,7 @@ psgd_status do_step(psgd_handle* h, const float* G, float* P_hat, float* D_hat, 
     cudaStream_t st = (cudaStream_t)stream;
     Launcher L{h, st};
     bool refresh = force || (h->tau > 0 && h->t % h->tau == 0);
-    if (h->mode == 1 && h->fused_ok && !refresh && aligned16(G)) {
+    if (h->mode == 1 && h->fused_ok && !refresh && aligned16(G) && h->power_steps == 1) {
         fused_ssp(L, h, G);
         if (D_hat) {
             float* Phat = (float*)(h->ws + h->lay.Phat);
@@ -751,6 +767,7 @@ psgd_status psgd_set_option(psgd_handle* h, int option, int value) {
         case PSGD_OPT_REFRESH_ITERS: if (value < 1 || value > 64) return PSGD_E_INVALID; h->refresh_iters = value; break;
         case PSGD_OPT_REFRESH_OVERSAMPLE: if (value < 0 || value > MAX_L) return PSGD_E_INVALID; h->oversample = value; break;
         case PSGD_OPT_REFRESH_TC: if (value != 0 && value != 1) return PSGD_E_INVALID; h->refresh_tc = value; break;
+        case PSGD_OPT_POWER_STEPS: if (value < 1 || value > 16) return PSGD_E_INVALID; h->power_steps = value; break;
         default: return PSGD_E_INVALID;
     }
     plan(h);

@@ -79,15 +79,15 @@ def compare_step(out, gpu, m, n, r, N, tag):
 
 
 def run_case(torch, m, n, r, N, tau, steps, workload=1, count=1, error_form="local", Einit=0.0, seed=7,
-             check_dense=False, mode="eager"):
+             check_dense=False, mode="eager", power_steps=1):
     from paper_2509_11254_b200 import PowerSGDPlus
 
     dev = "cuda:0"
     comp = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=seed, count=count, device=dev, error_form=error_form,
-                        mode=mode)
+                        mode=mode, power_steps=power_steps)
     rng = np.random.default_rng(seed)
     Q0 = np.stack([synth.init_Q(n, r, matrix_id=c, seed=seed) for c in range(count)])
-    oracles = [orc.PowerSGDPlusOracle(m, n, r, N, tau, Q0[c], error_form) for c in range(count)]
+    oracles = [orc.PowerSGDPlusOracle(m, n, r, N, tau, Q0[c], error_form, power_steps) for c in range(count)]
     if Einit:
         for o in oracles:
             o.E = (rng.standard_normal((N, m, n)) * Einit).astype(np.float32).astype(np.float64)
@@ -107,7 +107,7 @@ def run_case(torch, m, n, r, N, tau, steps, workload=1, count=1, error_form="loc
         assert comp.t == t + 1
         gp = dict(P_hat=comp.P_hat.cpu().numpy(), Q=comp.Q.cpu().numpy(), E=comp.E.cpu().numpy(),
                   Q_node=comp.debug("Q_node").cpu().numpy())
-        if mode == "eager":   # the single-pass kernel never materialises the per-node P_i
+        if mode == "eager" and power_steps == 1:   # (single-pass: no per-node P_i; K steps: P_i is the last round's)
             gp["P_node"] = comp.debug("P_node").cpu().numpy()
         for c, o in enumerate(oracles):
             out = o.step(G[c])
@@ -155,6 +155,12 @@ def test_large_rank_ssp(torch_cuda, r):
 def test_residual_on_tensor_cores(torch_cuda, m, n, r, N, count, form):
     """Ranks above 16: E = M - P~ Q_i^T as a split-TF32 tcgen05 product, against the oracle at 1e-5."""
     run_case(torch_cuda, m, n, r, N, tau=0, steps=2, workload=4, count=count, Einit=0.01, error_form=form, check_dense=True)
+
+
+@pytest.mark.parametrize("K,mode", [(2, "eager"), (3, "deferred")])
+def test_k_step_power_iteration(torch_cuda, K, mode):
+    """Eq. (8): K power steps per iteration (the deferred mode falls back to the three-pass kernels)."""
+    run_case(torch_cuda, 300, 200, 6, 3, tau=0, steps=3, workload=2, count=2, Einit=0.01, mode=mode, power_steps=K)
 
 
 def test_mean_error_form(torch_cuda):

@@ -275,6 +275,13 @@ def check_fixed_point(o):
     # many power steps converge to the optimal compressor (Eq. (8))
     Pk, Qk = o.power_iteration(Dbar, rng.standard_normal((n, r)), 400)
     np.testing.assert_allclose(Pk @ Qk.T, (U[:, :r] * s[:r]) @ Vt[:r], atol=1e-8)
+    # K power steps across the nodes (means of per-node products) are K power steps on the node mean
+    Qs = rng.standard_normal((n, r))
+    for K in (2, 5):
+        d = o.ssp_comp(Qs, D, power_steps=K)
+        Pk, Qk = o.power_iteration(Dbar, Qs, K)
+        np.testing.assert_allclose(d["P_hat"], Pk, atol=1e-12)
+        np.testing.assert_allclose(d["Q"], Qk, atol=1e-12)
 
 
 def check_counter_function(o):
