@@ -70,6 +70,8 @@ typedef enum {
                                       on the tensor cores in TF32, the last 8 in float32; 0: float32 throughout */
 #define PSGD_OPT_POWER_STEPS 6     /* K >= 1 power steps per SSP iteration (Eq. (8)); 1 (default) is PowerSGD's single
                                       step (Eq. (9)); K > 1 runs the three-pass kernels */
+#define PSGD_OPT_REFRESH_ADAPTIVE 7 /* 1 (default): a refresh whose block has <= 48 columns stops its sweeps once the top-r
+                                      basis has stopped moving between two checks (<= 1e-5 and halving, or <= 3e-6); 0: all the sweeps */
 
 /* buffers that psgd_debug_ptr exposes (test use only; valid until the next step) */
 #define PSGD_BUF_P_NODE 1   /* P^(i)   [count][N][m][r] */

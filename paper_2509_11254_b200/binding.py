@@ -11,6 +11,7 @@ PSGD_W_NOT_CONVERGED = 2
 PSGD_W_TIMEOUT = 4
 PSGD_OPT_ERROR_FORM, PSGD_OPT_MODE, PSGD_OPT_REFRESH_ITERS, PSGD_OPT_REFRESH_OVERSAMPLE, PSGD_OPT_REFRESH_TC = 1, 2, 3, 4, 5
 PSGD_OPT_POWER_STEPS = 6
+PSGD_OPT_REFRESH_ADAPTIVE = 7
 PSGD_BUF = {"P_node": 1, "Q_node": 2, "P_hat": 3, "Dbar": 4, "P_mean": 5}
 KERNEL_FAMILIES = ["project", "orth", "backproject", "residual", "refresh", "misc"]
 
@@ -89,7 +90,7 @@ class PowerSGDPlus:
     """
 
     def __init__(self, m, n, r, N, refresh_period=0, seed=0, count=1, device="cuda:0", error_form="local",
-                 mode="eager", refresh_iters=None, oversample=None, reset=True, refresh_tc=None, power_steps=None):
+                 mode="eager", refresh_iters=None, oversample=None, reset=True, refresh_tc=None, power_steps=None, refresh_adaptive=None):
         import torch
 
         self.torch = torch
@@ -111,6 +112,8 @@ class PowerSGDPlus:
             _check(L.psgd_set_option(h, PSGD_OPT_REFRESH_TC, int(bool(refresh_tc))))
         if power_steps is not None:
             _check(L.psgd_set_option(h, PSGD_OPT_POWER_STEPS, int(power_steps)))
+        if refresh_adaptive is not None:
+            _check(L.psgd_set_option(h, PSGD_OPT_REFRESH_ADAPTIVE, int(bool(refresh_adaptive))))
         eb, qb, wb = _sz(), _sz(), _sz()
         _check(L.psgd_sizes(h, C.byref(eb), C.byref(qb), C.byref(wb)))
         with torch.cuda.device(self.device):

@@ -31,6 +31,7 @@ struct Layout {
     size_t Qpad, Ppad, Qsub, Tacc, Pout, Wpart, Cmat, Cpart;  // deferred (single-pass) mode only
     size_t dbarT, Yt, Zt, gpart;                              // tensor-core refresh only
     size_t rtP, rtQ;                                          // tensor-core residual (r > 16) only
+    size_t Pold, dpart;                                       // stopping test of the refresh
 };
 
 struct ProfEvent {
@@ -44,7 +45,7 @@ struct psgd_handle {
     int64_t m, n;
     int r, N, count, tau;
     uint64_t seed;
-    int error_form = 0, mode = 0, refresh_iters = 20, oversample = -1, refresh_tc = 1, power_steps = 1;
+    int error_form = 0, mode = 0, refresh_iters = 20, oversample = -1, refresh_tc = 1, power_steps = 1, refresh_adaptive = 1;
     bool tc_ok = false;           // the refresh block is wide enough for the tensor-core sweeps
     size_t gpart_floats = 0;
     bool rtc_ok = false;          // ranks above 16 with 16-byte row strides: residual update on the tensor cores
@@ -127,6 +128,8 @@ void plan(psgd_handle* h) {
     size_t c2 = (c + 1) & ~(size_t)1;
     L.V = take(cnt * c2 * c2 * 8);
     L.U = take(cnt * ell * r * 8);
+    L.Pold = take(cnt * m * r * 4);
+    L.dpart = take(cnt * ((size_t)ceil_div(h->m, 64) + 1) * 8);
     // ---- tensor-core sweeps of the refresh: block of >= 32 columns, 16-byte row strides for TMA ----
     h->tc_ok = h->refresh_tc && ell >= 32 && ell <= TC_MAXN && h->n % 4 == 0 && h->m % 4 == 0;
     if (h->tc_ok) {
@@ -312,8 +315,8 @@ void launch_project_rp(Launcher& L, const ProjectArgs& a, int count, bool vec, b
 }
 // P = (A [+B]) Q for all matrices; `add` also stores A+B into Mout.
 void launch_project(Launcher& L, const float* A, const float* B, float* Mout, const float* Q, float* P, int rows, int n,
-                    int r, int nodes, int count, bool vec) {
-    ProjectArgs a{A, B, Mout, Q, P, rows, n, r, nodes, 1};
+                    int r, int nodes, int count, bool vec, const int* skip = nullptr) {
+    ProjectArgs a{A, B, Mout, Q, P, rows, n, r, nodes, 1, skip};
     bool add = B != nullptr;
     vec = vec && aligned16(A) && (!B || aligned16(B)) && (!Mout || aligned16(Mout));
     if (r <= 4) launch_project_rp<4>(L, a, count, vec, add);
@@ -337,8 +340,8 @@ void launch_back_rp(Launcher& L, BackArgs a, int mats, bool vec) {
     L.end();
 }
 void launch_back(Launcher& L, const float* M, const float* Phat, float* part, int rows, int n, int r, int nodes,
-                 int count, int rpc, int S, bool vec, const int* gate = nullptr) {
-    BackArgs a{M, Phat, part, rows, n, r, nodes, 1, rpc, S, gate};
+                 int count, int rpc, int S, bool vec, const int* gate = nullptr, const int* skip = nullptr) {
+    BackArgs a{M, Phat, part, rows, n, r, nodes, 1, rpc, S, gate, skip};
     vec = vec && aligned16(M);
     if (r <= 4) launch_back_rp<4>(L, a, count * nodes, vec);
     else if (r <= 8) launch_back_rp<8>(L, a, count * nodes, vec);
@@ -397,30 +400,30 @@ void launch_resid(Launcher& L, const float* M, float* Out, const float* Phat, co
 
 // ---- K2: X <- orthonormal factor of X (rows x c), in place or into Xout ------
 void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int rows, int c, int kind, float* XoutT = nullptr,
-                 bool complete = false) {
+                 bool complete = false, const int* skip = nullptr) {
     char* ws = h->ws;
     double* gram = (double*)(ws + h->lay.gram);
     double* T = (double*)(ws + h->lay.T);
     int* flags = (int*)(ws + h->lay.flags);
     int nparts = ceil_div(rows, GR_ROWS);
     int nblk = ceil_div(c, 64);
-    GramArgs g{X, gram, rows, c, nparts};
+    GramArgs g{X, gram, rows, c, nparts, nullptr, skip};
     L.begin(kind);
     k_gram<<<dim3(nparts, nblk * nblk, h->count), 256, 0, L.st>>>(g);
     L.end();
     if (nparts > 4) {   // fold the partials in parallel first; k_chol then reads partial 0 with the original stride
         size_t tot = (size_t)c * c * h->count;
         L.begin(kind);
-        k_gram_sum<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(gram, c * c, nparts, h->count);
+        k_gram_sum<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(gram, c * c, nparts, h->count, skip);
         L.end();
     }
     size_t smem = (size_t)c * chol_ld(c) * 8;
     allow_smem(k_chol, smem);
     L.begin(kind);
     int* defic = (int*)(ws + h->lay.defic);
-    k_chol<<<h->count, 256, smem, L.st>>>(gram, T, c, nparts > 4 ? -nparts : nparts, flags, nullptr, 0.0, complete ? defic : nullptr);
+    k_chol<<<h->count, 256, smem, L.st>>>(gram, T, c, nparts > 4 ? -nparts : nparts, flags, nullptr, 0.0, complete ? defic : nullptr, skip);
     L.end();
-    ApplyArgs ap{X, T, Xout, rows, c, c, c, 1, XoutT};
+    ApplyArgs ap{X, T, Xout, rows, c, c, c, 1, XoutT, skip};
     L.begin(kind);
     k_apply<<<dim3(ceil_div(rows, 32), h->count), 256, (size_t)32 * c * 4, L.st>>>(ap);
     L.end();
@@ -537,40 +540,78 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
     S = std::min(S, std::min(64, ceil_div(m, BP_SUB)));
     int rpc = (int)align_up(ceil_div(m, S), BP_SUB);
     S = ceil_div(m, rpc);
+    // Rayleigh-Ritz on the current block: eigenvectors of Z^T Z = Y^T Dbar Dbar^T Y, then P~ = Y U[:, :r]
+    int* done = flags + 3;                 // set on the device once the top-r basis has stopped moving
+    const bool adaptive = h->refresh_adaptive && ell <= 48 && h->refresh_iters - it0 > 6;
+    const int* skip = adaptive ? done : nullptr;
+    if (adaptive) cudaMemsetAsync(done, 0, 4, L.st);
+    auto rayleigh_ritz = [&]() {
+        int nparts = ceil_div(n, GR_ROWS);
+        int nblk = ceil_div(ell, 64);
+        GramArgs g{Z, gram, n, ell, nparts, nullptr, skip};
+        L.begin(K);
+        k_gram<<<dim3(nparts, nblk * nblk, cnt), 256, 0, L.st>>>(g);
+        L.end();
+        if (nparts > 4) {
+            size_t tot = (size_t)ell * ell * cnt;
+            L.begin(K);
+            k_gram_sum<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(gram, ell * ell, nparts, cnt, skip);
+            L.end();
+        }
+        int c2 = (ell + 1) & ~1;
+        size_t smem = (size_t)c2 * jac_ld(c2) * 8;
+        allow_smem(k_jacobi_top, smem);
+        L.begin(K);
+        k_jacobi_top<<<cnt, JAC_THREADS, smem, L.st>>>(gram, nparts > 4 ? -nparts : nparts, ell, r, V, U, flags, skip);
+        L.end();
+        ApplyArgs ap{Y, U, Phat, m, ell, r, r, 0, nullptr, skip};
+        L.begin(K);
+        k_apply<<<dim3(ceil_div(m, 32), cnt), 256, (size_t)32 * ell * 4, L.st>>>(ap);
+        L.end();
+    };
+    // Stopping test (blocks of <= 48 columns, where a Rayleigh-Ritz step is cheap): every third sweep the top-r
+    // Ritz basis is compared with the one of the previous check; once it has stopped moving in every matrix of
+    // the handle (rule in k_refresh_decide) the remaining kernels of this refresh return at once.  With geometric
+    // convergence the error left is below the last movement.  Inputs that never get there run all the sweeps.
+    float* Pold = (float*)(ws + h->lay.Pold);
+    double* dpart = (double*)(ws + h->lay.dpart);
+    double* dprev = dpart + (size_t)cnt * ceil_div(m, 64);
+    int nchecks = 0;
     for (int it = it0; it < h->refresh_iters; ++it) {
         // Y = Dbar Z, orthonormalise;  Z = Dbar^T Y, orthonormalise
-        launch_project(L, dbar, nullptr, nullptr, Z, Y, m, n, ell, 1, cnt, h->vec4);
-        launch_orth(L, h, Y, Y, m, ell, K);
-        launch_back(L, dbar, Y, part, m, n, ell, 1, cnt, rpc, S, h->vec4);
+        launch_project(L, dbar, nullptr, nullptr, Z, Y, m, n, ell, 1, cnt, h->vec4, skip);
+        launch_orth(L, h, Y, Y, m, ell, K, nullptr, false, skip);
+        launch_back(L, dbar, Y, part, m, n, ell, 1, cnt, rpc, S, h->vec4, nullptr, skip);
         size_t tot = (size_t)cnt * n * ell;
         L.begin(K);
-        k_reduce_q<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(part, nullptr, Z, n, ell, 1, S, cnt);
+        k_reduce_q<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(part, nullptr, Z, n, ell, 1, S, cnt, skip);
         L.end();
-        if (it + 1 < h->refresh_iters) launch_orth(L, h, Z, Z, n, ell, K);
+        if (it + 1 == h->refresh_iters) break;
+        if (adaptive && (it - it0 + 1) % 3 == 0) {
+            rayleigh_ritz();
+            if (nchecks > 0) {
+                const int nparts = ceil_div(m, GR_ROWS), nblk = ceil_div(r, 64), nb = ceil_div(m, 64);
+                GramArgs g{Pold, gram, m, r, nparts, Phat, skip};       // S = Pold^T Pnew
+                L.begin(K);
+                k_gram<<<dim3(nparts, nblk * nblk, cnt), 256, 0, L.st>>>(g);
+                L.end();
+                size_t tg = (size_t)r * r * cnt;
+                L.begin(K);
+                k_gram_sum<<<(unsigned)((tg + 255) / 256), 256, 0, L.st>>>(gram, r * r, nparts, cnt, skip);
+                L.end();
+                L.begin(K);
+                k_subspace_change<<<dim3(nb, cnt), 256, (size_t)r * r * 4, L.st>>>(Pold, Phat, gram, (size_t)nparts * r * r, dpart, m, r, skip);
+                L.end();
+                L.begin(K);
+                k_refresh_decide<<<1, 32, 0, L.st>>>(dpart, nb, cnt, dprev, nchecks > 1 ? 1 : 0, done);
+                L.end();
+            }
+            cudaMemcpyAsync(Pold, Phat, (size_t)cnt * m * r * 4, cudaMemcpyDeviceToDevice, L.st);
+            ++nchecks;
+        }
+        launch_orth(L, h, Z, Z, n, ell, K, nullptr, false, skip);
     }
-    // Rayleigh-Ritz: eigenvectors of Z^T Z = Y^T Dbar Dbar^T Y, then P~ = Y U[:, :r]
-    int nparts = ceil_div(n, GR_ROWS);
-    int nblk = ceil_div(ell, 64);
-    GramArgs g{Z, gram, n, ell, nparts};
-    L.begin(K);
-    k_gram<<<dim3(nparts, nblk * nblk, cnt), 256, 0, L.st>>>(g);
-    L.end();
-    int c2 = (ell + 1) & ~1;
-    size_t smem = (size_t)c2 * jac_ld(c2) * 8;
-    allow_smem(k_jacobi_top, smem);
-    L.begin(K);
-    if (nparts > 4) {
-        size_t tot = (size_t)ell * ell * cnt;
-        L.begin(K);
-        k_gram_sum<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(gram, ell * ell, nparts, cnt);
-        L.end();
-    }
-    k_jacobi_top<<<cnt, JAC_THREADS, smem, L.st>>>(gram, nparts > 4 ? -nparts : nparts, ell, r, V, U, flags);
-    L.end();
-    ApplyArgs ap{Y, U, Phat, m, ell, r, r, 0, nullptr};
-    L.begin(K);
-    k_apply<<<dim3(ceil_div(m, 32), cnt), 256, (size_t)32 * ell * 4, L.st>>>(ap);
-    L.end();
+    rayleigh_ritz();
     L.force_kind = -1;
 }
 
@@ -767,6 +808,7 @@ psgd_status psgd_set_option(psgd_handle* h, int option, int value) {
         case PSGD_OPT_REFRESH_ITERS: if (value < 1 || value > 64) return PSGD_E_INVALID; h->refresh_iters = value; break;
         case PSGD_OPT_REFRESH_OVERSAMPLE: if (value < 0 || value > MAX_L) return PSGD_E_INVALID; h->oversample = value; break;
         case PSGD_OPT_REFRESH_TC: if (value != 0 && value != 1) return PSGD_E_INVALID; h->refresh_tc = value; break;
+        case PSGD_OPT_REFRESH_ADAPTIVE: if (value != 0 && value != 1) return PSGD_E_INVALID; h->refresh_adaptive = value; break;
         case PSGD_OPT_POWER_STEPS: if (value < 1 || value > 16) return PSGD_E_INVALID; h->power_steps = value; break;
         default: return PSGD_E_INVALID;
     }

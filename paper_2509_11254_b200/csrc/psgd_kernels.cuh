@@ -55,6 +55,7 @@ struct ProjectArgs {
     const float* Q;   // [count][n][r]
     float* P;         // [mats][rows][r]
     int rows, n, r, nodes, nchunks;
+    const int* skip;  // when non-null the kernel does nothing if *skip != 0 (refresh already converged)
 };
 
 template <int RP, bool ADD>
@@ -69,6 +70,7 @@ __host__ __device__ constexpr size_t project_smem_bytes() {
 template <int RP, int VEC, bool ADD, bool STORE>
 __global__ void __launch_bounds__(PJ_THREADS) k_project(ProjectArgs a) {
     extern __shared__ __align__(16) float smem[];
+    if (a.skip && *a.skip) return;
     float* tA = smem;
     float* tB = tA + (ADD ? PJ_STAGES * PJ_TR * PJ_TCP : 0);
     float* tQ = tB + PJ_STAGES * PJ_TR * PJ_TCP;
@@ -218,6 +220,7 @@ struct BackArgs {
     float* part;        // [mats][S][n][r]
     int rows, n, r, nodes, nchunks, rows_per_chunk, S;
     const int* gate;    // when non-null the kernel does nothing unless *gate != 0
+    const int* skip;    // when non-null the kernel does nothing if *skip != 0
 };
 
 template <int RP, int VEC>
@@ -225,6 +228,7 @@ __global__ void __launch_bounds__(BP_THREADS) k_backproject(BackArgs a) {
     __shared__ __align__(16) float Ps[BP_SUB * RP];
     __shared__ __align__(16) float red[64 * 4 * RP];
     if (a.gate && *a.gate == 0) return;
+    if (a.skip && *a.skip) return;
     const int tid = threadIdx.x, tx = tid & 63, g = tid >> 6;
     const int col = blockIdx.x * BP_COLS + tx * 4;
     const int s = blockIdx.y;
@@ -311,7 +315,9 @@ __global__ void __launch_bounds__(BP_THREADS) k_backproject(BackArgs a) {
 
 // Q_i = sum over row chunks of the partials;  Q = (1/N) sum_i Q_i   (All-Reduce Mean).
 // One thread per (matrix, column, k); fixed summation order.
-__global__ void k_reduce_q(const float* part, float* Qi, float* Qmean, int n, int r, int nodes, int S, int count) {
+__global__ void k_reduce_q(const float* part, float* Qi, float* Qmean, int n, int r, int nodes, int S, int count,
+                           const int* skip = nullptr) {
+    if (skip && *skip) return;
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     size_t per = (size_t)n * r;
     if (idx >= per * count) return;
@@ -500,6 +506,8 @@ struct GramArgs {
     const float* X;  // [count][rows][c]
     double* part;    // [count][nparts][c][c]
     int rows, c, nparts;
+    const float* X2; // optional second factor: part = X^T X2 (all blocks computed); nullptr: X^T X, upper block triangle
+    const int* skip; // when non-null the kernel does nothing if *skip != 0
 };
 // grid: (nparts, nblk*nblk, count); 256 threads as 16x16; each thread a 4x4 block of a 64x64 tile.
 __global__ void __launch_bounds__(256) k_gram(GramArgs a) {
@@ -507,9 +515,11 @@ __global__ void __launch_bounds__(256) k_gram(GramArgs a) {
     __shared__ float sb[32][65];
     const int nblk = (a.c + 63) / 64;
     const int bi = blockIdx.y / nblk, bj = blockIdx.y % nblk;
-    if (bi > bj) return;  // symmetric: only the upper block triangle
+    if (a.skip && *a.skip) return;
+    if (!a.X2 && bi > bj) return;  // symmetric: only the upper block triangle
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     const float* Xb = a.X + (size_t)blockIdx.z * a.rows * a.c;
+    const float* X2b = (a.X2 ? a.X2 : a.X) + (size_t)blockIdx.z * a.rows * a.c;
     const int rbeg = blockIdx.x * GR_ROWS, rend = min(a.rows, rbeg + GR_ROWS);
     double acc[4][4];
 #pragma unroll
@@ -523,7 +533,7 @@ __global__ void __launch_bounds__(256) k_gram(GramArgs a) {
             int grow = r0 + rr;
             int ca = bi * 64 + cc, cb = bj * 64 + cc;
             sa[rr][cc] = (grow < rend && ca < a.c) ? Xb[(size_t)grow * a.c + ca] : 0.f;
-            sb[rr][cc] = (grow < rend && cb < a.c) ? Xb[(size_t)grow * a.c + cb] : 0.f;
+            sb[rr][cc] = (grow < rend && cb < a.c) ? X2b[(size_t)grow * a.c + cb] : 0.f;
         }
         __syncthreads();
 #pragma unroll 4
@@ -552,7 +562,8 @@ __global__ void __launch_bounds__(256) k_gram(GramArgs a) {
 
 // part[c][0][e] <- sum_p part[c][p][e]  (fixed order), so that the single-CTA kernels below read one
 // matrix instead of streaming every partial through one SM.  One thread per entry.
-__global__ void k_gram_sum(double* part, int cc, int nparts, int count) {
+__global__ void k_gram_sum(double* part, int cc, int nparts, int count, const int* skip = nullptr) {
+    if (skip && *skip) return;
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)cc * count) return;
     size_t c = idx / cc, e = idx % cc;
@@ -573,8 +584,10 @@ __host__ __device__ inline int chol_ld(int c) { return c | 1; }
 // `defic` (optional, [count][c]): 1 for every column whose pivot was rejected (zero or dependent column);
 // k_complete replaces those columns of P~ by an orthonormal completion.
 __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int c, int nparts, int* flags,
-                                              int* gate = nullptr, double gate_tol = 0.0, int* defic = nullptr) {
+                                              int* gate = nullptr, double gate_tol = 0.0, int* defic = nullptr,
+                                              const int* skip = nullptr) {
     extern __shared__ __align__(16) double Gs[];  // [c][ld]
+    if (skip && *skip) return;
     __shared__ double dinv[192];
     __shared__ int dcol[192];
     __shared__ int bad, illc;
@@ -715,9 +728,11 @@ struct ApplyArgs {
     float* Xout;      // [count][rows][kout]
     int rows, c, kout, ldt, upper;
     float* XoutT;     // optional transposed copy [count][kout][rows]
+    const int* skip;  // when non-null the kernel does nothing if *skip != 0
 };
 __global__ void __launch_bounds__(256) k_apply(ApplyArgs a) {
     extern __shared__ __align__(16) float xs[];  // [32][c]
+    if (a.skip && *a.skip) return;
     const int row0 = blockIdx.x * 32;
     const float* Xb = a.X + (size_t)blockIdx.y * a.rows * a.c;
     const double* Tb = a.T + (size_t)blockIdx.y * a.c * a.ldt;
@@ -751,8 +766,9 @@ constexpr int JAC_MAX_SWEEPS = 40;
 // leading dimension of the shared-memory matrix: odd number of doubles (no bank conflicts down a column)
 __host__ __device__ inline int jac_ld(int c2) { return c2 | 1; }
 __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, int nparts, int c, int r,
-                                                            double* Vws, double* U, int* flags) {
+                                                            double* Vws, double* U, int* flags, const int* skip = nullptr) {
     extern __shared__ __align__(16) double As[];  // [c2][ld]
+    if (skip && *skip) return;
     __shared__ double cs[128], sn[128];
     __shared__ int pp[128], qq[128];
     __shared__ double offn, diagn;
@@ -861,6 +877,60 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
         int i = e / r, k = e % r;
         Ub[e] = Vt[order[k] * c2 + i];
     }
+}
+
+// ----------------------------------------------------------------------------
+// Stopping test of the refresh: how far the top-r Ritz basis moved between two checks,
+//   d^2 = || Pnew - Pold (Pold^T Pnew) ||_F^2   (no cancellation: Pold is orthonormal to float32 rounding).
+// k_subspace_change forms the per-row-block sums of squares (S = Pold^T Pnew comes from k_gram / k_gram_sum,
+// [r][r] doubles); k_refresh_decide adds them in a fixed order and sets *done when every matrix of the
+// handle has stopped moving (rule below).  grid: (ceil(rows / 64), count), 256 threads, r * r floats of dynamic smem.
+// ----------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_subspace_change(const float* Pold, const float* Pnew, const double* S, size_t s_stride,
+                                                         double* dpart, int rows, int r, const int* skip) {
+    extern __shared__ __align__(16) float Ss[];   // [r][r]
+    __shared__ double red[8];
+    if (skip && *skip) return;
+    const int c = blockIdx.y, tid = threadIdx.x;
+    const double* Sb = S + (size_t)c * s_stride;
+    for (int e = tid; e < r * r; e += 256) Ss[e] = (float)Sb[e];
+    __syncthreads();
+    const int row0 = blockIdx.x * 64;
+    const float* po = Pold + (size_t)c * rows * r;
+    const float* pn = Pnew + (size_t)c * rows * r;
+    double acc = 0.0;
+    for (int e = tid; e < 64 * r; e += 256) {
+        const int row = row0 + e / r, k = e % r;
+        if (row >= rows) continue;
+        float v = pn[(size_t)row * r + k];
+        for (int j = 0; j < r; ++j) v = fmaf(-po[(size_t)row * r + j], Ss[j * r + k], v);
+        acc += (double)v * (double)v;
+    }
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if ((tid & 31) == 0) red[tid >> 5] = acc;
+    __syncthreads();
+    if (tid == 0) {
+        double t = 0.0;
+        for (int w = 0; w < 8; ++w) t += red[w];
+        dpart[(size_t)c * gridDim.x + blockIdx.x] = t;
+    }
+}
+// Rule per matrix (d = movement since the previous check, dprev the one before):
+//   d <= 1e-5 and still halving (d <= dprev / 2: geometric convergence, the error left is below d), or
+//   d <= 3e-6 (the float32 floor of two Ritz bases computed three sweeps apart).
+__global__ void k_refresh_decide(const double* dpart, int nb, int count, double* dprev, int have_prev, int* done) {
+    if (*done) return;
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    int all = 1;
+    for (int c = 0; c < count; ++c) {
+        double t = 0.0;
+        for (int b = 0; b < nb; ++b) t += dpart[(size_t)c * nb + b];
+        const double d = sqrt(t);
+        const bool ok = (d <= 3e-6) || (have_prev && d <= 1e-5 && d <= 0.5 * dprev[c]);
+        if (!ok) all = 0;
+        dprev[c] = d;
+    }
+    if (all) *done = 1;
 }
 
 }  // namespace psgd
