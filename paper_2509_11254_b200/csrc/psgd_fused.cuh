@@ -184,6 +184,23 @@ __device__ __forceinline__ void st_async_cluster_f32(unsigned local_addr, unsign
                  ::"r"(raddr), "r"(__float_as_uint(v)), "r"(rbar) : "memory");
 }
 
+// The same over each half warp (16 lanes) of NV in {8, 16} per-lane values: on return lane l holds the total of
+// value index l & 15 (NV == 16) or (l & 15) >> 1 (NV == 8) of its half in v[0].
+template <int NV>
+__device__ __forceinline__ void butterfly_reduce16(float (&v)[NV], int lane) {
+#pragma unroll
+    for (int o = 8, cnt = NV; cnt > 1; o >>= 1, cnt >>= 1) {
+        const bool up = (lane & o) != 0;
+#pragma unroll
+        for (int j = 0; j < cnt / 2; ++j) {
+            float send = up ? v[j] : v[j + cnt / 2];
+            float keep = up ? v[j + cnt / 2] : v[j];
+            v[j] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+        }
+    }
+    if (NV == 8) v[0] += __shfl_xor_sync(0xffffffffu, v[0], 1);
+}
+
 __device__ __forceinline__ void role_barrier(int id) {   // barrier among the 256 threads of one role
     asm volatile("bar.sync %0, 256;\n" ::"r"(id) : "memory");
 }
@@ -256,13 +273,20 @@ k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CU
         // =====================================================================================
         asm volatile("setmaxnreg.dec.sync.aligned.u32 88;\n");
         const float* Qc = a.Qpad + (size_t)c * n * RP;
-        // warp -> (column group, row group) of a stage, lane -> CPL adjacent columns (fixed for the kernel)
+        // warp -> (column group, row group) of a stage (fixed for the kernel).  Slices of >= 256 columns: a warp
+        // tile is 4 rows x 64 columns, lane -> (2 of the 4 rows, 4 adjacent columns), so that a half warp
+        // covers a row contiguously and only 16 values per lane have to be reduced over 16 lanes.
+        // Slices of 128 columns: 4 rows x 32 columns, lane -> one column.
+        constexpr bool WIDE = (CPL == 2);
+        constexpr int LC = WIDE ? 4 : 1;             // columns per lane
+        constexpr int LR = WIDE ? 2 : FU_RG;         // rows per lane
         const int cgp = warp % NCG, rgl = warp / NCG;
-        const int acol = cgp * 32 * CPL + lane * CPL;                       // column within the slice
+        const int hrow = WIDE ? (lane >> 4) : 0;     // which row pair of the warp tile
+        const int acol = WIDE ? cgp * 64 + 4 * (lane & 15) : cgp * 32 + lane;   // first column within the slice
         const int abox = acol / BW, aboxcol = acol % BW;                    // TMA tile and column inside it
-        f2p Qr[CPL][RP2];        // rows of Q' for this lane's columns, pairs over k
+        f2p Qr[LC][RP2];         // rows of Q' for this lane's columns, pairs over k
 #pragma unroll
-        for (int j = 0; j < CPL; ++j)
+        for (int j = 0; j < LC; ++j)
 #pragma unroll
             for (int k4 = 0; k4 < RP / 4; ++k4) {
                 ulonglong2 v = make_ulonglong2(0ull, 0ull);
@@ -299,9 +323,9 @@ k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CU
             advance_next();
         }
 
-        f2p sacc[FU_RG][RP2];
+        f2p sacc[LR][RP2];
 #pragma unroll
-        for (int rr = 0; rr < FU_RG; ++rr)
+        for (int rr = 0; rr < LR; ++rr)
 #pragma unroll
             for (int k = 0; k < RP2; ++k) sacc[rr][k] = ZERO2;
         int ss = 0, par = 0;                // ring slot and parity of the stage being consumed
@@ -324,16 +348,17 @@ k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CU
 
                     // ---- S = g + stored Delta -> tile; sacc += S Q' ----
                     mbar_wait(bar_full + 8 * ss, (unsigned)par, a.flags, dead);
-                    const float* sgp = ring + (size_t)ss * Ge::STAGE_FLOATS + (size_t)abox * (RS * BW) + (size_t)(rgl * FU_RG) * BW + aboxcol;
+                    const float* sgp = ring + (size_t)ss * Ge::STAGE_FLOATS + (size_t)abox * (RS * BW) + (size_t)(rgl * FU_RG + hrow * LR) * BW + aboxcol;
                     const float* smp = sgp + RS * WC;
-                    float* tp = tile + (((size_t)pbuf * N + i) * FU_R + rc * RS + rgl * FU_RG) * WC + acol;
-                    float sv[FU_RG][CPL];
+                    float* tp = tile + (((size_t)pbuf * N + i) * FU_R + rc * RS + rgl * FU_RG + hrow * LR) * WC + acol;
+                    float sv[LR][LC];
 #pragma unroll
-                    for (int rr = 0; rr < FU_RG; ++rr) {
-                        if (CPL == 2) {
-                            const float2 g2 = *reinterpret_cast<const float2*>(sgp + rr * BW);
-                            const float2 m2 = *reinterpret_cast<const float2*>(smp + rr * BW);
-                            sv[rr][0] = g2.x + m2.x; sv[rr][CPL - 1] = g2.y + m2.y;
+                    for (int rr = 0; rr < LR; ++rr) {
+                        if (WIDE) {
+                            const float4 g4 = *reinterpret_cast<const float4*>(sgp + rr * BW);
+                            const float4 m4 = *reinterpret_cast<const float4*>(smp + rr * BW);
+                            sv[rr][0] = g4.x + m4.x; sv[rr][LC > 1 ? 1 : 0] = g4.y + m4.y;
+                            sv[rr][LC > 2 ? 2 : 0] = g4.z + m4.z; sv[rr][LC > 3 ? 3 : 0] = g4.w + m4.w;
                         } else {
                             sv[rr][0] = sgp[rr * BW] + smp[rr * BW];
                         }
@@ -341,11 +366,11 @@ k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CU
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_empty + 8 * ss);   // the stage is in registers: release the slot
 #pragma unroll
-                    for (int rr = 0; rr < FU_RG; ++rr) {
-                        if (CPL == 2) *reinterpret_cast<float2*>(tp + rr * WC) = make_float2(sv[rr][0], sv[rr][CPL - 1]);
+                    for (int rr = 0; rr < LR; ++rr) {
+                        if (WIDE) *reinterpret_cast<float4*>(tp + rr * WC) = make_float4(sv[rr][0], sv[rr][LC > 1 ? 1 : 0], sv[rr][LC > 2 ? 2 : 0], sv[rr][LC > 3 ? 3 : 0]);
                         else tp[rr * WC] = sv[rr][0];
 #pragma unroll
-                        for (int j = 0; j < CPL; ++j) {
+                        for (int j = 0; j < LC; ++j) {
                             const f2p sd = pack2(sv[rr][j], sv[rr][j]);
 #pragma unroll
                             for (int k2 = 0; k2 < RP2; ++k2) sacc[rr][k2] = ffma2(sd, Qr[j][k2], sacc[rr][k2]);
@@ -354,9 +379,10 @@ k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CU
                     if (++ss == NST) { ss = 0; par ^= 1; }
 
                     if (i == N - 1) {   // the row chunk is complete for every node: reduce over the warp's columns
-                        float v[NV];
+                        constexpr int LV = LR * RP;      // values per lane
+                        float v[LV];
 #pragma unroll
-                        for (int rr = 0; rr < FU_RG; ++rr)
+                        for (int rr = 0; rr < LR; ++rr)
 #pragma unroll
                             for (int k2 = 0; k2 < RP2; ++k2) {
                                 const float2 u = unpack2(sacc[rr][k2]);
@@ -364,10 +390,16 @@ k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CU
                                 v[rr * RP + 2 * k2 + 1] = u.y;
                                 sacc[rr][k2] = ZERO2;
                             }
-                        butterfly_reduce<NV>(v, lane);
                         const int rgi = rc * Ge::NRG + rgl;     // row group within the block (0 or 1)
-                        if (NV == 32 || (lane & 1) == 0)
-                            PpartW[((pbuf * 2 + rgi) * NCG + cgp) * 32 + (NV == 32 ? lane : lane >> 1)] = v[0];
+                        float* pw = PpartW + ((pbuf * 2 + rgi) * NCG + cgp) * 32;   // [row in group][k]
+                        if (WIDE) {
+                            butterfly_reduce16<LV>(v, lane);
+                            if (LV == 16) pw[hrow * LV + (lane & 15)] = v[0];
+                            else if ((lane & 1) == 0) pw[hrow * LV + ((lane & 15) >> 1)] = v[0];
+                        } else {
+                            butterfly_reduce<LV>(v, lane);
+                            if (LV == 32 || (lane & 1) == 0) pw[LV == 32 ? lane : lane >> 1] = v[0];
+                        }
                     }
                 }
             }
