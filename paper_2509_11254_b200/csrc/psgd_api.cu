@@ -32,6 +32,7 @@ struct Layout {
     size_t dbarT, Yt, Zt, gpart;                              // tensor-core refresh only
     size_t rtP, rtQ;                                          // tensor-core residual (r > 16) only
     size_t Pold, dpart;                                       // stopping test of the refresh
+    size_t ptQ;                                               // tensor-core projection: split transposed Q
 };
 
 struct ProfEvent {
@@ -48,6 +49,8 @@ struct psgd_handle {
     int error_form = 0, mode = 0, refresh_iters = 20, oversample = -1, refresh_tc = 1, power_steps = 1, refresh_adaptive = 1;
     bool tc_ok = false;           // the refresh block is wide enough for the tensor-core sweeps
     size_t gpart_floats = 0;
+    bool ptc_ok = false;          // projections of more than 16 columns on the tensor cores
+    int ptc_ncp = 0;
     bool rtc_ok = false;          // ranks above 16 with 16-byte row strides: residual update on the tensor cores
     int rtc_KP = 0;
     int64_t t = 0;
@@ -141,6 +144,12 @@ void plan(psgd_handle* h) {
         size_t g2 = gemm_tc_splits(h->n, h->m, h->count) * cnt * n * ncp;
         h->gpart_floats = std::max(g1, g2);
         L.gpart = take(h->gpart_floats * 4);
+    }
+    // ---- projection on the tensor cores (r > 16, or refresh blocks of 17..128 columns) ----
+    h->ptc_ok = (h->r > 16 || ell > 16) && h->n % 4 == 0;
+    if (h->ptc_ok) {
+        h->ptc_ncp = (int)align_up(std::min<size_t>(128, std::max(r, ell)), 16);
+        L.ptQ = take(3 * cnt * (size_t)h->ptc_ncp * n * 4);
     }
     // ---- residual update on the tensor cores: split (head + tail) padded copies of P~ and Q_i ----
     h->rtc_ok = h->r > 16 && h->n % 4 == 0;
@@ -313,9 +322,40 @@ void launch_project_rp(Launcher& L, const ProjectArgs& a, int count, bool vec, b
         else launch_project_t<RP, 1, false, false>(L, a, count);
     }
 }
+// Tensor-core form for more than 16 columns (exactly split TF32 products, see psgd_gemm_tc.cuh).
+bool launch_project_tc(Launcher& L, const float* A, const float* B, float* Mout, const float* Q, float* P, int rows, int n,
+                       int r, int nodes, int count, const int* skip) {
+    psgd_handle* h = L.h;
+    const int Ncp = (int)align_up(r, 16);
+    if (!h->ptc_ok || Ncp > h->ptc_ncp || r > 128 || !aligned16(A) || (B && !aligned16(B)) || (Mout && !aligned16(Mout))) return false;
+    const int mats = count * nodes;
+    float* Qt = (float*)(h->ws + h->lay.ptQ);
+    const size_t tot = (size_t)count * Ncp * n;
+    L.begin(PSGD_K_PROJECT);
+    k_split_pad_t<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Q, Qt, n, r, Ncp, count, skip);
+    L.end();
+    CUtensorMap tA, tB, tQ[3];
+    bool ok = make_tile_map(&tA, A, n, rows, mats, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) &&
+              make_tile_map(&tB, B ? B : A, n, rows, mats, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B);
+    for (int t = 0; t < 3 && ok; ++t) ok = make_tile_map(&tQ[t], Qt + t * tot, n, Ncp, count, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!ok) {
+        snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
+        L.status = PSGD_E_CUDA;
+        return true;
+    }
+    ProjTcArgs a{B ? Mout : nullptr, P, rows, n, r, Ncp, proj_tc_stages(Ncp), B ? 1 : 0, nodes, (int*)(h->ws + h->lay.flags), skip};
+    size_t smem = proj_tc_smem_bytes(Ncp);
+    cudaFuncSetAttribute(k_project_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    L.begin(PSGD_K_PROJECT);
+    k_project_tc<<<dim3(ceil_div(rows, TC_BM), mats), PT_THREADS, smem, L.st>>>(tA, tB, tQ[0], tQ[1], tQ[2], a);
+    L.end();
+    return true;
+}
+
 // P = (A [+B]) Q for all matrices; `add` also stores A+B into Mout.
 void launch_project(Launcher& L, const float* A, const float* B, float* Mout, const float* Q, float* P, int rows, int n,
                     int r, int nodes, int count, bool vec, const int* skip = nullptr) {
+    if (r > 16 && launch_project_tc(L, A, B, Mout, Q, P, rows, n, r, nodes, count, skip)) return;
     ProjectArgs a{A, B, Mout, Q, P, rows, n, r, nodes, 1, skip};
     bool add = B != nullptr;
     vec = vec && aligned16(A) && (!B || aligned16(B)) && (!Mout || aligned16(Mout));
@@ -460,7 +500,7 @@ void ssp(Launcher& L, psgd_handle* h, const float* G) {
     float* Pmean = (float*)(ws + h->lay.Pmean);
     float* Phat = (float*)(ws + h->lay.Phat);
     const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count;
-    if (r <= 32) {
+    if (r <= 32 || (h->ptc_ok && aligned16(G))) {
         launch_project(L, G, h->E, h->E, h->Q, Pnode, m, n, r, N, cnt, h->vec4);
     } else {
         L.begin(PSGD_K_PROJECT);

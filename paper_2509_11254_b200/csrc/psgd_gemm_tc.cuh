@@ -407,3 +407,212 @@ k_residual_tc(const __grid_constant__ CUtensorMap tmPh, const __grid_constant__ 
 }
 
 }  // namespace psgd
+
+namespace psgd {
+
+// ---------------------------------------------------------------------------------------------
+// Projection on the tensor cores for ranks above 16:  P_i = (A_i [+ B_i]) Q  (Algorithm 1: P^(i) <-
+// Delta^(i) Q, with the error-feedback add of Eq. (7a) fused in; optionally stores M = A + B).
+// Per 32-column K block TMA brings the 128 x 32 tiles of A and B (128-byte swizzled); eight
+// converter warps form M in place, split it exactly into three TF32 terms (h + m + l, the head being
+// M itself, which the tensor core reads as TF32), write M back to HBM and hand the three tiles to
+// the MMA thread; Q^T arrives pre-split (k_split_pad_t).  Six tcgen05.mma products per 8 of K go
+// into two tensor-memory accumulators (h*h / the small terms); their sum is the float32-accurate P.
+// ---------------------------------------------------------------------------------------------
+constexpr int PT_THREADS = 320;   // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-9: converters (2-5 also epilogue)
+
+struct ProjTcArgs {
+    float* Mout;      // [mats][rows][n] or nullptr
+    float* P;         // [mats][rows][r]
+    int rows, n, r, Ncp, stages, has_b;
+    int nodes;        // matrices per Q
+    int* flags;
+    const int* skip;
+};
+
+__host__ __device__ inline size_t proj_tc_stage_bytes(int Ncp) { return (size_t)3 * TC_BM * TC_BK * 4 + (size_t)3 * Ncp * TC_BK * 4; }
+__host__ __device__ inline int proj_tc_stages(int Ncp) {
+    int s = (int)((size_t)220 * 1024 / proj_tc_stage_bytes(Ncp));
+    return s > 4 ? 4 : (s < 2 ? 2 : s);
+}
+__host__ __device__ inline size_t proj_tc_smem_bytes(int Ncp) { return (size_t)proj_tc_stages(Ncp) * proj_tc_stage_bytes(Ncp) + 1024 + 256; }
+
+// Q [count][n][r] -> Qt[t][count][Ncp][n], t = 0, 1, 2: the transposed factor split exactly into three TF32 terms,
+// rows k >= r zero.  One thread per (matrix, k, column).
+__global__ void k_split_pad_t(const float* Q, float* Qt, int n, int r, int Ncp, int count, const int* skip) {
+    if (skip && *skip) return;
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t per = (size_t)Ncp * n, tot = per * count;
+    if (idx >= tot) return;
+    const int c = (int)(idx / per);
+    const int k = (int)((idx % per) / n), col = (int)(idx % n);
+    float x = (k < r) ? Q[((size_t)c * n + col) * r + k] : 0.f;
+    float h = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
+    float r1 = x - h;
+    float mm = __uint_as_float(__float_as_uint(r1) & 0xFFFFE000u);
+    Qt[idx] = h;
+    Qt[tot + idx] = mm;
+    Qt[2 * tot + idx] = r1 - mm;
+}
+
+__global__ void __launch_bounds__(PT_THREADS, 1)
+k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+             const __grid_constant__ CUtensorMap tmQ0, const __grid_constant__ CUtensorMap tmQ1, const __grid_constant__ CUtensorMap tmQ2,
+             ProjTcArgs a) {
+    extern __shared__ __align__(16) unsigned char pt_smem_raw[];
+    if (a.skip && *a.skip) return;
+    unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pt_smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr unsigned A_BYTES = TC_BM * TC_BK * 4;
+    const unsigned B_BYTES = (unsigned)a.Ncp * TC_BK * 4;
+    const unsigned STAGE_BYTES = 3 * A_BYTES + 3 * B_BYTES;
+    const int NS = a.stages;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(base + (size_t)NS * STAGE_BYTES);
+    const unsigned bar_full = smem_u32(bars), bar_conv = bar_full + 8 * NS, bar_empty = bar_conv + 8 * NS, bar_acc = bar_empty + 8 * NS;
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 3 * NS + 1);
+    const unsigned smem_base = smem_u32(base);
+
+    const int rt = blockIdx.x, mat = blockIdx.y;
+    const int qz = mat / a.nodes;
+    const int KB = (a.n + TC_BK - 1) / TC_BK;
+    unsigned ncols = 32;
+    while ((int)ncols < 2 * a.Ncp) ncols <<= 1;
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_conv + 8 * s, 8); mbar_init(bar_empty + 8 * s, 1); }
+        mbar_init(bar_acc, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(ncols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    const unsigned tmem = *tmem_slot;
+    bool dead = false;
+
+    if (warp == 0) {
+        // ---- TMA producer ----
+        if (lane == 0) {
+            const unsigned tx = (a.has_b ? 2u : 1u) * A_BYTES + 3u * B_BYTES;
+            for (int kb = 0; kb < KB; ++kb) {
+                const int s = kb % NS;
+                if (kb >= NS) mbar_wait(bar_empty + 8 * s, (unsigned)((kb / NS - 1) & 1), a.flags, dead);
+                const unsigned dst = smem_base + s * STAGE_BYTES;
+                const unsigned bar = bar_full + 8 * s;
+                mbar_expect_tx(bar, tx);
+                tma_load_3d_sw(dst, &tmA, kb * TC_BK, rt * TC_BM, mat, bar);
+                if (a.has_b) tma_load_3d_sw(dst + A_BYTES, &tmB, kb * TC_BK, rt * TC_BM, mat, bar);
+                tma_load_3d_sw(dst + 3 * A_BYTES, &tmQ0, kb * TC_BK, 0, qz, bar);
+                tma_load_3d_sw(dst + 3 * A_BYTES + B_BYTES, &tmQ1, kb * TC_BK, 0, qz, bar);
+                tma_load_3d_sw(dst + 3 * A_BYTES + 2 * B_BYTES, &tmQ2, kb * TC_BK, 0, qz, bar);
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer ----
+        if (lane == 0) {
+            const unsigned idesc = tc_idesc(a.Ncp);
+            const unsigned d_big = tmem, d_small = tmem + (unsigned)a.Ncp;
+            const int tp[6] = {2, 0, 1, 1, 0, 0}, tq[6] = {0, 2, 1, 0, 1, 0};   // (M term, Q term), h = 0, m = 1, l = 2
+            for (int kb = 0; kb < KB; ++kb) {
+                const int s = kb % NS;
+                mbar_wait(bar_conv + 8 * s, (unsigned)((kb / NS) & 1), a.flags, dead);
+                asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                const unsigned sb = smem_base + s * STAGE_BYTES;
+                const unsigned long long dA[3] = {tc_smem_desc(sb), tc_smem_desc(sb + A_BYTES), tc_smem_desc(sb + 2 * A_BYTES)};
+                const unsigned long long dQ[3] = {tc_smem_desc(sb + 3 * A_BYTES), tc_smem_desc(sb + 3 * A_BYTES + B_BYTES),
+                                                  tc_smem_desc(sb + 3 * A_BYTES + 2 * B_BYTES)};
+#pragma unroll
+                for (int k = 0; k < TC_BK / 8; ++k) {
+                    const unsigned long long o = (unsigned long long)(2 * k);
+#pragma unroll
+                    for (int t = 0; t < 6; ++t) {
+                        const unsigned acc = (kb > 0 || k > 0 || (t > 0 && t < 5)) ? 1u : 0u;
+                        asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
+                                     ::"r"(t == 5 ? d_big : d_small), "l"(dA[tp[t]] + o), "l"(dQ[tq[t]] + o), "r"(idesc), "r"(acc) : "memory");
+                    }
+                }
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_empty + 8 * s) : "memory");
+            }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_acc) : "memory");
+        }
+    } else {
+        // ---- converters: M = A + B in place, exact three-way split, M back to HBM ----
+        const int ct = tid - 64;                       // 0 .. 255
+        for (int kb = 0; kb < KB; ++kb) {
+            const int s = kb % NS;
+            mbar_wait(bar_full + 8 * s, (unsigned)((kb / NS) & 1), a.flags, dead);
+            float4* t0 = reinterpret_cast<float4*>(base + (size_t)s * STAGE_BYTES);
+            float4* t1 = t0 + A_BYTES / 16;
+            float4* t2 = t1 + A_BYTES / 16;
+#pragma unroll
+            for (int u = 0; u < (TC_BM * TC_BK / 4) / 256; ++u) {
+                const int o = ct + u * 256;             // 16-byte unit of the swizzled tile
+                float4 mv = t0[o];
+                if (a.has_b) {
+                    const float4 e = t1[o];
+                    mv.x += e.x; mv.y += e.y; mv.z += e.z; mv.w += e.w;
+                    t0[o] = mv;                         // head: M itself (read as TF32 by the tensor core)
+                    if (a.Mout) {
+                        const int row = o >> 3, lc = (o & 7) ^ (row & 7);      // undo the 128-byte swizzle
+                        const int grow = rt * TC_BM + row, gcol = kb * TC_BK + lc * 4;
+                        if (grow < a.rows && gcol < a.n)
+                            *reinterpret_cast<float4*>(a.Mout + ((size_t)mat * a.rows + grow) * a.n + gcol) = mv;
+                    }
+                }
+                float4 d, mm, ll;
+                const float xs[4] = {mv.x, mv.y, mv.z, mv.w};
+                float ms[4], ls[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float h = __uint_as_float(__float_as_uint(xs[j]) & 0xFFFFE000u);
+                    const float r1 = xs[j] - h;
+                    ms[j] = __uint_as_float(__float_as_uint(r1) & 0xFFFFE000u);
+                    ls[j] = r1 - ms[j];
+                }
+                mm = make_float4(ms[0], ms[1], ms[2], ms[3]);
+                ll = make_float4(ls[0], ls[1], ls[2], ls[3]);
+                (void)d;
+                t1[o] = mm;
+                t2[o] = ll;
+            }
+            asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");    // generic writes -> visible to the tensor core
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_conv + 8 * s);
+        }
+        if (warp < 6) {
+            // ---- epilogue (warps 2-5): P = big + small accumulator ----
+            mbar_wait(bar_acc, 0u, a.flags, dead);
+            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+            const int quarter = warp & 3;
+            const int row = rt * TC_BM + quarter * 32 + lane;
+            float* out = a.P + ((size_t)mat * a.rows + (row < a.rows ? row : 0)) * a.r;
+            for (int col = 0; col < a.Ncp; col += 8) {
+                unsigned rb[8], rs[8];
+                const unsigned taddr = tmem + ((unsigned)(quarter * 32) << 16) + (unsigned)col;
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
+                             : "=r"(rb[0]), "=r"(rb[1]), "=r"(rb[2]), "=r"(rb[3]), "=r"(rb[4]), "=r"(rb[5]), "=r"(rb[6]), "=r"(rb[7])
+                             : "r"(taddr) : "memory");
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
+                             : "=r"(rs[0]), "=r"(rs[1]), "=r"(rs[2]), "=r"(rs[3]), "=r"(rs[4]), "=r"(rs[5]), "=r"(rs[6]), "=r"(rs[7])
+                             : "r"(taddr + (unsigned)a.Ncp) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+                if (row < a.rows) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (col + j < a.r) out[col + j] = __uint_as_float(rb[j]) + __uint_as_float(rs[j]);
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(ncols) : "memory");
+    }
+}
+
+}  // namespace psgd
