@@ -149,7 +149,7 @@ void plan(psgd_handle* h) {
     h->ptc_ok = (h->r > 16 || ell > 16) && h->n % 4 == 0;
     if (h->ptc_ok) {
         h->ptc_ncp = (int)align_up(std::min<size_t>(128, std::max(r, ell)), 16);
-        L.ptQ = take(3 * cnt * (size_t)h->ptc_ncp * n * 4);
+        L.ptQ = take(3 * cnt * (size_t)h->ptc_ncp * std::max(m, n) * 4);   // split Q^T (projection) or P~^T (back-projection)
     }
     // ---- residual update on the tensor cores: split (head + tail) padded copies of P~ and Q_i ----
     h->rtc_ok = h->r > 16 && h->n % 4 == 0;
@@ -379,13 +379,63 @@ void launch_back_rp(Launcher& L, BackArgs a, int mats, bool vec) {
     else k_backproject<RP, 1><<<grid, BP_THREADS, 0, L.st>>>(a);
     L.end();
 }
-void launch_back(Launcher& L, const float* M, const float* Phat, float* part, int rows, int n, int r, int nodes,
+// Tensor-core form for more than 16 columns (M as the MN-major operand, see psgd_gemm_tc.cuh).  Picks its own number of
+// row splits (at most S, the number the partial buffer was sized for) and returns it, 0 if the shape is not eligible.
+int launch_back_tc(Launcher& L, const float* M, const float* Phat, float* part, int rows, int n, int r, int nodes, int count,
+                   int S, const int* skip) {
+    psgd_handle* h = L.h;
+    const int Ncp = (int)align_up(r, 16);
+    if (!h->ptc_ok || Ncp > h->ptc_ncp || r > 128 || rows % 4 != 0 || !aligned16(M)) return 0;
+    const int mats = count * nodes;
+    const int KB = ceil_div(rows, TC_BK);
+    const int64_t base = (int64_t)ceil_div(n, TC_BM) * mats;
+    int best = 1;
+    int64_t best_cost = -1;
+    for (int s = 1; s <= std::min(S, 32); ++s) {       // cost: waves x (K blocks per CTA + fixed start-up and epilogue)
+        const int kbs = ceil_div(KB, s);
+        if (s > 1 && kbs < 16) break;
+        if ((int64_t)(s - 1) * kbs >= KB) continue;     // would leave an empty split
+        const int64_t cost = ((base * s + 147) / 148) * (kbs + 8);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+    }
+    if (const char* e = getenv("PSGD_BTC_OFF")) { if (atoi(e)) return 0; }   // PROBE
+    if (const char* e = getenv("PSGD_BTC_KBS")) { int k = atoi(e); if (k > 0) { best = std::min(S, ceil_div(KB, k)); } }   // PROBE
+    const int St = best, kbs = ceil_div(KB, St);
+    float* Pt = (float*)(h->ws + h->lay.ptQ);
+    const size_t tot = (size_t)count * Ncp * rows;
+    L.begin(PSGD_K_BACKPROJECT);
+    k_split_pad_t<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Phat, Pt, rows, r, Ncp, count, skip);
+    L.end();
+    CUtensorMap tM, tP[3];
+    bool ok = make_tile_map(&tM, M, n, rows, mats, 32, TC_BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
+    for (int t = 0; t < 3 && ok; ++t) ok = make_tile_map(&tP[t], Pt + t * tot, rows, Ncp, count, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!ok) {
+        snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
+        L.status = PSGD_E_CUDA;
+        return St;
+    }
+    BackTcArgs a{part, rows, n, r, Ncp, proj_tc_stages(Ncp), St, kbs, nodes, (int*)(h->ws + h->lay.flags), skip};
+    size_t smem = proj_tc_smem_bytes(Ncp);
+    cudaFuncSetAttribute(k_backproject_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    L.begin(PSGD_K_BACKPROJECT);
+    k_backproject_tc<<<dim3(ceil_div(n, TC_BM), St, mats), PT_THREADS, smem, L.st>>>(tM, tP[0], tP[1], tP[2], a);
+    L.end();
+    return St;
+}
+
+// Q_i partial sums for all matrices; returns the number of row splits written (the S to hand to k_reduce_q).
+int launch_back(Launcher& L, const float* M, const float* Phat, float* part, int rows, int n, int r, int nodes,
                  int count, int rpc, int S, bool vec, const int* gate = nullptr, const int* skip = nullptr) {
+    if (r > 16 && !gate) {
+        const int St = launch_back_tc(L, M, Phat, part, rows, n, r, nodes, count, S, skip);
+        if (St > 0) return St;
+    }
     BackArgs a{M, Phat, part, rows, n, r, nodes, 1, rpc, S, gate, skip};
     vec = vec && aligned16(M);
     if (r <= 4) launch_back_rp<4>(L, a, count * nodes, vec);
     else if (r <= 8) launch_back_rp<8>(L, a, count * nodes, vec);
     else launch_back_rp<16>(L, a, count * nodes, vec);
+    return S;
 }
 
 // ---- K4 dispatch ------------------------------------------------------------
@@ -481,10 +531,10 @@ void tail(Launcher& L, psgd_handle* h, float* D_hat) {
     float* Qnode = (float*)(ws + h->lay.Qnode);
     float* part = (float*)(ws + h->lay.part);
     const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count;
-    launch_back(L, h->E, Phat, part, m, n, r, N, cnt, h->rpc, h->S, h->vec4);
+    const int Sb = launch_back(L, h->E, Phat, part, m, n, r, N, cnt, h->rpc, h->S, h->vec4);
     size_t tot = (size_t)cnt * n * r;
     L.begin(PSGD_K_BACKPROJECT);
-    k_reduce_q<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(part, Qnode, h->Q, n, r, N, h->S, cnt);
+    k_reduce_q<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(part, Qnode, h->Q, n, r, N, Sb, cnt);
     L.end();
     if (h->error_form == 0)
         launch_resid(L, h->E, h->E, Phat, Qnode, m, n, r, N, cnt * N, 1, 1, h->vec4);
@@ -518,10 +568,10 @@ void ssp(Launcher& L, psgd_handle* h, const float* G) {
     float* Qnode = (float*)(ws + h->lay.Qnode);
     float* part = (float*)(ws + h->lay.part);
     for (int k = 1; k < h->power_steps; ++k) {
-        launch_back(L, h->E, Phat, part, m, n, r, N, cnt, h->rpc, h->S, h->vec4);
+        const int Sb = launch_back(L, h->E, Phat, part, m, n, r, N, cnt, h->rpc, h->S, h->vec4);
         size_t tq = (size_t)cnt * n * r;
         L.begin(PSGD_K_BACKPROJECT);
-        k_reduce_q<<<(unsigned)((tq + 255) / 256), 256, 0, L.st>>>(part, Qnode, h->Q, n, r, N, h->S, cnt);
+        k_reduce_q<<<(unsigned)((tq + 255) / 256), 256, 0, L.st>>>(part, Qnode, h->Q, n, r, N, Sb, cnt);
         L.end();
         launch_project(L, h->E, nullptr, nullptr, h->Q, Pnode, m, n, r, N, cnt, h->vec4);
         L.begin(PSGD_K_ORTH);
@@ -621,10 +671,10 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
         // Y = Dbar Z, orthonormalise;  Z = Dbar^T Y, orthonormalise
         launch_project(L, dbar, nullptr, nullptr, Z, Y, m, n, ell, 1, cnt, h->vec4, skip);
         launch_orth(L, h, Y, Y, m, ell, K, nullptr, false, skip);
-        launch_back(L, dbar, Y, part, m, n, ell, 1, cnt, rpc, S, h->vec4, nullptr, skip);
+        const int Sb = launch_back(L, dbar, Y, part, m, n, ell, 1, cnt, rpc, S, h->vec4, nullptr, skip);
         size_t tot = (size_t)cnt * n * ell;
         L.begin(K);
-        k_reduce_q<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(part, nullptr, Z, n, ell, 1, S, cnt, skip);
+        k_reduce_q<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(part, nullptr, Z, n, ell, 1, Sb, cnt, skip);
         L.end();
         if (it + 1 == h->refresh_iters) break;
         if (adaptive && (it - it0 + 1) % 3 == 0) {

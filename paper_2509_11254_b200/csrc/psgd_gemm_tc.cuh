@@ -416,10 +416,24 @@ namespace psgd {
 // Per 32-column K block TMA brings the 128 x 32 tiles of A and B (128-byte swizzled); eight
 // converter warps form M in place, split it exactly into three TF32 terms (h + m + l, the head being
 // M itself, which the tensor core reads as TF32), write M back to HBM and hand the three tiles to
-// the MMA thread; Q^T arrives pre-split (k_split_pad_t).  Six tcgen05.mma products per 8 of K go
-// into two tensor-memory accumulators (h*h / the small terms); their sum is the float32-accurate P.
+// the MMA thread; Q^T arrives pre-split (k_split_pad_t).  Of the six tcgen05.mma products per 8 of K
+// the five small ones go into one tensor-memory accumulator; the head product h*h goes through the
+// rotating accumulators described below and is summed in float32 registers.
 // ---------------------------------------------------------------------------------------------
-constexpr int PT_THREADS = 320;   // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-9: converters (2-5 also epilogue)
+constexpr int PT_THREADS = 320;   // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-9: converters, adders, epilogue
+// The tensor core adds to its float32 accumulator with truncation (measured on like-signed sums: 3e-8 relative per
+// accumulation, always toward zero, i.e. 2e-5 over the 512 steps of a 4096-long contraction).  The head product h*h
+// therefore accumulates only BT_F steps in tensor memory: BT_NB accumulators take turns and the converter warps add
+// each finished one to float32 registers (round to nearest) while the next ones fill.
+constexpr int BT_NB = 3;    // head accumulators in rotation
+constexpr int BT_F = 2;     // MMA steps (8 of K each) per head accumulator before it is added up in registers
+constexpr int BT_MAXG = 8;  // 8-column groups per thread: (Ncp / 2) / 8 for Ncp <= 128
+
+__device__ __forceinline__ void tmem_ld8(unsigned taddr, unsigned (&v)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "r"(taddr) : "memory");
+}
 
 struct ProjTcArgs {
     float* Mout;      // [mats][rows][n] or nullptr
@@ -464,22 +478,25 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pt_smem_raw) + 1023) & ~(uintptr_t)1023);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr unsigned A_BYTES = TC_BM * TC_BK * 4;
+    constexpr int CPB = (TC_BK / 8) / BT_F;                    // head chunks per K block
     const unsigned B_BYTES = (unsigned)a.Ncp * TC_BK * 4;
     const unsigned STAGE_BYTES = 3 * A_BYTES + 3 * B_BYTES;
     const int NS = a.stages;
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(base + (size_t)NS * STAGE_BYTES);
-    const unsigned bar_full = smem_u32(bars), bar_conv = bar_full + 8 * NS, bar_empty = bar_conv + 8 * NS, bar_acc = bar_empty + 8 * NS;
-    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 3 * NS + 1);
+    const unsigned bar_full = smem_u32(bars), bar_conv = bar_full + 8 * NS, bar_empty = bar_conv + 8 * NS;
+    const unsigned bar_hfull = bar_empty + 8 * NS, bar_hfree = bar_hfull + 8 * BT_NB, bar_acc = bar_hfree + 8 * BT_NB;
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 3 * NS + 2 * BT_NB + 1);
     const unsigned smem_base = smem_u32(base);
 
     const int rt = blockIdx.x, mat = blockIdx.y;
     const int qz = mat / a.nodes;
     const int KB = (a.n + TC_BK - 1) / TC_BK;
     unsigned ncols = 32;
-    while ((int)ncols < 2 * a.Ncp) ncols <<= 1;
+    while ((int)ncols < (BT_NB + 1) * a.Ncp) ncols <<= 1;
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_conv + 8 * s, 8); mbar_init(bar_empty + 8 * s, 1); }
+        for (int b = 0; b < BT_NB; ++b) { mbar_init(bar_hfull + 8 * b, 1); mbar_init(bar_hfree + 8 * b, 8); }
         mbar_init(bar_acc, 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -490,7 +507,7 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-    const unsigned tmem = *tmem_slot;
+    const unsigned tmem = *tmem_slot;      // small accumulator at column 0, head accumulator b at (1 + b) * Ncp
     bool dead = false;
 
     if (warp == 0) {
@@ -514,8 +531,9 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         // ---- MMA issuer ----
         if (lane == 0) {
             const unsigned idesc = tc_idesc(a.Ncp);
-            const unsigned d_big = tmem, d_small = tmem + (unsigned)a.Ncp;
+            const unsigned d_small = tmem;
             const int tp[6] = {2, 0, 1, 1, 0, 0}, tq[6] = {0, 2, 1, 0, 1, 0};   // (M term, Q term), h = 0, m = 1, l = 2
+            int chunk = 0;
             for (int kb = 0; kb < KB; ++kb) {
                 const int s = kb % NS;
                 mbar_wait(bar_conv + 8 * s, (unsigned)((kb / NS) & 1), a.flags, dead);
@@ -526,12 +544,22 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                                                   tc_smem_desc(sb + 3 * A_BYTES + 2 * B_BYTES)};
 #pragma unroll
                 for (int k = 0; k < TC_BK / 8; ++k) {
+                    const int hb = chunk % BT_NB;
+                    if (k % BT_F == 0 && chunk >= BT_NB) {     // the registers have taken this accumulator's last content
+                        mbar_wait(bar_hfree + 8 * hb, (unsigned)((chunk / BT_NB - 1) & 1), a.flags, dead);
+                        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                    }
+                    const unsigned d_head = tmem + (unsigned)((1 + hb) * a.Ncp);
                     const unsigned long long o = (unsigned long long)(2 * k);
 #pragma unroll
                     for (int t = 0; t < 6; ++t) {
-                        const unsigned acc = (kb > 0 || k > 0 || (t > 0 && t < 5)) ? 1u : 0u;
+                        const unsigned acc = (t == 5) ? ((k % BT_F != 0) ? 1u : 0u) : ((kb > 0 || k > 0 || t > 0) ? 1u : 0u);
                         asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
-                                     ::"r"(t == 5 ? d_big : d_small), "l"(dA[tp[t]] + o), "l"(dQ[tq[t]] + o), "r"(idesc), "r"(acc) : "memory");
+                                     ::"r"(t == 5 ? d_head : d_small), "l"(dA[tp[t]] + o), "l"(dQ[tq[t]] + o), "r"(idesc), "r"(acc) : "memory");
+                    }
+                    if (k % BT_F == BT_F - 1) {
+                        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_hfull + 8 * hb) : "memory");
+                        ++chunk;
                     }
                 }
                 asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_empty + 8 * s) : "memory");
@@ -539,8 +567,43 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_acc) : "memory");
         }
     } else {
-        // ---- converters: M = A + B in place, exact three-way split, M back to HBM ----
+        // ---- converters / adders (warps 2-9): M = A + B in place, exact three-way split, M back to HBM ----
         const int ct = tid - 64;                       // 0 .. 255
+        const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
+        const int half = (warp - 2) >> 2;              // which half of the columns this warp adds up
+        const int ng = a.Ncp >> 4;                     // 8-column groups per thread
+        const unsigned lane_base = (unsigned)(quarter * 32) << 16;
+        const unsigned col_base = (unsigned)(half * (a.Ncp >> 1));
+        float acc[BT_MAXG][8];
+#pragma unroll
+        for (int g = 0; g < BT_MAXG; ++g)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
+        // adds head accumulator (chunk c) to the registers and hands it back to the MMA thread
+        auto drain = [&](int c) {
+            const int hb = c % BT_NB;
+            mbar_wait(bar_hfull + 8 * hb, (unsigned)((c / BT_NB) & 1), a.flags, dead);
+            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+            const unsigned t0 = tmem + lane_base + (unsigned)((1 + hb) * a.Ncp) + col_base;
+#pragma unroll
+            for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
+                if (g2 < ng) {
+                    unsigned v0[8], v1[8];
+                    tmem_ld8(t0 + 8 * g2, v0);
+                    if (g2 + 1 < ng) tmem_ld8(t0 + 8 * (g2 + 1), v1);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc[g2][j] += __uint_as_float(v0[j]);
+                    if (g2 + 1 < ng) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) acc[g2 + 1][j] += __uint_as_float(v1[j]);
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_hfree + 8 * hb);
+        };
         for (int kb = 0; kb < KB; ++kb) {
             const int s = kb % NS;
             mbar_wait(bar_full + 8 * s, (unsigned)((kb / NS) & 1), a.flags, dead);
@@ -562,7 +625,6 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                             *reinterpret_cast<float4*>(a.Mout + ((size_t)mat * a.rows + grow) * a.n + gcol) = mv;
                     }
                 }
-                float4 d, mm, ll;
                 const float xs[4] = {mv.x, mv.y, mv.z, mv.w};
                 float ms[4], ls[4];
 #pragma unroll
@@ -572,37 +634,273 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     ms[j] = __uint_as_float(__float_as_uint(r1) & 0xFFFFE000u);
                     ls[j] = r1 - ms[j];
                 }
-                mm = make_float4(ms[0], ms[1], ms[2], ms[3]);
-                ll = make_float4(ls[0], ls[1], ls[2], ls[3]);
-                (void)d;
-                t1[o] = mm;
-                t2[o] = ll;
+                t1[o] = make_float4(ms[0], ms[1], ms[2], ms[3]);
+                t2[o] = make_float4(ls[0], ls[1], ls[2], ls[3]);
             }
             asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");    // generic writes -> visible to the tensor core
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_conv + 8 * s);
+            // one K block behind the conversion: the head products of block kb - 1 are done or nearly so
+            if (kb > 0) {
+#pragma unroll
+                for (int c = 0; c < CPB; ++c) drain((kb - 1) * CPB + c);
+            }
         }
-        if (warp < 6) {
-            // ---- epilogue (warps 2-5): P = big + small accumulator ----
-            mbar_wait(bar_acc, 0u, a.flags, dead);
-            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-            const int quarter = warp & 3;
-            const int row = rt * TC_BM + quarter * 32 + lane;
-            float* out = a.P + ((size_t)mat * a.rows + (row < a.rows ? row : 0)) * a.r;
-            for (int col = 0; col < a.Ncp; col += 8) {
-                unsigned rb[8], rs[8];
-                const unsigned taddr = tmem + ((unsigned)(quarter * 32) << 16) + (unsigned)col;
-                asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
-                             : "=r"(rb[0]), "=r"(rb[1]), "=r"(rb[2]), "=r"(rb[3]), "=r"(rb[4]), "=r"(rb[5]), "=r"(rb[6]), "=r"(rb[7])
-                             : "r"(taddr) : "memory");
-                asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
-                             : "=r"(rs[0]), "=r"(rs[1]), "=r"(rs[2]), "=r"(rs[3]), "=r"(rs[4]), "=r"(rs[5]), "=r"(rs[6]), "=r"(rs[7])
-                             : "r"(taddr + (unsigned)a.Ncp) : "memory");
+        if (KB > 0) {
+#pragma unroll
+            for (int c = 0; c < CPB; ++c) drain((KB - 1) * CPB + c);
+        }
+        // ---- epilogue: P = registers + small accumulator ----
+        mbar_wait(bar_acc, 0u, a.flags, dead);
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        const int row = rt * TC_BM + quarter * 32 + lane;
+        float* out = a.P + ((size_t)mat * a.rows + (row < a.rows ? row : 0)) * a.r;
+#pragma unroll
+        for (int g = 0; g < BT_MAXG; ++g) {
+            if (g < ng) {
+                unsigned v[8];
+                tmem_ld8(tmem + lane_base + col_base + 8 * g, v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
                 if (row < a.rows) {
+                    const int j0 = (int)col_base + 8 * g;
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        if (col + j < a.r) out[col + j] = __uint_as_float(rb[j]) + __uint_as_float(rs[j]);
+                        if (j0 + j < a.r) out[j0 + j] = acc[g][j] + __uint_as_float(v[j]);
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(ncols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Back-projection on the tensor cores for more than 16 columns:  Q_i = M_i^T P~  (Algorithm 1:
+// Q^(i) <- (Delta^(i))^T P~).  The contraction runs over the rows of M, so the tile of M is the
+// MN-major operand: TMA brings 32-row x 32-column boxes of M exactly as they lie in memory (128-byte
+// lines, 32-byte swizzle atoms, the one shared-memory form TF32 operands have in this orientation);
+// four boxes side by side give the 128 columns of one CTA.  P~^T arrives pre-split and K-major
+// (k_split_pad_t on P~).  Converters split the tile of M exactly into three TF32 terms; of the six
+// tcgen05.mma products per 8 rows the five small ones go into one tensor-memory accumulator for the
+// whole split; the head product h*h goes through the rotating accumulators (BT_NB, BT_F) and is
+// summed in float32 registers.  The rows are dealt to S splits; every split writes its partial
+// [n][r] block, k_reduce_q adds them in a fixed order.
+// ---------------------------------------------------------------------------------------------
+struct BackTcArgs {
+    float* part;      // [mats][S][n][r]
+    int rows, n, r, Ncp, stages, S, kb_per_split;
+    int nodes;        // matrices per P~
+    int* flags;
+    const int* skip;
+};
+
+// shared-memory descriptor of an MN-major TF32 tile: lines of 32 floats along MN, 4-row atoms of 512 bytes along K
+// (stride offset), the next 32 floats of MN `mn_block_bytes` further (leading offset); 128-byte swizzle on 32-byte atoms.
+__device__ __forceinline__ unsigned long long tc_smem_desc_mn(unsigned addr, unsigned mn_block_bytes) {
+    unsigned long long d = 0;
+    d |= (unsigned long long)((addr >> 4) & 0x3FFF);
+    d |= (unsigned long long)((mn_block_bytes >> 4) & 0x3FFF) << 16;
+    d |= (unsigned long long)(512 >> 4) << 32;
+    d |= (unsigned long long)1 << 46;
+    d |= (unsigned long long)1 << 61;
+    return d;
+}
+
+__global__ void __launch_bounds__(PT_THREADS, 1)
+k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmP0,
+                 const __grid_constant__ CUtensorMap tmP1, const __grid_constant__ CUtensorMap tmP2, BackTcArgs a) {
+    extern __shared__ __align__(16) unsigned char bt_smem_raw[];
+    if (a.skip && *a.skip) return;
+    unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(bt_smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr unsigned A_BYTES = TC_BM * TC_BK * 4;            // 128 columns x 32 rows
+    constexpr unsigned BOX_BYTES = 32 * TC_BK * 4;             // one 32-column box
+    constexpr int CPB = (TC_BK / 8) / BT_F;                    // head chunks per K block
+    const unsigned B_BYTES = (unsigned)a.Ncp * TC_BK * 4;
+    const unsigned STAGE_BYTES = 3 * A_BYTES + 3 * B_BYTES;
+    const int NS = a.stages;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(base + (size_t)NS * STAGE_BYTES);
+    const unsigned bar_full = smem_u32(bars), bar_conv = bar_full + 8 * NS, bar_empty = bar_conv + 8 * NS;
+    const unsigned bar_hfull = bar_empty + 8 * NS, bar_hfree = bar_hfull + 8 * BT_NB, bar_acc = bar_hfree + 8 * BT_NB;
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 3 * NS + 2 * BT_NB + 1);
+    const unsigned smem_base = smem_u32(base);
+
+    const int ct = blockIdx.x, sp = blockIdx.y, mat = blockIdx.z;
+    const int pz = mat / a.nodes;
+    const int KBall = (a.rows + TC_BK - 1) / TC_BK;
+    const int kb0 = sp * a.kb_per_split;
+    const int KB = max(0, min(KBall, kb0 + a.kb_per_split) - kb0);
+    unsigned ncols = 32;
+    while ((int)ncols < (BT_NB + 1) * a.Ncp) ncols <<= 1;
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_conv + 8 * s, 8); mbar_init(bar_empty + 8 * s, 1); }
+        for (int b = 0; b < BT_NB; ++b) { mbar_init(bar_hfull + 8 * b, 1); mbar_init(bar_hfree + 8 * b, 8); }
+        mbar_init(bar_acc, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(ncols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    const unsigned tmem = *tmem_slot;      // small accumulator at column 0, head accumulator b at (1 + b) * Ncp
+    bool dead = false;
+
+    if (warp == 0) {
+        // ---- TMA producer ----
+        if (lane == 0) {
+            const unsigned tx = A_BYTES + 3u * B_BYTES;
+            for (int kb = 0; kb < KB; ++kb) {
+                const int s = kb % NS;
+                if (kb >= NS) mbar_wait(bar_empty + 8 * s, (unsigned)((kb / NS - 1) & 1), a.flags, dead);
+                const unsigned dst = smem_base + s * STAGE_BYTES;
+                const unsigned bar = bar_full + 8 * s;
+                const int row = (kb0 + kb) * TC_BK;
+                mbar_expect_tx(bar, tx);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) tma_load_3d_sw(dst + j * BOX_BYTES, &tmM, ct * TC_BM + 32 * j, row, mat, bar);
+                tma_load_3d_sw(dst + 3 * A_BYTES, &tmP0, row, 0, pz, bar);
+                tma_load_3d_sw(dst + 3 * A_BYTES + B_BYTES, &tmP1, row, 0, pz, bar);
+                tma_load_3d_sw(dst + 3 * A_BYTES + 2 * B_BYTES, &tmP2, row, 0, pz, bar);
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer ----
+        if (lane == 0) {
+            const unsigned idesc = tc_idesc(a.Ncp) | (1u << 15);          // A is MN-major
+            const unsigned d_small = tmem;
+            const int tp[6] = {2, 0, 1, 1, 0, 0}, tq[6] = {0, 2, 1, 0, 1, 0};   // (M term, P~ term), h = 0, m = 1, l = 2
+            int chunk = 0;
+            for (int kb = 0; kb < KB; ++kb) {
+                const int s = kb % NS;
+                mbar_wait(bar_conv + 8 * s, (unsigned)((kb / NS) & 1), a.flags, dead);
+                asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                const unsigned sb = smem_base + s * STAGE_BYTES;
+                const unsigned long long dA[3] = {tc_smem_desc_mn(sb, BOX_BYTES), tc_smem_desc_mn(sb + A_BYTES, BOX_BYTES),
+                                                  tc_smem_desc_mn(sb + 2 * A_BYTES, BOX_BYTES)};
+                const unsigned long long dP[3] = {tc_smem_desc(sb + 3 * A_BYTES), tc_smem_desc(sb + 3 * A_BYTES + B_BYTES),
+                                                  tc_smem_desc(sb + 3 * A_BYTES + 2 * B_BYTES)};
+#pragma unroll
+                for (int k = 0; k < TC_BK / 8; ++k) {
+                    const int hb = chunk % BT_NB;
+                    if (k % BT_F == 0 && chunk >= BT_NB) {     // the registers have taken this accumulator's last content
+                        mbar_wait(bar_hfree + 8 * hb, (unsigned)((chunk / BT_NB - 1) & 1), a.flags, dead);
+                        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                    }
+                    const unsigned d_head = tmem + (unsigned)((1 + hb) * a.Ncp);
+                    const unsigned long long oa = (unsigned long long)(64 * k);   // 8 rows of 128 bytes, in 16-byte units
+                    const unsigned long long ob = (unsigned long long)(2 * k);    // 8 floats along the K-major line
+#pragma unroll
+                    for (int t = 0; t < 6; ++t) {
+                        const unsigned acc = (t == 5) ? ((k % BT_F != 0) ? 1u : 0u) : ((kb > 0 || k > 0 || t > 0) ? 1u : 0u);
+                        asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
+                                     ::"r"(t == 5 ? d_head : d_small), "l"(dA[tp[t]] + oa), "l"(dP[tq[t]] + ob), "r"(idesc), "r"(acc) : "memory");
+                    }
+                    if (k % BT_F == BT_F - 1) {
+                        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_hfull + 8 * hb) : "memory");
+                        ++chunk;
+                    }
+                }
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_empty + 8 * s) : "memory");
+            }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_acc) : "memory");
+        }
+    } else {
+        // ---- converters / adders (warps 2-9) ----
+        const int cv = tid - 64;                       // 0 .. 255
+        const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
+        const int half = (warp - 2) >> 2;              // which half of the columns this warp adds up
+        const int ng = a.Ncp >> 4;                     // 8-column groups per thread
+        const unsigned lane_base = (unsigned)(quarter * 32) << 16;
+        const unsigned col_base = (unsigned)(half * (a.Ncp >> 1));
+        float acc[BT_MAXG][8];
+#pragma unroll
+        for (int g = 0; g < BT_MAXG; ++g)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
+        // adds head accumulator (chunk c) to the registers and hands it back to the MMA thread
+        auto drain = [&](int c) {
+            const int hb = c % BT_NB;
+            mbar_wait(bar_hfull + 8 * hb, (unsigned)((c / BT_NB) & 1), a.flags, dead);
+            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+            const unsigned t0 = tmem + lane_base + (unsigned)((1 + hb) * a.Ncp) + col_base;
+#pragma unroll
+            for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
+                if (g2 < ng) {
+                    unsigned v0[8], v1[8];
+                    tmem_ld8(t0 + 8 * g2, v0);
+                    if (g2 + 1 < ng) tmem_ld8(t0 + 8 * (g2 + 1), v1);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc[g2][j] += __uint_as_float(v0[j]);
+                    if (g2 + 1 < ng) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) acc[g2 + 1][j] += __uint_as_float(v1[j]);
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_hfree + 8 * hb);
+        };
+        for (int kb = 0; kb < KB; ++kb) {
+            const int s = kb % NS;
+            mbar_wait(bar_full + 8 * s, (unsigned)((kb / NS) & 1), a.flags, dead);
+            const float4* t0 = reinterpret_cast<const float4*>(base + (size_t)s * STAGE_BYTES);
+            float4* t1 = reinterpret_cast<float4*>(base + (size_t)s * STAGE_BYTES + A_BYTES);
+            float4* t2 = t1 + A_BYTES / 16;
+#pragma unroll
+            for (int u = 0; u < (TC_BM * TC_BK / 4) / 256; ++u) {
+                const int o = cv + u * 256;
+                const float4 mv = t0[o];
+                const float xs[4] = {mv.x, mv.y, mv.z, mv.w};
+                float ms[4], ls[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float h = __uint_as_float(__float_as_uint(xs[j]) & 0xFFFFE000u);
+                    const float r1 = xs[j] - h;
+                    ms[j] = __uint_as_float(__float_as_uint(r1) & 0xFFFFE000u);
+                    ls[j] = r1 - ms[j];
+                }
+                t1[o] = make_float4(ms[0], ms[1], ms[2], ms[3]);
+                t2[o] = make_float4(ls[0], ls[1], ls[2], ls[3]);
+            }
+            asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_conv + 8 * s);
+            // one K block behind the conversion: the head products of block kb - 1 are done or nearly so
+            if (kb > 0) {
+#pragma unroll
+                for (int c = 0; c < CPB; ++c) drain((kb - 1) * CPB + c);
+            }
+        }
+        if (KB > 0) {
+#pragma unroll
+            for (int c = 0; c < CPB; ++c) drain((KB - 1) * CPB + c);
+        }
+        // ---- epilogue: partial Q_i rows of this split = registers + small accumulator ----
+        mbar_wait(bar_acc, 0u, a.flags, dead);
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        const int col = ct * TC_BM + quarter * 32 + lane;
+        float* out = a.part + (((size_t)mat * a.S + sp) * a.n + (col < a.n ? col : 0)) * a.r;
+#pragma unroll
+        for (int g = 0; g < BT_MAXG; ++g) {
+            if (g < ng) {
+                unsigned v[8];
+                tmem_ld8(tmem + lane_base + col_base + 8 * g, v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+                if (col < a.n) {
+                    const int j0 = (int)col_base + 8 * g;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (j0 + j < a.r) out[j0 + j] = (KB > 0) ? acc[g][j] + __uint_as_float(v[j]) : 0.f;
                 }
             }
         }
