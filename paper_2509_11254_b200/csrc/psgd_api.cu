@@ -398,8 +398,6 @@ int launch_back_tc(Launcher& L, const float* M, const float* Phat, float* part, 
         const int64_t cost = ((base * s + 147) / 148) * (kbs + 8);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
     }
-    if (const char* e = getenv("PSGD_BTC_OFF")) { if (atoi(e)) return 0; }   // PROBE
-    if (const char* e = getenv("PSGD_BTC_KBS")) { int k = atoi(e); if (k > 0) { best = std::min(S, ceil_div(KB, k)); } }   // PROBE
     const int St = best, kbs = ceil_div(KB, St);
     float* Pt = (float*)(h->ws + h->lay.ptQ);
     const size_t tot = (size_t)count * Ncp * rows;
@@ -426,7 +424,7 @@ int launch_back_tc(Launcher& L, const float* M, const float* Phat, float* part, 
 // Q_i partial sums for all matrices; returns the number of row splits written (the S to hand to k_reduce_q).
 int launch_back(Launcher& L, const float* M, const float* Phat, float* part, int rows, int n, int r, int nodes,
                  int count, int rpc, int S, bool vec, const int* gate = nullptr, const int* skip = nullptr) {
-    if (r > 16 && !gate) {
+    if (r > 32 && !gate) {     // up to 32 columns the float32 kernel is as fast
         const int St = launch_back_tc(L, M, Phat, part, rows, n, r, nodes, count, S, skip);
         if (St > 0) return St;
     }

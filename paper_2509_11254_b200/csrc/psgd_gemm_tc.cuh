@@ -285,12 +285,13 @@ k_residual_tc(const __grid_constant__ CUtensorMap tmPh, const __grid_constant__ 
                 const unsigned dst = smem_base + s * STAGE_BYTES;
                 const unsigned bar = bar_full + 8 * s;
                 mbar_expect_tx(bar, STAGE_BYTES);
-                tma_load_3d_sw(dst, &tmPh, kc * TC_BK, rt * TC_BM, c, bar);
-                tma_load_3d_sw(dst + A_BYTES, &tmPm, kc * TC_BK, rt * TC_BM, c, bar);
-                tma_load_3d_sw(dst + 2 * A_BYTES, &tmPl, kc * TC_BK, rt * TC_BM, c, bar);
-                tma_load_3d_sw(dst + 3 * A_BYTES, &tmQh, kc * TC_BK, ct * RT_BN, qz, bar);
-                tma_load_3d_sw(dst + 3 * A_BYTES + B_BYTES, &tmQm, kc * TC_BK, ct * RT_BN, qz, bar);
-                tma_load_3d_sw(dst + 3 * A_BYTES + 2 * B_BYTES, &tmQl, kc * TC_BK, ct * RT_BN, qz, bar);
+                const int kx = (nkc - 1 - kc) * TC_BK;      // last columns of the factors first (see the MMA issuer)
+                tma_load_3d_sw(dst, &tmPh, kx, rt * TC_BM, c, bar);
+                tma_load_3d_sw(dst + A_BYTES, &tmPm, kx, rt * TC_BM, c, bar);
+                tma_load_3d_sw(dst + 2 * A_BYTES, &tmPl, kx, rt * TC_BM, c, bar);
+                tma_load_3d_sw(dst + 3 * A_BYTES, &tmQh, kx, ct * RT_BN, qz, bar);
+                tma_load_3d_sw(dst + 3 * A_BYTES + B_BYTES, &tmQm, kx, ct * RT_BN, qz, bar);
+                tma_load_3d_sw(dst + 3 * A_BYTES + 2 * B_BYTES, &tmQl, kx, ct * RT_BN, qz, bar);
             }
         }
     } else if (warp == 1) {
@@ -309,13 +310,16 @@ k_residual_tc(const __grid_constant__ CUtensorMap tmPh, const __grid_constant__ 
                 const unsigned long long dQ[3] = {tc_smem_desc(sb + 3 * A_BYTES), tc_smem_desc(sb + 3 * A_BYTES + B_BYTES),
                                                   tc_smem_desc(sb + 3 * A_BYTES + 2 * B_BYTES)};
                 // two accumulators per tile: the h*h products (8 adds per 64 of K) and the five small products,
-                // so that the rounding of the tensor core's float32 adds hits the large running sum as rarely as possible
+                // so that the rounding of the tensor core's float32 adds hits the large running sum as rarely as possible.
+                // That add truncates toward zero, about 3e-8 of the running sum each time; the columns of P~ Q_i^T are
+                // summed from the last to the first because the leading columns carry the large terms (P~ comes out of
+                // a QR of M Q, or of Ritz vectors sorted by singular value): the running sum stays small until the end.
                 const unsigned d_big = tmem + (unsigned)(ab * 2 * RT_BN), d_small = d_big + RT_BN;
                 // (index of the P term, index of the Q term) with h = 0, m = 1, l = 2; small products first
                 const int tp[6] = {2, 0, 1, 1, 0, 0}, tq[6] = {0, 2, 1, 0, 1, 0};
 #pragma unroll
                 for (int k = 0; k < TC_BK / 8; ++k) {
-                    const unsigned long long o = (unsigned long long)(2 * k);
+                    const unsigned long long o = (unsigned long long)(2 * (TC_BK / 8 - 1 - k));
 #pragma unroll
                     for (int t = 0; t < 6; ++t) {
                         const unsigned acc = (kc > 0 || k > 0 || (t > 0 && t < 5)) ? 1u : 0u;
@@ -420,13 +424,16 @@ namespace psgd {
 // the five small ones go into one tensor-memory accumulator; the head product h*h goes through the
 // rotating accumulators described below and is summed in float32 registers.
 // ---------------------------------------------------------------------------------------------
-constexpr int PT_THREADS = 320;   // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-9: converters, adders, epilogue
+constexpr int PT_THREADS = 576;   // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-9: converters, warps 10-17: adders + epilogue
 // The tensor core adds to its float32 accumulator with truncation (measured on like-signed sums: 3e-8 relative per
 // accumulation, always toward zero, i.e. 2e-5 over the 512 steps of a 4096-long contraction).  The head product h*h
-// therefore accumulates only BT_F steps in tensor memory: BT_NB accumulators take turns and the converter warps add
+// therefore accumulates only BT_F steps in tensor memory: bt_heads() accumulators take turns and eight adder warps add
 // each finished one to float32 registers (round to nearest) while the next ones fill.
-constexpr int BT_NB = 3;    // head accumulators in rotation
-constexpr int BT_F = 2;     // MMA steps (8 of K each) per head accumulator before it is added up in registers
+constexpr int BT_NBMAX = 3; // most head accumulators in rotation
+// head accumulators in rotation: what fits beside the small accumulator in the 512 columns of tensor memory
+__host__ __device__ inline int bt_heads(int Ncp) { int nb = 512 / Ncp - 1; return nb > BT_NBMAX ? BT_NBMAX : nb; }
+constexpr int BT_F = 4;     // MMA steps (8 of K each) per head accumulator before it is added up in registers: one K block
+                            // (every hand-over costs the pipeline about 500 cycles per K block: 2 steps were 25 % slower)
 constexpr int BT_MAXG = 8;  // 8-column groups per thread: (Ncp / 2) / 8 for Ncp <= 128
 
 __device__ __forceinline__ void tmem_ld8(unsigned taddr, unsigned (&v)[8]) {
@@ -481,22 +488,22 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     constexpr int CPB = (TC_BK / 8) / BT_F;                    // head chunks per K block
     const unsigned B_BYTES = (unsigned)a.Ncp * TC_BK * 4;
     const unsigned STAGE_BYTES = 3 * A_BYTES + 3 * B_BYTES;
-    const int NS = a.stages;
+    const int NS = a.stages, NB = bt_heads(a.Ncp);
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(base + (size_t)NS * STAGE_BYTES);
     const unsigned bar_full = smem_u32(bars), bar_conv = bar_full + 8 * NS, bar_empty = bar_conv + 8 * NS;
-    const unsigned bar_hfull = bar_empty + 8 * NS, bar_hfree = bar_hfull + 8 * BT_NB, bar_acc = bar_hfree + 8 * BT_NB;
-    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 3 * NS + 2 * BT_NB + 1);
+    const unsigned bar_hfull = bar_empty + 8 * NS, bar_hfree = bar_hfull + 8 * NB, bar_acc = bar_hfree + 8 * NB;
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 3 * NS + 2 * NB + 1);
     const unsigned smem_base = smem_u32(base);
 
     const int rt = blockIdx.x, mat = blockIdx.y;
     const int qz = mat / a.nodes;
     const int KB = (a.n + TC_BK - 1) / TC_BK;
     unsigned ncols = 32;
-    while ((int)ncols < (BT_NB + 1) * a.Ncp) ncols <<= 1;
+    while ((int)ncols < (NB + 1) * a.Ncp) ncols <<= 1;
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_conv + 8 * s, 8); mbar_init(bar_empty + 8 * s, 1); }
-        for (int b = 0; b < BT_NB; ++b) { mbar_init(bar_hfull + 8 * b, 1); mbar_init(bar_hfree + 8 * b, 8); }
+        for (int b = 0; b < NB; ++b) { mbar_init(bar_hfull + 8 * b, 1); mbar_init(bar_hfree + 8 * b, 8); }
         mbar_init(bar_acc, 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -544,9 +551,9 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                                                   tc_smem_desc(sb + 3 * A_BYTES + 2 * B_BYTES)};
 #pragma unroll
                 for (int k = 0; k < TC_BK / 8; ++k) {
-                    const int hb = chunk % BT_NB;
-                    if (k % BT_F == 0 && chunk >= BT_NB) {     // the registers have taken this accumulator's last content
-                        mbar_wait(bar_hfree + 8 * hb, (unsigned)((chunk / BT_NB - 1) & 1), a.flags, dead);
+                    const int hb = chunk % NB;
+                    if (k % BT_F == 0 && chunk >= NB) {     // the registers have taken this accumulator's last content
+                        mbar_wait(bar_hfree + 8 * hb, (unsigned)((chunk / NB - 1) & 1), a.flags, dead);
                         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                     }
                     const unsigned d_head = tmem + (unsigned)((1 + hb) * a.Ncp);
@@ -566,44 +573,9 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             }
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_acc) : "memory");
         }
-    } else {
-        // ---- converters / adders (warps 2-9): M = A + B in place, exact three-way split, M back to HBM ----
+    } else if (warp < 10) {
+        // ---- converters (warps 2-9): M = A + B in place, exact three-way split, M back to HBM ----
         const int ct = tid - 64;                       // 0 .. 255
-        const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
-        const int half = (warp - 2) >> 2;              // which half of the columns this warp adds up
-        const int ng = a.Ncp >> 4;                     // 8-column groups per thread
-        const unsigned lane_base = (unsigned)(quarter * 32) << 16;
-        const unsigned col_base = (unsigned)(half * (a.Ncp >> 1));
-        float acc[BT_MAXG][8];
-#pragma unroll
-        for (int g = 0; g < BT_MAXG; ++g)
-#pragma unroll
-            for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
-        // adds head accumulator (chunk c) to the registers and hands it back to the MMA thread
-        auto drain = [&](int c) {
-            const int hb = c % BT_NB;
-            mbar_wait(bar_hfull + 8 * hb, (unsigned)((c / BT_NB) & 1), a.flags, dead);
-            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-            const unsigned t0 = tmem + lane_base + (unsigned)((1 + hb) * a.Ncp) + col_base;
-#pragma unroll
-            for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
-                if (g2 < ng) {
-                    unsigned v0[8], v1[8];
-                    tmem_ld8(t0 + 8 * g2, v0);
-                    if (g2 + 1 < ng) tmem_ld8(t0 + 8 * (g2 + 1), v1);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) acc[g2][j] += __uint_as_float(v0[j]);
-                    if (g2 + 1 < ng) {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[g2 + 1][j] += __uint_as_float(v1[j]);
-                    }
-                }
-            }
-            asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_hfree + 8 * hb);
-        };
         for (int kb = 0; kb < KB; ++kb) {
             const int s = kb % NS;
             mbar_wait(bar_full + 8 * s, (unsigned)((kb / NS) & 1), a.flags, dead);
@@ -640,16 +612,45 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");    // generic writes -> visible to the tensor core
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_conv + 8 * s);
-            // one K block behind the conversion: the head products of block kb - 1 are done or nearly so
-            if (kb > 0) {
+        }
+    } else {
+        // ---- adders (warps 10-17): head accumulators -> float32 registers; then the epilogue ----
+        const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
+        const int half = (warp - 10) >> 2;              // which half of the columns this warp adds up
+        const int ng = a.Ncp >> 4;                     // 8-column groups per thread
+        const unsigned lane_base = (unsigned)(quarter * 32) << 16;
+        const unsigned col_base = (unsigned)(half * (a.Ncp >> 1));
+        float acc[BT_MAXG][8];
 #pragma unroll
-                for (int c = 0; c < CPB; ++c) drain((kb - 1) * CPB + c);
+        for (int g = 0; g < BT_MAXG; ++g)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
+        // adds head accumulator (chunk c) to the registers and hands it back to the MMA thread
+        auto drain = [&](int c) {
+            const int hb = c % NB;
+            mbar_wait(bar_hfull + 8 * hb, (unsigned)((c / NB) & 1), a.flags, dead);
+            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+            const unsigned t0 = tmem + lane_base + (unsigned)((1 + hb) * a.Ncp) + col_base;
+#pragma unroll
+            for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
+                if (g2 < ng) {
+                    unsigned v0[8], v1[8];
+                    tmem_ld8(t0 + 8 * g2, v0);
+                    if (g2 + 1 < ng) tmem_ld8(t0 + 8 * (g2 + 1), v1);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc[g2][j] += __uint_as_float(v0[j]);
+                    if (g2 + 1 < ng) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) acc[g2 + 1][j] += __uint_as_float(v1[j]);
+                    }
+                }
             }
-        }
-        if (KB > 0) {
-#pragma unroll
-            for (int c = 0; c < CPB; ++c) drain((KB - 1) * CPB + c);
-        }
+            asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_hfree + 8 * hb);
+        };
+        for (int c = 0; c < KB * CPB; ++c) drain(c);
         // ---- epilogue: P = registers + small accumulator ----
         mbar_wait(bar_acc, 0u, a.flags, dead);
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
@@ -686,7 +687,7 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 // four boxes side by side give the 128 columns of one CTA.  P~^T arrives pre-split and K-major
 // (k_split_pad_t on P~).  Converters split the tile of M exactly into three TF32 terms; of the six
 // tcgen05.mma products per 8 rows the five small ones go into one tensor-memory accumulator for the
-// whole split; the head product h*h goes through the rotating accumulators (BT_NB, BT_F) and is
+// whole split; the head product h*h goes through the rotating accumulators (bt_heads, BT_F) and is
 // summed in float32 registers.  The rows are dealt to S splits; every split writes its partial
 // [n][r] block, k_reduce_q adds them in a fixed order.
 // ---------------------------------------------------------------------------------------------
@@ -722,11 +723,11 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     constexpr int CPB = (TC_BK / 8) / BT_F;                    // head chunks per K block
     const unsigned B_BYTES = (unsigned)a.Ncp * TC_BK * 4;
     const unsigned STAGE_BYTES = 3 * A_BYTES + 3 * B_BYTES;
-    const int NS = a.stages;
+    const int NS = a.stages, NB = bt_heads(a.Ncp);
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(base + (size_t)NS * STAGE_BYTES);
     const unsigned bar_full = smem_u32(bars), bar_conv = bar_full + 8 * NS, bar_empty = bar_conv + 8 * NS;
-    const unsigned bar_hfull = bar_empty + 8 * NS, bar_hfree = bar_hfull + 8 * BT_NB, bar_acc = bar_hfree + 8 * BT_NB;
-    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 3 * NS + 2 * BT_NB + 1);
+    const unsigned bar_hfull = bar_empty + 8 * NS, bar_hfree = bar_hfull + 8 * NB, bar_acc = bar_hfree + 8 * NB;
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 3 * NS + 2 * NB + 1);
     const unsigned smem_base = smem_u32(base);
 
     const int ct = blockIdx.x, sp = blockIdx.y, mat = blockIdx.z;
@@ -735,11 +736,11 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     const int kb0 = sp * a.kb_per_split;
     const int KB = max(0, min(KBall, kb0 + a.kb_per_split) - kb0);
     unsigned ncols = 32;
-    while ((int)ncols < (BT_NB + 1) * a.Ncp) ncols <<= 1;
+    while ((int)ncols < (NB + 1) * a.Ncp) ncols <<= 1;
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_conv + 8 * s, 8); mbar_init(bar_empty + 8 * s, 1); }
-        for (int b = 0; b < BT_NB; ++b) { mbar_init(bar_hfull + 8 * b, 1); mbar_init(bar_hfree + 8 * b, 8); }
+        for (int b = 0; b < NB; ++b) { mbar_init(bar_hfull + 8 * b, 1); mbar_init(bar_hfree + 8 * b, 8); }
         mbar_init(bar_acc, 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -789,9 +790,9 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
                                                   tc_smem_desc(sb + 3 * A_BYTES + 2 * B_BYTES)};
 #pragma unroll
                 for (int k = 0; k < TC_BK / 8; ++k) {
-                    const int hb = chunk % BT_NB;
-                    if (k % BT_F == 0 && chunk >= BT_NB) {     // the registers have taken this accumulator's last content
-                        mbar_wait(bar_hfree + 8 * hb, (unsigned)((chunk / BT_NB - 1) & 1), a.flags, dead);
+                    const int hb = chunk % NB;
+                    if (k % BT_F == 0 && chunk >= NB) {     // the registers have taken this accumulator's last content
+                        mbar_wait(bar_hfree + 8 * hb, (unsigned)((chunk / NB - 1) & 1), a.flags, dead);
                         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                     }
                     const unsigned d_head = tmem + (unsigned)((1 + hb) * a.Ncp);
@@ -812,44 +813,9 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
             }
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_acc) : "memory");
         }
-    } else {
-        // ---- converters / adders (warps 2-9) ----
+    } else if (warp < 10) {
+        // ---- converters (warps 2-9) ----
         const int cv = tid - 64;                       // 0 .. 255
-        const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
-        const int half = (warp - 2) >> 2;              // which half of the columns this warp adds up
-        const int ng = a.Ncp >> 4;                     // 8-column groups per thread
-        const unsigned lane_base = (unsigned)(quarter * 32) << 16;
-        const unsigned col_base = (unsigned)(half * (a.Ncp >> 1));
-        float acc[BT_MAXG][8];
-#pragma unroll
-        for (int g = 0; g < BT_MAXG; ++g)
-#pragma unroll
-            for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
-        // adds head accumulator (chunk c) to the registers and hands it back to the MMA thread
-        auto drain = [&](int c) {
-            const int hb = c % BT_NB;
-            mbar_wait(bar_hfull + 8 * hb, (unsigned)((c / BT_NB) & 1), a.flags, dead);
-            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-            const unsigned t0 = tmem + lane_base + (unsigned)((1 + hb) * a.Ncp) + col_base;
-#pragma unroll
-            for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
-                if (g2 < ng) {
-                    unsigned v0[8], v1[8];
-                    tmem_ld8(t0 + 8 * g2, v0);
-                    if (g2 + 1 < ng) tmem_ld8(t0 + 8 * (g2 + 1), v1);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) acc[g2][j] += __uint_as_float(v0[j]);
-                    if (g2 + 1 < ng) {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[g2 + 1][j] += __uint_as_float(v1[j]);
-                    }
-                }
-            }
-            asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_hfree + 8 * hb);
-        };
         for (int kb = 0; kb < KB; ++kb) {
             const int s = kb % NS;
             mbar_wait(bar_full + 8 * s, (unsigned)((kb / NS) & 1), a.flags, dead);
@@ -875,16 +841,45 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
             asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_conv + 8 * s);
-            // one K block behind the conversion: the head products of block kb - 1 are done or nearly so
-            if (kb > 0) {
+        }
+    } else {
+        // ---- adders (warps 10-17): head accumulators -> float32 registers; then the epilogue ----
+        const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
+        const int half = (warp - 10) >> 2;              // which half of the columns this warp adds up
+        const int ng = a.Ncp >> 4;                     // 8-column groups per thread
+        const unsigned lane_base = (unsigned)(quarter * 32) << 16;
+        const unsigned col_base = (unsigned)(half * (a.Ncp >> 1));
+        float acc[BT_MAXG][8];
 #pragma unroll
-                for (int c = 0; c < CPB; ++c) drain((kb - 1) * CPB + c);
+        for (int g = 0; g < BT_MAXG; ++g)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
+        // adds head accumulator (chunk c) to the registers and hands it back to the MMA thread
+        auto drain = [&](int c) {
+            const int hb = c % NB;
+            mbar_wait(bar_hfull + 8 * hb, (unsigned)((c / NB) & 1), a.flags, dead);
+            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+            const unsigned t0 = tmem + lane_base + (unsigned)((1 + hb) * a.Ncp) + col_base;
+#pragma unroll
+            for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
+                if (g2 < ng) {
+                    unsigned v0[8], v1[8];
+                    tmem_ld8(t0 + 8 * g2, v0);
+                    if (g2 + 1 < ng) tmem_ld8(t0 + 8 * (g2 + 1), v1);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc[g2][j] += __uint_as_float(v0[j]);
+                    if (g2 + 1 < ng) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) acc[g2 + 1][j] += __uint_as_float(v1[j]);
+                    }
+                }
             }
-        }
-        if (KB > 0) {
-#pragma unroll
-            for (int c = 0; c < CPB; ++c) drain((KB - 1) * CPB + c);
-        }
+            asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_hfree + 8 * hb);
+        };
+        for (int c = 0; c < KB * CPB; ++c) drain(c);
         // ---- epilogue: partial Q_i rows of this split = registers + small accumulator ----
         mbar_wait(bar_acc, 0u, a.flags, dead);
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
