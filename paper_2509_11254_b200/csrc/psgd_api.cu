@@ -424,7 +424,7 @@ int launch_back_tc(Launcher& L, const float* M, const float* Phat, float* part, 
 // Q_i partial sums for all matrices; returns the number of row splits written (the S to hand to k_reduce_q).
 int launch_back(Launcher& L, const float* M, const float* Phat, float* part, int rows, int n, int r, int nodes,
                  int count, int rpc, int S, bool vec, const int* gate = nullptr, const int* skip = nullptr) {
-    if (r > 32 && !gate) {     // up to 32 columns the float32 kernel is as fast
+    if (r > 16 && !gate) {
         const int St = launch_back_tc(L, M, Phat, part, rows, n, r, nodes, count, S, skip);
         if (St > 0) return St;
     }

@@ -723,7 +723,11 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     constexpr int CPB = (TC_BK / 8) / BT_F;                    // head chunks per K block
     const unsigned B_BYTES = (unsigned)a.Ncp * TC_BK * 4;
     const unsigned STAGE_BYTES = 3 * A_BYTES + 3 * B_BYTES;
-    const int NS = a.stages, NB = bt_heads(a.Ncp);
+    // Up to 80 columns the three terms of P~^T lie side by side as one B operand of 3 Ncp <= 256 rows, so that three
+    // MMAs per 8 rows (h x [h|m|l], m x [h|m], l x [h]) do the work of six and the slow MN-major operand is fetched
+    // half as often; an accumulator set is then [head | small | small], all of it added up in registers per K block.
+    const bool wide = 3 * a.Ncp <= 256;
+    const int NS = a.stages, NB = wide ? min(4, 512 / (3 * a.Ncp)) : bt_heads(a.Ncp);
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(base + (size_t)NS * STAGE_BYTES);
     const unsigned bar_full = smem_u32(bars), bar_conv = bar_full + 8 * NS, bar_empty = bar_conv + 8 * NS;
     const unsigned bar_hfull = bar_empty + 8 * NS, bar_hfree = bar_hfull + 8 * NB, bar_acc = bar_hfree + 8 * NB;
@@ -736,7 +740,7 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     const int kb0 = sp * a.kb_per_split;
     const int KB = max(0, min(KBall, kb0 + a.kb_per_split) - kb0);
     unsigned ncols = 32;
-    while ((int)ncols < (NB + 1) * a.Ncp) ncols <<= 1;
+    while ((int)ncols < (wide ? NB * 3 : NB + 1) * a.Ncp) ncols <<= 1;
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_conv + 8 * s, 8); mbar_init(bar_empty + 8 * s, 1); }
@@ -751,7 +755,7 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-    const unsigned tmem = *tmem_slot;      // small accumulator at column 0, head accumulator b at (1 + b) * Ncp
+    const unsigned tmem = *tmem_slot;      // small accumulator at column 0, head accumulator b at (1 + b) * Ncp; wide: set b at 3 b Ncp
     bool dead = false;
 
     if (warp == 0) {
@@ -788,6 +792,29 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
                                                   tc_smem_desc_mn(sb + 2 * A_BYTES, BOX_BYTES)};
                 const unsigned long long dP[3] = {tc_smem_desc(sb + 3 * A_BYTES), tc_smem_desc(sb + 3 * A_BYTES + B_BYTES),
                                                   tc_smem_desc(sb + 3 * A_BYTES + 2 * B_BYTES)};
+                if (wide) {
+                    const int hb = kb % NB;
+                    if (kb >= NB) {                        // the registers have taken this set's last content
+                        mbar_wait(bar_hfree + 8 * hb, (unsigned)((kb / NB - 1) & 1), a.flags, dead);
+                        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                    }
+                    const unsigned d_set = tmem + (unsigned)(3 * hb * a.Ncp);
+                    const unsigned id3 = tc_idesc(3 * a.Ncp) | (1u << 15), id2 = tc_idesc(2 * a.Ncp) | (1u << 15);
+#pragma unroll
+                    for (int k = 0; k < TC_BK / 8; ++k) {
+                        const unsigned long long oa = (unsigned long long)(64 * k), ob = (unsigned long long)(2 * k);
+                        const unsigned acc0 = k > 0 ? 1u : 0u;
+                        asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
+                                     ::"r"(d_set), "l"(dA[0] + oa), "l"(dP[0] + ob), "r"(id3), "r"(acc0) : "memory");
+                        asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
+                                     ::"r"(d_set + (unsigned)a.Ncp), "l"(dA[1] + oa), "l"(dP[0] + ob), "r"(id2), "r"(1u) : "memory");
+                        asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
+                                     ::"r"(d_set + (unsigned)a.Ncp), "l"(dA[2] + oa), "l"(dP[0] + ob), "r"(idesc), "r"(1u) : "memory");
+                    }
+                    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_hfull + 8 * hb) : "memory");
+                    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_empty + 8 * s) : "memory");
+                    continue;
+                }
 #pragma unroll
                 for (int k = 0; k < TC_BK / 8; ++k) {
                     const int hb = chunk % NB;
@@ -859,6 +886,25 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
             const int hb = c % NB;
             mbar_wait(bar_hfull + 8 * hb, (unsigned)((c / NB) & 1), a.flags, dead);
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+            if (wide) {
+                const unsigned ts = tmem + lane_base + (unsigned)(3 * hb * a.Ncp) + col_base;
+#pragma unroll
+                for (int g = 0; g < 5; ++g) {              // Ncp <= 80: at most 5 groups of 8 columns per thread
+                    if (g < ng) {
+                        unsigned vh[8], v1[8], v2[8];
+                        tmem_ld8(ts + 8 * g, vh);
+                        tmem_ld8(ts + (unsigned)a.Ncp + 8 * g, v1);
+                        tmem_ld8(ts + (unsigned)(2 * a.Ncp) + 8 * g, v2);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) acc[g][j] += __uint_as_float(vh[j]) + (__uint_as_float(v1[j]) + __uint_as_float(v2[j]));
+                    }
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_hfree + 8 * hb);
+                return;
+            }
             const unsigned t0 = tmem + lane_base + (unsigned)((1 + hb) * a.Ncp) + col_base;
 #pragma unroll
             for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
@@ -889,8 +935,13 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
         for (int g = 0; g < BT_MAXG; ++g) {
             if (g < ng) {
                 unsigned v[8];
-                tmem_ld8(tmem + lane_base + col_base + 8 * g, v);
-                asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+                if (!wide) {
+                    tmem_ld8(tmem + lane_base + col_base + 8 * g, v);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) v[j] = 0u;
+                }
                 if (col < a.n) {
                     const int j0 = (int)col_base + 8 * g;
 #pragma unroll
