@@ -335,9 +335,12 @@ def test_gemm_nt_tf32_matches_definition(torch_cuda, M, Nc, K, count):
 
 
 # ---- full-size workloads in the benchmark's launch configuration, checked on sampled matrices ----
-def _full_size_case(torch, workload, m, n, r, N, count, tau, sample, free_steps):
+def _full_size_case(torch, workload, m, n, r, N, count, tau, sample, free_steps, free_check=True):
     """Deferred mode as bench.py runs it: free-running steps against the oracle on the sampled
-    matrices (rotation-invariant outputs, 1e-3), then one more step from identical state (1e-5)."""
+    matrices (rotation-invariant outputs, 1e-3), then one more step from identical state (1e-5).
+    free_check=False skips the free-running comparison: without a spectral gap at r (directions r, r+1
+    both at the noise floor) two correct runs may keep different tail directions, so only the step from
+    identical state is a well-posed comparison."""
     from paper_2509_11254_b200 import PowerSGDPlus
 
     dev = "cuda:0"
@@ -353,7 +356,7 @@ def _full_size_case(torch, workload, m, n, r, N, count, tau, sample, free_steps)
         del G
     comp.materialize_error()
     assert comp.last_status() == 0
-    for c in sample:
+    for c in sample if free_check else ():
         normM = np.linalg.norm(out[c]["M"])
         assert projector_distance(comp.P_hat[c].cpu().numpy(), out[c]["P_hat"]) <= 1e-3, f"matrix {c}: projector"
         assert rel_fro(comp.E[c].cpu().numpy(), out[c]["E"], floor=1e-2 * normM) <= 1e-3, f"matrix {c}: residual"
@@ -395,6 +398,28 @@ def test_full_size_config5(torch_cuda, r):
     """BASELINE config 5: one 16384 x 4096 matrix on 4 nodes, plain PowerSGD steps (the step the sweep times)."""
     plan = _full_size_case(torch_cuda, 5, 16384, 4096, r, 4, 1, tau=0, sample=(0,), free_steps=3)
     assert plan["single_pass"] == 1 and plan["CS"] == 8 and plan["WC"] == 512
+
+
+@pytest.mark.parametrize("r", [64, 128])
+def test_full_size_config5_high_rank(torch_cuda, r):
+    """BASELINE config 5 at the ranks whose three passes run on the tensor cores (projection,
+    back-projection and residual as exactly split TF32 products).  The 0.9^k spectrum is at the noise
+    floor from k = 60 on, so there is no gap at r: a refresh at t = 0 aligns the state, the comparison is the
+    SSP step from identical state."""
+    plan = _full_size_case(torch_cuda, 5, 16384, 4096, r, 4, 1, tau=100, sample=(0,), free_steps=2, free_check=False)
+    assert plan["single_pass"] == 0
+
+
+def test_full_size_config4_attention_class(torch_cuda):
+    """BASELINE config 4, the 96 matrices of 2048 x 2048 (r = 32, N = 8, refresh at t = 0), two sampled."""
+    plan = _full_size_case(torch_cuda, 4, 2048, 2048, 32, 8, 96, tau=100, sample=(0, 95), free_steps=2)
+    assert plan["single_pass"] == 0
+
+
+def test_full_size_config4_ffn_class(torch_cuda):
+    """BASELINE config 4, the 72 matrices of 5504 x 2048, one sampled."""
+    plan = _full_size_case(torch_cuda, 4, 5504, 2048, 32, 8, 72, tau=100, sample=(71,), free_steps=2)
+    assert plan["single_pass"] == 0
 
 
 # ---- degenerate inputs ------------------------------------------------------------------------
