@@ -412,8 +412,8 @@ int launch_back_tc(Launcher& L, const float* M, const float* Phat, float* part, 
         L.status = PSGD_E_CUDA;
         return St;
     }
-    BackTcArgs a{part, rows, n, r, Ncp, proj_tc_stages(Ncp), St, kbs, nodes, (int*)(h->ws + h->lay.flags), skip};
-    size_t smem = proj_tc_smem_bytes(Ncp);
+    BackTcArgs a{part, rows, n, r, Ncp, back_tc_nh(Ncp), St, kbs, nodes, (int*)(h->ws + h->lay.flags), skip};
+    size_t smem = back_tc_smem_bytes(Ncp);
     cudaFuncSetAttribute(k_backproject_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     L.begin(PSGD_K_BACKPROJECT);
     k_backproject_tc<<<dim3(ceil_div(n, TC_BM), St, mats), PT_THREADS, smem, L.st>>>(tM, tP[0], tP[1], tP[2], a);

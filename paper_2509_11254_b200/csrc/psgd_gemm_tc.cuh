@@ -685,19 +685,45 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 // MN-major operand: TMA brings 32-row x 32-column boxes of M exactly as they lie in memory (128-byte
 // lines, 32-byte swizzle atoms, the one shared-memory form TF32 operands have in this orientation);
 // four boxes side by side give the 128 columns of one CTA.  P~^T arrives pre-split and K-major
-// (k_split_pad_t on P~).  Converters split the tile of M exactly into three TF32 terms; of the six
-// tcgen05.mma products per 8 rows the five small ones go into one tensor-memory accumulator for the
-// whole split; the head product h*h goes through the rotating accumulators (bt_heads, BT_F) and is
-// summed in float32 registers.  The rows are dealt to S splits; every split writes its partial
-// [n][r] block, k_reduce_q adds them in a fixed order.
+// (k_split_pad_t on P~, three exact terms).  The tile of M is used as two terms: the head is the tile
+// itself (read as TF32, i.e. truncated), the second term is x - head rounded to the nearest TF32
+// number, written by the converter warps; what is left of x (at most 2^-21 |x|, zero mean) averages
+// out over the hundreds of rows of a sum.  Products: h x [h|m|l] and m x [h|m]; m x l is below 2^-32.
+// Two shared-memory rings: a deep one for the tiles of M (16 KB stages) and a short one for what
+// lives only from the conversion to the end of the MMAs (the second term of the tile, the three
+// terms of P~^T).  One mbarrier per K block ("done", by tcgen05.commit) frees both stages and tells
+// the adder warps that the accumulators of that K block can be read.
+//   up to 80 columns: the three terms of P~^T lie side by side as one B operand of 3 Ncp <= 256 rows:
+//     two MMAs per 8 rows (the slow MN-major operand is fetched twice instead of six times); an
+//     accumulator set is [head | small | small], sets take turns and are added up in float32
+//     registers per K block;
+//   above: three MMAs (h x h, h x [m|l], m x [h|m]); the small products keep two accumulators for the
+//     whole split, the head product goes through rotating accumulators and float32 registers.
+// The rows are dealt to S splits; every split writes its partial [n][r] block, k_reduce_q adds them
+// in a fixed order.
 // ---------------------------------------------------------------------------------------------
+// stages of the short ring
+__host__ __device__ inline int back_tc_nm(int Ncp) { return 3 * Ncp <= 256 ? 3 : 2; }
+constexpr int BT_NHMAX = 8;       // most stages of the ring of M tiles
+
 struct BackTcArgs {
     float* part;      // [mats][S][n][r]
-    int rows, n, r, Ncp, stages, S, kb_per_split;
+    int rows, n, r, Ncp, nh, S, kb_per_split;
     int nodes;        // matrices per P~
     int* flags;
     const int* skip;
 };
+
+__host__ __device__ inline size_t back_tc_short_stage_bytes(int Ncp) { return (size_t)TC_BM * TC_BK * 4 + (size_t)3 * Ncp * TC_BK * 4; }
+// stages of the M ring that fit beside the short ring in 224 KB (0: does not fit)
+__host__ __device__ inline int back_tc_nh(int Ncp) {
+    const long long left = 224ll * 1024 - 1024 - 512 - (long long)back_tc_nm(Ncp) * (long long)back_tc_short_stage_bytes(Ncp);
+    const int nh = (int)(left / (TC_BM * TC_BK * 4));
+    return nh > BT_NHMAX ? BT_NHMAX : nh;
+}
+__host__ __device__ inline size_t back_tc_smem_bytes(int Ncp) {
+    return (size_t)back_tc_nh(Ncp) * TC_BM * TC_BK * 4 + back_tc_nm(Ncp) * back_tc_short_stage_bytes(Ncp) + 1024 + 512;
+}
 
 // shared-memory descriptor of an MN-major TF32 tile: lines of 32 floats along MN, 4-row atoms of 512 bytes along K
 // (stride offset), the next 32 floats of MN `mn_block_bytes` further (leading offset); 128-byte swizzle on 32-byte atoms.
@@ -710,6 +736,13 @@ __device__ __forceinline__ unsigned long long tc_smem_desc_mn(unsigned addr, uns
     d |= (unsigned long long)1 << 61;
     return d;
 }
+__device__ __forceinline__ void tc_mma_tf32(unsigned d, unsigned long long da, unsigned long long db, unsigned idesc, unsigned acc) {
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
+                 ::"r"(d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tc_commit(unsigned bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
 
 __global__ void __launch_bounds__(PT_THREADS, 1)
 k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmP0,
@@ -720,19 +753,17 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr unsigned A_BYTES = TC_BM * TC_BK * 4;            // 128 columns x 32 rows
     constexpr unsigned BOX_BYTES = 32 * TC_BK * 4;             // one 32-column box
-    constexpr int CPB = (TC_BK / 8) / BT_F;                    // head chunks per K block
     const unsigned B_BYTES = (unsigned)a.Ncp * TC_BK * 4;
-    const unsigned STAGE_BYTES = 3 * A_BYTES + 3 * B_BYTES;
-    // Up to 80 columns the three terms of P~^T lie side by side as one B operand of 3 Ncp <= 256 rows, so that three
-    // MMAs per 8 rows (h x [h|m|l], m x [h|m], l x [h]) do the work of six and the slow MN-major operand is fetched
-    // half as often; an accumulator set is then [head | small | small], all of it added up in registers per K block.
+    const unsigned SHORT_BYTES = A_BYTES + 3 * B_BYTES;        // [m tile][h, m, l of P~^T]
     const bool wide = 3 * a.Ncp <= 256;
-    const int NS = a.stages, NB = wide ? min(4, 512 / (3 * a.Ncp)) : bt_heads(a.Ncp);
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(base + (size_t)NS * STAGE_BYTES);
-    const unsigned bar_full = smem_u32(bars), bar_conv = bar_full + 8 * NS, bar_empty = bar_conv + 8 * NS;
-    const unsigned bar_hfull = bar_empty + 8 * NS, bar_hfree = bar_hfull + 8 * NB, bar_acc = bar_hfree + 8 * NB;
-    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 3 * NS + 2 * NB + 1);
-    const unsigned smem_base = smem_u32(base);
+    const int NM = back_tc_nm(a.Ncp);
+    const int NH = a.nh, NB = wide ? min(4, 512 / (3 * a.Ncp)) : min(3, (512 - 2 * a.Ncp) / a.Ncp);
+    unsigned char* short_base = base + (size_t)NH * A_BYTES;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(short_base + (size_t)NM * SHORT_BYTES);
+    const unsigned bar_hfull = smem_u32(bars), bar_done = bar_hfull + 8 * NH, bar_bfull = bar_done + 8 * NH;
+    const unsigned bar_conv = bar_bfull + 8 * NM, bar_free = bar_conv + 8 * NM, bar_acc = bar_free + 8 * NB;
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 2 * NH + 2 * NM + NB + 1);
+    const unsigned ring_u32 = smem_u32(base), short_u32 = smem_u32(short_base);
 
     const int ct = blockIdx.x, sp = blockIdx.y, mat = blockIdx.z;
     const int pz = mat / a.nodes;
@@ -740,11 +771,12 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     const int kb0 = sp * a.kb_per_split;
     const int KB = max(0, min(KBall, kb0 + a.kb_per_split) - kb0);
     unsigned ncols = 32;
-    while ((int)ncols < (wide ? NB * 3 : NB + 1) * a.Ncp) ncols <<= 1;
+    while ((int)ncols < (wide ? NB * 3 : NB + 2) * a.Ncp) ncols <<= 1;
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_conv + 8 * s, 8); mbar_init(bar_empty + 8 * s, 1); }
-        for (int b = 0; b < NB; ++b) { mbar_init(bar_hfull + 8 * b, 1); mbar_init(bar_hfree + 8 * b, 8); }
+        for (int s = 0; s < NH; ++s) { mbar_init(bar_hfull + 8 * s, 1); mbar_init(bar_done + 8 * s, 1); }
+        for (int s = 0; s < NM; ++s) { mbar_init(bar_bfull + 8 * s, 1); mbar_init(bar_conv + 8 * s, 8); }
+        for (int b = 0; b < NB; ++b) mbar_init(bar_free + 8 * b, 8);
         mbar_init(bar_acc, 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -755,124 +787,104 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-    const unsigned tmem = *tmem_slot;      // small accumulator at column 0, head accumulator b at (1 + b) * Ncp; wide: set b at 3 b Ncp
+    const unsigned tmem = *tmem_slot;      // wide: set b at 3 b Ncp; else two small accumulators at 0, head b at (2 + b) Ncp
     bool dead = false;
+    // K block j is "done" (all its MMAs have completed) in phase j / NH of bar_done[j % NH]
+    auto wait_done = [&](int j) { mbar_wait(bar_done + 8 * (j % NH), (unsigned)((j / NH) & 1), a.flags, dead); };
 
     if (warp == 0) {
-        // ---- TMA producer ----
+        // ---- TMA producer: tiles of M run NH - NM K blocks ahead of the terms of P~^T ----
         if (lane == 0) {
-            const unsigned tx = A_BYTES + 3u * B_BYTES;
-            for (int kb = 0; kb < KB; ++kb) {
-                const int s = kb % NS;
-                if (kb >= NS) mbar_wait(bar_empty + 8 * s, (unsigned)((kb / NS - 1) & 1), a.flags, dead);
-                const unsigned dst = smem_base + s * STAGE_BYTES;
-                const unsigned bar = bar_full + 8 * s;
-                const int row = (kb0 + kb) * TC_BK;
-                mbar_expect_tx(bar, tx);
+            const int lead = NH - NM;
+            auto issue_m = [&](int j) {
+                const int s = j % NH;
+                if (j >= NH) wait_done(j - NH);
+                const unsigned dst = ring_u32 + s * A_BYTES, bar = bar_hfull + 8 * s;
+                const int row = (kb0 + j) * TC_BK;
+                mbar_expect_tx(bar, A_BYTES);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) tma_load_3d_sw(dst + j * BOX_BYTES, &tmM, ct * TC_BM + 32 * j, row, mat, bar);
-                tma_load_3d_sw(dst + 3 * A_BYTES, &tmP0, row, 0, pz, bar);
-                tma_load_3d_sw(dst + 3 * A_BYTES + B_BYTES, &tmP1, row, 0, pz, bar);
-                tma_load_3d_sw(dst + 3 * A_BYTES + 2 * B_BYTES, &tmP2, row, 0, pz, bar);
+                for (int q = 0; q < 4; ++q) tma_load_3d_sw(dst + q * BOX_BYTES, &tmM, ct * TC_BM + 32 * q, row, mat, bar);
+            };
+            for (int j = 0; j < min(lead, KB); ++j) issue_m(j);
+            for (int kb = 0; kb < KB; ++kb) {
+                if (kb + lead < KB) issue_m(kb + lead);
+                const int s = kb % NM;
+                if (kb >= NM) wait_done(kb - NM);
+                const unsigned dst = short_u32 + s * SHORT_BYTES + A_BYTES, bar = bar_bfull + 8 * s;
+                const int row = (kb0 + kb) * TC_BK;
+                mbar_expect_tx(bar, 3u * B_BYTES);
+                tma_load_3d_sw(dst, &tmP0, row, 0, pz, bar);
+                tma_load_3d_sw(dst + B_BYTES, &tmP1, row, 0, pz, bar);
+                tma_load_3d_sw(dst + 2 * B_BYTES, &tmP2, row, 0, pz, bar);
             }
         }
     } else if (warp == 1) {
         // ---- MMA issuer ----
         if (lane == 0) {
-            const unsigned idesc = tc_idesc(a.Ncp) | (1u << 15);          // A is MN-major
-            const unsigned d_small = tmem;
-            const int tp[6] = {2, 0, 1, 1, 0, 0}, tq[6] = {0, 2, 1, 0, 1, 0};   // (M term, P~ term), h = 0, m = 1, l = 2
-            int chunk = 0;
+            const unsigned id1 = tc_idesc(a.Ncp) | (1u << 15);            // bit 15: A is MN-major
+            const unsigned id2 = tc_idesc(2 * a.Ncp) | (1u << 15), id3 = tc_idesc(wide ? 3 * a.Ncp : a.Ncp) | (1u << 15);
             for (int kb = 0; kb < KB; ++kb) {
-                const int s = kb % NS;
-                mbar_wait(bar_conv + 8 * s, (unsigned)((kb / NS) & 1), a.flags, dead);
+                const int sh = kb % NH, sm = kb % NM, hb = kb % NB;
+                mbar_wait(bar_conv + 8 * sm, (unsigned)((kb / NM) & 1), a.flags, dead);
+                mbar_wait(bar_bfull + 8 * sm, (unsigned)((kb / NM) & 1), a.flags, dead);
+                if (kb >= NB) mbar_wait(bar_free + 8 * hb, (unsigned)((kb / NB - 1) & 1), a.flags, dead);   // registers took its last content
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-                const unsigned sb = smem_base + s * STAGE_BYTES;
-                const unsigned long long dA[3] = {tc_smem_desc_mn(sb, BOX_BYTES), tc_smem_desc_mn(sb + A_BYTES, BOX_BYTES),
-                                                  tc_smem_desc_mn(sb + 2 * A_BYTES, BOX_BYTES)};
-                const unsigned long long dP[3] = {tc_smem_desc(sb + 3 * A_BYTES), tc_smem_desc(sb + 3 * A_BYTES + B_BYTES),
-                                                  tc_smem_desc(sb + 3 * A_BYTES + 2 * B_BYTES)};
+                const unsigned sb = short_u32 + sm * SHORT_BYTES;
+                const unsigned long long dAh = tc_smem_desc_mn(ring_u32 + sh * A_BYTES, BOX_BYTES), dAm = tc_smem_desc_mn(sb, BOX_BYTES);
+                const unsigned long long dPh = tc_smem_desc(sb + A_BYTES), dPm = tc_smem_desc(sb + A_BYTES + B_BYTES);
                 if (wide) {
-                    const int hb = kb % NB;
-                    if (kb >= NB) {                        // the registers have taken this set's last content
-                        mbar_wait(bar_hfree + 8 * hb, (unsigned)((kb / NB - 1) & 1), a.flags, dead);
-                        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-                    }
                     const unsigned d_set = tmem + (unsigned)(3 * hb * a.Ncp);
-                    const unsigned id3 = tc_idesc(3 * a.Ncp) | (1u << 15), id2 = tc_idesc(2 * a.Ncp) | (1u << 15);
+#pragma unroll
+                    for (int k = 0; k < TC_BK / 8; ++k) {
+                        const unsigned long long oa = (unsigned long long)(64 * k);   // 8 rows of 128 bytes, in 16-byte units
+                        const unsigned long long ob = (unsigned long long)(2 * k);    // 8 floats along the K-major line
+                        tc_mma_tf32(d_set, dAh + oa, dPh + ob, id3, k > 0 ? 1u : 0u);                      // h x [h|m|l]
+                        tc_mma_tf32(d_set + (unsigned)a.Ncp, dAm + oa, dPh + ob, id2, 1u);                 // m x [h|m]
+                    }
+                } else {
+                    const unsigned d_small = tmem, d_head = tmem + (unsigned)((2 + hb) * a.Ncp);
 #pragma unroll
                     for (int k = 0; k < TC_BK / 8; ++k) {
                         const unsigned long long oa = (unsigned long long)(64 * k), ob = (unsigned long long)(2 * k);
-                        const unsigned acc0 = k > 0 ? 1u : 0u;
-                        asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
-                                     ::"r"(d_set), "l"(dA[0] + oa), "l"(dP[0] + ob), "r"(id3), "r"(acc0) : "memory");
-                        asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
-                                     ::"r"(d_set + (unsigned)a.Ncp), "l"(dA[1] + oa), "l"(dP[0] + ob), "r"(id2), "r"(1u) : "memory");
-                        asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
-                                     ::"r"(d_set + (unsigned)a.Ncp), "l"(dA[2] + oa), "l"(dP[0] + ob), "r"(idesc), "r"(1u) : "memory");
-                    }
-                    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_hfull + 8 * hb) : "memory");
-                    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_empty + 8 * s) : "memory");
-                    continue;
-                }
-#pragma unroll
-                for (int k = 0; k < TC_BK / 8; ++k) {
-                    const int hb = chunk % NB;
-                    if (k % BT_F == 0 && chunk >= NB) {     // the registers have taken this accumulator's last content
-                        mbar_wait(bar_hfree + 8 * hb, (unsigned)((chunk / NB - 1) & 1), a.flags, dead);
-                        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-                    }
-                    const unsigned d_head = tmem + (unsigned)((1 + hb) * a.Ncp);
-                    const unsigned long long oa = (unsigned long long)(64 * k);   // 8 rows of 128 bytes, in 16-byte units
-                    const unsigned long long ob = (unsigned long long)(2 * k);    // 8 floats along the K-major line
-#pragma unroll
-                    for (int t = 0; t < 6; ++t) {
-                        const unsigned acc = (t == 5) ? ((k % BT_F != 0) ? 1u : 0u) : ((kb > 0 || k > 0 || t > 0) ? 1u : 0u);
-                        asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
-                                     ::"r"(t == 5 ? d_head : d_small), "l"(dA[tp[t]] + oa), "l"(dP[tq[t]] + ob), "r"(idesc), "r"(acc) : "memory");
-                    }
-                    if (k % BT_F == BT_F - 1) {
-                        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_hfull + 8 * hb) : "memory");
-                        ++chunk;
+                        tc_mma_tf32(d_small, dAh + oa, dPm + ob, id2, (kb > 0 || k > 0) ? 1u : 0u);        // h x [m|l]
+                        tc_mma_tf32(d_small, dAm + oa, dPh + ob, id2, 1u);                                 // m x [h|m]
+                        tc_mma_tf32(d_head, dAh + oa, dPh + ob, id1, k > 0 ? 1u : 0u);                     // h x h
                     }
                 }
-                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_empty + 8 * s) : "memory");
+                tc_commit(bar_done + 8 * sh);
             }
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_acc) : "memory");
+            tc_commit(bar_acc);
         }
     } else if (warp < 10) {
-        // ---- converters (warps 2-9) ----
+        // ---- converters (warps 2-9): the two lower TF32 terms of the tile of M ----
         const int cv = tid - 64;                       // 0 .. 255
         for (int kb = 0; kb < KB; ++kb) {
-            const int s = kb % NS;
-            mbar_wait(bar_full + 8 * s, (unsigned)((kb / NS) & 1), a.flags, dead);
-            const float4* t0 = reinterpret_cast<const float4*>(base + (size_t)s * STAGE_BYTES);
-            float4* t1 = reinterpret_cast<float4*>(base + (size_t)s * STAGE_BYTES + A_BYTES);
-            float4* t2 = t1 + A_BYTES / 16;
+            const int sh = kb % NH, sm = kb % NM;
+            mbar_wait(bar_hfull + 8 * sh, (unsigned)((kb / NH) & 1), a.flags, dead);
+            if (kb >= NM) wait_done(kb - NM);          // the MMAs that read this short stage have completed
+            const float4* t0 = reinterpret_cast<const float4*>(base + (size_t)sh * A_BYTES);
+            float4* t1 = reinterpret_cast<float4*>(short_base + (size_t)sm * SHORT_BYTES);
 #pragma unroll
             for (int u = 0; u < (TC_BM * TC_BK / 4) / 256; ++u) {
                 const int o = cv + u * 256;
                 const float4 mv = t0[o];
                 const float xs[4] = {mv.x, mv.y, mv.z, mv.w};
-                float ms[4], ls[4];
+                float ms[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float h = __uint_as_float(__float_as_uint(xs[j]) & 0xFFFFE000u);
-                    const float r1 = xs[j] - h;
-                    ms[j] = __uint_as_float(__float_as_uint(r1) & 0xFFFFE000u);
-                    ls[j] = r1 - ms[j];
+                    ms[j] = __uint_as_float((__float_as_uint(xs[j] - h) + 0x1000u) & 0xFFFFE000u);   // rounded to nearest TF32
                 }
                 t1[o] = make_float4(ms[0], ms[1], ms[2], ms[3]);
-                t2[o] = make_float4(ls[0], ls[1], ls[2], ls[3]);
             }
             asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_conv + 8 * s);
+            if (lane == 0) mbar_arrive(bar_conv + 8 * sm);
         }
     } else {
-        // ---- adders (warps 10-17): head accumulators -> float32 registers; then the epilogue ----
+        // ---- adders (warps 10-17): accumulators of each K block -> float32 registers; then the epilogue ----
         const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
-        const int half = (warp - 10) >> 2;              // which half of the columns this warp adds up
+        const int half = (warp - 10) >> 2;             // which half of the columns this warp adds up
         const int ng = a.Ncp >> 4;                     // 8-column groups per thread
         const unsigned lane_base = (unsigned)(quarter * 32) << 16;
         const unsigned col_base = (unsigned)(half * (a.Ncp >> 1));
@@ -881,10 +893,9 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
         for (int g = 0; g < BT_MAXG; ++g)
 #pragma unroll
             for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
-        // adds head accumulator (chunk c) to the registers and hands it back to the MMA thread
-        auto drain = [&](int c) {
+        for (int c = 0; c < KB; ++c) {
             const int hb = c % NB;
-            mbar_wait(bar_hfull + 8 * hb, (unsigned)((c / NB) & 1), a.flags, dead);
+            wait_done(c);
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
             if (wide) {
                 const unsigned ts = tmem + lane_base + (unsigned)(3 * hb * a.Ncp) + col_base;
@@ -900,33 +911,29 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
                         for (int j = 0; j < 8; ++j) acc[g][j] += __uint_as_float(vh[j]) + (__uint_as_float(v1[j]) + __uint_as_float(v2[j]));
                     }
                 }
-                asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_hfree + 8 * hb);
-                return;
-            }
-            const unsigned t0 = tmem + lane_base + (unsigned)((1 + hb) * a.Ncp) + col_base;
+            } else {
+                const unsigned t0 = tmem + lane_base + (unsigned)((2 + hb) * a.Ncp) + col_base;
 #pragma unroll
-            for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
-                if (g2 < ng) {
-                    unsigned v0[8], v1[8];
-                    tmem_ld8(t0 + 8 * g2, v0);
-                    if (g2 + 1 < ng) tmem_ld8(t0 + 8 * (g2 + 1), v1);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+                for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
+                    if (g2 < ng) {
+                        unsigned v0[8], v1[8];
+                        tmem_ld8(t0 + 8 * g2, v0);
+                        if (g2 + 1 < ng) tmem_ld8(t0 + 8 * (g2 + 1), v1);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) acc[g2][j] += __uint_as_float(v0[j]);
-                    if (g2 + 1 < ng) {
+                        for (int j = 0; j < 8; ++j) acc[g2][j] += __uint_as_float(v0[j]);
+                        if (g2 + 1 < ng) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[g2 + 1][j] += __uint_as_float(v1[j]);
+                            for (int j = 0; j < 8; ++j) acc[g2 + 1][j] += __uint_as_float(v1[j]);
+                        }
                     }
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_hfree + 8 * hb);
-        };
-        for (int c = 0; c < KB * CPB; ++c) drain(c);
-        // ---- epilogue: partial Q_i rows of this split = registers + small accumulator ----
+            if (lane == 0) mbar_arrive(bar_free + 8 * hb);
+        }
+        // ---- epilogue: partial Q_i rows of this split = registers (+ the small accumulator) ----
         mbar_wait(bar_acc, 0u, a.flags, dead);
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
         const int col = ct * TC_BM + quarter * 32 + lane;
@@ -936,8 +943,12 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
             if (g < ng) {
                 unsigned v[8];
                 if (!wide) {
+                    unsigned w[8];
                     tmem_ld8(tmem + lane_base + col_base + 8 * g, v);
+                    tmem_ld8(tmem + lane_base + (unsigned)a.Ncp + col_base + 8 * g, w);
                     asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(w[j]));
                 } else {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) v[j] = 0u;
