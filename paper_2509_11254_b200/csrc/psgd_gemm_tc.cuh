@@ -52,6 +52,12 @@ __device__ __forceinline__ unsigned long long tc_smem_desc(unsigned addr) {
 __device__ __forceinline__ unsigned tc_idesc(int n) {
     return (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(TC_BM >> 4) << 24);
 }
+// 32 lanes x 8 consecutive columns of tensor memory -> 8 registers per thread (lane = row of the accumulator)
+__device__ __forceinline__ void tmem_ld8(unsigned taddr, unsigned (&v)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tma_load_3d_sw(unsigned dst, const CUtensorMap* map, int x, int y, int z, unsigned bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"
@@ -207,6 +213,7 @@ namespace psgd {
 // ---------------------------------------------------------------------------------------------
 constexpr int RT_BN = 128;        // columns per output tile (= UMMA N)
 constexpr int RT_STAGES = 2;
+constexpr int RT_XPOSE_BYTES = 32 * 32 * 4;   // per epilogue warp: one 32 x 32 block turned from row-per-lane to row-contiguous
 constexpr int RT_THREADS = 320;   // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-9: epilogue (two per lane quarter)
 
 struct ResidTcArgs {
@@ -219,7 +226,7 @@ struct ResidTcArgs {
 };
 
 __host__ __device__ inline size_t resid_tc_smem_bytes() {
-    return (size_t)RT_STAGES * (3 * TC_BM * TC_BK * 4 + 3 * RT_BN * TC_BK * 4) + 1024 + 256;
+    return (size_t)RT_STAGES * (3 * TC_BM * TC_BK * 4 + 3 * RT_BN * TC_BK * 4) + 8 * RT_XPOSE_BYTES + 1024 + 256;
 }
 
 // X [rows][r] -> Xh, Xm, Xl [rows][KP], zero padded: x = h + m + l exactly, each term a TF32 number
@@ -334,68 +341,72 @@ k_residual_tc(const __grid_constant__ CUtensorMap tmPh, const __grid_constant__ 
         }
     } else {
         // ---- epilogue: E = M - accumulator ----
-        // Eight warps: warp w reads the tensor-memory lanes of quarter w % 4 (its accumulator rows) and the
-        // 32-column chunks of parity (w - 2) / 4.  The M values of a chunk are requested before the
-        // accumulator is read so that more loads are in flight.
+        // Eight warps: warp w reads the tensor-memory lanes of quarter w % 4 (its 32 accumulator rows) and the
+        // 32-column chunks of parity (w - 2) / 4.  Tensor memory hands a thread one row of the block; written like
+        // that to HBM every instruction would touch 32 lines, and the load-store unit, not HBM, would set the pace.
+        // So the block goes through a 4 KB shared-memory buffer of the warp (16-byte units XOR-swizzled by row) and
+        // comes back as 4 rows x 128 contiguous bytes per instruction, the layout M is loaded and E stored in.
+        // The M values of the next chunk are requested before the accumulator is read.
         const int quarter = warp & 3;
         const int half = (warp - 2) >> 2;
-        const int row = rt * TC_BM + quarter * 32 + lane;
-        const bool rok = row < a.rows;
-        const float* Mr = a.M ? a.M + ((size_t)mat * a.rows + (rok ? row : 0)) * a.n : nullptr;
-        float* Or = a.Out + ((size_t)mat * a.rows + (rok ? row : 0)) * a.n;
+        float4* xb = reinterpret_cast<float4*>(base + (size_t)RT_STAGES * STAGE_BYTES + 256 + (size_t)(warp - 2) * RT_XPOSE_BYTES);
+        const int lrow = lane >> 3, lch = lane & 7;           // coalesced phase: row within a group of 4, 16-byte unit
+        const int brow0 = rt * TC_BM + quarter * 32;          // first row of this warp's blocks
+        const size_t mrow = (size_t)mat * a.rows;
+        auto load_m = [&](int col0, float4 (&dst)[8]) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int row = brow0 + 4 * i + lrow, col = col0 + 4 * lch;
+                dst[i] = (a.M && row < a.rows && col < a.n) ? ldg_stream4(a.M + (mrow + row) * a.n + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        };
+        float4 mv[8];
+        load_m(half * 32, mv);
         for (int ct = 0; ct < nct; ++ct) {
             const int ab = ct & 1;
-            float4 mv[8];
-            const int cfirst = ct * RT_BN + half * 32;
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                mv[j] = (Mr && rok && cfirst + 4 * j < a.n) ? ldg_stream4(Mr + cfirst + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
             mbar_wait(bar_accf + 8 * ab, (unsigned)((ct >> 1) & 1), a.flags, dead);
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
 #pragma unroll 1
             for (int cc = half * 32; cc < RT_BN; cc += 64) {
                 const int col0 = ct * RT_BN + cc;
-                if (col0 >= a.n) break;
-                unsigned r[32], rs[32];
-                const unsigned taddr = tmem + ((unsigned)(quarter * 32) << 16) + (unsigned)(ab * 2 * RT_BN + cc);
-#define PSGD_TMEM_LD32(R, ADDR)                                                                                             \
-                asm volatile(                                                                                                  \
-                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "  \
-                    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"              \
-                    : "=r"(R[0]), "=r"(R[1]), "=r"(R[2]), "=r"(R[3]), "=r"(R[4]), "=r"(R[5]), "=r"(R[6]), "=r"(R[7]),          \
-                      "=r"(R[8]), "=r"(R[9]), "=r"(R[10]), "=r"(R[11]), "=r"(R[12]), "=r"(R[13]), "=r"(R[14]), "=r"(R[15]),    \
-                      "=r"(R[16]), "=r"(R[17]), "=r"(R[18]), "=r"(R[19]), "=r"(R[20]), "=r"(R[21]), "=r"(R[22]), "=r"(R[23]),  \
-                      "=r"(R[24]), "=r"(R[25]), "=r"(R[26]), "=r"(R[27]), "=r"(R[28]), "=r"(R[29]), "=r"(R[30]), "=r"(R[31])   \
-                    : "r"(ADDR) : "memory")
-                PSGD_TMEM_LD32(r, taddr);
-                PSGD_TMEM_LD32(rs, taddr + (unsigned)RT_BN);
-#undef PSGD_TMEM_LD32
-                asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-                // request the next chunk's M values (the next chunk of this tile, else nothing: the next tile's
-                // first chunk is requested at the top of the tile loop)
+                // next chunk of this warp: the other chunk of this tile, else the first chunk of the next tile
+                const int cnext = (cc + 64 < RT_BN) ? col0 + 64 : (ct + 1) * RT_BN + half * 32;
                 float4 mn[8];
-                const int cnext = col0 + 64;
-                const bool more = cc + 64 < RT_BN;
+                load_m(cnext < a.n && (cc + 64 < RT_BN || ct + 1 < nct) ? cnext : a.n, mn);
+                if (col0 < a.n) {
+                    const unsigned taddr = tmem + ((unsigned)(quarter * 32) << 16) + (unsigned)(ab * 2 * RT_BN + cc);
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    mn[j] = (more && Mr && rok && cnext + 4 * j < a.n) ? ldg_stream4(Mr + cnext + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
-                if (rok) {
+                    for (int p8 = 0; p8 < 4; ++p8) {
+                        unsigned rb[8], rs[8];
+                        tmem_ld8(taddr + 8 * p8, rb);
+                        tmem_ld8(taddr + (unsigned)RT_BN + 8 * p8, rs);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if (col0 + 4 * j < a.n) {      // n % 4 == 0: a group of 4 columns is all in or all out
-                            const float a0 = __uint_as_float(r[4 * j]) + __uint_as_float(rs[4 * j]);
-                            const float a1 = __uint_as_float(r[4 * j + 1]) + __uint_as_float(rs[4 * j + 1]);
-                            const float a2 = __uint_as_float(r[4 * j + 2]) + __uint_as_float(rs[4 * j + 2]);
-                            const float a3 = __uint_as_float(r[4 * j + 3]) + __uint_as_float(rs[4 * j + 3]);
-                            float4 o;
-                            if (Mr) o = make_float4(mv[j].x - a0, mv[j].y - a1, mv[j].z - a2, mv[j].w - a3);
-                            else o = make_float4(a0, a1, a2, a3);
-                            *reinterpret_cast<float4*>(Or + col0 + 4 * j) = o;
+                        for (int q = 0; q < 2; ++q) {
+                            const int j = 2 * p8 + q;            // 16-byte unit of this lane's row
+                            xb[lane * 8 + (j ^ (lane & 7))] =
+                                make_float4(__uint_as_float(rb[4 * q]) + __uint_as_float(rs[4 * q]),
+                                            __uint_as_float(rb[4 * q + 1]) + __uint_as_float(rs[4 * q + 1]),
+                                            __uint_as_float(rb[4 * q + 2]) + __uint_as_float(rs[4 * q + 2]),
+                                            __uint_as_float(rb[4 * q + 3]) + __uint_as_float(rs[4 * q + 3]));
                         }
                     }
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int br = 4 * i + lrow, row = brow0 + br, col = col0 + 4 * lch;
+                        const float4 pq = xb[br * 8 + (lch ^ (br & 7))];
+                        if (row < a.rows && col < a.n) {       // n % 4 == 0: a group of 4 columns is all in or all out
+                            float4 o;
+                            if (a.M) o = make_float4(mv[i].x - pq.x, mv[i].y - pq.y, mv[i].z - pq.z, mv[i].w - pq.w);
+                            else o = pq;
+                            *reinterpret_cast<float4*>(a.Out + (mrow + row) * a.n + col) = o;
+                        }
+                    }
+                    __syncwarp();
                 }
 #pragma unroll
-                for (int j = 0; j < 8; ++j) mv[j] = mn[j];
+                for (int i = 0; i < 8; ++i) mv[i] = mn[i];
             }
             asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
             __syncwarp();
@@ -436,11 +447,6 @@ constexpr int BT_F = 4;     // MMA steps (8 of K each) per head accumulator befo
                             // (every hand-over costs the pipeline about 500 cycles per K block: 2 steps were 25 % slower)
 constexpr int BT_MAXG = 8;  // 8-column groups per thread: (Ncp / 2) / 8 for Ncp <= 128
 
-__device__ __forceinline__ void tmem_ld8(unsigned taddr, unsigned (&v)[8]) {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
-                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
-                 : "r"(taddr) : "memory");
-}
 
 struct ProjTcArgs {
     float* Mout;      // [mats][rows][n] or nullptr
