@@ -343,7 +343,7 @@ bool launch_project_tc(Launcher& L, const float* A, const float* B, float* Mout,
         L.status = PSGD_E_CUDA;
         return true;
     }
-    ProjTcArgs a{B ? Mout : nullptr, P, rows, n, r, Ncp, proj_tc_stages(Ncp), B ? 1 : 0, nodes, (int*)(h->ws + h->lay.flags), skip};
+    ProjTcArgs a{B ? Mout : nullptr, P, rows, n, r, Ncp, proj_tc_nh(Ncp), B ? 1 : 0, nodes, (int*)(h->ws + h->lay.flags), skip};
     size_t smem = proj_tc_smem_bytes(Ncp);
     cudaFuncSetAttribute(k_project_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     L.begin(PSGD_K_PROJECT);

@@ -58,6 +58,13 @@ __device__ __forceinline__ void tmem_ld8(unsigned taddr, unsigned (&v)[8]) {
                  : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
                  : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tc_mma_tf32(unsigned d, unsigned long long da, unsigned long long db, unsigned idesc, unsigned acc) {
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
+                 ::"r"(d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tc_commit(unsigned bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void tma_load_3d_sw(unsigned dst, const CUtensorMap* map, int x, int y, int z, unsigned bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"
@@ -429,40 +436,48 @@ namespace psgd {
 // Projection on the tensor cores for ranks above 16:  P_i = (A_i [+ B_i]) Q  (Algorithm 1: P^(i) <-
 // Delta^(i) Q, with the error-feedback add of Eq. (7a) fused in; optionally stores M = A + B).
 // Per 32-column K block TMA brings the 128 x 32 tiles of A and B (128-byte swizzled); eight
-// converter warps form M in place, split it exactly into three TF32 terms (h + m + l, the head being
-// M itself, which the tensor core reads as TF32), write M back to HBM and hand the three tiles to
-// the MMA thread; Q^T arrives pre-split (k_split_pad_t).  Of the six tcgen05.mma products per 8 of K
-// the five small ones go into one tensor-memory accumulator; the head product h*h goes through the
-// rotating accumulators described below and is summed in float32 registers.
+// converter warps form M in place of A and write it back to HBM.  M is used as two TF32 terms: the
+// head is M itself (the tensor core reads a float32 as TF32, i.e. truncated), the second term is
+// M - head rounded to the nearest TF32 number, written over the tile of B; what is left (at most
+// 2^-21 |M|, zero mean) averages out over the hundreds of columns of a sum.  Q^T arrives pre-split
+// into three exact terms (k_split_pad_t).  Products: h x [h|m|l] and m x [h|m]; m x l is below 2^-32.
+//
+// Accumulation.  The tensor core adds to its float32 accumulator with truncation (measured on
+// like-signed sums: 3e-8 relative per accumulation, always toward zero, i.e. 2e-5 over the 512
+// steps of a 4096-long contraction).  The head product therefore accumulates one K block (4 steps)
+// at a time in tensor memory: accumulators take turns, and eight adder warps add each finished one
+// to float32 registers (round to nearest) while the next ones fill.  Adding up after every 2 steps
+// halves the bias again but was 25 % slower: every hand-over lengthens the life of a pipeline stage.
+//   up to 80 columns: the three terms of Q^T lie side by side as one B operand of 3 Ncp <= 256 rows:
+//     two MMAs per 8 of K into an accumulator set [head | small | small], all of it added up per K block;
+//   above: three MMAs (h x h, h x [m|l], m x [h|m]); the small products keep two accumulators for the
+//     whole contraction, the head product goes through the rotating accumulators.
+// One mbarrier per K block ("done", by tcgen05.commit) frees the shared-memory stages and tells the
+// adder warps that the accumulators of that K block can be read.
 // ---------------------------------------------------------------------------------------------
 constexpr int PT_THREADS = 576;   // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-9: converters, warps 10-17: adders + epilogue
-// The tensor core adds to its float32 accumulator with truncation (measured on like-signed sums: 3e-8 relative per
-// accumulation, always toward zero, i.e. 2e-5 over the 512 steps of a 4096-long contraction).  The head product h*h
-// therefore accumulates only BT_F steps in tensor memory: bt_heads() accumulators take turns and eight adder warps add
-// each finished one to float32 registers (round to nearest) while the next ones fill.
-constexpr int BT_NBMAX = 3; // most head accumulators in rotation
-// head accumulators in rotation: what fits beside the small accumulator in the 512 columns of tensor memory
-__host__ __device__ inline int bt_heads(int Ncp) { int nb = 512 / Ncp - 1; return nb > BT_NBMAX ? BT_NBMAX : nb; }
-constexpr int BT_F = 4;     // MMA steps (8 of K each) per head accumulator before it is added up in registers: one K block
-                            // (every hand-over costs the pipeline about 500 cycles per K block: 2 steps were 25 % slower)
-constexpr int BT_MAXG = 8;  // 8-column groups per thread: (Ncp / 2) / 8 for Ncp <= 128
-
+constexpr int BT_MAXG = 8;        // 8-column groups per thread: (Ncp / 2) / 8 for Ncp <= 128
 
 struct ProjTcArgs {
     float* Mout;      // [mats][rows][n] or nullptr
     float* P;         // [mats][rows][r]
-    int rows, n, r, Ncp, stages, has_b;
+    int rows, n, r, Ncp, nh, has_b;
     int nodes;        // matrices per Q
     int* flags;
     const int* skip;
 };
 
-__host__ __device__ inline size_t proj_tc_stage_bytes(int Ncp) { return (size_t)3 * TC_BM * TC_BK * 4 + (size_t)3 * Ncp * TC_BK * 4; }
-__host__ __device__ inline int proj_tc_stages(int Ncp) {
-    int s = (int)((size_t)220 * 1024 / proj_tc_stage_bytes(Ncp));
-    return s > 4 ? 4 : (s < 2 ? 2 : s);
+// Two shared-memory rings, as in the back-projection below: stages of 32 KB for the tiles of A and B (M and its second
+// TF32 term are formed in place) and a short ring for the three terms of Q^T.
+__host__ __device__ inline int proj_tc_nm(int Ncp) { return 3 * Ncp <= 256 ? 3 : 2; }
+__host__ __device__ inline int proj_tc_nh(int Ncp) {
+    const long long left = 224ll * 1024 - 1024 - 512 - (long long)proj_tc_nm(Ncp) * 3 * Ncp * TC_BK * 4;
+    const int nh = (int)(left / (2 * TC_BM * TC_BK * 4));
+    return nh > 6 ? 6 : nh;
 }
-__host__ __device__ inline size_t proj_tc_smem_bytes(int Ncp) { return (size_t)proj_tc_stages(Ncp) * proj_tc_stage_bytes(Ncp) + 1024 + 256; }
+__host__ __device__ inline size_t proj_tc_smem_bytes(int Ncp) {
+    return (size_t)proj_tc_nh(Ncp) * 2 * TC_BM * TC_BK * 4 + (size_t)proj_tc_nm(Ncp) * 3 * Ncp * TC_BK * 4 + 1024 + 512;
+}
 
 // Q [count][n][r] -> Qt[t][count][Ncp][n], t = 0, 1, 2: the transposed factor split exactly into three TF32 terms,
 // rows k >= r zero.  One thread per (matrix, k, column).
@@ -491,25 +506,29 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pt_smem_raw) + 1023) & ~(uintptr_t)1023);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr unsigned A_BYTES = TC_BM * TC_BK * 4;
-    constexpr int CPB = (TC_BK / 8) / BT_F;                    // head chunks per K block
+    constexpr unsigned LONG_BYTES = 2 * A_BYTES;               // [A tile -> M (head)][B tile -> second term]
     const unsigned B_BYTES = (unsigned)a.Ncp * TC_BK * 4;
-    const unsigned STAGE_BYTES = 3 * A_BYTES + 3 * B_BYTES;
-    const int NS = a.stages, NB = bt_heads(a.Ncp);
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(base + (size_t)NS * STAGE_BYTES);
-    const unsigned bar_full = smem_u32(bars), bar_conv = bar_full + 8 * NS, bar_empty = bar_conv + 8 * NS;
-    const unsigned bar_hfull = bar_empty + 8 * NS, bar_hfree = bar_hfull + 8 * NB, bar_acc = bar_hfree + 8 * NB;
-    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 3 * NS + 2 * NB + 1);
-    const unsigned smem_base = smem_u32(base);
+    const unsigned SHORT_BYTES = 3 * B_BYTES;                  // h, m, l of Q^T
+    const bool wide = 3 * a.Ncp <= 256;
+    const int NM = proj_tc_nm(a.Ncp);
+    const int NH = a.nh, NB = wide ? min(4, 512 / (3 * a.Ncp)) : min(3, (512 - 2 * a.Ncp) / a.Ncp);
+    unsigned char* short_base = base + (size_t)NH * LONG_BYTES;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(short_base + (size_t)NM * SHORT_BYTES);
+    const unsigned bar_hfull = smem_u32(bars), bar_conv = bar_hfull + 8 * NH, bar_done = bar_conv + 8 * NH;
+    const unsigned bar_bfull = bar_done + 8 * NH, bar_free = bar_bfull + 8 * NM, bar_acc = bar_free + 8 * NB;
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 3 * NH + NM + NB + 1);
+    const unsigned ring_u32 = smem_u32(base), short_u32 = smem_u32(short_base);
 
     const int rt = blockIdx.x, mat = blockIdx.y;
     const int qz = mat / a.nodes;
     const int KB = (a.n + TC_BK - 1) / TC_BK;
     unsigned ncols = 32;
-    while ((int)ncols < (NB + 1) * a.Ncp) ncols <<= 1;
+    while ((int)ncols < (wide ? NB * 3 : NB + 2) * a.Ncp) ncols <<= 1;
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_conv + 8 * s, 8); mbar_init(bar_empty + 8 * s, 1); }
-        for (int b = 0; b < NB; ++b) { mbar_init(bar_hfull + 8 * b, 1); mbar_init(bar_hfree + 8 * b, 8); }
+        for (int s = 0; s < NH; ++s) { mbar_init(bar_hfull + 8 * s, 1); mbar_init(bar_conv + 8 * s, 8); mbar_init(bar_done + 8 * s, 1); }
+        for (int s = 0; s < NM; ++s) mbar_init(bar_bfull + 8 * s, 1);
+        for (int b = 0; b < NB; ++b) mbar_init(bar_free + 8 * b, 8);
         mbar_init(bar_acc, 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -520,74 +539,78 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-    const unsigned tmem = *tmem_slot;      // small accumulator at column 0, head accumulator b at (1 + b) * Ncp
+    const unsigned tmem = *tmem_slot;      // wide: set b at 3 b Ncp; else two small accumulators at 0, head b at (2 + b) Ncp
     bool dead = false;
+    // K block j is "done" (all its MMAs have completed) in phase j / NH of bar_done[j % NH]
+    auto wait_done = [&](int j) { mbar_wait(bar_done + 8 * (j % NH), (unsigned)((j / NH) & 1), a.flags, dead); };
 
     if (warp == 0) {
-        // ---- TMA producer ----
+        // ---- TMA producer: tiles of A and B run NH - NM K blocks ahead of the terms of Q^T ----
         if (lane == 0) {
-            const unsigned tx = (a.has_b ? 2u : 1u) * A_BYTES + 3u * B_BYTES;
+            const int lead = NH - NM;
+            auto issue_ab = [&](int j) {
+                const int s = j % NH;
+                if (j >= NH) wait_done(j - NH);
+                const unsigned dst = ring_u32 + s * LONG_BYTES, bar = bar_hfull + 8 * s;
+                mbar_expect_tx(bar, (a.has_b ? 2u : 1u) * A_BYTES);
+                tma_load_3d_sw(dst, &tmA, j * TC_BK, rt * TC_BM, mat, bar);
+                if (a.has_b) tma_load_3d_sw(dst + A_BYTES, &tmB, j * TC_BK, rt * TC_BM, mat, bar);
+            };
+            for (int j = 0; j < min(lead, KB); ++j) issue_ab(j);
             for (int kb = 0; kb < KB; ++kb) {
-                const int s = kb % NS;
-                if (kb >= NS) mbar_wait(bar_empty + 8 * s, (unsigned)((kb / NS - 1) & 1), a.flags, dead);
-                const unsigned dst = smem_base + s * STAGE_BYTES;
-                const unsigned bar = bar_full + 8 * s;
-                mbar_expect_tx(bar, tx);
-                tma_load_3d_sw(dst, &tmA, kb * TC_BK, rt * TC_BM, mat, bar);
-                if (a.has_b) tma_load_3d_sw(dst + A_BYTES, &tmB, kb * TC_BK, rt * TC_BM, mat, bar);
-                tma_load_3d_sw(dst + 3 * A_BYTES, &tmQ0, kb * TC_BK, 0, qz, bar);
-                tma_load_3d_sw(dst + 3 * A_BYTES + B_BYTES, &tmQ1, kb * TC_BK, 0, qz, bar);
-                tma_load_3d_sw(dst + 3 * A_BYTES + 2 * B_BYTES, &tmQ2, kb * TC_BK, 0, qz, bar);
+                if (kb + lead < KB) issue_ab(kb + lead);
+                const int s = kb % NM;
+                if (kb >= NM) wait_done(kb - NM);
+                const unsigned dst = short_u32 + s * SHORT_BYTES, bar = bar_bfull + 8 * s;
+                mbar_expect_tx(bar, 3u * B_BYTES);
+                tma_load_3d_sw(dst, &tmQ0, kb * TC_BK, 0, qz, bar);
+                tma_load_3d_sw(dst + B_BYTES, &tmQ1, kb * TC_BK, 0, qz, bar);
+                tma_load_3d_sw(dst + 2 * B_BYTES, &tmQ2, kb * TC_BK, 0, qz, bar);
             }
         }
     } else if (warp == 1) {
         // ---- MMA issuer ----
         if (lane == 0) {
-            const unsigned idesc = tc_idesc(a.Ncp);
-            const unsigned d_small = tmem;
-            const int tp[6] = {2, 0, 1, 1, 0, 0}, tq[6] = {0, 2, 1, 0, 1, 0};   // (M term, Q term), h = 0, m = 1, l = 2
-            int chunk = 0;
+            const unsigned id1 = tc_idesc(a.Ncp), id2 = tc_idesc(2 * a.Ncp), id3 = tc_idesc(wide ? 3 * a.Ncp : a.Ncp);
             for (int kb = 0; kb < KB; ++kb) {
-                const int s = kb % NS;
-                mbar_wait(bar_conv + 8 * s, (unsigned)((kb / NS) & 1), a.flags, dead);
+                const int sh = kb % NH, sm = kb % NM, hb = kb % NB;
+                mbar_wait(bar_conv + 8 * sh, (unsigned)((kb / NH) & 1), a.flags, dead);
+                mbar_wait(bar_bfull + 8 * sm, (unsigned)((kb / NM) & 1), a.flags, dead);
+                if (kb >= NB) mbar_wait(bar_free + 8 * hb, (unsigned)((kb / NB - 1) & 1), a.flags, dead);   // registers took its last content
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-                const unsigned sb = smem_base + s * STAGE_BYTES;
-                const unsigned long long dA[3] = {tc_smem_desc(sb), tc_smem_desc(sb + A_BYTES), tc_smem_desc(sb + 2 * A_BYTES)};
-                const unsigned long long dQ[3] = {tc_smem_desc(sb + 3 * A_BYTES), tc_smem_desc(sb + 3 * A_BYTES + B_BYTES),
-                                                  tc_smem_desc(sb + 3 * A_BYTES + 2 * B_BYTES)};
+                const unsigned lb = ring_u32 + sh * LONG_BYTES, sb = short_u32 + sm * SHORT_BYTES;
+                const unsigned long long dAh = tc_smem_desc(lb), dAm = tc_smem_desc(lb + A_BYTES);
+                const unsigned long long dQh = tc_smem_desc(sb), dQm = tc_smem_desc(sb + B_BYTES);
+                if (wide) {
+                    const unsigned d_set = tmem + (unsigned)(3 * hb * a.Ncp);
 #pragma unroll
-                for (int k = 0; k < TC_BK / 8; ++k) {
-                    const int hb = chunk % NB;
-                    if (k % BT_F == 0 && chunk >= NB) {     // the registers have taken this accumulator's last content
-                        mbar_wait(bar_hfree + 8 * hb, (unsigned)((chunk / NB - 1) & 1), a.flags, dead);
-                        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                    for (int k = 0; k < TC_BK / 8; ++k) {
+                        const unsigned long long o = (unsigned long long)(2 * k);
+                        tc_mma_tf32(d_set, dAh + o, dQh + o, id3, k > 0 ? 1u : 0u);                        // h x [h|m|l]
+                        tc_mma_tf32(d_set + (unsigned)a.Ncp, dAm + o, dQh + o, id2, 1u);                   // m x [h|m]
                     }
-                    const unsigned d_head = tmem + (unsigned)((1 + hb) * a.Ncp);
-                    const unsigned long long o = (unsigned long long)(2 * k);
+                } else {
+                    const unsigned d_small = tmem, d_head = tmem + (unsigned)((2 + hb) * a.Ncp);
 #pragma unroll
-                    for (int t = 0; t < 6; ++t) {
-                        const unsigned acc = (t == 5) ? ((k % BT_F != 0) ? 1u : 0u) : ((kb > 0 || k > 0 || t > 0) ? 1u : 0u);
-                        asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
-                                     ::"r"(t == 5 ? d_head : d_small), "l"(dA[tp[t]] + o), "l"(dQ[tq[t]] + o), "r"(idesc), "r"(acc) : "memory");
-                    }
-                    if (k % BT_F == BT_F - 1) {
-                        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_hfull + 8 * hb) : "memory");
-                        ++chunk;
+                    for (int k = 0; k < TC_BK / 8; ++k) {
+                        const unsigned long long o = (unsigned long long)(2 * k);
+                        tc_mma_tf32(d_small, dAh + o, dQm + o, id2, (kb > 0 || k > 0) ? 1u : 0u);          // h x [m|l]
+                        tc_mma_tf32(d_small, dAm + o, dQh + o, id2, 1u);                                   // m x [h|m]
+                        tc_mma_tf32(d_head, dAh + o, dQh + o, id1, k > 0 ? 1u : 0u);                       // h x h
                     }
                 }
-                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_empty + 8 * s) : "memory");
+                tc_commit(bar_done + 8 * sh);
             }
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar_acc) : "memory");
+            tc_commit(bar_acc);
         }
     } else if (warp < 10) {
-        // ---- converters (warps 2-9): M = A + B in place, exact three-way split, M back to HBM ----
+        // ---- converters (warps 2-9): M = A + B in place and back to HBM; second TF32 term over the tile of B ----
         const int ct = tid - 64;                       // 0 .. 255
         for (int kb = 0; kb < KB; ++kb) {
-            const int s = kb % NS;
-            mbar_wait(bar_full + 8 * s, (unsigned)((kb / NS) & 1), a.flags, dead);
-            float4* t0 = reinterpret_cast<float4*>(base + (size_t)s * STAGE_BYTES);
+            const int sh = kb % NH;
+            mbar_wait(bar_hfull + 8 * sh, (unsigned)((kb / NH) & 1), a.flags, dead);
+            float4* t0 = reinterpret_cast<float4*>(base + (size_t)sh * LONG_BYTES);
             float4* t1 = t0 + A_BYTES / 16;
-            float4* t2 = t1 + A_BYTES / 16;
 #pragma unroll
             for (int u = 0; u < (TC_BM * TC_BK / 4) / 256; ++u) {
                 const int o = ct + u * 256;             // 16-byte unit of the swizzled tile
@@ -604,25 +627,22 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     }
                 }
                 const float xs[4] = {mv.x, mv.y, mv.z, mv.w};
-                float ms[4], ls[4];
+                float ms[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float h = __uint_as_float(__float_as_uint(xs[j]) & 0xFFFFE000u);
-                    const float r1 = xs[j] - h;
-                    ms[j] = __uint_as_float(__float_as_uint(r1) & 0xFFFFE000u);
-                    ls[j] = r1 - ms[j];
+                    ms[j] = __uint_as_float((__float_as_uint(xs[j] - h) + 0x1000u) & 0xFFFFE000u);   // rounded to nearest TF32
                 }
                 t1[o] = make_float4(ms[0], ms[1], ms[2], ms[3]);
-                t2[o] = make_float4(ls[0], ls[1], ls[2], ls[3]);
             }
             asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");    // generic writes -> visible to the tensor core
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_conv + 8 * s);
+            if (lane == 0) mbar_arrive(bar_conv + 8 * sh);
         }
     } else {
-        // ---- adders (warps 10-17): head accumulators -> float32 registers; then the epilogue ----
+        // ---- adders (warps 10-17): accumulators of each K block -> float32 registers; then the epilogue ----
         const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
-        const int half = (warp - 10) >> 2;              // which half of the columns this warp adds up
+        const int half = (warp - 10) >> 2;             // which half of the columns this warp adds up
         const int ng = a.Ncp >> 4;                     // 8-column groups per thread
         const unsigned lane_base = (unsigned)(quarter * 32) << 16;
         const unsigned col_base = (unsigned)(half * (a.Ncp >> 1));
@@ -631,33 +651,47 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         for (int g = 0; g < BT_MAXG; ++g)
 #pragma unroll
             for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
-        // adds head accumulator (chunk c) to the registers and hands it back to the MMA thread
-        auto drain = [&](int c) {
+        for (int c = 0; c < KB; ++c) {
             const int hb = c % NB;
-            mbar_wait(bar_hfull + 8 * hb, (unsigned)((c / NB) & 1), a.flags, dead);
+            wait_done(c);
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-            const unsigned t0 = tmem + lane_base + (unsigned)((1 + hb) * a.Ncp) + col_base;
+            if (wide) {
+                const unsigned ts = tmem + lane_base + (unsigned)(3 * hb * a.Ncp) + col_base;
 #pragma unroll
-            for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
-                if (g2 < ng) {
-                    unsigned v0[8], v1[8];
-                    tmem_ld8(t0 + 8 * g2, v0);
-                    if (g2 + 1 < ng) tmem_ld8(t0 + 8 * (g2 + 1), v1);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+                for (int g = 0; g < 5; ++g) {              // Ncp <= 80: at most 5 groups of 8 columns per thread
+                    if (g < ng) {
+                        unsigned vh[8], v1[8], v2[8];
+                        tmem_ld8(ts + 8 * g, vh);
+                        tmem_ld8(ts + (unsigned)a.Ncp + 8 * g, v1);
+                        tmem_ld8(ts + (unsigned)(2 * a.Ncp) + 8 * g, v2);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) acc[g2][j] += __uint_as_float(v0[j]);
-                    if (g2 + 1 < ng) {
+                        for (int j = 0; j < 8; ++j) acc[g][j] += __uint_as_float(vh[j]) + (__uint_as_float(v1[j]) + __uint_as_float(v2[j]));
+                    }
+                }
+            } else {
+                const unsigned t0 = tmem + lane_base + (unsigned)((2 + hb) * a.Ncp) + col_base;
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[g2 + 1][j] += __uint_as_float(v1[j]);
+                for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
+                    if (g2 < ng) {
+                        unsigned v0[8], v1[8];
+                        tmem_ld8(t0 + 8 * g2, v0);
+                        if (g2 + 1 < ng) tmem_ld8(t0 + 8 * (g2 + 1), v1);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) acc[g2][j] += __uint_as_float(v0[j]);
+                        if (g2 + 1 < ng) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) acc[g2 + 1][j] += __uint_as_float(v1[j]);
+                        }
                     }
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_hfree + 8 * hb);
-        };
-        for (int c = 0; c < KB * CPB; ++c) drain(c);
-        // ---- epilogue: P = registers + small accumulator ----
+            if (lane == 0) mbar_arrive(bar_free + 8 * hb);
+        }
+        // ---- epilogue: P = registers (+ the small accumulators) ----
         mbar_wait(bar_acc, 0u, a.flags, dead);
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
         const int row = rt * TC_BM + quarter * 32 + lane;
@@ -666,8 +700,17 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         for (int g = 0; g < BT_MAXG; ++g) {
             if (g < ng) {
                 unsigned v[8];
-                tmem_ld8(tmem + lane_base + col_base + 8 * g, v);
-                asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+                if (!wide) {
+                    unsigned w[8];
+                    tmem_ld8(tmem + lane_base + col_base + 8 * g, v);
+                    tmem_ld8(tmem + lane_base + (unsigned)a.Ncp + col_base + 8 * g, w);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(w[j]));
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) v[j] = 0u;
+                }
                 if (row < a.rows) {
                     const int j0 = (int)col_base + 8 * g;
 #pragma unroll
@@ -741,13 +784,6 @@ __device__ __forceinline__ unsigned long long tc_smem_desc_mn(unsigned addr, uns
     d |= (unsigned long long)1 << 46;
     d |= (unsigned long long)1 << 61;
     return d;
-}
-__device__ __forceinline__ void tc_mma_tf32(unsigned d, unsigned long long da, unsigned long long db, unsigned idesc, unsigned acc) {
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
-                 ::"r"(d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void tc_commit(unsigned bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
 }
 
 __global__ void __launch_bounds__(PT_THREADS, 1)
