@@ -31,7 +31,7 @@ UNIT = "GB/s"
 FALLBACK_HBM = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per element of one launch, from the ncu captures summarised under
 # profiles/ (taken on the 16384x4096, N=4 workload, where traffic grows in proportion to the elements)
-TRAFFIC_BYTES_PER_ELEMENT = {"k_fused_step": 11.86}
+TRAFFIC_BYTES_PER_ELEMENT = {"k_fused_step": 11.87}
 
 # default (rank, nodes, refresh period) per workload id
 DEFAULTS = {2: (8, 8, 50), 3: (16, 16, 20), 4: (32, 8, 100), 5: (16, 4, 0), 1: (4, 4, 5)}
