@@ -222,15 +222,14 @@ def make_inputs(workload, N, device, nbuf):
     return bufs
 
 
-def timed_steps(torch, handles, bufs, steps, dist_barrier):
+def timed_steps(torch, stack, bufs, steps, dist_barrier):
+    """K steps of the whole stack; every step forks from and joins the current stream, where the two events are."""
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     dist_barrier()
     torch.cuda.synchronize()
     ev0.record()
     for s in range(steps):
-        G = bufs[s % len(bufs)]
-        for h, g in zip(handles, G):
-            h.step(g)
+        stack.step(bufs[s % len(bufs)])
     ev1.record()
     torch.cuda.synchronize()
     dist_barrier()
@@ -307,16 +306,18 @@ def run_ours(args):
     handles = build_handles(args.workload, r, N, tau, device, args.mode)
     torch.cuda.synchronize()
 
+    from paper_2509_11254_b200 import StreamedStack
+
+    stack = StreamedStack(handles, device)       # one stream per shape class
     # warm-up (includes the t = 0 refresh when tau > 0)
     for s in range(max(args.warmup, 3)):
-        for h, g in zip(handles, bufs[s % nbuf]):
-            h.step(g)
+        stack.step(bufs[s % nbuf])
     torch.cuda.synchronize()
 
     sampler = ClockSampler(local)
     sampler.start()
     l0 = sum(h.launch_count() for h in handles)
-    ms_total = timed_steps(torch, handles, bufs, args.steps, barrier)
+    ms_total = timed_steps(torch, stack, bufs, args.steps, barrier)
     l1 = sum(h.launch_count() for h in handles)
     clocks = sampler.stop()
     ms_total = reps.max_over_ranks(ms_total)
@@ -369,6 +370,7 @@ def run_ours(args):
                        "r": r, "N": N, "refresh_period": tau, "mode": args.mode,
                        "launch_plan": [{k: p[k] for k in ("single_pass", "WC", "CS", "KC", "active_clusters")} for p in plans],
                        "l2": "inputs (%.2f GB of G per step, 2 alternating sets) exceed L2" % (g_bytes / 1e9),
+                       "streams": len(handles),
                        "parallelism": "replicas" if world > 1 else "single"},
             "north_star_frac": alg_bytes / ms_step / 1e6 / peak,
             "north_star_bytes_per_step": alg_bytes,
@@ -383,13 +385,11 @@ def run_ours(args):
         Ph = [torch.empty(h.P_hat.shape, dtype=torch.float32).pin_memory() for h in handles]
         Qh = [torch.empty(h.Q.shape, dtype=torch.float32).pin_memory() for h in handles]
         stage = bufs[0]
-        for h, gh, st, ph, qh in zip(handles, Gh, stage, Ph, Qh):
-            h.step_host(gh, st, ph, qh)
+        stack.step_host(Gh, stage, Ph, Qh)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         for s in range(e2e_steps):
-            for h, gh, st, ph, qh in zip(handles, Gh, stage, Ph, Qh):
-                h.step_host(gh, st, ph, qh)
+            stack.step_host(Gh, stage, Ph, Qh)
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) / e2e_steps
         line["e2e"] = {"value": g_bytes / dt / 1e9, "unit": UNIT, "h2d_bytes_per_step": g_bytes,

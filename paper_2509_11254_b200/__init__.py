@@ -14,3 +14,4 @@ from .binding import (  # noqa: F401
     PSGD_W_TIMEOUT,
     KERNEL_FAMILIES,
 )
+from .stack import StreamedStack  # noqa: F401,E402

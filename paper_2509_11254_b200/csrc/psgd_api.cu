@@ -657,8 +657,8 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
         k_apply<<<dim3(ceil_div(m, 32), cnt), 256, (size_t)32 * ell * 4, L.st>>>(ap);
         L.end();
     };
-    // Stopping test (blocks of <= 48 columns, where a Rayleigh-Ritz step is cheap): every third sweep the top-r
-    // Ritz basis is compared with the one of the previous check; once it has stopped moving in every matrix of
+    // Stopping test (blocks of <= 48 columns, where a Rayleigh-Ritz step is cheap): after sweeps 2, 4, 6, 9, 12, ... the
+    // top-r Ritz basis is compared with the one of the previous check; once it has stopped moving in every matrix of
     // the handle (rule in k_refresh_decide) the remaining kernels of this refresh return at once.  With geometric
     // convergence the error left is below the last movement.  Inputs that never get there run all the sweeps.
     float* Pold = (float*)(ws + h->lay.Pold);
@@ -675,7 +675,8 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
         k_reduce_q<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(part, nullptr, Z, n, ell, 1, Sb, cnt, skip);
         L.end();
         if (it + 1 == h->refresh_iters) break;
-        if (adaptive && (it - it0 + 1) % 3 == 0) {
+        const int swept = it - it0 + 1;
+        if (adaptive && (swept <= 6 ? swept % 2 == 0 : swept % 3 == 0)) {
             rayleigh_ritz();
             if (nchecks > 0) {
                 const int nparts = ceil_div(m, GR_ROWS), nblk = ceil_div(r, 64), nb = ceil_div(m, 64);

@@ -915,9 +915,10 @@ __global__ void __launch_bounds__(256) k_subspace_change(const float* Pold, cons
         dpart[(size_t)c * gridDim.x + blockIdx.x] = t;
     }
 }
-// Rule per matrix (d = movement since the previous check, dprev the one before):
-//   d <= 1e-5 and still halving (d <= dprev / 2: geometric convergence, the error left is below d), or
-//   d <= 3e-6 (the float32 floor of two Ritz bases computed three sweeps apart).
+// Rule per matrix (d = movement since the previous check, dprev the one before, q = d / dprev):
+//   q < 1 and d q / (1 - q) <= 1e-5: with geometric convergence the movements still to come add up to that
+//   (d <= 1e-5 while halving is the case q = 1/2), or
+//   d <= 3e-6 (the float32 floor of two Ritz bases computed a few sweeps apart).
 __global__ void k_refresh_decide(const double* dpart, int nb, int count, double* dprev, int have_prev, int* done) {
     if (*done) return;
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
@@ -926,7 +927,11 @@ __global__ void k_refresh_decide(const double* dpart, int nb, int count, double*
         double t = 0.0;
         for (int b = 0; b < nb; ++b) t += dpart[(size_t)c * nb + b];
         const double d = sqrt(t);
-        const bool ok = (d <= 3e-6) || (have_prev && d <= 1e-5 && d <= 0.5 * dprev[c]);
+        bool ok = d <= 3e-6;
+        if (!ok && have_prev && d < dprev[c]) {
+            const double q = d / dprev[c];
+            ok = d * q / (1.0 - q) <= 1e-5;
+        }
         if (!ok) all = 0;
         dprev[c] = d;
     }
