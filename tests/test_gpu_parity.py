@@ -422,6 +422,39 @@ def test_full_size_config4_ffn_class(torch_cuda):
     assert plan["single_pass"] == 0
 
 
+def test_streamed_stack_equals_sequential_steps(torch_cuda):
+    """Two shape classes stepped on one stream each (the benchmark's launch configuration) give bit for bit
+    what stepping them one after the other gives: the handles share nothing."""
+    from paper_2509_11254_b200 import PowerSGDPlus, StreamedStack
+
+    torch = torch_cuda
+    shapes = [(520, 256, 3), (384, 384, 2)]
+    N, r, tau = 4, 8, 3
+
+    def run(streamed):
+        hs = [PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=7 + i, count=c, mode="deferred") for i, (m, n, c) in enumerate(shapes)]
+        st = StreamedStack(hs)
+        for t in range(5):
+            G = [synth.make_gradients_torch(2, m, n, N, c, step=t, device="cuda:0") for (m, n, c) in shapes]
+            if streamed:
+                st.step(G)
+            else:
+                for h, g in zip(hs, G):
+                    h.step(g)
+        torch.cuda.synchronize()
+        for h in hs:
+            h.materialize_error()
+            assert h.last_status() == 0
+        out = [(h.P_hat.clone(), h.Q.clone(), h.E.clone()) for h in hs]
+        for h in hs:
+            h.close()
+        return out
+
+    for a, b in zip(run(True), run(False)):
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
+
+
 # ---- degenerate inputs ------------------------------------------------------------------------
 def _invariants(comp, M, P_mean, r, tag):
     """What must hold for ANY valid orthonormal factor (several are correct when P is rank deficient)."""
