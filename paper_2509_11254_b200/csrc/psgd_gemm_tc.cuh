@@ -458,6 +458,61 @@ namespace psgd {
 constexpr int PT_THREADS = 576;   // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-9: converters, warps 10-17: adders + epilogue
 constexpr int BT_MAXG = 8;        // 8-column groups per thread: (Ncp / 2) / 8 for Ncp <= 128
 
+// Adder warps of the projection and back-projection kernels: adds the accumulators of one K block (set / head
+// accumulator hb) to the thread's float32 registers.  The thread owns tensor-memory lane (lane_base) and the ng groups
+// of 8 columns starting at col_base.  wide: the set is [head | small | small] at 3 hb Ncp; else the head accumulator
+// at (2 + hb) Ncp (the two small accumulators at 0 stay for the whole contraction).
+__device__ __forceinline__ void tc_add_up(float (&acc)[BT_MAXG][8], unsigned tmem, unsigned lane_base, unsigned col_base,
+                                          int Ncp, int ng, bool wide, int hb) {
+    if (wide) {
+        const unsigned ts = tmem + lane_base + (unsigned)(3 * hb * Ncp) + col_base;
+#pragma unroll
+        for (int g = 0; g < 5; ++g) {              // Ncp <= 80: at most 5 groups of 8 columns per thread
+            if (g < ng) {
+                unsigned vh[8], v1[8], v2[8];
+                tmem_ld8(ts + 8 * g, vh);
+                tmem_ld8(ts + (unsigned)Ncp + 8 * g, v1);
+                tmem_ld8(ts + (unsigned)(2 * Ncp) + 8 * g, v2);
+                asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[g][j] += __uint_as_float(vh[j]) + (__uint_as_float(v1[j]) + __uint_as_float(v2[j]));
+            }
+        }
+    } else {
+        const unsigned t0 = tmem + lane_base + (unsigned)((2 + hb) * Ncp) + col_base;
+#pragma unroll
+        for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
+            if (g2 < ng) {
+                unsigned v0[8], v1[8];
+                tmem_ld8(t0 + 8 * g2, v0);
+                if (g2 + 1 < ng) tmem_ld8(t0 + 8 * (g2 + 1), v1);
+                asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[g2][j] += __uint_as_float(v0[j]);
+                if (g2 + 1 < ng) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc[g2 + 1][j] += __uint_as_float(v1[j]);
+                }
+            }
+        }
+    }
+}
+// The small accumulators (not wide) added to the registers of column group g; wide: nothing is left in tensor memory.
+__device__ __forceinline__ void tc_add_small(float (&v)[8], const float (&acc)[8], unsigned tmem, unsigned lane_base, unsigned col_base,
+                                             int Ncp, bool wide, int g) {
+    if (!wide) {
+        unsigned s1[8], s2[8];
+        tmem_ld8(tmem + lane_base + col_base + 8 * g, s1);
+        tmem_ld8(tmem + lane_base + (unsigned)Ncp + col_base + 8 * g, s2);
+        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = acc[j] + (__uint_as_float(s1[j]) + __uint_as_float(s2[j]));
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = acc[j];
+    }
+}
+
 struct ProjTcArgs {
     float* Mout;      // [mats][rows][n] or nullptr
     float* P;         // [mats][rows][r]
@@ -655,38 +710,7 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             const int hb = c % NB;
             wait_done(c);
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-            if (wide) {
-                const unsigned ts = tmem + lane_base + (unsigned)(3 * hb * a.Ncp) + col_base;
-#pragma unroll
-                for (int g = 0; g < 5; ++g) {              // Ncp <= 80: at most 5 groups of 8 columns per thread
-                    if (g < ng) {
-                        unsigned vh[8], v1[8], v2[8];
-                        tmem_ld8(ts + 8 * g, vh);
-                        tmem_ld8(ts + (unsigned)a.Ncp + 8 * g, v1);
-                        tmem_ld8(ts + (unsigned)(2 * a.Ncp) + 8 * g, v2);
-                        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[g][j] += __uint_as_float(vh[j]) + (__uint_as_float(v1[j]) + __uint_as_float(v2[j]));
-                    }
-                }
-            } else {
-                const unsigned t0 = tmem + lane_base + (unsigned)((2 + hb) * a.Ncp) + col_base;
-#pragma unroll
-                for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
-                    if (g2 < ng) {
-                        unsigned v0[8], v1[8];
-                        tmem_ld8(t0 + 8 * g2, v0);
-                        if (g2 + 1 < ng) tmem_ld8(t0 + 8 * (g2 + 1), v1);
-                        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[g2][j] += __uint_as_float(v0[j]);
-                        if (g2 + 1 < ng) {
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) acc[g2 + 1][j] += __uint_as_float(v1[j]);
-                        }
-                    }
-                }
-            }
+            tc_add_up(acc, tmem, lane_base, col_base, a.Ncp, ng, wide, hb);
             asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_free + 8 * hb);
@@ -699,23 +723,13 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 #pragma unroll
         for (int g = 0; g < BT_MAXG; ++g) {
             if (g < ng) {
-                unsigned v[8];
-                if (!wide) {
-                    unsigned w[8];
-                    tmem_ld8(tmem + lane_base + col_base + 8 * g, v);
-                    tmem_ld8(tmem + lane_base + (unsigned)a.Ncp + col_base + 8 * g, w);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(w[j]));
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) v[j] = 0u;
-                }
+                float v[8];
+                tc_add_small(v, acc[g], tmem, lane_base, col_base, a.Ncp, wide, g);
                 if (row < a.rows) {
                     const int j0 = (int)col_base + 8 * g;
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        if (j0 + j < a.r) out[j0 + j] = acc[g][j] + __uint_as_float(v[j]);
+                        if (j0 + j < a.r) out[j0 + j] = v[j];
                 }
             }
         }
@@ -939,38 +953,7 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
             const int hb = c % NB;
             wait_done(c);
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-            if (wide) {
-                const unsigned ts = tmem + lane_base + (unsigned)(3 * hb * a.Ncp) + col_base;
-#pragma unroll
-                for (int g = 0; g < 5; ++g) {              // Ncp <= 80: at most 5 groups of 8 columns per thread
-                    if (g < ng) {
-                        unsigned vh[8], v1[8], v2[8];
-                        tmem_ld8(ts + 8 * g, vh);
-                        tmem_ld8(ts + (unsigned)a.Ncp + 8 * g, v1);
-                        tmem_ld8(ts + (unsigned)(2 * a.Ncp) + 8 * g, v2);
-                        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[g][j] += __uint_as_float(vh[j]) + (__uint_as_float(v1[j]) + __uint_as_float(v2[j]));
-                    }
-                }
-            } else {
-                const unsigned t0 = tmem + lane_base + (unsigned)((2 + hb) * a.Ncp) + col_base;
-#pragma unroll
-                for (int g2 = 0; g2 < BT_MAXG; g2 += 2) {
-                    if (g2 < ng) {
-                        unsigned v0[8], v1[8];
-                        tmem_ld8(t0 + 8 * g2, v0);
-                        if (g2 + 1 < ng) tmem_ld8(t0 + 8 * (g2 + 1), v1);
-                        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[g2][j] += __uint_as_float(v0[j]);
-                        if (g2 + 1 < ng) {
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) acc[g2 + 1][j] += __uint_as_float(v1[j]);
-                        }
-                    }
-                }
-            }
+            tc_add_up(acc, tmem, lane_base, col_base, a.Ncp, ng, wide, hb);
             asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_free + 8 * hb);
@@ -983,23 +966,13 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
 #pragma unroll
         for (int g = 0; g < BT_MAXG; ++g) {
             if (g < ng) {
-                unsigned v[8];
-                if (!wide) {
-                    unsigned w[8];
-                    tmem_ld8(tmem + lane_base + col_base + 8 * g, v);
-                    tmem_ld8(tmem + lane_base + (unsigned)a.Ncp + col_base + 8 * g, w);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(w[j]));
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) v[j] = 0u;
-                }
+                float v[8];
+                tc_add_small(v, acc[g], tmem, lane_base, col_base, a.Ncp, wide, g);
                 if (col < a.n) {
                     const int j0 = (int)col_base + 8 * g;
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        if (j0 + j < a.r) out[j0 + j] = (KB > 0) ? acc[g][j] + __uint_as_float(v[j]) : 0.f;
+                        if (j0 + j < a.r) out[j0 + j] = (KB > 0) ? v[j] : 0.f;
                 }
             }
         }
