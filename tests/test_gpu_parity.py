@@ -157,6 +157,19 @@ def test_residual_on_tensor_cores(torch_cuda, m, n, r, N, count, form):
     run_case(torch_cuda, m, n, r, N, tau=0, steps=2, workload=4, count=count, Einit=0.01, error_form=form, check_dense=True)
 
 
+@pytest.mark.parametrize("m,n,r,N,count", [
+    (1100, 548, 17, 2, 2),     # 17 -> 32 columns: four accumulator sets, one group of 8 columns per adder thread
+    (772, 300, 40, 3, 1),      # 48 columns: three sets; ragged rows and columns, 7 K blocks per split
+    (1536, 640, 72, 2, 1),     # 80 columns: the widest one-operand form (3 x 80 = 240 <= 256), two sets
+    (900, 644, 88, 2, 1),      # 96 columns: three MMAs, three rotating head accumulators
+    (1028, 516, 128, 1, 2),    # 128 columns: two rotating head accumulators, a single node
+])
+def test_tensor_core_step_kernels_all_widths(torch_cuda, m, n, r, N, count):
+    """Every layout class of the r > 16 projection / back-projection / residual kernels (number of accumulator
+    sets, one-operand or three-MMA form, column groups per adder thread), P_i, P~, Q_i, Q and E against the oracle."""
+    run_case(torch_cuda, m, n, r, N, tau=0, steps=2, workload=4, count=count, Einit=0.01, check_dense=True)
+
+
 @pytest.mark.parametrize("K,mode", [(2, "eager"), (3, "deferred")])
 def test_k_step_power_iteration(torch_cuda, K, mode):
     """Eq. (8): K power steps per iteration (the deferred mode falls back to the three-pass kernels)."""
