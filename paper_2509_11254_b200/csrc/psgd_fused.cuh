@@ -155,26 +155,6 @@ __device__ __forceinline__ void butterfly_reduce(float (&v)[NV], int lane) {
     if (NV == 16) v[0] += __shfl_xor_sync(0xffffffffu, v[0], 1);
 }
 
-// Two packed floats in one 64-bit register (low half = .x), kept packed from the load to the last use so
-// that no pack / unpack moves are needed around the packed FMA.
-typedef unsigned long long f2p;
-__device__ __forceinline__ f2p pack2(float x, float y) {
-    f2p d;
-    asm("mov.b64 %0, {%1, %2};\n" : "=l"(d) : "f"(x), "f"(y));
-    return d;
-}
-__device__ __forceinline__ float2 unpack2(f2p v) {
-    float2 d;
-    asm("mov.b64 {%0, %1}, %2;\n" : "=f"(d.x), "=f"(d.y) : "l"(v));
-    return d;
-}
-// d = a * b + c on two packed floats (one instruction slot on sm_100)
-__device__ __forceinline__ f2p ffma2(f2p a, f2p b, f2p c) {
-    f2p d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-
 // A float delivered to a peer CTA's shared memory; the peer's mbarrier counts the 4 bytes.
 __device__ __forceinline__ void st_async_cluster_f32(unsigned local_addr, unsigned local_bar, unsigned rank, float v) {
     unsigned raddr, rbar;
