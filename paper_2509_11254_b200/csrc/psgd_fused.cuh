@@ -190,7 +190,6 @@ __global__ void __launch_bounds__(FU_THREADS, 1)
 k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmM, FusedArgs a) {
     using Ge = FusedGeom<WC>;
     constexpr int BW = Ge::BW, NBX = Ge::NBX, CPL = Ge::CPL, NCG = Ge::NCG, RS = Ge::RS, NRC = Ge::NRC, NST = Ge::NST, TPN = Ge::TPN;
-    constexpr int NV = FU_RG * RP;         // per-lane partial sums of one warp task
     constexpr int PR = FU_R * RP;          // entries of one block of P
     constexpr int RP2 = RP / 2;
     constexpr unsigned STAGE_BYTES = Ge::STAGE_FLOATS * 4;
