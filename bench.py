@@ -51,6 +51,8 @@ def parse():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-refresh", action="store_true", help="tau = 0 (plain PowerSGD steps only)")
     ap.add_argument("--refresh-period", type=int, default=None, help="override the workload's refresh period tau")
+    ap.add_argument("--grad-dtype", default="float32", choices=["float32", "bfloat16"],
+                    help="storage type of the gradients G (bfloat16: 2 bytes per element read instead of 4)")
     return ap.parse_args()
 
 
@@ -122,11 +124,11 @@ def stack_for(workload):
     return synth.STACKS[workload]
 
 
-def algorithmic_bytes(shapes, r, N):
-    """North-star accounting: read G, read E, write E per element (12 B) plus the P/Q traffic."""
+def algorithmic_bytes(shapes, r, N, g_bytes_per_element=4):
+    """North-star accounting: read G, read E, write E per element (12 B with float32 G) plus the P/Q traffic."""
     el = sum(m * n * c for m, n, c in shapes) * N
     pq = sum(4 * (2 * N * m * r + 2 * m * r + 2 * N * n * r + 2 * n * r) * c for m, n, c in shapes)
-    return 12 * el + pq, 4 * el
+    return (8 + g_bytes_per_element) * el + pq, g_bytes_per_element * el
 
 
 # ----------------------------------------------------------------------------
@@ -205,20 +207,24 @@ def run_reference(args):
 # ----------------------------------------------------------------------------
 # GPU arm
 # ----------------------------------------------------------------------------
-def build_handles(workload, r, N, tau, device, mode, seed=1):
+def build_handles(workload, r, N, tau, device, mode, seed=1, grad_dtype="float32"):
     from paper_2509_11254_b200 import PowerSGDPlus
 
-    return [PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=seed + i, count=c, device=device, mode=mode)
+    return [PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=seed + i, count=c, device=device, mode=mode, grad_dtype=grad_dtype)
             for i, (m, n, c) in enumerate(stack_for(workload))]
 
 
-def make_inputs(workload, N, device, nbuf):
+def make_inputs(workload, N, device, nbuf, grad_dtype="float32"):
+    import torch
     from paper_2509_11254_b200 import synth
 
     bufs = []
     for b in range(nbuf):
-        bufs.append([synth.make_gradients_torch(workload, m, n, N, c, step=b, device=device)
-                     for (m, n, c) in stack_for(workload)])
+        row = []
+        for (m, n, c) in stack_for(workload):
+            g = synth.make_gradients_torch(workload, m, n, N, c, step=b, device=device)
+            row.append(g.to(torch.bfloat16) if grad_dtype == "bfloat16" else g)
+        bufs.append(row)
     return bufs
 
 
@@ -299,11 +305,12 @@ def run_ours(args):
         tau = 0
     shapes = stack_for(args.workload)
     peak, peak_kind = peaks()
-    alg_bytes, g_bytes = algorithmic_bytes(shapes, r, N)
+    gbpe = 2 if args.grad_dtype == "bfloat16" else 4
+    alg_bytes, g_bytes = algorithmic_bytes(shapes, r, N, gbpe)
 
     nbuf = 1 if args.workload == 4 else 2
-    bufs = make_inputs(args.workload, N, device, nbuf)
-    handles = build_handles(args.workload, r, N, tau, device, args.mode)
+    bufs = make_inputs(args.workload, N, device, nbuf, args.grad_dtype)
+    handles = build_handles(args.workload, r, N, tau, device, args.mode, grad_dtype=args.grad_dtype)
     torch.cuda.synchronize()
 
     from paper_2509_11254_b200 import StreamedStack
@@ -342,7 +349,7 @@ def run_ours(args):
     n_refresh = sum(1 for h, t0 in zip(handles, t_now) for s in range(prof_steps) if tau > 0 and (t0 + s) % tau == 0)
     n_ssp = prof_steps * len(handles) - n_refresh
     el = sum(m * n * c for m, n, c in shapes) * N
-    per_family_bytes = {"project": 12 * el, "backproject": 4 * el, "residual": 8 * el}
+    per_family_bytes = {"project": (8 + gbpe) * el, "backproject": 4 * el, "residual": 8 * el}
     dom = max(("project", "backproject", "residual"), key=lambda k: fam.get(k, [0, 0])[0])
     # a family's kernels run once per handle per step; average duration of one launch set over all handles
     dom_ms_per_step = fam[dom][0] / prof_steps if prof_steps else float("nan")
@@ -355,7 +362,7 @@ def run_ours(args):
     kernel_name = "k_fused_step" if (dom == "project" and single_pass) else "k_" + dom
     # DRAM bytes per element of the dominant kernel from the committed ncu capture (profiles/), scaled to this
     # workload's elements; None for kernels without a current capture
-    traffic = TRAFFIC_BYTES_PER_ELEMENT.get(kernel_name)
+    traffic = TRAFFIC_BYTES_PER_ELEMENT.get(kernel_name) if args.grad_dtype == "float32" else None   # captured with float32 G
     traffic = traffic * el * ssp_frac if traffic is not None else None
     roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak if achieved else None, "traffic": traffic, "peak_source": f"of {peak_kind}",
@@ -370,7 +377,7 @@ def run_ours(args):
                        "r": r, "N": N, "refresh_period": tau, "mode": args.mode,
                        "launch_plan": [{k: p[k] for k in ("single_pass", "WC", "CS", "KC", "active_clusters")} for p in plans],
                        "l2": "inputs (%.2f GB of G per step, 2 alternating sets) exceed L2" % (g_bytes / 1e9),
-                       "streams": len(handles),
+                       "streams": len(handles), "grad_dtype": args.grad_dtype,
                        "parallelism": "replicas" if world > 1 else "single"},
             "north_star_frac": alg_bytes / ms_step / 1e6 / peak,
             "north_star_bytes_per_step": alg_bytes,
@@ -379,7 +386,7 @@ def run_ours(args):
     if rank == 0 and not args.no_e2e:
         # end to end through the host-buffer entry point: H2D of G and D2H of (P~, Q) inside the timed region
         e2e_steps = max(1, min(args.steps, 5))
-        Gh = [torch.empty(g.shape, dtype=torch.float32).pin_memory() for g in bufs[0]]
+        Gh = [torch.empty(g.shape, dtype=g.dtype).pin_memory() for g in bufs[0]]
         for gh, g in zip(Gh, bufs[0]):
             gh.copy_(g)
         Ph = [torch.empty(h.P_hat.shape, dtype=torch.float32).pin_memory() for h in handles]

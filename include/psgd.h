@@ -71,7 +71,12 @@ typedef enum {
 #define PSGD_OPT_POWER_STEPS 6     /* K >= 1 power steps per SSP iteration (Eq. (8)); 1 (default) is PowerSGD's single
                                       step (Eq. (9)); K > 1 runs the three-pass kernels */
 #define PSGD_OPT_REFRESH_ADAPTIVE 7 /* 1 (default): a refresh whose block has <= 48 columns stops its sweeps once the top-r
-                                      basis has stopped moving between two checks (<= 1e-5 and halving, or <= 3e-6); 0: all the sweeps */
+                                      basis has stopped moving (movement d between two checks, q = d / d_prev < 1 and d q / (1 - q) <= 1e-5,
+                                      or d <= 3e-6); 0: all the sweeps */
+
+#define PSGD_OPT_GRAD_BF16 8        /* 0 (default): the gradients G are float32; 1: bfloat16 (the same [count][N][m][n] layout, 2 bytes
+                                      per element), widened exactly to float32 as they are read.  The single-pass kernel then moves
+                                      10 instead of 12 bytes per element; the other paths first form M = G + E in the E buffer */
 
 /* buffers that psgd_debug_ptr exposes (test use only; valid until the next step) */
 #define PSGD_BUF_P_NODE 1   /* P^(i)   [count][N][m][r] */
@@ -126,14 +131,14 @@ psgd_status psgd_reset(psgd_handle* h, psgd_stream stream);
  * One iteration t of Algorithm 2 without the optimizer update:
  *   Delta_i = g_i + e_i (Eq. (7a));  SVD-Comp if refresh_period > 0 and
  *   t mod refresh_period == 0, else SSP-Comp (Algorithm 1);  e_i <- Delta_i - Delta^_i;  t <- t + 1.
- * G: DEVICE, read-only.  P_hat (DEVICE, may be NULL) receives P~_t.  D_hat
+ * G: DEVICE, read-only, float32 (bfloat16 with PSGD_OPT_GRAD_BF16).  P_hat (DEVICE, may be NULL) receives P~_t.  D_hat
  * (DEVICE, may be NULL) receives the dense global reconstruction P~_t Q_t^T.
  * Q (attached) is replaced by Q_t.  Enqueued on `stream`; does not synchronise.
  */
-psgd_status psgd_step(psgd_handle* h, const float* G, float* P_hat, float* D_hat, psgd_stream stream);
+psgd_status psgd_step(psgd_handle* h, const void* G, float* P_hat, float* D_hat, psgd_stream stream);
 
 /* The same iteration with SVD-Comp forced (Algorithm 1, second function; Definition 3). */
-psgd_status psgd_refresh(psgd_handle* h, const float* G, float* P_hat, float* D_hat, psgd_stream stream);
+psgd_status psgd_refresh(psgd_handle* h, const void* G, float* P_hat, float* D_hat, psgd_stream stream);
 
 /*
  * psgd_step with HOST buffers: copies G_host into the caller's DEVICE staging
@@ -141,7 +146,7 @@ psgd_status psgd_refresh(psgd_handle* h, const float* G, float* P_hat, float* D_
  * P_hat_host / Q_host (either may be NULL) and synchronises the stream.
  * Pinned host memory makes the copies asynchronous with respect to the host.
  */
-psgd_status psgd_step_host(psgd_handle* h, const float* G_host /*HOST*/, float* G_stage /*DEVICE*/,
+psgd_status psgd_step_host(psgd_handle* h, const void* G_host /*HOST*/, void* G_stage /*DEVICE*/,
                            float* P_hat_host /*HOST*/, float* Q_host /*HOST*/, psgd_stream stream);
 
 /*

@@ -12,6 +12,7 @@ PSGD_W_TIMEOUT = 4
 PSGD_OPT_ERROR_FORM, PSGD_OPT_MODE, PSGD_OPT_REFRESH_ITERS, PSGD_OPT_REFRESH_OVERSAMPLE, PSGD_OPT_REFRESH_TC = 1, 2, 3, 4, 5
 PSGD_OPT_POWER_STEPS = 6
 PSGD_OPT_REFRESH_ADAPTIVE = 7
+PSGD_OPT_GRAD_BF16 = 8
 PSGD_BUF = {"P_node": 1, "Q_node": 2, "P_hat": 3, "Dbar": 4, "P_mean": 5}
 KERNEL_FAMILIES = ["project", "orth", "backproject", "residual", "refresh", "misc"]
 
@@ -90,7 +91,8 @@ class PowerSGDPlus:
     """
 
     def __init__(self, m, n, r, N, refresh_period=0, seed=0, count=1, device="cuda:0", error_form="local",
-                 mode="eager", refresh_iters=None, oversample=None, reset=True, refresh_tc=None, power_steps=None, refresh_adaptive=None):
+                 mode="eager", refresh_iters=None, oversample=None, reset=True, refresh_tc=None, power_steps=None, refresh_adaptive=None,
+                 grad_dtype="float32"):
         import torch
 
         self.torch = torch
@@ -114,6 +116,9 @@ class PowerSGDPlus:
             _check(L.psgd_set_option(h, PSGD_OPT_POWER_STEPS, int(power_steps)))
         if refresh_adaptive is not None:
             _check(L.psgd_set_option(h, PSGD_OPT_REFRESH_ADAPTIVE, int(bool(refresh_adaptive))))
+        self.grad_dtype = {"float32": torch.float32, "bfloat16": torch.bfloat16}[grad_dtype]
+        if self.grad_dtype is torch.bfloat16:
+            _check(L.psgd_set_option(h, PSGD_OPT_GRAD_BF16, 1))
         eb, qb, wb = _sz(), _sz(), _sz()
         _check(L.psgd_sizes(h, C.byref(eb), C.byref(qb), C.byref(wb)))
         with torch.cuda.device(self.device):
@@ -132,8 +137,8 @@ class PowerSGDPlus:
 
     def _g(self, G):
         t = self.torch
-        if not (isinstance(G, t.Tensor) and G.is_cuda and G.dtype == t.float32 and G.is_contiguous()):
-            raise PSGDError("G must be a contiguous float32 CUDA tensor")
+        if not (isinstance(G, t.Tensor) and G.is_cuda and G.dtype == self.grad_dtype and G.is_contiguous()):
+            raise PSGDError(f"G must be a contiguous {self.grad_dtype} CUDA tensor")
         if G.numel() != self.count * self.N * self.m * self.n:
             raise PSGDError("G has the wrong number of elements")
         return G

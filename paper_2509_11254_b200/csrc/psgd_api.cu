@@ -49,6 +49,7 @@ struct psgd_handle {
     int error_form = 0, mode = 0, refresh_iters = 20, oversample = -1, refresh_tc = 1, power_steps = 1, refresh_adaptive = 1;
     bool tc_ok = false;           // the refresh block is wide enough for the tensor-core sweeps
     size_t gpart_floats = 0;
+    bool grad_bf16 = false;       // G arrives as bfloat16
     bool ptc_ok = false;          // projections of more than 16 columns on the tensor cores
     int ptc_ncp = 0;
     bool rtc_ok = false;          // ranks above 16 with 16-byte row strides: residual update on the tensor cores
@@ -260,15 +261,16 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 // Rank-3 map over [count*N][m][n] float32 with tiles of `rows` rows x bw columns of one node; out-of-range reads give zeros.
-bool make_tile_map(CUtensorMap* map, const float* base, int64_t n, int64_t m, int64_t mats, int bw, int rows,
-                   CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_NONE) {
+bool make_tile_map(CUtensorMap* map, const void* base, int64_t n, int64_t m, int64_t mats, int bw, int rows,
+                   CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_NONE, bool bf16 = false) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
+    const cuuint64_t es = bf16 ? 2 : 4;
     cuuint64_t dims[3] = {(cuuint64_t)n, (cuuint64_t)m, (cuuint64_t)mats};
-    cuuint64_t strides[2] = {(cuuint64_t)n * 4, (cuuint64_t)m * (cuuint64_t)n * 4};
+    cuuint64_t strides[2] = {(cuuint64_t)n * es, (cuuint64_t)m * (cuuint64_t)n * es};
     cuuint32_t box[3] = {(cuuint32_t)bw, (cuuint32_t)rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -542,13 +544,19 @@ void tail(Launcher& L, psgd_handle* h, float* D_hat) {
 }
 
 // ---- SSP-Comp (Algorithm 1, first function) ------------------------------------
-void ssp(Launcher& L, psgd_handle* h, const float* G) {
+void ssp(Launcher& L, psgd_handle* h, const void* Gv) {
     char* ws = h->ws;
     float* Pnode = (float*)(ws + h->lay.Pnode);
     float* Pmean = (float*)(ws + h->lay.Pmean);
     float* Phat = (float*)(ws + h->lay.Phat);
     const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count;
-    if (r <= 32 || (h->ptc_ok && aligned16(G))) {
+    const float* G = (const float*)Gv;
+    if (h->grad_bf16) {      // M = G + E formed in the E buffer first (10 B/element), then the projection reads M
+        L.begin(PSGD_K_PROJECT);
+        k_add_mean<<<148 * 8, 256, 0, L.st>>>((const unsigned short*)Gv, h->E, nullptr, (size_t)m * n, N, cnt);
+        L.end();
+        launch_project(L, h->E, nullptr, nullptr, h->Q, Pnode, m, n, r, N, cnt, h->vec4);
+    } else if (r <= 32 || (h->ptc_ok && aligned16(G))) {
         launch_project(L, G, h->E, h->E, h->Q, Pnode, m, n, r, N, cnt, h->vec4);
     } else {
         L.begin(PSGD_K_PROJECT);
@@ -581,7 +589,7 @@ void ssp(Launcher& L, psgd_handle* h, const float* G) {
 
 // ---- SVD-Comp (Algorithm 1, second function): top-r left singular subspace of the
 //      node mean by randomised block subspace iteration + Rayleigh-Ritz. ----------
-void svd(Launcher& L, psgd_handle* h, const float* G) {
+void svd(Launcher& L, psgd_handle* h, const void* G) {
     char* ws = h->ws;
     float* Phat = (float*)(ws + h->lay.Phat);
     float* dbar = (float*)(ws + h->lay.dbar);
@@ -596,7 +604,8 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
     const int K = PSGD_K_REFRESH;
     L.force_kind = K;
     L.begin(K);
-    k_add_mean<<<148 * 8, 256, 0, L.st>>>(G, h->E, dbar, (size_t)m * n, N, cnt);
+    if (h->grad_bf16) k_add_mean<<<148 * 8, 256, 0, L.st>>>((const unsigned short*)G, h->E, dbar, (size_t)m * n, N, cnt);
+    else k_add_mean<<<148 * 8, 256, 0, L.st>>>((const float*)G, h->E, dbar, (size_t)m * n, N, cnt);
     L.end();
     size_t zt = (size_t)cnt * n * ell;
     L.begin(K);
@@ -706,8 +715,10 @@ void svd(Launcher& L, psgd_handle* h, const float* G) {
 
 // ---- single-pass SSP-Comp step (deferred residual) --------------------------------
 template <int RP, int WC>
-void launch_fused_t(Launcher& L, psgd_handle* h, const float* G, FusedArgs a) {
-    void (*kern)(CUtensorMap, CUtensorMap, FusedArgs) = h->pending ? k_fused_step<RP, WC, true> : k_fused_step<RP, WC, false>;
+void launch_fused_t(Launcher& L, psgd_handle* h, const void* G, FusedArgs a) {
+    void (*kern)(CUtensorMap, CUtensorMap, FusedArgs) =
+        h->grad_bf16 ? (h->pending ? k_fused_step<RP, WC, true, true> : k_fused_step<RP, WC, false, true>)
+                     : (h->pending ? k_fused_step<RP, WC, true, false> : k_fused_step<RP, WC, false, false>);
     cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->fused_smem);
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(FU_THREADS);
@@ -743,7 +754,7 @@ void launch_fused_t(Launcher& L, psgd_handle* h, const float* G, FusedArgs a) {
     cfg.gridDim = dim3((unsigned)((size_t)h->CS * h->KC * h->count));
     CUtensorMap tmG, tmM;
     const int bw = FusedGeom<WC>::BW, rs = FusedGeom<WC>::RS;
-    if (!make_tile_map(&tmG, G, h->n, h->m, (int64_t)h->count * h->N, bw, rs) ||
+    if (!make_tile_map(&tmG, G, h->n, h->m, (int64_t)h->count * h->N, bw, rs, CU_TENSOR_MAP_SWIZZLE_NONE, h->grad_bf16) ||
         !make_tile_map(&tmM, h->E, h->n, h->m, (int64_t)h->count * h->N, bw, rs)) {
         snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
         L.status = PSGD_E_CUDA;
@@ -754,13 +765,13 @@ void launch_fused_t(Launcher& L, psgd_handle* h, const float* G, FusedArgs a) {
     L.end();
 }
 template <int RP>
-void launch_fused_rp(Launcher& L, psgd_handle* h, const float* G, const FusedArgs& a) {
+void launch_fused_rp(Launcher& L, psgd_handle* h, const void* G, const FusedArgs& a) {
     if (h->WC == 128) launch_fused_t<RP, 128>(L, h, G, a);
     else if (h->WC == 256) launch_fused_t<RP, 256>(L, h, G, a);
     else launch_fused_t<RP, 512>(L, h, G, a);
 }
 
-void fused_ssp(Launcher& L, psgd_handle* h, const float* G) {
+void fused_ssp(Launcher& L, psgd_handle* h, const void* G) {
     char* ws = h->ws;
     const Layout& Y = h->lay;
     float* Phat = (float*)(ws + Y.Phat);
@@ -837,14 +848,15 @@ psgd_status check_ready(const psgd_handle* h) {
     return PSGD_OK;
 }
 
-psgd_status do_step(psgd_handle* h, const float* G, float* P_hat, float* D_hat, psgd_stream stream, bool force) {
+psgd_status do_step(psgd_handle* h, const void* G, float* P_hat, float* D_hat, psgd_stream stream, bool force) {
     psgd_status s = check_ready(h);
     if (s != PSGD_OK) return s;
     if (!G) return PSGD_E_NULL;
     cudaStream_t st = (cudaStream_t)stream;
     Launcher L{h, st};
     bool refresh = force || (h->tau > 0 && h->t % h->tau == 0);
-    if (h->mode == 1 && h->fused_ok && !refresh && aligned16(G) && h->power_steps == 1) {
+    // (a bfloat16 row has to be a multiple of 16 bytes for the tensor map: n % 8 == 0)
+    if (h->mode == 1 && h->fused_ok && !refresh && aligned16(G) && h->power_steps == 1 && (!h->grad_bf16 || h->n % 8 == 0)) {
         fused_ssp(L, h, G);
         if (D_hat) {
             float* Phat = (float*)(h->ws + h->lay.Phat);
@@ -899,6 +911,7 @@ psgd_status psgd_set_option(psgd_handle* h, int option, int value) {
         case PSGD_OPT_REFRESH_TC: if (value != 0 && value != 1) return PSGD_E_INVALID; h->refresh_tc = value; break;
         case PSGD_OPT_REFRESH_ADAPTIVE: if (value != 0 && value != 1) return PSGD_E_INVALID; h->refresh_adaptive = value; break;
         case PSGD_OPT_POWER_STEPS: if (value < 1 || value > 16) return PSGD_E_INVALID; h->power_steps = value; break;
+        case PSGD_OPT_GRAD_BF16: if (value != 0 && value != 1) return PSGD_E_INVALID; h->grad_bf16 = value != 0; break;
         default: return PSGD_E_INVALID;
     }
     plan(h);
@@ -939,15 +952,15 @@ psgd_status psgd_reset(psgd_handle* h, psgd_stream stream) {
     return L.status;
 }
 
-psgd_status psgd_step(psgd_handle* h, const float* G, float* P_hat, float* D_hat, psgd_stream stream) {
+psgd_status psgd_step(psgd_handle* h, const void* G, float* P_hat, float* D_hat, psgd_stream stream) {
     return do_step(h, G, P_hat, D_hat, stream, false);
 }
 
-psgd_status psgd_refresh(psgd_handle* h, const float* G, float* P_hat, float* D_hat, psgd_stream stream) {
+psgd_status psgd_refresh(psgd_handle* h, const void* G, float* P_hat, float* D_hat, psgd_stream stream) {
     return do_step(h, G, P_hat, D_hat, stream, true);
 }
 
-psgd_status psgd_step_host(psgd_handle* h, const float* G_host, float* G_stage, float* P_hat_host, float* Q_host,
+psgd_status psgd_step_host(psgd_handle* h, const void* G_host, void* G_stage, float* P_hat_host, float* Q_host,
                            psgd_stream stream) {
     psgd_status s = check_ready(h);
     if (s != PSGD_OK) return s;
@@ -955,7 +968,7 @@ psgd_status psgd_step_host(psgd_handle* h, const float* G_host, float* G_stage, 
     cudaStream_t st = (cudaStream_t)stream;
     size_t eb, qb;
     psgd_sizes(h, &eb, &qb, nullptr);
-    PSGD_CUDA(h, cudaMemcpyAsync(G_stage, G_host, eb, cudaMemcpyHostToDevice, st));
+    PSGD_CUDA(h, cudaMemcpyAsync(G_stage, G_host, h->grad_bf16 ? eb / 2 : eb, cudaMemcpyHostToDevice, st));
     s = do_step(h, G_stage, nullptr, nullptr, stream, false);
     if (s != PSGD_OK) return s;
     if (P_hat_host)

@@ -185,7 +185,7 @@ __device__ __forceinline__ void role_barrier(int id) {   // barrier among the 25
     asm volatile("bar.sync %0, 256;\n" ::"r"(id) : "memory");
 }
 
-template <int RP, int WC, bool PENDING>
+template <int RP, int WC, bool PENDING, bool GBF = false>   // GBF: the gradient tiles are bfloat16 (half the bytes of their slot)
 __global__ void __launch_bounds__(FU_THREADS, 1)
 k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmM, FusedArgs a) {
     using Ge = FusedGeom<WC>;
@@ -282,10 +282,10 @@ k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CU
                 const int row = (slot + p_bl * a.KC) * FU_R + p_rc * RS;
                 const unsigned bar = bar_full + 8 * p_ss;
                 const unsigned dst = smem_u32(ring + (size_t)p_ss * Ge::STAGE_FLOATS);
-                mbar_expect_tx(bar, STAGE_BYTES);
+                mbar_expect_tx(bar, GBF ? STAGE_BYTES / 2 + STAGE_BYTES / 4 : STAGE_BYTES);
 #pragma unroll
                 for (int x = 0; x < NBX; ++x) {
-                    tma_load_3d(dst + x * BOX_BYTES, &tmG, colbase + x * BW, row, c * N + p_i, bar);
+                    tma_load_3d(dst + x * (GBF ? BOX_BYTES / 2 : BOX_BYTES), &tmG, colbase + x * BW, row, c * N + p_i, bar);
                     tma_load_3d(dst + STAGE_BYTES / 2 + x * BOX_BYTES, &tmM, colbase + x * BW, row, c * N + p_i, bar);
                 }
             }
@@ -327,19 +327,28 @@ k_fused_step(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CU
 
                     // ---- S = g + stored Delta -> tile; sacc += S Q' ----
                     mbar_wait(bar_full + 8 * ss, (unsigned)par, a.flags, dead);
-                    const float* sgp = ring + (size_t)ss * Ge::STAGE_FLOATS + (size_t)abox * (RS * BW) + (size_t)(rgl * FU_RG + hrow * LR) * BW + aboxcol;
+                    const size_t tile_off = (size_t)abox * (RS * BW) + (size_t)(rgl * FU_RG + hrow * LR) * BW + aboxcol;
+                    const float* sgp = ring + (size_t)ss * Ge::STAGE_FLOATS + tile_off;
+                    const unsigned short* sgb = reinterpret_cast<const unsigned short*>(ring + (size_t)ss * Ge::STAGE_FLOATS) + tile_off;
                     const float* smp = sgp + RS * WC;
                     float* tp = tile + (((size_t)pbuf * N + i) * FU_R + rc * RS + rgl * FU_RG + hrow * LR) * WC + acol;
                     float sv[LR][LC];
 #pragma unroll
                     for (int rr = 0; rr < LR; ++rr) {
                         if (WIDE) {
-                            const float4 g4 = *reinterpret_cast<const float4*>(sgp + rr * BW);
+                            float4 g4;
+                            if (GBF) {      // bfloat16 -> float32: its 16 bits are the upper half
+                                const uint2 gb = *reinterpret_cast<const uint2*>(sgb + rr * BW);
+                                g4 = make_float4(__uint_as_float(gb.x << 16), __uint_as_float(gb.x & 0xFFFF0000u),
+                                                 __uint_as_float(gb.y << 16), __uint_as_float(gb.y & 0xFFFF0000u));
+                            } else {
+                                g4 = *reinterpret_cast<const float4*>(sgp + rr * BW);
+                            }
                             const float4 m4 = *reinterpret_cast<const float4*>(smp + rr * BW);
                             sv[rr][0] = g4.x + m4.x; sv[rr][LC > 1 ? 1 : 0] = g4.y + m4.y;
                             sv[rr][LC > 2 ? 2 : 0] = g4.z + m4.z; sv[rr][LC > 3 ? 3 : 0] = g4.w + m4.w;
                         } else {
-                            sv[rr][0] = sgp[rr * BW] + smp[rr * BW];
+                            sv[rr][0] = (GBF ? __uint_as_float((unsigned)sgb[rr * BW] << 16) : sgp[rr * BW]) + smp[rr * BW];
                         }
                     }
                     __syncwarp();

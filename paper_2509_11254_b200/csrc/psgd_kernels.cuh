@@ -503,7 +503,12 @@ __global__ void __launch_bounds__(RS_THREADS) k_residual(ResidArgs a) {
 // elementwise helpers
 // ----------------------------------------------------------------------------
 // M = G + E (Eq. (7a)) written over E; optionally Dbar = (1/N) sum_i M_i (SVD-Comp, first line).
-__global__ void k_add_mean(const float* G, float* E, float* Dbar, size_t per_mat, int nodes, int count) {
+// float32 value of a gradient element: float32 as stored, bfloat16 widened exactly (its 16 bits are the top half)
+__device__ __forceinline__ float grad_value(const float* G, size_t i) { return __ldcs(G + i); }
+__device__ __forceinline__ float grad_value(const unsigned short* G, size_t i) { return __uint_as_float((unsigned)__ldcs(G + i) << 16); }
+
+template <typename TG>
+__global__ void k_add_mean(const TG* G, float* E, float* Dbar, size_t per_mat, int nodes, int count) {
     size_t total = per_mat * count;
     for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (size_t)gridDim.x * blockDim.x) {
@@ -511,7 +516,7 @@ __global__ void k_add_mean(const float* G, float* E, float* Dbar, size_t per_mat
         float s = 0.f;
         for (int i = 0; i < nodes; ++i) {
             size_t off = (c * nodes + i) * per_mat + e;
-            float mval = __ldcs(G + off) + E[off];
+            float mval = grad_value(G, off) + E[off];
             E[off] = mval;
             s += mval;
         }

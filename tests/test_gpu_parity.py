@@ -79,12 +79,12 @@ def compare_step(out, gpu, m, n, r, N, tag):
 
 
 def run_case(torch, m, n, r, N, tau, steps, workload=1, count=1, error_form="local", Einit=0.0, seed=7,
-             check_dense=False, mode="eager", power_steps=1):
+             check_dense=False, mode="eager", power_steps=1, grad_dtype="float32"):
     from paper_2509_11254_b200 import PowerSGDPlus
 
     dev = "cuda:0"
     comp = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=seed, count=count, device=dev, error_form=error_form,
-                        mode=mode, power_steps=power_steps)
+                        mode=mode, power_steps=power_steps, grad_dtype=grad_dtype)
     rng = np.random.default_rng(seed)
     Q0 = np.stack([synth.init_Q(n, r, matrix_id=c, seed=seed) for c in range(count)])
     oracles = [orc.PowerSGDPlusOracle(m, n, r, N, tau, Q0[c], error_form, power_steps) for c in range(count)]
@@ -99,6 +99,9 @@ def run_case(torch, m, n, r, N, tau, steps, workload=1, count=1, error_form="loc
             o.Q = o.Q.astype(np.float32).astype(np.float64)
         comp.set_state(E=np.stack([o.E for o in oracles]), Q=np.stack([o.Q for o in oracles]), t=t)
         Gd = torch.as_tensor(G, device=dev)
+        if grad_dtype == "bfloat16":     # the oracle gets the same bfloat16 values, widened
+            Gd = Gd.to(torch.bfloat16)
+            G = Gd.float().cpu().numpy()
         Dh = torch.empty((count, m, n), dtype=torch.float32, device=dev) if check_dense else None
         comp.step(Gd, D_hat=Dh)
         comp.materialize_error()
@@ -168,6 +171,19 @@ def test_tensor_core_step_kernels_all_widths(torch_cuda, m, n, r, N, count):
     """Every layout class of the r > 16 projection / back-projection / residual kernels (number of accumulator
     sets, one-operand or three-MMA form, column groups per adder thread), P_i, P~, Q_i, Q and E against the oracle."""
     run_case(torch_cuda, m, n, r, N, tau=0, steps=2, workload=4, count=count, Einit=0.01, check_dense=True)
+
+
+@pytest.mark.parametrize("m,n,r,N,count,mode,tau,Einit", [
+    (520, 256, 8, 4, 2, "deferred", 3, 0.0),     # single-pass kernel on bfloat16 tiles (128-column slices), refresh at t = 0, 3
+    (1100, 768, 4, 8, 1, "deferred", 0, 0.01),   # 256-column slices: 4 bfloat16 values per lane and row
+    (2054, 1004, 8, 2, 1, "deferred", 0, 0.01),  # n % 8 != 0: no bfloat16 tensor map, the three-pass kernels take over
+    (640, 256, 16, 2, 1, "eager", 0, 0.01),      # float32 kernels on M = G + E
+    (772, 300, 40, 3, 1, "eager", 0, 0.01),      # tensor-core kernels on M = G + E
+])
+def test_bfloat16_gradients(torch_cuda, m, n, r, N, count, mode, tau, Einit):
+    """PSGD_OPT_GRAD_BF16: G arrives as bfloat16 and is widened exactly as it is read; same tolerances as float32.
+    (The refresh case starts from E = 0: random E of the size the other cases use would bury the gap at r in noise.)"""
+    run_case(torch_cuda, m, n, r, N, tau=tau, steps=4, workload=2, count=count, Einit=Einit, mode=mode, grad_dtype="bfloat16")
 
 
 @pytest.mark.parametrize("K,mode", [(2, "eager"), (3, "deferred")])
