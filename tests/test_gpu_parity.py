@@ -451,6 +451,33 @@ def test_full_size_config4_ffn_class(torch_cuda):
     assert plan["single_pass"] == 0
 
 
+@pytest.mark.parametrize("grad_dtype", ["float32", "bfloat16"])
+def test_step_host_equals_step(torch_cuda, grad_dtype):
+    """psgd_step_host (pinned host G -> device staging buffer -> step -> P~, Q back to the host) gives bit for bit
+    what psgd_step gives on the same values already on the device."""
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    torch = torch_cuda
+    m, n, r, N, count = 520, 256, 8, 4, 2
+    dt = torch.float32 if grad_dtype == "float32" else torch.bfloat16
+    G = [synth.make_gradients_torch(2, m, n, N, count, step=t, device="cuda:0").to(dt) for t in range(3)]
+    a = PowerSGDPlus(m, n, r, N, refresh_period=2, seed=5, count=count, mode="deferred", grad_dtype=grad_dtype)
+    b = PowerSGDPlus(m, n, r, N, refresh_period=2, seed=5, count=count, mode="deferred", grad_dtype=grad_dtype)
+    stage = torch.empty_like(G[0])
+    Ph = torch.empty(a.P_hat.shape, dtype=torch.float32).pin_memory()
+    Qh = torch.empty(a.Q.shape, dtype=torch.float32).pin_memory()
+    for g in G:
+        a.step(g)
+        gh = torch.empty(g.shape, dtype=dt).pin_memory()
+        gh.copy_(g)
+        b.step_host(gh, stage, Ph, Qh)
+        torch.cuda.synchronize()
+        assert torch.equal(Ph, a.P_hat.cpu()) and torch.equal(Qh, a.Q.cpu())
+    assert torch.equal(a.E, b.E)
+    a.close()
+    b.close()
+
+
 def test_streamed_stack_equals_sequential_steps(torch_cuda):
     """Two shape classes stepped on one stream each (the benchmark's launch configuration) give bit for bit
     what stepping them one after the other gives: the handles share nothing."""
