@@ -141,6 +141,13 @@ psgd_status psgd_step(psgd_handle* h, const void* G, float* P_hat, float* D_hat,
 psgd_status psgd_refresh(psgd_handle* h, const void* G, float* P_hat, float* D_hat, psgd_stream stream);
 
 /*
+ * The optimizer step after the iteration, for momentum SGD (Eq. (7c)):  m_t = mu m_{t-1} + D^_t,
+ * X_{t+1} = X_t - eta m_t,  with D^_t = P~_t Q_t^T of the last psgd_step / psgd_refresh, formed on the fly and
+ * never stored.  X, mom: DEVICE, [count][m][n] float32, updated in place.  PSGD_E_STATE before the first step.
+ */
+psgd_status psgd_msgd_update(psgd_handle* h, float* X, float* mom, float eta, float mu, psgd_stream stream);
+
+/*
  * psgd_step with HOST buffers: copies G_host into the caller's DEVICE staging
  * buffer G_stage (same size as G), runs the step, copies P~ and Q_t back to
  * P_hat_host / Q_host (either may be NULL) and synchronises the stream.

@@ -261,6 +261,12 @@ def counter_stoch_grad(X, xi, sigma):
     return np.stack([g + x * (sigma * B_MAT - g) for x in xi])
 
 
+def msgd_update(X, mom, Dhat, eta, mu):
+    """Eq. (7c): m_t = mu m_{t-1} + Dhat_t;  X_{t+1} = X_t - eta m_t.  Returns (X_{t+1}, m_t)."""
+    mom = mu * np.asarray(mom, dtype=F64) + np.asarray(Dhat, dtype=F64)
+    return np.asarray(X, dtype=F64) - eta * mom, mom
+
+
 def run_counterexample(X0, Q_init, xi, sigma, tau, eta, mu, error_form="local"):
     """Algorithm 2 with the MSGD update of Eq. (7c) on the counterexample.
 
@@ -276,8 +282,8 @@ def run_counterexample(X0, Q_init, xi, sigma, tau, eta, mu, error_form="local"):
     for t in range(T):
         G = counter_stoch_grad(X, xi[t], sigma)
         out = orc.step(G)
-        mom = mu * mom + out["Dhat"]
+        Xn, mom = msgd_update(X, mom, out["Dhat"], eta, mu)
         rec = dict(X=X.copy(), grad=counter_grad(X), mom=mom.copy(), **out)
-        X = X - eta * mom
+        X = Xn
         hist.append(rec)
     return hist, X

@@ -31,6 +31,7 @@ SIGNATURES = {
     "psgd_step": (_int, [_vp, _vp, _vp, _vp, _vp]),
     "psgd_refresh": (_int, [_vp, _vp, _vp, _vp, _vp]),
     "psgd_step_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "psgd_msgd_update": (_int, [_vp, _vp, _vp, C.c_float, C.c_float, _vp]),
     "psgd_materialize_error": (_int, [_vp, _vp]),
     "psgd_state_written": (_int, [_vp]),
     "psgd_get_step": (_int, [_vp, C.POINTER(_i64)]),
@@ -164,6 +165,16 @@ class PowerSGDPlus:
                                         P_hat_host.data_ptr() if P_hat_host is not None else None,
                                         Q_host.data_ptr() if Q_host is not None else None,
                                         self._stream(stream)), self.h)
+
+    def msgd_update(self, X, mom, eta, mu, stream=None):
+        """Eq. (7c) with the reconstruction of the last step: mom <- mu mom + P~ Q^T, X <- X - eta mom (in place)."""
+        t = self.torch
+        for a in (X, mom):
+            if not (isinstance(a, t.Tensor) and a.is_cuda and a.dtype == t.float32 and a.is_contiguous()
+                    and a.numel() == self.count * self.m * self.n):
+                raise PSGDError("X and mom must be contiguous float32 CUDA tensors of count*m*n elements")
+        with t.cuda.device(self.device):
+            _check(lib().psgd_msgd_update(self.h, X.data_ptr(), mom.data_ptr(), float(eta), float(mu), self._stream(stream)), self.h)
 
     def materialize_error(self, stream=None):
         with self.torch.cuda.device(self.device):

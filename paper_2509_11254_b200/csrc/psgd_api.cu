@@ -488,6 +488,21 @@ void launch_resid(Launcher& L, const float* M, float* Out, const float* Phat, co
     L.end();
 }
 
+// Momentum-SGD hand-off (Eq. (7c)): mom <- mu mom + P~ Q^T, X <- X - eta mom, the reconstruction never stored.
+void launch_msgd(Launcher& L, float* X, float* Mom, float eta, float mu, const float* Phat, const float* Qf, int rows, int n,
+                 int r, int mats) {
+    int rpc = 128;
+    while (rpc > RS_SUB && (int64_t)mats * ceil_div(n, RS_COLS) * ceil_div(rows, rpc) < 4 * 148) rpc /= 2;
+    ResidArgs a{nullptr, nullptr, Phat, Qf, rows, n, r, 1, rpc, 0, 0};
+    a.X = X; a.Mom = Mom; a.eta = eta; a.mu = mu;
+    dim3 grid(ceil_div(n, RS_COLS), ceil_div(rows, rpc), mats);
+    L.begin(PSGD_K_RESIDUAL);
+    if (r <= 4) k_residual<4, 1><<<grid, RS_THREADS, 0, L.st>>>(a);
+    else if (r <= 8) k_residual<8, 1><<<grid, RS_THREADS, 0, L.st>>>(a);
+    else k_residual<16, 1><<<grid, RS_THREADS, 0, L.st>>>(a);
+    L.end();
+}
+
 // ---- K2: X <- orthonormal factor of X (rows x c), in place or into Xout ------
 void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int rows, int c, int kind, float* XoutT = nullptr,
                  bool complete = false, const int* skip = nullptr) {
@@ -958,6 +973,16 @@ psgd_status psgd_step(psgd_handle* h, const void* G, float* P_hat, float* D_hat,
 
 psgd_status psgd_refresh(psgd_handle* h, const void* G, float* P_hat, float* D_hat, psgd_stream stream) {
     return do_step(h, G, P_hat, D_hat, stream, true);
+}
+
+psgd_status psgd_msgd_update(psgd_handle* h, float* X, float* mom, float eta, float mu, psgd_stream stream) {
+    psgd_status s = check_ready(h);
+    if (s != PSGD_OK) return s;
+    if (!X || !mom) return PSGD_E_NULL;
+    if (h->t == 0) return PSGD_E_STATE;      // no P~_t, Q_t yet
+    Launcher L{h, (cudaStream_t)stream};
+    launch_msgd(L, X, mom, eta, mu, (const float*)(h->ws + h->lay.Phat), h->Q, (int)h->m, (int)h->n, h->r, h->count);
+    return L.status;
 }
 
 psgd_status psgd_step_host(psgd_handle* h, const void* G_host, void* G_stage, float* P_hat_host, float* Q_host,

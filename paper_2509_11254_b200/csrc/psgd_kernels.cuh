@@ -402,6 +402,11 @@ struct ResidArgs {
     int rows, n, r, nodes, rows_per_chunk;
     int q_per_node;     // 1: Qf indexed by (matrix,node); 0: by matrix only
     int out_per_node;   // 1: Out/M indexed by (matrix,node); 0: by matrix only (dense reconstruction)
+    // momentum-SGD hand-off (Eq. (7c)), only with M == nullptr: instead of storing the reconstruction D^,
+    // mom <- mu mom + D^ and X <- X - eta mom, both [mats][rows][n]
+    float* X = nullptr;
+    float* Mom = nullptr;
+    float eta = 0.f, mu = 0.f;
 };
 
 template <int RP, int VEC>
@@ -414,7 +419,8 @@ __global__ void __launch_bounds__(RS_THREADS) k_residual(ResidArgs a) {
     const int c = a.out_per_node ? mat / a.nodes : mat;
     const int rbeg = blockIdx.y * a.rows_per_chunk, rend = min(a.rows, rbeg + a.rows_per_chunk);
     const float* Mb = a.M ? a.M + (size_t)mat * a.rows * n : nullptr;
-    float* Ob = a.Out + (size_t)mat * a.rows * n;
+    float* Ob = a.X ? a.X + (size_t)mat * a.rows * n : a.Out + (size_t)mat * a.rows * n;
+    float* Vb = a.X ? a.Mom + (size_t)mat * a.rows * n : nullptr;
     const float* Pb = a.Phat + (size_t)c * a.rows * r;
     const float* Qb = a.Qf + (size_t)(a.q_per_node ? mat : c) * n * r;
     const int nch = (r + RP - 1) / RP;
@@ -487,6 +493,19 @@ __global__ void __launch_bounds__(RS_THREADS) k_residual(ResidArgs a) {
                 o = make_float4(rec[u][0], rec[u][1], rec[u][2], rec[u][3]);
             }
             float* p = Ob + (size_t)grow * n + col;
+            if (Vb) {               // o is the reconstruction D^ here
+                float* pv = Vb + (size_t)grow * n + col;
+                const float d[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (col + j < n) {
+                        const float mnew = fmaf(a.mu, pv[j], d[j]);
+                        pv[j] = mnew;
+                        p[j] = fmaf(-a.eta, mnew, p[j]);
+                    }
+                }
+                continue;
+            }
             if (VEC == 4) {
                 if (col < n) *reinterpret_cast<float4*>(p) = o;
             } else {

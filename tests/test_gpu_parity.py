@@ -451,6 +451,38 @@ def test_full_size_config4_ffn_class(torch_cuda):
     assert plan["single_pass"] == 0
 
 
+@pytest.mark.parametrize("m,n,r,mode", [(520, 256, 8, "deferred"), (300, 260, 40, "eager"), (257, 130, 3, "eager")])
+def test_msgd_update_after_the_step(torch_cuda, m, n, r, mode):
+    """Eq. (7c) through psgd_msgd_update: mom <- mu mom + P~ Q^T, X <- X - eta mom, against the oracle's update
+    fed with the oracle's own reconstruction, over three steps (one of them a refresh)."""
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    torch = torch_cuda
+    N, count, tau, eta, mu = 3, 2, 2, 0.05, 0.9
+    comp = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=11, count=count, mode=mode)
+    Q0 = comp.Q.cpu().numpy()
+    oracles = [orc.PowerSGDPlusOracle(m, n, r, N, tau, Q0[c]) for c in range(count)]
+    rng = np.random.default_rng(11)
+    X0 = rng.standard_normal((count, m, n)).astype(np.float32)
+    X = torch.as_tensor(X0, device="cuda:0").clone()
+    mom = torch.zeros_like(X)
+    Xo = [X0[c].astype(np.float64) for c in range(count)]
+    mo = [np.zeros((m, n)) for _ in range(count)]
+    for t in range(3):
+        G = np.stack([synth.make_gradients(2, m, n, N, step=t, matrix_id=c, seed=11) for c in range(count)])
+        comp.step(torch.as_tensor(G, device="cuda:0"))
+        comp.msgd_update(X, mom, eta, mu)
+        for c in range(count):
+            out = oracles[c].step(G[c])
+            Xo[c], mo[c] = orc.msgd_update(Xo[c], mo[c], out["Dhat"], eta, mu)
+    assert comp.last_status() == 0
+    for c in range(count):
+        assert rel_fro(mom[c].cpu().numpy(), mo[c]) <= 1e-4          # free-running over three steps
+        step_norm = np.linalg.norm(Xo[c] - X0[c])
+        assert np.linalg.norm(X[c].cpu().numpy() - Xo[c]) <= 1e-4 * step_norm + 1e-6 * np.linalg.norm(X0[c])
+    comp.close()
+
+
 @pytest.mark.parametrize("grad_dtype", ["float32", "bfloat16"])
 def test_step_host_equals_step(torch_cuda, grad_dtype):
     """psgd_step_host (pinned host G -> device staging buffer -> step -> P~, Q back to the host) gives bit for bit

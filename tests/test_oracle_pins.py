@@ -419,3 +419,17 @@ def test_planted_mistake_is_caught(name):
         except Exception:
             tripped.append(chk.__name__)
     assert tripped, f"no pin caught the planted mistake {name}"
+
+
+def test_msgd_update_closed_form():
+    """Eq. (7c) with a constant reconstruction D and m_{-1} = 0: m_t = D (1 - mu^(t+1)) / (1 - mu) and
+    X_T = X_0 - eta D sum_{t<T} (1 - mu^(t+1)) / (1 - mu); with mu = 0 plain SGD, X_T = X_0 - T eta D."""
+    rng = np.random.default_rng(3)
+    X0, D = rng.standard_normal((5, 4)), rng.standard_normal((5, 4))
+    for mu, eta, T in [(0.9, 0.05, 7), (0.0, 0.1, 4), (0.5, 1.0, 3)]:
+        X, mom = X0.copy(), np.zeros_like(X0)
+        for _ in range(T):
+            X, mom = orc.msgd_update(X, mom, D, eta, mu)
+        geo = [(1 - mu ** (t + 1)) / (1 - mu) for t in range(T)]
+        np.testing.assert_allclose(mom, D * geo[-1], rtol=1e-13, atol=1e-15)
+        np.testing.assert_allclose(X, X0 - eta * D * sum(geo), rtol=1e-13, atol=1e-13)
