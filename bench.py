@@ -125,7 +125,7 @@ def stack_for(workload):
 
 
 def algorithmic_bytes(shapes, r, N, g_bytes_per_element=4):
-    """North-star accounting: read G, read E, write E per element (12 B with float32 G) plus the P/Q traffic."""
+    """Minimum traffic of a step: read G, read E, write E per element (12 B with float32 G) plus the P/Q traffic."""
     el = sum(m * n * c for m, n, c in shapes) * N
     pq = sum(4 * (2 * N * m * r + 2 * m * r + 2 * N * n * r + 2 * n * r) * c for m, n, c in shapes)
     return (8 + g_bytes_per_element) * el + pq, g_bytes_per_element * el
@@ -243,7 +243,7 @@ def timed_steps(torch, stack, bufs, steps, dist_barrier):
 
 
 def sweep_config5(torch, device, peak, mode):
-    """BASELINE config 5: m=16384, n=4096, N=4, per-rank step and refresh latency."""
+    """Workload 5: m=16384, n=4096, N=4, per-rank step and refresh latency."""
     from paper_2509_11254_b200 import PowerSGDPlus, synth
 
     m, n, N = 16384, 4096, 4
@@ -274,7 +274,7 @@ def sweep_config5(torch, device, peak, mode):
         alg, gb = algorithmic_bytes([(m, n, 1)], r, N)
         plan = h.plan_info()
         out.append({"r": r, "kernel": "single-pass" if (mode == "deferred" and plan["single_pass"]) else "eager", "step_ms": round(ms, 4), "grad_GBps": round(gb / ms / 1e6, 1),
-                    "north_star_frac": round(alg / ms / 1e6 / peak, 4), "refresh_ms": round(rms, 3),
+                    "min_bytes_frac": round(alg / ms / 1e6 / peak, 4), "refresh_ms": round(rms, 3),
                     "flags": flags})
         h.close()
         del h
@@ -379,8 +379,8 @@ def run_ours(args):
                        "l2": "inputs (%.2f GB of G per step, 2 alternating sets) exceed L2" % (g_bytes / 1e9),
                        "streams": len(handles), "grad_dtype": args.grad_dtype,
                        "parallelism": "replicas" if world > 1 else "single"},
-            "north_star_frac": alg_bytes / ms_step / 1e6 / peak,
-            "north_star_bytes_per_step": alg_bytes,
+            "min_bytes_frac": alg_bytes / ms_step / 1e6 / peak,
+            "min_bytes_per_step": alg_bytes,
             "gpu_launches": l1 - l0, "clocks": clocks, "roofline": roofline}
 
     if rank == 0 and not args.no_e2e:

@@ -122,7 +122,7 @@ def run_case(torch, m, n, r, N, tau, steps, workload=1, count=1, error_form="loc
     comp.close()
 
 
-# ---- BASELINE config 1: tiny, 20 steps, refresh every 5 ------------------------
+# ---- workload 1: tiny, 20 steps, refresh every 5 ------------------------
 def test_config1_tiny_20_steps(torch_cuda):
     run_case(torch_cuda, 256, 128, 4, 4, tau=5, steps=20, workload=1)
 
@@ -411,27 +411,27 @@ def _full_size_case(torch, workload, m, n, r, N, count, tau, sample, free_steps,
 
 
 def test_full_size_config2_attention_class(torch_cuda):
-    """BASELINE config 2, the 48 matrices of 768 x 768 (r = 8, N = 8, refresh at t = 0), three sampled."""
+    """Workload 2, the 48 matrices of 768 x 768 (r = 8, N = 8, refresh at t = 0), three sampled."""
     plan = _full_size_case(torch_cuda, 2, 768, 768, 8, 8, 48, tau=50, sample=(0, 17, 47), free_steps=4)
     assert plan["single_pass"] == 1 and plan["CS"] == 3 and plan["WC"] == 256
 
 
 def test_full_size_config2_ffn_class(torch_cuda):
-    """BASELINE config 2, the 36 matrices of 2048 x 768, two sampled."""
+    """Workload 2, the 36 matrices of 2048 x 768, two sampled."""
     plan = _full_size_case(torch_cuda, 2, 2048, 768, 8, 8, 36, tau=50, sample=(5, 35), free_steps=3)
     assert plan["single_pass"] == 1
 
 
 @pytest.mark.parametrize("r", [4, 8])
 def test_full_size_config5(torch_cuda, r):
-    """BASELINE config 5: one 16384 x 4096 matrix on 4 nodes, plain PowerSGD steps (the step the sweep times)."""
+    """Workload 5: one 16384 x 4096 matrix on 4 nodes, plain PowerSGD steps (the step the sweep times)."""
     plan = _full_size_case(torch_cuda, 5, 16384, 4096, r, 4, 1, tau=0, sample=(0,), free_steps=3)
     assert plan["single_pass"] == 1 and plan["CS"] == 8 and plan["WC"] == 512
 
 
 @pytest.mark.parametrize("r", [64, 128])
 def test_full_size_config5_high_rank(torch_cuda, r):
-    """BASELINE config 5 at the ranks whose three passes run on the tensor cores (projection,
+    """Workload 5 at the ranks whose three passes run on the tensor cores (projection,
     back-projection and residual as exactly split TF32 products).  The 0.9^k spectrum is at the noise
     floor from k = 60 on, so there is no gap at r: a refresh at t = 0 aligns the state, the comparison is the
     SSP step from identical state."""
@@ -440,13 +440,13 @@ def test_full_size_config5_high_rank(torch_cuda, r):
 
 
 def test_full_size_config4_attention_class(torch_cuda):
-    """BASELINE config 4, the 96 matrices of 2048 x 2048 (r = 32, N = 8, refresh at t = 0), two sampled."""
+    """Workload 4, the 96 matrices of 2048 x 2048 (r = 32, N = 8, refresh at t = 0), two sampled."""
     plan = _full_size_case(torch_cuda, 4, 2048, 2048, 32, 8, 96, tau=100, sample=(0, 95), free_steps=2)
     assert plan["single_pass"] == 0
 
 
 def test_full_size_config4_ffn_class(torch_cuda):
-    """BASELINE config 4, the 72 matrices of 5504 x 2048, one sampled."""
+    """Workload 4, the 72 matrices of 5504 x 2048, one sampled."""
     plan = _full_size_case(torch_cuda, 4, 5504, 2048, 32, 8, 72, tau=100, sample=(71,), free_steps=2)
     assert plan["single_pass"] == 0
 
