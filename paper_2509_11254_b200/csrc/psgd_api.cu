@@ -753,13 +753,15 @@ void launch_fused_t(Launcher& L, psgd_handle* h, const void* G, FusedArgs a) {
         h->active_clusters = nc;
         // row slots: trade the idle tail of the last wave of clusters against the traffic of the
         // per-slot partial W (written and read once: 2 KC RP / (3 m) of the step's 12 bytes per element)
+        // and the start-up of every slot (loading Q', filling the ring, the first exchange: measured
+        // about 1.35 row blocks' worth of time per slot)
         int best = h->KCmax;
         if (nc > 0) {
             double best_cost = 1e30;
             for (int KC = 1; KC <= h->KCmax; ++KC) {
                 int64_t tot = (int64_t)h->count * KC;
                 double eff = (double)tot / (double)(((tot + nc - 1) / nc) * nc);
-                double cost = 1.0 / eff + 2.0 * KC * RP / (3.0 * (double)h->m);
+                double cost = 1.0 / eff + 2.0 * KC * RP / (3.0 * (double)h->m) + 1.35 * KC / (double)h->nblk;
                 if (cost < best_cost - 1e-9) { best_cost = cost; best = KC; }
             }
         }
