@@ -40,7 +40,7 @@ DEFAULTS = {2: (8, 8, 50), 3: (16, 16, 20), 4: (32, 8, 100), 5: (16, 4, 0), 1: (
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=2)
