@@ -73,6 +73,7 @@ struct psgd_handle {
     size_t fused_smem = 0;
     int active_clusters = -1;     // clusters of the single-pass kernel resident at once (known after its first launch)
     bool pending = false;         // E holds Delta_t; the residual is Delta_t - P~_t Qsub^T
+    bool pending_fused = false;   // ... and the padded factors the single-pass kernel subtracts are those of that step
     bool tacc_identity = true;    // no preconditioner yet
     bool qpad_valid = false;      // padded copy of Q is current
 };
@@ -324,6 +325,25 @@ void launch_project_rp(Launcher& L, const ProjectArgs& a, int count, bool vec, b
         else launch_project_t<RP, 1, false, false>(L, a, count);
     }
 }
+// P = (G + (Delta_prev - P~_prev Qsub^T)) Q, M = G + e stored over Delta_prev: the projection of the two-pass deferred
+// mode (r <= 16, one chunk of columns).
+void launch_project_pending(Launcher& L, const float* G, float* E, const float* Q, float* P, const float* Pprev, const float* Qsub,
+                            int qsub_per_node, int rows, int n, int r, int nodes, int count, bool vec) {
+    ProjectArgs a{G, E, E, Q, P, rows, n, r, nodes, 1, nullptr};
+    a.Pprev = Pprev; a.Qsub = Qsub; a.qsub_per_node = qsub_per_node;
+    vec = vec && aligned16(G) && aligned16(E);
+    dim3 grid(ceil_div(rows, PJ_TR), nodes, count);
+    auto go = [&](auto kern, size_t smem) {
+        allow_smem(kern, smem);
+        L.begin(PSGD_K_PROJECT);
+        kern<<<grid, PJ_THREADS, smem, L.st>>>(a);
+        L.end();
+    };
+    if (r <= 4) { if (vec) go(k_project<4, 4, true, true, true>, project_smem_bytes<4, true, true>()); else go(k_project<4, 1, true, true, true>, project_smem_bytes<4, true, true>()); }
+    else if (r <= 8) { if (vec) go(k_project<8, 4, true, true, true>, project_smem_bytes<8, true, true>()); else go(k_project<8, 1, true, true, true>, project_smem_bytes<8, true, true>()); }
+    else { if (vec) go(k_project<16, 4, true, true, true>, project_smem_bytes<16, true, true>()); else go(k_project<16, 1, true, true, true>, project_smem_bytes<16, true, true>()); }
+}
+
 // Tensor-core form for more than 16 columns (exactly split TF32 products, see psgd_gemm_tc.cuh).
 bool launch_project_tc(Launcher& L, const float* A, const float* B, float* Mout, const float* Q, float* P, int rows, int n,
                        int r, int nodes, int count, const int* skip) {
@@ -540,7 +560,8 @@ void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int r
 }
 
 // ---- Algorithm 1, common tail: Q_i, Q, residual, optional dense reconstruction --
-void tail(Launcher& L, psgd_handle* h, float* D_hat) {
+// defer: leave Delta_t in the E buffer (two-pass deferred mode); the next projection or psgd_materialize_error forms e_{t+1}
+void tail(Launcher& L, psgd_handle* h, float* D_hat, bool defer = false) {
     char* ws = h->ws;
     float* Phat = (float*)(ws + h->lay.Phat);
     float* Qnode = (float*)(ws + h->lay.Qnode);
@@ -551,7 +572,11 @@ void tail(Launcher& L, psgd_handle* h, float* D_hat) {
     L.begin(PSGD_K_BACKPROJECT);
     k_reduce_q<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(part, Qnode, h->Q, n, r, N, Sb, cnt);
     L.end();
-    if (h->error_form == 0)
+    if (defer) {
+        h->pending = true;
+        h->pending_fused = false;
+    }
+    else if (h->error_form == 0)
         launch_resid(L, h->E, h->E, Phat, Qnode, m, n, r, N, cnt * N, 1, 1, h->vec4);
     else
         launch_resid(L, h->E, h->E, Phat, h->Q, m, n, r, N, cnt * N, 0, 1, h->vec4);
@@ -566,7 +591,11 @@ void ssp(Launcher& L, psgd_handle* h, const void* Gv) {
     float* Phat = (float*)(ws + h->lay.Phat);
     const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count;
     const float* G = (const float*)Gv;
-    if (h->grad_bf16) {      // M = G + E formed in the E buffer first (10 B/element), then the projection reads M
+    if (h->pending) {        // two-pass deferred mode: E holds Delta_{t-1}; P~_{t-1} and Q_i of the last step are still in place
+        float* Qnode = (float*)(ws + h->lay.Qnode);
+        launch_project_pending(L, G, h->E, h->Q, Pnode, Phat, h->error_form == 0 ? Qnode : h->Q, h->error_form == 0 ? 1 : 0,
+                               m, n, r, N, cnt, h->vec4);
+    } else if (h->grad_bf16) {      // M = G + E formed in the E buffer first (10 B/element), then the projection reads M
         L.begin(PSGD_K_PROJECT);
         k_add_mean<<<148 * 8, 256, 0, L.st>>>((const unsigned short*)Gv, h->E, nullptr, (size_t)m * n, N, cnt);
         L.end();
@@ -844,6 +873,7 @@ void fused_ssp(Launcher& L, psgd_handle* h, const void* G) {
     k_sum_c<<<cnt, RP * RP, 0, L.st>>>(Cpart, Cmat, qblocks, RP);
     L.end();
     h->pending = true;
+    h->pending_fused = true;
     h->tacc_identity = false;
 }
 
@@ -874,15 +904,20 @@ psgd_status do_step(psgd_handle* h, const void* G, float* P_hat, float* D_hat, p
     bool refresh = force || (h->tau > 0 && h->t % h->tau == 0);
     // (a bfloat16 row has to be a multiple of 16 bytes for the tensor map: n % 8 == 0)
     if (h->mode == 1 && h->fused_ok && !refresh && aligned16(G) && h->power_steps == 1 && (!h->grad_bf16 || h->n % 8 == 0)) {
+        if (h->pending && !h->pending_fused) materialize(L, h);   // Delta_t left by a two-pass step: no padded factors for it
         fused_ssp(L, h, G);
         if (D_hat) {
             float* Phat = (float*)(h->ws + h->lay.Phat);
             launch_resid(L, nullptr, D_hat, Phat, h->Q, (int)h->m, (int)h->n, h->r, h->N, h->count, 0, 0, h->vec4);
         }
     } else {
-        materialize(L, h);   // refresh steps and shapes outside the single-pass plan run eagerly
+        // Refresh steps and shapes outside the single-pass plan run the three-pass kernels.  In deferred mode, up to
+        // 16 columns, SSP steps take two passes: the residual pass is dropped, the E buffer keeps Delta_t and the next
+        // projection forms e_{t+1} = Delta_t - P~_t Q_i^T on the fly (16 instead of 24 bytes per element).
+        const bool two_pass = h->mode == 1 && !refresh && h->r <= 16 && h->power_steps == 1 && !h->grad_bf16;
+        if (!two_pass) materialize(L, h);
         if (refresh) svd(L, h, G); else ssp(L, h, G);
-        tail(L, h, D_hat);
+        tail(L, h, D_hat, two_pass);
         h->tacc_identity = true;
         h->qpad_valid = false;
     }

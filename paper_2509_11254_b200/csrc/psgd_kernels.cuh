@@ -76,24 +76,30 @@ struct ProjectArgs {
     float* P;         // [mats][rows][r]
     int rows, n, r, nodes, nchunks;
     const int* skip;  // when non-null the kernel does nothing if *skip != 0 (refresh already converged)
+    // PEND only (two-pass deferred mode): B holds Delta_{t-1}; the residual e_t = Delta_{t-1} - P~_{t-1} Qsub^T
+    // (Algorithm 2, last line) is formed on the fly from the small factors instead of being read
+    const float* Pprev = nullptr;   // [count][rows][r]
+    const float* Qsub = nullptr;    // [mats][n][r] (qsub_per_node) or [count][n][r]
+    int qsub_per_node = 0;
 };
 
-template <int RP, bool ADD>
+template <int RP, bool ADD, bool PEND = false>
 __host__ __device__ constexpr size_t project_smem_bytes() {
     size_t tiles = (size_t)PJ_STAGES * PJ_TR * PJ_TCP * (ADD ? 2 : 1);
-    size_t q = (size_t)PJ_STAGES * PJ_TC * RP;
+    size_t q = (size_t)PJ_STAGES * PJ_TC * RP * (PEND ? 2 : 1);
     size_t red = (size_t)8 * 32 * RP;
     size_t body = tiles + q;
     return 4 * (body > red ? body : red);
 }
 
-template <int RP, int VEC, bool ADD, bool STORE>
+template <int RP, int VEC, bool ADD, bool STORE, bool PEND = false>
 __global__ void __launch_bounds__(PJ_THREADS) k_project(ProjectArgs a) {
     extern __shared__ __align__(16) float smem[];
     if (a.skip && *a.skip) return;
     float* tA = smem;
     float* tB = tA + (ADD ? PJ_STAGES * PJ_TR * PJ_TCP : 0);
     float* tQ = tB + PJ_STAGES * PJ_TR * PJ_TCP;
+    float* tQs = tQ + PJ_STAGES * PJ_TC * RP;      // PEND: tiles of Qsub beside those of Q
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row0 = blockIdx.x * PJ_TR;
@@ -105,6 +111,7 @@ __global__ void __launch_bounds__(PJ_THREADS) k_project(ProjectArgs a) {
     const float* Bb = ADD ? a.B + mat * (size_t)a.rows * a.n : nullptr;
     float* Mb = STORE ? a.Mout + mat * (size_t)a.rows * a.n : nullptr;
     const float* Qb = a.Q + (size_t)c * a.n * a.r;
+    const float* Qsb = PEND ? a.Qsub + (a.qsub_per_node ? mat : (size_t)c) * a.n * a.r : nullptr;
     const int n = a.n, r = a.r, rows = a.rows;
     const int ntiles = (n + PJ_TC - 1) / PJ_TC;
 
@@ -142,8 +149,15 @@ __global__ void __launch_bounds__(PJ_THREADS) k_project(ProjectArgs a) {
             int ok = (gcol < n && k0 + k < r) ? 4 : 0;
             size_t off = ok ? (size_t)gcol * r + k0 + k : 0;
             cp_async4(sq + e, Qb + off, ok);
+            if (PEND) cp_async4(tQs + stage * PJ_TC * RP + e, Qsb + off, ok);
         }
     };
+    float pp[PEND ? RP : 1];          // PEND: this lane's row of P~_{t-1}
+    if (PEND) {
+#pragma unroll
+        for (int k = 0; k < RP; ++k)
+            pp[k] = (row0 + lane < rows && k0 + k < r) ? __ldg(a.Pprev + ((size_t)c * rows + row0 + lane) * r + k0 + k) : 0.f;
+    }
 
     float acc[RP];
 #pragma unroll
@@ -168,6 +182,22 @@ __global__ void __launch_bounds__(PJ_THREADS) k_project(ProjectArgs a) {
             float4 v = *reinterpret_cast<const float4*>(sa + cb);
             if (ADD) {
                 float4 w = *reinterpret_cast<const float4*>(sb + cb);
+                if (PEND) {     // e = Delta_{t-1} - P~_{t-1} Qsub^T for the 4 columns, k ascending as in k_residual
+                    float corr[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        const float* qs = tQs + stage * PJ_TC * RP + (cb + cc) * RP;
+#pragma unroll
+                        for (int k4 = 0; k4 < RP / 4; ++k4) {
+                            const float4 q4 = *reinterpret_cast<const float4*>(qs + 4 * k4);
+                            corr[cc] = fmaf(pp[4 * k4 + 0], q4.x, corr[cc]);
+                            corr[cc] = fmaf(pp[4 * k4 + 1], q4.y, corr[cc]);
+                            corr[cc] = fmaf(pp[4 * k4 + 2], q4.z, corr[cc]);
+                            corr[cc] = fmaf(pp[4 * k4 + 3], q4.w, corr[cc]);
+                        }
+                    }
+                    w.x -= corr[0]; w.y -= corr[1]; w.z -= corr[2]; w.w -= corr[3];
+                }
                 v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
             }
             if (STORE) *reinterpret_cast<float4*>(sa + cb) = v;

@@ -483,6 +483,41 @@ def test_msgd_update_after_the_step(torch_cuda, m, n, r, mode):
     comp.close()
 
 
+@pytest.mark.parametrize("m,n,r,N,count,form", [
+    (640, 256, 16, 3, 2, "local"),     # the 16-column kernels
+    (1004, 500, 12, 2, 1, "local"),    # 12 -> 16 columns, ragged tiles
+    (520, 260, 9, 4, 1, "mean"),       # residual with the node-averaged Q
+    (333, 130, 5, 2, 1, "local"),      # n % 4 != 0: outside the single-pass plan, scalar loads
+])
+def test_two_pass_deferred_equals_three_pass(torch_cuda, m, n, r, N, count, form):
+    """Deferred mode outside the single-pass plan (r in 9..16, or n % 4 != 0): the residual pass is dropped and the
+    next projection forms e = Delta - P~ Q_i^T on the fly with the same float32 operations in the same order, so
+    free-running steps (with a refresh among them) equal the three-pass mode bit for bit."""
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    torch = torch_cuda
+    out = {}
+    for mode in ("eager", "deferred"):
+        comp = PowerSGDPlus(m, n, r, N, refresh_period=4, seed=9, count=count, mode=mode, error_form=form)
+        for t in range(7):
+            G = synth.make_gradients_torch(2, m, n, N, count, step=t, device="cuda:0")
+            comp.step(G)
+        launches = comp.launch_count()
+        comp.materialize_error()
+        assert comp.last_status() == 0
+        out[mode] = (comp.P_hat.clone(), comp.Q.clone(), comp.E.clone(), launches)
+        comp.close()
+    for a, b in zip(out["eager"][:3], out["deferred"][:3]):
+        assert torch.equal(a, b)
+    assert out["deferred"][3] < out["eager"][3]        # the residual launches really were dropped
+
+
+def test_full_size_config5_rank16_two_pass(torch_cuda):
+    """Workload 5 at r = 16 in deferred mode: projection with the on-the-fly residual and back-projection only."""
+    plan = _full_size_case(torch_cuda, 5, 16384, 4096, 16, 4, 1, tau=0, sample=(0,), free_steps=3)
+    assert plan["single_pass"] == 0
+
+
 @pytest.mark.parametrize("grad_dtype", ["float32", "bfloat16"])
 def test_step_host_equals_step(torch_cuda, grad_dtype):
     """psgd_step_host (pinned host G -> device staging buffer -> step -> P~, Q back to the host) gives bit for bit
