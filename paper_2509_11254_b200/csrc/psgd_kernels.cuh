@@ -149,15 +149,21 @@ __global__ void __launch_bounds__(PJ_THREADS) k_project(ProjectArgs a) {
             int ok = (gcol < n && k0 + k < r) ? 4 : 0;
             size_t off = ok ? (size_t)gcol * r + k0 + k : 0;
             cp_async4(sq + e, Qb + off, ok);
-            if (PEND) cp_async4(tQs + stage * PJ_TC * RP + e, Qsb + off, ok);
+            // Qsub tile with adjacent columns interleaved: {qs[2c][k], qs[2c+1][k]} is one 64-bit operand of the packed FMA
+            if (PEND) cp_async4(tQs + stage * PJ_TC * RP + ((cc >> 1) * RP + k) * 2 + (cc & 1), Qsb + off, ok);
         }
     };
-    float pp[PEND ? RP : 1];          // PEND: this lane's row of P~_{t-1}
+    f2p pp[PEND ? RP : 1];            // PEND: this lane's row of P~_{t-1}, every value twice (one per column of a pair)
     if (PEND) {
 #pragma unroll
-        for (int k = 0; k < RP; ++k)
-            pp[k] = (row0 + lane < rows && k0 + k < r) ? __ldg(a.Pprev + ((size_t)c * rows + row0 + lane) * r + k0 + k) : 0.f;
+        for (int k = 0; k < RP; ++k) {
+            const float pv = (row0 + lane < rows && k0 + k < r) ? __ldg(a.Pprev + ((size_t)c * rows + row0 + lane) * r + k0 + k) : 0.f;
+            pp[k] = pack2(pv, pv);
+        }
     }
+    f2p acc2[PEND ? RP / 2 : 1];      // PEND: the running sums packed in pairs of adjacent k (the kernel is FMA-bound then)
+#pragma unroll
+    for (int k = 0; k < (PEND ? RP / 2 : 1); ++k) acc2[k] = 0ull;
 
     float acc[RP];
 #pragma unroll
@@ -182,21 +188,20 @@ __global__ void __launch_bounds__(PJ_THREADS) k_project(ProjectArgs a) {
             float4 v = *reinterpret_cast<const float4*>(sa + cb);
             if (ADD) {
                 float4 w = *reinterpret_cast<const float4*>(sb + cb);
-                if (PEND) {     // e = Delta_{t-1} - P~_{t-1} Qsub^T for the 4 columns, k ascending as in k_residual
-                    float corr[4] = {0.f, 0.f, 0.f, 0.f};
+                if constexpr (PEND) {     // e = Delta_{t-1} - P~_{t-1} Qsub^T for the 4 columns, k ascending as in k_residual
+                    f2p corr2[2] = {0ull, 0ull};   // columns (0, 1) and (2, 3)
 #pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        const float* qs = tQs + stage * PJ_TC * RP + (cb + cc) * RP;
+                    for (int c2 = 0; c2 < 2; ++c2) {
+                        const ulonglong2* qs = reinterpret_cast<const ulonglong2*>(tQs + stage * PJ_TC * RP + ((cb >> 1) + c2) * RP * 2);
 #pragma unroll
-                        for (int k4 = 0; k4 < RP / 4; ++k4) {
-                            const float4 q4 = *reinterpret_cast<const float4*>(qs + 4 * k4);
-                            corr[cc] = fmaf(pp[4 * k4 + 0], q4.x, corr[cc]);
-                            corr[cc] = fmaf(pp[4 * k4 + 1], q4.y, corr[cc]);
-                            corr[cc] = fmaf(pp[4 * k4 + 2], q4.z, corr[cc]);
-                            corr[cc] = fmaf(pp[4 * k4 + 3], q4.w, corr[cc]);
+                        for (int k2 = 0; k2 < RP / 2; ++k2) {
+                            const ulonglong2 q2 = qs[k2];      // column pair at k = 2 k2 and 2 k2 + 1
+                            corr2[c2] = ffma2(pp[2 * k2 + 0], q2.x, corr2[c2]);
+                            corr2[c2] = ffma2(pp[2 * k2 + 1], q2.y, corr2[c2]);
                         }
                     }
-                    w.x -= corr[0]; w.y -= corr[1]; w.z -= corr[2]; w.w -= corr[3];
+                    const float2 c01 = unpack2(corr2[0]), c23 = unpack2(corr2[1]);
+                    w.x -= c01.x; w.y -= c01.y; w.z -= c23.x; w.w -= c23.y;
                 }
                 v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
             }
@@ -205,6 +210,16 @@ __global__ void __launch_bounds__(PJ_THREADS) k_project(ProjectArgs a) {
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) {
                 const float* q = sq + (cb + cc) * RP;
+                if constexpr (PEND) {
+                    const f2p md = pack2(mv[cc], mv[cc]);
+#pragma unroll
+                    for (int k4 = 0; k4 < RP / 4; ++k4) {
+                        const ulonglong2 qv = *reinterpret_cast<const ulonglong2*>(q + 4 * k4);
+                        acc2[2 * k4 + 0] = ffma2(md, qv.x, acc2[2 * k4 + 0]);
+                        acc2[2 * k4 + 1] = ffma2(md, qv.y, acc2[2 * k4 + 1]);
+                    }
+                    continue;
+                }
 #pragma unroll
                 for (int k4 = 0; k4 < RP / 4; ++k4) {
                     float4 qv = *reinterpret_cast<const float4*>(q + 4 * k4);
@@ -239,6 +254,14 @@ __global__ void __launch_bounds__(PJ_THREADS) k_project(ProjectArgs a) {
     }
     cp_async_wait<0>();
     __syncthreads();
+    if constexpr (PEND) {
+#pragma unroll
+        for (int k = 0; k < RP / 2; ++k) {
+            const float2 t2 = unpack2(acc2[k]);
+            acc[2 * k] = t2.x;
+            acc[2 * k + 1] = t2.y;
+        }
+    }
     // cross-warp reduction, fixed order
     float* red = smem;  // [8][32][RP]
 #pragma unroll
