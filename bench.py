@@ -273,7 +273,10 @@ def sweep_config5(torch, device, peak, mode):
         flags = h.last_status()
         alg, gb = algorithmic_bytes([(m, n, 1)], r, N)
         plan = h.plan_info()
-        out.append({"r": r, "kernel": "single-pass" if (mode == "deferred" and plan["single_pass"]) else "eager", "step_ms": round(ms, 4), "grad_GBps": round(gb / ms / 1e6, 1),
+        path = "three-pass"
+        if mode == "deferred":
+            path = "single-pass" if plan["single_pass"] else ("two-pass" if r <= 16 else "three-pass")
+        out.append({"r": r, "kernel": path, "step_ms": round(ms, 4), "grad_GBps": round(gb / ms / 1e6, 1),
                     "min_bytes_frac": round(alg / ms / 1e6 / peak, 4), "refresh_ms": round(rms, 3),
                     "flags": flags})
         h.close()
