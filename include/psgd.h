@@ -63,7 +63,9 @@ typedef enum {
 #define PSGD_OPT_MODE 2         /* 0: eager (E holds the true residual after every step)
                                    1: deferred (E holds Delta_t = g_t + e_t; the subtraction of
                                       P~_t Q_i^T is folded into the next step's first pass;
-                                      psgd_materialize_error produces the true residual) */
+                                      psgd_materialize_error produces the true residual).  Up to 8 columns the
+                                      whole SSP step is then one pass over G and E, up to 16 two passes; above,
+                                      and on refresh steps, the three-pass kernels run as in mode 0 */
 #define PSGD_OPT_REFRESH_ITERS 3   /* subspace iterations q of the refresh (default 20) */
 #define PSGD_OPT_REFRESH_OVERSAMPLE 4 /* extra columns of the refresh block (default max(8, r)) */
 #define PSGD_OPT_REFRESH_TC 5      /* 1 (default): the early sweeps of a refresh whose block has >= 32 columns run
