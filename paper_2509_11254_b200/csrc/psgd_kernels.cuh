@@ -326,6 +326,26 @@ __global__ void __launch_bounds__(BP_THREADS) k_backproject(BackArgs a) {
         for (int k = 0; k < (PACKED ? RP / 2 : 1); ++k) acc2[j][k] = 0ull;
     }
 
+    auto load8 = [&](int sub0, int rr, float4 (&dst)[8]) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int grow = sub0 + g + 2 * (rr + u);
+            dst[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (grow < rend) {
+                const float* p = Mb + (size_t)grow * n + col;
+                if (VEC == 4) {
+                    if (col < n) dst[u] = ldg_stream4(p);
+                } else {
+                    if (col + 0 < n) dst[u].x = __ldcs(p + 0);
+                    if (col + 1 < n) dst[u].y = __ldcs(p + 1);
+                    if (col + 2 < n) dst[u].z = __ldcs(p + 2);
+                    if (col + 3 < n) dst[u].w = __ldcs(p + 3);
+                }
+            }
+        }
+    };
+    float4 vn[8];
+    load8(rbeg, 0, vn);
     for (int sub0 = rbeg; sub0 < rend; sub0 += BP_SUB) {
         __syncthreads();
         for (int e = tid; e < BP_SUB * RP; e += BP_THREADS) {
@@ -338,22 +358,9 @@ __global__ void __launch_bounds__(BP_THREADS) k_backproject(BackArgs a) {
         for (int rr = 0; rr < BP_SUB / 2; rr += 8) {
             float4 v[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                int lr = g + 2 * (rr + u);
-                int grow = sub0 + lr;
-                v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (grow < rend) {
-                    const float* p = Mb + (size_t)grow * n + col;
-                    if (VEC == 4) {
-                        if (col < n) v[u] = ldg_stream4(p);
-                    } else {
-                        if (col + 0 < n) v[u].x = __ldcs(p + 0);
-                        if (col + 1 < n) v[u].y = __ldcs(p + 1);
-                        if (col + 2 < n) v[u].z = __ldcs(p + 2);
-                        if (col + 3 < n) v[u].w = __ldcs(p + 3);
-                    }
-                }
-            }
+            for (int u = 0; u < 8; ++u) v[u] = vn[u];
+            // the next 8 rows (of this sub-tile, else of the next one) are requested before these are used
+            if (rr + 8 < BP_SUB / 2) load8(sub0, rr + 8, vn); else load8(sub0 + BP_SUB, 0, vn);
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 const float* pr = Ps + (g + 2 * (rr + u)) * RP;
