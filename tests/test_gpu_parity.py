@@ -512,6 +512,32 @@ def test_two_pass_deferred_equals_three_pass(torch_cuda, m, n, r, N, count, form
     assert out["deferred"][3] < out["eager"][3]        # the residual launches really were dropped
 
 
+def test_two_pass_deferred_dense_output_and_state_reset(torch_cuda):
+    """The dense reconstruction asked for at every step and a set_state in the middle of a run (which discards the
+    pending Delta) leave the two-pass mode equal to the three-pass mode."""
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    torch = torch_cuda
+    m, n, r, N = 520, 256, 12, 3
+    res = {}
+    for mode in ("eager", "deferred"):
+        comp = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=4, mode=mode)
+        Dh = torch.empty((1, m, n), dtype=torch.float32, device="cuda:0")
+        outs = []
+        for t in range(5):
+            if t == 3:      # new state while Delta_2 is pending in the deferred mode
+                rng = np.random.default_rng(1)
+                comp.set_state(E=(rng.standard_normal((1, N, m, n)) * 0.01).astype(np.float32),
+                               Q=synth.init_Q(n, r, seed=2)[None], t=3)
+            comp.step(synth.make_gradients_torch(2, m, n, N, 1, step=t, device="cuda:0"), D_hat=Dh)
+            outs.append(Dh.clone())
+        comp.materialize_error()
+        res[mode] = outs + [comp.E.clone(), comp.Q.clone()]
+        comp.close()
+    for a, b in zip(res["eager"], res["deferred"]):
+        assert torch.equal(a, b)
+
+
 def test_full_size_config5_rank16_two_pass(torch_cuda):
     """Workload 5 at r = 16 in deferred mode: projection with the on-the-fly residual and back-projection only."""
     plan = _full_size_case(torch_cuda, 5, 16384, 4096, 16, 4, 1, tau=0, sample=(0,), free_steps=3)
