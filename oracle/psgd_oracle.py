@@ -28,7 +28,9 @@ Pins (tests/test_oracle_*.py): the counterexample's closed-form values, exact
 recovery of exactly-rank-r input, orthonormality, the Pythagoras identity
 Eq. (4), linearity of the compressor (Appendix B), Eq. (6), comparison with an
 independent eigen-solve and exhaustive subset search on tiny inputs, LAPACK QR
-with sign fix, and exact-rational Gram-Schmidt.  Nothing here is "parity
+with sign fix, exact-rational Gram-Schmidt, and for the TF32 product the values
+the number format fixes (last kept and first dropped mantissa bit, truncation
+not rounding) with a hand-computed 2 x 2 x 2 product.  Nothing here is "parity
 unpinned" except the trajectories of the large synthetic workloads, for which
 no published values exist.
 """

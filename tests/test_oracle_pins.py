@@ -306,6 +306,42 @@ def check_counter_function(o):
     np.testing.assert_allclose(gs.mean(axis=0), o.counter_grad(X), atol=1e-15)  # unbiased
 
 
+def check_tf32_product(o):
+    """TF32 keeps 1 sign + 8 exponent + 10 mantissa bits of a float32 and drops the 13 low ones by truncation.
+    Values the format fixes, chosen so that a mask one bit too short or too long, or rounding instead of
+    truncation, gives a different answer; then a 2 x 2 x 2 product worked out by hand."""
+    one = 1.0
+    keep = np.float32(1.0 + 2.0 ** -10)                     # last kept bit
+    drop = np.float32(1.0 + 2.0 ** -11)                     # first dropped bit: truncates to 1, rounding would not
+    drop2 = np.float32(1.0 + 2.0 ** -11 + 2.0 ** -12)       # above half an ulp: still truncates down
+    top = np.float32(2.0 - 2.0 ** -23)                      # all mantissa bits set -> 2 - 2^-10
+    x = np.array([keep, drop, drop2, top, -drop2, -top, 0.0, np.float32(2.0 ** -120) * drop2, np.float32(2.0 ** 100) * top], dtype=np.float32)
+    want = np.array([1.0 + 2.0 ** -10, one, one, 2.0 - 2.0 ** -10, -one, -(2.0 - 2.0 ** -10), 0.0,
+                     2.0 ** -120, 2.0 ** 100 * (2.0 - 2.0 ** -10)])
+    got = o.tf32_truncate(x)
+    assert got.dtype == np.float64
+    np.testing.assert_array_equal(got, want)                 # sign and exponent untouched, magnitude never grows
+    # every TF32 number is a fixed point; truncation is idempotent
+    rng = np.random.default_rng(12)
+    y = (rng.standard_normal(1000) * 10.0 ** rng.integers(-20, 20, 1000)).astype(np.float32)
+    t = o.tf32_truncate(y)
+    np.testing.assert_array_equal(o.tf32_truncate(t.astype(np.float32)), t)
+    assert np.all(np.abs(t) <= np.abs(y.astype(np.float64))) and np.all(np.abs(y - t) < 2.0 ** -10 * np.abs(y) + 1e-300)
+    assert np.all(np.mod(np.frexp(t)[0] * 2.0 ** 11, 1.0) == 0.0)      # at most 11 significant bits
+    # hand-computed product: a11 = 1 + 2^-10 (kept), a12 = 1 + 2^-11 (-> 1), a21 = 3, a22 = -(1 + 2^-11 + 2^-12) (-> -1);
+    # b11 = 2, b12 = 1 + 2^-10 + 2^-13 (-> 1 + 2^-10), b21 = -0.5, b22 = 4.   C = A B^T, C[i][j] = sum_k a[i][k] b[j][k]
+    A = np.array([[keep, drop], [3.0, -drop2]], dtype=np.float32)
+    B = np.array([[2.0, 1.0 + 2.0 ** -10 + 2.0 ** -13], [-0.5, 4.0]], dtype=np.float32)
+    e = 2.0 ** -10
+    C = np.array([[(1 + e) * 2 + 1 * (1 + e), (1 + e) * -0.5 + 1 * 4.0],
+                  [3 * 2 - 1 * (1 + e), 3 * -0.5 - 1 * 4.0]])
+    np.testing.assert_array_equal(o.gemm_nt_tf32(A, B), C)
+    # not transposed by mistake: a non-square case against the definition on already-representable operands
+    A2 = np.array([[1.0, 2.0, 3.0]], dtype=np.float32)
+    B2 = np.array([[1.0, 0.0, 0.0], [0.0, 0.0, 2.0]], dtype=np.float32)
+    np.testing.assert_array_equal(o.gemm_nt_tf32(A2, B2), np.array([[1.0, 6.0]]))
+
+
 ALL_CHECKS = [
     check_counterexample_t0,
     check_counterexample_induction,
@@ -316,6 +352,7 @@ ALL_CHECKS = [
     check_svd_tiny,
     check_fixed_point,
     check_counter_function,
+    check_tf32_product,
 ]
 
 
@@ -397,6 +434,24 @@ def _patch_psi_wrong_arg(mod):
     mod.counter_grad = lambda X: mod.psi_prime(X[0, 0] + X[0, 1] - X[1, 0] - X[1, 1]) * mod.A_MAT
 
 
+def _patch_tf32_mask(bits_dropped):
+    def patch(mod):
+        mask = np.uint32((0xFFFFFFFF << bits_dropped) & 0xFFFFFFFF)
+        mod.tf32_truncate = lambda X: (np.ascontiguousarray(X, dtype=np.float32).view(np.uint32) & mask).view(np.float32).astype(np.float64)
+    return patch
+
+
+def _patch_tf32_rounds(mod):
+    def rn(X):      # round to nearest instead of truncation
+        b = np.ascontiguousarray(X, dtype=np.float32).view(np.uint32)
+        return ((b + np.uint32(0x1000)) & np.uint32(0xFFFFE000)).view(np.float32).astype(np.float64)
+    mod.tf32_truncate = rn
+
+
+def _patch_gemm_not_transposed(mod):
+    mod.gemm_nt_tf32 = lambda A, B: mod.tf32_truncate(A) @ mod.tf32_truncate(B)
+
+
 MUTANTS = {
     "node_mean_used_for_local_Q": _patch_tail_transposed,
     "qr_sign_not_fixed": _patch_no_sign_fix,
@@ -406,6 +461,10 @@ MUTANTS = {
     "svd_trailing_vectors": _patch_svd_right_vectors,
     "psi_argument_garbled": _patch_psi_wrong_arg,
     "stale_Q_state": _patch_stale_q,
+    "tf32_mask_12_bits": _patch_tf32_mask(12),
+    "tf32_mask_14_bits": _patch_tf32_mask(14),
+    "tf32_rounds_to_nearest": _patch_tf32_rounds,
+    "tf32_product_not_transposed": _patch_gemm_not_transposed,
 }
 
 
