@@ -178,10 +178,13 @@ psgd_status psgd_last_status(psgd_handle* h, psgd_stream stream, int* flags /*HO
 psgd_status psgd_debug_ptr(psgd_handle* h, int which, void** ptr, size_t* bytes);
 
 /*
- * Launch plan of the handle, 8 ints (HOST): [0] 1 if the single-pass kernel serves this shape in
- * deferred mode, [1] rank padding, [2] columns per CTA, [3] CTAs per cluster, [4] row slots per
- * matrix, [5] clusters resident at once (-1 before the first single-pass launch), [6] its dynamic
- * shared memory in bytes, [7] row chunks of the eager back-projection.
+ * Launch plan and deferred-mode state of the handle, 12 ints (HOST): [0] 1 if the single-pass kernel
+ * serves this shape in deferred mode, [1] rank padding, [2] columns per CTA, [3] CTAs per cluster,
+ * [4] row slots per matrix, [5] clusters resident at once (-1 before the first single-pass launch),
+ * [6] its dynamic shared memory in bytes, [7] row chunks of the eager back-projection, [8] 1 while E
+ * holds Delta_t and the residual is still pending (deferred mode), [9] 1 if that pending residual is
+ * the single-pass kernel's (padded factors in place), [10] multiprocessors of the device that was
+ * current when the handle was created (148 when none was visible), [11] reserved (0).
  */
 psgd_status psgd_plan_info(const psgd_handle* h, int* info /*HOST*/);
 

@@ -216,9 +216,10 @@ class PowerSGDPlus:
         return flat.view(shape).clone()
 
     def plan_info(self):
-        v = (_int * 8)()
+        v = (_int * 12)()
         _check(lib().psgd_plan_info(self.h, v))
-        keys = ("single_pass", "RP", "WC", "CS", "KC", "active_clusters", "smem_bytes", "S")
+        keys = ("single_pass", "RP", "WC", "CS", "KC", "active_clusters", "smem_bytes", "S", "pending", "pending_single_pass",
+                "sm_count", "reserved")
         return dict(zip(keys, list(v)))
 
     def launch_count(self):

@@ -9,7 +9,10 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <map>
+#include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "psgd_kernels.cuh"
@@ -40,6 +43,14 @@ struct ProfEvent {
     int kind;
 };
 
+// An encoded TMA descriptor together with everything it was encoded from.
+struct CachedMap {
+    const void* base;
+    int64_t n, m, mats;
+    int bw, rows, swizzle, bf16;
+    CUtensorMap map;
+};
+
 }  // namespace
 
 struct psgd_handle {
@@ -65,6 +76,8 @@ struct psgd_handle {
     int64_t launches = 0;
     bool profiling = false;
     std::vector<ProfEvent> events;
+    std::vector<CachedMap> maps;  // tensor maps already encoded for this handle (E and the workspace never move after psgd_attach)
+    size_t map_next = 0;          // slot the next new map replaces once the cache is full
     char err[256] = "no error";
     bool vec4 = false;  // n % 4 == 0 (128-bit paths usable when pointers are 16-byte aligned)
     // single-pass (deferred residual) plan and state
@@ -76,16 +89,27 @@ struct psgd_handle {
     bool pending_fused = false;   // ... and the padded factors the single-pass kernel subtracts are those of that step
     bool tacc_identity = true;    // no preconditioner yet
     bool qpad_valid = false;      // padded copy of Q is current
+    int sm_count = 0;             // multiprocessors of the device that was current when the handle was created
 };
 
 namespace {
 
+// Multiprocessors of the current device; 148 (a B200) when no device is visible, so that a handle can still be
+// created and sized on a machine without one.
+int device_sms() {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+        return sms;
+    cudaGetLastError();
+    return 148;
+}
+
 // K splits of the tensor-core product with M rows and K columns: enough CTAs for about two per SM,
 // at least 8 K-blocks of 32 each
-int gemm_tc_splits(int64_t M, int64_t K, int count) {
+int gemm_tc_splits(int64_t M, int64_t K, int count, int sms) {
     int64_t tiles = ((M + TC_BM - 1) / TC_BM) * count;
     int64_t KB = (K + TC_BK - 1) / TC_BK;
-    int64_t S = std::max<int64_t>(1, std::min<int64_t>((2 * 148 + tiles - 1) / tiles, std::max<int64_t>(1, KB / 8)));
+    int64_t S = std::max<int64_t>(1, std::min<int64_t>((2 * sms + tiles - 1) / tiles, std::max<int64_t>(1, KB / 8)));
     int64_t kbps = (KB + S - 1) / S;
     return (int)((KB + kbps - 1) / kbps);
 }
@@ -100,7 +124,7 @@ int refresh_width(const psgd_handle* h) {
 void plan(psgd_handle* h) {
     h->ell = refresh_width(h);
     const int colblk = ceil_div(h->n, BP_COLS);
-    const int64_t target = 8 * 148;
+    const int64_t target = 8 * (int64_t)h->sm_count;
     int64_t base = (int64_t)h->count * h->N * colblk;
     int S = (int)std::max<int64_t>(1, (target + base - 1) / base);
     S = std::min<int64_t>(S, ceil_div(h->m, BP_SUB));
@@ -142,8 +166,8 @@ void plan(psgd_handle* h) {
         L.dbarT = take(cnt * m * n * 4);
         L.Yt = take(cnt * ell * m * 4);
         L.Zt = take(cnt * ell * n * 4);
-        size_t g1 = gemm_tc_splits(h->m, h->n, h->count) * cnt * m * ncp;
-        size_t g2 = gemm_tc_splits(h->n, h->m, h->count) * cnt * n * ncp;
+        size_t g1 = gemm_tc_splits(h->m, h->n, h->count, h->sm_count) * cnt * m * ncp;
+        size_t g2 = gemm_tc_splits(h->n, h->m, h->count, h->sm_count) * cnt * n * ncp;
         h->gpart_floats = std::max(g1, g2);
         L.gpart = take(h->gpart_floats * 4);
     }
@@ -184,9 +208,10 @@ void plan(psgd_handle* h) {
             // Row slots per matrix.  The workspace is sized here, on the host, for KCmax slots from a table of
             // the clusters of each size that a B200 keeps resident (one CTA per SM); the first launch asks the
             // device for the real number and picks KC <= KCmax for whole waves.
-            static const int resident[FU_MAXCS + 1] = {0, 148, 74, 48, 36, 28, 24, 20, 16};
+            // (upper bound for sizing: one CTA per multiprocessor, clusters packed without regard to the GPC borders)
+            const int resident = std::max(1, h->sm_count / bestCS);
             h->KCmax = (int)std::max<int64_t>(1, std::min<int64_t>(std::min(std::max(1, h->nblk / 4), 64),
-                                                                   (16 * resident[bestCS] + h->count - 1) / h->count));
+                                                                   (16 * resident + h->count - 1) / h->count));
             h->KC = h->KCmax;
             h->active_clusters = -1;
         }
@@ -239,9 +264,23 @@ struct Launcher {
     }
 };
 
+// Opt a kernel in to `bytes` of dynamic shared memory: the attribute is set once per (device, kernel) and raised
+// only when a larger size is asked for.
+void set_smem_attr(const void* kernel, size_t bytes) {
+    static std::mutex mu;
+    static std::map<std::pair<int, const void*>, size_t> done;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    std::lock_guard<std::mutex> lock(mu);
+    size_t& have = done[std::make_pair(dev, kernel)];
+    if (bytes > have) {
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+        have = bytes;
+    }
+}
 template <typename K>
 void allow_smem(K kernel, size_t bytes) {
-    if (bytes > 48 * 1024) cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (bytes > 48 * 1024) set_smem_attr((const void*)kernel, bytes);
 }
 
 inline bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
@@ -262,8 +301,8 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 // Rank-3 map over [count*N][m][n] float32 with tiles of `rows` rows x bw columns of one node; out-of-range reads give zeros.
-bool make_tile_map(CUtensorMap* map, const void* base, int64_t n, int64_t m, int64_t mats, int bw, int rows,
-                   CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_NONE, bool bf16 = false) {
+bool encode_tile_map(CUtensorMap* map, const void* base, int64_t n, int64_t m, int64_t mats, int bw, int rows,
+                     CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_NONE, bool bf16 = false) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     const cuuint64_t es = bf16 ? 2 : 4;
@@ -275,32 +314,70 @@ bool make_tile_map(CUtensorMap* map, const void* base, int64_t n, int64_t m, int
               swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same through the handle's cache: a descriptor is encoded once per distinct (pointer, shape, tile) and reused by
+// every later launch (E, Q and the workspace keep their addresses; gradient buffers usually alternate between a few).
+bool make_tile_map(psgd_handle* h, CUtensorMap* map, const void* base, int64_t n, int64_t m, int64_t mats, int bw, int rows,
+                   CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_NONE, bool bf16 = false) {
+    for (const CachedMap& c : h->maps)
+        if (c.base == base && c.n == n && c.m == m && c.mats == mats && c.bw == bw && c.rows == rows && c.swizzle == (int)swizzle &&
+            c.bf16 == (bf16 ? 1 : 0)) {
+            *map = c.map;
+            return true;
+        }
+    CachedMap c{base, n, m, mats, bw, rows, (int)swizzle, bf16 ? 1 : 0, {}};
+    if (!encode_tile_map(&c.map, base, n, m, mats, bw, rows, swizzle, bf16)) return false;
+    *map = c.map;
+    constexpr size_t kMaxCached = 96;
+    if (h->maps.size() < kMaxCached) h->maps.push_back(c);
+    else { h->maps[h->map_next] = c; h->map_next = (h->map_next + 1) % kMaxCached; }
+    return true;
+}
+
 
 // C = A B^T on the tensor cores: A [count][M][K], B [count][Nc][K] (both K-major), C [count][M][Nc].
 void launch_gemm_tc(Launcher& L, psgd_handle* h, const float* A, const float* B, float* C, int M, int Nc, int K, int kind) {
     const int cnt = h->count;
     const int Ncp = (int)align_up(Nc, 16);
     const int KB = ceil_div(K, TC_BK);
-    const int S = gemm_tc_splits(M, K, cnt);
+    const int S = gemm_tc_splits(M, K, cnt, h->sm_count);
     const int kbps = ceil_div(KB, S);
     float* Cpart = (float*)(h->ws + h->lay.gpart);
     if ((size_t)cnt * S * M * Ncp > h->gpart_floats) { L.status = PSGD_E_WORKSPACE; return; }
     CUtensorMap tmA, tmB;
-    if (!make_tile_map(&tmA, A, K, M, cnt, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tile_map(&tmB, B, K, Nc, cnt, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B)) {
+    if (!make_tile_map(h, &tmA, A, K, M, cnt, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tile_map(h, &tmB, B, K, Nc, cnt, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B)) {
         snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
         L.status = PSGD_E_CUDA;
         return;
     }
     GemmTcArgs g{Cpart, M, Ncp, K, S, kbps, (int*)(h->ws + h->lay.flags)};
     size_t smem = gemm_tc_smem_bytes(Ncp);
-    cudaFuncSetAttribute(k_gemm_tf32, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    set_smem_attr((const void*)k_gemm_tf32, smem);
     L.begin(kind);
     k_gemm_tf32<<<dim3(ceil_div(M, TC_BM), S, cnt), TC_THREADS, smem, L.st>>>(tmA, tmB, g);
     L.end();
     size_t tot = (size_t)cnt * M * Nc;
     L.begin(kind);
     k_gemm_reduce<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Cpart, C, M, Nc, Ncp, S, cnt);
+    L.end();
+}
+
+// M = G + E over E (Eq. (7a)), optionally Dbar = node mean of M (SVD-Comp, first line): 128-bit accesses when the
+// row-major arrays allow it.
+void launch_add_mean(Launcher& L, const void* G, bool bf16, float* E, float* dbar, size_t per_mat, int N, int cnt, int kind) {
+    const bool vec = per_mat % 4 == 0 && aligned16(E) && (!dbar || aligned16(dbar)) && (((uintptr_t)G & (bf16 ? 7 : 15)) == 0);
+    const int V = vec ? 4 : 1;
+    const size_t want = (per_mat + (size_t)V * 256 - 1) / ((size_t)V * 256);
+    const unsigned gx = (unsigned)std::max<size_t>(1, std::min<size_t>(want, (size_t)std::max(1, L.h->sm_count * 8 / cnt)));
+    dim3 grid(gx, (unsigned)cnt);
+    L.begin(kind);
+    if (bf16) {
+        if (vec) k_add_mean<unsigned short, 4><<<grid, 256, 0, L.st>>>((const unsigned short*)G, E, dbar, per_mat, N, cnt);
+        else k_add_mean<unsigned short, 1><<<grid, 256, 0, L.st>>>((const unsigned short*)G, E, dbar, per_mat, N, cnt);
+    } else {
+        if (vec) k_add_mean<float, 4><<<grid, 256, 0, L.st>>>((const float*)G, E, dbar, per_mat, N, cnt);
+        else k_add_mean<float, 1><<<grid, 256, 0, L.st>>>((const float*)G, E, dbar, per_mat, N, cnt);
+    }
     L.end();
 }
 
@@ -357,9 +434,9 @@ bool launch_project_tc(Launcher& L, const float* A, const float* B, float* Mout,
     k_split_pad_t<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Q, Qt, n, r, Ncp, count, skip);
     L.end();
     CUtensorMap tA, tB, tQ[3];
-    bool ok = make_tile_map(&tA, A, n, rows, mats, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) &&
-              make_tile_map(&tB, B ? B : A, n, rows, mats, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B);
-    for (int t = 0; t < 3 && ok; ++t) ok = make_tile_map(&tQ[t], Qt + t * tot, n, Ncp, count, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B);
+    bool ok = make_tile_map(h, &tA, A, n, rows, mats, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) &&
+              make_tile_map(h, &tB, B ? B : A, n, rows, mats, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B);
+    for (int t = 0; t < 3 && ok; ++t) ok = make_tile_map(h, &tQ[t], Qt + t * tot, n, Ncp, count, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) {
         snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
         L.status = PSGD_E_CUDA;
@@ -367,7 +444,7 @@ bool launch_project_tc(Launcher& L, const float* A, const float* B, float* Mout,
     }
     ProjTcArgs a{B ? Mout : nullptr, P, rows, n, r, Ncp, proj_tc_nh(Ncp), B ? 1 : 0, nodes, (int*)(h->ws + h->lay.flags), skip};
     size_t smem = proj_tc_smem_bytes(Ncp);
-    cudaFuncSetAttribute(k_project_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    set_smem_attr((const void*)k_project_tc, smem);
     L.begin(PSGD_K_PROJECT);
     k_project_tc<<<dim3(ceil_div(rows, TC_BM), mats), PT_THREADS, smem, L.st>>>(tA, tB, tQ[0], tQ[1], tQ[2], a);
     L.end();
@@ -417,7 +494,7 @@ int launch_back_tc(Launcher& L, const float* M, const float* Phat, float* part, 
         const int kbs = ceil_div(KB, s);
         if (s > 1 && kbs < 16) break;
         if ((int64_t)(s - 1) * kbs >= KB) continue;     // would leave an empty split
-        const int64_t cost = ((base * s + 147) / 148) * (kbs + 8);
+        const int64_t cost = ((base * s + h->sm_count - 1) / h->sm_count) * (kbs + 8);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
     }
     const int St = best, kbs = ceil_div(KB, St);
@@ -427,8 +504,8 @@ int launch_back_tc(Launcher& L, const float* M, const float* Phat, float* part, 
     k_split_pad_t<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Phat, Pt, rows, r, Ncp, count, skip);
     L.end();
     CUtensorMap tM, tP[3];
-    bool ok = make_tile_map(&tM, M, n, rows, mats, 32, TC_BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
-    for (int t = 0; t < 3 && ok; ++t) ok = make_tile_map(&tP[t], Pt + t * tot, rows, Ncp, count, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B);
+    bool ok = make_tile_map(h, &tM, M, n, rows, mats, 32, TC_BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
+    for (int t = 0; t < 3 && ok; ++t) ok = make_tile_map(h, &tP[t], Pt + t * tot, rows, Ncp, count, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) {
         snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
         L.status = PSGD_E_CUDA;
@@ -436,7 +513,7 @@ int launch_back_tc(Launcher& L, const float* M, const float* Phat, float* part, 
     }
     BackTcArgs a{part, rows, n, r, Ncp, back_tc_nh(Ncp), St, kbs, nodes, (int*)(h->ws + h->lay.flags), skip};
     size_t smem = back_tc_smem_bytes(Ncp);
-    cudaFuncSetAttribute(k_backproject_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    set_smem_attr((const void*)k_backproject_tc, smem);
     L.begin(PSGD_K_BACKPROJECT);
     k_backproject_tc<<<dim3(ceil_div(n, TC_BM), St, mats), PT_THREADS, smem, L.st>>>(tM, tP[0], tP[1], tP[2], a);
     L.end();
@@ -477,8 +554,8 @@ bool launch_resid_tc(Launcher& L, const float* M, float* Out, const float* Phat,
     L.end();
     CUtensorMap tP[3], tQ[3];
     for (int t = 0; t < 3; ++t) {
-        if (!make_tile_map(&tP[t], Pt[t], KP, rows, cnt, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-            !make_tile_map(&tQ[t], Qt[t], KP, n, qmats, TC_BK, RT_BN, CU_TENSOR_MAP_SWIZZLE_128B)) {
+        if (!make_tile_map(h, &tP[t], Pt[t], KP, rows, cnt, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tile_map(h, &tQ[t], Qt[t], KP, n, qmats, TC_BK, RT_BN, CU_TENSOR_MAP_SWIZZLE_128B)) {
             snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
             L.status = PSGD_E_CUDA;
             return true;
@@ -486,7 +563,7 @@ bool launch_resid_tc(Launcher& L, const float* M, float* Out, const float* Phat,
     }
     ResidTcArgs a{M, Out, rows, n, KP, out_per_node ? nodes : 1, q_per_node, (int*)(h->ws + h->lay.flags)};
     size_t smem = resid_tc_smem_bytes();
-    cudaFuncSetAttribute(k_residual_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    set_smem_attr((const void*)k_residual_tc, smem);
     L.begin(PSGD_K_RESIDUAL);
     k_residual_tc<<<dim3(ceil_div(rows, TC_BM), mats), RT_THREADS, smem, L.st>>>(tP[0], tP[1], tP[2], tQ[0], tQ[1], tQ[2], a);
     L.end();
@@ -497,7 +574,7 @@ void launch_resid(Launcher& L, const float* M, float* Out, const float* Phat, co
                   int nodes, int mats, int q_per_node, int out_per_node, bool vec) {
     if (r > 16 && launch_resid_tc(L, M, Out, Phat, Qf, rows, n, r, nodes, mats, q_per_node, out_per_node)) return;
     int rpc = 128;
-    while (rpc > RS_SUB && (int64_t)mats * ceil_div(n, RS_COLS) * ceil_div(rows, rpc) < 4 * 148) rpc /= 2;
+    while (rpc > RS_SUB && (int64_t)mats * ceil_div(n, RS_COLS) * ceil_div(rows, rpc) < 4 * L.h->sm_count) rpc /= 2;
     ResidArgs a{M, Out, Phat, Qf, rows, n, r, nodes, rpc, q_per_node, out_per_node};
     vec = vec && aligned16(Out) && (!M || aligned16(M));
     dim3 grid(ceil_div(n, RS_COLS), ceil_div(rows, rpc), mats);
@@ -512,7 +589,7 @@ void launch_resid(Launcher& L, const float* M, float* Out, const float* Phat, co
 void launch_msgd(Launcher& L, float* X, float* Mom, float eta, float mu, const float* Phat, const float* Qf, int rows, int n,
                  int r, int mats) {
     int rpc = 128;
-    while (rpc > RS_SUB && (int64_t)mats * ceil_div(n, RS_COLS) * ceil_div(rows, rpc) < 4 * 148) rpc /= 2;
+    while (rpc > RS_SUB && (int64_t)mats * ceil_div(n, RS_COLS) * ceil_div(rows, rpc) < 4 * L.h->sm_count) rpc /= 2;
     ResidArgs a{nullptr, nullptr, Phat, Qf, rows, n, r, 1, rpc, 0, 0};
     a.X = X; a.Mom = Mom; a.eta = eta; a.mu = mu;
     dim3 grid(ceil_div(n, RS_COLS), ceil_div(rows, rpc), mats);
@@ -596,16 +673,12 @@ void ssp(Launcher& L, psgd_handle* h, const void* Gv) {
         launch_project_pending(L, G, h->E, h->Q, Pnode, Phat, h->error_form == 0 ? Qnode : h->Q, h->error_form == 0 ? 1 : 0,
                                m, n, r, N, cnt, h->vec4);
     } else if (h->grad_bf16) {      // M = G + E formed in the E buffer first (10 B/element), then the projection reads M
-        L.begin(PSGD_K_PROJECT);
-        k_add_mean<<<148 * 8, 256, 0, L.st>>>((const unsigned short*)Gv, h->E, nullptr, (size_t)m * n, N, cnt);
-        L.end();
+        launch_add_mean(L, Gv, true, h->E, nullptr, (size_t)m * n, N, cnt, PSGD_K_PROJECT);
         launch_project(L, h->E, nullptr, nullptr, h->Q, Pnode, m, n, r, N, cnt, h->vec4);
     } else if (r <= 32 || (h->ptc_ok && aligned16(G))) {
         launch_project(L, G, h->E, h->E, h->Q, Pnode, m, n, r, N, cnt, h->vec4);
     } else {
-        L.begin(PSGD_K_PROJECT);
-        k_add_mean<<<148 * 8, 256, 0, L.st>>>(G, h->E, nullptr, (size_t)m * n, N, cnt);
-        L.end();
+        launch_add_mean(L, G, false, h->E, nullptr, (size_t)m * n, N, cnt, PSGD_K_PROJECT);
         launch_project(L, h->E, nullptr, nullptr, h->Q, Pnode, m, n, r, N, cnt, h->vec4);
     }
     size_t tot = (size_t)cnt * m * r;
@@ -647,10 +720,7 @@ void svd(Launcher& L, psgd_handle* h, const void* G) {
     const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count, ell = h->ell;
     const int K = PSGD_K_REFRESH;
     L.force_kind = K;
-    L.begin(K);
-    if (h->grad_bf16) k_add_mean<<<148 * 8, 256, 0, L.st>>>((const unsigned short*)G, h->E, dbar, (size_t)m * n, N, cnt);
-    else k_add_mean<<<148 * 8, 256, 0, L.st>>>((const float*)G, h->E, dbar, (size_t)m * n, N, cnt);
-    L.end();
+    launch_add_mean(L, G, h->grad_bf16, h->E, dbar, (size_t)m * n, N, cnt, K);
     size_t zt = (size_t)cnt * n * ell;
     L.begin(K);
     k_fill_normal<<<(unsigned)((zt + 255) / 256), 256, 0, L.st>>>(Z, zt, h->seed, 0x5eed0000ull + (uint64_t)h->t);
@@ -677,7 +747,7 @@ void svd(Launcher& L, psgd_handle* h, const void* G) {
     // chunking of Z = Dbar^T Y over rows
     int colblk = ceil_div(n, BP_COLS);
     int64_t base = (int64_t)cnt * colblk * ceil_div(ell, 16);
-    int S = (int)std::max<int64_t>(1, (8 * 148 + base - 1) / base);
+    int S = (int)std::max<int64_t>(1, (8 * (int64_t)h->sm_count + base - 1) / base);
     S = std::min(S, std::min(64, ceil_div(m, BP_SUB)));
     int rpc = (int)align_up(ceil_div(m, S), BP_SUB);
     S = ceil_div(m, rpc);
@@ -763,7 +833,7 @@ void launch_fused_t(Launcher& L, psgd_handle* h, const void* G, FusedArgs a) {
     void (*kern)(CUtensorMap, CUtensorMap, FusedArgs) =
         h->grad_bf16 ? (h->pending ? k_fused_step<RP, WC, true, true> : k_fused_step<RP, WC, false, true>)
                      : (h->pending ? k_fused_step<RP, WC, true, false> : k_fused_step<RP, WC, false, false>);
-    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->fused_smem);
+    set_smem_attr((const void*)kern, h->fused_smem);
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(FU_THREADS);
     cfg.dynamicSmemBytes = h->fused_smem;
@@ -800,8 +870,8 @@ void launch_fused_t(Launcher& L, psgd_handle* h, const void* G, FusedArgs a) {
     cfg.gridDim = dim3((unsigned)((size_t)h->CS * h->KC * h->count));
     CUtensorMap tmG, tmM;
     const int bw = FusedGeom<WC>::BW, rs = FusedGeom<WC>::RS;
-    if (!make_tile_map(&tmG, G, h->n, h->m, (int64_t)h->count * h->N, bw, rs, CU_TENSOR_MAP_SWIZZLE_NONE, h->grad_bf16) ||
-        !make_tile_map(&tmM, h->E, h->n, h->m, (int64_t)h->count * h->N, bw, rs)) {
+    if (!make_tile_map(h, &tmG, G, h->n, h->m, (int64_t)h->count * h->N, bw, rs, CU_TENSOR_MAP_SWIZZLE_NONE, h->grad_bf16) ||
+        !make_tile_map(h, &tmM, h->E, h->n, h->m, (int64_t)h->count * h->N, bw, rs)) {
         snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
         L.status = PSGD_E_CUDA;
         return;
@@ -943,6 +1013,7 @@ psgd_status psgd_create_batch(int64_t m, int64_t n, int r, int N, int count, int
     if (!h) return PSGD_E_INVALID;
     h->m = m; h->n = n; h->r = r; h->N = N; h->count = count; h->tau = refresh_period; h->seed = seed;
     h->vec4 = (n % 4 == 0);
+    h->sm_count = device_sms();
     plan(h);
     *out = h;
     return PSGD_OK;
@@ -1101,6 +1172,7 @@ psgd_status psgd_plan_info(const psgd_handle* h, int* info) {
     if (!h || !info) return PSGD_E_NULL;
     info[0] = h->fused_ok ? 1 : 0; info[1] = h->RP; info[2] = h->WC; info[3] = h->CS; info[4] = h->KC;
     info[5] = h->active_clusters; info[6] = (int)h->fused_smem; info[7] = h->S;
+    info[8] = h->pending ? 1 : 0; info[9] = (h->pending && h->pending_fused) ? 1 : 0; info[10] = h->sm_count; info[11] = 0;
     return PSGD_OK;
 }
 
@@ -1149,7 +1221,7 @@ extern "C" {
 psgd_status psgd_gemm_nt_tf32_scratch(int64_t M, int64_t Nc, int64_t K, int count, size_t* scratch_bytes) {
     if (!scratch_bytes) return PSGD_E_NULL;
     if (!(M >= 1 && Nc >= 1 && Nc <= TC_MAXN && K >= 4 && K % 4 == 0 && count >= 1 && count <= 65535)) return PSGD_E_INVALID;
-    *scratch_bytes = (size_t)gemm_tc_splits(M, K, count) * count * M * align_up(Nc, 16) * 4 + 256;
+    *scratch_bytes = (size_t)gemm_tc_splits(M, K, count, device_sms()) * count * M * align_up(Nc, 16) * 4 + 256;
     return PSGD_OK;
 }
 
@@ -1164,18 +1236,18 @@ psgd_status psgd_gemm_nt_tf32(const float* A, const float* B, float* C, int64_t 
     cudaStream_t cs = (cudaStream_t)stream;
     const int Ncp = (int)align_up(Nc, 16);
     const int KB = ceil_div(K, TC_BK);
-    const int S = gemm_tc_splits(M, K, count);
+    const int S = gemm_tc_splits(M, K, count, device_sms());
     const int kbps = ceil_div(KB, S);
     int* flags = (int*)scratch;                       // first 256 bytes: status word
     float* Cpart = (float*)((char*)scratch + 256);
     CUtensorMap tmA, tmB;
-    if (!make_tile_map(&tmA, A, K, M, count, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tile_map(&tmB, B, K, Nc, count, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B))
+    if (!encode_tile_map(&tmA, A, K, M, count, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !encode_tile_map(&tmB, B, K, Nc, count, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B))
         return PSGD_E_CUDA;
     if (cudaMemsetAsync(flags, 0, 4, cs) != cudaSuccess) return PSGD_E_CUDA;
     GemmTcArgs g{Cpart, (int)M, Ncp, (int)K, S, kbps, flags};
     size_t smem = gemm_tc_smem_bytes(Ncp);
-    cudaFuncSetAttribute(k_gemm_tf32, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    set_smem_attr((const void*)k_gemm_tf32, smem);
     k_gemm_tf32<<<dim3(ceil_div(M, TC_BM), S, count), TC_THREADS, smem, cs>>>(tmA, tmB, g);
     size_t tot = (size_t)count * M * Nc;
     k_gemm_reduce<<<(unsigned)((tot + 255) / 256), 256, 0, cs>>>(Cpart, C, (int)M, (int)Nc, Ncp, S, count);

@@ -586,20 +586,42 @@ __global__ void __launch_bounds__(RS_THREADS) k_residual(ResidArgs a) {
 __device__ __forceinline__ float grad_value(const float* G, size_t i) { return __ldcs(G + i); }
 __device__ __forceinline__ float grad_value(const unsigned short* G, size_t i) { return __uint_as_float((unsigned)__ldcs(G + i) << 16); }
 
-template <typename TG>
-__global__ void k_add_mean(const TG* G, float* E, float* Dbar, size_t per_mat, int nodes, int count) {
-    size_t total = per_mat * count;
-    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-         idx += (size_t)gridDim.x * blockDim.x) {
-        size_t c = idx / per_mat, e = idx % per_mat;
-        float s = 0.f;
-        for (int i = 0; i < nodes; ++i) {
-            size_t off = (c * nodes + i) * per_mat + e;
-            float mval = grad_value(G, off) + E[off];
-            E[off] = mval;
-            s += mval;
+__device__ __forceinline__ float4 grad_value4(const float* G, size_t i) { return __ldcs(reinterpret_cast<const float4*>(G + i)); }
+__device__ __forceinline__ float4 grad_value4(const unsigned short* G, size_t i) {
+    const uint2 b = __ldcs(reinterpret_cast<const uint2*>(G + i));
+    return make_float4(__uint_as_float(b.x << 16), __uint_as_float(b.x & 0xFFFF0000u), __uint_as_float(b.y << 16), __uint_as_float(b.y & 0xFFFF0000u));
+}
+
+// VEC == 4: per_mat % 4 == 0 and all three arrays 16-byte aligned (8-byte for bfloat16 G); a thread owns 4 adjacent
+// elements of one matrix for all its nodes (128-bit accesses, the matrix index comes from blockIdx.y: no division).
+// grid: (x: any, y: count).
+template <typename TG, int VEC>
+__global__ void __launch_bounds__(256) k_add_mean(const TG* G, float* E, float* Dbar, size_t per_mat, int nodes, int count) {
+    const size_t c = blockIdx.y;
+    const float nf = (float)nodes;
+    const size_t stride = (size_t)gridDim.x * blockDim.x * VEC;
+    for (size_t e = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * VEC; e < per_mat; e += stride) {
+        if (VEC == 4) {
+            float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int i = 0; i < nodes; ++i) {
+                const size_t off = (c * nodes + i) * per_mat + e;
+                const float4 g = grad_value4(G, off);
+                float4 m = *reinterpret_cast<const float4*>(E + off);
+                m.x += g.x; m.y += g.y; m.z += g.z; m.w += g.w;
+                *reinterpret_cast<float4*>(E + off) = m;
+                s.x += m.x; s.y += m.y; s.z += m.z; s.w += m.w;
+            }
+            if (Dbar) *reinterpret_cast<float4*>(Dbar + c * per_mat + e) = make_float4(s.x / nf, s.y / nf, s.z / nf, s.w / nf);
+        } else {
+            float s = 0.f;
+            for (int i = 0; i < nodes; ++i) {
+                const size_t off = (c * nodes + i) * per_mat + e;
+                const float mval = grad_value(G, off) + E[off];
+                E[off] = mval;
+                s += mval;
+            }
+            if (Dbar) Dbar[c * per_mat + e] = s / nf;
         }
-        if (Dbar) Dbar[idx] = s / (float)nodes;
     }
 }
 

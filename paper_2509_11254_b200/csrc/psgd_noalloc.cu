@@ -56,7 +56,7 @@ extern "C" psgd_status psgd_backproject_static(const float* M, const float* P_ha
     // row chunking: as many chunks as fill the GPU, but no more than the scratch holds
     const int colblk = ceil_div(n, BP_COLS);
     int64_t base = (int64_t)N * colblk;
-    int S = (int)std::max<int64_t>(1, (8 * 148 + base - 1) / base);
+    int S = (int)std::max<int64_t>(1, (8 * (int64_t)device_sms() + base - 1) / base);
     S = std::min<int64_t>(S, ceil_div(m, BP_SUB));
     S = (int)std::min<size_t>((size_t)S, max_floats / per_chunk);
     int rpc = (int)align_up(ceil_div(m, S), BP_SUB);
