@@ -1,14 +1,20 @@
 #!/usr/bin/env python
 """Benchmark of the PowerSGD+ compression hot path on B200.
 
-One "step" is one iteration of Algorithm 2 (without the optimizer) over ALL
-matrices of the workload: error-feedback add, SSP-Comp or (every tau steps)
-SVD-Comp, residual update.  Default workload: the 130M-parameter LLaMA-shaped
-stack (84 matrices, r = 8, N = 8 simulated nodes, refresh every 50 steps) with
-synthetic gradients.  Prints ONE JSON line (rank 0).
+One "step" is one iteration of Algorithm 2 (without the optimizer) over ALL matrices of a
+workload: error-feedback add, SSP-Comp or (every tau steps) SVD-Comp, residual update.
+
+The metric is quoted per rank r on the single large matrix (m = 16384, n = 4096, N = 4 simulated
+nodes, low-rank-plus-noise gradients), so that sweep is the body of the line: for every
+r in {1, 4, 8, 16, 64, 128} the step latency (median and minimum over blocks of steps), the
+gradient GB/s, the fraction of the 12-bytes-per-element HBM roofline, the dominant kernel with
+its own achieved bandwidth, and the latency of one SVD refresh.  The headline `value` is the one
+at r = 16, where the target binds.  The three model-shaped stacks follow as `stacks` (refreshes
+amortised at their period).  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                  [--workload 2|3|4|5] [--rank r] [--no-sweep] [--no-e2e] [--no-cpu]
+                  [--rank r] [--stacks 2,3,4|none] [--no-sweep] [--no-e2e] [--no-cpu]
+                  [--single-pass auto|cluster|none|l2] [--mode deferred|eager]
 
 Metric: gradient GB/s = bytes of G consumed per second, whole job.
 """
@@ -29,30 +35,31 @@ sys.path.insert(0, ROOT)
 METRIC = "powersgd_plus_step_gradient_throughput"
 UNIT = "GB/s"
 FALLBACK_HBM = 6650.0
+SWEEP_SHAPE = (16384, 4096, 4)          # m, n, N of the sweep workload
+SWEEP_RANKS = (1, 4, 8, 16, 64, 128)
+HEADLINE_RANK = 16
 # dram__bytes_read.sum + dram__bytes_write.sum per element of one launch, from the ncu captures summarised under
-# profiles/ (taken on the 16384x4096, N=4 workload, where traffic grows in proportion to the elements)
+# profiles/ (small case of the same kernel; traffic grows in proportion to the elements).  None: no current capture.
 TRAFFIC_BYTES_PER_ELEMENT = {"k_fused_step": 11.87}
 
-# default (rank, nodes, refresh period) per workload id
-DEFAULTS = {2: (8, 8, 50), 3: (16, 16, 20), 4: (32, 8, 100), 5: (16, 4, 0), 1: (4, 4, 5)}
+# (rank, nodes, refresh period) of the stacks
+STACK_DEFAULTS = {2: [(8, 8, 50)], 3: [(4, 16, 20), (16, 16, 20)], 4: [(32, 8, 100)]}
 
 
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=300, help="timed steps of the headline (r = 16) measurement")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=2)
-    ap.add_argument("--rank", type=int, default=None)
+    ap.add_argument("--rank", type=int, default=HEADLINE_RANK, help="rank of the headline measurement")
     ap.add_argument("--mode", default="deferred", choices=["eager", "deferred"])
-    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--single-pass", default="auto", choices=["auto", "cluster", "none", "l2"])
+    ap.add_argument("--stacks", default="2,3,4", help="model-shaped stacks to add (workload ids), or 'none'")
+    ap.add_argument("--no-sweep", action="store_true", help="only the headline rank")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--no-refresh", action="store_true", help="tau = 0 (plain PowerSGD steps only)")
-    ap.add_argument("--refresh-period", type=int, default=None, help="override the workload's refresh period tau")
-    ap.add_argument("--grad-dtype", default="float32", choices=["float32", "bfloat16"],
-                    help="storage type of the gradients G (bfloat16: 2 bytes per element read instead of 4)")
+    ap.add_argument("--small", action="store_true", help="a quarter of the sweep matrix (m = 4096): for profiler captures")
     return ap.parse_args()
 
 
@@ -64,6 +71,13 @@ def peaks():
         except Exception:
             pass
     return FALLBACK_HBM, "fallback"
+
+
+def host_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count()
 
 
 class ClockSampler:
@@ -118,12 +132,6 @@ class ClockSampler:
         return out
 
 
-def stack_for(workload):
-    from paper_2509_11254_b200 import synth
-
-    return synth.STACKS[workload]
-
-
 def algorithmic_bytes(shapes, r, N, g_bytes_per_element=4):
     """Minimum traffic of a step: read G, read E, write E per element (12 B with float32 G) plus the P/Q traffic."""
     el = sum(m * n * c for m, n, c in shapes) * N
@@ -131,57 +139,199 @@ def algorithmic_bytes(shapes, r, N, g_bytes_per_element=4):
     return (8 + g_bytes_per_element) * el + pq, g_bytes_per_element * el
 
 
+FAMILY_BYTES = {"project": 12, "backproject": 4, "residual": 8}   # algorithmic bytes per element of one launch set
+
+
+def kernel_name(family, r, step_kernel):
+    if family == "project":
+        if step_kernel == 1:
+            return "k_fused_step"
+        if step_kernel == 2:
+            return "k_stream_step"
+        return "k_project_tc" if r > 16 else "k_project"
+    return ("k_%s_tc" if r > 16 else "k_%s") % family
+
+
+# ----------------------------------------------------------------------------
+# timing helpers
+# ----------------------------------------------------------------------------
+def time_blocks(torch, step_fn, total_steps, block=50, min_seconds=0.0, max_blocks=40):
+    """Blocks of `block` steps timed with CUDA events on the current stream until `total_steps` steps and
+    `min_seconds` of device time have passed.  Returns (ms per step of every block, steps done)."""
+    per_block, done, spent = [], 0, 0.0
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    while (done < total_steps or spent < min_seconds * 1e3) and len(per_block) < max_blocks:
+        k = min(block, max(1, total_steps - done)) if done < total_steps else block
+        torch.cuda.synchronize()
+        ev0.record()
+        for s in range(k):
+            step_fn(done + s)
+        ev1.record()
+        torch.cuda.synchronize()
+        ms = ev0.elapsed_time(ev1)
+        per_block.append(ms / k)
+        done += k
+        spent += ms
+    return per_block, done
+
+
+def family_profile(handles, step_fn, steps):
+    """Second pass with per-launch CUDA events on the launching stream: milliseconds per step of every kernel family."""
+    for h in handles:
+        h.profile_begin()
+    for s in range(steps):
+        step_fn(s)
+    fam = {}
+    for h in handles:
+        for k, (ms, ln) in h.profile_read().items():
+            a = fam.setdefault(k, [0.0, 0])
+            a[0] += ms
+            a[1] += ln
+    return {k: (v[0] / steps, v[1] / steps) for k, v in fam.items() if v[1]}
+
+
+def roofline_entry(fam, r, step_kernel, elements, peak, peak_kind):
+    dom = max(("project", "backproject", "residual"), key=lambda k: fam.get(k, (0.0, 0))[0])
+    ms = fam[dom][0]
+    name = kernel_name(dom, r, step_kernel)
+    achieved = FAMILY_BYTES[dom] * elements / ms / 1e6
+    tb = TRAFFIC_BYTES_PER_ELEMENT.get(name)
+    return {"bound": "hbm", "kernel": name, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+            "frac": round(achieved / peak, 4), "traffic": tb * elements if tb is not None else None,
+            "peak_source": f"of {peak_kind}", "ms_per_launch_set": round(ms, 4),
+            "algorithmic_bytes_per_launch_set": FAMILY_BYTES[dom] * elements,
+            "per_family_ms_per_step": {k: round(v[0], 4) for k, v in fam.items()}}
+
+
+# ----------------------------------------------------------------------------
+# the sweep (workload 5)
+# ----------------------------------------------------------------------------
+def sweep_point(torch, device, r, bufs, mode, single_pass, steps, min_seconds, peak, peak_kind, refresh=True):
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    N, m, n = bufs[0].shape[1], bufs[0].shape[2], bufs[0].shape[3]
+    h = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=5, device=device, mode=mode, single_pass=single_pass)
+    for s in range(5):
+        h.step(bufs[s % 2])
+    l0 = h.launch_count()
+    blocks, done = time_blocks(torch, lambda s: h.step(bufs[s % 2]), steps, min_seconds=min_seconds)
+    launches = h.launch_count() - l0
+    fam = family_profile([h], lambda s: h.step(bufs[s % 2]), 20)
+    plan = h.plan_info()
+    out = {"r": r, "step_ms": round(statistics.median(blocks), 4), "step_ms_min": round(min(blocks), 4), "steps_timed": done,
+           "blocks": len(blocks)}
+    alg, gb = algorithmic_bytes([(m, n, 1)], r, N)
+    ms = out["step_ms"]
+    out.update(grad_GBps=round(gb / ms / 1e6, 1), min_bytes_frac=round(alg / ms / 1e6 / peak, 4),
+               path={0: ("two-pass" if (mode == "deferred" and r <= 16) else "three-pass"), 1: "single-pass (cluster kernel)",
+                     2: "single-pass (L2-pipelined kernel)"}[plan["step_kernel"]],
+               roofline=roofline_entry(fam, r, plan["step_kernel"], m * n * N, peak, peak_kind),
+               launches_per_step=round(launches / done, 2))
+    if refresh:
+        h.refresh(bufs[0])
+        rb, _ = time_blocks(torch, lambda s: h.refresh(bufs[s % 2]), 3, block=1)
+        out["refresh_ms"] = round(statistics.median(rb), 3)
+        out["refresh_ms_min"] = round(min(rb), 3)
+    out["flags"] = h.last_status()
+    return out, h, launches, done
+
+
+# ----------------------------------------------------------------------------
+# the model-shaped stacks (workloads 2, 3, 4)
+# ----------------------------------------------------------------------------
+def stack_bench(torch, device, workload, r, N, tau, mode, single_pass, peak, peak_kind):
+    from paper_2509_11254_b200 import PowerSGDPlus, StreamedStack, synth
+
+    shapes = synth.STACKS[workload]
+    nbuf = 1 if workload == 4 else 2
+    bufs = [[synth.make_gradients_torch(workload, m, n, N, c, step=b, device=device) for (m, n, c) in shapes] for b in range(nbuf)]
+    handles = [PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=1 + i, count=c, device=device, mode=mode, single_pass=single_pass)
+               for i, (m, n, c) in enumerate(shapes)]
+    stack = StreamedStack(handles, device)
+    for s in range(3):            # t = 0 is a refresh
+        stack.step(bufs[s % nbuf])
+    # SSP steps only (t = 3 .. < tau), then one refresh step on its own; the amortised figure follows from the two
+    n_ssp = max(4, min(40 if workload != 4 else 10, tau - 8))
+    blocks, done = time_blocks(torch, lambda s: stack.step(bufs[s % nbuf]), n_ssp, block=max(1, n_ssp // 2), max_blocks=2)
+    ssp_ms = statistics.median(blocks)
+    fam = family_profile(handles, lambda s: [h.step(g) for h, g in zip(handles, bufs[s % nbuf])], 3)
+    plans = [h.plan_info() for h in handles]
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for h, g in zip(handles, bufs[0]):
+        h.refresh(g)
+    ev1.record()
+    torch.cuda.synchronize()
+    refresh_ms = ev0.elapsed_time(ev1)
+    flags = [h.last_status() for h in handles]
+    alg, gb = algorithmic_bytes(shapes, r, N)
+    ms = ((tau - 1) * ssp_ms + refresh_ms) / tau if tau > 0 else ssp_ms
+    el = sum(m * n * c for m, n, c in shapes) * N
+    out = {"workload": synth.WORKLOADS[workload]["name"], "r": r, "N": N, "refresh_period": tau,
+           "ms_per_step": round(ms, 4), "ssp_step_ms": round(ssp_ms, 4), "refresh_step_ms": round(refresh_ms, 3),
+           "grad_GBps": round(gb / ms / 1e6, 1), "min_bytes_frac": round(alg / ms / 1e6 / peak, 4),
+           "min_bytes_frac_ssp_only": round(alg / ssp_ms / 1e6 / peak, 4),
+           "roofline": roofline_entry(fam, r, plans[0]["step_kernel"], el, peak, peak_kind),
+           "gradient_sets": nbuf, "g_bytes_per_step": gb, "flags": flags}
+    for h in handles:
+        h.close()
+    del handles, bufs, stack
+    torch.cuda.empty_cache()
+    return out
+
+
 # ----------------------------------------------------------------------------
 # CPU baseline: the oracle as it stands, on a bounded sample
 # ----------------------------------------------------------------------------
-def cpu_baseline(workload, r, N, budget_s=12.0):
+def cpu_baseline(r, budget_s=10.0, small=False):
+    """SSP steps of the oracle on the sweep matrix at rank r, and its dense-SVD refresh on a row sample of it."""
     import numpy as np
 
     from oracle import psgd_oracle as orc
     from paper_2509_11254_b200 import synth
 
-    shapes = stack_for(workload)
-    t_used, g_bytes, nsteps = 0.0, 0, 0
-    desc = []
-    for (m, n, _c) in shapes:
-        G = synth.make_gradients(workload, m, n, N, step=1, matrix_id=0)
-        o = orc.PowerSGDPlusOracle(m, n, r, N, 0, synth.init_Q(n, r))
-        reps = 0
-        t0 = time.perf_counter()
-        while True:
-            o.step(G)
-            reps += 1
-            if time.perf_counter() - t0 > budget_s / len(shapes) or reps >= 20:
-                break
-        dt = time.perf_counter() - t0
-        t_used += dt
-        g_bytes += reps * G.nbytes
-        nsteps += reps
-        desc.append(f"{reps} SSP steps of one {m}x{n} matrix (N={N})")
-    try:
-        cores = len(os.sched_getaffinity(0))
-    except Exception:
-        cores = os.cpu_count()
-    return {"value": g_bytes / t_used / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": "; ".join(desc) + f"; r={r}; numpy float64 (OpenBLAS threads = cores)"}
+    m, n, N = SWEEP_SHAPE
+    ms_rows = 2048                 # the SSP sample: the first 2048 rows of the sweep matrix (all columns, all nodes)
+    G = synth.make_gradients(5, ms_rows, n, N, step=1)
+    o = orc.PowerSGDPlusOracle(ms_rows, n, r, N, 0, synth.init_Q(n, r))
+    o.step(G)
+    reps, t0 = 0, time.perf_counter()
+    while True:
+        o.step(G)
+        reps += 1
+        if time.perf_counter() - t0 > budget_s or reps >= 20:
+            break
+    dt = (time.perf_counter() - t0) / reps
+    val = G.nbytes / dt / 1e9
+    # refresh: svd_comp on a square row sample (n x n): the dense SVD is what the oracle's refresh costs
+    sv_rows = n if not small else n // 4
+    Gs = synth.make_gradients(5, sv_rows, n, N, step=2)
+    t1 = time.perf_counter()
+    orc.svd_comp(Gs.astype(np.float64), r)
+    svd_s = time.perf_counter() - t1
+    return {"value": val, "unit": UNIT, "cores": host_cores(), "kind": "oracle",
+            "sample": f"{reps} SSP steps (r={r}) of the first {ms_rows} rows of the {m}x{n} sweep matrix, N={N}; "
+                      f"refresh: one svd_comp (dense SVD) of a {sv_rows}x{n} row sample; numpy float64, OpenBLAS threads = cores",
+            "ssp_step_ms_sample": round(dt * 1e3, 2), "ssp_step_ms_scaled_to_full_matrix": round(dt * 1e3 * m / ms_rows, 1),
+            "refresh_ms_sample": round(svd_s * 1e3, 1)}
 
 
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    r, N, tau = DEFAULTS[args.workload]
-    r = args.rank or r
-    import numpy as np
+    import numpy as np  # noqa: F401
 
     from oracle import psgd_oracle as orc
     from paper_2509_11254_b200 import synth
 
-    shapes = stack_for(args.workload)
-    m, n, _ = shapes[0]
-    o = orc.PowerSGDPlusOracle(m, n, r, N, 0, synth.init_Q(n, r))
-    Gs = [synth.make_gradients(args.workload, m, n, N, step=s) for s in range(2)]
-    steps = max(1, min(args.steps, 50))
+    m, n, N = SWEEP_SHAPE
+    r = args.rank
+    rows = 2048
+    o = orc.PowerSGDPlusOracle(rows, n, r, N, 0, synth.init_Q(n, r))
+    Gs = [synth.make_gradients(5, rows, n, N, step=s) for s in range(2)]
+    steps = max(1, min(args.steps, 30))
     for w in range(max(1, min(args.warmup, 3))):
         o.step(Gs[w % 2])
     t0 = time.perf_counter()
@@ -189,16 +339,12 @@ def run_reference(args):
         o.step(Gs[s % 2])
     dt = time.perf_counter() - t0
     val = steps * Gs[0].nbytes / dt / 1e9
-    try:
-        cores = len(os.sched_getaffinity(0))
-    except Exception:
-        cores = os.cpu_count()
-    sample = f"each step = one SSP step of one {m}x{n} matrix (N={N}, r={r}) of workload {args.workload}"
+    sample = f"each step = one SSP step (r={r}) of the first {rows} rows of the {m}x{n} sweep matrix, N={N}"
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
             "warmup": args.warmup, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": synth.WORKLOADS[args.workload]["name"], "r": r, "N": N, "sample": sample},
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "config": {"workload": "sweep", "m": m, "n": n, "N": N, "r": r, "sample": sample},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": host_cores(), "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -207,84 +353,6 @@ def run_reference(args):
 # ----------------------------------------------------------------------------
 # GPU arm
 # ----------------------------------------------------------------------------
-def build_handles(workload, r, N, tau, device, mode, seed=1, grad_dtype="float32"):
-    from paper_2509_11254_b200 import PowerSGDPlus
-
-    return [PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=seed + i, count=c, device=device, mode=mode, grad_dtype=grad_dtype)
-            for i, (m, n, c) in enumerate(stack_for(workload))]
-
-
-def make_inputs(workload, N, device, nbuf, grad_dtype="float32"):
-    import torch
-    from paper_2509_11254_b200 import synth
-
-    bufs = []
-    for b in range(nbuf):
-        row = []
-        for (m, n, c) in stack_for(workload):
-            g = synth.make_gradients_torch(workload, m, n, N, c, step=b, device=device)
-            row.append(g.to(torch.bfloat16) if grad_dtype == "bfloat16" else g)
-        bufs.append(row)
-    return bufs
-
-
-def timed_steps(torch, stack, bufs, steps, dist_barrier):
-    """K steps of the whole stack; every step forks from and joins the current stream, where the two events are."""
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    dist_barrier()
-    torch.cuda.synchronize()
-    ev0.record()
-    for s in range(steps):
-        stack.step(bufs[s % len(bufs)])
-    ev1.record()
-    torch.cuda.synchronize()
-    dist_barrier()
-    return ev0.elapsed_time(ev1)
-
-
-def sweep_config5(torch, device, peak, mode):
-    """Workload 5: m=16384, n=4096, N=4, per-rank step and refresh latency."""
-    from paper_2509_11254_b200 import PowerSGDPlus, synth
-
-    m, n, N = 16384, 4096, 4
-    bufs = [synth.make_gradients_torch(5, m, n, N, 1, step=b, device=device) for b in range(2)]
-    out = []
-    for r in (1, 4, 16, 64, 128):
-        h = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=5, device=device, mode=mode)
-        for s in range(3):
-            h.step(bufs[s % 2])
-        steps = 10
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        ev0.record()
-        for s in range(steps):
-            h.step(bufs[s % 2])
-        ev1.record()
-        torch.cuda.synchronize()
-        ms = ev0.elapsed_time(ev1) / steps
-        h.refresh(bufs[0])
-        torch.cuda.synchronize()
-        ev0.record()
-        for s in range(2):
-            h.refresh(bufs[s % 2])
-        ev1.record()
-        torch.cuda.synchronize()
-        rms = ev0.elapsed_time(ev1) / 2
-        flags = h.last_status()
-        alg, gb = algorithmic_bytes([(m, n, 1)], r, N)
-        plan = h.plan_info()
-        path = "three-pass"
-        if mode == "deferred":
-            path = "single-pass" if plan["single_pass"] else ("two-pass" if r <= 16 else "three-pass")
-        out.append({"r": r, "kernel": path, "step_ms": round(ms, 4), "grad_GBps": round(gb / ms / 1e6, 1),
-                    "min_bytes_frac": round(alg / ms / 1e6 / peak, 4), "refresh_ms": round(rms, 3),
-                    "flags": flags})
-        h.close()
-        del h
-        torch.cuda.empty_cache()
-    return out
-
-
 def run_ours(args):
     import torch
 
@@ -296,126 +364,102 @@ def run_ours(args):
     torch.cuda.set_device(local)
     device = f"cuda:{local}"
     reps = Replicas("nccl", device)
-    barrier = reps.barrier
 
     from paper_2509_11254_b200 import synth
 
-    r, N, tau = DEFAULTS[args.workload]
-    r = args.rank or r
-    if args.refresh_period is not None:
-        tau = args.refresh_period
-    if args.no_refresh:
-        tau = 0
-    shapes = stack_for(args.workload)
+    m, n, N = SWEEP_SHAPE
+    if args.small:
+        m //= 4
     peak, peak_kind = peaks()
-    gbpe = 2 if args.grad_dtype == "bfloat16" else 4
-    alg_bytes, g_bytes = algorithmic_bytes(shapes, r, N, gbpe)
+    bufs = [synth.make_gradients_torch(5, m, n, N, 1, step=b, device=device) for b in range(2)]
+    r = args.rank
+    alg_bytes, g_bytes = algorithmic_bytes([(m, n, 1)], r, N)
 
-    nbuf = 1 if args.workload == 4 else 2
-    bufs = make_inputs(args.workload, N, device, nbuf, args.grad_dtype)
-    handles = build_handles(args.workload, r, N, tau, device, args.mode, grad_dtype=args.grad_dtype)
-    torch.cuda.synchronize()
+    # ---- headline: the step at the headline rank, on every replica, max over ranks ----
+    from paper_2509_11254_b200 import PowerSGDPlus
 
-    from paper_2509_11254_b200 import StreamedStack
-
-    stack = StreamedStack(handles, device)       # one stream per shape class
-    # warm-up (includes the t = 0 refresh when tau > 0)
+    h = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=5, device=device, mode=args.mode, single_pass=args.single_pass)
     for s in range(max(args.warmup, 3)):
-        stack.step(bufs[s % nbuf])
+        h.step(bufs[s % 2])
     torch.cuda.synchronize()
-
     sampler = ClockSampler(local)
     sampler.start()
-    l0 = sum(h.launch_count() for h in handles)
-    ms_total = timed_steps(torch, stack, bufs, args.steps, barrier)
-    l1 = sum(h.launch_count() for h in handles)
-    clocks = sampler.stop()
-    ms_total = reps.max_over_ranks(ms_total)
+    l0 = h.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps.barrier()
+    torch.cuda.synchronize()
+    ev0.record()
+    for s in range(args.steps):
+        h.step(bufs[s % 2])
+    ev1.record()
+    torch.cuda.synchronize()
+    reps.barrier()
+    ms_total = reps.max_over_ranks(ev0.elapsed_time(ev1))
+    launches = h.launch_count() - l0
     ms_step = ms_total / args.steps
-    value = reps.job_throughput(g_bytes, ms_step) / 1e9  # GB/s of gradient, all replicas
-
-    # second pass over the same number of steps with per-launch CUDA events (roofline of the dominant kernel)
-    for h in handles:
-        h.profile_begin()
-    prof_steps = min(args.steps, 20)
-    t_now = [h.t for h in handles]
-    ssp_only = [s for s in range(prof_steps)]
-    for s in ssp_only:
-        for h, g in zip(handles, bufs[s % nbuf]):
-            h.step(g)
-    fam = {}
-    for h in handles:
-        for k, (ms, ln) in h.profile_read().items():
-            a = fam.setdefault(k, [0.0, 0])
-            a[0] += ms
-            a[1] += ln
-    n_refresh = sum(1 for h, t0 in zip(handles, t_now) for s in range(prof_steps) if tau > 0 and (t0 + s) % tau == 0)
-    n_ssp = prof_steps * len(handles) - n_refresh
-    el = sum(m * n * c for m, n, c in shapes) * N
-    per_family_bytes = {"project": (8 + gbpe) * el, "backproject": 4 * el, "residual": 8 * el}
-    dom = max(("project", "backproject", "residual"), key=lambda k: fam.get(k, [0, 0])[0])
-    # a family's kernels run once per handle per step; average duration of one launch set over all handles
-    dom_ms_per_step = fam[dom][0] / prof_steps if prof_steps else float("nan")
-    ssp_frac = n_ssp / max(1, prof_steps * len(handles))
-    if dom != "project":
-        ssp_frac = 1.0  # the tail kernels run on refresh steps too
-    achieved = per_family_bytes[dom] * ssp_frac / dom_ms_per_step / 1e6 if dom_ms_per_step else None
-    plans = [h.plan_info() for h in handles]
-    single_pass = args.mode == "deferred" and all(p["single_pass"] for p in plans)
-    kernel_name = "k_fused_step" if (dom == "project" and single_pass) else "k_" + dom
-    # DRAM bytes per element of the dominant kernel from the committed ncu capture (profiles/), scaled to this
-    # workload's elements; None for kernels without a current capture
-    traffic = TRAFFIC_BYTES_PER_ELEMENT.get(kernel_name) if args.grad_dtype == "float32" else None   # captured with float32 G
-    traffic = traffic * el * ssp_frac if traffic is not None else None
-    roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak if achieved else None, "traffic": traffic, "peak_source": f"of {peak_kind}",
-                "algorithmic_bytes_per_launch_set": per_family_bytes[dom],
-                "per_family_ms_per_step": {k: round(v[0] / prof_steps, 4) for k, v in fam.items()},
-                "note": "second pass of the same steps with per-launch CUDA events on the launching stream"}
+    value = reps.job_throughput(g_bytes, ms_step) / 1e9          # GB/s of gradient, all replicas
+    # a longer look at the same step: blocks of 50 steps for at least half a second of device time
+    blocks, done = time_blocks(torch, lambda s: h.step(bufs[s % 2]), 100, min_seconds=0.5)
+    clocks = sampler.stop()
+    fam = family_profile([h], lambda s: h.step(bufs[s % 2]), 20)
+    plan = h.plan_info()
+    roofline = roofline_entry(fam, r, plan["step_kernel"], m * n * N, peak, peak_kind)
+    roofline["note"] = "dominant kernel family of the headline step; a second pass of 20 steps with per-launch CUDA events on the launching stream"
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": synth.WORKLOADS[args.workload]["name"], "matrices": [list(s) for s in shapes],
-                       "r": r, "N": N, "refresh_period": tau, "mode": args.mode,
-                       "launch_plan": [{k: p[k] for k in ("single_pass", "WC", "CS", "KC", "active_clusters")} for p in plans],
-                       "l2": "inputs (%.2f GB of G per step, 2 alternating sets) exceed L2" % (g_bytes / 1e9),
-                       "streams": len(handles), "grad_dtype": args.grad_dtype,
+            "config": {"workload": "sweep", "m": m, "n": n, "N": N, "ranks": list(SWEEP_RANKS), "headline_rank": r,
+                       "refresh_period": 0, "mode": args.mode, "single_pass": args.single_pass,
+                       "gradients": "low rank (s_k = 0.9^k, 256 terms) plus 5 % Gaussian noise, 2 alternating sets generated on the device",
+                       "l2": "inputs (%.2f GB of G and as much of E per step) exceed L2" % (g_bytes / 1e9),
                        "parallelism": "replicas" if world > 1 else "single"},
             "min_bytes_frac": alg_bytes / ms_step / 1e6 / peak,
             "min_bytes_per_step": alg_bytes,
-            "gpu_launches": l1 - l0, "clocks": clocks, "roofline": roofline}
+            "step_ms_blocks": {"median": round(statistics.median(blocks), 4), "min": round(min(blocks), 4), "blocks": len(blocks), "steps": done},
+            "gpu_launches": launches, "clocks": clocks, "roofline": roofline}
 
     if rank == 0 and not args.no_e2e:
         # end to end through the host-buffer entry point: H2D of G and D2H of (P~, Q) inside the timed region
-        e2e_steps = max(1, min(args.steps, 5))
-        Gh = [torch.empty(g.shape, dtype=g.dtype).pin_memory() for g in bufs[0]]
-        for gh, g in zip(Gh, bufs[0]):
-            gh.copy_(g)
-        Ph = [torch.empty(h.P_hat.shape, dtype=torch.float32).pin_memory() for h in handles]
-        Qh = [torch.empty(h.Q.shape, dtype=torch.float32).pin_memory() for h in handles]
-        stage = bufs[0]
-        stack.step_host(Gh, stage, Ph, Qh)
+        e2e_steps = 5
+        Gh = torch.empty(bufs[0].shape, dtype=bufs[0].dtype).pin_memory()
+        Gh.copy_(bufs[0])
+        Ph = torch.empty(h.P_hat.shape, dtype=torch.float32).pin_memory()
+        Qh = torch.empty(h.Q.shape, dtype=torch.float32).pin_memory()
+        stage = torch.empty_like(bufs[0])
+        h.step_host(Gh, stage, Ph, Qh)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         for s in range(e2e_steps):
-            stack.step_host(Gh, stage, Ph, Qh)
+            h.step_host(Gh, stage, Ph, Qh)
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) / e2e_steps
         line["e2e"] = {"value": g_bytes / dt / 1e9, "unit": UNIT, "h2d_bytes_per_step": g_bytes,
-                       "d2h_bytes_per_step": sum(p.numel() * 4 for p in Ph) + sum(q.numel() * 4 for q in Qh),
-                       "steps": e2e_steps, "ms_per_step": dt * 1e3}
-        del Gh
-
-    for h in handles:
-        h.close()
-    del handles, bufs
+                       "d2h_bytes_per_step": Ph.numel() * 4 + Qh.numel() * 4, "steps": e2e_steps, "ms_per_step": dt * 1e3}
+        del Gh, stage
+    h.close()
+    del h
     torch.cuda.empty_cache()
 
     if rank == 0 and world == 1 and not args.no_sweep:
-        line["sweep_config5"] = sweep_config5(torch, device, peak, args.mode)
+        sweep = []
+        for rr in SWEEP_RANKS:
+            pt, hh, _, _ = sweep_point(torch, device, rr, bufs, args.mode, args.single_pass, 100, 0.5, peak, peak_kind)
+            hh.close()
+            del hh
+            torch.cuda.empty_cache()
+            sweep.append(pt)
+        line["sweep"] = sweep
+    del bufs
+    torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and args.stacks != "none":
+        stacks = []
+        for w in [int(x) for x in args.stacks.split(",") if x]:
+            for (sr, sN, stau) in STACK_DEFAULTS[w]:
+                stacks.append(stack_bench(torch, device, w, sr, sN, stau, args.mode, args.single_pass, peak, peak_kind))
+        line["stacks"] = stacks
     if rank == 0 and world == 1 and not args.no_cpu:
-        line["cpu_baseline"] = cpu_baseline(args.workload if args.workload != 4 else 4, r, N)
+        line["cpu_baseline"] = cpu_baseline(r, small=args.small)
     if rank == 0:
         print(json.dumps(line))
     reps.close()

@@ -66,10 +66,11 @@ typedef enum {
                                       psgd_materialize_error produces the true residual).  Up to 8 columns the
                                       whole SSP step is then one pass over G and E, up to 16 two passes; above,
                                       and on refresh steps, the three-pass kernels run as in mode 0 */
-#define PSGD_OPT_REFRESH_ITERS 3   /* subspace iterations q of the refresh (default 20) */
+#define PSGD_OPT_REFRESH_ITERS 3   /* subspace iterations q of the refresh; 0 (default): 12 where the early sweeps run on the tensor cores, else
+                                      at most 20 with the stopping test.  The start block is [Q_{t-1} | random columns] */
 #define PSGD_OPT_REFRESH_OVERSAMPLE 4 /* extra columns of the refresh block (default max(8, r)) */
 #define PSGD_OPT_REFRESH_TC 5      /* 1 (default): the early sweeps of a refresh whose block has >= 32 columns run
-                                      on the tensor cores in TF32, the last 8 in float32; 0: float32 throughout */
+                                      on the tensor cores in TF32, the last 4 in float32; 0: float32 throughout */
 #define PSGD_OPT_POWER_STEPS 6     /* K >= 1 power steps per SSP iteration (Eq. (8)); 1 (default) is PowerSGD's single
                                       step (Eq. (9)); K > 1 runs the three-pass kernels */
 #define PSGD_OPT_REFRESH_ADAPTIVE 7 /* 1 (default): a refresh whose block has <= 48 columns stops its sweeps once the top-r
@@ -79,6 +80,12 @@ typedef enum {
 #define PSGD_OPT_GRAD_BF16 8        /* 0 (default): the gradients G are float32; 1: bfloat16 (the same [count][N][m][n] layout, 2 bytes
                                       per element), widened exactly to float32 as they are read.  The single-pass kernel then moves
                                       10 instead of 12 bytes per element; the other paths first form M = G + E in the E buffer */
+
+#define PSGD_OPT_SINGLE_PASS 9       /* which kernels serve the SSP steps of the deferred mode.  0 (default): the fastest known for the
+                                      shape (the cluster single-pass kernel up to 4 columns, the two-pass kernels from 5 to 16);
+                                      1: the cluster single-pass kernel where it applies (up to 8 columns; also bfloat16 gradients);
+                                      2: the two-pass kernels; 3: the L2-pipelined single-pass kernel where it applies (up to 16
+                                      columns, n % 4 == 0, float32 gradients).  A choice that does not apply falls back to two passes */
 
 /* buffers that psgd_debug_ptr exposes (test use only; valid until the next step) */
 #define PSGD_BUF_P_NODE 1   /* P^(i)   [count][N][m][r] */
@@ -184,7 +191,8 @@ psgd_status psgd_debug_ptr(psgd_handle* h, int which, void** ptr, size_t* bytes)
  * [6] its dynamic shared memory in bytes, [7] row chunks of the eager back-projection, [8] 1 while E
  * holds Delta_t and the residual is still pending (deferred mode), [9] 1 if that pending residual is
  * the single-pass kernel's (padded factors in place), [10] multiprocessors of the device that was
- * current when the handle was created (148 when none was visible), [11] reserved (0).
+ * current when the handle was created (148 when none was visible), [11] what ran the last
+ * step: 0 the three- or two-pass kernels, 1 the cluster single-pass kernel, 2 the L2-pipelined single-pass kernel.
  */
 psgd_status psgd_plan_info(const psgd_handle* h, int* info /*HOST*/);
 

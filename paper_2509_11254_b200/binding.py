@@ -13,6 +13,7 @@ PSGD_OPT_ERROR_FORM, PSGD_OPT_MODE, PSGD_OPT_REFRESH_ITERS, PSGD_OPT_REFRESH_OVE
 PSGD_OPT_POWER_STEPS = 6
 PSGD_OPT_REFRESH_ADAPTIVE = 7
 PSGD_OPT_GRAD_BF16 = 8
+PSGD_OPT_SINGLE_PASS = 9
 PSGD_BUF = {"P_node": 1, "Q_node": 2, "P_hat": 3, "Dbar": 4, "P_mean": 5}
 KERNEL_FAMILIES = ["project", "orth", "backproject", "residual", "refresh", "misc"]
 
@@ -93,7 +94,7 @@ class PowerSGDPlus:
 
     def __init__(self, m, n, r, N, refresh_period=0, seed=0, count=1, device="cuda:0", error_form="local",
                  mode="eager", refresh_iters=None, oversample=None, reset=True, refresh_tc=None, power_steps=None, refresh_adaptive=None,
-                 grad_dtype="float32"):
+                 grad_dtype="float32", single_pass=None):
         import torch
 
         self.torch = torch
@@ -117,6 +118,8 @@ class PowerSGDPlus:
             _check(L.psgd_set_option(h, PSGD_OPT_POWER_STEPS, int(power_steps)))
         if refresh_adaptive is not None:
             _check(L.psgd_set_option(h, PSGD_OPT_REFRESH_ADAPTIVE, int(bool(refresh_adaptive))))
+        if single_pass is not None:
+            _check(L.psgd_set_option(h, PSGD_OPT_SINGLE_PASS, {"auto": 0, "cluster": 1, "none": 2, "l2": 3}[single_pass]))
         self.grad_dtype = {"float32": torch.float32, "bfloat16": torch.bfloat16}[grad_dtype]
         if self.grad_dtype is torch.bfloat16:
             _check(L.psgd_set_option(h, PSGD_OPT_GRAD_BF16, 1))
@@ -219,7 +222,7 @@ class PowerSGDPlus:
         v = (_int * 12)()
         _check(lib().psgd_plan_info(self.h, v))
         keys = ("single_pass", "RP", "WC", "CS", "KC", "active_clusters", "smem_bytes", "S", "pending", "pending_single_pass",
-                "sm_count", "reserved")
+                "sm_count", "step_kernel")
         return dict(zip(keys, list(v)))
 
     def launch_count(self):

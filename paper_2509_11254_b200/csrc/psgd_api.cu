@@ -18,6 +18,7 @@
 #include "psgd_kernels.cuh"
 #include "psgd_fused.cuh"
 #include "psgd_gemm_tc.cuh"
+#include "psgd_stream.cuh"
 
 using namespace psgd;
 
@@ -25,6 +26,7 @@ namespace {
 
 constexpr int MAX_R = 128;
 constexpr int MAX_L = 160;  // widest refresh block
+constexpr int REFRESH_F32_TAIL = 4;   // float32-accurate sweeps that end a refresh whose early sweeps ran in TF32
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
@@ -36,6 +38,7 @@ struct Layout {
     size_t rtP, rtQ;                                          // tensor-core residual (r > 16) only
     size_t Pold, dpart;                                       // stopping test of the refresh
     size_t ptQ;                                               // tensor-core projection: split transposed Q
+    size_t sPpart, sCnt, sGram;                               // L2-pipelined single-pass kernel: per-unit partial products, counters and flags, Gram partials
 };
 
 struct ProfEvent {
@@ -57,7 +60,7 @@ struct psgd_handle {
     int64_t m, n;
     int r, N, count, tau;
     uint64_t seed;
-    int error_form = 0, mode = 0, refresh_iters = 20, oversample = -1, refresh_tc = 1, power_steps = 1, refresh_adaptive = 1;
+    int error_form = 0, mode = 0, refresh_iters = 0 /* 0: chosen from the block width */, refresh_warm = 1, oversample = -1, refresh_tc = 1, power_steps = 1, refresh_adaptive = 1;
     bool tc_ok = false;           // the refresh block is wide enough for the tensor-core sweeps
     size_t gpart_floats = 0;
     bool grad_bf16 = false;       // G arrives as bfloat16
@@ -89,6 +92,11 @@ struct psgd_handle {
     bool pending_fused = false;   // ... and the padded factors the single-pass kernel subtracts are those of that step
     bool tacc_identity = true;    // no preconditioner yet
     bool qpad_valid = false;      // padded copy of Q is current
+    // L2-pipelined single-pass kernel (psgd_stream.cuh)
+    int single_pass_kernel = 0;   // PSGD_OPT_SINGLE_PASS: 0 the fastest known for the shape, 1 cluster kernel, 2 two-pass kernels, 3 L2-pipelined kernel
+    bool stream_ok = false;       // the shape fits the L2-pipelined kernel
+    int s_nrb = 0, s_ngrp = 0, s_tpu = 0, s_csplit = 0, s_KC = 1, s_CB = 0, s_grid = -1;
+    int step_kernel = 0;          // what ran the last step: 0 three-/two-pass kernels, 1 cluster kernel, 2 L2-pipelined kernel
     int sm_count = 0;             // multiprocessors of the device that was current when the handle was created
 };
 
@@ -216,8 +224,30 @@ void plan(psgd_handle* h) {
             h->active_clusters = -1;
         }
     }
-    if (h->fused_ok) {
-        const size_t RP = h->RP, KC = h->KCmax;
+    // ---- L2-pipelined single-pass kernel: up to 16 columns, 16-byte row strides ----
+    // Which kernel serves the SSP steps of the deferred mode (PSGD_OPT_SINGLE_PASS).  Measured on a B200 (16384 x 4096, N = 4):
+    // up to 4 columns the cluster kernel is the fastest (0.76 of the 12 B/element roofline), from 5 to 16 columns the two-pass
+    // kernels are (0.57 at 8 columns against 0.48 for either single-pass kernel: both are bound by instruction issue there).
+    if (h->single_pass_kernel == 2 || (h->single_pass_kernel == 0 && h->r > 4 && !h->grad_bf16)) h->fused_ok = false;
+    h->stream_ok = h->mode == 1 && h->single_pass_kernel == 3 && h->r <= 16 && h->n % 4 == 0 && h->N <= 16 && !h->grad_bf16;
+    size_t wslots = h->fused_ok ? (size_t)h->KCmax : 0;
+    if (h->stream_ok) {
+        if (!h->fused_ok) h->RP = h->r <= 4 ? 4 : (h->r <= 8 ? 8 : 16);
+        h->s_nrb = ceil_div(h->m, SS_ROWS);
+        h->s_ngrp = ceil_div(h->s_nrb, SS_GROUP);
+        const int ntiles = ceil_div(h->n, SS_TCOLS);
+        h->s_tpu = std::min(SS_MAXTPU, ntiles);
+        h->s_csplit = ceil_div(ntiles, h->s_tpu);
+        h->s_CB = ceil_div(h->n, SS_BCOLS);
+        // row slots per (matrix, node, column block): as many as there are back-projection workers to take them
+        const int64_t pairs = (int64_t)h->count * h->N * h->s_CB;
+        const int64_t workers = (int64_t)(4 - (h->RP >= 16 ? 2 : 3)) * h->sm_count;     // 4 - stream_groups<RP>() per CTA
+        h->s_KC = (int)std::max<int64_t>(1, std::min<int64_t>(std::min(h->s_ngrp, 32), workers / pairs));
+        h->s_grid = -1;
+        wslots = std::max<size_t>(wslots, 2 * (size_t)h->s_KC);
+    }
+    if (h->fused_ok || h->stream_ok) {
+        const size_t RP = h->RP, KC = wslots;
         L.Qpad = take(cnt * n * RP * 4);
         L.Ppad = take(cnt * m * RP * 4);
         L.Qsub = take(cnt * N * n * RP * 4);
@@ -226,6 +256,11 @@ void plan(psgd_handle* h) {
         L.Wpart = take(cnt * KC * N * n * RP * 4);
         L.Cmat = take(cnt * RP * RP * 4);
         L.Cpart = take(cnt * (size_t)ceil_div(h->n, 16) * RP * RP * 8);
+    }
+    if (h->stream_ok) {
+        L.sPpart = take(cnt * (size_t)h->s_nrb * N * h->s_csplit * SS_ROWS * h->RP * 4);
+        L.sCnt = take(cnt * (size_t)h->s_nrb * 2 * 4);
+        L.sGram = take(cnt * (size_t)h->s_nrb * r * r * 8);
     }
     L.total = off;
 }
@@ -720,15 +755,29 @@ void svd(Launcher& L, psgd_handle* h, const void* G) {
     const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count, ell = h->ell;
     const int K = PSGD_K_REFRESH;
     L.force_kind = K;
+    // Sweeps.  Blocks of up to 31 columns run in float32 with the device-side stopping test, so the number is only an upper
+    // limit (20); wider blocks have no such test (their Rayleigh-Ritz step is too dear to repeat) and run 12 sweeps, the
+    // first 8 of them in TF32: measured on a 16384 x 4096 mean with a 0.9^k spectrum, 4 sweeps already bring the top-16
+    // projector within 1e-5 and 8 sweeps the energy left behind at r = 64 within 1e-9 of the optimum.
+    const int iters = h->refresh_iters > 0 ? h->refresh_iters : (h->tc_ok ? 12 : 20);
     launch_add_mean(L, G, h->grad_bf16, h->E, dbar, (size_t)m * n, N, cnt, K);
     size_t zt = (size_t)cnt * n * ell;
     L.begin(K);
     k_fill_normal<<<(unsigned)((zt + 255) / 256), 256, 0, L.st>>>(Z, zt, h->seed, 0x5eed0000ull + (uint64_t)h->t);
     L.end();
+    // Warm start: Algorithm 2 carries Q_{t-1} across the refresh, and its columns already span most of the subspace
+    // wanted (the right factor of the last compression).  They replace the first r random columns of the start block;
+    // the converged result is the same subspace, reached in fewer sweeps.
+    if (h->t > 0 && h->refresh_warm) {
+        L.begin(K);
+        k_copy_columns<<<(unsigned)(((size_t)cnt * n * r + 255) / 256), 256, 0, L.st>>>(h->Q, Z, (size_t)cnt * n, r, ell);
+        L.end();
+    }
     // Early sweeps on the tensor cores (TF32 operands): they bring the block close to the subspace, the
     // float32 sweeps that follow remove the TF32 rounding.  Needs Dbar^T and transposed copies of the blocks.
     int it0 = 0;
-    const bool tc = h->tc_ok && aligned16(dbar) && h->refresh_iters > 8;
+    const int tail32 = REFRESH_F32_TAIL;
+    const bool tc = h->tc_ok && aligned16(dbar) && iters > tail32;
     float* dbarT = tc ? (float*)(ws + h->lay.dbarT) : nullptr;
     float* Yt = tc ? (float*)(ws + h->lay.Yt) : nullptr;
     float* Zt = tc ? (float*)(ws + h->lay.Zt) : nullptr;
@@ -737,7 +786,7 @@ void svd(Launcher& L, psgd_handle* h, const void* G) {
         L.begin(K);
         k_transpose<<<dim3(ceil_div(n, 32), ceil_div(m, 32), cnt), dim3(32, 8), 0, L.st>>>(dbar, dbarT, m, n);
         L.end();
-        for (; it0 < h->refresh_iters - 8; ++it0) {
+        for (; it0 < iters - tail32; ++it0) {
             launch_gemm_tc(L, h, dbar, Zt, Y, m, ell, n, K);       // Y = Dbar Z
             launch_orth(L, h, Y, Y, m, ell, K, Yt);
             launch_gemm_tc(L, h, dbarT, Yt, Z, n, ell, m, K);      // Z = Dbar^T Y
@@ -753,7 +802,7 @@ void svd(Launcher& L, psgd_handle* h, const void* G) {
     S = ceil_div(m, rpc);
     // Rayleigh-Ritz on the current block: eigenvectors of Z^T Z = Y^T Dbar Dbar^T Y, then P~ = Y U[:, :r]
     int* done = flags + 3;                 // set on the device once the top-r basis has stopped moving
-    const bool adaptive = h->refresh_adaptive && ell <= 48 && h->refresh_iters - it0 > 6;
+    const bool adaptive = h->refresh_adaptive && ell <= 48 && iters - it0 > 6;
     const int* skip = adaptive ? done : nullptr;
     if (adaptive) cudaMemsetAsync(done, 0, 4, L.st);
     auto rayleigh_ritz = [&]() {
@@ -788,7 +837,7 @@ void svd(Launcher& L, psgd_handle* h, const void* G) {
     double* dpart = (double*)(ws + h->lay.dpart);
     double* dprev = dpart + (size_t)cnt * ceil_div(m, 64);
     int nchecks = 0;
-    for (int it = it0; it < h->refresh_iters; ++it) {
+    for (int it = it0; it < iters; ++it) {
         // Y = Dbar Z, orthonormalise;  Z = Dbar^T Y, orthonormalise
         launch_project(L, dbar, nullptr, nullptr, Z, Y, m, n, ell, 1, cnt, h->vec4, skip);
         launch_orth(L, h, Y, Y, m, ell, K, nullptr, false, skip);
@@ -797,7 +846,7 @@ void svd(Launcher& L, psgd_handle* h, const void* G) {
         L.begin(K);
         k_reduce_q<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(part, nullptr, Z, n, ell, 1, Sb, cnt, skip);
         L.end();
-        if (it + 1 == h->refresh_iters) break;
+        if (it + 1 == iters) break;
         const int swept = it - it0 + 1;
         if (adaptive && (swept <= 6 ? swept % 2 == 0 : swept % 3 == 0)) {
             rayleigh_ritz();
@@ -947,6 +996,101 @@ void fused_ssp(Launcher& L, psgd_handle* h, const void* G) {
     h->tacc_identity = false;
 }
 
+// ---- single-pass SSP-Comp step, L2-pipelined kernel (psgd_stream.cuh) ----------------
+template <int RP>
+bool launch_stream_t(Launcher& L, psgd_handle* h, StreamArgs a) {
+    void (*kern)(StreamArgs) = h->pending ? k_stream_step<RP, true> : k_stream_step<RP, false>;
+    const size_t smem = stream_smem_bytes<RP>();
+    set_smem_attr((const void*)kern, smem);
+    if (h->s_grid < 0) {     // one persistent CTA per multiprocessor, all of them resident (they wait on one another's flags)
+        int per_sm = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, SS_THREADS, smem) != cudaSuccess) { per_sm = 0; cudaGetLastError(); }
+        h->s_grid = std::min(per_sm, 1) * h->sm_count;
+    }
+    if (h->s_grid <= 0) return false;
+    const int64_t units = (int64_t)h->count * h->s_nrb * h->N * h->s_csplit;
+    const int grid = (int)std::min<int64_t>(h->s_grid, units);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(SS_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = L.st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    L.begin(PSGD_K_PROJECT);
+    cudaLaunchKernelEx(&cfg, kern, a);
+    L.end();
+    return true;
+}
+
+bool stream_ssp(Launcher& L, psgd_handle* h, const void* G) {
+    char* ws = h->ws;
+    const Layout& Y = h->lay;
+    float* Phat = (float*)(ws + Y.Phat);
+    float* Qnode = (float*)(ws + Y.Qnode);
+    float* part = (float*)(ws + Y.part);
+    double* gram = (double*)(ws + Y.sGram);
+    double* T = (double*)(ws + Y.T);
+    int* flags = (int*)(ws + Y.flags);
+    int* gate = flags + 1;
+    float* Qpad = (float*)(ws + Y.Qpad);
+    float* Ppad = (float*)(ws + Y.Ppad);
+    float* Qsub = (float*)(ws + Y.Qsub);
+    float* Tacc = (float*)(ws + Y.Tacc);
+    float* Pout = (float*)(ws + Y.Pout);
+    float* Wpart = (float*)(ws + Y.Wpart);
+    float* Cmat = (float*)(ws + Y.Cmat);
+    double* Cpart = (double*)(ws + Y.Cpart);
+    unsigned* cnts = (unsigned*)(ws + Y.sCnt);
+    const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count, RP = h->RP, nrb = h->s_nrb;
+    if (!h->qpad_valid) {   // first single-pass step after an eager one: no accumulated transform yet, Q' = Q
+        size_t tot = (size_t)cnt * n * RP;
+        L.begin(PSGD_K_MISC);
+        k_pad_rows<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(h->Q, Qpad, (size_t)cnt * n, r, RP);
+        L.end();
+        h->qpad_valid = true;
+    }
+    cudaMemsetAsync(gate, 0, 4, L.st);
+    cudaMemsetAsync(cnts, 0, (size_t)cnt * nrb * 2 * 4, L.st);
+    StreamArgs a{(const float*)G, h->E, Qpad, Qsub, Ppad, (float*)(ws + Y.sPpart), Pout, Wpart, gram, cnts, cnts + (size_t)cnt * nrb, flags,
+                 m, n, r, N, cnt, nrb, h->s_ngrp, h->s_tpu, h->s_csplit, h->s_KC, h->s_CB, h->error_form == 0 ? 1 : 0};
+    bool ok = RP == 4 ? launch_stream_t<4>(L, h, a) : (RP == 8 ? launch_stream_t<8>(L, h, a) : launch_stream_t<16>(L, h, a));
+    if (!ok) return false;
+    if (L.status != PSGD_OK) return true;
+    // P'^T P' = L L^T  ->  T'; scaled pivot^2 < 2e-2 raises the gate for the precise back-projection (as in the cluster kernel's path)
+    size_t tg = (size_t)r * r * cnt;
+    L.begin(PSGD_K_ORTH);
+    k_gram_sum<<<(unsigned)((tg + 255) / 256), 256, 0, L.st>>>(gram, r * r, nrb, cnt);
+    L.end();
+    L.begin(PSGD_K_ORTH);
+    int* defic = (int*)(ws + Y.defic);
+    k_chol<<<cnt, 256, (size_t)r * chol_ld(r) * 8, L.st>>>(gram, T, r, -nrb, flags, gate, 2e-2, defic);
+    L.end();
+    FinishPArgs fp{Pout, T, Phat, Ppad, Tacc, Tacc, m, r, RP, h->tacc_identity ? 1 : 0};
+    L.begin(PSGD_K_ORTH);
+    k_finish_p<<<dim3(ceil_div(m, 64), cnt), 256, 0, L.st>>>(fp);
+    L.end();
+    L.begin(PSGD_K_ORTH);
+    k_complete<<<cnt, 256, 0, L.st>>>(Phat, Ppad, defic, flags, m, r, RP, h->seed + (uint64_t)h->t);
+    L.end();
+    launch_back(L, h->E, Phat, part, m, n, r, N, cnt, h->rpc, h->S, h->vec4, gate);
+    const int qblocks = ceil_div(n, 16);
+    FinishQArgs fq{Wpart, part, T, Tacc, gate, Qnode, h->Q, Qpad, Qsub, Cpart, n, r, RP, N, 2 * h->s_KC, h->S, h->error_form};
+    L.begin(PSGD_K_BACKPROJECT);
+    k_finish_q<<<dim3(qblocks, cnt), 16 * RP, 0, L.st>>>(fq);
+    L.end();
+    L.begin(PSGD_K_BACKPROJECT);
+    k_sum_c<<<cnt, RP * RP, 0, L.st>>>(Cpart, Cmat, qblocks, RP);
+    L.end();
+    h->pending = true;
+    h->pending_fused = true;
+    h->tacc_identity = false;
+    return true;
+}
+
 // e_{t+1} = Delta_t - P~_t Qsub^T in place (Algorithm 2, last line), if it is still pending
 void materialize(Launcher& L, psgd_handle* h) {
     if (!h->pending) return;
@@ -973,9 +1117,20 @@ psgd_status do_step(psgd_handle* h, const void* G, float* P_hat, float* D_hat, p
     Launcher L{h, st};
     bool refresh = force || (h->tau > 0 && h->t % h->tau == 0);
     // (a bfloat16 row has to be a multiple of 16 bytes for the tensor map: n % 8 == 0)
-    if (h->mode == 1 && h->fused_ok && !refresh && aligned16(G) && h->power_steps == 1 && (!h->grad_bf16 || h->n % 8 == 0)) {
+    const bool one_pass = h->mode == 1 && !refresh && aligned16(G) && h->power_steps == 1;
+    bool done = false;
+    if (one_pass && h->stream_ok && h->s_grid != 0) {
         if (h->pending && !h->pending_fused) materialize(L, h);   // Delta_t left by a two-pass step: no padded factors for it
+        done = stream_ssp(L, h, G);
+        if (done) h->step_kernel = 2;
+    }
+    if (!done && one_pass && h->fused_ok && (!h->grad_bf16 || h->n % 8 == 0)) {
+        if (h->pending && !h->pending_fused) materialize(L, h);
         fused_ssp(L, h, G);
+        done = true;
+        h->step_kernel = 1;
+    }
+    if (done) {
         if (D_hat) {
             float* Phat = (float*)(h->ws + h->lay.Phat);
             launch_resid(L, nullptr, D_hat, Phat, h->Q, (int)h->m, (int)h->n, h->r, h->N, h->count, 0, 0, h->vec4);
@@ -984,12 +1139,15 @@ psgd_status do_step(psgd_handle* h, const void* G, float* P_hat, float* D_hat, p
         // Refresh steps and shapes outside the single-pass plan run the three-pass kernels.  In deferred mode, up to
         // 16 columns, SSP steps take two passes: the residual pass is dropped, the E buffer keeps Delta_t and the next
         // projection forms e_{t+1} = Delta_t - P~_t Q_i^T on the fly (16 instead of 24 bytes per element).
-        const bool two_pass = h->mode == 1 && !refresh && h->r <= 16 && h->power_steps == 1 && !h->grad_bf16;
-        if (!two_pass) materialize(L, h);
+        // A refresh step needs the true residual before it (SVD-Comp works on g + e), but may leave its own residual pending
+        // like any other step of that mode.
+        const bool two_pass = h->mode == 1 && h->r <= 16 && h->power_steps == 1 && !h->grad_bf16;
+        if (!two_pass || refresh) materialize(L, h);
         if (refresh) svd(L, h, G); else ssp(L, h, G);
         tail(L, h, D_hat, two_pass);
         h->tacc_identity = true;
         h->qpad_valid = false;
+        h->step_kernel = 0;
     }
     if (L.status != PSGD_OK) return L.status;
     if (P_hat) {
@@ -1029,12 +1187,13 @@ psgd_status psgd_set_option(psgd_handle* h, int option, int value) {
     switch (option) {
         case PSGD_OPT_ERROR_FORM: if (value != 0 && value != 1) return PSGD_E_INVALID; h->error_form = value; break;
         case PSGD_OPT_MODE: if (value != 0 && value != 1) return PSGD_E_INVALID; h->mode = value; break;
-        case PSGD_OPT_REFRESH_ITERS: if (value < 1 || value > 64) return PSGD_E_INVALID; h->refresh_iters = value; break;
+        case PSGD_OPT_REFRESH_ITERS: if (value < 0 || value > 64) return PSGD_E_INVALID; h->refresh_iters = value; break;
         case PSGD_OPT_REFRESH_OVERSAMPLE: if (value < 0 || value > MAX_L) return PSGD_E_INVALID; h->oversample = value; break;
         case PSGD_OPT_REFRESH_TC: if (value != 0 && value != 1) return PSGD_E_INVALID; h->refresh_tc = value; break;
         case PSGD_OPT_REFRESH_ADAPTIVE: if (value != 0 && value != 1) return PSGD_E_INVALID; h->refresh_adaptive = value; break;
         case PSGD_OPT_POWER_STEPS: if (value < 1 || value > 16) return PSGD_E_INVALID; h->power_steps = value; break;
         case PSGD_OPT_GRAD_BF16: if (value != 0 && value != 1) return PSGD_E_INVALID; h->grad_bf16 = value != 0; break;
+        case PSGD_OPT_SINGLE_PASS: if (value < 0 || value > 3) return PSGD_E_INVALID; h->single_pass_kernel = value; break;
         default: return PSGD_E_INVALID;
     }
     plan(h);
@@ -1170,9 +1329,9 @@ psgd_status psgd_debug_ptr(psgd_handle* h, int which, void** ptr, size_t* bytes)
 
 psgd_status psgd_plan_info(const psgd_handle* h, int* info) {
     if (!h || !info) return PSGD_E_NULL;
-    info[0] = h->fused_ok ? 1 : 0; info[1] = h->RP; info[2] = h->WC; info[3] = h->CS; info[4] = h->KC;
+    info[0] = (h->fused_ok || h->stream_ok) ? 1 : 0; info[1] = h->RP; info[2] = h->WC; info[3] = h->CS; info[4] = h->KC;
     info[5] = h->active_clusters; info[6] = (int)h->fused_smem; info[7] = h->S;
-    info[8] = h->pending ? 1 : 0; info[9] = (h->pending && h->pending_fused) ? 1 : 0; info[10] = h->sm_count; info[11] = 0;
+    info[8] = h->pending ? 1 : 0; info[9] = (h->pending && h->pending_fused) ? 1 : 0; info[10] = h->sm_count; info[11] = h->step_kernel;
     return PSGD_OK;
 }
 

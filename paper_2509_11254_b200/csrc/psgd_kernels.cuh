@@ -313,9 +313,9 @@ __global__ void __launch_bounds__(BP_THREADS) k_backproject(BackArgs a) {
     const float* Mb = a.M + (size_t)mat * a.rows * n;
     const float* Pb = a.Phat + (size_t)c * a.rows * r;
 
-    // Up to 8 columns of P~ the sums are kept packed in pairs of adjacent k (fma.rn.f32x2: half the FMA issue slots,
-    // measured 15-25 % faster); at 16 the extra registers cost more than the issue slots give.
-    constexpr bool PACKED = RP <= 8;
+    // The sums are kept packed in pairs of adjacent k (fma.rn.f32x2: half the FMA issue slots; measured 15-25 % faster up
+    // to 8 columns, 7 % at 16).
+    constexpr bool PACKED = RP <= 16;
     float acc[4][RP];
     f2p acc2[4][PACKED ? RP / 2 : 1];
 #pragma unroll
@@ -623,6 +623,15 @@ __global__ void __launch_bounds__(256) k_add_mean(const TG* G, float* E, float* 
             if (Dbar) Dbar[c * per_mat + e] = s / nf;
         }
     }
+}
+
+// Dst[row][k] = Src[row][k] for k < c_src: the first columns of a wider row-major block.  One thread per source entry.
+__global__ void k_copy_columns(const float* Src, float* Dst, size_t rows, int c_src, int c_dst) {
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= rows * c_src) return;
+    size_t row = idx / c_src;
+    int k = (int)(idx % c_src);
+    Dst[row * c_dst + k] = Src[idx];
 }
 
 // X = (1/N) sum_i X_i  for the small factor arrays (All-Reduce Mean of P).

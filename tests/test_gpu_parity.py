@@ -3,13 +3,13 @@
 Every comparison starts both sides from IDENTICAL state: the oracle's state is
 rounded to float32, uploaded, and the oracle continues from the rounded values.
 Tolerances (float32 path vs double oracle):
-  relative Frobenius error <= 1e-5 on P~, Q, Q_i, P_i and E
-  (E's denominator is floored at 1e-2 * ||M||_F: E = M - P~Q_i^T is a cancellation whose
-  float32 rounding error is about eps * ||M||_F ~ 1e-7 ||M||_F whatever the size of E, so a
-  relative bound of 1e-5 is only meaningful down to ||E||_F ~ 1e-2 ||M||_F);
+  relative Frobenius error <= 1e-5 on P~, Q, Q_i, P_i and E.  E = M - P~Q_i^T is a cancellation whose
+  float32 rounding error is about eps * ||M||_F whatever the size of E, so two bounds are asserted:
+  ||E_gpu - E_ref||_F <= 8 eps_float32 ||M||_F always, and the relative 1e-5 bound (no floor on the
+  denominator) wherever ||E||_F >= 1e-2 ||M||_F, which the first bound then implies;
   after a refresh: projector distance ||P~P~^T - P~_ref P~_ref^T||_F <= 1e-4 when
-  the spectrum of the node mean has a gap (sigma_r - sigma_{r+1}) / sigma_1 >= 2e-3,
-  otherwise only the residual norm ||Dbar - P~P~^T Dbar||_F must match (1e-5).
+  the spectrum of the node mean has a gap (sigma_r - sigma_{r+1}) / sigma_1 >= 2e-3;
+  always: the energy left behind, ||Dbar - P~P~^T Dbar||_F^2, within 2e-6 ||Dbar||^2 of the optimum (Eq. (6)).
 """
 import numpy as np
 import pytest
@@ -23,6 +23,8 @@ pytestmark = pytest.mark.gpu
 TOL = 1e-5
 PROJ_TOL = 1e-4
 GAP_MIN = 2e-3
+EPS32 = float(np.finfo(np.float32).eps)
+E_ABS = 8.0          # ||E_gpu - E_ref||_F <= E_ABS * eps_float32 * ||M||_F
 
 
 @pytest.fixture(scope="module")
@@ -45,7 +47,7 @@ def projector_distance(P, Pref):
     return float(np.sqrt(2.0) * np.linalg.norm(P - Pref @ (Pref.T @ P)))
 
 
-def compare_step(out, gpu, m, n, r, N, tag):
+def compare_step(out, gpu, m, n, r, N, tag, e_abs=E_ABS):
     """out: oracle dict for one matrix; gpu: dict of numpy arrays for the same matrix."""
     normM = np.linalg.norm(out["M"])
     P_ref = out["P_hat"]
@@ -55,11 +57,16 @@ def compare_step(out, gpu, m, n, r, N, tag):
         s = out["sigma"]
         gap = (s[r - 1] - (s[r] if r < len(s) else 0.0)) / s[0]
         Dbar = out["Dbar"]
+        if "Dbar" in gpu:      # node mean of Delta (SVD-Comp, first line) as the GPU formed it
+            assert rel_fro(gpu["Dbar"], Dbar) <= 1e-6, f"{tag}: Dbar {rel_fro(gpu['Dbar'], Dbar)}"
         Pg = gpu["P_hat"].astype(np.float64)
         res_g = np.linalg.norm(Dbar - Pg @ (Pg.T @ Dbar))
         res_o = np.linalg.norm(Dbar - P_ref @ (P_ref.T @ Dbar))
-        # 1e-5 relative, with an absolute floor of 1e-6 ||Dbar|| (float32 rounding of P~ itself)
-        assert abs(res_g - res_o) <= TOL * max(res_o, 0.1 * np.linalg.norm(Dbar)), f"{tag}: refresh residual"
+        # Optimality of the compressor in the terms of Eq. (6), i.e. squared norms relative to ||Dbar||^2: the energy the
+        # GPU's subspace leaves behind exceeds the optimum sum_{i>r} sigma_i^2 by at most 2e-6 ||Dbar||^2 (and, P~ being
+        # orthonormal, cannot fall below it by more than rounding).  This is the whole check when sigma_r has no gap.
+        nD2 = float(np.linalg.norm(Dbar)) ** 2
+        assert -1e-6 * nD2 <= res_g ** 2 - res_o ** 2 <= 2e-6 * nD2, f"{tag}: refresh residual {(res_g ** 2 - res_o ** 2) / nD2}"
         if gap >= GAP_MIN:
             d = projector_distance(Pg, P_ref)
             assert d <= PROJ_TOL, f"{tag}: projector distance {d} (gap {gap})"
@@ -74,17 +81,25 @@ def compare_step(out, gpu, m, n, r, N, tag):
     assert rel_fro(gpu["P_hat"], P_ref) <= TOL, f"{tag}: P~ {rel_fro(gpu['P_hat'], P_ref)}"
     assert rel_fro(gpu["Q"], out["Q"]) <= TOL, f"{tag}: Q"
     assert rel_fro(gpu["Q_node"], out["Q_i"]) <= TOL, f"{tag}: Q_i"
-    e = rel_fro(gpu["E"], out["E"], floor=1e-2 * normM)
-    assert e <= TOL, f"{tag}: E {e}"
+    check_residual(gpu["E"], out["E"], normM, tag, e_abs)
+
+
+def check_residual(E_gpu, E_ref, normM, tag, e_abs=E_ABS):
+    """The two bounds on the residual (see the module docstring)."""
+    err = float(np.linalg.norm(np.asarray(E_gpu, dtype=np.float64) - E_ref))
+    assert err <= e_abs * EPS32 * normM, f"{tag}: E off by {err / (EPS32 * normM):.2f} eps ||M||"
+    normE = float(np.linalg.norm(E_ref))
+    if normE >= 1e-2 * normM:
+        assert err <= TOL * normE, f"{tag}: E {err / normE}"
 
 
 def run_case(torch, m, n, r, N, tau, steps, workload=1, count=1, error_form="local", Einit=0.0, seed=7,
-             check_dense=False, mode="eager", power_steps=1, grad_dtype="float32"):
+             check_dense=False, mode="eager", power_steps=1, grad_dtype="float32", single_pass=None):
     from paper_2509_11254_b200 import PowerSGDPlus
 
     dev = "cuda:0"
     comp = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=seed, count=count, device=dev, error_form=error_form,
-                        mode=mode, power_steps=power_steps, grad_dtype=grad_dtype)
+                        mode=mode, power_steps=power_steps, grad_dtype=grad_dtype, single_pass=single_pass)
     rng = np.random.default_rng(seed)
     Q0 = np.stack([synth.init_Q(n, r, matrix_id=c, seed=seed) for c in range(count)])
     oracles = [orc.PowerSGDPlusOracle(m, n, r, N, tau, Q0[c], error_form, power_steps) for c in range(count)]
@@ -112,6 +127,8 @@ def run_case(torch, m, n, r, N, tau, steps, workload=1, count=1, error_form="loc
                   Q_node=comp.debug("Q_node").cpu().numpy())
         if mode == "eager" and power_steps == 1:   # (single-pass: no per-node P_i; K steps: P_i is the last round's)
             gp["P_node"] = comp.debug("P_node").cpu().numpy()
+        if tau > 0 and t % tau == 0:
+            gp["Dbar"] = comp.debug("Dbar").cpu().numpy()
         for c, o in enumerate(oracles):
             out = o.step(G[c])
             compare_step(out, {k: v[c] for k, v in gp.items()}, m, n, r, N, f"t={t} c={c}")
@@ -220,6 +237,34 @@ def test_refresh_tensor_core_sweeps(torch_cuda, m, n, r, N, workload):
     run_case(torch_cuda, m, n, r, N, tau=2, steps=3, workload=workload)
 
 
+@pytest.mark.parametrize("m,n,r,N,workload", [(1024, 512, 8, 2, 2), (1536, 1024, 32, 2, 5)])
+def test_refresh_with_few_sweeps_is_contractive(torch_cuda, m, n, r, N, workload):
+    """A refresh cut short at q = 1, 2, 4 sweeps (PSGD_OPT_REFRESH_ITERS) is no longer the SVD, but it is still a contractive
+    compressor in the sense the convergence analysis needs (Sec. 4; Eq. (6)): the energy it leaves behind stays below
+    (1 - r/n) ||Dbar||^2, it approaches the oracle's optimum sum_{i>r} sigma_i^2 as q grows, and P~ stays orthonormal."""
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    torch = torch_cuda
+    G = synth.make_gradients(workload, m, n, N, step=0)
+    Dbar = orc._mean(G.astype(np.float64))
+    sig = np.linalg.svd(Dbar, compute_uv=False)
+    nD2, opt = float(np.sum(sig ** 2)), float(np.sum(sig[r:] ** 2))
+    excess = []
+    for q in (1, 2, 4, 8):
+        comp = PowerSGDPlus(m, n, r, N, refresh_period=100, seed=5, refresh_iters=q)
+        comp.step(torch.as_tensor(G[None], device="cuda:0"))          # t = 0: a refresh
+        assert comp.last_status() == 0
+        P = comp.P_hat[0].cpu().numpy().astype(np.float64)
+        assert np.linalg.norm(P.T @ P - np.eye(r)) <= 1e-5
+        left = float(np.linalg.norm(Dbar - P @ (P.T @ Dbar)) ** 2)
+        assert left <= (1.0 - r / n) * nD2, f"q = {q}: not contractive"
+        assert left >= opt * (1.0 - 1e-6) - 1e-6 * nD2             # nothing beats the optimal compressor
+        excess.append((left - opt) / nD2)
+        comp.close()
+    assert excess[-1] <= 2e-6
+    assert excess[0] >= excess[1] - 1e-7 and excess[1] >= excess[2] - 1e-7 and excess[2] >= excess[3] - 1e-7, excess
+
+
 def test_refresh_every_step(torch_cuda):
     run_case(torch_cuda, 256, 128, 4, 4, tau=1, steps=3, workload=1)
 
@@ -277,22 +322,24 @@ def test_deferred_config1_tiny_20_steps(torch_cuda):
     run_case(torch_cuda, 256, 128, 4, 4, tau=5, steps=20, workload=1, mode="deferred")
 
 
+@pytest.mark.parametrize("single_pass", ["auto", "cluster", "l2"])
 @pytest.mark.parametrize("m,n,r,N,count,workload", [
-    (300, 200, 8, 2, 3, 2),      # one CTA per cluster, 256-column slice, ragged rows, batch of 3
-    (96, 96, 1, 5, 1, 2),        # r = 1, five nodes, 128-column slice
-    (64, 8, 8, 2, 1, 2),         # n == r
-    (513, 260, 7, 1, 1, 5),      # N = 1 (two stages per block), ragged rows, slice of 4 valid columns in the last CTA
-    (768, 768, 8, 8, 2, 2),      # cluster of 3 CTAs x 256 columns (config-2 shape)
-    (2056, 768, 8, 8, 1, 2),     # config-2 FFN shape, m % 8 == 0 with several row slots
-    (4099, 4096, 8, 4, 1, 5),    # cluster of 8 CTAs x 512 columns (config-5 columns), last block has 3 valid rows
-    (2054, 2048, 4, 8, 1, 4),    # cluster of 8 CTAs x 256 columns (config-4 columns), r = 4
-    (784, 768, 4, 16, 1, 3),     # 16 nodes: cluster of 6 CTAs x 128 columns
-    (1004, 1000, 6, 4, 2, 2),    # n not a multiple of the slice: padded columns, last row chunk empty
-    (513, 260, 16, 1, 1, 5),     # r = 16: outside the single-pass plan, runs the eager kernels
+    (300, 200, 8, 2, 3, 2),      # ragged rows and columns (7 tiles of 32 columns, the last with 8), batch of 3
+    (96, 96, 1, 5, 1, 2),        # r = 1, five nodes, a single row block
+    (64, 8, 8, 2, 1, 2),         # n == r: one tile with 8 valid columns
+    (513, 260, 7, 1, 1, 5),      # N = 1, ragged rows (5 row blocks, one valid row in the last), 9 tiles -> 2 column splits
+    (768, 768, 8, 8, 2, 2),      # config-2 attention shape: 3 column splits of 8 tiles (cluster kernel: 3 CTAs x 256 columns)
+    (2056, 768, 8, 8, 1, 2),     # config-2 FFN shape plus a ragged row block
+    (4099, 4096, 8, 4, 1, 5),    # config-5 columns: 16 column splits, 16 column blocks per node, last block has 3 valid rows
+    (2054, 2048, 4, 8, 1, 4),    # config-4 columns, r = 4
+    (784, 768, 4, 16, 1, 3),     # 16 nodes
+    (1004, 1000, 6, 4, 2, 2),    # n not a multiple of 32: last tile holds 8 columns
+    (513, 260, 16, 1, 1, 5),     # r = 16 (L2-pipelined kernel only; with it switched off: the two-pass kernels)
+    (1100, 516, 12, 3, 2, 2),    # 12 -> 16 columns, 3 nodes, 17 tiles -> 3 column splits, the last with one tile
     (130, 66, 5, 2, 2, 2),       # n % 4 != 0: falls back to the eager kernels
 ])
-def test_deferred_step_by_step(torch_cuda, m, n, r, N, count, workload):
-    run_case(torch_cuda, m, n, r, N, tau=0, steps=3, workload=workload, count=count, Einit=0.01, mode="deferred")
+def test_deferred_step_by_step(torch_cuda, m, n, r, N, count, workload, single_pass):
+    run_case(torch_cuda, m, n, r, N, tau=0, steps=3, workload=workload, count=count, Einit=0.01, mode="deferred", single_pass=single_pass)
 
 
 def test_deferred_mean_error_form(torch_cuda):
@@ -364,16 +411,32 @@ def test_gemm_nt_tf32_matches_definition(torch_cuda, M, Nc, K, count):
 
 
 # ---- full-size workloads in the benchmark's launch configuration, checked on sampled matrices ----
-def _full_size_case(torch, workload, m, n, r, N, count, tau, sample, free_steps, free_check=True):
+def _implied_residual(comp, c):
+    """The residual the GPU state stands for, in double: E itself, or, while a deferred step's residual is
+    still pending, e = Delta - P~ Q_i^T from the stored Delta and the factors of that step (Algorithm 2, last line)."""
+    E = comp.E[c].cpu().numpy().astype(np.float64)
+    if comp.plan_info()["pending"]:
+        P = comp.P_hat[c].cpu().numpy().astype(np.float64)
+        Qn = comp.debug("Q_node")[c].cpu().numpy().astype(np.float64)
+        for i in range(E.shape[0]):
+            E[i] -= P @ Qn[i].T
+    return E
+
+
+def _full_size_case(torch, workload, m, n, r, N, count, tau, sample, free_steps, free_check=True, expect_pending=None,
+                    single_pass=None):
     """Deferred mode as bench.py runs it: free-running steps against the oracle on the sampled
     matrices (rotation-invariant outputs, 1e-3), then one more step from identical state (1e-5).
+    The GPU is NOT asked to materialise its residual in between: the oracle takes over the state the GPU
+    holds (stored Delta, P~ and Q_i of the last step -> e in double on the host, and Q), so the step that is
+    compared is the steady-state one, with the pending residual folded into its first pass.
     free_check=False skips the free-running comparison: without a spectral gap at r (directions r, r+1
     both at the noise floor) two correct runs may keep different tail directions, so only the step from
     identical state is a well-posed comparison."""
     from paper_2509_11254_b200 import PowerSGDPlus
 
     dev = "cuda:0"
-    comp = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=3, count=count, device=dev, mode="deferred")
+    comp = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=3, count=count, device=dev, mode="deferred", single_pass=single_pass)
     Q0 = comp.Q.cpu().numpy()
     oracles = {c: orc.PowerSGDPlusOracle(m, n, r, N, tau, Q0[c]) for c in sample}
     out = {}
@@ -383,20 +446,24 @@ def _full_size_case(torch, workload, m, n, r, N, count, tau, sample, free_steps,
         for c in sample:
             out[c] = oracles[c].step(G[c].cpu().numpy())
         del G
-    comp.materialize_error()
     assert comp.last_status() == 0
-    for c in sample if free_check else ():
-        normM = np.linalg.norm(out[c]["M"])
-        assert projector_distance(comp.P_hat[c].cpu().numpy(), out[c]["P_hat"]) <= 1e-3, f"matrix {c}: projector"
-        assert rel_fro(comp.E[c].cpu().numpy(), out[c]["E"], floor=1e-2 * normM) <= 1e-3, f"matrix {c}: residual"
-    # one step from identical state: the oracle continues from the GPU's float32 state
+    plan = comp.plan_info()
+    if expect_pending is not None:
+        assert plan["pending"] == int(expect_pending), plan
     t = free_steps
     for c in sample:
-        oracles[c].E = comp.E[c].cpu().numpy().astype(np.float64)
+        e = _implied_residual(comp, c)
+        if free_check:
+            normM = np.linalg.norm(out[c]["M"])
+            assert projector_distance(comp.P_hat[c].cpu().numpy(), out[c]["P_hat"]) <= 1e-3, f"matrix {c}: projector"
+            assert rel_fro(e, out[c]["E"], floor=1e-2 * normM) <= 1e-3, f"matrix {c}: residual"
+        # one step from identical state: the oracle continues from the state the GPU holds
+        oracles[c].E = e
         oracles[c].Q = comp.Q[c].cpu().numpy().astype(np.float64)
         oracles[c].t = t
     G = synth.make_gradients_torch(workload, m, n, N, count, step=t, device=dev)
     comp.step(G)
+    plan = comp.plan_info()
     comp.materialize_error()
     assert comp.last_status() == 0
     Qn = comp.debug("Q_node")
@@ -405,28 +472,115 @@ def _full_size_case(torch, workload, m, n, r, N, count, tau, sample, free_steps,
         gp = dict(P_hat=comp.P_hat[c].cpu().numpy(), Q=comp.Q[c].cpu().numpy(), E=comp.E[c].cpu().numpy(),
                   Q_node=Qn[c].cpu().numpy())
         compare_step(o, gp, m, n, r, N, f"full size, matrix {c}")
-    plan = comp.plan_info()
     comp.close()
     return plan
 
 
+def _full_size_refresh(torch, workload, m, n, r, N, count, sample, svd_cache=None, refresh_iters=None):
+    """SVD-Comp at full size from identical state: t = 0 of a fresh handle (E = 0), the step psgd_refresh times in the
+    benchmark.  The oracle's dense SVD of the node mean runs once per sampled matrix (svd_cache keeps U, sigma per
+    matrix so that several ranks of the same workload share it: at t = 0 with E = 0 the node mean does not depend on r).
+    With a spectral gap at r: projector <= 1e-4, Q after alignment, E, and Dbar itself; without one: the residual norm of
+    Eq. (6), which every basis of a correct top-r subspace attains."""
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    dev = "cuda:0"
+    comp = PowerSGDPlus(m, n, r, N, refresh_period=1000, seed=3, count=count, device=dev, mode="deferred", refresh_iters=refresh_iters)
+    G = synth.make_gradients_torch(workload, m, n, N, count, step=0, device=dev)
+    comp.step(G)                       # t = 0: a refresh
+    comp.materialize_error()
+    assert comp.last_status() == 0
+    Dbar_g = comp.debug("Dbar")
+    Qn = comp.debug("Q_node")
+    for c in sample:
+        Gc = G[c].cpu().numpy().astype(np.float64)
+        Dbar = orc._mean(Gc)
+        if svd_cache is not None and c in svd_cache:
+            U, sig = svd_cache[c]
+        else:
+            U, sig = orc.svd_top_r(Dbar, min(n, 160))
+            if svd_cache is not None:
+                svd_cache[c] = (U, sig)
+        P_ref = U[:, :r]
+        tail_ = orc._tail(P_ref, Gc)
+        o = dict(refresh=True, sigma=sig, Dbar=Dbar, P_hat=P_ref, M=Gc, Q=tail_["Q"], Q_i=tail_["Q_i"], E=Gc - tail_["Dhat_i"])
+        gp = dict(P_hat=comp.P_hat[c].cpu().numpy(), Q=comp.Q[c].cpu().numpy(), E=comp.E[c].cpu().numpy(),
+                  Q_node=Qn[c].cpu().numpy(), Dbar=Dbar_g[c].cpu().numpy())
+        compare_step(o, gp, m, n, r, N, f"full-size refresh, matrix {c}, r = {r}")
+    comp.close()
+
+
+@pytest.mark.parametrize("single_pass", ["auto", "cluster", "none", "l2"])
+@pytest.mark.parametrize("m,n,r,N,count,workload", [
+    (520, 256, 8, 4, 2, 2),
+    (1100, 516, 4, 3, 2, 2),
+    (1040, 1024, 16, 4, 1, 5),     # r = 16: the cluster kernel does not take it (two-pass kernels instead)
+])
+def test_pending_step_from_identical_state(torch_cuda, m, n, r, N, count, workload, single_pass):
+    """The steady-state step of the deferred mode at 1e-5: three free steps, then the oracle takes over the state the GPU
+    holds WITHOUT the GPU materialising its residual, and the next step (pending residual folded into the first pass) is
+    compared.  For each of the ways the deferred mode runs an SSP step (cluster single-pass kernel, two-pass kernels,
+    L2-pipelined single-pass kernel, and the default choice among them)."""
+    plan = _full_size_case(torch_cuda, workload, m, n, r, N, count, tau=0, sample=tuple(range(count)), free_steps=3,
+                           expect_pending=True, single_pass=single_pass)
+    want = {"auto": 1 if r <= 4 else 0, "cluster": 1 if r <= 8 else 0, "none": 0, "l2": 2}[single_pass]
+    assert plan["step_kernel"] == want
+
+
 def test_full_size_config2_attention_class(torch_cuda):
     """Workload 2, the 48 matrices of 768 x 768 (r = 8, N = 8, refresh at t = 0), three sampled."""
-    plan = _full_size_case(torch_cuda, 2, 768, 768, 8, 8, 48, tau=50, sample=(0, 17, 47), free_steps=4)
-    assert plan["single_pass"] == 1 and plan["CS"] == 3 and plan["WC"] == 256
+    plan = _full_size_case(torch_cuda, 2, 768, 768, 8, 8, 48, tau=50, sample=(0, 17, 47), free_steps=4, expect_pending=True)
+    assert plan["step_kernel"] == 0        # r = 8: the two-pass kernels are the default
 
 
 def test_full_size_config2_ffn_class(torch_cuda):
     """Workload 2, the 36 matrices of 2048 x 768, two sampled."""
-    plan = _full_size_case(torch_cuda, 2, 2048, 768, 8, 8, 36, tau=50, sample=(5, 35), free_steps=3)
-    assert plan["single_pass"] == 1
+    plan = _full_size_case(torch_cuda, 2, 2048, 768, 8, 8, 36, tau=50, sample=(5, 35), free_steps=3, expect_pending=True)
+    assert plan["step_kernel"] == 0
 
 
-@pytest.mark.parametrize("r", [4, 8])
+def test_full_size_config2_l2_pipelined_kernel(torch_cuda):
+    """The FFN class of workload 2 through the L2-pipelined single-pass kernel."""
+    plan = _full_size_case(torch_cuda, 2, 2048, 768, 8, 8, 36, tau=50, sample=(9,), free_steps=3, expect_pending=True, single_pass="l2")
+    assert plan["step_kernel"] == 2
+
+
+def test_full_size_config2_cluster_kernel(torch_cuda):
+    """The attention class through the cluster single-pass kernel (3 CTAs x 256 columns per cluster)."""
+    plan = _full_size_case(torch_cuda, 2, 768, 768, 8, 8, 48, tau=50, sample=(3,), free_steps=3, expect_pending=True, single_pass="cluster")
+    assert plan["step_kernel"] == 1 and plan["CS"] == 3 and plan["WC"] == 256
+
+
+@pytest.mark.parametrize("m,n,count,sample", [(768, 768, 48, (0, 31)), (2048, 768, 36, (20,))])
+@pytest.mark.parametrize("r", [4, 16])
+def test_full_size_config3(torch_cuda, m, n, count, sample, r):
+    """Workload 3: the same stack on 16 nodes whose top-8 left subspaces differ, r = 4 and r = 16, both shape classes."""
+    plan = _full_size_case(torch_cuda, 3, m, n, r, 16, count, tau=20, sample=sample, free_steps=3, expect_pending=True)
+    assert plan["step_kernel"] == (1 if r <= 4 else 0)
+    if r <= 4:
+        assert plan["CS"] == 6 and plan["WC"] == 128          # 16 nodes: 6 CTAs x 128 columns per cluster
+
+
+def test_full_size_config3_l2_pipelined_kernel(torch_cuda):
+    """Workload 3 at r = 16 through the L2-pipelined single-pass kernel (16 nodes, 3 column splits per row block)."""
+    plan = _full_size_case(torch_cuda, 3, 768, 768, 16, 16, 48, tau=20, sample=(7,), free_steps=3, expect_pending=True, single_pass="l2")
+    assert plan["step_kernel"] == 2
+
+
+@pytest.mark.parametrize("r", [1, 4, 8, 16])
 def test_full_size_config5(torch_cuda, r):
     """Workload 5: one 16384 x 4096 matrix on 4 nodes, plain PowerSGD steps (the step the sweep times)."""
-    plan = _full_size_case(torch_cuda, 5, 16384, 4096, r, 4, 1, tau=0, sample=(0,), free_steps=3)
-    assert plan["single_pass"] == 1 and plan["CS"] == 8 and plan["WC"] == 512
+    plan = _full_size_case(torch_cuda, 5, 16384, 4096, r, 4, 1, tau=0, sample=(0,), free_steps=3, expect_pending=True)
+    assert plan["step_kernel"] == (1 if r <= 4 else 0)
+    if r <= 4:
+        assert plan["CS"] == 8 and plan["WC"] == 512
+
+
+@pytest.mark.parametrize("r,single_pass", [(8, "cluster"), (8, "l2"), (16, "l2")])
+def test_full_size_config5_single_pass_kernels(torch_cuda, r, single_pass):
+    """The same workload through the single-pass kernels that are not the default at these ranks."""
+    plan = _full_size_case(torch_cuda, 5, 16384, 4096, r, 4, 1, tau=0, sample=(0,), free_steps=3, expect_pending=True, single_pass=single_pass)
+    assert plan["step_kernel"] == {"cluster": 1, "l2": 2}[single_pass]
 
 
 @pytest.mark.parametrize("r", [64, 128])
@@ -437,6 +591,27 @@ def test_full_size_config5_high_rank(torch_cuda, r):
     SSP step from identical state."""
     plan = _full_size_case(torch_cuda, 5, 16384, 4096, r, 4, 1, tau=100, sample=(0,), free_steps=2, free_check=False)
     assert plan["single_pass"] == 0
+
+
+_SVD_CACHE_W5 = {}
+
+
+@pytest.mark.parametrize("r", [1, 4, 16, 64, 128])
+def test_full_size_config5_refresh(torch_cuda, r):
+    """SVD-Comp of the 16384 x 4096 node mean at every rank of the sweep, against the oracle's dense SVD.  Gaps of the
+    generated spectrum at r = 1, 4, 16: about 0.1, 0.07, 0.02 (projector bound applies); r = 64, 128 sit in the noise
+    floor (residual-norm identity of Eq. (6))."""
+    _full_size_refresh(torch_cuda, 5, 16384, 4096, r, 4, 1, sample=(0,), svd_cache=_SVD_CACHE_W5)
+
+
+@pytest.mark.parametrize("workload,m,n,r,N,count,sample", [
+    (2, 768, 768, 8, 8, 48, (0, 47)), (2, 2048, 768, 8, 8, 36, (11,)),
+    (3, 768, 768, 4, 16, 48, (5,)), (3, 2048, 768, 16, 16, 36, (2,)),
+    (4, 2048, 2048, 32, 8, 96, (95,)), (4, 5504, 2048, 32, 8, 72, (0,)),
+])
+def test_full_size_stack_refresh(torch_cuda, workload, m, n, r, N, count, sample):
+    """The t = 0 refresh of the stacks (workloads 2, 3, 4) at full size from identical state."""
+    _full_size_refresh(torch_cuda, workload, m, n, r, N, count, sample=sample)
 
 
 def test_full_size_config4_attention_class(torch_cuda):
@@ -490,7 +665,7 @@ def test_msgd_update_after_the_step(torch_cuda, m, n, r, mode):
     (333, 130, 5, 2, 1, "local"),      # n % 4 != 0: outside the single-pass plan, scalar loads
 ])
 def test_two_pass_deferred_equals_three_pass(torch_cuda, m, n, r, N, count, form):
-    """Deferred mode outside the single-pass plan (r in 9..16, or n % 4 != 0): the residual pass is dropped and the
+    """Deferred mode with the single-pass kernels switched off (what also serves n % 4 != 0): the residual pass is dropped and the
     next projection forms e = Delta - P~ Q_i^T on the fly with the same float32 operations in the same order, so
     free-running steps (with a refresh among them) equal the three-pass mode bit for bit."""
     from paper_2509_11254_b200 import PowerSGDPlus
@@ -498,7 +673,7 @@ def test_two_pass_deferred_equals_three_pass(torch_cuda, m, n, r, N, count, form
     torch = torch_cuda
     out = {}
     for mode in ("eager", "deferred"):
-        comp = PowerSGDPlus(m, n, r, N, refresh_period=4, seed=9, count=count, mode=mode, error_form=form)
+        comp = PowerSGDPlus(m, n, r, N, refresh_period=4, seed=9, count=count, mode=mode, error_form=form, single_pass="none")
         for t in range(7):
             G = synth.make_gradients_torch(2, m, n, N, count, step=t, device="cuda:0")
             comp.step(G)
@@ -521,7 +696,7 @@ def test_two_pass_deferred_dense_output_and_state_reset(torch_cuda):
     m, n, r, N = 520, 256, 12, 3
     res = {}
     for mode in ("eager", "deferred"):
-        comp = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=4, mode=mode)
+        comp = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=4, mode=mode, single_pass="none")
         Dh = torch.empty((1, m, n), dtype=torch.float32, device="cuda:0")
         outs = []
         for t in range(5):
@@ -536,12 +711,6 @@ def test_two_pass_deferred_dense_output_and_state_reset(torch_cuda):
         comp.close()
     for a, b in zip(res["eager"], res["deferred"]):
         assert torch.equal(a, b)
-
-
-def test_full_size_config5_rank16_two_pass(torch_cuda):
-    """Workload 5 at r = 16 in deferred mode: projection with the on-the-fly residual and back-projection only."""
-    plan = _full_size_case(torch_cuda, 5, 16384, 4096, 16, 4, 1, tau=0, sample=(0,), free_steps=3)
-    assert plan["single_pass"] == 0
 
 
 @pytest.mark.parametrize("grad_dtype", ["float32", "bfloat16"])
@@ -675,4 +844,6 @@ def test_ill_conditioned_projection_takes_the_precise_path(torch_cuda):
     out = o.step(G)
     gp = dict(P_hat=comp.P_hat[0].cpu().numpy(), Q=comp.Q[0].cpu().numpy(), E=comp.E[0].cpu().numpy(),
               Q_node=comp.debug("Q_node")[0].cpu().numpy())
-    compare_step(out, gp, m, n, r, N, "ill-conditioned Q")
+    # (columns 2 and 3 of P = M Q are 0.02 apart in angle: the float32 rounding of P is amplified by 1 / 0.02 in P~, so the
+    #  absolute bound on E is widened by that factor's share; the 1e-5 bounds on P~, Q and Q_i are not)
+    compare_step(out, gp, m, n, r, N, "ill-conditioned Q", e_abs=32.0)

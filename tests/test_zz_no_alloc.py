@@ -6,7 +6,11 @@ stall the device), so `psgd_backproject_static` keeps its partial sums in a fixe
 inside the library instead of a caller-provided workspace.  This file checks, through
 the C ABI, that it returns what `psgd_step` computes for the same inputs: Q_i = M_i^T P~
 per node and their mean, twice in a row (the second call finds the first call's
-leftovers in the shared array), and that oversized problems are refused.
+leftovers in the shared array), and that oversized problems are refused.  Because the
+two entry points share their kernels, the result is also compared with M_i^T P~ and its
+node mean evaluated in double precision on the host.  The shapes include one where the
+fixed array, not the GPU's size, limits the number of row chunks, and one with more
+than 16 columns (several column chunks per launch).
 
 Collected last on purpose (file name), and independent of every other test.
 """
@@ -40,7 +44,9 @@ def test_static_backprojection_matches_step_twice_in_a_row():
         pytest.skip("no CUDA device")
     from paper_2509_11254_b200.binding import backproject_static
 
-    problems = [(1024, 512, 8, 4, 21), (300, 130, 5, 3, 22), (1024, 512, 8, 4, 21)]
+    # (m, n, r, N, seed).  4096 x 1024, r = 16, N = 16: one row chunk of partial sums is 1 MiB, so the 8 MiB array allows
+    # 8 chunks where the GPU alone would get 19; r = 24: two column chunks of 16
+    problems = [(1024, 512, 8, 4, 21), (300, 130, 5, 3, 22), (4096, 1024, 16, 16, 23), (640, 256, 24, 2, 24), (1024, 512, 8, 4, 21)]
     prepared = [_step_outputs(torch, *p) for p in problems]
     # back-to-back calls on one stream: each finds the previous call's partial sums in the array
     results = []
@@ -50,9 +56,14 @@ def test_static_backprojection_matches_step_twice_in_a_row():
         backproject_static(G, P_hat, Qm, Qn)
         results.append((Qn, Qm))
     torch.cuda.synchronize()
-    for (Qn, Qm), (_, _, Qn_ref, Qm_ref) in zip(results, prepared):
+    for (Qn, Qm), (G, P_hat, Qn_ref, Qm_ref) in zip(results, prepared):
         assert rel_fro(Qn.cpu().numpy(), Qn_ref.cpu().numpy()) <= TOL
         assert rel_fro(Qm.cpu().numpy(), Qm_ref.cpu().numpy()) <= TOL
+        # the definition, in double on the host: Q_i = M_i^T P~, Q = (1/N) sum_i Q_i
+        M64, P64 = G.cpu().numpy().astype(np.float64), P_hat.cpu().numpy().astype(np.float64)
+        Q64 = np.stack([M64[i].T @ P64 for i in range(M64.shape[0])])
+        assert rel_fro(Qn.cpu().numpy(), Q64) <= TOL
+        assert rel_fro(Qm.cpu().numpy(), Q64.mean(axis=0)) <= TOL
     # Q_node is optional
     G, P_hat, _, Qm_ref = prepared[0]
     Qm = torch.empty_like(Qm_ref)
