@@ -40,7 +40,7 @@ SWEEP_RANKS = (1, 4, 8, 16, 64, 128)
 HEADLINE_RANK = 16
 # dram__bytes_read.sum + dram__bytes_write.sum per element of one launch, from the ncu captures summarised under
 # profiles/ (small case of the same kernel; traffic grows in proportion to the elements).  None: no current capture.
-TRAFFIC_BYTES_PER_ELEMENT = {"k_fused_step": 11.87}
+TRAFFIC_BYTES_PER_ELEMENT = {"k_fused_step": 11.87, "k_project": 11.4, "k_backproject": 4.1, "k_stream_step": 13.6}
 
 # (rank, nodes, refresh period) of the stacks
 STACK_DEFAULTS = {2: [(8, 8, 50)], 3: [(4, 16, 20), (16, 16, 20)], 4: [(32, 8, 100)]}
@@ -59,6 +59,7 @@ def parse():
     ap.add_argument("--no-sweep", action="store_true", help="only the headline rank")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--refresh-period", type=int, default=0, help="refresh period tau of the headline handle (0: SSP steps only, as the metric asks)")
     ap.add_argument("--small", action="store_true", help="a quarter of the sweep matrix (m = 4096): for profiler captures")
     return ap.parse_args()
 
@@ -292,7 +293,7 @@ def cpu_baseline(r, budget_s=10.0, small=False):
     from paper_2509_11254_b200 import synth
 
     m, n, N = SWEEP_SHAPE
-    ms_rows = 2048                 # the SSP sample: the first 2048 rows of the sweep matrix (all columns, all nodes)
+    ms_rows = n                    # the SSP sample: a square (n x n) row sample of the sweep matrix, all nodes (the method needs m >= n)
     G = synth.make_gradients(5, ms_rows, n, N, step=1)
     o = orc.PowerSGDPlusOracle(ms_rows, n, r, N, 0, synth.init_Q(n, r))
     o.step(G)
@@ -311,7 +312,7 @@ def cpu_baseline(r, budget_s=10.0, small=False):
     orc.svd_comp(Gs.astype(np.float64), r)
     svd_s = time.perf_counter() - t1
     return {"value": val, "unit": UNIT, "cores": host_cores(), "kind": "oracle",
-            "sample": f"{reps} SSP steps (r={r}) of the first {ms_rows} rows of the {m}x{n} sweep matrix, N={N}; "
+            "sample": f"{reps} SSP steps (r={r}) of a {ms_rows}x{n} row sample of the {m}x{n} sweep matrix, N={N}; "
                       f"refresh: one svd_comp (dense SVD) of a {sv_rows}x{n} row sample; numpy float64, OpenBLAS threads = cores",
             "ssp_step_ms_sample": round(dt * 1e3, 2), "ssp_step_ms_scaled_to_full_matrix": round(dt * 1e3 * m / ms_rows, 1),
             "refresh_ms_sample": round(svd_s * 1e3, 1)}
@@ -328,10 +329,10 @@ def run_reference(args):
 
     m, n, N = SWEEP_SHAPE
     r = args.rank
-    rows = 2048
+    rows = n                       # a square row sample: the method needs m >= n
     o = orc.PowerSGDPlusOracle(rows, n, r, N, 0, synth.init_Q(n, r))
     Gs = [synth.make_gradients(5, rows, n, N, step=s) for s in range(2)]
-    steps = max(1, min(args.steps, 30))
+    steps = max(1, min(args.steps, 20))
     for w in range(max(1, min(args.warmup, 3))):
         o.step(Gs[w % 2])
     t0 = time.perf_counter()
@@ -339,7 +340,7 @@ def run_reference(args):
         o.step(Gs[s % 2])
     dt = time.perf_counter() - t0
     val = steps * Gs[0].nbytes / dt / 1e9
-    sample = f"each step = one SSP step (r={r}) of the first {rows} rows of the {m}x{n} sweep matrix, N={N}"
+    sample = f"each step = one SSP step (r={r}) of a {rows}x{n} row sample of the {m}x{n} sweep matrix, N={N}"
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
             "warmup": args.warmup, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -378,7 +379,7 @@ def run_ours(args):
     # ---- headline: the step at the headline rank, on every replica, max over ranks ----
     from paper_2509_11254_b200 import PowerSGDPlus
 
-    h = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=5, device=device, mode=args.mode, single_pass=args.single_pass)
+    h = PowerSGDPlus(m, n, r, N, refresh_period=args.refresh_period, seed=5, device=device, mode=args.mode, single_pass=args.single_pass)
     for s in range(max(args.warmup, 3)):
         h.step(bufs[s % 2])
     torch.cuda.synchronize()
@@ -399,9 +400,10 @@ def run_ours(args):
     ms_step = ms_total / args.steps
     value = reps.job_throughput(g_bytes, ms_step) / 1e9          # GB/s of gradient, all replicas
     # a longer look at the same step: blocks of 50 steps for at least half a second of device time
-    blocks, done = time_blocks(torch, lambda s: h.step(bufs[s % 2]), 100, min_seconds=0.5)
+    # (--small is the profiler's case: no more launches than needed)
+    blocks, done = time_blocks(torch, lambda s: h.step(bufs[s % 2]), 100, min_seconds=0.5) if not args.small else ([ms_step], args.steps)
     clocks = sampler.stop()
-    fam = family_profile([h], lambda s: h.step(bufs[s % 2]), 20)
+    fam = family_profile([h], lambda s: h.step(bufs[s % 2]), 20 if not args.small else 2)
     plan = h.plan_info()
     roofline = roofline_entry(fam, r, plan["step_kernel"], m * n * N, peak, peak_kind)
     roofline["note"] = "dominant kernel family of the headline step; a second pass of 20 steps with per-launch CUDA events on the launching stream"
@@ -410,7 +412,7 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": "sweep", "m": m, "n": n, "N": N, "ranks": list(SWEEP_RANKS), "headline_rank": r,
-                       "refresh_period": 0, "mode": args.mode, "single_pass": args.single_pass,
+                       "refresh_period": args.refresh_period, "mode": args.mode, "single_pass": args.single_pass,
                        "gradients": "low rank (s_k = 0.9^k, 256 terms) plus 5 % Gaussian noise, 2 alternating sets generated on the device",
                        "l2": "inputs (%.2f GB of G and as much of E per step) exceed L2" % (g_bytes / 1e9),
                        "parallelism": "replicas" if world > 1 else "single"},

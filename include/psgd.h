@@ -82,7 +82,8 @@ typedef enum {
                                       10 instead of 12 bytes per element; the other paths first form M = G + E in the E buffer */
 
 #define PSGD_OPT_SINGLE_PASS 9       /* which kernels serve the SSP steps of the deferred mode.  0 (default): the fastest known for the
-                                      shape (the cluster single-pass kernel up to 4 columns, the two-pass kernels from 5 to 16);
+                                      shape (the cluster single-pass kernel up to 4 columns, and up to 8 where its clusters have at most 4 CTAs;
+                                      the two-pass kernels otherwise);
                                       1: the cluster single-pass kernel where it applies (up to 8 columns; also bfloat16 gradients);
                                       2: the two-pass kernels; 3: the L2-pipelined single-pass kernel where it applies (up to 16
                                       columns, n % 4 == 0, float32 gradients).  A choice that does not apply falls back to two passes */

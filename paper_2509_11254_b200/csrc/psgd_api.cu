@@ -225,10 +225,12 @@ void plan(psgd_handle* h) {
         }
     }
     // ---- L2-pipelined single-pass kernel: up to 16 columns, 16-byte row strides ----
-    // Which kernel serves the SSP steps of the deferred mode (PSGD_OPT_SINGLE_PASS).  Measured on a B200 (16384 x 4096, N = 4):
-    // up to 4 columns the cluster kernel is the fastest (0.76 of the 12 B/element roofline), from 5 to 16 columns the two-pass
-    // kernels are (0.57 at 8 columns against 0.48 for either single-pass kernel: both are bound by instruction issue there).
-    if (h->single_pass_kernel == 2 || (h->single_pass_kernel == 0 && h->r > 4 && !h->grad_bf16)) h->fused_ok = false;
+    // Which kernel serves the SSP steps of the deferred mode (PSGD_OPT_SINGLE_PASS).  Measured on a B200: up to 4 columns the
+    // cluster kernel is the fastest everywhere (0.76 of the 12 B/element roofline on 16384 x 4096, N = 4).  From 5 to 8
+    // columns it still is where its clusters are small enough to fill the chip (3 CTAs for n = 768: 2.06 against 2.21 ms per
+    // step of the 130M-shaped stack), while with clusters of more than 4 CTAs (8 for n = 4096: 120 of 148 multiprocessors
+    // busy) the two-pass kernels win (0.86 against 1.04 ms).  Above 8 columns the two-pass kernels are the fastest.
+    if (h->single_pass_kernel == 2 || (h->single_pass_kernel == 0 && h->r > 4 && h->CS > 4 && !h->grad_bf16)) h->fused_ok = false;
     h->stream_ok = h->mode == 1 && h->single_pass_kernel == 3 && h->r <= 16 && h->n % 4 == 0 && h->N <= 16 && !h->grad_bf16;
     size_t wslots = h->fused_ok ? (size_t)h->KCmax : 0;
     if (h->stream_ok) {

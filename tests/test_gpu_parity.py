@@ -523,20 +523,20 @@ def test_pending_step_from_identical_state(torch_cuda, m, n, r, N, count, worklo
     L2-pipelined single-pass kernel, and the default choice among them)."""
     plan = _full_size_case(torch_cuda, workload, m, n, r, N, count, tau=0, sample=tuple(range(count)), free_steps=3,
                            expect_pending=True, single_pass=single_pass)
-    want = {"auto": 1 if r <= 4 else 0, "cluster": 1 if r <= 8 else 0, "none": 0, "l2": 2}[single_pass]
+    want = {"auto": 1 if r <= 8 else 0, "cluster": 1 if r <= 8 else 0, "none": 0, "l2": 2}[single_pass]     # (clusters of <= 4 CTAs here)
     assert plan["step_kernel"] == want
 
 
 def test_full_size_config2_attention_class(torch_cuda):
     """Workload 2, the 48 matrices of 768 x 768 (r = 8, N = 8, refresh at t = 0), three sampled."""
     plan = _full_size_case(torch_cuda, 2, 768, 768, 8, 8, 48, tau=50, sample=(0, 17, 47), free_steps=4, expect_pending=True)
-    assert plan["step_kernel"] == 0        # r = 8: the two-pass kernels are the default
+    assert plan["step_kernel"] == 1 and plan["CS"] == 3 and plan["WC"] == 256     # clusters of 3 CTAs x 256 columns
 
 
 def test_full_size_config2_ffn_class(torch_cuda):
     """Workload 2, the 36 matrices of 2048 x 768, two sampled."""
     plan = _full_size_case(torch_cuda, 2, 2048, 768, 8, 8, 36, tau=50, sample=(5, 35), free_steps=3, expect_pending=True)
-    assert plan["step_kernel"] == 0
+    assert plan["step_kernel"] == 1
 
 
 def test_full_size_config2_l2_pipelined_kernel(torch_cuda):
@@ -545,10 +545,10 @@ def test_full_size_config2_l2_pipelined_kernel(torch_cuda):
     assert plan["step_kernel"] == 2
 
 
-def test_full_size_config2_cluster_kernel(torch_cuda):
-    """The attention class through the cluster single-pass kernel (3 CTAs x 256 columns per cluster)."""
-    plan = _full_size_case(torch_cuda, 2, 768, 768, 8, 8, 48, tau=50, sample=(3,), free_steps=3, expect_pending=True, single_pass="cluster")
-    assert plan["step_kernel"] == 1 and plan["CS"] == 3 and plan["WC"] == 256
+def test_full_size_config2_two_pass_kernels(torch_cuda):
+    """The attention class through the two-pass kernels (projection with the residual formed on the fly, back-projection)."""
+    plan = _full_size_case(torch_cuda, 2, 768, 768, 8, 8, 48, tau=50, sample=(3,), free_steps=3, expect_pending=True, single_pass="none")
+    assert plan["step_kernel"] == 0
 
 
 @pytest.mark.parametrize("m,n,count,sample", [(768, 768, 48, (0, 31)), (2048, 768, 36, (20,))])
