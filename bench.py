@@ -59,6 +59,8 @@ def parse():
     ap.add_argument("--no-sweep", action="store_true", help="only the headline rank")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--grad-dtype", default="float32", choices=["float32", "bfloat16"],
+                    help="storage type of the gradients G of the headline measurement (bfloat16: 2 bytes per element read instead of 4)")
     ap.add_argument("--refresh-period", type=int, default=0, help="refresh period tau of the headline handle (0: SSP steps only, as the metric asks)")
     ap.add_argument("--small", action="store_true", help="a quarter of the sweep matrix (m = 4096): for profiler captures")
     return ap.parse_args()
@@ -374,14 +376,17 @@ def run_ours(args):
     peak, peak_kind = peaks()
     bufs = [synth.make_gradients_torch(5, m, n, N, 1, step=b, device=device) for b in range(2)]
     r = args.rank
-    alg_bytes, g_bytes = algorithmic_bytes([(m, n, 1)], r, N)
+    gbpe = 2 if args.grad_dtype == "bfloat16" else 4
+    alg_bytes, g_bytes = algorithmic_bytes([(m, n, 1)], r, N, gbpe)
+    hbufs = [b.to(torch.bfloat16) for b in bufs] if gbpe == 2 else bufs
 
     # ---- headline: the step at the headline rank, on every replica, max over ranks ----
     from paper_2509_11254_b200 import PowerSGDPlus
 
-    h = PowerSGDPlus(m, n, r, N, refresh_period=args.refresh_period, seed=5, device=device, mode=args.mode, single_pass=args.single_pass)
+    h = PowerSGDPlus(m, n, r, N, refresh_period=args.refresh_period, seed=5, device=device, mode=args.mode, single_pass=args.single_pass,
+                     grad_dtype=args.grad_dtype)
     for s in range(max(args.warmup, 3)):
-        h.step(bufs[s % 2])
+        h.step(hbufs[s % 2])
     torch.cuda.synchronize()
     sampler = ClockSampler(local)
     sampler.start()
@@ -391,7 +396,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     ev0.record()
     for s in range(args.steps):
-        h.step(bufs[s % 2])
+        h.step(hbufs[s % 2])
     ev1.record()
     torch.cuda.synchronize()
     reps.barrier()
@@ -401,9 +406,9 @@ def run_ours(args):
     value = reps.job_throughput(g_bytes, ms_step) / 1e9          # GB/s of gradient, all replicas
     # a longer look at the same step: blocks of 50 steps for at least half a second of device time
     # (--small is the profiler's case: no more launches than needed)
-    blocks, done = time_blocks(torch, lambda s: h.step(bufs[s % 2]), 100, min_seconds=0.5) if not args.small else ([ms_step], args.steps)
+    blocks, done = time_blocks(torch, lambda s: h.step(hbufs[s % 2]), 100, min_seconds=0.5) if not args.small else ([ms_step], args.steps)
     clocks = sampler.stop()
-    fam = family_profile([h], lambda s: h.step(bufs[s % 2]), 20 if not args.small else 2)
+    fam = family_profile([h], lambda s: h.step(hbufs[s % 2]), 20 if not args.small else 2)
     plan = h.plan_info()
     roofline = roofline_entry(fam, r, plan["step_kernel"], m * n * N, peak, peak_kind)
     roofline["note"] = "dominant kernel family of the headline step; a second pass of 20 steps with per-launch CUDA events on the launching stream"
@@ -412,7 +417,7 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": "sweep", "m": m, "n": n, "N": N, "ranks": list(SWEEP_RANKS), "headline_rank": r,
-                       "refresh_period": args.refresh_period, "mode": args.mode, "single_pass": args.single_pass,
+                       "refresh_period": args.refresh_period, "mode": args.mode, "single_pass": args.single_pass, "grad_dtype": args.grad_dtype,
                        "gradients": "low rank (s_k = 0.9^k, 256 terms) plus 5 % Gaussian noise, 2 alternating sets generated on the device",
                        "l2": "inputs (%.2f GB of G and as much of E per step) exceed L2" % (g_bytes / 1e9),
                        "parallelism": "replicas" if world > 1 else "single"},
@@ -424,11 +429,11 @@ def run_ours(args):
     if rank == 0 and not args.no_e2e:
         # end to end through the host-buffer entry point: H2D of G and D2H of (P~, Q) inside the timed region
         e2e_steps = 5
-        Gh = torch.empty(bufs[0].shape, dtype=bufs[0].dtype).pin_memory()
-        Gh.copy_(bufs[0])
+        Gh = torch.empty(hbufs[0].shape, dtype=hbufs[0].dtype).pin_memory()
+        Gh.copy_(hbufs[0])
         Ph = torch.empty(h.P_hat.shape, dtype=torch.float32).pin_memory()
         Qh = torch.empty(h.Q.shape, dtype=torch.float32).pin_memory()
-        stage = torch.empty_like(bufs[0])
+        stage = torch.empty_like(hbufs[0])
         h.step_host(Gh, stage, Ph, Qh)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
