@@ -88,6 +88,11 @@ typedef enum {
                                       2: the two-pass kernels; 3: the L2-pipelined single-pass kernel where it applies (up to 16
                                       columns, n % 4 == 0, float32 gradients).  A choice that does not apply falls back to two passes */
 
+#define PSGD_OPT_TRANSPOSED 10       /* 1: G, E (and D_hat, X, mom) are stored as [count][N][n][m], i.e. each matrix as the row-major
+                                      n x m transpose of the m x n problem (Sec. 1: X in R^{m x n}, m >= n): a weight kept as its transpose
+                                      needs no copy.  P_hat [m][r] and Q [n][r] keep their layouts.  Runs the three-pass kernels with their
+                                      roles exchanged (28 bytes per element); the deferred mode and bfloat16 gradients do not apply */
+
 /* buffers that psgd_debug_ptr exposes (test use only; valid until the next step) */
 #define PSGD_BUF_P_NODE 1   /* P^(i)   [count][N][m][r] */
 #define PSGD_BUF_Q_NODE 2   /* Q^(i)   [count][N][n][r] */
@@ -214,6 +219,20 @@ const char* psgd_last_cuda_error(const psgd_handle* h);
 
 /* Frees host memory of the handle.  Never touches caller-owned device buffers. */
 psgd_status psgd_destroy(psgd_handle* h);
+
+/*
+ * Several handles of different shapes stepped by ONE call (a model's matrices come in a few shape classes: Sec. 5 trains
+ * LLaMA- and RoBERTa-style stacks).  Each handle runs on a stream of the group's own, forked from `stream` and joined back into
+ * it, so that the small finishing kernels and the ragged last wave of one class overlap the streaming kernels of the others; for
+ * the caller's stream the call is one stream-ordered operation.  The handles share nothing, so the results equal those of
+ * stepping them one after the other bit for bit.  psgd_group_create creates CUDA streams and events on the current device (no
+ * device memory); handles must outlive the group.  G[i] / P_hat[i] (DEVICE; P_hat[i] and P_hat itself may be NULL) belong to handle i.
+ */
+typedef struct psgd_group psgd_group;
+psgd_status psgd_group_create(psgd_handle* const* handles /*HOST*/, int count, psgd_group** out);
+psgd_status psgd_group_step(psgd_group* g, const void* const* G /*HOST array of DEVICE pointers*/,
+                            float* const* P_hat /*HOST array of DEVICE pointers, or NULL*/, psgd_stream stream);
+psgd_status psgd_group_destroy(psgd_group* g);
 
 /*
  * The tensor-core contraction the refresh uses for its early subspace sweeps (SVD-Comp of

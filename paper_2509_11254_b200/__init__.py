@@ -7,6 +7,7 @@ There is no CPU fallback: using the binding without the built library raises.
 from .binding import (  # noqa: F401
     PSGDError,
     PowerSGDPlus,
+    StepGroup,
     lib,
     library_path,
     PSGD_W_RANK_DEFICIENT,

@@ -14,6 +14,7 @@ PSGD_OPT_POWER_STEPS = 6
 PSGD_OPT_REFRESH_ADAPTIVE = 7
 PSGD_OPT_GRAD_BF16 = 8
 PSGD_OPT_SINGLE_PASS = 9
+PSGD_OPT_TRANSPOSED = 10
 PSGD_BUF = {"P_node": 1, "Q_node": 2, "P_hat": 3, "Dbar": 4, "P_mean": 5}
 KERNEL_FAMILIES = ["project", "orth", "backproject", "residual", "refresh", "misc"]
 
@@ -48,6 +49,9 @@ SIGNATURES = {
     "psgd_gemm_nt_tf32_scratch": (_int, [_i64, _i64, _i64, _int, C.POINTER(_sz)]),
     "psgd_gemm_nt_tf32": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _int, _vp, _sz, _vp]),
     "psgd_backproject_static": (_int, [_vp, _vp, _vp, _vp, _i64, _i64, _int, _int, _vp]),
+    "psgd_group_create": (_int, [C.POINTER(_vp), _int, C.POINTER(_vp)]),
+    "psgd_group_step": (_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), _vp]),
+    "psgd_group_destroy": (_int, [_vp]),
 }
 
 
@@ -94,7 +98,7 @@ class PowerSGDPlus:
 
     def __init__(self, m, n, r, N, refresh_period=0, seed=0, count=1, device="cuda:0", error_form="local",
                  mode="eager", refresh_iters=None, oversample=None, reset=True, refresh_tc=None, power_steps=None, refresh_adaptive=None,
-                 grad_dtype="float32", single_pass=None):
+                 grad_dtype="float32", single_pass=None, transposed=False):
         import torch
 
         self.torch = torch
@@ -118,6 +122,9 @@ class PowerSGDPlus:
             _check(L.psgd_set_option(h, PSGD_OPT_POWER_STEPS, int(power_steps)))
         if refresh_adaptive is not None:
             _check(L.psgd_set_option(h, PSGD_OPT_REFRESH_ADAPTIVE, int(bool(refresh_adaptive))))
+        self.transposed = bool(transposed)
+        if self.transposed:
+            _check(L.psgd_set_option(h, PSGD_OPT_TRANSPOSED, 1))
         if single_pass is not None:
             _check(L.psgd_set_option(h, PSGD_OPT_SINGLE_PASS, {"auto": 0, "cluster": 1, "none": 2, "l2": 3}[single_pass]))
         self.grad_dtype = {"float32": torch.float32, "bfloat16": torch.bfloat16}[grad_dtype]
@@ -126,7 +133,7 @@ class PowerSGDPlus:
         eb, qb, wb = _sz(), _sz(), _sz()
         _check(L.psgd_sizes(h, C.byref(eb), C.byref(qb), C.byref(wb)))
         with torch.cuda.device(self.device):
-            self.E = torch.empty((count, N, m, n), dtype=torch.float32, device=self.device)
+            self.E = torch.empty((count, N, n, m) if self.transposed else (count, N, m, n), dtype=torch.float32, device=self.device)
             self.Q = torch.empty((count, n, r), dtype=torch.float32, device=self.device)
             self.ws = torch.empty((wb.value,), dtype=torch.uint8, device=self.device)
             self.P_hat = torch.empty((count, m, r), dtype=torch.float32, device=self.device)
@@ -243,6 +250,40 @@ class PowerSGDPlus:
         if getattr(self, "h", None) is not None and self.h.value:
             lib().psgd_destroy(self.h)
             self.h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class StepGroup:
+    """Handles of different shapes stepped by one call (psgd_group_*): each on a stream of the group's own,
+    forked from and joined into the caller's stream."""
+
+    def __init__(self, handles):
+        import torch
+
+        self.torch = torch
+        self.handles = list(handles)
+        arr = (_vp * len(self.handles))(*[h.h for h in self.handles])
+        g = _vp()
+        with torch.cuda.device(self.handles[0].device):
+            _check(lib().psgd_group_create(arr, len(self.handles), C.byref(g)))
+        self.g = g
+
+    def step(self, G_list, stream=None):
+        hs = self.handles
+        Gs = (_vp * len(hs))(*[h._g(g).data_ptr() for h, g in zip(hs, G_list)])
+        Ps = (_vp * len(hs))(*[h.P_hat.data_ptr() for h in hs])
+        with self.torch.cuda.device(hs[0].device):
+            _check(lib().psgd_group_step(self.g, Gs, Ps, hs[0]._stream(stream)))
+
+    def close(self):
+        if getattr(self, "g", None) is not None and self.g.value:
+            lib().psgd_group_destroy(self.g)
+            self.g = _vp()
 
     def __del__(self):
         try:

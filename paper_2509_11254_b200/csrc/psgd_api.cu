@@ -96,6 +96,8 @@ struct psgd_handle {
     int single_pass_kernel = 0;   // PSGD_OPT_SINGLE_PASS: 0 the fastest known for the shape, 1 cluster kernel, 2 two-pass kernels, 3 L2-pipelined kernel
     bool stream_ok = false;       // the shape fits the L2-pipelined kernel
     int s_nrb = 0, s_ngrp = 0, s_tpu = 0, s_csplit = 0, s_KC = 1, s_CB = 0, s_grid = -1;
+    bool transposed = false;      // PSGD_OPT_TRANSPOSED: G and E are stored as [n][m] (the transpose of the m x n problem)
+    int t_S = 1, t_rpc = 0;       // row chunks of the contraction over the n stored rows (transposed storage)
     int step_kernel = 0;          // what ran the last step: 0 three-/two-pass kernels, 1 cluster kernel, 2 L2-pipelined kernel
     int sm_count = 0;             // multiprocessors of the device that was current when the handle was created
 };
@@ -155,6 +157,14 @@ void plan(psgd_handle* h) {
     size_t part_step = cnt * N * (size_t)h->S * n * r * 4;
     size_t part_ref = cnt * (size_t)ceil_div(h->m, BP_SUB) * n * ell * 4;  // upper bound on chunks
     part_ref = std::min(part_ref, cnt * (size_t)64 * n * ell * 4);          // refresh uses <= 64 chunks
+    if (h->transposed) {   // P_i = S_i^T Q contracts over the n stored rows and has m outputs per column of Q
+        const int colblk_t = ceil_div(h->m, BP_COLS);
+        int St = (int)std::max<int64_t>(1, (target + (int64_t)h->count * h->N * colblk_t - 1) / ((int64_t)h->count * h->N * colblk_t));
+        St = std::min<int64_t>(St, ceil_div(h->n, BP_SUB));
+        h->t_rpc = (int)align_up(ceil_div(h->n, St), BP_SUB);
+        h->t_S = ceil_div(h->n, h->t_rpc);
+        part_step = std::max(part_step, cnt * N * (size_t)h->t_S * m * r * 4);
+    }
     L.part = take(std::max(part_step, part_ref));
     size_t nparts = std::max<size_t>(ceil_div(std::max(m, n), GR_ROWS), 64);  // 64: most clusters per matrix
     L.gram = take(cnt * nparts * c * c * 8);
@@ -169,6 +179,7 @@ void plan(psgd_handle* h) {
     L.dpart = take(cnt * ((size_t)ceil_div(h->m, 64) + 1) * 8);
     // ---- tensor-core sweeps of the refresh: block of >= 32 columns, 16-byte row strides for TMA ----
     h->tc_ok = h->refresh_tc && ell >= 32 && ell <= TC_MAXN && h->n % 4 == 0 && h->m % 4 == 0;
+    if (h->transposed && !h->tc_ok) L.dbarT = take(cnt * m * n * 4);   // the node mean in storage orientation, before it is transposed
     if (h->tc_ok) {
         const size_t ncp = align_up(ell, 16);
         L.dbarT = take(cnt * m * n * 4);
@@ -197,7 +208,7 @@ void plan(psgd_handle* h) {
     // A CTA owns WC in {128, 256, 512} columns of every node; the tile of S it keeps on chip and the
     // registers of its back-projection bound N * WC by 2048.  CS = ceil(n / WC) CTAs form a cluster.
     h->fused_ok = false;
-    if (h->mode == 1 && h->r <= 8 && h->n % 4 == 0 && h->N <= 16) {
+    if (h->mode == 1 && h->r <= 8 && h->n % 4 == 0 && h->N <= 16 && !h->transposed) {
         const int RP = h->r <= 4 ? 4 : 8;
         const int wcmax = h->N <= 4 ? 512 : (h->N <= 8 ? 256 : 128);
         int bestWC = 0, bestCS = 0;
@@ -231,7 +242,7 @@ void plan(psgd_handle* h) {
     // step of the 130M-shaped stack), while with clusters of more than 4 CTAs (8 for n = 4096: 120 of 148 multiprocessors
     // busy) the two-pass kernels win (0.86 against 1.04 ms).  Above 8 columns the two-pass kernels are the fastest.
     if (h->single_pass_kernel == 2 || (h->single_pass_kernel == 0 && h->r > 4 && h->CS > 4 && !h->grad_bf16)) h->fused_ok = false;
-    h->stream_ok = h->mode == 1 && h->single_pass_kernel == 3 && h->r <= 16 && h->n % 4 == 0 && h->N <= 16 && !h->grad_bf16;
+    h->stream_ok = !h->transposed && h->mode == 1 && h->single_pass_kernel == 3 && h->r <= 16 && h->n % 4 == 0 && h->N <= 16 && !h->grad_bf16;
     size_t wslots = h->fused_ok ? (size_t)h->KCmax : 0;
     if (h->stream_ok) {
         if (!h->fused_ok) h->RP = h->r <= 4 ? 4 : (h->r <= 8 ? 8 : 16);
@@ -608,11 +619,12 @@ bool launch_resid_tc(Launcher& L, const float* M, float* Out, const float* Phat,
 }
 
 void launch_resid(Launcher& L, const float* M, float* Out, const float* Phat, const float* Qf, int rows, int n, int r,
-                  int nodes, int mats, int q_per_node, int out_per_node, bool vec) {
-    if (r > 16 && launch_resid_tc(L, M, Out, Phat, Qf, rows, n, r, nodes, mats, q_per_node, out_per_node)) return;
+                  int nodes, int mats, int q_per_node, int out_per_node, bool vec, int p_per_node = 0) {
+    if (r > 16 && !p_per_node && launch_resid_tc(L, M, Out, Phat, Qf, rows, n, r, nodes, mats, q_per_node, out_per_node)) return;
     int rpc = 128;
     while (rpc > RS_SUB && (int64_t)mats * ceil_div(n, RS_COLS) * ceil_div(rows, rpc) < 4 * L.h->sm_count) rpc /= 2;
     ResidArgs a{M, Out, Phat, Qf, rows, n, r, nodes, rpc, q_per_node, out_per_node};
+    a.p_per_node = p_per_node;
     vec = vec && aligned16(Out) && (!M || aligned16(M));
     dim3 grid(ceil_div(n, RS_COLS), ceil_div(rows, rpc), mats);
     L.begin(PSGD_K_RESIDUAL);
@@ -743,7 +755,7 @@ void ssp(Launcher& L, psgd_handle* h, const void* Gv) {
 
 // ---- SVD-Comp (Algorithm 1, second function): top-r left singular subspace of the
 //      node mean by randomised block subspace iteration + Rayleigh-Ritz. ----------
-void svd(Launcher& L, psgd_handle* h, const void* G) {
+void svd(Launcher& L, psgd_handle* h, const void* G, bool have_dbar = false) {
     char* ws = h->ws;
     float* Phat = (float*)(ws + h->lay.Phat);
     float* dbar = (float*)(ws + h->lay.dbar);
@@ -762,7 +774,7 @@ void svd(Launcher& L, psgd_handle* h, const void* G) {
     // first 8 of them in TF32: measured on a 16384 x 4096 mean with a 0.9^k spectrum, 4 sweeps already bring the top-16
     // projector within 1e-5 and 8 sweeps the energy left behind at r = 64 within 1e-9 of the optimum.
     const int iters = h->refresh_iters > 0 ? h->refresh_iters : (h->tc_ok ? 12 : 20);
-    launch_add_mean(L, G, h->grad_bf16, h->E, dbar, (size_t)m * n, N, cnt, K);
+    if (!have_dbar) launch_add_mean(L, G, h->grad_bf16, h->E, dbar, (size_t)m * n, N, cnt, K);
     size_t zt = (size_t)cnt * n * ell;
     L.begin(K);
     k_fill_normal<<<(unsigned)((zt + 255) / 256), 256, 0, L.st>>>(Z, zt, h->seed, 0x5eed0000ull + (uint64_t)h->t);
@@ -876,6 +888,50 @@ void svd(Launcher& L, psgd_handle* h, const void* G) {
     }
     rayleigh_ritz();
     L.force_kind = -1;
+}
+
+// ---- one iteration with G and E stored transposed ([n][m] row-major, Sec. 1: X in R^{m x n} kept as X^T) ----------
+// The same kernels with their roles exchanged: the contraction over the stored rows (the back-projection kernels) gives
+// P_i = S_i^T Q, the contraction over the stored columns (the projection kernels) gives Q_i = S_i P~, and the residual kernel
+// takes Q_i as its row factor and P~ as its column factor.  Three passes plus the error-feedback add (28 bytes per element).
+void step_transposed(Launcher& L, psgd_handle* h, const void* G, bool refresh, float* D_hat) {
+    char* ws = h->ws;
+    float* Pnode = (float*)(ws + h->lay.Pnode);
+    float* Pmean = (float*)(ws + h->lay.Pmean);
+    float* Phat = (float*)(ws + h->lay.Phat);
+    float* Qnode = (float*)(ws + h->lay.Qnode);
+    float* part = (float*)(ws + h->lay.part);
+    const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count;
+    const bool vec_s = h->m % 4 == 0;          // stored rows have m entries
+    if (refresh) {
+        // node mean in storage orientation, transposed once into the [m][n] array SVD-Comp works on
+        float* dbar_s = (float*)(ws + h->lay.dbarT);
+        float* dbar = (float*)(ws + h->lay.dbar);
+        launch_add_mean(L, G, h->grad_bf16, h->E, dbar_s, (size_t)m * n, N, cnt, PSGD_K_REFRESH);
+        L.begin(PSGD_K_REFRESH);
+        k_transpose<<<dim3(ceil_div(m, 32), ceil_div(n, 32), cnt), dim3(32, 8), 0, L.st>>>(dbar_s, dbar, n, m);
+        L.end();
+        svd(L, h, G, true);
+    } else {
+        launch_add_mean(L, G, h->grad_bf16, h->E, nullptr, (size_t)m * n, N, cnt, PSGD_K_PROJECT);
+        // P_i = S_i^T Q_{t-1} and their node mean
+        const int Sb = launch_back(L, h->E, h->Q, part, n, m, r, N, cnt, h->t_rpc, h->t_S, vec_s);
+        size_t tot = (size_t)cnt * m * r;
+        L.begin(PSGD_K_PROJECT);
+        k_reduce_q<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(part, Pnode, Pmean, m, r, N, Sb, cnt);
+        L.end();
+        launch_orth(L, h, Pmean, Phat, m, r, PSGD_K_ORTH, nullptr, true);
+    }
+    // Q_i = S_i P~, Q = mean_i Q_i
+    launch_project(L, h->E, nullptr, nullptr, Phat, Qnode, n, m, r, N, cnt, vec_s);
+    size_t tq = (size_t)cnt * n * r;
+    L.begin(PSGD_K_BACKPROJECT);
+    k_node_mean<<<(unsigned)((tq + 255) / 256), 256, 0, L.st>>>(Qnode, h->Q, (size_t)n * r, N, cnt);
+    L.end();
+    // E_s = S - Q_i P~^T (stored orientation)
+    if (h->error_form == 0) launch_resid(L, h->E, h->E, Qnode, Phat, n, m, r, N, cnt * N, 0, 1, vec_s, 1);
+    else launch_resid(L, h->E, h->E, h->Q, Phat, n, m, r, N, cnt * N, 0, 1, vec_s, 0);
+    if (D_hat) launch_resid(L, nullptr, D_hat, h->Q, Phat, n, m, r, N, cnt, 0, 0, vec_s, 0);
 }
 
 // ---- single-pass SSP-Comp step (deferred residual) --------------------------------
@@ -1119,6 +1175,17 @@ psgd_status do_step(psgd_handle* h, const void* G, float* P_hat, float* D_hat, p
     Launcher L{h, st};
     bool refresh = force || (h->tau > 0 && h->t % h->tau == 0);
     // (a bfloat16 row has to be a multiple of 16 bytes for the tensor map: n % 8 == 0)
+    if (h->transposed) {
+        step_transposed(L, h, G, refresh, D_hat);
+        h->step_kernel = 0;
+        if (L.status != PSGD_OK) return L.status;
+        if (P_hat) {
+            PSGD_CUDA(h, cudaMemcpyAsync(P_hat, h->ws + h->lay.Phat, (size_t)h->count * h->m * h->r * 4,
+                                         cudaMemcpyDeviceToDevice, st));
+        }
+        h->t += 1;
+        return PSGD_OK;
+    }
     const bool one_pass = h->mode == 1 && !refresh && aligned16(G) && h->power_steps == 1;
     bool done = false;
     if (one_pass && h->stream_ok && h->s_grid != 0) {
@@ -1195,6 +1262,7 @@ psgd_status psgd_set_option(psgd_handle* h, int option, int value) {
         case PSGD_OPT_REFRESH_ADAPTIVE: if (value != 0 && value != 1) return PSGD_E_INVALID; h->refresh_adaptive = value; break;
         case PSGD_OPT_POWER_STEPS: if (value < 1 || value > 16) return PSGD_E_INVALID; h->power_steps = value; break;
         case PSGD_OPT_GRAD_BF16: if (value != 0 && value != 1) return PSGD_E_INVALID; h->grad_bf16 = value != 0; break;
+        case PSGD_OPT_TRANSPOSED: if (value != 0 && value != 1) return PSGD_E_INVALID; h->transposed = value != 0; break;
         case PSGD_OPT_SINGLE_PASS: if (value < 0 || value > 3) return PSGD_E_INVALID; h->single_pass_kernel = value; break;
         default: return PSGD_E_INVALID;
     }
@@ -1250,7 +1318,8 @@ psgd_status psgd_msgd_update(psgd_handle* h, float* X, float* mom, float eta, fl
     if (!X || !mom) return PSGD_E_NULL;
     if (h->t == 0) return PSGD_E_STATE;      // no P~_t, Q_t yet
     Launcher L{h, (cudaStream_t)stream};
-    launch_msgd(L, X, mom, eta, mu, (const float*)(h->ws + h->lay.Phat), h->Q, (int)h->m, (int)h->n, h->r, h->count);
+    if (h->transposed) launch_msgd(L, X, mom, eta, mu, h->Q, (const float*)(h->ws + h->lay.Phat), (int)h->n, (int)h->m, h->r, h->count);
+    else launch_msgd(L, X, mom, eta, mu, (const float*)(h->ws + h->lay.Phat), h->Q, (int)h->m, (int)h->n, h->r, h->count);
     return L.status;
 }
 
@@ -1417,6 +1486,73 @@ psgd_status psgd_gemm_nt_tf32(const float* A, const float* B, float* C, int64_t 
     if (cudaMemcpyAsync(&hflags, flags, 4, cudaMemcpyDeviceToHost, cs) != cudaSuccess || cudaStreamSynchronize(cs) != cudaSuccess)
         return PSGD_E_CUDA;
     return hflags ? PSGD_E_STATE : PSGD_OK;
+}
+
+}  // extern "C"
+
+struct psgd_group {
+    std::vector<psgd_handle*> hs;
+    std::vector<cudaStream_t> streams;
+    std::vector<cudaEvent_t> join;
+    cudaEvent_t fork = nullptr;
+};
+
+extern "C" {
+
+psgd_status psgd_group_create(psgd_handle* const* handles, int count, psgd_group** out) {
+    if (!handles || !out) return PSGD_E_NULL;
+    if (count < 1 || count > 4096) return PSGD_E_INVALID;
+    for (int i = 0; i < count; ++i)
+        if (!handles[i]) return PSGD_E_NULL;
+    psgd_group* g = new (std::nothrow) psgd_group();
+    if (!g) return PSGD_E_INVALID;
+    bool ok = cudaEventCreateWithFlags(&g->fork, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < count && ok; ++i) {
+        cudaStream_t s = nullptr;
+        cudaEvent_t e = nullptr;
+        ok = cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) == cudaSuccess;
+        if (ok) g->streams.push_back(s);
+        ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+        if (ok) g->join.push_back(e);
+        if (ok) g->hs.push_back(handles[i]);
+    }
+    if (!ok) {
+        cudaGetLastError();
+        psgd_group_destroy(g);
+        return PSGD_E_CUDA;
+    }
+    *out = g;
+    return PSGD_OK;
+}
+
+psgd_status psgd_group_step(psgd_group* g, const void* const* G, float* const* P_hat, psgd_stream stream) {
+    if (!g || !G) return PSGD_E_NULL;
+    for (size_t i = 0; i < g->hs.size(); ++i) {
+        psgd_status s = check_ready(g->hs[i]);
+        if (s != PSGD_OK) return s;
+        if (!G[i]) return PSGD_E_NULL;
+    }
+    cudaStream_t main = (cudaStream_t)stream;
+    if (cudaEventRecord(g->fork, main) != cudaSuccess) return PSGD_E_CUDA;
+    psgd_status worst = PSGD_OK;
+    for (size_t i = 0; i < g->hs.size(); ++i) {
+        if (cudaStreamWaitEvent(g->streams[i], g->fork, 0) != cudaSuccess) return PSGD_E_CUDA;
+        psgd_status s = psgd_step(g->hs[i], G[i], P_hat ? P_hat[i] : nullptr, nullptr, (psgd_stream)g->streams[i]);
+        if (s != PSGD_OK && worst == PSGD_OK) worst = s;
+        if (cudaEventRecord(g->join[i], g->streams[i]) != cudaSuccess) return PSGD_E_CUDA;
+    }
+    for (size_t i = 0; i < g->hs.size(); ++i)
+        if (cudaStreamWaitEvent(main, g->join[i], 0) != cudaSuccess) return PSGD_E_CUDA;
+    return worst;
+}
+
+psgd_status psgd_group_destroy(psgd_group* g) {
+    if (!g) return PSGD_E_NULL;
+    for (cudaStream_t s : g->streams) { cudaStreamSynchronize(s); cudaStreamDestroy(s); }
+    for (cudaEvent_t e : g->join) cudaEventDestroy(e);
+    if (g->fork) cudaEventDestroy(g->fork);
+    delete g;
+    return PSGD_OK;
 }
 
 }  // extern "C"

@@ -462,6 +462,7 @@ struct ResidArgs {
     int rows, n, r, nodes, rows_per_chunk;
     int q_per_node;     // 1: Qf indexed by (matrix,node); 0: by matrix only
     int out_per_node;   // 1: Out/M indexed by (matrix,node); 0: by matrix only (dense reconstruction)
+    int p_per_node = 0; // 1: Phat (the row factor) indexed by (matrix,node); 0: by matrix only
     // momentum-SGD hand-off (Eq. (7c)), only with M == nullptr: instead of storing the reconstruction D^,
     // mom <- mu mom + D^ and X <- X - eta mom, both [mats][rows][n]
     float* X = nullptr;
@@ -481,7 +482,7 @@ __global__ void __launch_bounds__(RS_THREADS) k_residual(ResidArgs a) {
     const float* Mb = a.M ? a.M + (size_t)mat * a.rows * n : nullptr;
     float* Ob = a.X ? a.X + (size_t)mat * a.rows * n : a.Out + (size_t)mat * a.rows * n;
     float* Vb = a.X ? a.Mom + (size_t)mat * a.rows * n : nullptr;
-    const float* Pb = a.Phat + (size_t)c * a.rows * r;
+    const float* Pb = a.Phat + (size_t)(a.p_per_node ? mat : c) * a.rows * r;
     const float* Qb = a.Qf + (size_t)(a.q_per_node ? mat : c) * n * r;
     const int nch = (r + RP - 1) / RP;
     const int rpad = nch * RP;

@@ -94,12 +94,13 @@ def check_residual(E_gpu, E_ref, normM, tag, e_abs=E_ABS):
 
 
 def run_case(torch, m, n, r, N, tau, steps, workload=1, count=1, error_form="local", Einit=0.0, seed=7,
-             check_dense=False, mode="eager", power_steps=1, grad_dtype="float32", single_pass=None):
+             check_dense=False, mode="eager", power_steps=1, grad_dtype="float32", single_pass=None, transposed=False):
     from paper_2509_11254_b200 import PowerSGDPlus
 
     dev = "cuda:0"
     comp = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=seed, count=count, device=dev, error_form=error_form,
-                        mode=mode, power_steps=power_steps, grad_dtype=grad_dtype, single_pass=single_pass)
+                        mode=mode, power_steps=power_steps, grad_dtype=grad_dtype, single_pass=single_pass, transposed=transposed)
+    tr = (lambda a: np.ascontiguousarray(np.swapaxes(a, -1, -2))) if transposed else (lambda a: a)   # problem <-> storage orientation
     rng = np.random.default_rng(seed)
     Q0 = np.stack([synth.init_Q(n, r, matrix_id=c, seed=seed) for c in range(count)])
     oracles = [orc.PowerSGDPlusOracle(m, n, r, N, tau, Q0[c], error_form, power_steps) for c in range(count)]
@@ -112,18 +113,18 @@ def run_case(torch, m, n, r, N, tau, steps, workload=1, count=1, error_form="loc
         for o in oracles:
             o.E = o.E.astype(np.float32).astype(np.float64)
             o.Q = o.Q.astype(np.float32).astype(np.float64)
-        comp.set_state(E=np.stack([o.E for o in oracles]), Q=np.stack([o.Q for o in oracles]), t=t)
-        Gd = torch.as_tensor(G, device=dev)
+        comp.set_state(E=tr(np.stack([o.E for o in oracles])), Q=np.stack([o.Q for o in oracles]), t=t)
+        Gd = torch.as_tensor(tr(G), device=dev)
         if grad_dtype == "bfloat16":     # the oracle gets the same bfloat16 values, widened
             Gd = Gd.to(torch.bfloat16)
             G = Gd.float().cpu().numpy()
-        Dh = torch.empty((count, m, n), dtype=torch.float32, device=dev) if check_dense else None
+        Dh = torch.empty((count, n, m) if transposed else (count, m, n), dtype=torch.float32, device=dev) if check_dense else None
         comp.step(Gd, D_hat=Dh)
         comp.materialize_error()
         flags = comp.last_status()
         assert flags == 0, f"step {t}: warning flags {flags}"
         assert comp.t == t + 1
-        gp = dict(P_hat=comp.P_hat.cpu().numpy(), Q=comp.Q.cpu().numpy(), E=comp.E.cpu().numpy(),
+        gp = dict(P_hat=comp.P_hat.cpu().numpy(), Q=comp.Q.cpu().numpy(), E=tr(comp.E.cpu().numpy()),
                   Q_node=comp.debug("Q_node").cpu().numpy())
         if mode == "eager" and power_steps == 1:   # (single-pass: no per-node P_i; K steps: P_i is the last round's)
             gp["P_node"] = comp.debug("P_node").cpu().numpy()
@@ -135,7 +136,7 @@ def run_case(torch, m, n, r, N, tau, steps, workload=1, count=1, error_form="loc
             if check_dense:
                 Pg = gp["P_hat"][c].astype(np.float64)
                 Qg = gp["Q"][c].astype(np.float64)
-                assert rel_fro(Dh[c].cpu().numpy(), Pg @ Qg.T) <= TOL
+                assert rel_fro(tr(Dh[c].cpu().numpy()), Pg @ Qg.T) <= TOL
     comp.close()
 
 
@@ -207,6 +208,23 @@ def test_bfloat16_gradients(torch_cuda, m, n, r, N, count, mode, tau, Einit):
 def test_k_step_power_iteration(torch_cuda, K, mode):
     """Eq. (8): K power steps per iteration (the deferred mode falls back to the three-pass kernels)."""
     run_case(torch_cuda, 300, 200, 6, 3, tau=0, steps=3, workload=2, count=2, Einit=0.01, mode=mode, power_steps=K)
+
+
+@pytest.mark.parametrize("m,n,r,N,count,tau,form,workload", [
+    (300, 200, 8, 2, 3, 0, "local", 2),      # ragged both ways, batch of 3
+    (513, 260, 16, 1, 1, 0, "local", 5),     # a single node
+    (1004, 500, 12, 3, 1, 0, "mean", 2),     # residual with the node-averaged Q
+    (640, 256, 40, 2, 1, 0, "local", 4),     # more than 16 columns: tensor-core contractions, float32 residual kernel
+    (256, 128, 4, 4, 1, 3, "local", 1),      # refreshes at t = 0 and 3 (the node mean is transposed once per refresh)
+    (1000, 520, 32, 2, 1, 2, "local", 5),    # refresh with tensor-core sweeps
+    (257, 130, 3, 2, 2, 0, "local", 2),      # m % 4 != 0: scalar loads along the stored rows
+])
+def test_transposed_storage(torch_cuda, m, n, r, N, count, tau, form, workload):
+    """PSGD_OPT_TRANSPOSED: G and E kept as the row-major n x m transposes of the m x n problem (Sec. 1 fixes m >= n for the
+    problem, not for how a weight lies in memory).  Same outputs, same tolerances; E and the dense reconstruction are compared
+    after transposing them back."""
+    run_case(torch_cuda, m, n, r, N, tau=tau, steps=4, workload=workload, count=count, Einit=0.0 if tau else 0.01, error_form=form,
+             check_dense=True, transposed=True)
 
 
 def test_mean_error_form(torch_cuda):
@@ -847,3 +865,49 @@ def test_ill_conditioned_projection_takes_the_precise_path(torch_cuda):
     # (columns 2 and 3 of P = M Q are 0.02 apart in angle: the float32 rounding of P is amplified by 1 / 0.02 in P~, so the
     #  absolute bound on E is widened by that factor's share; the 1e-5 bounds on P~, Q and Q_i are not)
     compare_step(out, gp, m, n, r, N, "ill-conditioned Q", e_abs=32.0)
+
+
+def test_group_step_of_mixed_shapes_equals_separate_steps():
+    """psgd_group_step: handles of different shapes, ranks, modes and storage stepped by one call give, bit for bit, what stepping
+    them one after the other gives (they share nothing), over several steps including refreshes."""
+    import torch
+
+    from paper_2509_11254_b200 import PowerSGDPlus, StepGroup, synth
+
+    specs = [  # (m, n, r, N, count, kwargs)
+        (512, 256, 4, 2, 3, dict(refresh_period=3)),
+        (300, 130, 5, 3, 1, dict(refresh_period=0, mode="deferred")),
+        (1024, 512, 16, 4, 2, dict(refresh_period=3, mode="deferred", single_pass="l2")),
+        (640, 256, 40, 2, 1, dict(refresh_period=0, mode="deferred")),
+        (130, 300, 6, 2, 2, dict(refresh_period=3, transposed=True)),
+    ]
+
+    def make():
+        return [PowerSGDPlus(max(m, n), min(m, n), r, N, count=c, seed=7 + i, device="cuda:0", **kw)
+                for i, (m, n, r, N, c, kw) in enumerate(specs)]
+
+    def grads(step):
+        out = []
+        for i, (m, n, r, N, c, kw) in enumerate(specs):
+            g = np.stack([synth.make_gradients(2, max(m, n), min(m, n), N, step=step, seed=100 * i + j) for j in range(c)])
+            if kw.get("transposed"):
+                g = np.ascontiguousarray(np.swapaxes(g, -1, -2))
+            out.append(torch.as_tensor(g, device="cuda:0"))
+        return out
+
+    one, many = make(), make()
+    group = StepGroup(many)
+    for step in range(5):
+        Gs = grads(step)
+        for h, g in zip(one, Gs):
+            h.step(g)
+        group.step(Gs)
+        torch.cuda.synchronize()
+        for a, b in zip(one, many):
+            assert torch.equal(a.P_hat, b.P_hat) and torch.equal(a.Q, b.Q)
+            a.materialize_error(); b.materialize_error()
+            assert torch.equal(a.E, b.E)
+            assert a.last_status() == b.last_status()
+    group.close()
+    for h in one + many:
+        h.close()
