@@ -221,6 +221,34 @@ const char* psgd_last_cuda_error(const psgd_handle* h);
 psgd_status psgd_destroy(psgd_handle* h);
 
 /*
+ * One iteration of Algorithm 2 with the nodes spread over several processes (one or more nodes per GPU).  Algorithm 2
+ * averages three arrays over the nodes: P = mean_i P_i, Q = mean_i Q_i and, when t mod tau = 0, Delta = mean_i (g_i + e_i).
+ * A handle created with N nodes forms the mean over ITS nodes; the caller averages over the processes between the phases
+ * (an all-reduce with the mean as its operation, every process holding the same N) and hands the result back:
+ *
+ *   psgd_exchange_plan   whether the next step is a refresh (t mod tau = 0, or force_refresh) and how many floats each exchange carries:
+ *                        first = count*m*r (P), or count*m*n at a refresh (Delta); second = count*n*r (Q)
+ *   psgd_exchange_begin  M_i = G_i + e_i, then `first` <- local mean of P_i = M_i Q_{t-1} (at a refresh: of M_i,
+ *                        in storage orientation)
+ *        ... caller: first <- mean over processes of first ...
+ *   psgd_exchange_orth   P~ = orth(first) (at a refresh: SVD-Comp on first), then `second` <- local mean of Q_i = M_i^T P~
+ *        ... caller: second <- mean over processes of second ...
+ *   psgd_exchange_end    Q_t <- second, e_{t+1,i} = M_i - P~ Q_i^T (or - P~ Q_t^T, PSGD_OPT_ERROR_FORM = 1), P_hat and
+ *                        D_hat as in psgd_step, t <- t + 1
+ *
+ * `first` and `second` are DEVICE arrays of the caller (16-byte aligned; typically slots of one flat buffer per exchange that
+ * serves all handles of a model, so that each exchange is one all-reduce); the library reads and writes them in stream
+ * order and keeps no pointer to them.  All processes must use the same seed, options and step count: each then factorises
+ * the same averaged array with the same deterministic kernels and obtains the same P~.  With one process the three phases
+ * equal psgd_step (eager mode) or its two-pass form (PSGD_OPT_MODE = 1: up to 16 columns the residual stays pending in E);
+ * the single-pass kernels are not used.  PSGD_E_INVALID: phases out of order, PSGD_OPT_POWER_STEPS > 1, misaligned arrays.
+ */
+psgd_status psgd_exchange_plan(const psgd_handle* h, int force_refresh, int* refresh, size_t* first_floats, size_t* second_floats);
+psgd_status psgd_exchange_begin(psgd_handle* h, const void* G, int force_refresh, float* first, psgd_stream stream);
+psgd_status psgd_exchange_orth(psgd_handle* h, const float* first, float* second, psgd_stream stream);
+psgd_status psgd_exchange_end(psgd_handle* h, const float* second, float* P_hat, float* D_hat, psgd_stream stream);
+
+/*
  * Several handles of different shapes stepped by ONE call (a model's matrices come in a few shape classes: Sec. 5 trains
  * LLaMA- and RoBERTa-style stacks).  Each handle runs on a stream of the group's own, forked from `stream` and joined back into
  * it, so that the small finishing kernels and the ragged last wave of one class overlap the streaming kernels of the others; for

@@ -16,3 +16,4 @@ from .binding import (  # noqa: F401
     KERNEL_FAMILIES,
 )
 from .stack import StreamedStack  # noqa: F401,E402
+from .exchange import ExchangedStack, slot_offsets  # noqa: F401,E402

@@ -49,6 +49,10 @@ SIGNATURES = {
     "psgd_gemm_nt_tf32_scratch": (_int, [_i64, _i64, _i64, _int, C.POINTER(_sz)]),
     "psgd_gemm_nt_tf32": (_int, [_vp, _vp, _vp, _i64, _i64, _i64, _int, _vp, _sz, _vp]),
     "psgd_backproject_static": (_int, [_vp, _vp, _vp, _vp, _i64, _i64, _int, _int, _vp]),
+    "psgd_exchange_plan": (_int, [_vp, _int, C.POINTER(_int), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
+    "psgd_exchange_begin": (_int, [_vp, _vp, _int, _vp, _vp]),
+    "psgd_exchange_orth": (_int, [_vp, _vp, _vp, _vp]),
+    "psgd_exchange_end": (_int, [_vp, _vp, _vp, _vp, _vp]),
     "psgd_group_create": (_int, [C.POINTER(_vp), _int, C.POINTER(_vp)]),
     "psgd_group_step": (_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), _vp]),
     "psgd_group_destroy": (_int, [_vp]),
@@ -175,6 +179,38 @@ class PowerSGDPlus:
                                         P_hat_host.data_ptr() if P_hat_host is not None else None,
                                         Q_host.data_ptr() if Q_host is not None else None,
                                         self._stream(stream)), self.h)
+
+    # One iteration with the nodes spread over several processes: the caller averages `first` and `second` over the
+    # processes between the phases (exchange.ExchangedStack does, with torch.distributed).
+    def exchange_plan(self, force_refresh=False):
+        """(refresh, first_floats, second_floats) of the next step."""
+        rf, a, b = _int(), C.c_size_t(), C.c_size_t()
+        _check(lib().psgd_exchange_plan(self.h, int(bool(force_refresh)), C.byref(rf), C.byref(a), C.byref(b)))
+        return bool(rf.value), a.value, b.value
+
+    def _slot(self, t, floats):
+        tt = self.torch
+        if not (isinstance(t, tt.Tensor) and t.is_cuda and t.dtype == tt.float32 and t.is_contiguous() and t.numel() >= floats):
+            raise PSGDError(f"an exchange array must be a contiguous float32 CUDA tensor of at least {floats} elements")
+        return t.data_ptr()
+
+    def exchange_begin(self, G, first, force_refresh=False, stream=None):
+        G = self._g(G)
+        floats = self.exchange_plan(force_refresh)[1]
+        with self.torch.cuda.device(self.device):
+            _check(lib().psgd_exchange_begin(self.h, G.data_ptr(), int(bool(force_refresh)), self._slot(first, floats),
+                                             self._stream(stream)), self.h)
+
+    def exchange_orth(self, first, second, stream=None):
+        _, a, b = self.exchange_plan()
+        with self.torch.cuda.device(self.device):
+            _check(lib().psgd_exchange_orth(self.h, self._slot(first, a), self._slot(second, b), self._stream(stream)), self.h)
+
+    def exchange_end(self, second, D_hat=None, stream=None):
+        b = self.exchange_plan()[2]
+        with self.torch.cuda.device(self.device):
+            _check(lib().psgd_exchange_end(self.h, self._slot(second, b), self.P_hat.data_ptr(),
+                                           D_hat.data_ptr() if D_hat is not None else None, self._stream(stream)), self.h)
 
     def msgd_update(self, X, mom, eta, mu, stream=None):
         """Eq. (7c) with the reconstruction of the last step: mom <- mu mom + P~ Q^T, X <- X - eta mom (in place)."""

@@ -99,6 +99,8 @@ struct psgd_handle {
     bool transposed = false;      // PSGD_OPT_TRANSPOSED: G and E are stored as [n][m] (the transpose of the m x n problem)
     int t_S = 1, t_rpc = 0;       // row chunks of the contraction over the n stored rows (transposed storage)
     int step_kernel = 0;          // what ran the last step: 0 three-/two-pass kernels, 1 cluster kernel, 2 L2-pipelined kernel
+    int ex_phase = 0;             // psgd_exchange_*: 0 between steps, 1 after _begin, 2 after _orth
+    bool ex_refresh = false;      // the step in flight is a refresh
     int sm_count = 0;             // multiprocessors of the device that was current when the handle was created
 };
 
@@ -300,6 +302,12 @@ struct Launcher {
         cudaEventCreate(&ev.b);
         cudaEventRecord(ev.a, st);
         h->events.push_back(ev);
+    }
+    void check(cudaError_t e) {   // a runtime call that is not a launch of this library's kernels
+        if (e != cudaSuccess && status == PSGD_OK) {
+            snprintf(h->err, sizeof(h->err), "runtime call: %s", cudaGetErrorString(e));
+            status = PSGD_E_CUDA;
+        }
     }
     void end() {
         if (h->profiling) cudaEventRecord(h->events.back().b, st);
@@ -710,10 +718,10 @@ void tail(Launcher& L, psgd_handle* h, float* D_hat, bool defer = false) {
 }
 
 // ---- SSP-Comp (Algorithm 1, first function) ------------------------------------
-void ssp(Launcher& L, psgd_handle* h, const void* Gv) {
+// P_i = (G_i + e_i) Q_{t-1} for every node, M_i left in the E buffer
+void ssp_project(Launcher& L, psgd_handle* h, const void* Gv) {
     char* ws = h->ws;
     float* Pnode = (float*)(ws + h->lay.Pnode);
-    float* Pmean = (float*)(ws + h->lay.Pmean);
     float* Phat = (float*)(ws + h->lay.Phat);
     const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count;
     const float* G = (const float*)Gv;
@@ -730,6 +738,15 @@ void ssp(Launcher& L, psgd_handle* h, const void* Gv) {
         launch_add_mean(L, G, false, h->E, nullptr, (size_t)m * n, N, cnt, PSGD_K_PROJECT);
         launch_project(L, h->E, nullptr, nullptr, h->Q, Pnode, m, n, r, N, cnt, h->vec4);
     }
+}
+
+void ssp(Launcher& L, psgd_handle* h, const void* Gv) {
+    char* ws = h->ws;
+    float* Pnode = (float*)(ws + h->lay.Pnode);
+    float* Pmean = (float*)(ws + h->lay.Pmean);
+    float* Phat = (float*)(ws + h->lay.Phat);
+    const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count;
+    ssp_project(L, h, Gv);
     size_t tot = (size_t)cnt * m * r;
     L.begin(PSGD_K_ORTH);
     k_node_mean<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Pnode, Pmean, (size_t)m * r, N, cnt);
@@ -1161,6 +1178,99 @@ void materialize(Launcher& L, psgd_handle* h) {
     h->pending = false;
 }
 
+// ---- one iteration with the nodes spread over several processes --------------------------------------------------
+// Algorithm 2 averages P (line "P <- allreduce-mean"), Q and, at a refresh, Delta over the nodes.  Here this handle holds
+// N of the nodes; the caller averages three small arrays over the processes between the phases.  Every process then
+// factorises the same averaged P (or runs SVD-Comp on the same averaged Delta) and gets the same P~ bit for bit.
+// Deferred mode runs the two-pass form (the residual stays pending between steps); the single-pass kernels fuse the
+// node mean and have no place for an exchange.
+bool ex_two_pass(const psgd_handle* h) { return h->mode == 1 && h->r <= 16 && !h->grad_bf16; }
+
+void exchange_begin(Launcher& L, psgd_handle* h, const void* G, float* out, bool refresh) {
+    char* ws = h->ws;
+    float* Pnode = (float*)(ws + h->lay.Pnode);
+    float* part = (float*)(ws + h->lay.part);
+    const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count;
+    const size_t tot = (size_t)cnt * m * r;
+    if (h->transposed) {
+        launch_add_mean(L, G, h->grad_bf16, h->E, refresh ? out : nullptr, (size_t)m * n, N, cnt, refresh ? PSGD_K_REFRESH : PSGD_K_PROJECT);
+        if (refresh) return;     // out: the local mean in storage orientation
+        const int Sb = launch_back(L, h->E, h->Q, part, n, m, r, N, cnt, h->t_rpc, h->t_S, h->m % 4 == 0);
+        L.begin(PSGD_K_PROJECT);
+        k_reduce_q<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(part, Pnode, out, m, r, N, Sb, cnt);
+        L.end();
+        return;
+    }
+    if (!ex_two_pass(h) || refresh) materialize(L, h);
+    if (refresh) {
+        launch_add_mean(L, G, h->grad_bf16, h->E, out, (size_t)m * n, N, cnt, PSGD_K_REFRESH);
+        return;
+    }
+    ssp_project(L, h, G);
+    L.begin(PSGD_K_ORTH);
+    k_node_mean<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Pnode, out, (size_t)m * r, N, cnt);
+    L.end();
+}
+
+void exchange_orth(Launcher& L, psgd_handle* h, const float* in, float* out, bool refresh) {
+    char* ws = h->ws;
+    float* Phat = (float*)(ws + h->lay.Phat);
+    float* Qnode = (float*)(ws + h->lay.Qnode);
+    float* part = (float*)(ws + h->lay.part);
+    float* dbar = (float*)(ws + h->lay.dbar);
+    const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count;
+    const size_t tq = (size_t)cnt * n * r;
+    if (refresh) {
+        if (h->transposed) {
+            L.begin(PSGD_K_REFRESH);
+            k_transpose<<<dim3(ceil_div(m, 32), ceil_div(n, 32), cnt), dim3(32, 8), 0, L.st>>>(in, dbar, n, m);
+            L.end();
+        } else {
+            L.check(cudaMemcpyAsync(dbar, in, (size_t)cnt * m * n * 4, cudaMemcpyDeviceToDevice, L.st));
+        }
+        svd(L, h, nullptr, true);
+    } else {
+        launch_orth(L, h, in, Phat, m, r, PSGD_K_ORTH, nullptr, true);
+    }
+    if (h->transposed) {
+        launch_project(L, h->E, nullptr, nullptr, Phat, Qnode, n, m, r, N, cnt, h->m % 4 == 0);
+        L.begin(PSGD_K_BACKPROJECT);
+        k_node_mean<<<(unsigned)((tq + 255) / 256), 256, 0, L.st>>>(Qnode, out, (size_t)n * r, N, cnt);
+        L.end();
+    } else {
+        const int Sb = launch_back(L, h->E, Phat, part, m, n, r, N, cnt, h->rpc, h->S, h->vec4);
+        L.begin(PSGD_K_BACKPROJECT);
+        k_reduce_q<<<(unsigned)((tq + 255) / 256), 256, 0, L.st>>>(part, Qnode, out, n, r, N, Sb, cnt);
+        L.end();
+    }
+}
+
+void exchange_end(Launcher& L, psgd_handle* h, const float* in, float* D_hat) {
+    char* ws = h->ws;
+    float* Phat = (float*)(ws + h->lay.Phat);
+    float* Qnode = (float*)(ws + h->lay.Qnode);
+    const int m = (int)h->m, n = (int)h->n, r = h->r, N = h->N, cnt = h->count;
+    if (in != h->Q) L.check(cudaMemcpyAsync(h->Q, in, (size_t)cnt * n * r * 4, cudaMemcpyDeviceToDevice, L.st));
+    if (h->transposed) {
+        const bool vec_s = h->m % 4 == 0;
+        if (h->error_form == 0) launch_resid(L, h->E, h->E, Qnode, Phat, n, m, r, N, cnt * N, 0, 1, vec_s, 1);
+        else launch_resid(L, h->E, h->E, h->Q, Phat, n, m, r, N, cnt * N, 0, 1, vec_s, 0);
+        if (D_hat) launch_resid(L, nullptr, D_hat, h->Q, Phat, n, m, r, N, cnt, 0, 0, vec_s, 0);
+        return;
+    }
+    if (ex_two_pass(h)) {
+        h->pending = true;
+        h->pending_fused = false;
+    } else if (h->error_form == 0) {
+        launch_resid(L, h->E, h->E, Phat, Qnode, m, n, r, N, cnt * N, 1, 1, h->vec4);
+    } else {
+        launch_resid(L, h->E, h->E, Phat, h->Q, m, n, r, N, cnt * N, 0, 1, h->vec4);
+    }
+    if (D_hat) launch_resid(L, nullptr, D_hat, Phat, h->Q, m, n, r, N, cnt, 0, 0, h->vec4);
+    h->tacc_identity = true;
+    h->qpad_valid = false;
+}
+
 psgd_status check_ready(const psgd_handle* h) {
     if (!h) return PSGD_E_NULL;
     if (!h->E || !h->Q || !h->ws) return PSGD_E_WORKSPACE;
@@ -1171,6 +1281,7 @@ psgd_status do_step(psgd_handle* h, const void* G, float* P_hat, float* D_hat, p
     psgd_status s = check_ready(h);
     if (s != PSGD_OK) return s;
     if (!G) return PSGD_E_NULL;
+    if (h->ex_phase != 0) return PSGD_E_INVALID;   // an iteration begun by psgd_exchange_begin is still open
     cudaStream_t st = (cudaStream_t)stream;
     Launcher L{h, st};
     bool refresh = force || (h->tau > 0 && h->t % h->tau == 0);
@@ -1301,6 +1412,7 @@ psgd_status psgd_reset(psgd_handle* h, psgd_stream stream) {
     L.end();
     h->t = 0;
     h->pending = false; h->tacc_identity = true; h->qpad_valid = false;
+    h->ex_phase = 0;
     return L.status;
 }
 
@@ -1310,6 +1422,57 @@ psgd_status psgd_step(psgd_handle* h, const void* G, float* P_hat, float* D_hat,
 
 psgd_status psgd_refresh(psgd_handle* h, const void* G, float* P_hat, float* D_hat, psgd_stream stream) {
     return do_step(h, G, P_hat, D_hat, stream, true);
+}
+
+psgd_status psgd_exchange_plan(const psgd_handle* h, int force_refresh, int* refresh, size_t* first_floats, size_t* second_floats) {
+    if (!h) return PSGD_E_NULL;
+    const bool rf = h->ex_phase != 0 ? h->ex_refresh : (force_refresh || (h->tau > 0 && h->t % h->tau == 0));
+    if (refresh) *refresh = rf ? 1 : 0;
+    if (first_floats) *first_floats = (size_t)h->count * h->m * (rf ? (size_t)h->n : (size_t)h->r);
+    if (second_floats) *second_floats = (size_t)h->count * h->n * h->r;
+    return PSGD_OK;
+}
+
+psgd_status psgd_exchange_begin(psgd_handle* h, const void* G, int force_refresh, float* first, psgd_stream stream) {
+    psgd_status s = check_ready(h);
+    if (s != PSGD_OK) return s;
+    if (!G || !first) return PSGD_E_NULL;
+    if (h->ex_phase != 0 || h->power_steps != 1 || !aligned16(first)) return PSGD_E_INVALID;
+    Launcher L{h, (cudaStream_t)stream};
+    h->ex_refresh = force_refresh || (h->tau > 0 && h->t % h->tau == 0);
+    exchange_begin(L, h, G, first, h->ex_refresh);
+    if (L.status != PSGD_OK) return L.status;
+    h->ex_phase = 1;
+    return PSGD_OK;
+}
+
+psgd_status psgd_exchange_orth(psgd_handle* h, const float* first, float* second, psgd_stream stream) {
+    psgd_status s = check_ready(h);
+    if (s != PSGD_OK) return s;
+    if (!first || !second) return PSGD_E_NULL;
+    if (h->ex_phase != 1 || !aligned16(first) || !aligned16(second)) return PSGD_E_INVALID;
+    Launcher L{h, (cudaStream_t)stream};
+    exchange_orth(L, h, first, second, h->ex_refresh);
+    if (L.status != PSGD_OK) return L.status;
+    h->ex_phase = 2;
+    return PSGD_OK;
+}
+
+psgd_status psgd_exchange_end(psgd_handle* h, const float* second, float* P_hat, float* D_hat, psgd_stream stream) {
+    psgd_status s = check_ready(h);
+    if (s != PSGD_OK) return s;
+    if (!second) return PSGD_E_NULL;
+    if (h->ex_phase != 2 || !aligned16(second)) return PSGD_E_INVALID;
+    cudaStream_t st = (cudaStream_t)stream;
+    Launcher L{h, st};
+    exchange_end(L, h, second, D_hat);
+    if (L.status != PSGD_OK) return L.status;
+    h->step_kernel = 0;
+    if (P_hat)
+        PSGD_CUDA(h, cudaMemcpyAsync(P_hat, h->ws + h->lay.Phat, (size_t)h->count * h->m * h->r * 4, cudaMemcpyDeviceToDevice, st));
+    h->ex_phase = 0;
+    h->t += 1;
+    return PSGD_OK;
 }
 
 psgd_status psgd_msgd_update(psgd_handle* h, float* X, float* mom, float eta, float mu, psgd_stream stream) {

@@ -911,3 +911,126 @@ def test_group_step_of_mixed_shapes_equals_separate_steps():
     group.close()
     for h in one + many:
         h.close()
+
+
+# ---- nodes spread over processes: the three phases around the caller's two averages ------------------------------
+EXCHANGE_CASES = [  # (m, n, r, N, count, tau, kwargs)
+    (512, 256, 4, 4, 2, 3, dict()),                                        # eager, refreshes at t = 0 and 3
+    (300, 130, 5, 2, 1, 0, dict(error_form="mean")),                       # node-averaged Q in the residual, scalar paths
+    (1024, 512, 16, 4, 1, 3, dict(mode="deferred", single_pass="none")),   # two-pass form: the residual stays pending
+    (640, 256, 40, 2, 1, 3, dict(mode="deferred")),                        # tensor-core contractions and refresh sweeps
+    (300, 130, 6, 2, 2, 3, dict(transposed=True)),                         # transposed storage
+]
+
+
+@pytest.mark.parametrize("m,n,r,N,count,tau,kw", EXCHANGE_CASES)
+def test_exchange_phases_with_one_process_equal_the_step(torch_cuda, m, n, r, N, count, tau, kw):
+    """psgd_exchange_begin / _orth / _end with nothing to average in between run the same kernels on the same data as
+    psgd_step (three- or two-pass form): P~, Q, E and the warning flags agree bit for bit over steps with refreshes."""
+    torch = torch_cuda
+    from paper_2509_11254_b200 import ExchangedStack, PowerSGDPlus
+
+    a = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=5, count=count, device="cuda:0", **kw)
+    b = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=5, count=count, device="cuda:0", **kw)
+    stack = ExchangedStack([b])
+    assert stack.world == 1
+    for t in range(5):
+        G = np.stack([synth.make_gradients(2, m, n, N, step=t, matrix_id=c, seed=5) for c in range(count)])
+        if kw.get("transposed"):
+            G = np.ascontiguousarray(np.swapaxes(G, -1, -2))
+        Gd = torch.as_tensor(G, device="cuda:0")
+        a.step(Gd)
+        refreshed = stack.step([Gd])
+        assert refreshed == [tau > 0 and t % tau == 0]
+        assert a.t == b.t == t + 1
+        assert torch.equal(a.P_hat, b.P_hat) and torch.equal(a.Q, b.Q)
+        assert a.plan_info()["pending"] == b.plan_info()["pending"]
+        assert a.last_status() == b.last_status() == 0
+    a.materialize_error(); b.materialize_error()
+    assert torch.equal(a.E, b.E)
+    # a step cannot start while an iteration is open, and the phases cannot be taken out of order
+    first = torch.zeros(b.exchange_plan()[1] + 64, device="cuda:0")
+    second = torch.zeros(b.exchange_plan()[2] + 64, device="cuda:0")
+    from paper_2509_11254_b200 import PSGDError
+    with pytest.raises(PSGDError):
+        b.exchange_orth(first, second)
+    b.exchange_begin(Gd, first)
+    with pytest.raises(PSGDError):
+        b.step(Gd)
+    with pytest.raises(PSGDError):
+        b.exchange_end(second)
+    b.exchange_orth(first, second)
+    b.exchange_end(second)
+    a.step(Gd)
+    assert torch.equal(a.Q, b.Q) and b.t == 6
+    a.close(); b.close()
+
+
+@pytest.mark.parametrize("m,n,r,N,count,tau,kw", EXCHANGE_CASES)
+def test_exchange_two_halves_of_the_nodes_against_the_oracle(torch_cuda, m, n, r, N, count, tau, kw):
+    """Two handles stand for two processes, each holding N of the 2N nodes; the test averages `first` and `second`
+    between the phases (what the all-reduce does).  The result is Algorithm 2 on all 2N nodes: P~ (projector), Q and
+    every node's e_{t+1} against the oracle, and the two halves agree on P~ and Q bit for bit."""
+    torch = torch_cuda
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    dev = "cuda:0"
+    halves = [PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=9, count=count, device=dev, **kw) for _ in range(2)]
+    tr = (lambda x: np.ascontiguousarray(np.swapaxes(x, -1, -2))) if kw.get("transposed") else (lambda x: x)
+    form = kw.get("error_form", "local")
+    Q0 = np.stack([synth.init_Q(n, r, matrix_id=c, seed=9) for c in range(count)])
+    oracles = [orc.PowerSGDPlusOracle(m, n, r, 2 * N, tau, Q0[c], form) for c in range(count)]
+    for h in halves:
+        h.set_state(E=np.zeros((count, N) + ((n, m) if kw.get("transposed") else (m, n)), np.float32), Q=Q0, t=0)
+    for t in range(5):
+        G = np.stack([synth.make_gradients(2, m, n, 2 * N, step=t, matrix_id=c, seed=9) for c in range(count)])   # [count][2N][m][n]
+        rf, f1, f2 = halves[0].exchange_plan()
+        assert rf == (tau > 0 and t % tau == 0) and f2 == count * n * r and f1 == count * m * (n if rf else r)
+        firsts = [torch.zeros(f1, device=dev) for _ in halves]
+        seconds = [torch.zeros(f2, device=dev) for _ in halves]
+        for k, h in enumerate(halves):
+            h.exchange_begin(torch.as_tensor(tr(G[:, k * N:(k + 1) * N]), device=dev), firsts[k])
+        mean1 = (firsts[0] + firsts[1]) * 0.5
+        for k, h in enumerate(halves):
+            firsts[k].copy_(mean1)
+            h.exchange_orth(firsts[k], seconds[k])
+        mean2 = (seconds[0] + seconds[1]) * 0.5
+        for k, h in enumerate(halves):
+            seconds[k].copy_(mean2)
+            h.exchange_end(seconds[k])
+        assert torch.equal(halves[0].P_hat, halves[1].P_hat) and torch.equal(halves[0].Q, halves[1].Q)
+        E_parts = []
+        for h in halves:
+            assert h.last_status() == 0
+            if t == 4:
+                h.materialize_error()
+                E_parts.append(tr(h.E.cpu().numpy()))
+        for c, o in enumerate(oracles):
+            # the oracle continues from its own double-precision state: five steps of float32 drift stay within the tolerances
+            out = o.step(G[c])
+            P_ref, P_gpu = out["P_hat"], halves[0].P_hat[c].cpu().numpy().astype(np.float64)
+            assert np.abs(P_gpu.T @ P_gpu - np.eye(r)).max() <= 1e-5
+            M = out["M"]
+            gap = 1.0
+            if out["refresh"]:
+                sg = out["sigma"]
+                gap = (sg[r - 1] - sg[r]) / sg[0]
+            if gap >= GAP_MIN:
+                assert np.linalg.norm(P_gpu @ P_gpu.T - P_ref @ P_ref.T) <= (1e-4 if out["refresh"] else 2e-5) * np.sqrt(r)
+                R = P_ref.T @ P_gpu                  # the two bases differ by (nearly) a rotation at a refresh
+                assert rel_fro(halves[0].Q[c].cpu().numpy(), out["Q"] @ R) <= 2e-4
+            else:                                    # no gap at sigma_r: any basis that leaves the optimal energy behind
+                Dbar = out["Dbar"]
+                left = np.linalg.norm(Dbar - P_gpu @ (P_gpu.T @ Dbar)) ** 2
+                assert -1e-6 * np.linalg.norm(Dbar) ** 2 <= left - np.sum(out["sigma"][r:] ** 2) <= 2e-6 * np.linalg.norm(Dbar) ** 2
+                o.Q = M.mean(axis=0).T @ P_gpu       # the oracle goes on from the basis the GPU chose
+                o.E = M - np.einsum("mr,inr->imn", P_gpu, np.einsum("imn,mr->inr", M, P_gpu)) if form == "local" \
+                    else M - (P_gpu @ o.Q.T)[None]
+                out = dict(out, Q=o.Q, E=o.E)
+            # Q from its definition on the oracle's M with the GPU's basis: mean over all 2N nodes of M_i^T P~
+            assert rel_fro(halves[0].Q[c].cpu().numpy(), M.mean(axis=0).T @ P_gpu) <= 2e-4
+            if t == 4:
+                E_gpu = np.concatenate([E_parts[0][c], E_parts[1][c]], axis=0)
+                assert np.linalg.norm(E_gpu - out["E"]) <= 2e-4 * np.linalg.norm(M)
+    for h in halves:
+        h.close()
