@@ -55,6 +55,8 @@ def parse():
     ap.add_argument("--rank", type=int, default=HEADLINE_RANK, help="rank of the headline measurement")
     ap.add_argument("--mode", default="deferred", choices=["eager", "deferred"])
     ap.add_argument("--single-pass", default="auto", choices=["auto", "cluster", "none", "l2"])
+    ap.add_argument("--pending-tc", default=None, choices=["auto", "always", "never"],
+                    help="two-pass steps: fold the pending residual in on the tensor cores (default: the library's choice per rank)")
     ap.add_argument("--stacks", default="2,3,4", help="model-shaped stacks to add (workload ids), or 'none'")
     ap.add_argument("--no-sweep", action="store_true", help="only the headline rank")
     ap.add_argument("--no-e2e", action="store_true")
@@ -209,11 +211,14 @@ def roofline_entry(fam, r, step_kernel, elements, peak, peak_kind):
 # ----------------------------------------------------------------------------
 # the sweep (workload 5)
 # ----------------------------------------------------------------------------
+PENDING_TC = None      # --pending-tc: which projection folds the pending residual in (None: the library's choice)
+
+
 def sweep_point(torch, device, r, bufs, mode, single_pass, steps, min_seconds, peak, peak_kind, refresh=True):
     from paper_2509_11254_b200 import PowerSGDPlus
 
     N, m, n = bufs[0].shape[1], bufs[0].shape[2], bufs[0].shape[3]
-    h = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=5, device=device, mode=mode, single_pass=single_pass)
+    h = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=5, device=device, mode=mode, single_pass=single_pass, pending_tc=PENDING_TC)
     for s in range(5):
         h.step(bufs[s % 2])
     l0 = h.launch_count()
@@ -248,7 +253,7 @@ def stack_bench(torch, device, workload, r, N, tau, mode, single_pass, peak, pea
     shapes = synth.STACKS[workload]
     nbuf = 1 if workload == 4 else 2
     bufs = [[synth.make_gradients_torch(workload, m, n, N, c, step=b, device=device) for (m, n, c) in shapes] for b in range(nbuf)]
-    handles = [PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=1 + i, count=c, device=device, mode=mode, single_pass=single_pass)
+    handles = [PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=1 + i, count=c, device=device, mode=mode, single_pass=single_pass, pending_tc=PENDING_TC)
                for i, (m, n, c) in enumerate(shapes)]
     stack = StreamedStack(handles, device)
     for s in range(3):            # t = 0 is a refresh
@@ -383,7 +388,7 @@ def run_ours(args):
     # ---- headline: the step at the headline rank, on every replica, max over ranks ----
     from paper_2509_11254_b200 import PowerSGDPlus
 
-    h = PowerSGDPlus(m, n, r, N, refresh_period=args.refresh_period, seed=5, device=device, mode=args.mode, single_pass=args.single_pass,
+    h = PowerSGDPlus(m, n, r, N, refresh_period=args.refresh_period, seed=5, device=device, mode=args.mode, single_pass=args.single_pass, pending_tc=PENDING_TC,
                      grad_dtype=args.grad_dtype)
     for s in range(max(args.warmup, 3)):
         h.step(hbufs[s % 2])
@@ -417,7 +422,7 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": "sweep", "m": m, "n": n, "N": N, "ranks": list(SWEEP_RANKS), "headline_rank": r,
-                       "refresh_period": args.refresh_period, "mode": args.mode, "single_pass": args.single_pass, "grad_dtype": args.grad_dtype,
+                       "refresh_period": args.refresh_period, "mode": args.mode, "single_pass": args.single_pass, "pending_tc": args.pending_tc or "auto", "grad_dtype": args.grad_dtype,
                        "gradients": "low rank (s_k = 0.9^k, 256 terms) plus 5 % Gaussian noise, 2 alternating sets generated on the device",
                        "l2": "inputs (%.2f GB of G and as much of E per step) exceed L2" % (g_bytes / 1e9),
                        "parallelism": "replicas" if world > 1 else "single"},
@@ -473,7 +478,9 @@ def run_ours(args):
 
 
 def main():
+    global PENDING_TC
     args = parse()
+    PENDING_TC = args.pending_tc
     if args.impl == "reference":
         run_reference(args)
     else:

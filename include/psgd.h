@@ -93,6 +93,12 @@ typedef enum {
                                       needs no copy.  P_hat [m][r] and Q [n][r] keep their layouts.  Runs the three-pass kernels with their
                                       roles exchanged (28 bytes per element); the deferred mode and bfloat16 gradients do not apply */
 
+#define PSGD_OPT_PENDING_TC 11       /* two-pass form of the deferred mode: which projection folds in the pending residual
+                                      e = Delta - P~ Qsub^T.  0 (default): the tensor-core kernel (the rank-r product as extra MMAs,
+                                      up to 32 columns, n % 4 == 0) from the number of columns on where it is the faster one, the float32
+                                      kernel (up to 16 columns) below; 1: the tensor-core kernel wherever it fits; 2: never (more than 16
+                                      columns then take three passes) */
+
 /* buffers that psgd_debug_ptr exposes (test use only; valid until the next step) */
 #define PSGD_BUF_P_NODE 1   /* P^(i)   [count][N][m][r] */
 #define PSGD_BUF_Q_NODE 2   /* Q^(i)   [count][N][n][r] */
@@ -198,7 +204,8 @@ psgd_status psgd_debug_ptr(psgd_handle* h, int which, void** ptr, size_t* bytes)
  * holds Delta_t and the residual is still pending (deferred mode), [9] 1 if that pending residual is
  * the single-pass kernel's (padded factors in place), [10] multiprocessors of the device that was
  * current when the handle was created (148 when none was visible), [11] what ran the last
- * step: 0 the three- or two-pass kernels, 1 the cluster single-pass kernel, 2 the L2-pipelined single-pass kernel.
+ * step: 0 the three- or two-pass kernels, 1 the cluster single-pass kernel, 2 the L2-pipelined single-pass kernel,
+ * 3 the two-pass kernels with the pending residual folded in on the tensor cores (PSGD_OPT_PENDING_TC).
  */
 psgd_status psgd_plan_info(const psgd_handle* h, int* info /*HOST*/);
 

@@ -26,6 +26,7 @@ namespace {
 
 constexpr int MAX_R = 128;
 constexpr int MAX_L = 160;  // widest refresh block
+constexpr int PENDING_TC_MIN_R = 8;    // above this many columns the pending-residual projection runs on the tensor cores by default
 constexpr int REFRESH_F32_TAIL = 4;   // float32-accurate sweeps that end a refresh whose early sweeps ran in TF32
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -38,6 +39,7 @@ struct Layout {
     size_t rtP, rtQ;                                          // tensor-core residual (r > 16) only
     size_t Pold, dpart;                                       // stopping test of the refresh
     size_t ptQ;                                               // tensor-core projection: split transposed Q
+    size_t ppP, ppQ;                                          // ... of the two-pass deferred mode: images of P~_prev and Qsub
     size_t sPpart, sCnt, sGram;                               // L2-pipelined single-pass kernel: per-unit partial products, counters and flags, Gram partials
 };
 
@@ -65,6 +67,8 @@ struct psgd_handle {
     size_t gpart_floats = 0;
     bool grad_bf16 = false;       // G arrives as bfloat16
     bool ptc_ok = false;          // projections of more than 16 columns on the tensor cores
+    bool ppt_ok = false;          // pending-residual projection (two-pass deferred mode) on the tensor cores
+    int pend_tc = 0;              // PSGD_OPT_PENDING_TC: 0 where it is the faster form, 1 wherever it fits, 2 never
     int ptc_ncp = 0;
     bool rtc_ok = false;          // ranks above 16 with 16-byte row strides: residual update on the tensor cores
     int rtc_KP = 0;
@@ -99,6 +103,7 @@ struct psgd_handle {
     bool transposed = false;      // PSGD_OPT_TRANSPOSED: G and E are stored as [n][m] (the transpose of the m x n problem)
     int t_S = 1, t_rpc = 0;       // row chunks of the contraction over the n stored rows (transposed storage)
     int step_kernel = 0;          // what ran the last step: 0 three-/two-pass kernels, 1 cluster kernel, 2 L2-pipelined kernel
+    bool ran_pending_tc = false;  // the projection of the step in flight folded the pending residual in on the tensor cores
     int ex_phase = 0;             // psgd_exchange_*: 0 between steps, 1 after _begin, 2 after _orth
     bool ex_refresh = false;      // the step in flight is a refresh
     int sm_count = 0;             // multiprocessors of the device that was current when the handle was created
@@ -194,9 +199,16 @@ void plan(psgd_handle* h) {
     }
     // ---- projection on the tensor cores (r > 16, or refresh blocks of 17..128 columns) ----
     h->ptc_ok = (h->r > 16 || ell > 16) && h->n % 4 == 0;
-    if (h->ptc_ok) {
-        h->ptc_ncp = (int)align_up(std::min<size_t>(128, std::max(r, ell)), 16);
-        L.ptQ = take(3 * cnt * (size_t)h->ptc_ncp * std::max(m, n) * 4);   // split Q^T (projection) or P~^T (back-projection)
+    // ... and the projection of the two-pass deferred mode (pending residual folded in as a tensor-core product), up to 32 columns
+    h->ppt_ok = h->mode == 1 && h->r <= 32 && h->n % 4 == 0 && !h->transposed && !h->grad_bf16 && h->power_steps == 1 && h->pend_tc != 2;
+    h->ptc_ncp = h->ptc_ok ? (int)align_up(std::min<size_t>(128, std::max(r, ell)), 16) : 0;
+    if (h->ptc_ok || h->ppt_ok) {
+        const size_t ncp = std::max<size_t>(h->ptc_ncp, h->ppt_ok ? align_up(r, 16) : 0);
+        L.ptQ = take(3 * cnt * ncp * align_up(std::max(m, n), TC_BK) * 4);   // split Q^T (projection) or P~^T (back-projection)
+    }
+    if (h->ppt_ok) {
+        L.ppP = take(cnt * align_up(m, TC_BM) * 2 * TC_BK * 4);         // two terms of P~_prev, one image per 128-row block
+        L.ppQ = take(cnt * N * align_up(n, TC_BK) * 3 * TC_BK * 4);     // three terms of Qsub, one image per 32-column block
     }
     // ---- residual update on the tensor cores: split (head + tail) padded copies of P~ and Q_i ----
     h->rtc_ok = h->r > 16 && h->n % 4 == 0;
@@ -484,15 +496,15 @@ bool launch_project_tc(Launcher& L, const float* A, const float* B, float* Mout,
     const int Ncp = (int)align_up(r, 16);
     if (!h->ptc_ok || Ncp > h->ptc_ncp || r > 128 || !aligned16(A) || (B && !aligned16(B)) || (Mout && !aligned16(Mout))) return false;
     const int mats = count * nodes;
-    float* Qt = (float*)(h->ws + h->lay.ptQ);
-    const size_t tot = (size_t)count * Ncp * n;
+    float* Qimg = (float*)(h->ws + h->lay.ptQ);
+    const int KB = ceil_div(n, TC_BK);
+    const size_t tot = (size_t)count * KB * Ncp * TC_BK;
     L.begin(PSGD_K_PROJECT);
-    k_split_pad_t<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Q, Qt, n, r, Ncp, count, skip);
+    k_split_img_t<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Q, Qimg, n, r, Ncp, KB, count, skip);
     L.end();
-    CUtensorMap tA, tB, tQ[3];
+    CUtensorMap tA, tB;
     bool ok = make_tile_map(h, &tA, A, n, rows, mats, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) &&
               make_tile_map(h, &tB, B ? B : A, n, rows, mats, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B);
-    for (int t = 0; t < 3 && ok; ++t) ok = make_tile_map(h, &tQ[t], Qt + t * tot, n, Ncp, count, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) {
         snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
         L.status = PSGD_E_CUDA;
@@ -500,9 +512,48 @@ bool launch_project_tc(Launcher& L, const float* A, const float* B, float* Mout,
     }
     ProjTcArgs a{B ? Mout : nullptr, P, rows, n, r, Ncp, proj_tc_nh(Ncp), B ? 1 : 0, nodes, (int*)(h->ws + h->lay.flags), skip};
     size_t smem = proj_tc_smem_bytes(Ncp);
-    set_smem_attr((const void*)k_project_tc, smem);
+    set_smem_attr((const void*)k_project_tc<false>, smem);
     L.begin(PSGD_K_PROJECT);
-    k_project_tc<<<dim3(ceil_div(rows, TC_BM), mats), PT_THREADS, smem, L.st>>>(tA, tB, tQ[0], tQ[1], tQ[2], a);
+    k_project_tc<false><<<dim3(ceil_div(rows, TC_BM), mats), PT_THREADS, smem, L.st>>>(tA, tB, Qimg, a);
+    L.end();
+    return true;
+}
+
+// The projection of the two-pass deferred mode on the tensor cores (up to 32 columns): P = (G + (Delta_prev - P~_prev Qsub^T)) Q,
+// M stored over Delta_prev.  False when the shape or the pointers do not allow it (nothing has been launched then).
+bool launch_project_pending_tc(Launcher& L, const float* G, float* E, const float* Q, float* P, const float* Pprev, const float* Qsub,
+                               int qsub_per_node, int rows, int n, int r, int nodes, int count) {
+    psgd_handle* h = L.h;
+    if (!h->ppt_ok || r > 32 || !aligned16(G) || !aligned16(E)) return false;
+    const int Ncp = (int)align_up(r, 16);
+    const int mats = count * nodes, qmats = qsub_per_node ? mats : count;
+    const int KB = ceil_div(n, TC_BK), RT = ceil_div(rows, TC_BM);
+    float* Qimg = (float*)(h->ws + h->lay.ptQ);
+    float* Pimg = (float*)(h->ws + h->lay.ppP);
+    float* QSimg = (float*)(h->ws + h->lay.ppQ);
+    CUtensorMap tA, tB;
+    if (!make_tile_map(h, &tA, G, n, rows, mats, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tile_map(h, &tB, E, n, rows, mats, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_128B)) {
+        snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
+        L.status = PSGD_E_CUDA;
+        return true;
+    }
+    const size_t tq = (size_t)count * KB * Ncp * TC_BK, tp = (size_t)count * RT * TC_BM * TC_BK, ts = (size_t)qmats * KB * 32 * TC_BK;
+    L.begin(PSGD_K_PROJECT);
+    k_split_img_t<<<(unsigned)((tq + 255) / 256), 256, 0, L.st>>>(Q, Qimg, n, r, Ncp, KB, count, nullptr);
+    L.end();
+    L.begin(PSGD_K_PROJECT);
+    k_split_img_rows<<<(unsigned)((tp + 255) / 256), 256, 0, L.st>>>(Pprev, Pimg, rows, r, TC_BM, 2, count);
+    L.end();
+    L.begin(PSGD_K_PROJECT);
+    k_split_img_rows<<<(unsigned)((ts + 255) / 256), 256, 0, L.st>>>(Qsub, QSimg, n, r, 32, 3, qmats);
+    L.end();
+    ProjTcArgs a{E, P, rows, n, r, Ncp, proj_tc_nh(Ncp, true), 1, nodes, (int*)(h->ws + h->lay.flags), nullptr,
+                 Pimg, QSimg, qsub_per_node, ceil_div(r, 8)};
+    size_t smem = proj_tc_smem_bytes(Ncp, true);
+    set_smem_attr((const void*)k_project_tc<true>, smem);
+    L.begin(PSGD_K_PROJECT);
+    k_project_tc<true><<<dim3(RT, mats), PT_THREADS_PEND, smem, L.st>>>(tA, tB, Qimg, a);
     L.end();
     return true;
 }
@@ -718,6 +769,19 @@ void tail(Launcher& L, psgd_handle* h, float* D_hat, bool defer = false) {
 }
 
 // ---- SSP-Comp (Algorithm 1, first function) ------------------------------------
+// Which projection carries the pending residual of the two-pass deferred mode.  The tensor-core form does not depend on the
+// number of columns; the float32 form costs 2r multiply-adds per element and is the faster one only for few columns.
+bool pending_on_tc(const psgd_handle* h) {
+    if (!h->ppt_ok) return false;
+    return h->pend_tc == 1 || h->r > PENDING_TC_MIN_R;
+}
+// SSP steps of the deferred mode in two passes (the residual stays pending in E): up to 16 columns, or up to 32 on the tensor cores
+bool two_pass_ok(const psgd_handle* h) {
+    return h->mode == 1 && h->power_steps == 1 && !h->grad_bf16 && (h->r <= 16 || pending_on_tc(h));
+}
+
+void materialize(Launcher& L, psgd_handle* h);
+
 // P_i = (G_i + e_i) Q_{t-1} for every node, M_i left in the E buffer
 void ssp_project(Launcher& L, psgd_handle* h, const void* Gv) {
     char* ws = h->ws;
@@ -727,8 +791,17 @@ void ssp_project(Launcher& L, psgd_handle* h, const void* Gv) {
     const float* G = (const float*)Gv;
     if (h->pending) {        // two-pass deferred mode: E holds Delta_{t-1}; P~_{t-1} and Q_i of the last step are still in place
         float* Qnode = (float*)(ws + h->lay.Qnode);
-        launch_project_pending(L, G, h->E, h->Q, Pnode, Phat, h->error_form == 0 ? Qnode : h->Q, h->error_form == 0 ? 1 : 0,
-                               m, n, r, N, cnt, h->vec4);
+        const float* Qsub = h->error_form == 0 ? Qnode : h->Q;
+        const int per_node = h->error_form == 0 ? 1 : 0;
+        h->ran_pending_tc = pending_on_tc(h) && launch_project_pending_tc(L, G, h->E, h->Q, Pnode, Phat, Qsub, per_node, m, n, r, N, cnt);
+        if (!h->ran_pending_tc) {
+            if (r > 16) {      // no float32 kernel folds a residual of more than 16 columns in: form it first (a third pass)
+                materialize(L, h);
+                ssp_project(L, h, Gv);
+                return;
+            }
+            launch_project_pending(L, G, h->E, h->Q, Pnode, Phat, Qsub, per_node, m, n, r, N, cnt, h->vec4);
+        }
     } else if (h->grad_bf16) {      // M = G + E formed in the E buffer first (10 B/element), then the projection reads M
         launch_add_mean(L, Gv, true, h->E, nullptr, (size_t)m * n, N, cnt, PSGD_K_PROJECT);
         launch_project(L, h->E, nullptr, nullptr, h->Q, Pnode, m, n, r, N, cnt, h->vec4);
@@ -1184,7 +1257,7 @@ void materialize(Launcher& L, psgd_handle* h) {
 // factorises the same averaged P (or runs SVD-Comp on the same averaged Delta) and gets the same P~ bit for bit.
 // Deferred mode runs the two-pass form (the residual stays pending between steps); the single-pass kernels fuse the
 // node mean and have no place for an exchange.
-bool ex_two_pass(const psgd_handle* h) { return h->mode == 1 && h->r <= 16 && !h->grad_bf16; }
+bool ex_two_pass(const psgd_handle* h) { return two_pass_ok(h); }
 
 void exchange_begin(Launcher& L, psgd_handle* h, const void* G, float* out, bool refresh) {
     char* ws = h->ws;
@@ -1299,6 +1372,7 @@ psgd_status do_step(psgd_handle* h, const void* G, float* P_hat, float* D_hat, p
     }
     const bool one_pass = h->mode == 1 && !refresh && aligned16(G) && h->power_steps == 1;
     bool done = false;
+    h->ran_pending_tc = false;
     if (one_pass && h->stream_ok && h->s_grid != 0) {
         if (h->pending && !h->pending_fused) materialize(L, h);   // Delta_t left by a two-pass step: no padded factors for it
         done = stream_ssp(L, h, G);
@@ -1321,13 +1395,13 @@ psgd_status do_step(psgd_handle* h, const void* G, float* P_hat, float* D_hat, p
         // projection forms e_{t+1} = Delta_t - P~_t Q_i^T on the fly (16 instead of 24 bytes per element).
         // A refresh step needs the true residual before it (SVD-Comp works on g + e), but may leave its own residual pending
         // like any other step of that mode.
-        const bool two_pass = h->mode == 1 && h->r <= 16 && h->power_steps == 1 && !h->grad_bf16;
+        const bool two_pass = two_pass_ok(h);
         if (!two_pass || refresh) materialize(L, h);
         if (refresh) svd(L, h, G); else ssp(L, h, G);
         tail(L, h, D_hat, two_pass);
         h->tacc_identity = true;
         h->qpad_valid = false;
-        h->step_kernel = 0;
+        h->step_kernel = h->ran_pending_tc ? 3 : 0;
     }
     if (L.status != PSGD_OK) return L.status;
     if (P_hat) {
@@ -1375,6 +1449,7 @@ psgd_status psgd_set_option(psgd_handle* h, int option, int value) {
         case PSGD_OPT_GRAD_BF16: if (value != 0 && value != 1) return PSGD_E_INVALID; h->grad_bf16 = value != 0; break;
         case PSGD_OPT_TRANSPOSED: if (value != 0 && value != 1) return PSGD_E_INVALID; h->transposed = value != 0; break;
         case PSGD_OPT_SINGLE_PASS: if (value < 0 || value > 3) return PSGD_E_INVALID; h->single_pass_kernel = value; break;
+        case PSGD_OPT_PENDING_TC: if (value < 0 || value > 2) return PSGD_E_INVALID; h->pend_tc = value; break;
         default: return PSGD_E_INVALID;
     }
     plan(h);
@@ -1440,6 +1515,7 @@ psgd_status psgd_exchange_begin(psgd_handle* h, const void* G, int force_refresh
     if (h->ex_phase != 0 || h->power_steps != 1 || !aligned16(first)) return PSGD_E_INVALID;
     Launcher L{h, (cudaStream_t)stream};
     h->ex_refresh = force_refresh || (h->tau > 0 && h->t % h->tau == 0);
+    h->ran_pending_tc = false;
     exchange_begin(L, h, G, first, h->ex_refresh);
     if (L.status != PSGD_OK) return L.status;
     h->ex_phase = 1;
@@ -1467,7 +1543,7 @@ psgd_status psgd_exchange_end(psgd_handle* h, const float* second, float* P_hat,
     Launcher L{h, st};
     exchange_end(L, h, second, D_hat);
     if (L.status != PSGD_OK) return L.status;
-    h->step_kernel = 0;
+    h->step_kernel = h->ran_pending_tc ? 3 : 0;
     if (P_hat)
         PSGD_CUDA(h, cudaMemcpyAsync(P_hat, h->ws + h->lay.Phat, (size_t)h->count * h->m * h->r * 4, cudaMemcpyDeviceToDevice, st));
     h->ex_phase = 0;
@@ -1719,5 +1795,11 @@ psgd_status psgd_group_destroy(psgd_group* g) {
 }
 
 }  // extern "C"
+
+#ifdef PSGD_PTC_TIMING
+extern "C" int psgd_debug_ptc_times(unsigned* host /*[12][512]*/) {
+    return (int)cudaMemcpyFromSymbol(host, psgd::g_ptc_t, sizeof(unsigned) * 12 * 512);
+}
+#endif
 
 #include "psgd_noalloc.cu"

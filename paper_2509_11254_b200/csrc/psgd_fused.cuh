@@ -105,7 +105,11 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
     unsigned ok;
     asm volatile(
         "{\n.reg .pred p;\n"
+#ifdef PSGD_MBAR_TEST_WAIT
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+#else
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+#endif
         "selp.u32 %0, 1, 0, p;\n}\n"
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
@@ -118,6 +122,37 @@ __device__ __forceinline__ void mbar_wait(unsigned bar, unsigned parity, int* fl
         if (mbar_try_wait(bar, parity)) return;
     dead = true;
     atomicOr(flags, FU_W_TIMEOUT);
+}
+// For a role played by a single thread whose barrier has usually completed already: a non-blocking test first.
+__device__ __forceinline__ void mbar_wait_ready(unsigned bar, unsigned parity, int* flags, bool& dead) {
+    unsigned ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (!ok) mbar_wait(bar, parity, flags, dead);
+}
+// The same wait for a whole warp (all 32 lanes must call it): lane 0 polls, pausing between polls, so that a waiting
+// warp puts one request at a time on the barrier instead of 32 (many warps polling at full rate slow down every other
+// barrier operation of the CTA, the single MMA-issuing thread's first of all); once the phase has completed every lane
+// observes it itself with one more try_wait, which returns at once and gives that lane its own acquire.
+__device__ __forceinline__ void mbar_wait_warp(unsigned bar, unsigned parity, int* flags, bool& dead) {
+    if (dead) return;                        // (uniform across the warp: set from lane 0 below)
+    int gave_up = 0;
+    if ((threadIdx.x & 31) == 0) {
+        bool ok = false;
+        for (unsigned it = 0; it < FU_WAIT_LIMIT && !ok; ++it) {
+            ok = mbar_try_wait(bar, parity);
+            if (!ok) __nanosleep(40);
+        }
+        if (!ok) { gave_up = 1; atomicOr(flags, FU_W_TIMEOUT); }
+    }
+    gave_up = __shfl_sync(0xffffffffu, gave_up, 0);
+    if (gave_up) { dead = true; return; }
+#ifndef PSGD_MBAR_NO_REWAIT
+    (void)mbar_try_wait(bar, parity);
+#endif
 }
 // TMA: one tile {x: columns, y: rows, z: (matrix, node)} of a rank-3 tensor map into shared memory.
 // x must be a multiple of 4 floats (16 bytes); coordinates past the extents read zeros.

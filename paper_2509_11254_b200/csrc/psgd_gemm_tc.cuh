@@ -456,6 +456,7 @@ namespace psgd {
 // adder warps that the accumulators of that K block can be read.
 // ---------------------------------------------------------------------------------------------
 constexpr int PT_THREADS = 576;   // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-9: converters, warps 10-17: adders + epilogue
+constexpr int PT_THREADS_PEND = 608;   // ... and warp 18: issues the MMAs of the pending-residual correction
 constexpr int BT_MAXG = 8;        // 8-column groups per thread: (Ncp / 2) / 8 for Ncp <= 128
 
 // Adder warps of the projection and back-projection kernels: adds the accumulators of one K block (set / head
@@ -520,18 +521,31 @@ struct ProjTcArgs {
     int nodes;        // matrices per Q
     int* flags;
     const int* skip;
+    // pending residual (two-pass deferred mode): M = A + (B - P~_prev Qsub^T), the product formed by the tensor core
+    const float* Pimg;    // [count][row tiles][2][128][32]: two TF32 terms of P~_prev, shared-memory image (k_split_img_rows)
+    const float* QSimg;   // [mats or count][KB][3][32][32]: three terms of Qsub, one image per K block
+    int qs_per_node;      // Qsub is per (matrix, node) (1) or per matrix (0)
+    int ksteps;           // ceil(r / 8): MMAs along the rank
 };
+constexpr int PT_CORR_COLS = 96;                     // one correction accumulator: [head | small | small] x 32 columns
+constexpr unsigned PT_QS_BYTES = 3 * 32 * TC_BK * 4; // three terms of a 32-row block of Qsub
+constexpr unsigned PT_PIMG_BYTES = 2 * TC_BM * TC_BK * 4;
 
 // Two shared-memory rings, as in the back-projection below: stages of 32 KB for the tiles of A and B (M and its second
 // TF32 term are formed in place) and a short ring for the three terms of Q^T.
+// (pend: every stage of the short ring also holds the three terms of a block of Qsub, and the two terms of P~_prev stay resident)
 __host__ __device__ inline int proj_tc_nm(int Ncp) { return 3 * Ncp <= 256 ? 3 : 2; }
-__host__ __device__ inline int proj_tc_nh(int Ncp) {
-    const long long left = 224ll * 1024 - 1024 - 512 - (long long)proj_tc_nm(Ncp) * 3 * Ncp * TC_BK * 4;
+__host__ __device__ inline long long proj_tc_short_bytes(int Ncp, bool pend) {
+    return 3ll * Ncp * TC_BK * 4 + (pend ? (long long)PT_QS_BYTES : 0);
+}
+__host__ __device__ inline int proj_tc_nh(int Ncp, bool pend = false) {
+    const long long left = 224ll * 1024 - 1024 - 512 - proj_tc_nm(Ncp) * proj_tc_short_bytes(Ncp, pend) - (pend ? (long long)PT_PIMG_BYTES : 0);
     const int nh = (int)(left / (2 * TC_BM * TC_BK * 4));
     return nh > 6 ? 6 : nh;
 }
-__host__ __device__ inline size_t proj_tc_smem_bytes(int Ncp) {
-    return (size_t)proj_tc_nh(Ncp) * 2 * TC_BM * TC_BK * 4 + (size_t)proj_tc_nm(Ncp) * 3 * Ncp * TC_BK * 4 + 1024 + 512;
+__host__ __device__ inline size_t proj_tc_smem_bytes(int Ncp, bool pend = false) {
+    return (size_t)proj_tc_nh(Ncp, pend) * 2 * TC_BM * TC_BK * 4 + (size_t)(proj_tc_nm(Ncp) * proj_tc_short_bytes(Ncp, pend)) +
+           (pend ? PT_PIMG_BYTES : 0) + 1024 + 512;
 }
 
 // Q [count][n][r] -> Qt[t][count][Ncp][n], t = 0, 1, 2: the transposed factor split exactly into three TF32 terms,
@@ -552,9 +566,83 @@ __global__ void k_split_pad_t(const float* Q, float* Qt, int n, int r, int Ncp, 
     Qt[2 * tot + idx] = r1 - mm;
 }
 
-__global__ void __launch_bounds__(PT_THREADS, 1)
-k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-             const __grid_constant__ CUtensorMap tmQ0, const __grid_constant__ CUtensorMap tmQ1, const __grid_constant__ CUtensorMap tmQ2,
+// Q [count][n][r] -> Qimg[count][KB][t][Ncp][32], t = 0, 1, 2: the same three exact terms, laid out as the shared-memory
+// image of one K block after the other (rows of 128 bytes, 128-byte swizzle: the 16-byte unit u of row k sits at unit
+// u ^ (k & 7)), so that ONE untiled bulk copy of 3 Ncp 128 bytes brings what a K block needs.  Columns beyond n and rows
+// k >= r are zero.  One thread per (matrix, K block, k, column).
+__global__ void k_split_img_t(const float* Q, float* Qimg, int n, int r, int Ncp, int KB, int count, const int* skip) {
+    if (skip && *skip) return;
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t per_kb = (size_t)Ncp * TC_BK, tot = per_kb * KB * count;
+    if (idx >= tot) return;
+    const int c = (int)(idx / (per_kb * KB));
+    const int kb = (int)((idx / per_kb) % KB);
+    const int k = (int)((idx % per_kb) / TC_BK), cc = (int)(idx % TC_BK);
+    const int col = kb * TC_BK + cc;
+    float x = (k < r && col < n) ? Q[((size_t)c * n + col) * r + k] : 0.f;
+    float h = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
+    float r1 = x - h;
+    float mm = __uint_as_float(__float_as_uint(r1) & 0xFFFFE000u);
+    float* blk = Qimg + ((size_t)c * KB + kb) * 3 * per_kb;
+    const size_t o = (size_t)k * TC_BK + ((((cc >> 2) ^ (k & 7)) << 2) | (cc & 3));
+    blk[o] = h;
+    blk[per_kb + o] = mm;
+    blk[2 * per_kb + o] = r1 - mm;
+}
+// X [mats][rows][r] -> img[mats][ceil(rows / TR)][T][TR][32]: blocks of TR rows as K-major shared-memory images (rows of 128
+// bytes holding columns 0..31, zero beyond r and beyond `rows`; 128-byte swizzle).  T = 3: the three exact TF32 terms;
+// T = 2: head and the rest rounded to the nearest TF32 number.  One thread per (matrix, row, column).
+__global__ void k_split_img_rows(const float* X, float* img, int rows, int r, int TR, int T, int mats) {
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int tiles = (rows + TR - 1) / TR;
+    const size_t per_mat = (size_t)tiles * TR * TC_BK, tot = per_mat * mats;
+    if (idx >= tot) return;
+    const int mt = (int)(idx / per_mat);
+    const size_t w = idx % per_mat;
+    const int tile = (int)(w / ((size_t)TR * TC_BK)), rr = (int)((w / TC_BK) % TR), k = (int)(w % TC_BK);
+    const int row = tile * TR + rr;
+    const float x = (row < rows && k < r) ? X[((size_t)mt * rows + row) * r + k] : 0.f;
+    const float h = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
+    const float r1 = x - h;
+    float* blk = img + ((size_t)mt * tiles + tile) * T * TR * TC_BK;
+    const size_t o = (size_t)rr * TC_BK + ((((k >> 2) ^ (rr & 7)) << 2) | (k & 3));
+    blk[o] = h;
+    if (T == 2) {
+        blk[(size_t)TR * TC_BK + o] = __uint_as_float((__float_as_uint(r1) + 0x1000u) & 0xFFFFE000u);
+    } else {
+        const float mm = __uint_as_float(__float_as_uint(r1) & 0xFFFFE000u);
+        blk[(size_t)TR * TC_BK + o] = mm;
+        blk[2 * (size_t)TR * TC_BK + o] = r1 - mm;
+    }
+}
+__device__ __forceinline__ void tmem_ld16(unsigned taddr, unsigned (&v)[16]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void bulk_load_1d(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// PEND (two-pass deferred mode, up to 32 columns): the tile of B holds Delta_{t-1} and M = A + (B - P~_prev Qsub^T).  The
+// rank-r product of a K block, C = P~_prev[128 rows] Qsub[32 columns]^T, is formed by the tensor core into one of two
+// correction accumulators before the converters need it (P~_prev as two TF32 terms resident in shared memory, the block of
+// Qsub as three terms in the short ring: h x [h|m|l] and m x [h|m], `ksteps` pairs of MMAs).  The converters then work one
+// accumulator row per lane: they read C with tcgen05.ld, form M in the (swizzled, hence conflict-free) tile and its second
+// term, and after a barrier among themselves write the tile of M back to HBM with the row-contiguous mapping.
+#ifdef PSGD_PTC_TIMING
+// Per-K-block time stamps of CTA (0, 0) (instrumented builds only): [event][K block], SM clock, low 32 bits.
+__device__ unsigned g_ptc_t[12][512];
+#define PTC_STAMP(ev, kb) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (kb) < 512) g_ptc_t[ev][kb] = (unsigned)clock64(); } while (0)
+#else
+#define PTC_STAMP(ev, kb) do { } while (0)
+#endif
+
+template <bool PEND>
+__global__ void __launch_bounds__(PEND ? PT_THREADS_PEND : PT_THREADS, 1)
+k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const float* __restrict__ Qimg,
              ProjTcArgs a) {
     extern __shared__ __align__(16) unsigned char pt_smem_raw[];
     if (a.skip && *a.skip) return;
@@ -563,28 +651,35 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     constexpr unsigned A_BYTES = TC_BM * TC_BK * 4;
     constexpr unsigned LONG_BYTES = 2 * A_BYTES;               // [A tile -> M (head)][B tile -> second term]
     const unsigned B_BYTES = (unsigned)a.Ncp * TC_BK * 4;
-    const unsigned SHORT_BYTES = 3 * B_BYTES;                  // h, m, l of Q^T
+    const unsigned SHORT_BYTES = 3 * B_BYTES + (PEND ? PT_QS_BYTES : 0u);   // h, m, l of Q^T [, h, m, l of the block of Qsub]
     const bool wide = 3 * a.Ncp <= 256;
     const int NM = proj_tc_nm(a.Ncp);
-    const int NH = a.nh, NB = wide ? min(4, 512 / (3 * a.Ncp)) : min(3, (512 - 2 * a.Ncp) / a.Ncp);
+    const int CORR = PEND ? 2 * PT_CORR_COLS : 0;              // tensor-memory columns of the two correction accumulators
+    const int NH = a.nh, NB = wide ? min(4, (512 - CORR) / (3 * a.Ncp)) : min(3, (512 - 2 * a.Ncp) / a.Ncp);
     unsigned char* short_base = base + (size_t)NH * LONG_BYTES;
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(short_base + (size_t)NM * SHORT_BYTES);
+    unsigned char* pimg_base = short_base + (size_t)NM * SHORT_BYTES;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(pimg_base + (PEND ? PT_PIMG_BYTES : 0u));
     const unsigned bar_hfull = smem_u32(bars), bar_conv = bar_hfull + 8 * NH, bar_done = bar_conv + 8 * NH;
     const unsigned bar_bfull = bar_done + 8 * NH, bar_free = bar_bfull + 8 * NM, bar_acc = bar_free + 8 * NB;
-    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 3 * NH + NM + NB + 1);
-    const unsigned ring_u32 = smem_u32(base), short_u32 = smem_u32(short_base);
+    const unsigned bar_stored = bar_acc + 8, bar_corr = bar_stored + 8 * NH, bar_cfree = bar_corr + 16, bar_pfull = bar_cfree + 16;
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 4 * NH + NM + NB + 1 + 5);
+    const unsigned ring_u32 = smem_u32(base), short_u32 = smem_u32(short_base), pimg_u32 = smem_u32(pimg_base);
 
     const int rt = blockIdx.x, mat = blockIdx.y;
     const int qz = mat / a.nodes;
     const int KB = (a.n + TC_BK - 1) / TC_BK;
     unsigned ncols = 32;
-    while ((int)ncols < (wide ? NB * 3 : NB + 2) * a.Ncp) ncols <<= 1;
+    while ((int)ncols < CORR + (wide ? NB * 3 : NB + 2) * a.Ncp) ncols <<= 1;
 
     if (tid == 0) {
-        for (int s = 0; s < NH; ++s) { mbar_init(bar_hfull + 8 * s, 1); mbar_init(bar_conv + 8 * s, 8); mbar_init(bar_done + 8 * s, 1); }
+        for (int s = 0; s < NH; ++s) {
+            mbar_init(bar_hfull + 8 * s, 1); mbar_init(bar_conv + 8 * s, 4); mbar_init(bar_done + 8 * s, 1); mbar_init(bar_stored + 8 * s, 4);
+        }
         for (int s = 0; s < NM; ++s) mbar_init(bar_bfull + 8 * s, 1);
         for (int b = 0; b < NB; ++b) mbar_init(bar_free + 8 * b, 8);
         mbar_init(bar_acc, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(bar_corr + 8 * b, 1); mbar_init(bar_cfree + 8 * b, 4); }
+        mbar_init(bar_pfull, 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     if (warp == 1) {
@@ -594,7 +689,8 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-    const unsigned tmem = *tmem_slot;      // wide: set b at 3 b Ncp; else two small accumulators at 0, head b at (2 + b) Ncp
+    const unsigned tmem_all = *tmem_slot;  // pend: correction accumulators at 0 and 96, the rest behind them
+    const unsigned tmem = tmem_all + (unsigned)CORR;   // wide: set b at 3 b Ncp; else two small accumulators at 0, head b at (2 + b) Ncp
     bool dead = false;
     // K block j is "done" (all its MMAs have completed) in phase j / NH of bar_done[j % NH]
     auto wait_done = [&](int j) { mbar_wait(bar_done + 8 * (j % NH), (unsigned)((j / NH) & 1), a.flags, dead); };
@@ -603,10 +699,19 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         // ---- TMA producer: tiles of A and B run NH - NM K blocks ahead of the terms of Q^T ----
         if (lane == 0) {
             const int lead = NH - NM;
+            if (PEND) {
+                mbar_expect_tx(bar_pfull, PT_PIMG_BYTES);
+                bulk_load_1d(pimg_u32, a.Pimg + ((size_t)qz * gridDim.x + rt) * (PT_PIMG_BYTES / 4), PT_PIMG_BYTES, bar_pfull);
+            }
+            const float* qs_src = PEND ? a.QSimg + (size_t)(a.qs_per_node ? mat : qz) * KB * (PT_QS_BYTES / 4) : nullptr;
             auto issue_ab = [&](int j) {
                 const int s = j % NH;
-                if (j >= NH) wait_done(j - NH);
+                if (j >= NH) {
+                    wait_done(j - NH);
+                    if (PEND) mbar_wait(bar_stored + 8 * s, (unsigned)(((j - NH) / NH) & 1), a.flags, dead);   // its M has left for HBM
+                }
                 const unsigned dst = ring_u32 + s * LONG_BYTES, bar = bar_hfull + 8 * s;
+                PTC_STAMP(0, j);
                 mbar_expect_tx(bar, (a.has_b ? 2u : 1u) * A_BYTES);
                 tma_load_3d_sw(dst, &tmA, j * TC_BK, rt * TC_BM, mat, bar);
                 if (a.has_b) tma_load_3d_sw(dst + A_BYTES, &tmB, j * TC_BK, rt * TC_BM, mat, bar);
@@ -617,25 +722,31 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 const int s = kb % NM;
                 if (kb >= NM) wait_done(kb - NM);
                 const unsigned dst = short_u32 + s * SHORT_BYTES, bar = bar_bfull + 8 * s;
-                mbar_expect_tx(bar, 3u * B_BYTES);
-                tma_load_3d_sw(dst, &tmQ0, kb * TC_BK, 0, qz, bar);
-                tma_load_3d_sw(dst + B_BYTES, &tmQ1, kb * TC_BK, 0, qz, bar);
-                tma_load_3d_sw(dst + 2 * B_BYTES, &tmQ2, kb * TC_BK, 0, qz, bar);
+                mbar_expect_tx(bar, SHORT_BYTES);
+                bulk_load_1d(dst, Qimg + ((size_t)qz * KB + kb) * (3u * B_BYTES / 4), 3u * B_BYTES, bar);
+                if (PEND) bulk_load_1d(dst + 3u * B_BYTES, qs_src + (size_t)kb * (PT_QS_BYTES / 4), PT_QS_BYTES, bar);
             }
         }
     } else if (warp == 1) {
-        // ---- MMA issuer ----
+        // ---- MMA issuer: one thread, so every instruction of its loop is on the critical path of the whole CTA.  Ring
+        //      positions and barrier parities are carried along as counters (no division), descriptors are offsets from
+        //      those of stage 0 (the address field holds addr >> 4 and shared memory ends below 2^18). ----
         if (lane == 0) {
             const unsigned id1 = tc_idesc(a.Ncp), id2 = tc_idesc(2 * a.Ncp), id3 = tc_idesc(wide ? 3 * a.Ncp : a.Ncp);
+            const unsigned long long dA0 = tc_smem_desc(ring_u32), dS0 = tc_smem_desc(short_u32);
+            const unsigned long long long_step = LONG_BYTES >> 4, short_step = SHORT_BYTES >> 4;
+            const unsigned long long a_off = A_BYTES >> 4, b_off = B_BYTES >> 4;
+            int sh = 0, phh = 0, sm = 0, phm = 0, hb = 0, phb = 1;     // kb % NH, (kb / NH) & 1, ... ; phb: parity of kb / NB - 1
             for (int kb = 0; kb < KB; ++kb) {
-                const int sh = kb % NH, sm = kb % NM, hb = kb % NB;
-                mbar_wait(bar_conv + 8 * sh, (unsigned)((kb / NH) & 1), a.flags, dead);
-                mbar_wait(bar_bfull + 8 * sm, (unsigned)((kb / NM) & 1), a.flags, dead);
-                if (kb >= NB) mbar_wait(bar_free + 8 * hb, (unsigned)((kb / NB - 1) & 1), a.flags, dead);   // registers took its last content
+                PTC_STAMP(10, kb);
+                mbar_wait_ready(bar_conv + 8 * sh, (unsigned)phh, a.flags, dead);
+                PTC_STAMP(11, kb);
+                mbar_wait_ready(bar_bfull + 8 * sm, (unsigned)phm, a.flags, dead);
+                if (kb >= NB) mbar_wait_ready(bar_free + 8 * hb, (unsigned)phb, a.flags, dead);   // registers took its last content
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-                const unsigned lb = ring_u32 + sh * LONG_BYTES, sb = short_u32 + sm * SHORT_BYTES;
-                const unsigned long long dAh = tc_smem_desc(lb), dAm = tc_smem_desc(lb + A_BYTES);
-                const unsigned long long dQh = tc_smem_desc(sb), dQm = tc_smem_desc(sb + B_BYTES);
+                PTC_STAMP(5, kb);
+                const unsigned long long dAh = dA0 + (unsigned long long)sh * long_step, dAm = dAh + a_off;
+                const unsigned long long dQh = dS0 + (unsigned long long)sm * short_step, dQm = dQh + b_off;
                 if (wide) {
                     const unsigned d_set = tmem + (unsigned)(3 * hb * a.Ncp);
 #pragma unroll
@@ -654,21 +765,93 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                         tc_mma_tf32(d_head, dAh + o, dQh + o, id1, k > 0 ? 1u : 0u);                       // h x h
                     }
                 }
+                PTC_STAMP(8, kb);
                 tc_commit(bar_done + 8 * sh);
+                PTC_STAMP(9, kb);
+                if (++sh == NH) { sh = 0; phh ^= 1; }
+                if (++sm == NM) { sm = 0; phm ^= 1; }
+                if (++hb == NB) { hb = 0; phb ^= 1; }
             }
             tc_commit(bar_acc);
         }
     } else if (warp < 10) {
-        // ---- converters (warps 2-9): M = A + B in place and back to HBM; second TF32 term over the tile of B ----
-        const int ct = tid - 64;                       // 0 .. 255
-        for (int kb = 0; kb < KB; ++kb) {
+        // ---- converters: two groups of four warps (one warp per quarter of the tensor-memory lanes) take the K blocks in
+        //      turn, so that the waits of one K block (tile arrival, tensor-memory reads, the group's barrier, the stores)
+        //      overlap the arithmetic of the next ----
+        const int grp = (warp - 2) >> 2;
+        const int ct = tid - 64 - 128 * grp;           // 0 .. 127 within the group
+        if (PEND) {
+            // one accumulator row per lane: M = A + B - C, second term, then the tile of M to HBM
+            const int quarter = warp & 3;              // tensor-memory lanes of this warp
+            const int row = quarter * 32 + lane;
+            const unsigned lane_base = (unsigned)(quarter * 32) << 16;
+            for (int kb = grp; kb < KB; kb += 2) {
+                const int sh = kb % NH, cb = grp;      // correction accumulator kb & 1
+                mbar_wait_warp(bar_hfull + 8 * sh, (unsigned)((kb / NH) & 1), a.flags, dead);
+                if (quarter == 2 && lane == 0) PTC_STAMP(1, kb);
+                mbar_wait_warp(bar_corr + 8 * cb, (unsigned)((kb >> 1) & 1), a.flags, dead);
+                if (quarter == 2 && lane == 0) PTC_STAMP(2, kb);
+                asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                float4* t0 = reinterpret_cast<float4*>(base + (size_t)sh * LONG_BYTES);
+                float4* t1 = t0 + A_BYTES / 16;
+#pragma unroll
+                for (int chalf = 0; chalf < 2; ++chalf) {
+                    unsigned ch[16], c1[16], c2[16];
+                    const unsigned tc = tmem_all + lane_base + (unsigned)(cb * PT_CORR_COLS + 16 * chalf);
+                    tmem_ld16(tc, ch);
+                    tmem_ld16(tc + 32u, c1);
+                    tmem_ld16(tc + 64u, c2);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+                    if (chalf == 1) {
+                        asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_cfree + 8 * cb);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int o = row * 8 + ((4 * chalf + j) ^ (row & 7));       // 16-byte unit of the swizzled tile
+                        const float4 g = t0[o], e = t1[o];
+                        float xs[4] = {g.x + e.x, g.y + e.y, g.z + e.z, g.w + e.w};
+                        float ms[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            xs[q] -= __uint_as_float(ch[4 * j + q]) + (__uint_as_float(c1[4 * j + q]) + __uint_as_float(c2[4 * j + q]));
+                            const float h = __uint_as_float(__float_as_uint(xs[q]) & 0xFFFFE000u);
+                            ms[q] = __uint_as_float((__float_as_uint(xs[q] - h) + 0x1000u) & 0xFFFFE000u);
+                        }
+                        t0[o] = make_float4(xs[0], xs[1], xs[2], xs[3]);
+                        t1[o] = make_float4(ms[0], ms[1], ms[2], ms[3]);
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");    // generic writes -> visible to the tensor core
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_conv + 8 * sh);
+                if (quarter == 2 && lane == 0) PTC_STAMP(3, kb);
+                if (grp == 0) asm volatile("bar.sync 1, 128;\n" ::: "memory");    // every row of M is in the tile
+                else asm volatile("bar.sync 2, 128;\n" ::: "memory");
+#pragma unroll
+                for (int u = 0; u < (TC_BM * TC_BK / 4) / 128; ++u) {
+                    const int o = ct + u * 128;
+                    const int r2 = o >> 3, lc = (o & 7) ^ (r2 & 7);
+                    const int grow = rt * TC_BM + r2, gcol = kb * TC_BK + lc * 4;
+                    if (grow < a.rows && gcol < a.n)
+                        *reinterpret_cast<float4*>(a.Mout + ((size_t)mat * a.rows + grow) * a.n + gcol) = t0[o];
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_stored + 8 * sh);
+                if (quarter == 2 && lane == 0) PTC_STAMP(4, kb);
+            }
+        } else {
+        // M = A + B in place and back to HBM; second TF32 term over the tile of B
+        for (int kb = grp; kb < KB; kb += 2) {
             const int sh = kb % NH;
-            mbar_wait(bar_hfull + 8 * sh, (unsigned)((kb / NH) & 1), a.flags, dead);
+            mbar_wait_warp(bar_hfull + 8 * sh, (unsigned)((kb / NH) & 1), a.flags, dead);
+            if ((warp & 3) == 2 && lane == 0) PTC_STAMP(1, kb);
             float4* t0 = reinterpret_cast<float4*>(base + (size_t)sh * LONG_BYTES);
             float4* t1 = t0 + A_BYTES / 16;
 #pragma unroll
-            for (int u = 0; u < (TC_BM * TC_BK / 4) / 256; ++u) {
-                const int o = ct + u * 256;             // 16-byte unit of the swizzled tile
+            for (int u = 0; u < (TC_BM * TC_BK / 4) / 128; ++u) {
+                const int o = ct + u * 128;             // 16-byte unit of the swizzled tile
                 float4 mv = t0[o];
                 if (a.has_b) {
                     const float4 e = t1[o];
@@ -693,6 +876,35 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");    // generic writes -> visible to the tensor core
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_conv + 8 * sh);
+            if ((warp & 3) == 2 && lane == 0) PTC_STAMP(3, kb);
+        }
+        }
+    } else if (warp == 18) {
+        // ---- (pend) issuer of the correction MMAs, a thread of its own so that the projection's issuer does not wait for
+        //      them: C_j = P~_prev Qsub_j^T into accumulator j & 1, whose last reader was K block j - 2.  The short-ring stage
+        //      it reads is released by the "done" of the projection of the same K block, which cannot be issued before the
+        //      converters have consumed C_j. ----
+        if (PEND && lane == 0) {
+            const unsigned idc3 = tc_idesc(96), idc2 = tc_idesc(64);
+            const unsigned long long dPh = tc_smem_desc(pimg_u32), dPm = tc_smem_desc(pimg_u32 + A_BYTES);
+            const unsigned long long dS0 = tc_smem_desc(short_u32) + ((3u * B_BYTES) >> 4), short_step = SHORT_BYTES >> 4;
+            mbar_wait(bar_pfull, 0u, a.flags, dead);
+            int sm = 0, phm = 0;
+            for (int j = 0; j < KB; ++j) {
+                const int cb = j & 1;
+                mbar_wait_ready(bar_bfull + 8 * sm, (unsigned)phm, a.flags, dead);
+                if (j >= 2) mbar_wait_ready(bar_cfree + 8 * cb, (unsigned)(((j >> 1) - 1) & 1), a.flags, dead);
+                asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+                const unsigned long long dS = dS0 + (unsigned long long)sm * short_step;
+                const unsigned d_c = tmem_all + (unsigned)(cb * PT_CORR_COLS);
+                for (int k = 0; k < a.ksteps; ++k) {
+                    const unsigned long long o = (unsigned long long)(2 * k);
+                    tc_mma_tf32(d_c, dPh + o, dS + o, idc3, k > 0 ? 1u : 0u);          // h x [h|m|l]
+                    tc_mma_tf32(d_c + 32u, dPm + o, dS + o, idc2, 1u);                  // m x [h|m]
+                }
+                tc_commit(bar_corr + 8 * cb);
+                if (++sm == NM) { sm = 0; phm ^= 1; }
+            }
         }
     } else {
         // ---- adders (warps 10-17): accumulators of each K block -> float32 registers; then the epilogue ----
@@ -708,15 +920,17 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
         for (int c = 0; c < KB; ++c) {
             const int hb = c % NB;
-            wait_done(c);
+            mbar_wait_warp(bar_done + 8 * (c % NH), (unsigned)((c / NH) & 1), a.flags, dead);
+            if (warp == 10 && lane == 0) PTC_STAMP(6, c);
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
             tc_add_up(acc, tmem, lane_base, col_base, a.Ncp, ng, wide, hb);
             asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_free + 8 * hb);
+            if (warp == 10 && lane == 0) PTC_STAMP(7, c);
         }
         // ---- epilogue: P = registers (+ the small accumulators) ----
-        mbar_wait(bar_acc, 0u, a.flags, dead);
+        mbar_wait_warp(bar_acc, 0u, a.flags, dead);
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
         const int row = rt * TC_BM + quarter * 32 + lane;
         float* out = a.P + ((size_t)mat * a.rows + (row < a.rows ? row : 0)) * a.r;
@@ -738,7 +952,7 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(ncols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_all), "r"(ncols) : "memory");
     }
 }
 

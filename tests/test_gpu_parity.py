@@ -429,20 +429,21 @@ def test_gemm_nt_tf32_matches_definition(torch_cuda, M, Nc, K, count):
 
 
 # ---- full-size workloads in the benchmark's launch configuration, checked on sampled matrices ----
-def _implied_residual(comp, c):
+def _implied_residual(comp, c, mean_form=False):
     """The residual the GPU state stands for, in double: E itself, or, while a deferred step's residual is
     still pending, e = Delta - P~ Q_i^T from the stored Delta and the factors of that step (Algorithm 2, last line)."""
     E = comp.E[c].cpu().numpy().astype(np.float64)
     if comp.plan_info()["pending"]:
         P = comp.P_hat[c].cpu().numpy().astype(np.float64)
         Qn = comp.debug("Q_node")[c].cpu().numpy().astype(np.float64)
+        Qm = comp.Q[c].cpu().numpy().astype(np.float64)
         for i in range(E.shape[0]):
-            E[i] -= P @ Qn[i].T
+            E[i] -= P @ (Qm.T if mean_form else Qn[i].T)
     return E
 
 
 def _full_size_case(torch, workload, m, n, r, N, count, tau, sample, free_steps, free_check=True, expect_pending=None,
-                    single_pass=None):
+                    single_pass=None, pending_tc=None, error_form="local"):
     """Deferred mode as bench.py runs it: free-running steps against the oracle on the sampled
     matrices (rotation-invariant outputs, 1e-3), then one more step from identical state (1e-5).
     The GPU is NOT asked to materialise its residual in between: the oracle takes over the state the GPU
@@ -454,9 +455,10 @@ def _full_size_case(torch, workload, m, n, r, N, count, tau, sample, free_steps,
     from paper_2509_11254_b200 import PowerSGDPlus
 
     dev = "cuda:0"
-    comp = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=3, count=count, device=dev, mode="deferred", single_pass=single_pass)
+    comp = PowerSGDPlus(m, n, r, N, refresh_period=tau, seed=3, count=count, device=dev, mode="deferred", single_pass=single_pass,
+                        pending_tc=pending_tc, error_form=error_form)
     Q0 = comp.Q.cpu().numpy()
-    oracles = {c: orc.PowerSGDPlusOracle(m, n, r, N, tau, Q0[c]) for c in sample}
+    oracles = {c: orc.PowerSGDPlusOracle(m, n, r, N, tau, Q0[c], error_form) for c in sample}
     out = {}
     for t in range(free_steps):
         G = synth.make_gradients_torch(workload, m, n, N, count, step=t, device=dev)
@@ -470,7 +472,7 @@ def _full_size_case(torch, workload, m, n, r, N, count, tau, sample, free_steps,
         assert plan["pending"] == int(expect_pending), plan
     t = free_steps
     for c in sample:
-        e = _implied_residual(comp, c)
+        e = _implied_residual(comp, c, error_form == "mean")
         if free_check:
             normM = np.linalg.norm(out[c]["M"])
             assert projector_distance(comp.P_hat[c].cpu().numpy(), out[c]["P_hat"]) <= 1e-3, f"matrix {c}: projector"
@@ -543,6 +545,25 @@ def test_pending_step_from_identical_state(torch_cuda, m, n, r, N, count, worklo
                            expect_pending=True, single_pass=single_pass)
     want = {"auto": 1 if r <= 8 else 0, "cluster": 1 if r <= 8 else 0, "none": 0, "l2": 2}[single_pass]     # (clusters of <= 4 CTAs here)
     assert plan["step_kernel"] == want
+
+
+@pytest.mark.parametrize("m,n,r,N,count,workload,form", [
+    (520, 256, 8, 4, 2, 2, "local"),        # 5 row blocks (the last with 8 rows), 8 K blocks, one rank step
+    (1100, 516, 5, 3, 2, 2, "local"),       # n % 32 = 4: the last K block holds 4 columns; r = 5 (one rank step, 3 zero columns)
+    (1040, 1024, 16, 4, 1, 5, "local"),     # two rank steps; 32 K blocks (more than the rings and accumulators hold)
+    (640, 260, 12, 2, 1, 2, "mean"),        # the node-averaged Q in the residual: one block of Qsub per matrix
+    (772, 388, 20, 3, 1, 4, "local"),       # 17..32 columns: accumulator sets of 96 columns, three rank steps
+    (1536, 640, 32, 2, 2, 4, "local"),      # 32 columns, four rank steps
+    (128, 32, 16, 1, 1, 2, "local"),        # a single tile and a single K block
+])
+def test_pending_step_on_tensor_cores(torch_cuda, m, n, r, N, count, workload, form):
+    """The steady-state two-pass step with the pending residual folded into the tensor-core projection (the rank-r product
+    P~_{t-1} Qsub^T as extra MMAs whose accumulator the converter warps subtract): three free steps, then the oracle takes
+    over the state the GPU holds without the GPU materialising its residual, and the next step is compared at 1e-5
+    (P_i's mean through P~, Q_i, Q, and E within 8 eps of norm(M))."""
+    plan = _full_size_case(torch_cuda, workload, m, n, r, N, count, tau=0, sample=tuple(range(count)), free_steps=3,
+                           expect_pending=True, single_pass="none", pending_tc="always", error_form=form)
+    assert plan["step_kernel"] == 3
 
 
 def test_full_size_config2_attention_class(torch_cuda):
