@@ -489,6 +489,15 @@ void launch_project_pending(Launcher& L, const float* G, float* E, const float* 
     else { if (vec) go(k_project<16, 4, true, true, true>, project_smem_bytes<16, true, true>()); else go(k_project<16, 1, true, true, true>, project_smem_bytes<16, true, true>()); }
 }
 
+// K splits of the tensor-core projection: one CTA per multiprocessor runs at a time, so a grid that ends in a short last
+// wave leaves most of the chip idle for a whole row block; two CTAs per row block (half of the columns each) make the waves
+// twice as many and half as long.  Cost model: waves x (K blocks per CTA + a fixed cost for filling and draining its rings).
+int proj_tc_ksplit(int tiles, int KB, int sms) {
+    if (KB < 16) return 1;
+    const long long c1 = (long long)ceil_div(tiles, sms) * (KB + 8), c2 = (long long)ceil_div(2 * tiles, sms) * (KB / 2 + 8);
+    return c2 * 100 < c1 * 97 ? 2 : 1;
+}
+
 // Tensor-core form for more than 16 columns (exactly split TF32 products, see psgd_gemm_tc.cuh).
 bool launch_project_tc(Launcher& L, const float* A, const float* B, float* Mout, const float* Q, float* P, int rows, int n,
                        int r, int nodes, int count, const int* skip) {
@@ -513,8 +522,11 @@ bool launch_project_tc(Launcher& L, const float* A, const float* B, float* Mout,
     ProjTcArgs a{B ? Mout : nullptr, P, rows, n, r, Ncp, proj_tc_nh(Ncp), B ? 1 : 0, nodes, (int*)(h->ws + h->lay.flags), skip};
     size_t smem = proj_tc_smem_bytes(Ncp);
     set_smem_attr((const void*)k_project_tc<false>, smem);
+    // (a launch that a device-side flag may skip must leave P alone: no zeroing, hence no split)
+    const int KS = skip ? 1 : proj_tc_ksplit(ceil_div(rows, TC_BM) * mats, KB, h->sm_count);
+    if (KS > 1) L.check(cudaMemsetAsync(P, 0, (size_t)mats * rows * r * 4, L.st));
     L.begin(PSGD_K_PROJECT);
-    k_project_tc<false><<<dim3(ceil_div(rows, TC_BM), mats), PT_THREADS, smem, L.st>>>(tA, tB, Qimg, a);
+    k_project_tc<false><<<dim3(ceil_div(rows, TC_BM), mats, KS), PT_THREADS, smem, L.st>>>(tA, tB, Qimg, a);
     L.end();
     return true;
 }
@@ -552,8 +564,10 @@ bool launch_project_pending_tc(Launcher& L, const float* G, float* E, const floa
                  Pimg, QSimg, qsub_per_node, ceil_div(r, 8)};
     size_t smem = proj_tc_smem_bytes(Ncp, true);
     set_smem_attr((const void*)k_project_tc<true>, smem);
+    const int KS = proj_tc_ksplit(RT * mats, KB, h->sm_count);
+    if (KS > 1) L.check(cudaMemsetAsync(P, 0, (size_t)mats * rows * r * 4, L.st));
     L.begin(PSGD_K_PROJECT);
-    k_project_tc<true><<<dim3(RT, mats), PT_THREADS_PEND, smem, L.st>>>(tA, tB, Qimg, a);
+    k_project_tc<true><<<dim3(RT, mats, KS), PT_THREADS_PEND, smem, L.st>>>(tA, tB, Qimg, a);
     L.end();
     return true;
 }

@@ -667,7 +667,11 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
     const int rt = blockIdx.x, mat = blockIdx.y;
     const int qz = mat / a.nodes;
-    const int KB = (a.n + TC_BK - 1) / TC_BK;
+    // the K blocks (32 columns each) of this row block are dealt to gridDim.z CTAs; with more than one the partial
+    // products are added into a zeroed P (two addends per element: the sum does not depend on their order)
+    const int KBt = (a.n + TC_BK - 1) / TC_BK;
+    const int kb_lo = (int)((long long)KBt * blockIdx.z / gridDim.z);
+    const int KB = (int)((long long)KBt * (blockIdx.z + 1) / gridDim.z) - kb_lo;
     unsigned ncols = 32;
     while ((int)ncols < CORR + (wide ? NB * 3 : NB + 2) * a.Ncp) ncols <<= 1;
 
@@ -703,7 +707,7 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 mbar_expect_tx(bar_pfull, PT_PIMG_BYTES);
                 bulk_load_1d(pimg_u32, a.Pimg + ((size_t)qz * gridDim.x + rt) * (PT_PIMG_BYTES / 4), PT_PIMG_BYTES, bar_pfull);
             }
-            const float* qs_src = PEND ? a.QSimg + (size_t)(a.qs_per_node ? mat : qz) * KB * (PT_QS_BYTES / 4) : nullptr;
+            const float* qs_src = PEND ? a.QSimg + ((size_t)(a.qs_per_node ? mat : qz) * KBt + kb_lo) * (PT_QS_BYTES / 4) : nullptr;
             auto issue_ab = [&](int j) {
                 const int s = j % NH;
                 if (j >= NH) {
@@ -713,8 +717,8 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 const unsigned dst = ring_u32 + s * LONG_BYTES, bar = bar_hfull + 8 * s;
                 PTC_STAMP(0, j);
                 mbar_expect_tx(bar, (a.has_b ? 2u : 1u) * A_BYTES);
-                tma_load_3d_sw(dst, &tmA, j * TC_BK, rt * TC_BM, mat, bar);
-                if (a.has_b) tma_load_3d_sw(dst + A_BYTES, &tmB, j * TC_BK, rt * TC_BM, mat, bar);
+                tma_load_3d_sw(dst, &tmA, (kb_lo + j) * TC_BK, rt * TC_BM, mat, bar);
+                if (a.has_b) tma_load_3d_sw(dst + A_BYTES, &tmB, (kb_lo + j) * TC_BK, rt * TC_BM, mat, bar);
             };
             for (int j = 0; j < min(lead, KB); ++j) issue_ab(j);
             for (int kb = 0; kb < KB; ++kb) {
@@ -723,7 +727,7 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 if (kb >= NM) wait_done(kb - NM);
                 const unsigned dst = short_u32 + s * SHORT_BYTES, bar = bar_bfull + 8 * s;
                 mbar_expect_tx(bar, SHORT_BYTES);
-                bulk_load_1d(dst, Qimg + ((size_t)qz * KB + kb) * (3u * B_BYTES / 4), 3u * B_BYTES, bar);
+                bulk_load_1d(dst, Qimg + ((size_t)qz * KBt + kb_lo + kb) * (3u * B_BYTES / 4), 3u * B_BYTES, bar);
                 if (PEND) bulk_load_1d(dst + 3u * B_BYTES, qs_src + (size_t)kb * (PT_QS_BYTES / 4), PT_QS_BYTES, bar);
             }
         }
@@ -833,7 +837,7 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 for (int u = 0; u < (TC_BM * TC_BK / 4) / 128; ++u) {
                     const int o = ct + u * 128;
                     const int r2 = o >> 3, lc = (o & 7) ^ (r2 & 7);
-                    const int grow = rt * TC_BM + r2, gcol = kb * TC_BK + lc * 4;
+                    const int grow = rt * TC_BM + r2, gcol = (kb_lo + kb) * TC_BK + lc * 4;
                     if (grow < a.rows && gcol < a.n)
                         *reinterpret_cast<float4*>(a.Mout + ((size_t)mat * a.rows + grow) * a.n + gcol) = t0[o];
                 }
@@ -859,7 +863,7 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     t0[o] = mv;                         // head: M itself (read as TF32 by the tensor core)
                     if (a.Mout) {
                         const int row = o >> 3, lc = (o & 7) ^ (row & 7);      // undo the 128-byte swizzle
-                        const int grow = rt * TC_BM + row, gcol = kb * TC_BK + lc * 4;
+                        const int grow = rt * TC_BM + row, gcol = (kb_lo + kb) * TC_BK + lc * 4;
                         if (grow < a.rows && gcol < a.n)
                             *reinterpret_cast<float4*>(a.Mout + ((size_t)mat * a.rows + grow) * a.n + gcol) = mv;
                     }
@@ -943,7 +947,10 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     const int j0 = (int)col_base + 8 * g;
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        if (j0 + j < a.r) out[j0 + j] = v[j];
+                        if (j0 + j < a.r) {
+                            if (gridDim.z > 1) atomicAdd(out + j0 + j, v[j]);
+                            else out[j0 + j] = v[j];
+                        }
                 }
             }
         }

@@ -543,7 +543,8 @@ def test_pending_step_from_identical_state(torch_cuda, m, n, r, N, count, worklo
     L2-pipelined single-pass kernel, and the default choice among them)."""
     plan = _full_size_case(torch_cuda, workload, m, n, r, N, count, tau=0, sample=tuple(range(count)), free_steps=3,
                            expect_pending=True, single_pass=single_pass)
-    want = {"auto": 1 if r <= 8 else 0, "cluster": 1 if r <= 8 else 0, "none": 0, "l2": 2}[single_pass]     # (clusters of <= 4 CTAs here)
+    two_pass = 3 if r > 8 else 0      # more than 8 columns: the pending residual is folded in on the tensor cores
+    want = {"auto": 1 if r <= 8 else two_pass, "cluster": 1 if r <= 8 else two_pass, "none": two_pass, "l2": 2}[single_pass]     # (clusters of <= 4 CTAs here)
     assert plan["step_kernel"] == want
 
 
@@ -595,7 +596,7 @@ def test_full_size_config2_two_pass_kernels(torch_cuda):
 def test_full_size_config3(torch_cuda, m, n, count, sample, r):
     """Workload 3: the same stack on 16 nodes whose top-8 left subspaces differ, r = 4 and r = 16, both shape classes."""
     plan = _full_size_case(torch_cuda, 3, m, n, r, 16, count, tau=20, sample=sample, free_steps=3, expect_pending=True)
-    assert plan["step_kernel"] == (1 if r <= 4 else 0)
+    assert plan["step_kernel"] == (1 if r <= 4 else 3)
     if r <= 4:
         assert plan["CS"] == 6 and plan["WC"] == 128          # 16 nodes: 6 CTAs x 128 columns per cluster
 
@@ -610,7 +611,7 @@ def test_full_size_config3_l2_pipelined_kernel(torch_cuda):
 def test_full_size_config5(torch_cuda, r):
     """Workload 5: one 16384 x 4096 matrix on 4 nodes, plain PowerSGD steps (the step the sweep times)."""
     plan = _full_size_case(torch_cuda, 5, 16384, 4096, r, 4, 1, tau=0, sample=(0,), free_steps=3, expect_pending=True)
-    assert plan["step_kernel"] == (1 if r <= 4 else 0)
+    assert plan["step_kernel"] == (1 if r <= 4 else (0 if r <= 8 else 3))
     if r <= 4:
         assert plan["CS"] == 8 and plan["WC"] == 512
 
@@ -655,14 +656,14 @@ def test_full_size_stack_refresh(torch_cuda, workload, m, n, r, N, count, sample
 
 def test_full_size_config4_attention_class(torch_cuda):
     """Workload 4, the 96 matrices of 2048 x 2048 (r = 32, N = 8, refresh at t = 0), two sampled."""
-    plan = _full_size_case(torch_cuda, 4, 2048, 2048, 32, 8, 96, tau=100, sample=(0, 95), free_steps=2)
-    assert plan["single_pass"] == 0
+    plan = _full_size_case(torch_cuda, 4, 2048, 2048, 32, 8, 96, tau=100, sample=(0, 95), free_steps=2, expect_pending=True)
+    assert plan["single_pass"] == 0 and plan["step_kernel"] == 3      # two passes, the residual folded in on the tensor cores
 
 
 def test_full_size_config4_ffn_class(torch_cuda):
     """Workload 4, the 72 matrices of 5504 x 2048, one sampled."""
-    plan = _full_size_case(torch_cuda, 4, 5504, 2048, 32, 8, 72, tau=100, sample=(71,), free_steps=2)
-    assert plan["single_pass"] == 0
+    plan = _full_size_case(torch_cuda, 4, 5504, 2048, 32, 8, 72, tau=100, sample=(71,), free_steps=2, expect_pending=True)
+    assert plan["single_pass"] == 0 and plan["step_kernel"] == 3
 
 
 @pytest.mark.parametrize("m,n,r,mode", [(520, 256, 8, "deferred"), (300, 260, 40, "eager"), (257, 130, 3, "eager")])
@@ -704,15 +705,16 @@ def test_msgd_update_after_the_step(torch_cuda, m, n, r, mode):
     (333, 130, 5, 2, 1, "local"),      # n % 4 != 0: outside the single-pass plan, scalar loads
 ])
 def test_two_pass_deferred_equals_three_pass(torch_cuda, m, n, r, N, count, form):
-    """Deferred mode with the single-pass kernels switched off (what also serves n % 4 != 0): the residual pass is dropped and the
-    next projection forms e = Delta - P~ Q_i^T on the fly with the same float32 operations in the same order, so
-    free-running steps (with a refresh among them) equal the three-pass mode bit for bit."""
+    """Deferred mode with the single-pass kernels and the tensor-core projection switched off (what also serves n % 4 != 0): the
+    residual pass is dropped and the next projection forms e = Delta - P~ Q_i^T on the fly with the same float32 operations in
+    the same order, so free-running steps (with a refresh among them) equal the three-pass mode bit for bit."""
     from paper_2509_11254_b200 import PowerSGDPlus
 
     torch = torch_cuda
     out = {}
     for mode in ("eager", "deferred"):
-        comp = PowerSGDPlus(m, n, r, N, refresh_period=4, seed=9, count=count, mode=mode, error_form=form, single_pass="none")
+        comp = PowerSGDPlus(m, n, r, N, refresh_period=4, seed=9, count=count, mode=mode, error_form=form, single_pass="none",
+                            pending_tc="never")
         for t in range(7):
             G = synth.make_gradients_torch(2, m, n, N, count, step=t, device="cuda:0")
             comp.step(G)
@@ -735,7 +737,7 @@ def test_two_pass_deferred_dense_output_and_state_reset(torch_cuda):
     m, n, r, N = 520, 256, 12, 3
     res = {}
     for mode in ("eager", "deferred"):
-        comp = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=4, mode=mode, single_pass="none")
+        comp = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=4, mode=mode, single_pass="none", pending_tc="never")
         Dh = torch.empty((1, m, n), dtype=torch.float32, device="cuda:0")
         outs = []
         for t in range(5):
