@@ -550,7 +550,8 @@ bool launch_project_pending_tc(Launcher& L, const float* G, float* E, const floa
         L.status = PSGD_E_CUDA;
         return true;
     }
-    const size_t tq = (size_t)count * KB * Ncp * TC_BK, tp = (size_t)count * RT * TC_BM * TC_BK, ts = (size_t)qmats * KB * 32 * TC_BK;
+    const int GQ = r <= 8 ? 4 : (r <= 16 ? 2 : 1), groups = ceil_div(KB, GQ);     // K blocks whose rank columns share one image of Qsub
+    const size_t tq = (size_t)count * KB * Ncp * TC_BK, tp = (size_t)count * RT * TC_BM * TC_BK, ts = (size_t)qmats * groups * 32 * TC_BK;
     L.begin(PSGD_K_PROJECT);
     k_split_img_t<<<(unsigned)((tq + 255) / 256), 256, 0, L.st>>>(Q, Qimg, n, r, Ncp, KB, count, nullptr);
     L.end();
@@ -558,10 +559,10 @@ bool launch_project_pending_tc(Launcher& L, const float* G, float* E, const floa
     k_split_img_rows<<<(unsigned)((tp + 255) / 256), 256, 0, L.st>>>(Pprev, Pimg, rows, r, TC_BM, 2, count);
     L.end();
     L.begin(PSGD_K_PROJECT);
-    k_split_img_rows<<<(unsigned)((ts + 255) / 256), 256, 0, L.st>>>(Qsub, QSimg, n, r, 32, 3, qmats);
+    k_split_img_qs<<<(unsigned)((ts + 255) / 256), 256, 0, L.st>>>(Qsub, QSimg, n, r, GQ, groups, qmats);
     L.end();
     ProjTcArgs a{E, P, rows, n, r, Ncp, proj_tc_nh(Ncp, true), 1, nodes, (int*)(h->ws + h->lay.flags), nullptr,
-                 Pimg, QSimg, qsub_per_node, ceil_div(r, 8)};
+                 Pimg, QSimg, qsub_per_node, ceil_div(r, 8), GQ, groups};
     size_t smem = proj_tc_smem_bytes(Ncp, true);
     set_smem_attr((const void*)k_project_tc<true>, smem);
     const int KS = proj_tc_ksplit(RT * mats, KB, h->sm_count);

@@ -523,29 +523,32 @@ struct ProjTcArgs {
     const int* skip;
     // pending residual (two-pass deferred mode): M = A + (B - P~_prev Qsub^T), the product formed by the tensor core
     const float* Pimg;    // [count][row tiles][2][128][32]: two TF32 terms of P~_prev, shared-memory image (k_split_img_rows)
-    const float* QSimg;   // [mats or count][KB][3][32][32]: three terms of Qsub, one image per K block
+    const float* QSimg;   // [mats or count][groups][3][32][32]: three terms of Qsub, one image per group of K blocks (k_split_img_qs)
     int qs_per_node;      // Qsub is per (matrix, node) (1) or per matrix (0)
     int ksteps;           // ceil(r / 8): MMAs along the rank
+    int qs_group;         // K blocks per image: 4 (r <= 8), 2 (r <= 16) or 1; their 32 / qs_group rank columns lie side by side in a row
+    int qs_groups;        // images per matrix: ceil(KB / qs_group)
 };
+constexpr int PT_NQ = 3;                             // stages of the ring of Qsub images (pend)
 constexpr int PT_CORR_COLS = 96;                     // one correction accumulator: [head | small | small] x 32 columns
 constexpr unsigned PT_QS_BYTES = 3 * 32 * TC_BK * 4; // three terms of a 32-row block of Qsub
 constexpr unsigned PT_PIMG_BYTES = 2 * TC_BM * TC_BK * 4;
 
 // Two shared-memory rings, as in the back-projection below: stages of 32 KB for the tiles of A and B (M and its second
 // TF32 term are formed in place) and a short ring for the three terms of Q^T.
-// (pend: every stage of the short ring also holds the three terms of a block of Qsub, and the two terms of P~_prev stay resident)
+// (pend: the two terms of P~_prev stay resident, and the images of Qsub have a ring of their own, filled by the thread that
+// issues the correction MMAs and released as soon as those have completed, so that it runs ahead of the other rings)
 __host__ __device__ inline int proj_tc_nm(int Ncp) { return 3 * Ncp <= 256 ? 3 : 2; }
-__host__ __device__ inline long long proj_tc_short_bytes(int Ncp, bool pend) {
-    return 3ll * Ncp * TC_BK * 4 + (pend ? (long long)PT_QS_BYTES : 0);
-}
+__host__ __device__ inline long long proj_tc_short_bytes(int Ncp) { return 3ll * Ncp * TC_BK * 4; }
+__host__ __device__ inline long long proj_tc_pend_bytes(bool pend) { return pend ? (long long)PT_PIMG_BYTES + (long long)PT_NQ * PT_QS_BYTES : 0; }
 __host__ __device__ inline int proj_tc_nh(int Ncp, bool pend = false) {
-    const long long left = 224ll * 1024 - 1024 - 512 - proj_tc_nm(Ncp) * proj_tc_short_bytes(Ncp, pend) - (pend ? (long long)PT_PIMG_BYTES : 0);
+    const long long left = 224ll * 1024 - 1024 - 512 - proj_tc_nm(Ncp) * proj_tc_short_bytes(Ncp) - proj_tc_pend_bytes(pend);
     const int nh = (int)(left / (2 * TC_BM * TC_BK * 4));
     return nh > 6 ? 6 : nh;
 }
 __host__ __device__ inline size_t proj_tc_smem_bytes(int Ncp, bool pend = false) {
-    return (size_t)proj_tc_nh(Ncp, pend) * 2 * TC_BM * TC_BK * 4 + (size_t)(proj_tc_nm(Ncp) * proj_tc_short_bytes(Ncp, pend)) +
-           (pend ? PT_PIMG_BYTES : 0) + 1024 + 512;
+    return (size_t)proj_tc_nh(Ncp, pend) * 2 * TC_BM * TC_BK * 4 + (size_t)(proj_tc_nm(Ncp) * proj_tc_short_bytes(Ncp)) +
+           (size_t)proj_tc_pend_bytes(pend) + 1024 + 512;
 }
 
 // Q [count][n][r] -> Qt[t][count][Ncp][n], t = 0, 1, 2: the transposed factor split exactly into three TF32 terms,
@@ -615,6 +618,27 @@ __global__ void k_split_img_rows(const float* X, float* img, int rows, int r, in
         blk[2 * (size_t)TR * TC_BK + o] = r1 - mm;
     }
 }
+// Qsub [mats][n][r] -> img[mats][groups][3][32][32]: image gi holds the K blocks G gi .. G gi + G - 1 (32 rows of Qsub each).
+// Row `row` of the image is [block 0: k = 0 .. 32/G - 1 | block 1 | ...] of those blocks' row `row`, as three exact TF32 terms,
+// 128-byte swizzled; zero beyond r and beyond n.  One thread per (matrix, image, row, float).
+__global__ void k_split_img_qs(const float* X, float* img, int n, int r, int G, int groups, int mats) {
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t per_img = 32 * TC_BK, tot = per_img * groups * mats;
+    if (idx >= tot) return;
+    const int mt = (int)(idx / (per_img * groups));
+    const int gi = (int)((idx / per_img) % groups), row = (int)((idx / TC_BK) % 32), f = (int)(idx % TC_BK);
+    const int kpad = TC_BK / G, q = f / kpad, k = f % kpad;
+    const int col = (gi * G + q) * 32 + row;
+    const float x = (col < n && k < r) ? X[((size_t)mt * n + col) * r + k] : 0.f;
+    const float h = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
+    const float r1 = x - h;
+    const float mm = __uint_as_float(__float_as_uint(r1) & 0xFFFFE000u);
+    float* blk = img + ((size_t)mt * groups + gi) * 3 * per_img;
+    const size_t o = (size_t)row * TC_BK + ((((f >> 2) ^ (row & 7)) << 2) | (f & 3));
+    blk[o] = h;
+    blk[per_img + o] = mm;
+    blk[2 * per_img + o] = r1 - mm;
+}
 __device__ __forceinline__ void tmem_ld16(unsigned taddr, unsigned (&v)[16]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
                  : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
@@ -651,19 +675,21 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     constexpr unsigned A_BYTES = TC_BM * TC_BK * 4;
     constexpr unsigned LONG_BYTES = 2 * A_BYTES;               // [A tile -> M (head)][B tile -> second term]
     const unsigned B_BYTES = (unsigned)a.Ncp * TC_BK * 4;
-    const unsigned SHORT_BYTES = 3 * B_BYTES + (PEND ? PT_QS_BYTES : 0u);   // h, m, l of Q^T [, h, m, l of the block of Qsub]
+    const unsigned SHORT_BYTES = 3 * B_BYTES;                  // h, m, l of Q^T
     const bool wide = 3 * a.Ncp <= 256;
     const int NM = proj_tc_nm(a.Ncp);
     const int CORR = PEND ? 2 * PT_CORR_COLS : 0;              // tensor-memory columns of the two correction accumulators
     const int NH = a.nh, NB = wide ? min(4, (512 - CORR) / (3 * a.Ncp)) : min(3, (512 - 2 * a.Ncp) / a.Ncp);
     unsigned char* short_base = base + (size_t)NH * LONG_BYTES;
     unsigned char* pimg_base = short_base + (size_t)NM * SHORT_BYTES;
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(pimg_base + (PEND ? PT_PIMG_BYTES : 0u));
+    unsigned char* qs_base = pimg_base + (PEND ? PT_PIMG_BYTES : 0u);       // ring of Qsub images (pend)
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(qs_base + (PEND ? PT_NQ * PT_QS_BYTES : 0u));
     const unsigned bar_hfull = smem_u32(bars), bar_conv = bar_hfull + 8 * NH, bar_done = bar_conv + 8 * NH;
     const unsigned bar_bfull = bar_done + 8 * NH, bar_free = bar_bfull + 8 * NM, bar_acc = bar_free + 8 * NB;
     const unsigned bar_stored = bar_acc + 8, bar_corr = bar_stored + 8 * NH, bar_cfree = bar_corr + 16, bar_pfull = bar_cfree + 16;
-    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 4 * NH + NM + NB + 1 + 5);
-    const unsigned ring_u32 = smem_u32(base), short_u32 = smem_u32(short_base), pimg_u32 = smem_u32(pimg_base);
+    const unsigned bar_qfull = bar_pfull + 8, bar_qfree = bar_qfull + 8 * PT_NQ;
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 4 * NH + NM + NB + 1 + 5 + 2 * PT_NQ);
+    const unsigned ring_u32 = smem_u32(base), short_u32 = smem_u32(short_base), pimg_u32 = smem_u32(pimg_base), qs_u32 = smem_u32(qs_base);
 
     const int rt = blockIdx.x, mat = blockIdx.y;
     const int qz = mat / a.nodes;
@@ -684,6 +710,7 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         mbar_init(bar_acc, 1);
         for (int b = 0; b < 2; ++b) { mbar_init(bar_corr + 8 * b, 1); mbar_init(bar_cfree + 8 * b, 4); }
         mbar_init(bar_pfull, 1);
+        for (int b = 0; b < PT_NQ; ++b) { mbar_init(bar_qfull + 8 * b, 1); mbar_init(bar_qfree + 8 * b, 1); }
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     if (warp == 1) {
@@ -707,7 +734,6 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 mbar_expect_tx(bar_pfull, PT_PIMG_BYTES);
                 bulk_load_1d(pimg_u32, a.Pimg + ((size_t)qz * gridDim.x + rt) * (PT_PIMG_BYTES / 4), PT_PIMG_BYTES, bar_pfull);
             }
-            const float* qs_src = PEND ? a.QSimg + ((size_t)(a.qs_per_node ? mat : qz) * KBt + kb_lo) * (PT_QS_BYTES / 4) : nullptr;
             auto issue_ab = [&](int j) {
                 const int s = j % NH;
                 if (j >= NH) {
@@ -728,7 +754,6 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 const unsigned dst = short_u32 + s * SHORT_BYTES, bar = bar_bfull + 8 * s;
                 mbar_expect_tx(bar, SHORT_BYTES);
                 bulk_load_1d(dst, Qimg + ((size_t)qz * KBt + kb_lo + kb) * (3u * B_BYTES / 4), 3u * B_BYTES, bar);
-                if (PEND) bulk_load_1d(dst + 3u * B_BYTES, qs_src + (size_t)kb * (PT_QS_BYTES / 4), PT_QS_BYTES, bar);
             }
         }
     } else if (warp == 1) {
@@ -891,15 +916,26 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         if (PEND && lane == 0) {
             const unsigned idc3 = tc_idesc(96), idc2 = tc_idesc(64);
             const unsigned long long dPh = tc_smem_desc(pimg_u32), dPm = tc_smem_desc(pimg_u32 + A_BYTES);
-            const unsigned long long dS0 = tc_smem_desc(short_u32) + ((3u * B_BYTES) >> 4), short_step = SHORT_BYTES >> 4;
+            const unsigned long long dS0 = tc_smem_desc(qs_u32), qs_step = PT_QS_BYTES >> 4;
+            // images of Qsub: image gi serves the K blocks G gi .. G gi + G - 1, block q at 32 / G floats (8 / G units) into every row
+            const int G = a.qs_group, gsh = G == 4 ? 2 : (G == 2 ? 1 : 0);
+            const unsigned long long blk_units = 8u >> gsh;
+            const int g_lo = kb_lo >> gsh, ngr = ((kb_lo + KB - 1) >> gsh) - g_lo + 1;
+            const float* qs_src = a.QSimg + ((size_t)(a.qs_per_node ? mat : qz) * a.qs_groups + g_lo) * (PT_QS_BYTES / 4);
+            auto load_group = [&](int gl, int s) {
+                mbar_expect_tx(bar_qfull + 8 * s, PT_QS_BYTES);
+                bulk_load_1d(qs_u32 + s * PT_QS_BYTES, qs_src + (size_t)gl * (PT_QS_BYTES / 4), PT_QS_BYTES, bar_qfull + 8 * s);
+            };
+            for (int gl = 0; gl < min(PT_NQ, ngr); ++gl) load_group(gl, gl);
             mbar_wait(bar_pfull, 0u, a.flags, dead);
-            int sm = 0, phm = 0;
+            int s = 0, phq = 0, gl = 0;             // stage, parity and local index of the current image
+            unsigned free_par = 0;                  // bit s: parity of the next completion of qfree[s] to wait for
             for (int j = 0; j < KB; ++j) {
-                const int cb = j & 1;
-                mbar_wait_ready(bar_bfull + 8 * sm, (unsigned)phm, a.flags, dead);
+                const int q = (kb_lo + j) & (G - 1), cb = j & 1;
+                if (j == 0 || q == 0) mbar_wait_ready(bar_qfull + 8 * s, (unsigned)phq, a.flags, dead);
                 if (j >= 2) mbar_wait_ready(bar_cfree + 8 * cb, (unsigned)(((j >> 1) - 1) & 1), a.flags, dead);
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-                const unsigned long long dS = dS0 + (unsigned long long)sm * short_step;
+                const unsigned long long dS = dS0 + (unsigned long long)s * qs_step + (unsigned long long)q * blk_units;
                 const unsigned d_c = tmem_all + (unsigned)(cb * PT_CORR_COLS);
                 for (int k = 0; k < a.ksteps; ++k) {
                     const unsigned long long o = (unsigned long long)(2 * k);
@@ -907,7 +943,18 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     tc_mma_tf32(d_c + 32u, dPm + o, dS + o, idc2, 1u);                  // m x [h|m]
                 }
                 tc_commit(bar_corr + 8 * cb);
-                if (++sm == NM) { sm = 0; phm ^= 1; }
+                if (q == G - 1 || j == KB - 1) {
+                    tc_commit(bar_qfree + 8 * s);           // the image is free once these MMAs have completed
+                    // refill the stage that was released one image ago (its MMAs are long done): image gl - 1 + PT_NQ
+                    if (gl >= 1 && gl - 1 + PT_NQ < ngr) {
+                        const int ps = s == 0 ? PT_NQ - 1 : s - 1;
+                        mbar_wait_ready(bar_qfree + 8 * ps, (free_par >> ps) & 1u, a.flags, dead);
+                        free_par ^= 1u << ps;
+                        load_group(gl - 1 + PT_NQ, ps);
+                    }
+                    ++gl;
+                    if (++s == PT_NQ) { s = 0; phq ^= 1; }
+                }
             }
         }
     } else {
@@ -1100,15 +1147,18 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
         if (lane == 0) {
             const unsigned id1 = tc_idesc(a.Ncp) | (1u << 15);            // bit 15: A is MN-major
             const unsigned id2 = tc_idesc(2 * a.Ncp) | (1u << 15), id3 = tc_idesc(wide ? 3 * a.Ncp : a.Ncp) | (1u << 15);
+            // one thread: ring positions and parities as counters, descriptors as offsets from those of stage 0
+            const unsigned long long dA0 = tc_smem_desc_mn(ring_u32, BOX_BYTES), dM0 = tc_smem_desc_mn(short_u32, BOX_BYTES);
+            const unsigned long long dP0 = tc_smem_desc(short_u32 + A_BYTES);
+            const unsigned long long long_step = A_BYTES >> 4, short_step = SHORT_BYTES >> 4, b_off = B_BYTES >> 4;
+            int sh = 0, sm = 0, phm = 0, hb = 0, phb = 1;
             for (int kb = 0; kb < KB; ++kb) {
-                const int sh = kb % NH, sm = kb % NM, hb = kb % NB;
-                mbar_wait(bar_conv + 8 * sm, (unsigned)((kb / NM) & 1), a.flags, dead);
-                mbar_wait(bar_bfull + 8 * sm, (unsigned)((kb / NM) & 1), a.flags, dead);
-                if (kb >= NB) mbar_wait(bar_free + 8 * hb, (unsigned)((kb / NB - 1) & 1), a.flags, dead);   // registers took its last content
+                mbar_wait_ready(bar_conv + 8 * sm, (unsigned)phm, a.flags, dead);
+                mbar_wait_ready(bar_bfull + 8 * sm, (unsigned)phm, a.flags, dead);
+                if (kb >= NB) mbar_wait_ready(bar_free + 8 * hb, (unsigned)phb, a.flags, dead);   // registers took its last content
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-                const unsigned sb = short_u32 + sm * SHORT_BYTES;
-                const unsigned long long dAh = tc_smem_desc_mn(ring_u32 + sh * A_BYTES, BOX_BYTES), dAm = tc_smem_desc_mn(sb, BOX_BYTES);
-                const unsigned long long dPh = tc_smem_desc(sb + A_BYTES), dPm = tc_smem_desc(sb + A_BYTES + B_BYTES);
+                const unsigned long long dAh = dA0 + (unsigned long long)sh * long_step, dAm = dM0 + (unsigned long long)sm * short_step;
+                const unsigned long long dPh = dP0 + (unsigned long long)sm * short_step, dPm = dPh + b_off;
                 if (wide) {
                     const unsigned d_set = tmem + (unsigned)(3 * hb * a.Ncp);
 #pragma unroll
@@ -1129,6 +1179,9 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
                     }
                 }
                 tc_commit(bar_done + 8 * sh);
+                if (++sh == NH) sh = 0;
+                if (++sm == NM) { sm = 0; phm ^= 1; }
+                if (++hb == NB) { hb = 0; phb ^= 1; }
             }
             tc_commit(bar_acc);
         }
