@@ -180,7 +180,7 @@ void plan(psgd_handle* h) {
     L.Y = take(cnt * m * ell * 4);
     L.Z = take(cnt * n * ell * 4);
     size_t c2 = (c + 1) & ~(size_t)1;
-    L.V = take(cnt * c2 * c2 * 8);
+    L.V = take(std::max<size_t>(8, cnt * jac_log_doubles((int)c2) * 8));   // rotation log of the Rayleigh-Ritz step (blocks too wide for shared memory)
     L.U = take(cnt * ell * r * 8);
     L.Pold = take(cnt * m * r * 4);
     L.dpart = take(cnt * ((size_t)ceil_div(h->m, 64) + 1) * 8);
@@ -905,11 +905,17 @@ void svd(Launcher& L, psgd_handle* h, const void* G, bool have_dbar = false) {
         L.begin(K);
         k_transpose<<<dim3(ceil_div(n, 32), ceil_div(m, 32), cnt), dim3(32, 8), 0, L.st>>>(dbar, dbarT, m, n);
         L.end();
+        // Only Y is orthonormalised in a sweep (as in the float32 sweeps below): Z = Dbar^T Y with orthonormal Y is bounded by
+        // the largest singular value, and the Gram matrix of the next Y is formed in double.
         for (; it0 < iters - tail32; ++it0) {
             launch_gemm_tc(L, h, dbar, Zt, Y, m, ell, n, K);       // Y = Dbar Z
             launch_orth(L, h, Y, Y, m, ell, K, Yt);
             launch_gemm_tc(L, h, dbarT, Yt, Z, n, ell, m, K);      // Z = Dbar^T Y
-            launch_orth(L, h, Z, Z, n, ell, K, Zt);
+            if (it0 + 1 < iters - tail32) {
+                L.begin(K);
+                k_transpose<<<dim3(ceil_div(ell, 32), ceil_div(n, 32), cnt), dim3(32, 8), 0, L.st>>>(Z, Zt, n, ell);
+                L.end();
+            }
         }
     }
     // chunking of Z = Dbar^T Y over rows
@@ -938,11 +944,18 @@ void svd(Launcher& L, psgd_handle* h, const void* G, bool have_dbar = false) {
             L.end();
         }
         int c2 = (ell + 1) & ~1;
-        size_t smem = (size_t)c2 * jac_ld(c2) * 8;
+        size_t smem = jac_smem_bytes(c2);
         allow_smem(k_jacobi_top, smem);
         L.begin(K);
         k_jacobi_top<<<cnt, JAC_THREADS, smem, L.st>>>(gram, nparts > 4 ? -nparts : nparts, ell, r, V, U, flags, skip);
         L.end();
+        if (!jac_v_in_smem(c2)) {      // eigenvectors replayed from the rotation log
+            size_t vs = jacv_smem_bytes(c2);
+            allow_smem(k_jacobi_vectors, vs);
+            L.begin(K);
+            k_jacobi_vectors<<<dim3(ceil_div(c2, JV_ROWS), cnt), JV_THREADS, vs, L.st>>>(V, ell, r, U, skip);
+            L.end();
+        }
         ApplyArgs ap{Y, U, Phat, m, ell, r, r, 0, nullptr, skip};
         L.begin(K);
         k_apply<<<dim3(ceil_div(m, 32), cnt), 256, (size_t)32 * ell * 4, L.st>>>(ap);

@@ -931,9 +931,26 @@ constexpr int JAC_THREADS = 512;
 constexpr int JAC_MAX_SWEEPS = 40;
 // leading dimension of the shared-memory matrix: odd number of doubles (no bank conflicts down a column)
 __host__ __device__ inline int jac_ld(int c2) { return c2 | 1; }
+// The eigenvector matrix is kept in shared memory beside A while both fit; wider blocks log their rotations
+// (cos, sin per pair and round: the pairs follow from the round-robin schedule) and k_jacobi_vectors replays them.
+__host__ __device__ inline bool jac_v_in_smem(int c2) { return (size_t)c2 * jac_ld(c2) * 8 + (size_t)c2 * c2 * 8 <= 200 * 1024; }
+__host__ __device__ inline size_t jac_smem_bytes(int c2) {
+    return (size_t)c2 * jac_ld(c2) * 8 + (jac_v_in_smem(c2) ? (size_t)c2 * c2 * 8 : 0);
+}
+// doubles per matrix of the rotation log: a header of 2 + c2 values (sweeps done, unused, order of the eigenvalues), then
+// [sweep][round][pair](cos, sin)
+__host__ __device__ inline size_t jac_log_doubles(int c2) {
+    return jac_v_in_smem(c2) ? 0 : 2 + (size_t)c2 + (size_t)JAC_MAX_SWEEPS * (c2 - 1) * (c2 / 2) * 2;
+}
+// pair k of round `round` in the round-robin tournament on c2 players: position 0 fixed, the others rotate
+__device__ __forceinline__ void jac_pair(int k, int round, int c2, int& p, int& q) {
+    const int a0 = (k == 0) ? 0 : 1 + (k - 1 + round) % (c2 - 1);
+    const int b0 = 1 + (c2 - 2 - k + round) % (c2 - 1);
+    p = min(a0, b0); q = max(a0, b0);
+}
 __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, int nparts, int c, int r,
-                                                            double* Vws, double* U, int* flags, const int* skip = nullptr) {
-    extern __shared__ __align__(16) double As[];  // [c2][ld]
+                                                            double* rotlog, double* U, int* flags, const int* skip = nullptr) {
+    extern __shared__ __align__(16) double As[];  // [c2][ld] (+ [c2][c2] eigenvectors, transposed, when they fit)
     if (skip && *skip) return;
     __shared__ double cs[128], sn[128];
     __shared__ int pp[128], qq[128];
@@ -943,7 +960,10 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
     const int c2 = (c + 1) & ~1;
     const int ld = jac_ld(c2);
     const int np = c2 / 2;
-    double* Vt = Vws + (size_t)blockIdx.x * c2 * c2;   // eigenvector matrix, stored transposed: Vt[p][i] = V[i][p]
+    const bool vsm = jac_v_in_smem(c2);
+    double* Vt = As + (size_t)c2 * ld;                 // Vt[p][i] = V[i][p] (only when vsm)
+    double* logb = vsm ? nullptr : rotlog + (size_t)blockIdx.x * jac_log_doubles(c2);
+    double* rots = vsm ? nullptr : logb + 2 + c2;
     const int pstride = nparts < 0 ? -nparts : nparts;   // nparts < 0: partials already folded into partial 0
     if (nparts < 0) nparts = 1;
     const double* pb = part + (size_t)blockIdx.x * pstride * c * c;
@@ -956,7 +976,7 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
             for (int p = 0; p < nparts; ++p) s += pb[(size_t)p * c * c + (size_t)ii * c + jj];
         }
         As[i * ld + j] = s;
-        Vt[e] = (i == j) ? 1.0 : 0.0;
+        if (vsm) Vt[e] = (i == j) ? 1.0 : 0.0;
     }
     __syncthreads();
     // symmetrise (the two triangles of a diagonal block were accumulated separately)
@@ -965,14 +985,13 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
         if (i < j) { double v = 0.5 * (As[i * ld + j] + As[j * ld + i]); As[i * ld + j] = v; As[j * ld + i] = v; }
     }
     __syncthreads();
-    int converged = 0;
+    int converged = 0, sweeps = 0;
+    const int k_first = tid / c2, i_first = tid % c2, k_step = JAC_THREADS / c2, i_step = JAC_THREADS % c2;
     for (int sweep = 0; sweep < JAC_MAX_SWEEPS && !converged; ++sweep) {
         for (int round = 0; round < c2 - 1; ++round) {
-            // round-robin tournament: position 0 fixed, the others rotate
             if (tid < np) {
-                int a0 = (tid == 0) ? 0 : 1 + (tid - 1 + round) % (c2 - 1);
-                int b0 = 1 + (c2 - 2 - tid + round) % (c2 - 1);
-                int p = min(a0, b0), q = max(a0, b0);
+                int p, q;
+                jac_pair(tid, round, c2, p, q);
                 pp[tid] = p; qq[tid] = q;
                 double apq = As[p * ld + q], app = As[p * ld + p], aqq = As[q * ld + q];
                 double cc = 1.0, ss = 0.0;
@@ -983,32 +1002,41 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
                     ss = t * cc;
                 }
                 cs[tid] = cc; sn[tid] = ss;
+                if (!vsm) {
+                    double* o = rots + (((size_t)sweep * (c2 - 1) + round) * np + tid) * 2;
+                    o[0] = cc; o[1] = ss;
+                }
             }
             __syncthreads();
-            // columns: A <- A J, V <- V J   (thread index runs down the column)
-            for (int e = tid; e < np * c2; e += JAC_THREADS) {
-                int k = e / c2, i = e % c2;
+            // columns: A <- A J, V <- V J   (thread index runs down the column; (k, i) advance without a division)
+            for (int e = tid, k = k_first, i = i_first; e < np * c2; e += JAC_THREADS) {
                 int p = pp[k], q = qq[k];
                 double cc = cs[k], ss = sn[k];
                 double aip = As[i * ld + p], aiq = As[i * ld + q];
                 As[i * ld + p] = cc * aip - ss * aiq;
                 As[i * ld + q] = ss * aip + cc * aiq;
-                double vip = Vt[p * c2 + i], viq = Vt[q * c2 + i];
-                Vt[p * c2 + i] = cc * vip - ss * viq;
-                Vt[q * c2 + i] = ss * vip + cc * viq;
+                if (vsm) {
+                    double vip = Vt[p * c2 + i], viq = Vt[q * c2 + i];
+                    Vt[p * c2 + i] = cc * vip - ss * viq;
+                    Vt[q * c2 + i] = ss * vip + cc * viq;
+                }
+                k += k_step; i += i_step;
+                if (i >= c2) { i -= c2; ++k; }
             }
             __syncthreads();
             // rows: A <- J^T A
-            for (int e = tid; e < np * c2; e += JAC_THREADS) {
-                int k = e / c2, j = e % c2;
+            for (int e = tid, k = k_first, j = i_first; e < np * c2; e += JAC_THREADS) {
                 int p = pp[k], q = qq[k];
                 double cc = cs[k], ss = sn[k];
                 double apj = As[p * ld + j], aqj = As[q * ld + j];
                 As[p * ld + j] = cc * apj - ss * aqj;
                 As[q * ld + j] = ss * apj + cc * aqj;
+                k += k_step; j += i_step;
+                if (j >= c2) { j -= c2; ++k; }
             }
             __syncthreads();
         }
+        ++sweeps;
         if (tid == 0) { offn = 0.0; diagn = 0.0; }
         __syncthreads();
         double lo = 0.0, ldg = 0.0;
@@ -1038,10 +1066,61 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
         order[rank] = i;
     }
     __syncthreads();
-    double* Ub = U + (size_t)blockIdx.x * c * r;
-    for (int e = tid; e < c * r; e += JAC_THREADS) {
-        int i = e / r, k = e % r;
-        Ub[e] = Vt[order[k] * c2 + i];
+    if (vsm) {
+        double* Ub = U + (size_t)blockIdx.x * c * r;
+        for (int e = tid; e < c * r; e += JAC_THREADS) {
+            int i = e / r, k = e % r;
+            Ub[e] = Vt[order[k] * c2 + i];
+        }
+    } else {
+        if (tid == 0) logb[0] = (double)sweeps;
+        for (int i = tid; i < c2; i += JAC_THREADS) logb[2 + i] = (double)order[i];
+    }
+}
+
+// The eigenvectors of a block too wide for k_jacobi_top's shared memory: V = J_1 J_2 ... replayed from the rotation log.
+// Row i of V only ever mixes with itself, and the rotations of one round touch disjoint columns: a CTA carries JV_ROWS rows
+// in shared memory, eight lanes share a row and split the pairs of a round between them, a warp-level barrier separates
+// the rounds.  The players of the round-robin schedule come from a doubled table (no division per rotation).
+constexpr int JV_ROWS = 16, JV_THREADS = 128;
+__host__ __device__ inline size_t jacv_smem_bytes(int c2) {
+    return (size_t)JV_ROWS * (c2 + 1) * 8 + (size_t)2 * (c2 / 2) * 16 + (size_t)2 * (c2 - 1) * 4;
+}
+__global__ void __launch_bounds__(JV_THREADS) k_jacobi_vectors(const double* rotlog, int c, int r, double* U, const int* skip = nullptr) {
+    extern __shared__ __align__(16) double Vs[];   // [JV_ROWS][c2 + 1], two rounds of (cos, sin), then the table of players
+    if (skip && *skip) return;
+    const int c2 = (c + 1) & ~1, np = c2 / 2, ldv = c2 + 1;
+    double2* rbuf = reinterpret_cast<double2*>(Vs + (size_t)((JV_ROWS * ldv + 1) & ~1));     // [2][np]
+    int* perm = reinterpret_cast<int*>(rbuf + 2 * np);                    // perm[j] = 1 + j mod (c2 - 1), j < 2 (c2 - 1)
+    const double* logb = rotlog + (size_t)blockIdx.y * jac_log_doubles(c2);
+    const double2* rots = reinterpret_cast<const double2*>(logb + 2 + c2);
+    const int tid = threadIdx.x, rl = tid >> 3, l8 = tid & 7;
+    const int i = blockIdx.x * JV_ROWS + rl;
+    for (int j = tid; j < 2 * (c2 - 1); j += JV_THREADS) perm[j] = 1 + j % (c2 - 1);
+    double* row = Vs + (size_t)rl * ldv;
+    for (int p = l8; p < c2; p += 8) row[p] = (p == i) ? 1.0 : 0.0;
+    const int rounds = (int)logb[0] * (c2 - 1);           // the log is one run of rounds, np rotations each
+    for (int k = tid; k < np && rounds > 0; k += JV_THREADS) rbuf[k] = __ldg(rots + k);
+    __syncthreads();
+    for (int g = 0, round = 0; g < rounds; ++g) {
+        const double2* cur = rbuf + (g & 1) * np;
+        double2 nxt = make_double2(1.0, 0.0);
+        if (tid < np && g + 1 < rounds) nxt = __ldg(rots + (size_t)(g + 1) * np + tid);       // np <= JV_THREADS
+        for (int k = l8; k < np; k += 8) {
+            const int a0 = (k == 0) ? 0 : perm[k - 1 + round], b0 = perm[c2 - 2 - k + round];
+            const int p = min(a0, b0), q = max(a0, b0);
+            const double2 csn = cur[k];
+            const double vp = row[p], vq = row[q];
+            row[p] = csn.x * vp - csn.y * vq;
+            row[q] = csn.y * vp + csn.x * vq;
+        }
+        if (tid < np) rbuf[((g + 1) & 1) * np + tid] = nxt;
+        __syncthreads();
+        if (++round == c2 - 1) round = 0;
+    }
+    if (i < c) {
+        double* Ub = U + (size_t)blockIdx.y * c * r;
+        for (int k = l8; k < r; k += 8) Ub[(size_t)i * r + k] = row[(int)logb[2 + k]];
     }
 }
 
