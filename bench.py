@@ -40,7 +40,7 @@ SWEEP_RANKS = (1, 4, 8, 16, 64, 128)
 HEADLINE_RANK = 16
 # dram__bytes_read.sum + dram__bytes_write.sum per element of one launch, from the ncu captures summarised under
 # profiles/ (small case of the same kernel; traffic grows in proportion to the elements).  None: no current capture.
-TRAFFIC_BYTES_PER_ELEMENT = {"k_fused_step": 11.87, "k_project": 11.4, "k_backproject": 4.1, "k_stream_step": 13.6}
+TRAFFIC_BYTES_PER_ELEMENT = {"k_fused_step": 11.87, "k_project": 11.4, "k_project_tc<pend>": 11.49, "k_backproject": 4.1, "k_stream_step": 13.6}
 
 # (rank, nodes, refresh period) of the stacks
 STACK_DEFAULTS = {2: [(8, 8, 50)], 3: [(4, 16, 20), (16, 16, 20)], 4: [(32, 8, 100)]}
@@ -153,6 +153,8 @@ def kernel_name(family, r, step_kernel):
             return "k_fused_step"
         if step_kernel == 2:
             return "k_stream_step"
+        if step_kernel == 3:
+            return "k_project_tc<pend>"
         return "k_project_tc" if r > 16 else "k_project"
     return ("k_%s_tc" if r > 16 else "k_%s") % family
 
@@ -232,7 +234,7 @@ def sweep_point(torch, device, r, bufs, mode, single_pass, steps, min_seconds, p
     ms = out["step_ms"]
     out.update(grad_GBps=round(gb / ms / 1e6, 1), min_bytes_frac=round(alg / ms / 1e6 / peak, 4),
                path={0: ("two-pass" if (mode == "deferred" and r <= 16) else "three-pass"), 1: "single-pass (cluster kernel)",
-                     2: "single-pass (L2-pipelined kernel)"}[plan["step_kernel"]],
+                     2: "single-pass (L2-pipelined kernel)", 3: "two-pass (pending residual folded in on the tensor cores)"}[plan["step_kernel"]],
                roofline=roofline_entry(fam, r, plan["step_kernel"], m * n * N, peak, peak_kind),
                launches_per_step=round(launches / done, 2))
     if refresh:
