@@ -754,7 +754,7 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
                                               const int* skip = nullptr) {
     extern __shared__ __align__(16) double Gs[];  // [c][ld]
     if (skip && *skip) return;
-    __shared__ double dinv[192];
+    __shared__ double dinv[192], rdiag[192];   // column scaling; reciprocals of the diagonal of L
     __shared__ int dcol[192];
     __shared__ int bad, illc;
     const int tid = threadIdx.x;
@@ -786,17 +786,20 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
         Gs[i * ld + j] = v;
     }
     __syncthreads();
-    // right-looking Cholesky on the lower triangle: Gs = L L^T
+    // right-looking Cholesky on the lower triangle: Gs = L L^T.  Every thread evaluates the pivot of the step itself (no
+    // serial step by one thread): two barriers per column.
     for (int k = 0; k < c; ++k) {
+        double p = Gs[k * ld + k];
+        const bool reject = !(p > CHOL_PIVOT_TOL);
         if (tid == 0) {
-            double p = Gs[k * ld + k];
             if (!(p > gate_tol)) illc = 1;
-            if (!(p > CHOL_PIVOT_TOL)) { bad = 1; dcol[k] = 1; p = 1.0; for (int i = k + 1; i < c; ++i) Gs[i * ld + k] = 0.0; }
-            Gs[k * ld + k] = sqrt(p);
+            if (reject) { bad = 1; dcol[k] = 1; }
         }
-        __syncthreads();
-        double lkk = Gs[k * ld + k];
-        for (int i = k + 1 + tid; i < c; i += 256) Gs[i * ld + k] /= lkk;
+        if (reject) p = 1.0;
+        const double rl = rsqrt(p);
+        __syncthreads();                       // every thread has read the pivot
+        if (tid == 0) { Gs[k * ld + k] = sqrt(p); rdiag[k] = rl; }
+        for (int i = k + 1 + tid; i < c; i += 256) Gs[i * ld + k] = reject ? 0.0 : Gs[i * ld + k] * rl;
         __syncthreads();
         // trailing update, one row per warp pass: lanes walk along the row
         const int rem = c - k - 1;
@@ -807,26 +810,28 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
         }
         __syncthreads();
     }
-    // in-place inverse of the lower-triangular L, row by row
-    for (int i = 0; i < c; ++i) {
-        double lii = Gs[i * ld + i];
-        double val = 0.0;
-        int j = tid;  // c <= 192 <= 256: one column per thread
-        if (j < i) {
-            double s = 0.0;
-            for (int k = j; k < i; ++k) s += Gs[i * ld + k] * Gs[k * ld + j];
-            val = -s / lii;
+    // Inverse of the lower-triangular L by forward substitution, one column per thread and no barrier: column j of
+    // X = L^-1 is x_j = 1 / l_jj, x_i = -(sum_{k = j}^{i - 1} l_ik x_k) / l_ii; it is kept in row j of the unused upper
+    // triangle (X[i][j] at Gs[j][i]), the diagonal in rdiag.
+    if (tid < c) {
+        const int j = tid;
+        double* xr = Gs + (size_t)j * ld;       // xr[i] = X[i][j] for i > j
+        const double xj = rdiag[j];
+        for (int i = j + 1; i < c; ++i) {
+            const double* li = Gs + (size_t)i * ld;
+            double s0 = li[j] * xj, s1 = 0.0;
+            int k = j + 1;
+            for (; k + 1 < i; k += 2) { s0 = fma(li[k], xr[k], s0); s1 = fma(li[k + 1], xr[k + 1], s1); }
+            if (k < i) s0 = fma(li[k], xr[k], s0);
+            xr[i] = -(s0 + s1) * rdiag[i];
         }
-        __syncthreads();
-        if (j < i) Gs[i * ld + j] = val;
-        if (j == i) Gs[i * ld + i] = 1.0 / lii;
-        __syncthreads();
     }
+    __syncthreads();
     // T[j][k] = dinv[j] * Linv[k][j]  for j <= k
     double* Tb = T + (size_t)blockIdx.x * c * c;
     for (int e = tid; e < c * c; e += 256) {
         int j = e / c, k = e % c;
-        Tb[e] = (j <= k) ? dinv[j] * Gs[k * ld + j] : 0.0;
+        Tb[e] = (j < k) ? dinv[j] * Gs[j * ld + k] : (j == k ? dinv[j] * rdiag[j] : 0.0);
     }
     if (defic)
         for (int k = tid; k < c; k += 256) defic[(size_t)blockIdx.x * c + k] = dcol[k];
