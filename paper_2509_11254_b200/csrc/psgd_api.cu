@@ -616,18 +616,17 @@ int launch_back_tc(Launcher& L, const float* M, const float* Phat, float* part, 
         const int kbs = ceil_div(KB, s);
         if (s > 1 && kbs < 16) break;
         if ((int64_t)(s - 1) * kbs >= KB) continue;     // would leave an empty split
-        const int64_t cost = ((base * s + h->sm_count - 1) / h->sm_count) * (kbs + 8);
+        const int64_t cost = ((base * s + h->sm_count - 1) / h->sm_count) * (kbs + 10);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
     }
     const int St = best, kbs = ceil_div(KB, St);
-    float* Pt = (float*)(h->ws + h->lay.ptQ);
-    const size_t tot = (size_t)count * Ncp * rows;
+    float* Pimg = (float*)(h->ws + h->lay.ptQ);        // P~^T as one shared-memory image per K block of 32 rows
+    const size_t tot = (size_t)count * KB * Ncp * TC_BK;
     L.begin(PSGD_K_BACKPROJECT);
-    k_split_pad_t<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Phat, Pt, rows, r, Ncp, count, skip);
+    k_split_img_t<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(Phat, Pimg, rows, r, Ncp, KB, count, skip);
     L.end();
-    CUtensorMap tM, tP[3];
+    CUtensorMap tM;
     bool ok = make_tile_map(h, &tM, M, n, rows, mats, 32, TC_BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
-    for (int t = 0; t < 3 && ok; ++t) ok = make_tile_map(h, &tP[t], Pt + t * tot, rows, Ncp, count, TC_BK, Ncp, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) {
         snprintf(h->err, sizeof(h->err), "cuTensorMapEncodeTiled failed");
         L.status = PSGD_E_CUDA;
@@ -637,7 +636,7 @@ int launch_back_tc(Launcher& L, const float* M, const float* Phat, float* part, 
     size_t smem = back_tc_smem_bytes(Ncp);
     set_smem_attr((const void*)k_backproject_tc, smem);
     L.begin(PSGD_K_BACKPROJECT);
-    k_backproject_tc<<<dim3(ceil_div(n, TC_BM), St, mats), PT_THREADS, smem, L.st>>>(tM, tP[0], tP[1], tP[2], a);
+    k_backproject_tc<<<dim3(ceil_div(n, TC_BM), St, mats), PT_THREADS, smem, L.st>>>(tM, Pimg, a);
     L.end();
     return St;
 }

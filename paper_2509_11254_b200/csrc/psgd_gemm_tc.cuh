@@ -433,14 +433,16 @@ k_residual_tc(const __grid_constant__ CUtensorMap tmPh, const __grid_constant__ 
 namespace psgd {
 
 // ---------------------------------------------------------------------------------------------
-// Projection on the tensor cores for ranks above 16:  P_i = (A_i [+ B_i]) Q  (Algorithm 1: P^(i) <-
-// Delta^(i) Q, with the error-feedback add of Eq. (7a) fused in; optionally stores M = A + B).
+// Projection on the tensor cores (ranks above 16; with the pending residual of the two-pass deferred mode
+// from 9 columns on):  P_i = (A_i [+ B_i]) Q  (Algorithm 1: P^(i) <- Delta^(i) Q, with the error-feedback
+// add of Eq. (7a) fused in; optionally stores M = A + B).
 // Per 32-column K block TMA brings the 128 x 32 tiles of A and B (128-byte swizzled); eight
 // converter warps form M in place of A and write it back to HBM.  M is used as two TF32 terms: the
 // head is M itself (the tensor core reads a float32 as TF32, i.e. truncated), the second term is
 // M - head rounded to the nearest TF32 number, written over the tile of B; what is left (at most
 // 2^-21 |M|, zero mean) averages out over the hundreds of columns of a sum.  Q^T arrives pre-split
-// into three exact terms (k_split_pad_t).  Products: h x [h|m|l] and m x [h|m]; m x l is below 2^-32.
+// into three exact terms, one untiled bulk copy per K block of an image in shared-memory order
+// (k_split_img_t).  Products: h x [h|m|l] and m x [h|m]; m x l is below 2^-32.
 //
 // Accumulation.  The tensor core adds to its float32 accumulator with truncation (measured on
 // like-signed sums: 3e-8 relative per accumulation, always toward zero, i.e. 2e-5 over the 512
@@ -551,25 +553,8 @@ __host__ __device__ inline size_t proj_tc_smem_bytes(int Ncp, bool pend = false)
            (size_t)proj_tc_pend_bytes(pend) + 1024 + 512;
 }
 
-// Q [count][n][r] -> Qt[t][count][Ncp][n], t = 0, 1, 2: the transposed factor split exactly into three TF32 terms,
-// rows k >= r zero.  One thread per (matrix, k, column).
-__global__ void k_split_pad_t(const float* Q, float* Qt, int n, int r, int Ncp, int count, const int* skip) {
-    if (skip && *skip) return;
-    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const size_t per = (size_t)Ncp * n, tot = per * count;
-    if (idx >= tot) return;
-    const int c = (int)(idx / per);
-    const int k = (int)((idx % per) / n), col = (int)(idx % n);
-    float x = (k < r) ? Q[((size_t)c * n + col) * r + k] : 0.f;
-    float h = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
-    float r1 = x - h;
-    float mm = __uint_as_float(__float_as_uint(r1) & 0xFFFFE000u);
-    Qt[idx] = h;
-    Qt[tot + idx] = mm;
-    Qt[2 * tot + idx] = r1 - mm;
-}
-
-// Q [count][n][r] -> Qimg[count][KB][t][Ncp][32], t = 0, 1, 2: the same three exact terms, laid out as the shared-memory
+// Q [count][n][r] -> Qimg[count][KB][t][Ncp][32], t = 0, 1, 2: the transposed factor split exactly into three TF32 terms
+// (h = x with its 13 low mantissa bits cleared, m the same of x - h, l the rest), laid out as the shared-memory
 // image of one K block after the other (rows of 128 bytes, 128-byte swizzle: the 16-byte unit u of row k sits at unit
 // u ^ (k & 7)), so that ONE untiled bulk copy of 3 Ncp 128 bytes brings what a K block needs.  Columns beyond n and rows
 // k >= r are zero.  One thread per (matrix, K block, k, column).
@@ -1016,13 +1001,14 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 // MN-major operand: TMA brings 32-row x 32-column boxes of M exactly as they lie in memory (128-byte
 // lines, 32-byte swizzle atoms, the one shared-memory form TF32 operands have in this orientation);
 // four boxes side by side give the 128 columns of one CTA.  P~^T arrives pre-split and K-major
-// (k_split_pad_t on P~, three exact terms).  The tile of M is used as two terms: the head is the tile
+// (k_split_img_t on P~, three exact terms).  The tile of M is used as two terms: the head is the tile
 // itself (read as TF32, i.e. truncated), the second term is x - head rounded to the nearest TF32
 // number, written by the converter warps; what is left of x (at most 2^-21 |x|, zero mean) averages
 // out over the hundreds of rows of a sum.  Products: h x [h|m|l] and m x [h|m]; m x l is below 2^-32.
-// Two shared-memory rings: a deep one for the tiles of M (16 KB stages) and a short one for what
-// lives only from the conversion to the end of the MMAs (the second term of the tile, the three
-// terms of P~^T).  One mbarrier per K block ("done", by tcgen05.commit) frees both stages and tells
+// Three shared-memory rings: a deep one for the tiles of M (16 KB stages), a short one for the second
+// term of the tile (it lives only from the conversion to the end of the MMAs) and one for the three
+// terms of P~^T, one untiled bulk copy per K block of an image in shared-memory order (k_split_img_t);
+// the last is requested as many K blocks ahead as it has stages, because the MMAs wait for it.  One mbarrier per K block ("done", by tcgen05.commit) frees both stages and tells
 // the adder warps that the accumulators of that K block can be read.
 //   up to 80 columns: the three terms of P~^T lie side by side as one B operand of 3 Ncp <= 256 rows:
 //     two MMAs per 8 rows (the slow MN-major operand is fetched twice instead of six times); an
@@ -1045,15 +1031,20 @@ struct BackTcArgs {
     const int* skip;
 };
 
-__host__ __device__ inline size_t back_tc_short_stage_bytes(int Ncp) { return (size_t)TC_BM * TC_BK * 4 + (size_t)3 * Ncp * TC_BK * 4; }
-// stages of the M ring that fit beside the short ring in 224 KB (0: does not fit)
+// Stages of the ring of P~^T terms.  Its loads are small but wanted early (the MMAs of a K block cannot start without them)
+// and take a full memory latency, so for narrow factors the ring is deeper than the ring of second terms it used to share.
+__host__ __device__ inline int back_tc_np(int Ncp) { return Ncp <= 16 ? 8 : (Ncp <= 32 ? 6 : (Ncp <= 48 ? 4 : back_tc_nm(Ncp))); }
+__host__ __device__ inline size_t back_tc_fixed_bytes(int Ncp) {
+    return (size_t)back_tc_nm(Ncp) * TC_BM * TC_BK * 4 + (size_t)back_tc_np(Ncp) * 3 * Ncp * TC_BK * 4;
+}
+// stages of the M ring that fit beside the two short rings in 224 KB (0: does not fit)
 __host__ __device__ inline int back_tc_nh(int Ncp) {
-    const long long left = 224ll * 1024 - 1024 - 512 - (long long)back_tc_nm(Ncp) * (long long)back_tc_short_stage_bytes(Ncp);
+    const long long left = 224ll * 1024 - 1024 - 512 - (long long)back_tc_fixed_bytes(Ncp);
     const int nh = (int)(left / (TC_BM * TC_BK * 4));
     return nh > BT_NHMAX ? BT_NHMAX : nh;
 }
 __host__ __device__ inline size_t back_tc_smem_bytes(int Ncp) {
-    return (size_t)back_tc_nh(Ncp) * TC_BM * TC_BK * 4 + back_tc_nm(Ncp) * back_tc_short_stage_bytes(Ncp) + 1024 + 512;
+    return (size_t)back_tc_nh(Ncp) * TC_BM * TC_BK * 4 + back_tc_fixed_bytes(Ncp) + 1024 + 512;
 }
 
 // shared-memory descriptor of an MN-major TF32 tile: lines of 32 floats along MN, 4-row atoms of 512 bytes along K
@@ -1069,8 +1060,7 @@ __device__ __forceinline__ unsigned long long tc_smem_desc_mn(unsigned addr, uns
 }
 
 __global__ void __launch_bounds__(PT_THREADS, 1)
-k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmP0,
-                 const __grid_constant__ CUtensorMap tmP1, const __grid_constant__ CUtensorMap tmP2, BackTcArgs a) {
+k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const float* __restrict__ Pimg, BackTcArgs a) {
     extern __shared__ __align__(16) unsigned char bt_smem_raw[];
     if (a.skip && *a.skip) return;
     unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(bt_smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -1078,16 +1068,17 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     constexpr unsigned A_BYTES = TC_BM * TC_BK * 4;            // 128 columns x 32 rows
     constexpr unsigned BOX_BYTES = 32 * TC_BK * 4;             // one 32-column box
     const unsigned B_BYTES = (unsigned)a.Ncp * TC_BK * 4;
-    const unsigned SHORT_BYTES = A_BYTES + 3 * B_BYTES;        // [m tile][h, m, l of P~^T]
+    const unsigned P_BYTES = 3 * B_BYTES;                      // h, m, l of P~^T of one K block
     const bool wide = 3 * a.Ncp <= 256;
-    const int NM = back_tc_nm(a.Ncp);
+    const int NM = back_tc_nm(a.Ncp), NP = back_tc_np(a.Ncp);
     const int NH = a.nh, NB = wide ? min(4, 512 / (3 * a.Ncp)) : min(3, (512 - 2 * a.Ncp) / a.Ncp);
-    unsigned char* short_base = base + (size_t)NH * A_BYTES;
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(short_base + (size_t)NM * SHORT_BYTES);
+    unsigned char* short_base = base + (size_t)NH * A_BYTES;             // second terms of the tiles of M: NM stages
+    unsigned char* p_base = short_base + (size_t)NM * A_BYTES;           // terms of P~^T: NP stages
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(p_base + (size_t)NP * P_BYTES);
     const unsigned bar_hfull = smem_u32(bars), bar_done = bar_hfull + 8 * NH, bar_bfull = bar_done + 8 * NH;
-    const unsigned bar_conv = bar_bfull + 8 * NM, bar_free = bar_conv + 8 * NM, bar_acc = bar_free + 8 * NB;
-    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 2 * NH + 2 * NM + NB + 1);
-    const unsigned ring_u32 = smem_u32(base), short_u32 = smem_u32(short_base);
+    const unsigned bar_conv = bar_bfull + 8 * NP, bar_free = bar_conv + 8 * NM, bar_acc = bar_free + 8 * NB;
+    unsigned* tmem_slot = reinterpret_cast<unsigned*>(bars + 2 * NH + NP + NM + NB + 1);
+    const unsigned ring_u32 = smem_u32(base), short_u32 = smem_u32(short_base), p_u32 = smem_u32(p_base);
 
     const int ct = blockIdx.x, sp = blockIdx.y, mat = blockIdx.z;
     const int pz = mat / a.nodes;
@@ -1099,7 +1090,8 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
 
     if (tid == 0) {
         for (int s = 0; s < NH; ++s) { mbar_init(bar_hfull + 8 * s, 1); mbar_init(bar_done + 8 * s, 1); }
-        for (int s = 0; s < NM; ++s) { mbar_init(bar_bfull + 8 * s, 1); mbar_init(bar_conv + 8 * s, 8); }
+        for (int s = 0; s < NP; ++s) mbar_init(bar_bfull + 8 * s, 1);
+        for (int s = 0; s < NM; ++s) mbar_init(bar_conv + 8 * s, 8);
         for (int b = 0; b < NB; ++b) mbar_init(bar_free + 8 * b, 8);
         mbar_init(bar_acc, 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
@@ -1117,9 +1109,10 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     auto wait_done = [&](int j) { mbar_wait(bar_done + 8 * (j % NH), (unsigned)((j / NH) & 1), a.flags, dead); };
 
     if (warp == 0) {
-        // ---- TMA producer: tiles of M run NH - NM K blocks ahead of the terms of P~^T ----
+        // ---- TMA producer: tiles of M run NH - NP K blocks ahead of the terms of P~^T (one bulk copy per K block) ----
         if (lane == 0) {
-            const int lead = NH - NM;
+            const int lead = max(NH - NP, 0);
+            const float* psrc = Pimg + ((size_t)pz * KBall + kb0) * (P_BYTES / 4);
             auto issue_m = [&](int j) {
                 const int s = j % NH;
                 if (j >= NH) wait_done(j - NH);
@@ -1132,14 +1125,11 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
             for (int j = 0; j < min(lead, KB); ++j) issue_m(j);
             for (int kb = 0; kb < KB; ++kb) {
                 if (kb + lead < KB) issue_m(kb + lead);
-                const int s = kb % NM;
-                if (kb >= NM) wait_done(kb - NM);
-                const unsigned dst = short_u32 + s * SHORT_BYTES + A_BYTES, bar = bar_bfull + 8 * s;
-                const int row = (kb0 + kb) * TC_BK;
-                mbar_expect_tx(bar, 3u * B_BYTES);
-                tma_load_3d_sw(dst, &tmP0, row, 0, pz, bar);
-                tma_load_3d_sw(dst + B_BYTES, &tmP1, row, 0, pz, bar);
-                tma_load_3d_sw(dst + 2 * B_BYTES, &tmP2, row, 0, pz, bar);
+                const int s = kb % NP;
+                if (kb >= NP) wait_done(kb - NP);
+                const unsigned dst = p_u32 + s * P_BYTES, bar = bar_bfull + 8 * s;
+                mbar_expect_tx(bar, P_BYTES);
+                bulk_load_1d(dst, psrc + (size_t)kb * (P_BYTES / 4), P_BYTES, bar);
             }
         }
     } else if (warp == 1) {
@@ -1149,16 +1139,16 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
             const unsigned id2 = tc_idesc(2 * a.Ncp) | (1u << 15), id3 = tc_idesc(wide ? 3 * a.Ncp : a.Ncp) | (1u << 15);
             // one thread: ring positions and parities as counters, descriptors as offsets from those of stage 0
             const unsigned long long dA0 = tc_smem_desc_mn(ring_u32, BOX_BYTES), dM0 = tc_smem_desc_mn(short_u32, BOX_BYTES);
-            const unsigned long long dP0 = tc_smem_desc(short_u32 + A_BYTES);
-            const unsigned long long long_step = A_BYTES >> 4, short_step = SHORT_BYTES >> 4, b_off = B_BYTES >> 4;
-            int sh = 0, sm = 0, phm = 0, hb = 0, phb = 1;
+            const unsigned long long dP0 = tc_smem_desc(p_u32);
+            const unsigned long long long_step = A_BYTES >> 4, p_step = P_BYTES >> 4, b_off = B_BYTES >> 4;
+            int sh = 0, sm = 0, phm = 0, sp_ = 0, php = 0, hb = 0, phb = 1;
             for (int kb = 0; kb < KB; ++kb) {
                 mbar_wait_ready(bar_conv + 8 * sm, (unsigned)phm, a.flags, dead);
-                mbar_wait_ready(bar_bfull + 8 * sm, (unsigned)phm, a.flags, dead);
+                mbar_wait_ready(bar_bfull + 8 * sp_, (unsigned)php, a.flags, dead);
                 if (kb >= NB) mbar_wait_ready(bar_free + 8 * hb, (unsigned)phb, a.flags, dead);   // registers took its last content
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-                const unsigned long long dAh = dA0 + (unsigned long long)sh * long_step, dAm = dM0 + (unsigned long long)sm * short_step;
-                const unsigned long long dPh = dP0 + (unsigned long long)sm * short_step, dPm = dPh + b_off;
+                const unsigned long long dAh = dA0 + (unsigned long long)sh * long_step, dAm = dM0 + (unsigned long long)sm * long_step;
+                const unsigned long long dPh = dP0 + (unsigned long long)sp_ * p_step, dPm = dPh + b_off;
                 if (wide) {
                     const unsigned d_set = tmem + (unsigned)(3 * hb * a.Ncp);
 #pragma unroll
@@ -1181,6 +1171,7 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
                 tc_commit(bar_done + 8 * sh);
                 if (++sh == NH) sh = 0;
                 if (++sm == NM) { sm = 0; phm ^= 1; }
+                if (++sp_ == NP) { sp_ = 0; php ^= 1; }
                 if (++hb == NB) { hb = 0; phb ^= 1; }
             }
             tc_commit(bar_acc);
@@ -1193,7 +1184,7 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
             mbar_wait(bar_hfull + 8 * sh, (unsigned)((kb / NH) & 1), a.flags, dead);
             if (kb >= NM) wait_done(kb - NM);          // the MMAs that read this short stage have completed
             const float4* t0 = reinterpret_cast<const float4*>(base + (size_t)sh * A_BYTES);
-            float4* t1 = reinterpret_cast<float4*>(short_base + (size_t)sm * SHORT_BYTES);
+            float4* t1 = reinterpret_cast<float4*>(short_base + (size_t)sm * A_BYTES);
 #pragma unroll
             for (int u = 0; u < (TC_BM * TC_BK / 4) / 256; ++u) {
                 const int o = cv + u * 256;
