@@ -719,26 +719,34 @@ k_project_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 mbar_expect_tx(bar_pfull, PT_PIMG_BYTES);
                 bulk_load_1d(pimg_u32, a.Pimg + ((size_t)qz * gridDim.x + rt) * (PT_PIMG_BYTES / 4), PT_PIMG_BYTES, bar_pfull);
             }
-            auto issue_ab = [&](int j) {
-                const int s = j % NH;
-                if (j >= NH) {
-                    wait_done(j - NH);
-                    if (PEND) mbar_wait(bar_stored + 8 * s, (unsigned)(((j - NH) / NH) & 1), a.flags, dead);   // its M has left for HBM
+            // (one thread: positions and parities as counters, a non-blocking test before every wait)
+            int aj = 0, as = 0, aph = 1;             // next tile pair: index, stage j % NH, parity of "done"/"stored" of tile j - NH
+            auto issue_ab = [&]() {
+                if (aj >= NH) {
+                    mbar_wait_ready(bar_done + 8 * as, (unsigned)aph, a.flags, dead);
+                    if (PEND) mbar_wait_ready(bar_stored + 8 * as, (unsigned)aph, a.flags, dead);   // its M has left for HBM
                 }
-                const unsigned dst = ring_u32 + s * LONG_BYTES, bar = bar_hfull + 8 * s;
-                PTC_STAMP(0, j);
+                const unsigned dst = ring_u32 + as * LONG_BYTES, bar = bar_hfull + 8 * as;
+                PTC_STAMP(0, aj);
                 mbar_expect_tx(bar, (a.has_b ? 2u : 1u) * A_BYTES);
-                tma_load_3d_sw(dst, &tmA, (kb_lo + j) * TC_BK, rt * TC_BM, mat, bar);
-                if (a.has_b) tma_load_3d_sw(dst + A_BYTES, &tmB, (kb_lo + j) * TC_BK, rt * TC_BM, mat, bar);
+                tma_load_3d_sw(dst, &tmA, (kb_lo + aj) * TC_BK, rt * TC_BM, mat, bar);
+                if (a.has_b) tma_load_3d_sw(dst + A_BYTES, &tmB, (kb_lo + aj) * TC_BK, rt * TC_BM, mat, bar);
+                ++aj;
+                if (++as == NH) { as = 0; aph ^= 1; }
             };
-            for (int j = 0; j < min(lead, KB); ++j) issue_ab(j);
+            for (int j = 0; j < min(lead, KB); ++j) issue_ab();
+            const float* qsrc = Qimg + ((size_t)qz * KBt + kb_lo) * (3u * B_BYTES / 4);
+            int ss = 0, ds = 0, dph = 0;             // stage kb % NM; stage and parity of "done" of K block kb - NM
             for (int kb = 0; kb < KB; ++kb) {
-                if (kb + lead < KB) issue_ab(kb + lead);
-                const int s = kb % NM;
-                if (kb >= NM) wait_done(kb - NM);
-                const unsigned dst = short_u32 + s * SHORT_BYTES, bar = bar_bfull + 8 * s;
+                if (aj < KB) issue_ab();
+                if (kb >= NM) {
+                    mbar_wait_ready(bar_done + 8 * ds, (unsigned)dph, a.flags, dead);
+                    if (++ds == NH) { ds = 0; dph ^= 1; }
+                }
+                const unsigned dst = short_u32 + ss * SHORT_BYTES, bar = bar_bfull + 8 * ss;
                 mbar_expect_tx(bar, SHORT_BYTES);
-                bulk_load_1d(dst, Qimg + ((size_t)qz * KBt + kb_lo + kb) * (3u * B_BYTES / 4), 3u * B_BYTES, bar);
+                bulk_load_1d(dst, qsrc + (size_t)kb * (3u * B_BYTES / 4), 3u * B_BYTES, bar);
+                if (++ss == NM) ss = 0;
             }
         }
     } else if (warp == 1) {
@@ -1113,23 +1121,30 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const float* __restric
         if (lane == 0) {
             const int lead = max(NH - NP, 0);
             const float* psrc = Pimg + ((size_t)pz * KBall + kb0) * (P_BYTES / 4);
-            auto issue_m = [&](int j) {
-                const int s = j % NH;
-                if (j >= NH) wait_done(j - NH);
-                const unsigned dst = ring_u32 + s * A_BYTES, bar = bar_hfull + 8 * s;
-                const int row = (kb0 + j) * TC_BK;
+            // (one thread: positions and parities as counters, a non-blocking test before every wait)
+            int mj = 0, ms = 0, mph = 1;             // next tile of M: index, stage j % NH, parity of "done" of tile j - NH
+            auto issue_m = [&]() {
+                if (mj >= NH) mbar_wait_ready(bar_done + 8 * ms, (unsigned)mph, a.flags, dead);
+                const unsigned dst = ring_u32 + ms * A_BYTES, bar = bar_hfull + 8 * ms;
+                const int row = (kb0 + mj) * TC_BK;
                 mbar_expect_tx(bar, A_BYTES);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) tma_load_3d_sw(dst + q * BOX_BYTES, &tmM, ct * TC_BM + 32 * q, row, mat, bar);
+                ++mj;
+                if (++ms == NH) { ms = 0; mph ^= 1; }
             };
-            for (int j = 0; j < min(lead, KB); ++j) issue_m(j);
+            for (int j = 0; j < min(lead, KB); ++j) issue_m();
+            int ps = 0, ds = 0, dph = 0;             // stage kb % NP; stage and parity of "done" of K block kb - NP
             for (int kb = 0; kb < KB; ++kb) {
-                if (kb + lead < KB) issue_m(kb + lead);
-                const int s = kb % NP;
-                if (kb >= NP) wait_done(kb - NP);
-                const unsigned dst = p_u32 + s * P_BYTES, bar = bar_bfull + 8 * s;
+                if (mj < KB) issue_m();
+                if (kb >= NP) {
+                    mbar_wait_ready(bar_done + 8 * ds, (unsigned)dph, a.flags, dead);
+                    if (++ds == NH) { ds = 0; dph ^= 1; }
+                }
+                const unsigned dst = p_u32 + ps * P_BYTES, bar = bar_bfull + 8 * ps;
                 mbar_expect_tx(bar, P_BYTES);
                 bulk_load_1d(dst, psrc + (size_t)kb * (P_BYTES / 4), P_BYTES, bar);
+                if (++ps == NP) ps = 0;
             }
         }
     } else if (warp == 1) {
