@@ -110,7 +110,7 @@ k_gemm_tf32(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (lane == 0) {
             for (int kb = 0; kb < nkb; ++kb) {
                 const int s = kb % TC_STAGES;
-                if (kb >= TC_STAGES) mbar_wait(bar_empty + 8 * s, (unsigned)((kb / TC_STAGES - 1) & 1), a.flags, dead);
+                if (kb >= TC_STAGES) mbar_wait_ready(bar_empty + 8 * s, (unsigned)((kb / TC_STAGES - 1) & 1), a.flags, dead);
                 const unsigned dst = smem_base + s * stage_bytes;
                 mbar_expect_tx(bar_full + 8 * s, stage_bytes);
                 tma_load_3d_sw(dst, &tmA, (kb0 + kb) * TC_BK, mt * TC_BM, c, bar_full + 8 * s);
@@ -123,7 +123,7 @@ k_gemm_tf32(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const unsigned idesc = tc_idesc(a.Ncp);
             for (int kb = 0; kb < nkb; ++kb) {
                 const int s = kb % TC_STAGES;
-                mbar_wait(bar_full + 8 * s, (unsigned)((kb / TC_STAGES) & 1), a.flags, dead);
+                mbar_wait_ready(bar_full + 8 * s, (unsigned)((kb / TC_STAGES) & 1), a.flags, dead);
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                 const unsigned long long da = tc_smem_desc(smem_base + s * stage_bytes);
                 const unsigned long long db = tc_smem_desc(smem_base + s * stage_bytes + a_bytes);
@@ -292,10 +292,9 @@ k_residual_tc(const __grid_constant__ CUtensorMap tmPh, const __grid_constant__ 
     if (warp == 0) {
         // ---- TMA producer: per (column tile, K chunk) the heads and tails of both factors ----
         if (lane == 0) {
-            for (int it = 0; it < total; ++it) {
+            for (int it = 0, ct = 0, kc = 0; it < total; ++it, ct += (kc + 1 == nkc), kc = (kc + 1 == nkc) ? 0 : kc + 1) {
                 const int s = it % RT_STAGES;
-                const int ct = it / nkc, kc = it % nkc;
-                if (it >= RT_STAGES) mbar_wait(bar_empty + 8 * s, (unsigned)((it / RT_STAGES - 1) & 1), a.flags, dead);
+                if (it >= RT_STAGES) mbar_wait_ready(bar_empty + 8 * s, (unsigned)((it / RT_STAGES - 1) & 1), a.flags, dead);
                 const unsigned dst = smem_base + s * STAGE_BYTES;
                 const unsigned bar = bar_full + 8 * s;
                 mbar_expect_tx(bar, STAGE_BYTES);
@@ -312,12 +311,11 @@ k_residual_tc(const __grid_constant__ CUtensorMap tmPh, const __grid_constant__ 
         // ---- MMA issuer ----
         if (lane == 0) {
             const unsigned idesc = tc_idesc(RT_BN);
-            for (int it = 0; it < total; ++it) {
+            for (int it = 0, ct = 0, kc = 0; it < total; ++it, ct += (kc + 1 == nkc), kc = (kc + 1 == nkc) ? 0 : kc + 1) {
                 const int s = it % RT_STAGES;
-                const int ct = it / nkc, kc = it % nkc;
                 const int ab = ct & 1;                                   // accumulator buffer
-                if (kc == 0 && ct >= 2) mbar_wait(bar_acce + 8 * ab, (unsigned)(((ct >> 1) - 1) & 1), a.flags, dead);
-                mbar_wait(bar_full + 8 * s, (unsigned)((it / RT_STAGES) & 1), a.flags, dead);
+                if (kc == 0 && ct >= 2) mbar_wait_ready(bar_acce + 8 * ab, (unsigned)(((ct >> 1) - 1) & 1), a.flags, dead);
+                mbar_wait_ready(bar_full + 8 * s, (unsigned)((it / RT_STAGES) & 1), a.flags, dead);
                 asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
                 const unsigned sb = smem_base + s * STAGE_BYTES;
                 const unsigned long long dP[3] = {tc_smem_desc(sb), tc_smem_desc(sb + A_BYTES), tc_smem_desc(sb + 2 * A_BYTES)};
@@ -1148,15 +1146,21 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const float* __restric
             }
         }
     } else if (warp == 1) {
-        // ---- MMA issuer ----
+        // ---- MMA issuer (one thread; a second one taking every other K block was measured and changed nothing) ----
         if (lane == 0) {
             const unsigned id1 = tc_idesc(a.Ncp) | (1u << 15);            // bit 15: A is MN-major
             const unsigned id2 = tc_idesc(2 * a.Ncp) | (1u << 15), id3 = tc_idesc(wide ? 3 * a.Ncp : a.Ncp) | (1u << 15);
-            // one thread: ring positions and parities as counters, descriptors as offsets from those of stage 0
+            // ring positions and parities as counters, descriptors as offsets from those of stage 0
             const unsigned long long dA0 = tc_smem_desc_mn(ring_u32, BOX_BYTES), dM0 = tc_smem_desc_mn(short_u32, BOX_BYTES);
             const unsigned long long dP0 = tc_smem_desc(p_u32);
             const unsigned long long long_step = A_BYTES >> 4, p_step = P_BYTES >> 4, b_off = B_BYTES >> 4;
             int sh = 0, sm = 0, phm = 0, sp_ = 0, php = 0, hb = 0, phb = 1;
+            auto advance = [&]() {
+                if (++sh == NH) sh = 0;
+                if (++sm == NM) { sm = 0; phm ^= 1; }
+                if (++sp_ == NP) { sp_ = 0; php ^= 1; }
+                if (++hb == NB) { hb = 0; phb ^= 1; }
+            };
             for (int kb = 0; kb < KB; ++kb) {
                 mbar_wait_ready(bar_conv + 8 * sm, (unsigned)phm, a.flags, dead);
                 mbar_wait_ready(bar_bfull + 8 * sp_, (unsigned)php, a.flags, dead);
@@ -1184,10 +1188,7 @@ k_backproject_tc(const __grid_constant__ CUtensorMap tmM, const float* __restric
                     }
                 }
                 tc_commit(bar_done + 8 * sh);
-                if (++sh == NH) sh = 0;
-                if (++sm == NM) { sm = 0; phm ^= 1; }
-                if (++sp_ == NP) { sp_ = 0; php ^= 1; }
-                if (++hb == NB) { hb = 0; phb ^= 1; }
+                advance();
             }
             tc_commit(bar_acc);
         }
