@@ -744,6 +744,7 @@ __global__ void k_gram_sum(double* part, int cc, int nparts, int count, const in
 // Dynamic shared memory: c * chol_ld(c) doubles (rows padded to an odd number of doubles so that
 // walking down a column is free of bank conflicts).
 constexpr double CHOL_PIVOT_TOL = 1e-11;  // squared sine of the angle to the previous columns
+constexpr int CHOL_NB = 8;                // columns per panel of the factorisation
 __host__ __device__ inline int chol_ld(int c) { return c | 1; }
 // `gate` (optional): set to 1 when a scaled pivot^2 falls below gate_tol, i.e. when the columns
 // are too ill-conditioned for results derived from W = M^T P to keep float32 accuracy.
@@ -764,14 +765,15 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
     if (nparts < 0) nparts = 1;
     const double* pb = part + (size_t)blockIdx.x * pstride * c * c;
     if (tid == 0) { bad = 0; illc = 0; }
-    for (int e = tid; e < c * c; e += 256) {
-        int i = e / c, j = e % c;
-        int ii = i, jj = j;
-        if (i / 64 > j / 64) { ii = j; jj = i; }   // lower block triangle was not computed: mirror
-        double s = 0.0;
-        for (int p = 0; p < nparts; ++p) s += pb[(size_t)p * c * c + (size_t)ii * c + jj];
-        Gs[i * ld + j] = s;
-    }
+    const int tx = tid & 31, ty = tid >> 5;          // lanes along a row, 8 rows at a time
+    for (int i = ty; i < c; i += 8)
+        for (int j = tx; j < c; j += 32) {
+            int ii = i, jj = j;
+            if ((i >> 6) > (j >> 6)) { ii = j; jj = i; }   // lower block triangle was not computed: mirror
+            double s = 0.0;
+            for (int p = 0; p < nparts; ++p) s += pb[(size_t)p * c * c + (size_t)ii * c + jj];
+            Gs[i * ld + j] = s;
+        }
     __syncthreads();
     for (int k = tid; k < c; k += 256) {
         double d = Gs[k * ld + k];
@@ -779,60 +781,88 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
         if (!(d > 0.0)) { dinv[k] = 0.0; bad = 1; dcol[k] = 1; } else dinv[k] = 1.0 / sqrt(d);
     }
     __syncthreads();
-    for (int e = tid; e < c * c; e += 256) {
-        int i = e / c, j = e % c;
-        double v = Gs[i * ld + j] * dinv[i] * dinv[j];
-        if (i == j && dinv[i] == 0.0) v = 1.0;  // zero column: decouple it (fixed up later)
-        Gs[i * ld + j] = v;
-    }
+    for (int i = ty; i < c; i += 8)
+        for (int j = tx; j < c; j += 32) {
+            double v = Gs[i * ld + j] * dinv[i] * dinv[j];
+            if (i == j && dinv[i] == 0.0) v = 1.0;  // zero column: decouple it (fixed up later)
+            Gs[i * ld + j] = v;
+        }
     __syncthreads();
-    // right-looking Cholesky on the lower triangle: Gs = L L^T.  Every thread evaluates the pivot of the step itself (no
-    // serial step by one thread): two barriers per column.
-    for (int k = 0; k < c; ++k) {
-        double p = Gs[k * ld + k];
-        const bool reject = !(p > CHOL_PIVOT_TOL);
-        if (tid == 0) {
-            if (!(p > gate_tol)) illc = 1;
-            if (reject) { bad = 1; dcol[k] = 1; }
+    // Right-looking Cholesky on the lower triangle, Gs = L L^T, in panels of CHOL_NB columns: a column's update is applied at
+    // once only to the rest of its panel (a few entries per thread between barriers); the matrix behind the panel receives the
+    // panel's CHOL_NB rank-one updates in one pass (same terms in the same order, one load and store per entry instead of
+    // CHOL_NB).  Every thread evaluates the pivot of a column itself (no serial step by one thread).
+    for (int k0 = 0; k0 < c; k0 += CHOL_NB) {
+        const int kend = min(c, k0 + CHOL_NB);
+        for (int k = k0; k < kend; ++k) {
+            double p = Gs[k * ld + k];
+            const bool reject = !(p > CHOL_PIVOT_TOL);
+            if (tid == 0) {
+                if (!(p > gate_tol)) illc = 1;
+                if (reject) { bad = 1; dcol[k] = 1; }
+            }
+            if (reject) p = 1.0;
+            const double rl = rsqrt(p);
+            __syncthreads();                       // every thread has read the pivot
+            if (tid == 0) { Gs[k * ld + k] = sqrt(p); rdiag[k] = rl; }
+            for (int i = k + 1 + tid; i < c; i += 256) Gs[i * ld + k] = reject ? 0.0 : Gs[i * ld + k] * rl;
+            __syncthreads();
+            const int w = kend - k - 1;            // columns of the panel still to come
+            if (w > 0) {                           // eight threads per row (one per panel column, CHOL_NB = 8), 32 rows per pass
+                const int j = k + 1 + (tid & 7);
+                if ((tid & 7) < w) {
+                    const double ljk = Gs[j * ld + k];
+                    for (int i = k + 1 + (tid >> 3); i < c; i += 32)
+                        if (i >= j) Gs[i * ld + j] = fma(-Gs[i * ld + k], ljk, Gs[i * ld + j]);
+                }
+                __syncthreads();
+            }
         }
-        if (reject) p = 1.0;
-        const double rl = rsqrt(p);
-        __syncthreads();                       // every thread has read the pivot
-        if (tid == 0) { Gs[k * ld + k] = sqrt(p); rdiag[k] = rl; }
-        for (int i = k + 1 + tid; i < c; i += 256) Gs[i * ld + k] = reject ? 0.0 : Gs[i * ld + k] * rl;
-        __syncthreads();
-        // trailing update, one row per warp pass: lanes walk along the row
-        const int rem = c - k - 1;
-        for (int ri = (tid >> 5); ri < rem; ri += 8) {
-            const int i = k + 1 + ri;
-            const double lik = Gs[i * ld + k];
-            for (int j = k + 1 + (tid & 31); j <= i; j += 32) Gs[i * ld + j] -= lik * Gs[j * ld + k];
+        // behind the panel, one row per warp pass: lanes walk along the row
+        if (kend < c) {
+            for (int i = kend + (tid >> 5); i < c; i += 8) {
+                double li[CHOL_NB];
+#pragma unroll
+                for (int q = 0; q < CHOL_NB; ++q) li[q] = Gs[i * ld + k0 + q];
+                for (int j = kend + (tid & 31); j <= i; j += 32) {
+                    double g = Gs[i * ld + j];
+#pragma unroll
+                    for (int q = 0; q < CHOL_NB; ++q) g = fma(-li[q], Gs[j * ld + k0 + q], g);
+                    Gs[i * ld + j] = g;
+                }
+            }
+            __syncthreads();
         }
-        __syncthreads();
     }
-    // Inverse of the lower-triangular L by forward substitution, one column per thread and no barrier: column j of
-    // X = L^-1 is x_j = 1 / l_jj, x_i = -(sum_{k = j}^{i - 1} l_ik x_k) / l_ii; it is kept in row j of the unused upper
-    // triangle (X[i][j] at Gs[j][i]), the diagonal in rdiag.
-    if (tid < c) {
-        const int j = tid;
-        double* xr = Gs + (size_t)j * ld;       // xr[i] = X[i][j] for i > j
-        const double xj = rdiag[j];
-        for (int i = j + 1; i < c; ++i) {
-            const double* li = Gs + (size_t)i * ld;
-            double s0 = li[j] * xj, s1 = 0.0;
-            int k = j + 1;
-            for (; k + 1 < i; k += 2) { s0 = fma(li[k], xr[k], s0); s1 = fma(li[k + 1], xr[k + 1], s1); }
-            if (k < i) s0 = fma(li[k], xr[k], s0);
-            xr[i] = -(s0 + s1) * rdiag[i];
+    // Inverse of the lower-triangular L by forward substitution, no block-wide barrier: column j of X = L^-1 is
+    // x_j = 1 / l_jj, x_i = -(sum_{k = j}^{i - 1} l_ik x_k) / l_ii, kept in row j of the unused upper triangle (X[i][j] at
+    // Gs[j][i]), the diagonal in rdiag.  Two adjacent lanes share a column and take alternate terms of every sum (the first
+    // column's c^2 / 2 dependent steps set the time of the whole phase).
+    for (int j0 = 0; j0 < c; j0 += 128) {
+        const int j = j0 + (tid >> 1), hlf = tid & 1;
+        if (j < c) {
+            const unsigned pair = 3u << ((tid & 31) & ~1);
+            double* xr = Gs + (size_t)j * ld;       // xr[i] = X[i][j] for i > j
+            const double xj = rdiag[j];
+            for (int i = j + 1; i < c; ++i) {
+                const double* li = Gs + (size_t)i * ld;
+                double s0 = hlf ? 0.0 : li[j] * xj, s1 = 0.0;
+                int k = j + 1 + hlf;
+                for (; k + 2 < i; k += 4) { s0 = fma(li[k], xr[k], s0); s1 = fma(li[k + 2], xr[k + 2], s1); }
+                if (k < i) s0 = fma(li[k], xr[k], s0);
+                double sum = s0 + s1;
+                sum += __shfl_xor_sync(pair, sum, 1);
+                if (!hlf) xr[i] = -sum * rdiag[i];
+                __syncwarp(pair);
+            }
         }
     }
     __syncthreads();
     // T[j][k] = dinv[j] * Linv[k][j]  for j <= k
     double* Tb = T + (size_t)blockIdx.x * c * c;
-    for (int e = tid; e < c * c; e += 256) {
-        int j = e / c, k = e % c;
-        Tb[e] = (j < k) ? dinv[j] * Gs[j * ld + k] : (j == k ? dinv[j] * rdiag[j] : 0.0);
-    }
+    for (int j = ty; j < c; j += 8)
+        for (int k = tx; k < c; k += 32)
+            Tb[(size_t)j * c + k] = (j < k) ? dinv[j] * Gs[j * ld + k] : (j == k ? dinv[j] * rdiag[j] : 0.0);
     if (defic)
         for (int k = tid; k < c; k += 256) defic[(size_t)blockIdx.x * c + k] = dcol[k];
     if (tid == 0 && bad) atomicOr(flags, 1);
