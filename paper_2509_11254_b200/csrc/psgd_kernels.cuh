@@ -943,14 +943,24 @@ __global__ void __launch_bounds__(256) k_apply(ApplyArgs a) {
         xs[e] = (row0 + rr < a.rows) ? Xb[(size_t)(row0 + rr) * a.c + j] : 0.f;
     }
     __syncthreads();
-    for (int e = threadIdx.x; e < 32 * a.kout; e += 256) {
-        int rr = e / a.kout, k = e % a.kout;
-        int jend = a.upper ? min(a.c, k + 1) : a.c;
-        double s = 0.0;
-        for (int j = 0; j < jend; ++j) s = fma((double)xs[rr * a.c + j], __ldg(Tb + (size_t)j * a.ldt + k), s);
-        if (row0 + rr < a.rows) {
-            Ob[(size_t)(row0 + rr) * a.kout + k] = (float)s;
-            if (a.XoutT) a.XoutT[((size_t)blockIdx.y * a.kout + k) * a.rows + row0 + rr] = (float)s;
+    // a thread carries column k of four rows (rr, rr + 8, rr + 16, rr + 24): one load of T[j][k] feeds four independent sums
+    for (int e = threadIdx.x; e < 8 * a.kout; e += 256) {
+        const int rr = e / a.kout, k = e % a.kout;
+        const int jend = a.upper ? min(a.c, k + 1) : a.c;
+        double s[4] = {0.0, 0.0, 0.0, 0.0};
+        const float* x0 = xs + rr * a.c;
+        for (int j = 0; j < jend; ++j) {
+            const double t = __ldg(Tb + (size_t)j * a.ldt + k);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) s[q] = fma((double)x0[q * 8 * a.c + j], t, s[q]);
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int row = row0 + rr + 8 * q;
+            if (row < a.rows) {
+                Ob[(size_t)row * a.kout + k] = (float)s[q];
+                if (a.XoutT) a.XoutT[((size_t)blockIdx.y * a.kout + k) * a.rows + row] = (float)s[q];
+            }
         }
     }
 }
