@@ -1032,6 +1032,7 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
     __syncthreads();
     int converged = 0, sweeps = 0;
     const int k_first = tid / c2, i_first = tid % c2, k_step = JAC_THREADS / c2, i_step = JAC_THREADS % c2;
+    const int ka_first = tid / np, kb_first = tid % np, ka_step = JAC_THREADS / np, kb_step = JAC_THREADS % np;
     for (int sweep = 0; sweep < JAC_MAX_SWEEPS && !converged; ++sweep) {
         for (int round = 0; round < c2 - 1; ++round) {
             if (tid < np) {
@@ -1053,31 +1054,33 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
                 }
             }
             __syncthreads();
-            // columns: A <- A J, V <- V J   (thread index runs down the column; (k, i) advance without a division)
-            for (int e = tid, k = k_first, i = i_first; e < np * c2; e += JAC_THREADS) {
-                int p = pp[k], q = qq[k];
-                double cc = cs[k], ss = sn[k];
-                double aip = As[i * ld + p], aiq = As[i * ld + q];
-                As[i * ld + p] = cc * aip - ss * aiq;
-                As[i * ld + q] = ss * aip + cc * aiq;
-                if (vsm) {
-                    double vip = Vt[p * c2 + i], viq = Vt[q * c2 + i];
+            // A <- J^T A J in one pass over 2 x 2 blocks: the block of pairs (a, b), rows {p_a, q_a} x columns {p_b, q_b}, only
+            // needs its own four entries and the two rotations ((a, b) advance without a division)
+            for (int e = tid, ka = ka_first, kb = kb_first; e < np * np; e += JAC_THREADS) {
+                const int pa = pp[ka], qa = qq[ka], pb2 = pp[kb], qb = qq[kb];
+                const double ca = cs[ka], sa = sn[ka], cb = cs[kb], sb = sn[kb];
+                const double a00 = As[pa * ld + pb2], a01 = As[pa * ld + qb], a10 = As[qa * ld + pb2], a11 = As[qa * ld + qb];
+                // columns: (x_p, x_q) <- (c x_p - s x_q, s x_p + c x_q) with the rotation of pair b
+                const double b00 = cb * a00 - sb * a01, b01 = sb * a00 + cb * a01;
+                const double b10 = cb * a10 - sb * a11, b11 = sb * a10 + cb * a11;
+                // rows: the same with the rotation of pair a
+                As[pa * ld + pb2] = ca * b00 - sa * b10;
+                As[pa * ld + qb] = ca * b01 - sa * b11;
+                As[qa * ld + pb2] = sa * b00 + ca * b10;
+                As[qa * ld + qb] = sa * b01 + ca * b11;
+                ka += ka_step; kb += kb_step;
+                if (kb >= np) { kb -= np; ++ka; }
+            }
+            if (vsm) {      // V <- V J (thread index runs down the column)
+                for (int e = tid, k = k_first, i = i_first; e < np * c2; e += JAC_THREADS) {
+                    const int p = pp[k], q = qq[k];
+                    const double cc = cs[k], ss = sn[k];
+                    const double vip = Vt[p * c2 + i], viq = Vt[q * c2 + i];
                     Vt[p * c2 + i] = cc * vip - ss * viq;
                     Vt[q * c2 + i] = ss * vip + cc * viq;
+                    k += k_step; i += i_step;
+                    if (i >= c2) { i -= c2; ++k; }
                 }
-                k += k_step; i += i_step;
-                if (i >= c2) { i -= c2; ++k; }
-            }
-            __syncthreads();
-            // rows: A <- J^T A
-            for (int e = tid, k = k_first, j = i_first; e < np * c2; e += JAC_THREADS) {
-                int p = pp[k], q = qq[k];
-                double cc = cs[k], ss = sn[k];
-                double apj = As[p * ld + j], aqj = As[q * ld + j];
-                As[p * ld + j] = cc * apj - ss * aqj;
-                As[q * ld + j] = ss * apj + cc * aqj;
-                k += k_step; j += i_step;
-                if (j >= c2) { j -= c2; ++k; }
             }
             __syncthreads();
         }
