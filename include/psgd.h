@@ -99,6 +99,10 @@ typedef enum {
                                       kernel (up to 16 columns) below; 1: the tensor-core kernel wherever it fits; 2: never (more than 16
                                       columns then take three passes) */
 
+#define PSGD_OPT_BACKPROJECT_TMA 12   /* 1 (default): the float32 back-projection Q_i = M_i^T P~ of 4, 8 or 16 columns stages its tiles of M
+                                      by TMA in shared memory (n >= 256, n % 4 == 0, aligned pointers); 0: always the kernel that
+                                      prefetches into registers.  The two add the same products in a different order */
+
 /* buffers that psgd_debug_ptr exposes (test use only; valid until the next step) */
 #define PSGD_BUF_P_NODE 1   /* P^(i)   [count][N][m][r] */
 #define PSGD_BUF_Q_NODE 2   /* Q^(i)   [count][N][n][r] */

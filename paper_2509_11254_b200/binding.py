@@ -16,6 +16,7 @@ PSGD_OPT_GRAD_BF16 = 8
 PSGD_OPT_SINGLE_PASS = 9
 PSGD_OPT_TRANSPOSED = 10
 PSGD_OPT_PENDING_TC = 11
+PSGD_OPT_BACKPROJECT_TMA = 12
 PSGD_BUF = {"P_node": 1, "Q_node": 2, "P_hat": 3, "Dbar": 4, "P_mean": 5}
 KERNEL_FAMILIES = ["project", "orth", "backproject", "residual", "refresh", "misc"]
 
@@ -103,7 +104,7 @@ class PowerSGDPlus:
 
     def __init__(self, m, n, r, N, refresh_period=0, seed=0, count=1, device="cuda:0", error_form="local",
                  mode="eager", refresh_iters=None, oversample=None, reset=True, refresh_tc=None, power_steps=None, refresh_adaptive=None,
-                 grad_dtype="float32", single_pass=None, transposed=False, pending_tc=None):
+                 grad_dtype="float32", single_pass=None, transposed=False, pending_tc=None, backproject_tma=None):
         import torch
 
         self.torch = torch
@@ -134,6 +135,8 @@ class PowerSGDPlus:
             _check(L.psgd_set_option(h, PSGD_OPT_SINGLE_PASS, {"auto": 0, "cluster": 1, "none": 2, "l2": 3}[single_pass]))
         if pending_tc is not None:      # "auto" | "always" | "never": which projection folds in the pending residual of the two-pass form
             _check(L.psgd_set_option(h, PSGD_OPT_PENDING_TC, {"auto": 0, "always": 1, "never": 2}[pending_tc]))
+        if backproject_tma is not None:
+            _check(L.psgd_set_option(h, PSGD_OPT_BACKPROJECT_TMA, int(bool(backproject_tma))))
         self.grad_dtype = {"float32": torch.float32, "bfloat16": torch.bfloat16}[grad_dtype]
         if self.grad_dtype is torch.bfloat16:
             _check(L.psgd_set_option(h, PSGD_OPT_GRAD_BF16, 1))

@@ -19,6 +19,7 @@
 #include "psgd_fused.cuh"
 #include "psgd_gemm_tc.cuh"
 #include "psgd_stream.cuh"
+#include "psgd_backproject_tma.cuh"
 
 using namespace psgd;
 
@@ -103,6 +104,7 @@ struct psgd_handle {
     bool transposed = false;      // PSGD_OPT_TRANSPOSED: G and E are stored as [n][m] (the transpose of the m x n problem)
     int t_S = 1, t_rpc = 0;       // row chunks of the contraction over the n stored rows (transposed storage)
     int step_kernel = 0;          // what ran the last step: 0 three-/two-pass kernels, 1 cluster kernel, 2 L2-pipelined kernel
+    bool bq_ok = true;            // back-projection with TMA-staged tiles where the shape allows (PSGD_OPT_BACKPROJECT_TMA)
     bool ran_pending_tc = false;  // the projection of the step in flight folded the pending residual in on the tensor cores
     int ex_phase = 0;             // psgd_exchange_*: 0 between steps, 1 after _begin, 2 after _orth
     bool ex_refresh = false;      // the step in flight is a refresh
@@ -650,6 +652,36 @@ int launch_back(Launcher& L, const float* M, const float* Phat, float* part, int
     }
     BackArgs a{M, Phat, part, rows, n, r, nodes, 1, rpc, S, gate, skip};
     vec = vec && aligned16(M);
+    // 4, 8 or 16 columns exactly, whole 256-column blocks of 16-byte aligned rows: tiles of M staged by TMA
+    if (!gate && vec && (r == 4 || r == 8 || r == 16) && n >= BP_COLS && rpc % BQ_ROWS == 0 && aligned16(Phat) && L.h->bq_ok) {
+        CUtensorMap tM;
+        if (make_tile_map(L.h, &tM, M, n, rows, (int64_t)count * nodes, BP_COLS, BQ_ROWS)) {
+            // row chunks: two CTAs per multiprocessor run at a time; fewest waves x (tiles per CTA + start-up), at most the S
+            // chunks the partial buffer was sized for
+            const int64_t base = (int64_t)ceil_div(n, BP_COLS) * count * nodes, slots = 2 * (int64_t)L.h->sm_count;
+            int bestS = S, best_rpc = rpc;
+            int64_t best_cost = -1;
+            for (int s2 = 1; s2 <= S; ++s2) {
+                const int rpc2 = (int)align_up(ceil_div(rows, s2), BP_SUB), sc = ceil_div(rows, rpc2);
+                const int64_t cost = ((base * sc + slots - 1) / slots) * (ceil_div(rpc2, BQ_ROWS) + 3);
+                if (best_cost < 0 || cost < best_cost) { best_cost = cost; bestS = sc; best_rpc = rpc2; }
+            }
+            S = bestS;
+            a.S = S; a.rows_per_chunk = best_rpc;
+            dim3 grid(ceil_div(n, BP_COLS), S, count * nodes);
+            int* flags = (int*)(L.h->ws + L.h->lay.flags);
+            auto go = [&](auto kern, size_t smem) {
+                set_smem_attr((const void*)kern, smem);
+                L.begin(PSGD_K_BACKPROJECT);
+                kern<<<grid, BQ_THREADS, smem, L.st>>>(tM, a, flags);
+                L.end();
+            };
+            if (r == 4) go(k_backproject_tma<4>, backq_smem_bytes<4>());
+            else if (r == 8) go(k_backproject_tma<8>, backq_smem_bytes<8>());
+            else go(k_backproject_tma<16>, backq_smem_bytes<16>());
+            return S;
+        }
+    }
     if (r <= 4) launch_back_rp<4>(L, a, count * nodes, vec);
     else if (r <= 8) launch_back_rp<8>(L, a, count * nodes, vec);
     else launch_back_rp<16>(L, a, count * nodes, vec);
@@ -1477,6 +1509,7 @@ psgd_status psgd_set_option(psgd_handle* h, int option, int value) {
         case PSGD_OPT_TRANSPOSED: if (value != 0 && value != 1) return PSGD_E_INVALID; h->transposed = value != 0; break;
         case PSGD_OPT_SINGLE_PASS: if (value < 0 || value > 3) return PSGD_E_INVALID; h->single_pass_kernel = value; break;
         case PSGD_OPT_PENDING_TC: if (value < 0 || value > 2) return PSGD_E_INVALID; h->pend_tc = value; break;
+        case PSGD_OPT_BACKPROJECT_TMA: if (value != 0 && value != 1) return PSGD_E_INVALID; h->bq_ok = value != 0; break;
         default: return PSGD_E_INVALID;
     }
     plan(h);

@@ -1057,3 +1057,33 @@ def test_exchange_two_halves_of_the_nodes_against_the_oracle(torch_cuda, m, n, r
                 assert np.linalg.norm(E_gpu - out["E"]) <= 2e-4 * np.linalg.norm(M)
     for h in halves:
         h.close()
+
+
+@pytest.mark.parametrize("m,n,r,N,count", [
+    (1000, 516, 16, 3, 2),      # ragged last tile of 32 rows (8 valid), last column block of 4 valid columns
+    (4100, 1024, 8, 2, 1),      # several row chunks, the last with 4 valid rows
+    (640, 256, 4, 4, 1),        # a single column block, 4 columns
+    (2048, 768, 16, 8, 3),      # config-2 FFN shape
+])
+def test_backprojection_with_tma_staged_tiles(torch_cuda, m, n, r, N, count):
+    """Q_i = M_i^T P~ with the tiles of M staged by TMA (the default for 4, 8 or 16 columns) against the kernel that prefetches
+    into registers (same products, different order of the partial sums) and against the definition in double on the host."""
+    torch = torch_cuda
+    from paper_2509_11254_b200 import PowerSGDPlus
+
+    res = []
+    G = torch.as_tensor(np.stack([synth.make_gradients(2, m, n, N, step=0, matrix_id=c, seed=11) for c in range(count)]), device="cuda:0")
+    for tma in (True, False):
+        comp = PowerSGDPlus(m, n, r, N, refresh_period=0, seed=11, count=count, device="cuda:0", backproject_tma=tma)
+        comp.step(G)
+        assert comp.last_status() == 0
+        res.append((comp.P_hat.clone(), comp.debug("Q_node").clone(), comp.Q.clone()))
+        comp.close()
+    (Pa, Qa, Qma), (Pb, Qb, Qmb) = res
+    assert torch.equal(Pa, Pb)                       # the projection does not depend on the option
+    M64, P64 = G.cpu().numpy().astype(np.float64), Pa.cpu().numpy().astype(np.float64)
+    for c in range(count):
+        ref = np.stack([M64[c, i].T @ P64[c] for i in range(N)])
+        assert rel_fro(Qa[c].cpu().numpy(), ref) <= 1e-6 and rel_fro(Qb[c].cpu().numpy(), ref) <= 1e-6
+        assert rel_fro(Qma[c].cpu().numpy(), ref.mean(axis=0)) <= 1e-6
+    assert rel_fro(Qa.cpu().numpy(), Qb.cpu().numpy()) <= 1e-6
