@@ -505,7 +505,8 @@ bool launch_project_tc(Launcher& L, const float* A, const float* B, float* Mout,
                        int r, int nodes, int count, const int* skip) {
     psgd_handle* h = L.h;
     const int Ncp = (int)align_up(r, 16);
-    if (!h->ptc_ok || Ncp > h->ptc_ncp || r > 128 || !aligned16(A) || (B && !aligned16(B)) || (Mout && !aligned16(Mout))) return false;
+    // (n is the row length of the matrices handed in, which with transposed storage is not the handle's n: 16-byte rows for TMA)
+    if (!h->ptc_ok || Ncp > h->ptc_ncp || r > 128 || n % 4 != 0 || !aligned16(A) || (B && !aligned16(B)) || (Mout && !aligned16(Mout))) return false;
     const int mats = count * nodes;
     float* Qimg = (float*)(h->ws + h->lay.ptQ);
     const int KB = ceil_div(n, TC_BK);
@@ -608,7 +609,7 @@ int launch_back_tc(Launcher& L, const float* M, const float* Phat, float* part, 
                    int S, const int* skip) {
     psgd_handle* h = L.h;
     const int Ncp = (int)align_up(r, 16);
-    if (!h->ptc_ok || Ncp > h->ptc_ncp || r > 128 || rows % 4 != 0 || !aligned16(M)) return 0;
+    if (!h->ptc_ok || Ncp > h->ptc_ncp || r > 128 || n % 4 != 0 || !aligned16(M)) return 0;
     const int mats = count * nodes;
     const int KB = ceil_div(rows, TC_BK);
     const int64_t base = (int64_t)ceil_div(n, TC_BM) * mats;
@@ -693,9 +694,11 @@ int launch_back(Launcher& L, const float* M, const float* Phat, float* part, int
 bool launch_resid_tc(Launcher& L, const float* M, float* Out, const float* Phat, const float* Qf, int rows, int n, int r,
                      int nodes, int mats, int q_per_node, int out_per_node) {
     psgd_handle* h = L.h;
-    if (!h->rtc_ok || !aligned16(Out) || (M && !aligned16(M))) return false;
+    if (!h->rtc_ok || n % 4 != 0 || !aligned16(Out) || (M && !aligned16(M))) return false;
     const int KP = h->rtc_KP, cnt = h->count;
     const int qmats = q_per_node ? mats : cnt;
+    // the split copies of the factors were sized for the handle's own orientation (rows = m, Q_i per node of n rows)
+    if (rows > h->m || (int64_t)qmats * n > (int64_t)cnt * h->N * h->n) return false;
     const size_t tp = (size_t)cnt * rows * KP, tq = (size_t)qmats * n * KP;
     float* Pt[3] = {(float*)(h->ws + h->lay.rtP), (float*)(h->ws + h->lay.rtP) + tp, (float*)(h->ws + h->lay.rtP) + 2 * tp};
     float* Qt[3] = {(float*)(h->ws + h->lay.rtQ), (float*)(h->ws + h->lay.rtQ) + tq, (float*)(h->ws + h->lay.rtQ) + 2 * tq};

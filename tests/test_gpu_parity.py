@@ -218,6 +218,9 @@ def test_k_step_power_iteration(torch_cuda, K, mode):
     (256, 128, 4, 4, 1, 3, "local", 1),      # refreshes at t = 0 and 3 (the node mean is transposed once per refresh)
     (1000, 520, 32, 2, 1, 2, "local", 5),    # refresh with tensor-core sweeps
     (257, 130, 3, 2, 2, 0, "local", 2),      # m % 4 != 0: scalar loads along the stored rows
+    (769, 256, 20, 4, 2, 0, "local", 2),    # more than 16 columns with m % 4 != 0: no tensor-core form along the stored rows, float32 kernels
+    (1000, 64, 20, 2, 1, 0, "mean", 2),     # m > N n: the tensor-core residual's split factors would not fit their buffers, float32 kernel
+    (1024, 128, 24, 2, 1, 0, "mean", 4),    # ... and a shape where they fit: tensor-core residual on stored rows of m entries
 ])
 def test_transposed_storage(torch_cuda, m, n, r, N, count, tau, form, workload):
     """PSGD_OPT_TRANSPOSED: G and E kept as the row-major n x m transposes of the m x n problem (Sec. 1 fixes m >= n for the
