@@ -687,6 +687,25 @@ __global__ void __launch_bounds__(256) k_gram(GramArgs a) {
     const float* Xb = a.X + (size_t)blockIdx.z * a.rows * a.c;
     const float* X2b = (a.X2 ? a.X2 : a.X) + (size_t)blockIdx.z * a.rows * a.c;
     const int rbeg = blockIdx.x * GR_ROWS, rend = min(a.rows, rbeg + GR_ROWS);
+    if (a.c <= 16) {
+        // up to 16 columns (every orthogonalisation of an SSP step): one entry of the c x c block per thread instead of a
+        // 4 x 4 patch of a 64 x 64 tile of which 15/16 would be padding
+        double s = 0.0;
+        for (int r0 = rbeg; r0 < rend; r0 += 32) {
+            __syncthreads();
+            for (int e = threadIdx.x; e < 32 * 16; e += 256) {
+                const int rr = e >> 4, cc = e & 15, grow = r0 + rr;
+                const bool in = grow < rend && cc < a.c;
+                sa[rr][cc] = in ? Xb[(size_t)grow * a.c + cc] : 0.f;
+                sb[rr][cc] = in ? X2b[(size_t)grow * a.c + cc] : 0.f;
+            }
+            __syncthreads();
+#pragma unroll 8
+            for (int rr = 0; rr < 32; ++rr) s = fma((double)sa[rr][ty], (double)sb[rr][tx], s);
+        }
+        if (ty < a.c && tx < a.c) a.part[((size_t)blockIdx.z * a.nparts + blockIdx.x) * a.c * a.c + (size_t)ty * a.c + tx] = s;
+        return;
+    }
     double acc[4][4];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
@@ -734,9 +753,18 @@ __global__ void k_gram_sum(double* part, int cc, int nparts, int count, const in
     if (idx >= (size_t)cc * count) return;
     size_t c = idx / cc, e = idx % cc;
     double* pb = part + c * (size_t)nparts * cc;
-    double s = 0.0;
-    for (int p = 0; p < nparts; ++p) s += pb[(size_t)p * cc + e];
-    pb[e] = s;
+    // four running sums over the partials p = 0, 1, 2, 3 (mod 4), combined in a fixed order: the loads of a round do not
+    // depend on one another
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+    int p = 0;
+    for (; p + 3 < nparts; p += 4) {
+        s0 += pb[(size_t)p * cc + e];
+        s1 += pb[(size_t)(p + 1) * cc + e];
+        s2 += pb[(size_t)(p + 2) * cc + e];
+        s3 += pb[(size_t)(p + 3) * cc + e];
+    }
+    for (; p < nparts; ++p) s0 += pb[(size_t)p * cc + e];
+    pb[e] = (s0 + s1) + (s2 + s3);
 }
 
 // Sum the Gram partials, scale to unit diagonal, Cholesky, invert, and write
