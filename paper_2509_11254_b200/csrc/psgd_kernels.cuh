@@ -773,6 +773,7 @@ __global__ void k_gram_sum(double* part, int cc, int nparts, int count, const in
 // walking down a column is free of bank conflicts).
 constexpr double CHOL_PIVOT_TOL = 1e-11;  // squared sine of the angle to the previous columns
 constexpr int CHOL_NB = 8;                // columns per panel of the factorisation
+constexpr int CHOL_IB = 32;               // block size of the triangular inverse
 __host__ __device__ inline int chol_ld(int c) { return c | 1; }
 // `gate` (optional): set to 1 when a scaled pivot^2 falls below gate_tol, i.e. when the columns
 // are too ill-conditioned for results derived from W = M^T P to keep float32 accuracy.
@@ -862,17 +863,18 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
             __syncthreads();
         }
     }
-    // Inverse of the lower-triangular L by forward substitution, no block-wide barrier: column j of X = L^-1 is
-    // x_j = 1 / l_jj, x_i = -(sum_{k = j}^{i - 1} l_ik x_k) / l_ii, kept in row j of the unused upper triangle (X[i][j] at
-    // Gs[j][i]), the diagonal in rdiag.  Two adjacent lanes share a column and take alternate terms of every sum (the first
-    // column's c^2 / 2 dependent steps set the time of the whole phase).
+    // Inverse X = L^-1 of the lower-triangular factor, in blocks of CHOL_IB rows and columns; X[i][j] (i > j) is kept at
+    // Gs[j][i] in the unused upper triangle, the diagonal in rdiag.
+    // (1) Diagonal blocks, all at once: column j of a block by forward substitution inside the block,
+    //     x_j = 1 / l_jj, x_i = -(sum_{k = j}^{i - 1} l_ik x_k) / l_ii; two adjacent lanes share a column and take alternate terms.
     for (int j0 = 0; j0 < c; j0 += 128) {
         const int j = j0 + (tid >> 1), hlf = tid & 1;
         if (j < c) {
             const unsigned pair = 3u << ((tid & 31) & ~1);
             double* xr = Gs + (size_t)j * ld;       // xr[i] = X[i][j] for i > j
             const double xj = rdiag[j];
-            for (int i = j + 1; i < c; ++i) {
+            const int iend = min(c, (j / CHOL_IB + 1) * CHOL_IB);
+            for (int i = j + 1; i < iend; ++i) {
                 const double* li = Gs + (size_t)i * ld;
                 double s0 = hlf ? 0.0 : li[j] * xj, s1 = 0.0;
                 int k = j + 1 + hlf;
@@ -886,6 +888,38 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
         }
     }
     __syncthreads();
+    // (2) Block rows below the first, one after the other: for the rows a of block row bi and every column b to its left,
+    //     S[a][b] = sum_{k = b}^{bi CHOL_IB - 1} l_ak x_kb (parked where X[a][b] will live), then X[a][b] = -sum_{t <= a} x_at S[t][b]
+    //     with t running over the rows of the block: two passes in which every entry is independent of the others.
+    for (int a0 = CHOL_IB; a0 < c; a0 += CHOL_IB) {
+        const int na = min(CHOL_IB, c - a0), ne = na * a0;          // entries (a, b): a0 <= a < a0 + na, b < a0
+        for (int e = tid; e < ne; e += 256) {
+            const int aa = a0 + e % na, bb = e / na;
+            const double* la = Gs + (size_t)aa * ld;
+            const double* xb = Gs + (size_t)bb * ld;
+            double s0 = la[bb] * rdiag[bb], s1 = 0.0;
+            int k = bb + 1;
+            for (; k + 1 < a0; k += 2) { s0 = fma(la[k], xb[k], s0); s1 = fma(la[k + 1], xb[k + 1], s1); }
+            if (k < a0) s0 = fma(la[k], xb[k], s0);
+            Gs[(size_t)bb * ld + aa] = s0 + s1;                     // S[a][b]; nobody reads X[a][b] in this pass
+        }
+        __syncthreads();
+        double xv[(CHOL_IB * 160 + 255) / 256];                     // at most 32 x 160 entries over 256 threads
+        int q = 0;
+        for (int e = tid; e < ne; e += 256, ++q) {
+            const int aa = a0 + e % na, bb = e / na;
+            const double* sb = Gs + (size_t)bb * ld;                // S[t][b] at sb[t]
+            double s0 = rdiag[aa] * sb[aa], s1 = 0.0;               // t = a: x_aa = 1 / l_aa
+            int t = a0;
+            for (; t + 1 < aa; t += 2) { s0 = fma(Gs[(size_t)t * ld + aa], sb[t], s0); s1 = fma(Gs[(size_t)(t + 1) * ld + aa], sb[t + 1], s1); }
+            if (t < aa) s0 = fma(Gs[(size_t)t * ld + aa], sb[t], s0);
+            xv[q] = -(s0 + s1);
+        }
+        __syncthreads();
+        q = 0;
+        for (int e = tid; e < ne; e += 256, ++q) Gs[(size_t)(e / na) * ld + a0 + e % na] = xv[q];
+        __syncthreads();
+    }
     // T[j][k] = dinv[j] * Linv[k][j]  for j <= k
     double* Tb = T + (size_t)blockIdx.x * c * c;
     for (int j = ty; j < c; j += 8)
