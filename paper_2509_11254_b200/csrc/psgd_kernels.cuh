@@ -820,7 +820,7 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
     // Right-looking Cholesky on the lower triangle, Gs = L L^T, in panels of CHOL_NB columns: a column's update is applied at
     // once only to the rest of its panel (a few entries per thread between barriers); the matrix behind the panel receives the
     // panel's CHOL_NB rank-one updates in one pass (same terms in the same order, one load and store per entry instead of
-    // CHOL_NB).  Every thread evaluates the pivot of a column itself (no serial step by one thread).
+    // CHOL_NB).  Every thread evaluates the pivot of a column itself (no serial step by one thread, two barriers per column).
     for (int k0 = 0; k0 < c; k0 += CHOL_NB) {
         const int kend = min(c, k0 + CHOL_NB);
         for (int k = k0; k < kend; ++k) {
@@ -831,9 +831,8 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
                 if (reject) { bad = 1; dcol[k] = 1; }
             }
             if (reject) p = 1.0;
-            const double rl = rsqrt(p);
-            __syncthreads();                       // every thread has read the pivot
-            if (tid == 0) { Gs[k * ld + k] = sqrt(p); rdiag[k] = rl; }
+            const double rl = rsqrt(p);            // 1 / l_kk: all that the later phases need of the diagonal (Gs[k][k] keeps the pivot)
+            if (tid == 0) rdiag[k] = rl;
             for (int i = k + 1 + tid; i < c; i += 256) Gs[i * ld + k] = reject ? 0.0 : Gs[i * ld + k] * rl;
             __syncthreads();
             const int w = kend - k - 1;            // columns of the panel still to come
