@@ -67,9 +67,9 @@ typedef enum {
                                       whole SSP step is then one pass over G and E, up to 16 two passes; above,
                                       and on refresh steps, the three-pass kernels run as in mode 0 */
 #define PSGD_OPT_REFRESH_ITERS 3   /* subspace iterations q of the refresh; 0 (default): where the early sweeps run on the tensor cores 12 (blocks of
-                                      32 columns and more) or 20 (16 to 31 columns), else at most 20 with the stopping test.  The start block is [Q_{t-1} | random columns] */
+                                      32 columns and more) or 20 (8 to 31 columns), else at most 20 with the stopping test.  The start block is [Q_{t-1} | random columns] */
 #define PSGD_OPT_REFRESH_OVERSAMPLE 4 /* extra columns of the refresh block (default max(8, r)) */
-#define PSGD_OPT_REFRESH_TC 5      /* 1 (default): the early sweeps of a refresh whose block has >= 16 columns run
+#define PSGD_OPT_REFRESH_TC 5      /* 1 (default): the early sweeps of a refresh whose block has >= 8 columns run
                                       on the tensor cores in TF32, the last 4 in float32; 0: float32 throughout */
 #define PSGD_OPT_POWER_STEPS 6     /* K >= 1 power steps per SSP iteration (Eq. (8)); 1 (default) is PowerSGD's single
                                       step (Eq. (9)); K > 1 runs the three-pass kernels */

@@ -186,8 +186,8 @@ void plan(psgd_handle* h) {
     L.U = take(cnt * ell * r * 8);
     L.Pold = take(cnt * m * r * 4);
     L.dpart = take(cnt * ((size_t)ceil_div(h->m, 64) + 1) * 8);
-    // ---- tensor-core sweeps of the refresh: block of >= 16 columns, 16-byte row strides for TMA ----
-    h->tc_ok = h->refresh_tc && ell >= 16 && ell <= TC_MAXN && h->n % 4 == 0 && h->m % 4 == 0;
+    // ---- tensor-core sweeps of the refresh: block of >= 8 columns, 16-byte row strides for TMA ----
+    h->tc_ok = h->refresh_tc && ell >= 8 && ell <= TC_MAXN && h->n % 4 == 0 && h->m % 4 == 0;
     if (h->transposed && !h->tc_ok) L.dbarT = take(cnt * m * n * 4);   // the node mean in storage orientation, before it is transposed
     if (h->tc_ok) {
         const size_t ncp = align_up(ell, 16);
@@ -912,7 +912,7 @@ void svd(Launcher& L, psgd_handle* h, const void* G, bool have_dbar = false) {
     // limit (20); wider blocks have no such test (their Rayleigh-Ritz step is too dear to repeat) and run 12 sweeps, the
     // first 8 of them in TF32: measured on a 16384 x 4096 mean with a 0.9^k spectrum, 4 sweeps already bring the top-16
     // projector within 1e-5 and 8 sweeps the energy left behind at r = 64 within 1e-9 of the optimum.
-    // Blocks of 16 to 31 columns (r = 8 .. 15 with their 8 extra columns) converge more slowly once error feedback has filled
+    // Blocks of 8 to 31 columns (r up to 15 with their 8 or more extra columns) converge more slowly once error feedback has filled
     // the directions right below r: 12 sweeps left the projector 3e-2 off in a free-running run, 20 (16 in TF32) pass every test.
     const int iters = h->refresh_iters > 0 ? h->refresh_iters : (h->tc_ok ? (ell < 32 ? 20 : 12) : 20);
     if (!have_dbar) launch_add_mean(L, G, h->grad_bf16, h->E, dbar, (size_t)m * n, N, cnt, K);
