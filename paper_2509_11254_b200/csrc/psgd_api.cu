@@ -773,7 +773,7 @@ void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int r
     if (nparts > 4) {   // fold the partials in parallel first; k_chol then reads partial 0 with the original stride
         size_t tot = (size_t)c * c * h->count;
         L.begin(kind);
-        k_gram_sum<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(gram, c * c, nparts, h->count, skip);
+        k_gram_sum<<<(unsigned)((tot + 31) / 32), 256, 0, L.st>>>(gram, c * c, nparts, h->count, skip);
         L.end();
     }
     size_t smem = (size_t)c * chol_ld(c) * 8;
@@ -976,7 +976,7 @@ void svd(Launcher& L, psgd_handle* h, const void* G, bool have_dbar = false) {
         if (nparts > 4) {
             size_t tot = (size_t)ell * ell * cnt;
             L.begin(K);
-            k_gram_sum<<<(unsigned)((tot + 255) / 256), 256, 0, L.st>>>(gram, ell * ell, nparts, cnt, skip);
+            k_gram_sum<<<(unsigned)((tot + 31) / 32), 256, 0, L.st>>>(gram, ell * ell, nparts, cnt, skip);
             L.end();
         }
         int c2 = (ell + 1) & ~1;
@@ -1026,7 +1026,7 @@ void svd(Launcher& L, psgd_handle* h, const void* G, bool have_dbar = false) {
                 L.end();
                 size_t tg = (size_t)r * r * cnt;
                 L.begin(K);
-                k_gram_sum<<<(unsigned)((tg + 255) / 256), 256, 0, L.st>>>(gram, r * r, nparts, cnt, skip);
+                k_gram_sum<<<(unsigned)((tg + 31) / 32), 256, 0, L.st>>>(gram, r * r, nparts, cnt, skip);
                 L.end();
                 L.begin(K);
                 k_subspace_change<<<dim3(nb, cnt), 256, (size_t)r * r * 4, L.st>>>(Pold, Phat, gram, (size_t)nparts * r * r, dpart, m, r, skip);
@@ -1275,7 +1275,7 @@ bool stream_ssp(Launcher& L, psgd_handle* h, const void* G) {
     // P'^T P' = L L^T  ->  T'; scaled pivot^2 < 2e-2 raises the gate for the precise back-projection (as in the cluster kernel's path)
     size_t tg = (size_t)r * r * cnt;
     L.begin(PSGD_K_ORTH);
-    k_gram_sum<<<(unsigned)((tg + 255) / 256), 256, 0, L.st>>>(gram, r * r, nrb, cnt);
+    k_gram_sum<<<(unsigned)((tg + 31) / 32), 256, 0, L.st>>>(gram, r * r, nrb, cnt);
     L.end();
     L.begin(PSGD_K_ORTH);
     int* defic = (int*)(ws + Y.defic);

@@ -746,25 +746,36 @@ __global__ void __launch_bounds__(256) k_gram(GramArgs a) {
 }
 
 // part[c][0][e] <- sum_p part[c][p][e]  (fixed order), so that the single-CTA kernels below read one
-// matrix instead of streaming every partial through one SM.  One thread per entry.
-__global__ void k_gram_sum(double* part, int cc, int nparts, int count, const int* skip = nullptr) {
+// matrix instead of streaming every partial through one SM.  A CTA of 8 warps takes 32 consecutive entries: warp w adds the
+// partials p = w (mod 8) of its entries in four independent running sums (256-byte rows, coalesced), the eight warp sums are
+// added in a fixed order.  grid: ceil(cc * count / 32), 256 threads.
+__global__ void __launch_bounds__(256) k_gram_sum(double* part, int cc, int nparts, int count, const int* skip = nullptr) {
+    __shared__ double red[8][33];
     if (skip && *skip) return;
-    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= (size_t)cc * count) return;
-    size_t c = idx / cc, e = idx % cc;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const size_t idx = (size_t)blockIdx.x * 32 + lane;
+    const bool in = idx < (size_t)cc * count;
+    const size_t c = in ? idx / cc : 0, e = in ? idx % cc : 0;
     double* pb = part + c * (size_t)nparts * cc;
-    // four running sums over the partials p = 0, 1, 2, 3 (mod 4), combined in a fixed order: the loads of a round do not
-    // depend on one another
     double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-    int p = 0;
-    for (; p + 3 < nparts; p += 4) {
-        s0 += pb[(size_t)p * cc + e];
-        s1 += pb[(size_t)(p + 1) * cc + e];
-        s2 += pb[(size_t)(p + 2) * cc + e];
-        s3 += pb[(size_t)(p + 3) * cc + e];
+    if (in) {
+        int p = w;
+        for (; p + 24 < nparts; p += 32) {
+            s0 += pb[(size_t)p * cc + e];
+            s1 += pb[(size_t)(p + 8) * cc + e];
+            s2 += pb[(size_t)(p + 16) * cc + e];
+            s3 += pb[(size_t)(p + 24) * cc + e];
+        }
+        for (; p < nparts; p += 8) s0 += pb[(size_t)p * cc + e];
     }
-    for (; p < nparts; ++p) s0 += pb[(size_t)p * cc + e];
-    pb[e] = (s0 + s1) + (s2 + s3);
+    red[w][lane] = (s0 + s1) + (s2 + s3);
+    __syncthreads();       // every read of partial 0 (warp 0's own) is done before it is overwritten
+    if (w == 0 && in) {
+        double t = red[0][lane];
+#pragma unroll
+        for (int k = 1; k < 8; ++k) t += red[k][lane];
+        pb[e] = t;
+    }
 }
 
 // Sum the Gram partials, scale to unit diagonal, Cholesky, invert, and write
@@ -1035,6 +1046,9 @@ __global__ void __launch_bounds__(256) k_apply(ApplyArgs a) {
 // ----------------------------------------------------------------------------
 constexpr int JAC_THREADS = 512;
 constexpr int JAC_MAX_SWEEPS = 40;
+// stop once the squared off-diagonal norm is this fraction of the squared diagonal norm: 1e-13 relative, two orders below
+// anything the float32 basis built from the eigenvectors can show and above the rounding floor of a 256-column block
+constexpr double JAC_OFF_TOL = 1e-26;
 // leading dimension of the shared-memory matrix: odd number of doubles (no bank conflicts down a column)
 __host__ __device__ inline int jac_ld(int c2) { return c2 | 1; }
 // The eigenvector matrix is kept in shared memory beside A while both fit; wider blocks log their rotations
@@ -1160,7 +1174,7 @@ __global__ void __launch_bounds__(JAC_THREADS) k_jacobi_top(const double* part, 
         }
         if ((tid & 31) == 0) { atomicAdd(&offn, lo); atomicAdd(&diagn, ldg); }
         __syncthreads();
-        converged = (offn <= 1e-30 * diagn) || (diagn == 0.0);
+        converged = (offn <= JAC_OFF_TOL * diagn) || (diagn == 0.0);
         __syncthreads();
     }
     if (tid == 0 && !converged) atomicOr(flags, 2);
