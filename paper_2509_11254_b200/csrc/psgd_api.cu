@@ -770,17 +770,30 @@ void launch_orth(Launcher& L, psgd_handle* h, const float* X, float* Xout, int r
     L.begin(kind);
     k_gram<<<dim3(nparts, nblk * nblk, h->count), 256, 0, L.st>>>(g);
     L.end();
-    if (nparts > 4) {   // fold the partials in parallel first; k_chol then reads partial 0 with the original stride
+    if (nparts > 4) {   // fold the partials in parallel first; the Cholesky kernel then reads partial 0 with the original stride
         size_t tot = (size_t)c * c * h->count;
         L.begin(kind);
         k_gram_sum<<<(unsigned)((tot + 31) / 32), 256, 0, L.st>>>(gram, c * c, nparts, h->count, skip);
         L.end();
     }
     size_t smem = (size_t)c * chol_ld(c) * 8;
-    allow_smem(k_chol, smem);
     L.begin(kind);
     int* defic = (int*)(ws + h->lay.defic);
-    k_chol<<<h->count, 256, smem, L.st>>>(gram, T, c, nparts > 4 ? -nparts : nparts, flags, nullptr, 0.0, complete ? defic : nullptr, skip);
+    const int np = nparts > 4 ? -nparts : nparts;
+    int* dfc = complete ? defic : nullptr;
+    // wide CTAs only while every matrix has a multiprocessor to itself: with more matrices than that the narrow ones share
+    // the multiprocessors and finish sooner together
+    const int nt = h->count <= h->sm_count ? chol_threads(c) : 256;
+    if (nt == 1024) {
+        allow_smem(k_chol_t<1024>, smem);
+        k_chol_t<1024><<<h->count, 1024, smem, L.st>>>(gram, T, c, np, flags, nullptr, 0.0, dfc, skip);
+    } else if (nt == 512) {
+        allow_smem(k_chol_t<512>, smem);
+        k_chol_t<512><<<h->count, 512, smem, L.st>>>(gram, T, c, np, flags, nullptr, 0.0, dfc, skip);
+    } else {
+        allow_smem(k_chol_t<256>, smem);
+        k_chol_t<256><<<h->count, 256, smem, L.st>>>(gram, T, c, np, flags, nullptr, 0.0, dfc, skip);
+    }
     L.end();
     ApplyArgs ap{X, T, Xout, rows, c, c, c, 1, XoutT, skip};
     L.begin(kind);
@@ -1184,7 +1197,7 @@ void fused_ssp(Launcher& L, psgd_handle* h, const void* G) {
     // P'^T P' = L L^T  ->  T'; scaled pivot^2 < 2e-2 (rounding of W T amplified > 7x) raises the gate for the precise path
     L.begin(PSGD_K_ORTH);
     int* defic = (int*)(ws + Y.defic);
-    k_chol<<<cnt, 256, (size_t)r * chol_ld(r) * 8, L.st>>>(gram, T, r, h->KC, flags, gate, 2e-2, defic);
+    k_chol_t<256><<<cnt, 256, (size_t)r * chol_ld(r) * 8, L.st>>>(gram, T, r, h->KC, flags, gate, 2e-2, defic);
     L.end();
     FinishPArgs fp{Pout, T, Phat, Ppad, Tacc, Tacc, m, r, RP, h->tacc_identity ? 1 : 0};
     L.begin(PSGD_K_ORTH);
@@ -1279,7 +1292,7 @@ bool stream_ssp(Launcher& L, psgd_handle* h, const void* G) {
     L.end();
     L.begin(PSGD_K_ORTH);
     int* defic = (int*)(ws + Y.defic);
-    k_chol<<<cnt, 256, (size_t)r * chol_ld(r) * 8, L.st>>>(gram, T, r, -nrb, flags, gate, 2e-2, defic);
+    k_chol_t<256><<<cnt, 256, (size_t)r * chol_ld(r) * 8, L.st>>>(gram, T, r, -nrb, flags, gate, 2e-2, defic);
     L.end();
     FinishPArgs fp{Pout, T, Phat, Ppad, Tacc, Tacc, m, r, RP, h->tacc_identity ? 1 : 0};
     L.begin(PSGD_K_ORTH);

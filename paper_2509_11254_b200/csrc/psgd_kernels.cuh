@@ -781,18 +781,23 @@ __global__ void __launch_bounds__(256) k_gram_sum(double* part, int cc, int npar
 // Sum the Gram partials, scale to unit diagonal, Cholesky, invert, and write
 // T = D^-1 L^-T (upper triangular, double) so that P~ = P T.  One CTA per matrix.
 // Dynamic shared memory: c * chol_ld(c) doubles (rows padded to an odd number of doubles so that
-// walking down a column is free of bank conflicts).
+// walking down a column is free of bank conflicts).  NT threads: 256 for the narrow factors of a step; the wide blocks of a
+// refresh take chol_threads(c) (every phase is a chain of short dependent steps between barriers, so more warps per
+// scheduler shorten it; each entry sees the same operations in the same order whatever NT).
 constexpr double CHOL_PIVOT_TOL = 1e-11;  // squared sine of the angle to the previous columns
 constexpr int CHOL_NB = 8;                // columns per panel of the factorisation
 constexpr int CHOL_IB = 32;               // block size of the triangular inverse
 __host__ __device__ inline int chol_ld(int c) { return c | 1; }
+__host__ __device__ inline int chol_threads(int c) { return c >= 96 ? 1024 : (c >= 48 ? 512 : 256); }
 // `gate` (optional): set to 1 when a scaled pivot^2 falls below gate_tol, i.e. when the columns
 // are too ill-conditioned for results derived from W = M^T P to keep float32 accuracy.
 // `defic` (optional, [count][c]): 1 for every column whose pivot was rejected (zero or dependent column);
 // k_complete replaces those columns of P~ by an orthonormal completion.
-__global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int c, int nparts, int* flags,
-                                              int* gate = nullptr, double gate_tol = 0.0, int* defic = nullptr,
-                                              const int* skip = nullptr) {
+template <int NT>
+__global__ void __launch_bounds__(NT) k_chol_t(const double* part, double* T, int c, int nparts, int* flags,
+                                               int* gate = nullptr, double gate_tol = 0.0, int* defic = nullptr,
+                                               const int* skip = nullptr) {
+    constexpr int NW = NT / 32;                       // warps; NT / 8 rows per pass inside a panel
     extern __shared__ __align__(16) double Gs[];  // [c][ld]
     if (skip && *skip) return;
     __shared__ double dinv[192], rdiag[192];   // column scaling; reciprocals of the diagonal of L
@@ -805,8 +810,8 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
     if (nparts < 0) nparts = 1;
     const double* pb = part + (size_t)blockIdx.x * pstride * c * c;
     if (tid == 0) { bad = 0; illc = 0; }
-    const int tx = tid & 31, ty = tid >> 5;          // lanes along a row, 8 rows at a time
-    for (int i = ty; i < c; i += 8)
+    const int tx = tid & 31, ty = tid >> 5;          // lanes along a row, one row per warp at a time
+    for (int i = ty; i < c; i += NW)
         for (int j = tx; j < c; j += 32) {
             int ii = i, jj = j;
             if ((i >> 6) > (j >> 6)) { ii = j; jj = i; }   // lower block triangle was not computed: mirror
@@ -815,13 +820,13 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
             Gs[i * ld + j] = s;
         }
     __syncthreads();
-    for (int k = tid; k < c; k += 256) {
+    for (int k = tid; k < c; k += NT) {
         double d = Gs[k * ld + k];
         dcol[k] = 0;
         if (!(d > 0.0)) { dinv[k] = 0.0; bad = 1; dcol[k] = 1; } else dinv[k] = 1.0 / sqrt(d);
     }
     __syncthreads();
-    for (int i = ty; i < c; i += 8)
+    for (int i = ty; i < c; i += NW)
         for (int j = tx; j < c; j += 32) {
             double v = Gs[i * ld + j] * dinv[i] * dinv[j];
             if (i == j && dinv[i] == 0.0) v = 1.0;  // zero column: decouple it (fixed up later)
@@ -844,14 +849,14 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
             if (reject) p = 1.0;
             const double rl = rsqrt(p);            // 1 / l_kk: all that the later phases need of the diagonal (Gs[k][k] keeps the pivot)
             if (tid == 0) rdiag[k] = rl;
-            for (int i = k + 1 + tid; i < c; i += 256) Gs[i * ld + k] = reject ? 0.0 : Gs[i * ld + k] * rl;
+            for (int i = k + 1 + tid; i < c; i += NT) Gs[i * ld + k] = reject ? 0.0 : Gs[i * ld + k] * rl;
             __syncthreads();
             const int w = kend - k - 1;            // columns of the panel still to come
-            if (w > 0) {                           // eight threads per row (one per panel column, CHOL_NB = 8), 32 rows per pass
+            if (w > 0) {                           // eight threads per row (one per panel column, CHOL_NB = 8), NT / 8 rows per pass
                 const int j = k + 1 + (tid & 7);
                 if ((tid & 7) < w) {
                     const double ljk = Gs[j * ld + k];
-                    for (int i = k + 1 + (tid >> 3); i < c; i += 32)
+                    for (int i = k + 1 + (tid >> 3); i < c; i += NT / 8)
                         if (i >= j) Gs[i * ld + j] = fma(-Gs[i * ld + k], ljk, Gs[i * ld + j]);
                 }
                 __syncthreads();
@@ -859,7 +864,7 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
         }
         // behind the panel, one row per warp pass: lanes walk along the row
         if (kend < c) {
-            for (int i = kend + (tid >> 5); i < c; i += 8) {
+            for (int i = kend + (tid >> 5); i < c; i += NW) {
                 double li[CHOL_NB];
 #pragma unroll
                 for (int q = 0; q < CHOL_NB; ++q) li[q] = Gs[i * ld + k0 + q];
@@ -877,7 +882,7 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
     // Gs[j][i] in the unused upper triangle, the diagonal in rdiag.
     // (1) Diagonal blocks, all at once: column j of a block by forward substitution inside the block,
     //     x_j = 1 / l_jj, x_i = -(sum_{k = j}^{i - 1} l_ik x_k) / l_ii; two adjacent lanes share a column and take alternate terms.
-    for (int j0 = 0; j0 < c; j0 += 128) {
+    for (int j0 = 0; j0 < c; j0 += NT / 2) {
         const int j = j0 + (tid >> 1), hlf = tid & 1;
         if (j < c) {
             const unsigned pair = 3u << ((tid & 31) & ~1);
@@ -903,7 +908,7 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
     //     with t running over the rows of the block: two passes in which every entry is independent of the others.
     for (int a0 = CHOL_IB; a0 < c; a0 += CHOL_IB) {
         const int na = min(CHOL_IB, c - a0), ne = na * a0;          // entries (a, b): a0 <= a < a0 + na, b < a0
-        for (int e = tid; e < ne; e += 256) {
+        for (int e = tid; e < ne; e += NT) {
             const int aa = a0 + e % na, bb = e / na;
             const double* la = Gs + (size_t)aa * ld;
             const double* xb = Gs + (size_t)bb * ld;
@@ -914,9 +919,9 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
             Gs[(size_t)bb * ld + aa] = s0 + s1;                     // S[a][b]; nobody reads X[a][b] in this pass
         }
         __syncthreads();
-        double xv[(CHOL_IB * 160 + 255) / 256];                     // at most 32 x 160 entries over 256 threads
+        double xv[(CHOL_IB * 160 + NT - 1) / NT];                   // at most 32 x 160 entries over NT threads
         int q = 0;
-        for (int e = tid; e < ne; e += 256, ++q) {
+        for (int e = tid; e < ne; e += NT, ++q) {
             const int aa = a0 + e % na, bb = e / na;
             const double* sb = Gs + (size_t)bb * ld;                // S[t][b] at sb[t]
             double s0 = rdiag[aa] * sb[aa], s1 = 0.0;               // t = a: x_aa = 1 / l_aa
@@ -927,22 +932,22 @@ __global__ void __launch_bounds__(256) k_chol(const double* part, double* T, int
         }
         __syncthreads();
         q = 0;
-        for (int e = tid; e < ne; e += 256, ++q) Gs[(size_t)(e / na) * ld + a0 + e % na] = xv[q];
+        for (int e = tid; e < ne; e += NT, ++q) Gs[(size_t)(e / na) * ld + a0 + e % na] = xv[q];
         __syncthreads();
     }
     // T[j][k] = dinv[j] * Linv[k][j]  for j <= k
     double* Tb = T + (size_t)blockIdx.x * c * c;
-    for (int j = ty; j < c; j += 8)
+    for (int j = ty; j < c; j += NW)
         for (int k = tx; k < c; k += 32)
             Tb[(size_t)j * c + k] = (j < k) ? dinv[j] * Gs[j * ld + k] : (j == k ? dinv[j] * rdiag[j] : 0.0);
     if (defic)
-        for (int k = tid; k < c; k += 256) defic[(size_t)blockIdx.x * c + k] = dcol[k];
+        for (int k = tid; k < c; k += NT) defic[(size_t)blockIdx.x * c + k] = dcol[k];
     if (tid == 0 && bad) atomicOr(flags, 1);
     if (tid == 0 && illc && gate) atomicOr(gate, 1);
 }
 
 // Orthonormal completion of a rank-deficient factor (the paper is silent on QR of a rank-deficient P; any
-// orthonormal P~ whose span contains range(P) is a valid result).  Every column that k_chol rejected is
+// orthonormal P~ whose span contains range(P) is a valid result).  Every column that k_chol_t rejected is
 // replaced by a seeded pseudo-random vector, orthogonalised twice (modified Gram-Schmidt, double sums)
 // against the valid columns and normalised.  One CTA per matrix; does nothing unless the status word
 // carries PSGD_W_RANK_DEFICIENT.  Ppad (optional) is the padded copy [count][rows][RP] kept in step.
@@ -995,6 +1000,7 @@ __global__ void __launch_bounds__(256) k_complete(float* Phat, float* Ppad, cons
 
 // Xout[row][k] = sum_j X[row][j] * T[j][k]  (double accumulate), k < kout.
 // grid: (row tiles of 32, count); 256 threads.  X and Xout may alias (rows are staged).
+// (1024 threads per tile, one pass over the items instead of four, were measured on blocks of 128 columns: 113 us against 79 us.)
 struct ApplyArgs {
     const float* X;   // [count][rows][c]
     const double* T;  // [count][c][ldt]
